@@ -1,0 +1,198 @@
+/*
+ * razor.h - C ABI of the B200 (sm_100a) RazorAttention hot path.
+ *
+ * RazorAttention (arXiv 2407.15891) keeps the whole KV cache only for "retrieval" heads.  Every
+ * other head keeps its first N0 attention-sink tokens and its most recent L tokens (Algorithm 1,
+ * lines 2-3) and folds all dropped tokens into one compensation token, the mean of the dropped
+ * keys and values (Eq. 4).  At decode time that token enters the softmax with weight N_d, the
+ * number of dropped tokens (Eq. 5); retrieval heads use ordinary attention (Algorithm 1, line 5).
+ *
+ * This library builds that head-heterogeneous cache at the end of prefill (razor_compress), adds
+ * decode tokens to it (razor_append) and runs decode attention over it (razor_decode_attention).
+ *
+ * Conventions
+ *   - Every function returns RAZOR_OK (0) or a negative razor_status code.  Nothing throws, aborts
+ *     or traps on the device.
+ *   - "device" pointers are CUDA device memory of the current device; "host" pointers are ordinary
+ *     host memory, read before the call returns.
+ *   - The caller owns every device buffer: dense K/V, queries, outputs, the page pool and the
+ *     workspace.  The library never allocates device memory; it owns only the host-side handle
+ *     (and a small pinned host staging area), released by razor_cache_destroy.
+ *   - Work is enqueued on the CUDA stream passed as `stream` (a cudaStream_t cast to void*; NULL is
+ *     the default stream) and is asynchronous with respect to the host.  All calls on one cache
+ *     must be stream-ordered with respect to each other (they share scratch buffers).
+ *   - Storage dtype of K, V and q is config.dtype; compensation sums/means and outputs are fp32.
+ *   - The library never applies rotary embeddings: K and q arrive after the rotary transformation,
+ *     as the paper's cache does (Section 3.2, text below Eq. 4).
+ */
+#ifndef RAZOR_H_
+#define RAZOR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define RAZOR_API __attribute__((visibility("default")))
+#else
+#define RAZOR_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  RAZOR_OK = 0,
+  RAZOR_E_INVALID_ARG = -1,     /* a size, index or flag is out of range */
+  RAZOR_E_NULL_PTR = -2,        /* a required pointer is NULL */
+  RAZOR_E_UNSUPPORTED_DIM = -3, /* head_dim / dtype / group size / page size not supported */
+  RAZOR_E_POOL_TOO_SMALL = -4,  /* page pool or workspace smaller than razor_query_bytes reports */
+  RAZOR_E_CAPACITY = -5,        /* append beyond max_new_tokens, or context beyond max_ctx_len */
+  RAZOR_E_NOT_COMPRESSED = -6,  /* append/decode/export on a layer (or sequence) not yet compressed */
+  RAZOR_E_CUDA = -7,            /* a CUDA runtime call failed; razor_last_cuda_error() has the code */
+  RAZOR_E_MISALIGNED = -8       /* a device pointer or stride breaks the 16-byte alignment rule */
+} razor_status;
+
+enum { RAZOR_F32 = 0, RAZOR_BF16 = 1 };
+
+typedef struct razor_cache razor_cache_t; /* opaque host object */
+
+typedef struct {
+  int32_t batch;            /* B: sequences                                                        */
+  int32_t n_layers;         /* L                                                                   */
+  int32_t n_q_heads;        /* Hq; must be a multiple of n_kv_heads; group = Hq/Hkv in {1,2,4,8}   */
+  int32_t n_kv_heads;       /* Hkv                                                                 */
+  int32_t head_dim;         /* D: 64 or 128                                                        */
+  int32_t dtype;            /* RAZOR_F32 or RAZOR_BF16: storage of K, V and q                      */
+  int32_t page_tokens;      /* tokens per page; must be 16                                         */
+  int32_t n_sink;           /* N0 of Algorithm 1 (Table 2: 4); >= 0                                */
+  int32_t max_ctx_len;      /* largest context length any sequence has at compression time        */
+  int32_t max_new_tokens;   /* append capacity per sequence after compression                      */
+  int32_t use_compensation; /* 1: Eq. 5.  0: plain truncation (sinks + window only, Table 1 scheme) */
+  int32_t page_shuffle_seed;/* 0: pages of a head are consecutive.  != 0: page ids are permuted
+                               (exercises the page indirection the way a serving allocator would)  */
+  float sm_scale;           /* multiplies every logit, the compensation logit included; 0 means
+                               1/sqrt(head_dim).  Eq. 3 and Eq. 5 print no scale: that is 1.0f     */
+} razor_config_t;
+
+/*
+ * Sizes of the two caller-owned device buffers (Algorithm 1, line 2 fixes how many tokens each
+ * head keeps).  ctx_len[B], window[B]: host; head_is_retrieval[L*Hkv]: host, 1 = the KV head keeps
+ * every token (for grouped-query models the caller ORs the flags of the group's query heads,
+ * Section 4.1).  pool_bytes covers every layer compressed once, with room for max_new_tokens
+ * appends; workspace_bytes depends on the config only.  Both are multiples of 256.
+ */
+RAZOR_API int razor_query_bytes(const razor_config_t* cfg, const int32_t* ctx_len, const int32_t* window,
+                      const uint8_t* head_is_retrieval, size_t* pool_bytes, size_t* workspace_bytes);
+
+/*
+ * Create a cache over caller-owned device memory.  pool_dev and workspace_dev must be 256-byte
+ * aligned and stay valid until razor_cache_destroy.  The workspace is cleared on `stream`.
+ * Errors: NULL_PTR, INVALID_ARG, UNSUPPORTED_DIM, MISALIGNED, POOL_TOO_SMALL (workspace), CUDA.
+ */
+RAZOR_API int razor_cache_create(razor_cache_t** out, const razor_config_t* cfg, void* pool_dev, size_t pool_bytes,
+                       void* workspace_dev, size_t workspace_bytes, void* stream);
+
+/*
+ * Prefill-end compression of one layer (Algorithm 1 lines 1-4, Eq. 4).
+ *   K, V     device, [B, Hkv, N, D] with element strides stride_b / stride_h / stride_n (innermost
+ *            dimension contiguous); rows at or beyond ctx_len[b] are never read.  Base pointers
+ *            16-byte aligned, strides multiples of 16 bytes.
+ *   ctx_len  host [B]: tokens of each sequence (0 <= ctx_len[b] <= max_ctx_len)
+ *   head_is_retrieval  host [Hkv] for this layer
+ *   n_sink   must equal config.n_sink
+ *   window   host [B]: recent-window length L_h of each sequence (>= 0); the caller evaluates
+ *            max(S0, N/C) of Algorithm 1 line 2
+ * A retrieval head, and any head with ctx_len <= n_sink + window, keeps positions [0, N).  Any
+ * other head keeps [0, n_sink) and [N - window, N); positions [n_sink, N - window) are summed in
+ * fp32 into its compensation sums, and the means and the count N_d are stored.  Kept rows are
+ * copied bit for bit into the page pool in ascending position order.  Compressing a layer again
+ * reuses its pages when the new plan fits in them.
+ * Errors: NULL_PTR, INVALID_ARG, MISALIGNED, CAPACITY (ctx_len > max_ctx_len), POOL_TOO_SMALL, CUDA.
+ */
+RAZOR_API int razor_compress(razor_cache_t* cache, int32_t layer, const void* K, const void* V, int64_t stride_b,
+                   int64_t stride_h, int64_t stride_n, const int32_t* ctx_len,
+                   const uint8_t* head_is_retrieval, int32_t n_sink, const int32_t* window, void* stream);
+
+/*
+ * The same for ONE sequence b of the batch (serving admission: sequences arrive one at a time and
+ * their dense K/V need not coexist).  K, V device [Hkv, N, D] with strides stride_h / stride_n.
+ * head_is_retrieval must be the same for every sequence of a layer.
+ */
+RAZOR_API int razor_compress_seq(razor_cache_t* cache, int32_t layer, int32_t b, const void* K, const void* V,
+                       int64_t stride_h, int64_t stride_n, int32_t ctx_len, const uint8_t* head_is_retrieval,
+                       int32_t n_sink, int32_t window, void* stream);
+
+/*
+ * Add one decode token per sequence to a compressed layer.  k_new, v_new: device [B, Hkv, D],
+ * contiguous.  Retrieval heads, and heads whose window is not yet full, store the row in the next
+ * slot.  A head with a full window first folds its oldest recent token into the compensation sums
+ * (count + 1, means recomputed: Eq. 4 over all tokens dropped so far), then stores the new row in
+ * that slot; the window length stays what it was at compression (the paper does not say how the
+ * cache grows while decoding).  Hence t appends leave exactly the state that compressing the
+ * (N + t)-token context with the same window would.
+ * Errors: NULL_PTR, INVALID_ARG, NOT_COMPRESSED, CAPACITY (more than max_new_tokens appends), CUDA.
+ */
+RAZOR_API int razor_append(razor_cache_t* cache, int32_t layer, const void* k_new, const void* v_new, void* stream);
+
+/*
+ * Decode attention of one query token per sequence over the compressed layer (Eq. 5; Algorithm 1
+ * line 5).  q: device [B, Hq, D] contiguous, config.dtype.  out: device [B, Hq, D] fp32.
+ * Query head j reads KV head j / group.  For a head with N_d > 0 dropped tokens
+ *   out = (N_d e^{s_c} v_hat + sum_kept e^{s_n} v_n) / (N_d e^{s_c} + sum_kept e^{s_n}),
+ *   s_n = sm_scale q.k_n,  s_c = sm_scale q.k_hat;
+ * other heads get softmax attention over all their tokens.  A sequence with no tokens gives zeros.
+ * Call razor_append first when the query token should attend to itself.
+ * Errors: NULL_PTR, INVALID_ARG, NOT_COMPRESSED, CUDA.
+ */
+RAZOR_API int razor_decode_attention(razor_cache_t* cache, int32_t layer, const void* q, float* out, void* stream);
+
+/*
+ * Read back the compressed state of one (layer, sequence, KV head) in LOGICAL order (ascending
+ * original position), whatever the physical slot order is.  Device outputs, any of which may be
+ * NULL: kept_pos int32[n_kept]; K, V [n_kept, D] in config.dtype; comp_mean_k/v and comp_sum_k/v
+ * fp32[D].  Host outputs (may be NULL): n_kept, n_drop.  n_kept is known on the host without a
+ * device read, so call once with NULL device pointers to size the buffers.  Snapshot and parity probe.
+ */
+RAZOR_API int razor_cache_export(razor_cache_t* cache, int32_t layer, int32_t b, int32_t kv_head, int32_t* kept_pos,
+                       void* K, void* V, float* comp_mean_k, float* comp_mean_v, float* comp_sum_k,
+                       float* comp_sum_v, int32_t* n_kept, int32_t* n_drop, void* stream);
+
+/* Host-side accounting of one layer: bytes of kept K+V rows and of the dense cache they stand for. */
+RAZOR_API int razor_cache_stats(const razor_cache_t* cache, int32_t layer, size_t* kept_bytes, size_t* dense_bytes);
+
+/*
+ * The decode work schedule (host only; no device is touched).  Every (sequence, KV head) token
+ * stream is cut into page ranges of near-equal size so that one launch is balanced over the SMs
+ * whatever the mix of full-length and short heads; ranges are ordered longest first.
+ *   razor_schedule_plan   plans for given stream lengths: tokens host int32[n_heads] (tokens stored
+ *                         per head), target_items = how many ranges to aim for (>= 1).
+ *   razor_schedule_query  the plan the next razor_decode_attention of `layer` would use.
+ * items: host int32[max_items][4] = {head index b*Hkv + kv_head, first_page, end_page,
+ * parts_of_this_head}, may be NULL; n_items receives the count.  A page is 16 tokens.
+ * Errors: NULL_PTR, INVALID_ARG (also when max_items is too small), NOT_COMPRESSED.
+ */
+RAZOR_API int razor_schedule_plan(const int32_t* tokens, int32_t n_heads, int32_t target_items, int32_t* items,
+                        int32_t max_items, int32_t* n_items);
+RAZOR_API int razor_schedule_query(razor_cache_t* cache, int32_t layer, int32_t* items, int32_t max_items,
+                         int32_t* n_items);
+
+/* Forget every compressed layer and give all pages back (the handle and buffers stay usable). */
+RAZOR_API int razor_cache_reset(razor_cache_t* cache);
+
+/* Free the host-side handle.  Device buffers belong to the caller. */
+RAZOR_API int razor_cache_destroy(razor_cache_t* cache);
+
+/* Text for a status code; never NULL. */
+RAZOR_API const char* razor_status_string(int status);
+
+/* cudaError_t value of the last failed CUDA call seen by this library in this thread (0 if none). */
+RAZOR_API int razor_last_cuda_error(void);
+
+/* Library version, "major.minor". */
+RAZOR_API const char* razor_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RAZOR_H_ */

@@ -1,0 +1,289 @@
+"""Thin ctypes binding of librazor.so (include/razor.h).  Argument marshalling only.
+
+Every step of the hot path runs in the library's CUDA kernels; torch is used here for device
+memory (`torch.empty`, `data_ptr`) and for the current stream.  There is no CPU or PyTorch
+fallback: if the library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Sequence, Tuple
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "librazor.so")
+
+RAZOR_F32, RAZOR_BF16 = 0, 1
+STATUS = {
+    0: "RAZOR_OK", -1: "RAZOR_E_INVALID_ARG", -2: "RAZOR_E_NULL_PTR", -3: "RAZOR_E_UNSUPPORTED_DIM",
+    -4: "RAZOR_E_POOL_TOO_SMALL", -5: "RAZOR_E_CAPACITY", -6: "RAZOR_E_NOT_COMPRESSED", -7: "RAZOR_E_CUDA",
+    -8: "RAZOR_E_MISALIGNED",
+}
+
+# every symbol include/razor.h declares
+SYMBOLS = [
+    "razor_query_bytes", "razor_cache_create", "razor_compress", "razor_compress_seq", "razor_append",
+    "razor_decode_attention", "razor_cache_export", "razor_cache_stats", "razor_schedule_plan",
+    "razor_schedule_query", "razor_cache_reset", "razor_cache_destroy", "razor_status_string",
+    "razor_last_cuda_error", "razor_version",
+]
+
+
+class RazorError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        lib = _lib
+        msg = lib.razor_status_string(status).decode() if lib is not None else "?"
+        extra = f" (cudaError {lib.razor_last_cuda_error()})" if status == -7 and lib is not None else ""
+        super().__init__(f"{where}: {STATUS.get(status, status)}: {msg}{extra}")
+
+
+class RazorConfig(C.Structure):
+    _fields_ = [
+        ("batch", C.c_int32), ("n_layers", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
+        ("head_dim", C.c_int32), ("dtype", C.c_int32), ("page_tokens", C.c_int32), ("n_sink", C.c_int32),
+        ("max_ctx_len", C.c_int32), ("max_new_tokens", C.c_int32), ("use_compensation", C.c_int32),
+        ("page_shuffle_seed", C.c_int32), ("sm_scale", C.c_float),
+    ]
+
+
+_lib: Optional[C.CDLL] = None
+
+
+def load() -> C.CDLL:
+    """Load librazor.so; raises if it has not been built (python -m paper_2407_15891_b200.build)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2407_15891_b200.build` "
+                          "(there is no fallback path)")
+    lib = C.CDLL(LIB_PATH)
+    vp, i32, i64, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_size_t
+    cfgp = C.POINTER(RazorConfig)
+    lib.razor_query_bytes.argtypes = [cfgp, vp, vp, vp, C.POINTER(sz), C.POINTER(sz)]
+    lib.razor_cache_create.argtypes = [C.POINTER(vp), cfgp, vp, sz, vp, sz, vp]
+    lib.razor_compress.argtypes = [vp, i32, vp, vp, i64, i64, i64, vp, vp, i32, vp, vp]
+    lib.razor_compress_seq.argtypes = [vp, i32, i32, vp, vp, i64, i64, i32, vp, i32, i32, vp]
+    lib.razor_append.argtypes = [vp, i32, vp, vp, vp]
+    lib.razor_decode_attention.argtypes = [vp, i32, vp, vp, vp]
+    lib.razor_cache_export.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, C.POINTER(i32),
+                                       C.POINTER(i32), vp]
+    lib.razor_cache_stats.argtypes = [vp, i32, C.POINTER(sz), C.POINTER(sz)]
+    lib.razor_schedule_plan.argtypes = [vp, i32, i32, vp, i32, C.POINTER(i32)]
+    lib.razor_schedule_query.argtypes = [vp, i32, vp, i32, C.POINTER(i32)]
+    lib.razor_cache_reset.argtypes = [vp]
+    lib.razor_cache_destroy.argtypes = [vp]
+    lib.razor_status_string.argtypes = [C.c_int]
+    lib.razor_status_string.restype = C.c_char_p
+    lib.razor_last_cuda_error.argtypes = []
+    lib.razor_version.argtypes = []
+    lib.razor_version.restype = C.c_char_p
+    for name in SYMBOLS:
+        fn = getattr(lib, name)
+        if fn.restype is C.c_int and name not in ("razor_status_string", "razor_version"):
+            fn.restype = C.c_int
+    _lib = lib
+    return lib
+
+
+def _check(status: int, where: str) -> None:
+    if status != 0:
+        raise RazorError(status, where)
+
+
+def _i32(a: Sequence[int]) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(a, dtype=np.int32))
+
+
+def _u8(a: Sequence[int]) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(a, dtype=np.uint8))
+
+
+def _ptr(t) -> Optional[int]:
+    if t is None:
+        return None
+    if isinstance(t, torch.Tensor):
+        return t.data_ptr()
+    if isinstance(t, np.ndarray):
+        return t.ctypes.data
+    return int(t)
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    return int(stream) or None
+
+
+def make_config(batch, n_layers, n_q_heads, n_kv_heads, head_dim, dtype, n_sink, max_ctx_len, max_new_tokens,
+                use_compensation=1, page_shuffle_seed=0, sm_scale=0.0, page_tokens=16) -> RazorConfig:
+    dt = {torch.float32: RAZOR_F32, torch.bfloat16: RAZOR_BF16, "f32": RAZOR_F32, "bf16": RAZOR_BF16}.get(dtype, dtype)
+    return RazorConfig(batch, n_layers, n_q_heads, n_kv_heads, head_dim, dt, page_tokens, n_sink, max_ctx_len,
+                       max_new_tokens, use_compensation, page_shuffle_seed, sm_scale)
+
+
+# ----------------------------------------------------------------------------- the C-ABI calls, same names
+def razor_version() -> str:
+    return load().razor_version().decode()
+
+
+def razor_status_string(status: int) -> str:
+    return load().razor_status_string(status).decode()
+
+
+def razor_query_bytes(cfg: RazorConfig, ctx_len, window, head_is_retrieval) -> Tuple[int, int]:
+    """-> (pool_bytes, workspace_bytes).  head_is_retrieval: [L*Hkv] (or [L, Hkv])."""
+    a, w, r = _i32(ctx_len), _i32(window), _u8(np.asarray(head_is_retrieval).reshape(-1))
+    pool, ws = C.c_size_t(0), C.c_size_t(0)
+    _check(load().razor_query_bytes(C.byref(cfg), a.ctypes.data, w.ctypes.data, r.ctypes.data, C.byref(pool),
+                                    C.byref(ws)), "razor_query_bytes")
+    return pool.value, ws.value
+
+
+def razor_cache_create(cfg: RazorConfig, pool, pool_bytes: int, workspace, workspace_bytes: int, stream=None) -> int:
+    h = C.c_void_p(None)
+    _check(load().razor_cache_create(C.byref(h), C.byref(cfg), _ptr(pool), pool_bytes, _ptr(workspace),
+                                     workspace_bytes, _stream(stream)), "razor_cache_create")
+    return h.value
+
+
+def razor_compress(cache: int, layer: int, K, V, stride_b: int, stride_h: int, stride_n: int, ctx_len,
+                   head_is_retrieval, n_sink: int, window, stream=None) -> None:
+    a, w, r = _i32(ctx_len), _i32(window), _u8(head_is_retrieval)
+    _check(load().razor_compress(cache, layer, _ptr(K), _ptr(V), stride_b, stride_h, stride_n, a.ctypes.data,
+                                 r.ctypes.data, n_sink, w.ctypes.data, _stream(stream)), "razor_compress")
+
+
+def razor_compress_seq(cache: int, layer: int, b: int, K, V, stride_h: int, stride_n: int, ctx_len: int,
+                       head_is_retrieval, n_sink: int, window: int, stream=None) -> None:
+    r = _u8(head_is_retrieval)
+    _check(load().razor_compress_seq(cache, layer, b, _ptr(K), _ptr(V), stride_h, stride_n, ctx_len, r.ctypes.data,
+                                     n_sink, window, _stream(stream)), "razor_compress_seq")
+
+
+def razor_append(cache: int, layer: int, k_new, v_new, stream=None) -> None:
+    _check(load().razor_append(cache, layer, _ptr(k_new), _ptr(v_new), _stream(stream)), "razor_append")
+
+
+def razor_decode_attention(cache: int, layer: int, q, out, stream=None) -> None:
+    _check(load().razor_decode_attention(cache, layer, _ptr(q), _ptr(out), _stream(stream)),
+           "razor_decode_attention")
+
+
+def razor_cache_export(cache: int, layer: int, b: int, kv_head: int, kept_pos=None, K=None, V=None, comp_mean_k=None,
+                       comp_mean_v=None, comp_sum_k=None, comp_sum_v=None, stream=None) -> Tuple[int, int]:
+    """-> (n_kept, n_drop); fills whichever device buffers are given."""
+    nk, nd = C.c_int32(0), C.c_int32(0)
+    _check(load().razor_cache_export(cache, layer, b, kv_head, _ptr(kept_pos), _ptr(K), _ptr(V), _ptr(comp_mean_k),
+                                     _ptr(comp_mean_v), _ptr(comp_sum_k), _ptr(comp_sum_v), C.byref(nk), C.byref(nd),
+                                     _stream(stream)), "razor_cache_export")
+    return nk.value, nd.value
+
+
+def razor_cache_stats(cache: int, layer: int) -> Tuple[int, int]:
+    """-> (kept_bytes, dense_bytes) of the layer's K+V rows."""
+    k, d = C.c_size_t(0), C.c_size_t(0)
+    _check(load().razor_cache_stats(cache, layer, C.byref(k), C.byref(d)), "razor_cache_stats")
+    return k.value, d.value
+
+
+def razor_schedule_plan(tokens, target_items: int) -> np.ndarray:
+    """Host-only: -> int32 [n_items, 4] = (head, first_page, end_page (-1: open), parts_of_head)."""
+    t = _i32(tokens)
+    n = C.c_int32(0)
+    lib = load()
+    _check(lib.razor_schedule_plan(t.ctypes.data, len(t), target_items, None, 0, C.byref(n)), "razor_schedule_plan")
+    items = np.zeros((n.value, 4), dtype=np.int32)
+    _check(lib.razor_schedule_plan(t.ctypes.data, len(t), target_items, items.ctypes.data, n.value, C.byref(n)),
+           "razor_schedule_plan")
+    return items
+
+
+def razor_schedule_query(cache: int, layer: int) -> np.ndarray:
+    n = C.c_int32(0)
+    lib = load()
+    _check(lib.razor_schedule_query(cache, layer, None, 0, C.byref(n)), "razor_schedule_query")
+    items = np.zeros((n.value, 4), dtype=np.int32)
+    _check(lib.razor_schedule_query(cache, layer, items.ctypes.data, n.value, C.byref(n)), "razor_schedule_query")
+    return items
+
+
+def razor_cache_reset(cache: int) -> None:
+    _check(load().razor_cache_reset(cache), "razor_cache_reset")
+
+
+def razor_cache_destroy(cache: int) -> None:
+    _check(load().razor_cache_destroy(cache), "razor_cache_destroy")
+
+
+# ----------------------------------------------------------------------------- convenience owner of the buffers
+class RazorCache:
+    """Owns the pool / workspace tensors and the handle.  Still marshalling only."""
+
+    def __init__(self, cfg: RazorConfig, ctx_len, window, head_is_retrieval, device="cuda:0", extra_pool_bytes=0):
+        if not torch.cuda.is_available():
+            raise RuntimeError("RazorCache needs a CUDA device (there is no CPU path)")
+        self.cfg = cfg
+        self.device = torch.device(device)
+        self.pool_bytes, self.ws_bytes = razor_query_bytes(cfg, ctx_len, window, head_is_retrieval)
+        self.pool_bytes += extra_pool_bytes
+        with torch.cuda.device(self.device):
+            self.pool = torch.empty(self.pool_bytes, dtype=torch.uint8, device=self.device)
+            self.workspace = torch.empty(self.ws_bytes, dtype=torch.uint8, device=self.device)
+            self.handle = razor_cache_create(cfg, self.pool, self.pool_bytes, self.workspace, self.ws_bytes)
+        self.tdtype = torch.bfloat16 if cfg.dtype == RAZOR_BF16 else torch.float32
+
+    def compress(self, layer: int, K: torch.Tensor, V: torch.Tensor, ctx_len, head_is_retrieval, window) -> None:
+        """K, V: [B, Hkv, N, D] device tensors (innermost dim contiguous, same strides)."""
+        assert K.stride() == V.stride() and K.stride(3) == 1
+        razor_compress(self.handle, layer, K, V, K.stride(0), K.stride(1), K.stride(2), ctx_len, head_is_retrieval,
+                       self.cfg.n_sink, window)
+
+    def compress_seq(self, layer: int, b: int, K: torch.Tensor, V: torch.Tensor, ctx_len: int, head_is_retrieval,
+                     window: int) -> None:
+        """K, V: [Hkv, N, D] device tensors of one sequence."""
+        assert K.stride() == V.stride() and K.stride(2) == 1
+        razor_compress_seq(self.handle, layer, b, K, V, K.stride(0), K.stride(1), ctx_len, head_is_retrieval,
+                           self.cfg.n_sink, window)
+
+    def append(self, layer: int, k_new: torch.Tensor, v_new: torch.Tensor) -> None:
+        assert k_new.is_contiguous() and v_new.is_contiguous()
+        razor_append(self.handle, layer, k_new, v_new)
+
+    def decode(self, layer: int, q: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        assert q.is_contiguous()
+        if out is None:
+            out = torch.empty(q.shape, dtype=torch.float32, device=q.device)
+        razor_decode_attention(self.handle, layer, q, out)
+        return out
+
+    def export(self, layer: int, b: int, kv_head: int):
+        """-> dict(kept_pos, K, V, mean_k, mean_v, sum_k, sum_v, n_drop) in logical order (device tensors)."""
+        n_kept, n_drop = razor_cache_export(self.handle, layer, b, kv_head)
+        D = self.cfg.head_dim
+        dev = self.device
+        kp = torch.empty(max(n_kept, 1), dtype=torch.int32, device=dev)
+        K = torch.empty((max(n_kept, 1), D), dtype=self.tdtype, device=dev)
+        V = torch.empty_like(K)
+        f = [torch.empty(D, dtype=torch.float32, device=dev) for _ in range(4)]
+        razor_cache_export(self.handle, layer, b, kv_head, kp, K, V, f[0], f[1], f[2], f[3])
+        return dict(kept_pos=kp[:n_kept], K=K[:n_kept], V=V[:n_kept], mean_k=f[0], mean_v=f[1], sum_k=f[2],
+                    sum_v=f[3], n_drop=n_drop)
+
+    def stats(self, layer: int):
+        return razor_cache_stats(self.handle, layer)
+
+    def close(self) -> None:
+        if getattr(self, "handle", None):
+            razor_cache_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,561 @@
+// Host side of the C ABI declared in include/razor.h: argument checks, the per-head plan
+// (Algorithm 1 line 2: how many tokens each head keeps), page allocation, host mirrors of the
+// per-head lengths (they are deterministic, so no device->host read is ever needed), the cached
+// decode schedule, and the kernel launches.
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "razor_internal.h"
+
+using namespace razor;
+
+namespace {
+
+thread_local int g_last_cuda_error = 0;
+
+#define RZ_CUDA(call)                          \
+  do {                                         \
+    cudaError_t e__ = (call);                  \
+    if (e__ != cudaSuccess) {                  \
+      g_last_cuda_error = (int)e__;            \
+      (void)cudaGetLastError();                \
+      return RAZOR_E_CUDA;                     \
+    }                                          \
+  } while (0)
+
+constexpr int kItemBudget = 16384;     // upper bound on split parts beyond one per head
+constexpr size_t kAlign = 256;
+
+inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+inline int ceil_div(long long a, long long b) { return (int)((a + b - 1) / b); }
+
+struct Layout {
+  size_t state, comp_sum, comp_mean, page_table, items, partials, tickets, queue, scratch, seq_desc, total;
+  int max_pages, max_items;
+};
+
+int check_config(const razor_config_t* c) {
+  if (!c) return RAZOR_E_NULL_PTR;
+  if (c->batch < 1 || c->n_layers < 1 || c->n_kv_heads < 1 || c->n_q_heads < 1) return RAZOR_E_INVALID_ARG;
+  if (c->n_q_heads % c->n_kv_heads) return RAZOR_E_INVALID_ARG;
+  const int g = c->n_q_heads / c->n_kv_heads;
+  if (g != 1 && g != 2 && g != 4 && g != 8) return RAZOR_E_UNSUPPORTED_DIM;
+  if (c->head_dim != 64 && c->head_dim != 128) return RAZOR_E_UNSUPPORTED_DIM;
+  if (c->dtype != RAZOR_F32 && c->dtype != RAZOR_BF16) return RAZOR_E_UNSUPPORTED_DIM;
+  if (c->page_tokens != kPageTokens) return RAZOR_E_UNSUPPORTED_DIM;
+  if (c->n_sink < 0 || c->max_ctx_len < 0 || c->max_new_tokens < 0) return RAZOR_E_INVALID_ARG;
+  if ((long long)c->max_ctx_len + c->max_new_tokens > (1LL << 30)) return RAZOR_E_INVALID_ARG;
+  if ((long long)c->batch * c->n_kv_heads > (1 << 20)) return RAZOR_E_INVALID_ARG;
+  if (!(c->sm_scale >= 0.f) || std::isinf(c->sm_scale)) return RAZOR_E_INVALID_ARG;
+  return RAZOR_OK;
+}
+
+inline size_t esz(const razor_config_t& c) { return c.dtype == RAZOR_BF16 ? 2 : 4; }
+inline size_t row_bytes(const razor_config_t& c) { return (size_t)c.head_dim * esz(c); }
+inline size_t page_bytes(const razor_config_t& c) { return 2 * (size_t)kPageTokens * row_bytes(c); }
+
+Layout make_layout(const razor_config_t& c) {
+  Layout l;
+  const size_t nh = (size_t)c.batch * c.n_kv_heads, L = c.n_layers, D = c.head_dim;
+  const int g = c.n_q_heads / c.n_kv_heads;
+  l.max_pages = std::max(1, ceil_div((long long)c.max_ctx_len + c.max_new_tokens, kPageTokens));
+  l.max_items = (int)nh + kItemBudget;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+  l.state = take(L * nh * sizeof(HeadState));
+  l.comp_sum = take(L * nh * 2 * D * sizeof(float));
+  l.comp_mean = take(L * nh * 2 * D * sizeof(float));
+  l.page_table = take(L * nh * (size_t)l.max_pages * sizeof(int32_t));
+  l.items = take(L * (size_t)l.max_items * sizeof(WorkItem));
+  l.partials = take((size_t)l.max_items * g * (kPartialPad + D) * sizeof(float));
+  l.tickets = take(nh * sizeof(int32_t));
+  l.queue = take(4 * sizeof(int32_t));
+  l.scratch = take(nh * kCompressMaxSlices * 2 * D * sizeof(float));
+  l.seq_desc = take((size_t)c.batch * sizeof(SeqDesc));
+  l.total = off;
+  return l;
+}
+
+// Tokens a head can ever hold (Algorithm 1 line 3 plus room for appended decode tokens).
+inline long long head_capacity_tokens(const razor_config_t& c, int n_ctx, int window, bool retrieval) {
+  const long long grown = (long long)n_ctx + c.max_new_tokens;
+  return retrieval ? grown : std::min(grown, (long long)c.n_sink + window);
+}
+
+struct LayerHost {
+  bool any = false;
+  int n_done = 0;
+  std::vector<uint8_t> retr;        // [Hkv]
+  std::vector<uint8_t> seq_done;    // [B]
+  std::vector<HeadState> hs;        // [B*Hkv] mirror of the device state
+  std::vector<long long> region_start, region_count;   // pages owned by (layer, b)
+  int appended = 0;
+  // decode schedule
+  bool sched_valid = false;
+  int n_items = 0, chunk_pages = 0, growth_tokens = 0;
+  WorkItem* items = nullptr;        // pinned host, [max_items]
+  cudaEvent_t upload_done = nullptr;
+};
+
+uint64_t mix64(uint64_t x) {
+  x += 0x9E3779B97F4A7C15ull;
+  x = (x ^ (x >> 30)) * 0xBF58476D1CE4E5B9ull;
+  x = (x ^ (x >> 27)) * 0x94D049BB133111EBull;
+  return x ^ (x >> 31);
+}
+
+}  // namespace
+
+struct razor_cache {
+  razor_config_t cfg;
+  Layout lay;
+  DeviceView dv;
+  long long pool_pages = 0, next_page = 0;
+  int n_sms = 148;
+  std::vector<LayerHost> layers;
+  WorkItem* pinned_items = nullptr;   // [L][max_items]
+};
+
+extern "C" {
+
+const char* razor_version(void) { return "0.1"; }
+
+int razor_last_cuda_error(void) { return g_last_cuda_error; }
+
+const char* razor_status_string(int s) {
+  switch (s) {
+    case RAZOR_OK: return "ok";
+    case RAZOR_E_INVALID_ARG: return "invalid argument";
+    case RAZOR_E_NULL_PTR: return "null pointer";
+    case RAZOR_E_UNSUPPORTED_DIM: return "unsupported head_dim, dtype, group size or page size";
+    case RAZOR_E_POOL_TOO_SMALL: return "page pool or workspace too small";
+    case RAZOR_E_CAPACITY: return "capacity exceeded (max_new_tokens or max_ctx_len)";
+    case RAZOR_E_NOT_COMPRESSED: return "layer or sequence not compressed yet";
+    case RAZOR_E_CUDA: return "CUDA runtime error (see razor_last_cuda_error)";
+    case RAZOR_E_MISALIGNED: return "pointer or stride not 16-byte aligned";
+    default: return "unknown status";
+  }
+}
+
+int razor_query_bytes(const razor_config_t* cfg, const int32_t* ctx_len, const int32_t* window,
+                      const uint8_t* head_is_retrieval, size_t* pool_bytes, size_t* workspace_bytes) {
+  int rc = check_config(cfg);
+  if (rc) return rc;
+  if (!ctx_len || !window || !head_is_retrieval) return RAZOR_E_NULL_PTR;
+  if (!pool_bytes && !workspace_bytes) return RAZOR_E_NULL_PTR;
+  unsigned long long pages = 0;
+  for (int b = 0; b < cfg->batch; ++b) {
+    if (ctx_len[b] < 0 || window[b] < 0) return RAZOR_E_INVALID_ARG;
+    if (ctx_len[b] > cfg->max_ctx_len) return RAZOR_E_CAPACITY;
+    for (int l = 0; l < cfg->n_layers; ++l)
+      for (int g = 0; g < cfg->n_kv_heads; ++g)
+        pages += ceil_div(head_capacity_tokens(*cfg, ctx_len[b], window[b],
+                                               head_is_retrieval[(size_t)l * cfg->n_kv_heads + g] != 0),
+                          kPageTokens);
+  }
+  if (pool_bytes) *pool_bytes = align_up(std::max<size_t>(1, pages) * page_bytes(*cfg));
+  if (workspace_bytes) *workspace_bytes = make_layout(*cfg).total;
+  return RAZOR_OK;
+}
+
+int razor_cache_create(razor_cache_t** out, const razor_config_t* cfg, void* pool_dev, size_t pool_bytes,
+                       void* workspace_dev, size_t workspace_bytes, void* stream) {
+  if (!out) return RAZOR_E_NULL_PTR;
+  *out = nullptr;
+  int rc = check_config(cfg);
+  if (rc) return rc;
+  if (!pool_dev || !workspace_dev) return RAZOR_E_NULL_PTR;
+  if (((uintptr_t)pool_dev | (uintptr_t)workspace_dev) & (kAlign - 1)) return RAZOR_E_MISALIGNED;
+  const Layout lay = make_layout(*cfg);
+  if (workspace_bytes < lay.total) return RAZOR_E_POOL_TOO_SMALL;
+  if (pool_bytes < page_bytes(*cfg)) return RAZOR_E_POOL_TOO_SMALL;
+
+  int dev = 0, sms = 0;
+  RZ_CUDA(cudaGetDevice(&dev));
+  RZ_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+
+  razor_cache* c = new (std::nothrow) razor_cache();
+  if (!c) return RAZOR_E_INVALID_ARG;
+  c->cfg = *cfg;
+  if (c->cfg.sm_scale == 0.f) c->cfg.sm_scale = 1.0f / std::sqrt((float)cfg->head_dim);
+  c->lay = lay;
+  c->n_sms = sms;
+  c->pool_pages = (long long)(pool_bytes / page_bytes(*cfg));
+  uint8_t* ws = (uint8_t*)workspace_dev;
+  DeviceView& dv = c->dv;
+  dv.pool = (uint8_t*)pool_dev;
+  dv.state = (HeadState*)(ws + lay.state);
+  dv.comp_sum = (float*)(ws + lay.comp_sum);
+  dv.comp_mean = (float*)(ws + lay.comp_mean);
+  dv.page_table = (int32_t*)(ws + lay.page_table);
+  dv.items = (WorkItem*)(ws + lay.items);
+  dv.partials = (float*)(ws + lay.partials);
+  dv.tickets = (int32_t*)(ws + lay.tickets);
+  dv.queue = (int32_t*)(ws + lay.queue);
+  dv.compress_scratch = (float*)(ws + lay.scratch);
+  dv.seq_desc = (SeqDesc*)(ws + lay.seq_desc);
+  dv.n_heads = cfg->batch * cfg->n_kv_heads;
+  dv.n_kv_heads = cfg->n_kv_heads;
+  dv.max_pages = lay.max_pages;
+  dv.max_items = lay.max_items;
+  dv.head_dim = cfg->head_dim;
+  dv.n_sink = cfg->n_sink;
+  dv.group = cfg->n_q_heads / cfg->n_kv_heads;
+  dv.use_comp = cfg->use_compensation ? 1 : 0;
+  dv.page_bytes = page_bytes(*cfg);
+  dv.scale_log2 = c->cfg.sm_scale * 1.4426950408889634f;
+
+  cudaError_t e = cudaMemsetAsync(workspace_dev, 0, lay.total, (cudaStream_t)stream);
+  if (e == cudaSuccess)
+    e = cudaHostAlloc((void**)&c->pinned_items, (size_t)cfg->n_layers * lay.max_items * sizeof(WorkItem),
+                      cudaHostAllocDefault);
+  if (e != cudaSuccess) {
+    g_last_cuda_error = (int)e;
+    (void)cudaGetLastError();
+    delete c;
+    return RAZOR_E_CUDA;
+  }
+  c->layers.resize(cfg->n_layers);
+  for (int l = 0; l < cfg->n_layers; ++l) {
+    LayerHost& L = c->layers[l];
+    L.retr.assign(cfg->n_kv_heads, 0);
+    L.seq_done.assign(cfg->batch, 0);
+    L.hs.assign((size_t)dv.n_heads, HeadState{0, 0, 0, 0});
+    L.region_start.assign(cfg->batch, 0);
+    L.region_count.assign(cfg->batch, 0);
+    L.items = c->pinned_items + (size_t)l * lay.max_items;
+  }
+  *out = c;
+  return RAZOR_OK;
+}
+
+int razor_cache_reset(razor_cache_t* c) {
+  if (!c) return RAZOR_E_NULL_PTR;
+  c->next_page = 0;
+  for (LayerHost& L : c->layers) {
+    L.any = false;
+    L.n_done = 0;
+    L.appended = 0;
+    L.sched_valid = false;
+    std::fill(L.seq_done.begin(), L.seq_done.end(), 0);
+    std::fill(L.region_count.begin(), L.region_count.end(), 0);
+    std::fill(L.hs.begin(), L.hs.end(), HeadState{0, 0, 0, 0});
+  }
+  return RAZOR_OK;
+}
+
+int razor_cache_destroy(razor_cache_t* c) {
+  if (!c) return RAZOR_E_NULL_PTR;
+  for (LayerHost& L : c->layers)
+    if (L.upload_done) cudaEventDestroy(L.upload_done);
+  if (c->pinned_items) cudaFreeHost(c->pinned_items);
+  delete c;
+  return RAZOR_OK;
+}
+
+}  // extern "C"
+
+namespace {
+
+struct SeqIn {
+  int b;
+  const void* K;
+  const void* V;
+  int64_t stride_h, stride_n;
+  int n_ctx, window;
+};
+
+// Shared body of razor_compress / razor_compress_seq: the plan (C0), page allocation, uploads, launch.
+int compress_impl(razor_cache* c, int layer, const std::vector<SeqIn>& seqs, const uint8_t* retr, int n_sink,
+                  cudaStream_t stream) {
+  const razor_config_t& cfg = c->cfg;
+  if (layer < 0 || layer >= cfg.n_layers) return RAZOR_E_INVALID_ARG;
+  if (n_sink != cfg.n_sink) return RAZOR_E_INVALID_ARG;
+  LayerHost& L = c->layers[layer];
+  const int H = cfg.n_kv_heads;
+  const size_t es = esz(cfg);
+  std::vector<uint8_t> flags(H);
+  for (int g = 0; g < H; ++g) flags[g] = retr[g] ? 1 : 0;
+
+  // The retrieval set belongs to the layer: sequences compressed one at a time must agree on it.
+  bool others_done = false;
+  {
+    std::vector<uint8_t> in_call(cfg.batch, 0);
+    for (const SeqIn& s : seqs) in_call[s.b] = 1;
+    for (int b = 0; b < cfg.batch; ++b) others_done |= (L.seq_done[b] && !in_call[b]);
+  }
+  if (others_done && std::memcmp(flags.data(), L.retr.data(), H) != 0) return RAZOR_E_INVALID_ARG;
+
+  int n_max = 0;
+  for (const SeqIn& s : seqs) {
+    if (s.b < 0 || s.b >= cfg.batch) return RAZOR_E_INVALID_ARG;
+    if (s.n_ctx < 0 || s.window < 0) return RAZOR_E_INVALID_ARG;
+    if (s.n_ctx > cfg.max_ctx_len) return RAZOR_E_CAPACITY;
+    if (s.n_ctx > 0) {
+      if (!s.K || !s.V) return RAZOR_E_NULL_PTR;
+      if (((uintptr_t)s.K | (uintptr_t)s.V) & 15) return RAZOR_E_MISALIGNED;
+      if (((s.stride_h * (int64_t)es) | (s.stride_n * (int64_t)es)) & 15) return RAZOR_E_MISALIGNED;
+      if (s.stride_n < cfg.head_dim || s.stride_h < 0) return RAZOR_E_INVALID_ARG;
+    }
+    n_max = std::max(n_max, s.n_ctx);
+  }
+
+  // Page plan per sequence; allocate (or reuse) the sequence's region, all-or-nothing.
+  std::vector<long long> need(seqs.size());
+  long long next = c->next_page;
+  std::vector<long long> new_start(seqs.size(), -1);
+  for (size_t i = 0; i < seqs.size(); ++i) {
+    long long pages = 0;
+    for (int g = 0; g < H; ++g)
+      pages += ceil_div(head_capacity_tokens(cfg, seqs[i].n_ctx, seqs[i].window, flags[g] != 0), kPageTokens);
+    need[i] = pages;
+    if (pages > L.region_count[seqs[i].b]) {
+      if (next + pages > c->pool_pages) return RAZOR_E_POOL_TOO_SMALL;
+      new_start[i] = next;
+      next += pages;
+    }
+  }
+  c->next_page = next;
+
+  std::vector<int32_t> rows((size_t)H * c->lay.max_pages);
+  std::vector<HeadState> states(H);
+  std::vector<SeqDesc> descs(seqs.size());
+  for (size_t i = 0; i < seqs.size(); ++i) {
+    const SeqIn& s = seqs[i];
+    if (new_start[i] >= 0) {
+      L.region_start[s.b] = new_start[i];
+      L.region_count[s.b] = need[i];
+    }
+    // page ids of the region, optionally permuted
+    std::vector<int32_t> ids((size_t)need[i]);
+    for (long long k = 0; k < need[i]; ++k) ids[(size_t)k] = (int32_t)(L.region_start[s.b] + k);
+    if (cfg.page_shuffle_seed) {
+      uint64_t st = mix64((uint64_t)cfg.page_shuffle_seed * 1315423911ull + (uint64_t)layer * 2654435761ull + s.b);
+      for (long long k = need[i] - 1; k > 0; --k) {
+        st = mix64(st);
+        std::swap(ids[(size_t)k], ids[(size_t)(st % (uint64_t)(k + 1))]);
+      }
+    }
+    std::fill(rows.begin(), rows.end(), 0);
+    size_t cursor = 0;
+    for (int g = 0; g < H; ++g) {
+      const bool r = flags[g] != 0;
+      const int cap_pages = ceil_div(head_capacity_tokens(cfg, s.n_ctx, s.window, r), kPageTokens);
+      for (int k = 0; k < cap_pages; ++k) rows[(size_t)g * c->lay.max_pages + k] = ids[cursor++];
+      const bool keep_all = r || s.n_ctx <= cfg.n_sink + s.window;
+      HeadState h;
+      h.len = keep_all ? s.n_ctx : cfg.n_sink + s.window;
+      h.n_drop = keep_all ? 0 : s.n_ctx - cfg.n_sink - s.window;
+      h.ring_head = 0;
+      h.window = r ? -1 : s.window;
+      states[g] = h;
+      L.hs[(size_t)s.b * H + g] = h;
+    }
+    const size_t head0 = (size_t)layer * c->dv.n_heads + (size_t)s.b * H;
+    RZ_CUDA(cudaMemcpyAsync(c->dv.page_table + head0 * c->lay.max_pages, rows.data(), rows.size() * sizeof(int32_t),
+                            cudaMemcpyHostToDevice, stream));
+    RZ_CUDA(cudaMemcpyAsync(c->dv.state + head0, states.data(), states.size() * sizeof(HeadState),
+                            cudaMemcpyHostToDevice, stream));
+    SeqDesc d;
+    d.K = s.K; d.V = s.V; d.stride_h = s.stride_h; d.stride_n = s.stride_n;
+    d.n_ctx = s.n_ctx; d.window = s.window; d.b = s.b; d.pad = 0;
+    descs[i] = d;
+    if (!L.seq_done[s.b]) { L.seq_done[s.b] = 1; L.n_done += 1; }
+  }
+  RZ_CUDA(cudaMemcpyAsync(c->dv.seq_desc, descs.data(), descs.size() * sizeof(SeqDesc), cudaMemcpyHostToDevice,
+                          stream));
+  L.retr = flags;
+  L.any = true;
+  L.appended = 0;
+  L.sched_valid = false;
+
+  // Slices per head: enough CTAs to fill the machine, slices no shorter than 64 rows.
+  int slices = ceil_div((long long)c->n_sms * 8, (long long)seqs.size() * H);
+  slices = std::max(1, std::min({slices, kCompressMaxSlices, std::max(1, n_max / 64)}));
+  RZ_CUDA(launch_compress(c->dv, cfg.dtype, layer, (int)seqs.size(), slices, stream));
+  return RAZOR_OK;
+}
+
+int ensure_schedule(razor_cache* c, int layer, cudaStream_t stream, bool upload) {
+  LayerHost& L = c->layers[layer];
+  const bool stale = !L.sched_valid || (long long)L.growth_tokens * 4 >= (long long)L.chunk_pages * kPageTokens;
+  if (!stale) return RAZOR_OK;
+  const int nh = c->dv.n_heads;
+  std::vector<int32_t> pages(nh);
+  for (int h = 0; h < nh; ++h) pages[h] = ceil_div(L.hs[h].len, kPageTokens);
+  if (L.upload_done) RZ_CUDA(cudaEventSynchronize(L.upload_done));   // previous upload has left the staging area
+  const int warps = c->n_sms * (c->dv.group == 1 ? 16 : 8);
+  const int n = build_schedule(pages.data(), nh, warps * 4, c->lay.max_items, L.items, &L.chunk_pages);
+  if (n < 0) return RAZOR_E_INVALID_ARG;
+  L.n_items = n;
+  L.growth_tokens = 0;
+  if (upload) {
+    if (!L.upload_done) RZ_CUDA(cudaEventCreateWithFlags(&L.upload_done, cudaEventDisableTiming));
+    RZ_CUDA(cudaMemcpyAsync(c->dv.items + (size_t)layer * c->lay.max_items, L.items, (size_t)n * sizeof(WorkItem),
+                            cudaMemcpyHostToDevice, stream));
+    RZ_CUDA(cudaEventRecord(L.upload_done, stream));
+    L.sched_valid = true;
+  } else {
+    L.sched_valid = false;   // the device copy no longer matches; the next decode uploads again
+  }
+  return RAZOR_OK;
+}
+
+inline int layer_ready(const razor_cache* c, int layer) {
+  if (layer < 0 || layer >= c->cfg.n_layers) return RAZOR_E_INVALID_ARG;
+  const LayerHost& L = c->layers[layer];
+  if (!L.any || L.n_done != c->cfg.batch) return RAZOR_E_NOT_COMPRESSED;
+  return RAZOR_OK;
+}
+
+int emit_items(const WorkItem* w, int n, int32_t* items, int32_t max_items, int32_t* n_items) {
+  *n_items = n;
+  if (!items) return RAZOR_OK;
+  if (max_items < n) return RAZOR_E_INVALID_ARG;
+  for (int i = 0; i < n; ++i) {
+    items[4 * i + 0] = w[i].head;
+    items[4 * i + 1] = w[i].page_begin;
+    items[4 * i + 2] = w[i].page_end;
+    items[4 * i + 3] = w[i].n_parts;
+  }
+  return RAZOR_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int razor_compress(razor_cache_t* c, int32_t layer, const void* K, const void* V, int64_t stride_b, int64_t stride_h,
+                   int64_t stride_n, const int32_t* ctx_len, const uint8_t* head_is_retrieval, int32_t n_sink,
+                   const int32_t* window, void* stream) {
+  if (!c || !ctx_len || !head_is_retrieval || !window) return RAZOR_E_NULL_PTR;
+  const size_t es = esz(c->cfg);
+  if ((stride_b * (int64_t)es) & 15) return RAZOR_E_MISALIGNED;
+  if (stride_b < 0) return RAZOR_E_INVALID_ARG;
+  std::vector<SeqIn> seqs(c->cfg.batch);
+  for (int b = 0; b < c->cfg.batch; ++b) {
+    SeqIn s;
+    s.b = b;
+    s.K = K ? (const char*)K + (size_t)b * stride_b * es : nullptr;
+    s.V = V ? (const char*)V + (size_t)b * stride_b * es : nullptr;
+    s.stride_h = stride_h;
+    s.stride_n = stride_n;
+    s.n_ctx = ctx_len[b];
+    s.window = window[b];
+    seqs[b] = s;
+  }
+  return compress_impl(c, layer, seqs, head_is_retrieval, n_sink, (cudaStream_t)stream);
+}
+
+int razor_compress_seq(razor_cache_t* c, int32_t layer, int32_t b, const void* K, const void* V, int64_t stride_h,
+                       int64_t stride_n, int32_t ctx_len, const uint8_t* head_is_retrieval, int32_t n_sink,
+                       int32_t window, void* stream) {
+  if (!c || !head_is_retrieval) return RAZOR_E_NULL_PTR;
+  std::vector<SeqIn> seqs(1);
+  seqs[0] = SeqIn{b, K, V, stride_h, stride_n, ctx_len, window};
+  return compress_impl(c, layer, seqs, head_is_retrieval, n_sink, (cudaStream_t)stream);
+}
+
+int razor_append(razor_cache_t* c, int32_t layer, const void* k_new, const void* v_new, void* stream) {
+  if (!c || !k_new || !v_new) return RAZOR_E_NULL_PTR;
+  int rc = layer_ready(c, layer);
+  if (rc) return rc;
+  if (((uintptr_t)k_new | (uintptr_t)v_new) & 15) return RAZOR_E_MISALIGNED;
+  LayerHost& L = c->layers[layer];
+  if (L.appended >= c->cfg.max_new_tokens) return RAZOR_E_CAPACITY;
+  RZ_CUDA(launch_append(c->dv, c->cfg.dtype, layer, k_new, v_new, (cudaStream_t)stream));
+  // Host mirror of the kernel's state update.
+  const int n_sink = c->cfg.n_sink;
+  for (HeadState& h : L.hs) {
+    if (h.window < 0 || h.len < n_sink + h.window) {
+      h.len += 1;
+    } else if (h.window == 0) {
+      h.n_drop += 1;
+    } else {
+      h.n_drop += 1;
+      h.ring_head = (h.ring_head + 1 == h.window) ? 0 : h.ring_head + 1;
+    }
+  }
+  L.appended += 1;
+  L.growth_tokens += 1;
+  return RAZOR_OK;
+}
+
+int razor_decode_attention(razor_cache_t* c, int32_t layer, const void* q, float* out, void* stream) {
+  if (!c || !q || !out) return RAZOR_E_NULL_PTR;
+  int rc = layer_ready(c, layer);
+  if (rc) return rc;
+  if (((uintptr_t)q | (uintptr_t)out) & 15) return RAZOR_E_MISALIGNED;
+  rc = ensure_schedule(c, layer, (cudaStream_t)stream, true);
+  if (rc) return rc;
+  RZ_CUDA(launch_decode(c->dv, c->cfg.dtype, layer, c->layers[layer].n_items, q, out, c->n_sms,
+                        (cudaStream_t)stream));
+  return RAZOR_OK;
+}
+
+int razor_cache_export(razor_cache_t* c, int32_t layer, int32_t b, int32_t kv_head, int32_t* kept_pos, void* K,
+                       void* V, float* comp_mean_k, float* comp_mean_v, float* comp_sum_k, float* comp_sum_v,
+                       int32_t* n_kept, int32_t* n_drop, void* stream) {
+  if (!c) return RAZOR_E_NULL_PTR;
+  if (layer < 0 || layer >= c->cfg.n_layers || b < 0 || b >= c->cfg.batch || kv_head < 0 ||
+      kv_head >= c->cfg.n_kv_heads)
+    return RAZOR_E_INVALID_ARG;
+  const LayerHost& L = c->layers[layer];
+  if (!L.any || !L.seq_done[b]) return RAZOR_E_NOT_COMPRESSED;
+  const int head = b * c->cfg.n_kv_heads + kv_head;
+  if (n_kept) *n_kept = L.hs[head].len;
+  if (n_drop) *n_drop = L.hs[head].n_drop;
+  if (kept_pos || K || V || comp_mean_k || comp_mean_v || comp_sum_k || comp_sum_v) {
+    if (((uintptr_t)K | (uintptr_t)V) & 15) return RAZOR_E_MISALIGNED;
+    RZ_CUDA(launch_export(c->dv, c->cfg.dtype, layer, head, kept_pos, K, V, comp_mean_k, comp_mean_v, comp_sum_k,
+                          comp_sum_v, (cudaStream_t)stream));
+  }
+  return RAZOR_OK;
+}
+
+int razor_cache_stats(const razor_cache_t* c, int32_t layer, size_t* kept_bytes, size_t* dense_bytes) {
+  if (!c) return RAZOR_E_NULL_PTR;
+  if (layer < 0 || layer >= c->cfg.n_layers) return RAZOR_E_INVALID_ARG;
+  const LayerHost& L = c->layers[layer];
+  if (!L.any) return RAZOR_E_NOT_COMPRESSED;
+  size_t kept = 0, dense = 0;
+  for (const HeadState& h : L.hs) {
+    kept += (size_t)h.len;
+    dense += (size_t)h.len + (size_t)h.n_drop;
+  }
+  const size_t per_token = 2 * row_bytes(c->cfg);
+  if (kept_bytes) *kept_bytes = kept * per_token;
+  if (dense_bytes) *dense_bytes = dense * per_token;
+  return RAZOR_OK;
+}
+
+int razor_schedule_plan(const int32_t* tokens, int32_t n_heads, int32_t target_items, int32_t* items,
+                        int32_t max_items, int32_t* n_items) {
+  if (!tokens || !n_items) return RAZOR_E_NULL_PTR;
+  if (n_heads < 1 || target_items < 1) return RAZOR_E_INVALID_ARG;
+  std::vector<int32_t> pages(n_heads);
+  for (int h = 0; h < n_heads; ++h) {
+    if (tokens[h] < 0) return RAZOR_E_INVALID_ARG;
+    pages[h] = ceil_div(tokens[h], kPageTokens);
+  }
+  const int cap = n_heads + kItemBudget;
+  std::vector<WorkItem> w(cap);
+  int chunk = 0;
+  const int n = build_schedule(pages.data(), n_heads, target_items, cap, w.data(), &chunk);
+  if (n < 0) return RAZOR_E_INVALID_ARG;
+  return emit_items(w.data(), n, items, max_items, n_items);
+}
+
+int razor_schedule_query(razor_cache_t* c, int32_t layer, int32_t* items, int32_t max_items, int32_t* n_items) {
+  if (!c || !n_items) return RAZOR_E_NULL_PTR;
+  int rc = layer_ready(c, layer);
+  if (rc) return rc;
+  rc = ensure_schedule(c, layer, nullptr, false);
+  if (rc) return rc;
+  return emit_items(c->layers[layer].items, c->layers[layer].n_items, items, max_items, n_items);
+}
+
+}  // extern "C"

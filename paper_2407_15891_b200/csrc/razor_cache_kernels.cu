@@ -1,0 +1,267 @@
+// Cache-building kernels: prefill-end compression (Algorithm 1 lines 2-3, Eq. 4), decode-token
+// append with fold-on-evict, and the logical-order export used for snapshots and parity checks.
+#include "razor_common.cuh"
+
+namespace razor {
+
+// ---------------------------------------------------------------------------------------------
+// Compression.  grid = (slices, Hkv, sequences); a CTA streams one slice of the rows of one
+// (sequence, KV head).  Every dense row is read exactly once: a kept row is copied bit for bit to its
+// page slot, a dropped row is added into per-thread fp32 accumulators.  The per-slice sums go to
+// scratch and are reduced in a fixed order by compress_finalize_kernel, so the compensation token
+// (Eq. 4) is reproducible from run to run.
+// Slot of a kept position p (ascending position order): retrieval head or N <= N0 + W: slot = p;
+// otherwise sinks p < N0 keep slot p and recent tokens p >= N - W go to N0 + (p - (N - W)).
+template <typename T, int D>
+__global__ void __launch_bounds__(256) compress_kernel(DeviceView dv, int layer, int n_slices) {
+  using Geo = RowGeom<T, D>;
+  constexpr int LPR = Geo::kLpr, EPL = Geo::kEpl, NGRP = 256 / LPR;
+  __shared__ float red[NGRP][2][D];
+
+  const SeqDesc sd = dv.seq_desc[blockIdx.z];
+  const int g = blockIdx.y;
+  const int head = sd.b * dv.n_kv_heads + g;
+  const HeadState st = dv.state[(size_t)layer * dv.n_heads + head];
+  const int N = sd.n_ctx, n_sink = dv.n_sink;
+  const bool keep_all = st.window < 0 || N <= n_sink + st.window;
+  const int recent0 = keep_all ? 0 : N - st.window;
+
+  const int rows_per_slice = (((N + n_slices - 1) / n_slices) + 15) & ~15;
+  const int r0 = blockIdx.x * rows_per_slice;
+  const int r1 = min(N, r0 + rows_per_slice);
+  const int lir = threadIdx.x % LPR, grp = threadIdx.x / LPR;
+
+  const char* Kb = (const char*)sd.K + (size_t)g * sd.stride_h * sizeof(T);
+  const char* Vb = (const char*)sd.V + (size_t)g * sd.stride_h * sizeof(T);
+  const size_t row_stride = (size_t)sd.stride_n * sizeof(T);
+  const int32_t* pt = dv.page_table + ((size_t)layer * dv.n_heads + head) * dv.max_pages;
+
+  float accK[EPL], accV[EPL];
+#pragma unroll
+  for (int i = 0; i < EPL; ++i) accK[i] = accV[i] = 0.f;
+
+  constexpr int UNROLL = 4;
+  for (int p0 = r0 + grp; p0 < r1; p0 += NGRP * UNROLL) {
+    uint4 kf[UNROLL], vf[UNROLL];
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+      const int p = p0 + u * NGRP;
+      if (p < r1) {
+        kf[u] = ld_stream((const uint4*)(Kb + (size_t)p * row_stride) + lir);
+        vf[u] = ld_stream((const uint4*)(Vb + (size_t)p * row_stride) + lir);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+      const int p = p0 + u * NGRP;
+      if (p >= r1) continue;
+      int slot;
+      if (keep_all || p < n_sink) slot = p;
+      else if (p >= recent0) slot = n_sink + (p - recent0);
+      else slot = -1;
+      if (slot >= 0) {
+        const size_t page = (size_t)pt[slot >> 4];
+        uint4* dst = (uint4*)(dv.pool + page * dv.page_bytes + (size_t)(slot & 15) * Geo::kRowBytes) + lir;
+        dst[0] = kf[u];
+        dst[kPageTokens * LPR] = vf[u];   // V rows follow the 16 K rows of the page
+      } else {
+        float a[EPL], b[EPL];
+        Elem<T>::unpack(kf[u], a);
+        Elem<T>::unpack(vf[u], b);
+#pragma unroll
+        for (int i = 0; i < EPL; ++i) { accK[i] += a[i]; accV[i] += b[i]; }
+      }
+    }
+  }
+
+#pragma unroll
+  for (int i = 0; i < EPL; ++i) {
+    red[grp][0][lir * EPL + i] = accK[i];
+    red[grp][1][lir * EPL + i] = accV[i];
+  }
+  __syncthreads();
+  float* scratch = dv.compress_scratch + ((size_t)head * kCompressMaxSlices + blockIdx.x) * 2 * D;
+  for (int e = threadIdx.x; e < 2 * D; e += 256) {
+    float s = 0.f;
+#pragma unroll
+    for (int r = 0; r < NGRP; ++r) s += (&red[r][0][0])[e];
+    scratch[e] = s;
+  }
+}
+
+// grid = (Hkv, sequences), block = 2*D threads: fixed-order sum of the slice partials, then the
+// means of Eq. 4 (zero when nothing was dropped, so no 0/0 is ever formed).
+template <int D>
+__global__ void compress_finalize_kernel(DeviceView dv, int layer, int n_slices) {
+  const SeqDesc sd = dv.seq_desc[blockIdx.y];
+  const int head = sd.b * dv.n_kv_heads + blockIdx.x;
+  const size_t hs = (size_t)layer * dv.n_heads + head;
+  const int n_drop = dv.state[hs].n_drop;
+  const float* scratch = dv.compress_scratch + (size_t)head * kCompressMaxSlices * 2 * D;
+  const int e = threadIdx.x;
+  float s = 0.f;
+  for (int i = 0; i < n_slices; ++i) s += scratch[(size_t)i * 2 * D + e];
+  if (n_drop == 0) s = 0.f;
+  dv.comp_sum[hs * 2 * D + e] = s;
+  dv.comp_mean[hs * 2 * D + e] = n_drop > 0 ? __fdiv_rn(s, (float)n_drop) : 0.f;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Append: one warp per (sequence, KV head).  A head that keeps everything, or whose window is not
+// full yet, stores the new row in slot `len`.  Otherwise the oldest recent token (ring slot
+// ring_head) is folded into the fp32 compensation sums, the count grows by one, the means are
+// recomputed (Eq. 4 over every token dropped so far) and the new row takes that slot.
+template <typename T, int D>
+__global__ void __launch_bounds__(128) append_kernel(DeviceView dv, int layer, const T* __restrict__ k_new,
+                                                     const T* __restrict__ v_new) {
+  using Geo = RowGeom<T, D>;
+  constexpr int LPR = Geo::kLpr, EPL = Geo::kEpl;
+  const int lane = threadIdx.x & 31;
+  const int head = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (head >= dv.n_heads) return;
+  const size_t hs = (size_t)layer * dv.n_heads + head;
+  HeadState st = dv.state[hs];
+  __syncwarp();
+  const int n_sink = dv.n_sink;
+  const bool keeps_all = st.window < 0;
+
+  int slot = -1;
+  bool evict = false, fold_new = false;
+  if (keeps_all || st.len < n_sink + st.window) {
+    slot = st.len;
+    st.len += 1;
+  } else if (st.window == 0) {
+    fold_new = true;                 // no recent window at all: the token is dropped at once
+    st.n_drop += 1;
+  } else {
+    slot = n_sink + st.ring_head;
+    evict = true;
+    st.n_drop += 1;
+    st.ring_head = (st.ring_head + 1 == st.window) ? 0 : st.ring_head + 1;
+  }
+
+  if (lane < LPR) {
+    const uint4 kf = ((const uint4*)(k_new + (size_t)head * D))[lane];
+    const uint4 vf = ((const uint4*)(v_new + (size_t)head * D))[lane];
+    uint4* krow = nullptr;
+    if (slot >= 0) {
+      const size_t page = (size_t)dv.page_table[hs * dv.max_pages + (slot >> 4)];
+      krow = (uint4*)(dv.pool + page * dv.page_bytes + (size_t)(slot & 15) * Geo::kRowBytes) + lane;
+    }
+    if (evict || fold_new) {
+      const uint4 ok = evict ? krow[0] : kf;
+      const uint4 ov = evict ? krow[kPageTokens * LPR] : vf;
+      float a[EPL], b[EPL];
+      Elem<T>::unpack(ok, a);
+      Elem<T>::unpack(ov, b);
+      float* sum = dv.comp_sum + hs * 2 * D + lane * EPL;
+      float* mean = dv.comp_mean + hs * 2 * D + lane * EPL;
+      const float cnt = (float)st.n_drop;
+#pragma unroll
+      for (int i = 0; i < EPL; ++i) {
+        const float sk = sum[i] + a[i], sv = sum[D + i] + b[i];
+        sum[i] = sk;
+        sum[D + i] = sv;
+        mean[i] = __fdiv_rn(sk, cnt);
+        mean[D + i] = __fdiv_rn(sv, cnt);
+      }
+    }
+    if (slot >= 0) {
+      krow[0] = kf;
+      krow[kPageTokens * LPR] = vf;
+    }
+  }
+  __syncwarp();
+  if (lane == 0) dv.state[hs] = st;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Export in logical order (ascending original position).  With T = len + n_drop tokens seen so far:
+// logical index i < N0 (or any i while nothing has been dropped) is position i in slot i; otherwise
+// j = i - N0 is the j-th oldest recent token: slot N0 + (ring_head + j) mod W, position T - W + j.
+template <typename T, int D>
+__global__ void __launch_bounds__(256) export_kernel(DeviceView dv, int layer, int head, int32_t* kept_pos, T* K,
+                                                     T* V, float* mean_k, float* mean_v, float* sum_k, float* sum_v) {
+  using Geo = RowGeom<T, D>;
+  constexpr int LPR = Geo::kLpr, NGRP = 256 / LPR;
+  const size_t hs = (size_t)layer * dv.n_heads + head;
+  const HeadState st = dv.state[hs];
+  const int n_sink = dv.n_sink;
+  const int lir = threadIdx.x % LPR, grp = threadIdx.x / LPR;
+  const int total = st.len + st.n_drop;
+  for (int i = blockIdx.x * NGRP + grp; i < st.len; i += gridDim.x * NGRP) {
+    int slot = i, pos = i;
+    if (st.n_drop > 0 && i >= n_sink) {
+      const int j = i - n_sink;
+      slot = n_sink + (st.ring_head + j) % st.window;
+      pos = total - st.window + j;
+    }
+    const size_t page = (size_t)dv.page_table[hs * dv.max_pages + (slot >> 4)];
+    const uint4* src = (const uint4*)(dv.pool + page * dv.page_bytes + (size_t)(slot & 15) * Geo::kRowBytes) + lir;
+    if (K) ((uint4*)(K + (size_t)i * D))[lir] = src[0];
+    if (V) ((uint4*)(V + (size_t)i * D))[lir] = src[kPageTokens * LPR];
+    if (kept_pos && lir == 0) kept_pos[i] = pos;
+  }
+  if (blockIdx.x == 0) {
+    for (int e = threadIdx.x; e < D; e += 256) {
+      if (mean_k) mean_k[e] = dv.comp_mean[hs * 2 * D + e];
+      if (mean_v) mean_v[e] = dv.comp_mean[hs * 2 * D + D + e];
+      if (sum_k) sum_k[e] = dv.comp_sum[hs * 2 * D + e];
+      if (sum_v) sum_v[e] = dv.comp_sum[hs * 2 * D + D + e];
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+template <typename T, int D>
+static cudaError_t compress_t(const DeviceView& dv, int layer, int n_seqs, int n_slices, cudaStream_t s) {
+  dim3 grid(n_slices, dv.n_kv_heads, n_seqs);
+  compress_kernel<T, D><<<grid, 256, 0, s>>>(dv, layer, n_slices);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  compress_finalize_kernel<D><<<dim3(dv.n_kv_heads, n_seqs), 2 * D, 0, s>>>(dv, layer, n_slices);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_compress(const DeviceView& dv, int dtype, int layer, int n_seqs, int n_slices, cudaStream_t s) {
+  if (dtype == RAZOR_BF16) {
+    return dv.head_dim == 128 ? compress_t<__nv_bfloat16, 128>(dv, layer, n_seqs, n_slices, s)
+                              : compress_t<__nv_bfloat16, 64>(dv, layer, n_seqs, n_slices, s);
+  }
+  return dv.head_dim == 128 ? compress_t<float, 128>(dv, layer, n_seqs, n_slices, s)
+                            : compress_t<float, 64>(dv, layer, n_seqs, n_slices, s);
+}
+
+template <typename T, int D>
+static cudaError_t append_t(const DeviceView& dv, int layer, const void* k, const void* v, cudaStream_t s) {
+  const int warps = 4;
+  append_kernel<T, D><<<(dv.n_heads + warps - 1) / warps, warps * 32, 0, s>>>(dv, layer, (const T*)k, (const T*)v);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_append(const DeviceView& dv, int dtype, int layer, const void* k, const void* v, cudaStream_t s) {
+  if (dtype == RAZOR_BF16) {
+    return dv.head_dim == 128 ? append_t<__nv_bfloat16, 128>(dv, layer, k, v, s)
+                              : append_t<__nv_bfloat16, 64>(dv, layer, k, v, s);
+  }
+  return dv.head_dim == 128 ? append_t<float, 128>(dv, layer, k, v, s) : append_t<float, 64>(dv, layer, k, v, s);
+}
+
+template <typename T, int D>
+static cudaError_t export_t(const DeviceView& dv, int layer, int head, int32_t* kp, void* K, void* V, float* mk,
+                            float* mv, float* sk, float* sv, cudaStream_t s) {
+  export_kernel<T, D><<<64, 256, 0, s>>>(dv, layer, head, kp, (T*)K, (T*)V, mk, mv, sk, sv);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_export(const DeviceView& dv, int dtype, int layer, int head, int32_t* kp, void* K, void* V,
+                          float* mk, float* mv, float* sk, float* sv, cudaStream_t s) {
+  if (dtype == RAZOR_BF16) {
+    return dv.head_dim == 128 ? export_t<__nv_bfloat16, 128>(dv, layer, head, kp, K, V, mk, mv, sk, sv, s)
+                              : export_t<__nv_bfloat16, 64>(dv, layer, head, kp, K, V, mk, mv, sk, sv, s);
+  }
+  return dv.head_dim == 128 ? export_t<float, 128>(dv, layer, head, kp, K, V, mk, mv, sk, sv, s)
+                            : export_t<float, 64>(dv, layer, head, kp, K, V, mk, mv, sk, sv, s);
+}
+
+}  // namespace razor

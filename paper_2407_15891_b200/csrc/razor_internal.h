@@ -1,0 +1,95 @@
+// Internal declarations shared by the host side (razor_api.cu, razor_schedule.cpp) and the kernels.
+// Nothing here is part of the public ABI (that is include/razor.h).
+#ifndef RAZOR_INTERNAL_H_
+#define RAZOR_INTERNAL_H_
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "razor.h"
+
+namespace razor {
+
+constexpr int kPageTokens = 16;        // tokens per page
+constexpr int kMaxGroup = 8;           // query heads per KV head
+constexpr int kCompressMaxSlices = 64; // row slices per (sequence, KV head) in the compression kernel
+constexpr int kMinChunkPages = 4;      // smallest decode work item
+constexpr int kPartialPad = 4;         // floats before o[] in a partial record: m, l, 2 x pad
+
+// Device-resident state of one (layer, sequence, KV head).  window < 0 marks a head that keeps every
+// token (retrieval head).  Physical slots: [0, n_sink) sinks, then the recent window as a ring whose
+// oldest element sits at ring index ring_head (Algorithm 1 line 3 keeps sinks + recent tokens).
+struct HeadState {
+  int32_t len;        // tokens stored (physical slots in use)
+  int32_t n_drop;     // N_d of Eq. 4: tokens folded into the compensation sums so far
+  int32_t ring_head;  // ring index of the oldest recent token
+  int32_t window;     // recent-window length; < 0: keeps everything
+};
+
+// One decode work item: pages [page_begin, page_end) of one head's token stream.  page_end < 0 means
+// "to the end of the stream as it is now" (the last part of a head grows with appends).
+struct WorkItem {
+  int32_t head;       // b * Hkv + kv_head
+  int32_t page_begin;
+  int32_t page_end;
+  int32_t part_idx;   // index of this part within its head
+  int32_t n_parts;    // parts of this head
+  int32_t part_base;  // first partial-record slot of this head
+  int32_t pad0, pad1;
+};
+
+// One sequence handed to the compression kernel.
+struct SeqDesc {
+  const void* K;
+  const void* V;
+  int64_t stride_h;   // elements
+  int64_t stride_n;   // elements
+  int32_t n_ctx;
+  int32_t window;
+  int32_t b;
+  int32_t pad;
+};
+
+// Pointers into the caller's workspace, plus the dimensions the kernels need.
+struct DeviceView {
+  uint8_t* pool;            // pages: [page][K rows | V rows][16][D]
+  HeadState* state;         // [L][B*Hkv]
+  float* comp_sum;          // [L][B*Hkv][2][D]  (K sums then V sums)
+  float* comp_mean;         // [L][B*Hkv][2][D]
+  int32_t* page_table;      // [L][B*Hkv][max_pages]
+  WorkItem* items;          // [L][max_items]
+  float* partials;          // [max_items][G][kPartialPad + D]
+  int32_t* tickets;         // [B*Hkv]
+  int32_t* queue;           // [4]: next item, warps done, spare
+  float* compress_scratch;  // [B*Hkv][kCompressMaxSlices][2][D]
+  SeqDesc* seq_desc;        // [B]
+  int32_t n_heads;          // B*Hkv
+  int32_t n_kv_heads;
+  int32_t max_pages;        // page-table row length
+  int32_t max_items;
+  int32_t head_dim;
+  int32_t n_sink;
+  int32_t group;
+  int32_t use_comp;
+  size_t page_bytes;
+  float scale_log2;         // sm_scale * log2(e)
+};
+
+// Kernel launchers (defined in the .cu files).  Each returns the cudaError_t of the launch.
+cudaError_t launch_compress(const DeviceView& dv, int dtype, int layer, int n_seqs, int n_slices,
+                            cudaStream_t stream);
+cudaError_t launch_append(const DeviceView& dv, int dtype, int layer, const void* k_new, const void* v_new,
+                          cudaStream_t stream);
+cudaError_t launch_decode(const DeviceView& dv, int dtype, int layer, int n_items, const void* q, float* out,
+                          int n_sms, cudaStream_t stream);
+cudaError_t launch_export(const DeviceView& dv, int dtype, int layer, int head, int32_t* kept_pos, void* K, void* V,
+                          float* mean_k, float* mean_v, float* sum_k, float* sum_v, cudaStream_t stream);
+
+// Host-only schedule builder (razor_schedule.cpp).  pages[h] = pages of head h's token stream now.
+// Returns the number of items written (<= max_items).
+int build_schedule(const int32_t* pages, int n_heads, int target_items, int max_items, WorkItem* out,
+                   int* chunk_pages_out);
+
+}  // namespace razor
+#endif

@@ -85,8 +85,13 @@ def stream_key(seed: int, tag: int, sub: int = 0) -> int:
 
 
 def normal_bf16(seed: int, tag: int, shape: Sequence[int], device="cpu", sub: int = 0,
-                out: Optional[torch.Tensor] = None, chunk: int = 1 << 26) -> torch.Tensor:
-    """Tensor of N(0,1) values rounded to bf16; element i depends on (seed, tag, sub, i) only."""
+                out: Optional[torch.Tensor] = None, chunk: int = 1 << 26, offset: int = 0) -> torch.Tensor:
+    """Tensor of N(0,1) values rounded to bf16; element i depends on (seed, tag, sub, offset + i) only.
+
+    `offset` (a multiple of 4) selects a window of a larger virtual tensor, so that one head of a
+    layer can be generated without the rest.
+    """
+    assert offset % 4 == 0
     n = int(np.prod(shape)) if len(shape) else 1
     dev = torch.device(device)
     if out is None:
@@ -98,12 +103,12 @@ def normal_bf16(seed: int, tag: int, shape: Sequence[int], device="cpu", sub: in
     shifts = torch.tensor([0, 16, 32, 48], dtype=torch.int64, device=dev)
     for start in range(0, n, chunk):
         stop = min(n, start + chunk)
-        g0, g1 = start >> 2, (stop + 3) >> 2
+        g0, g1 = (offset + start) >> 2, (offset + stop + 3) >> 2
         g = torch.arange(g0, g1, dtype=torch.int64, device=dev)
         h = _splitmix64_t(g ^ key)
         lanes = ((h.unsqueeze(1) >> shifts) & 0xFFFF).reshape(-1)
         vals = table[lanes]
-        lo = start - (g0 << 2)
+        lo = offset + start - (g0 << 2)
         flat[start:stop] = vals[lo:lo + (stop - start)]
     return out.view(*shape)
 
@@ -270,6 +275,19 @@ def make_dense_kv(w: Workload, layer: int, device="cpu", needle_beta: float = 20
                 for p in needle_positions(w, layer, b, h):
                     if p < w.ctx_len[b]:
                         k[b, h, p, :] = needle[b, h]
+    if w.dtype == "f32":
+        return k.float(), v.float()
+    return k, v
+
+
+def make_dense_head(w: Workload, layer: int, b: int, g: int, device="cpu"):
+    """K, V [N_max, D] of one (sequence, KV head): the same values make_dense_kv gives at [b, g],
+    generated alone (needle keys excepted: they depend on the queries and are not planted here)."""
+    N, D = w.n_max, w.head_dim
+    off = ((b * w.n_kv_heads) + g) * N * D
+    k = normal_bf16(w.seed, TAG_K, (N, D), device, sub=layer, offset=off)
+    v = normal_bf16(w.seed, TAG_V, (N, D), device, sub=layer, offset=off)
+    k[: w.n_sink, :] *= 4.0
     if w.dtype == "f32":
         return k.float(), v.float()
     return k, v

@@ -1,0 +1,240 @@
+"""GPU parity tests: the CUDA library (through its C ABI) against the CPU oracle on the same seeded
+inputs.  Layout bit-exact; means within 1e-3 relative; outputs within 3e-3 (bf16) / 1e-5 (fp32)."""
+import copy
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import razor_oracle as orc
+from paper_2407_15891_b200 import binding as rz
+from paper_2407_15891_b200 import synth
+
+from _harness import TOL_OUT, bits, make_cache, run_parity, sample_heads, to_f64
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def small(name, **kw):
+    w = copy.copy(synth.workload(name))
+    for k, v in kw.items():
+        setattr(w, k, v)
+    return w
+
+
+# ------------------------------------------------------------------ the five configurations
+def test_cfg1_tiny_fp32_every_head():
+    w = synth.workload("cfg1")
+    st = {}
+    r = run_parity(w, steps=0, stats=st)
+    assert r["heads"] == 4 and r["outputs"] == 4
+    # and with one appended token (the query then attends to itself)
+    r = run_parity(w, steps=1)
+    assert r["out"] <= 1e-5
+
+
+def test_cfg1_needle_recalled_only_by_retrieval_head():
+    w = synth.workload("cfg1")
+    cache = make_cache(w)
+    K, V = synth.make_dense_kv(w, 0, DEV)
+    cache.compress(0, K, V, w.ctx_len, w.retrieval(0), w.window)
+    out = cache.decode(0, synth.make_queries(w, 0, 0, DEV)).cpu()
+    v200 = V[0, :, 200, :].cpu()
+    assert (out[0, 0] - v200[0]).abs().max() < 0.05
+    for h in (1, 2, 3):
+        assert (out[0, h] - v200[h]).abs().max() > 0.5
+    cache.close()
+
+
+def test_cfg2_llama2_7b_shaped_32k_every_head():
+    w = synth.workload("cfg2")
+    st = {}
+    r = run_parity(w, steps=0, stats=st)
+    assert r["heads"] == 8 * 32
+    assert st["kept_bytes"] == w.compressed_bytes(0) and st["dense_bytes"] == w.dense_bytes()
+
+
+def test_cfg3_llama2_13b_64k_full_stack_16_steps_sampled():
+    w = synth.workload("cfg3")
+    layers = [0, 13, 26, 39]
+    heads = {l: sample_heads(w, l, 2, 3, range(w.batch)) for l in layers}
+    r = run_parity(w, layers=layers, heads_for=heads, steps=16, check_layout_every=5)
+    assert r["outputs"] == 4 * 4 * 5 * 16
+
+
+def test_cfg4_gqa_llama3_8b_shaped_128k_sampled():
+    w = synth.workload("cfg4")
+    layers = [0, 15, 31]
+    heads = {l: sample_heads(w, l, 2, 3, range(w.batch)) for l in layers}
+    r = run_parity(w, layers=layers, heads_for=heads, steps=0)
+    assert r["outputs"] == 3 * 2 * 5 * 4
+    r = run_parity(w, layers=layers, heads_for={l: heads[l][:3] for l in layers}, steps=2)
+
+
+def test_cfg5_ragged_serving_mix_64_steps_sampled():
+    w = synth.workload("cfg5")
+    order = np.argsort(w.ctx_len)
+    bs = [int(order[0]), int(order[len(order) // 2]), int(order[-1])]      # shortest, median, longest
+    heads = {0: sample_heads(w, 0, 1, 2, bs)}
+    r = run_parity(w, layers=[0], heads_for=heads, steps=64, per_seq=True, check_layout_every=16)
+    assert r["outputs"] == 3 * 3 * 64
+
+
+# ------------------------------------------------------------------ scaled copies, every head, paged
+@pytest.mark.parametrize("name,scale", [("cfg2", 1 / 16), ("cfg3", 1 / 32), ("cfg4", 1 / 32), ("cfg5", 1 / 32)])
+def test_scaled_configs_every_head_with_shuffled_pages(name, scale):
+    w = synth.workload(name, scale)
+    if name == "cfg3":
+        w.n_layers = 3
+    if name == "cfg4":
+        w.n_layers = 2
+    if name == "cfg5":
+        w.batch, w.ctx_len, w.window = 8, w.ctx_len[:8], w.window[:8]
+    w.decode_steps = min(w.decode_steps, 8)
+    run_parity(w, steps=w.decode_steps if w.decode_steps > 1 else 0, shuffle=12345, per_seq=(name == "cfg5"),
+               check_layout_every=3)
+
+
+# ------------------------------------------------------------------ property sweep over small shapes
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("D", [64, 128])
+@pytest.mark.parametrize("group", [1, 2, 4, 8])
+def test_small_shape_sweep(dtype, D, group):
+    rng = np.random.default_rng(D * 100 + group + (7 if dtype == "f32" else 0))
+    for trial in range(6):
+        B = int(rng.integers(1, 4))
+        Hkv = int(rng.integers(1, 4))
+        n_sink = int(rng.integers(0, 6))
+        ctx = [int(rng.integers(0 if trial == 0 else 1, 301)) for _ in range(B)]
+        win = [int(rng.integers(0, 80)) for _ in range(B)]
+        if trial == 1:
+            win = [max(ctx) + 5] * B                         # window covers everything: nothing dropped
+        if trial == 2:
+            win = [max(0, c - n_sink - 1) for c in ctx]      # exactly one dropped token where possible
+        w = synth.Workload(f"sweep{trial}", B, 2, Hkv * group, Hkv, D, dtype, ctx, win, n_sink,
+                           n_retrieval_kv=min(1, Hkv - 1) if trial % 2 else 0, decode_steps=5,
+                           seed=9000 + trial + D + group)
+        run_parity(w, steps=5 if trial != 3 else 0, shuffle=trial, check_layout_every=1)
+
+
+def test_append_many_tokens_crosses_pages_evicts_and_rebuilds_schedule():
+    w = synth.Workload("long_append", 2, 1, 4, 4, 128, "bf16", [700, 90], [64, 200], 4, 1, 300, 4242)
+    run_parity(w, steps=300, check_layout_every=37)
+
+
+def test_plain_truncation_mode_and_literal_scale():
+    w = synth.workload("cfg2", 1 / 32)
+    run_parity(w, steps=3, use_comp=0)                      # sinks + window only (no compensation term)
+    w1 = synth.workload("cfg1")
+    run_parity(w1, steps=2, sm_scale=1.0)                   # Eq. 5 as printed: no 1/sqrt(d)
+
+
+def test_invariants_on_gpu_window_covers_context_equals_full_attention():
+    """A window >= N reproduces full attention; compared here against the oracle's full attention."""
+    w = synth.Workload("fullwin", 1, 1, 2, 2, 128, "bf16", [333], [400], 4, 0, 1, 77)
+    cache = make_cache(w)
+    K, V = synth.make_dense_kv(w, 0, DEV)
+    cache.compress(0, K, V, w.ctx_len, w.retrieval(0), w.window)
+    q = synth.make_queries(w, 0, 0, DEV)
+    out = to_f64(cache.decode(0, q))
+    for h in range(2):
+        ref = orc.full_attention(to_f64(q[0, h]), to_f64(K[0, h]), to_f64(V[0, h]), 1 / math.sqrt(128))
+        assert np.abs(out[0, h] - ref).max() <= 3e-3
+    cache.close()
+
+
+# ------------------------------------------------------------------ error paths on a live cache
+def test_error_codes_on_a_live_cache():
+    w = synth.Workload("err", 2, 2, 2, 2, 64, "bf16", [100, 50], [20, 20], 4, 1, 2, 5)
+    cache = make_cache(w)
+    q = synth.make_queries(w, 0, 0, DEV)
+    out = torch.empty(q.shape, dtype=torch.float32, device=DEV)
+    k_new, v_new = synth.make_new_kv(w, 0, 0, DEV)
+    with pytest.raises(rz.RazorError) as e:
+        cache.decode(0, q)
+    assert e.value.status == -6                                   # not compressed
+    with pytest.raises(rz.RazorError) as e:
+        cache.append(0, k_new, v_new)
+    assert e.value.status == -6
+    K, V = synth.make_dense_kv(w, 0, DEV)
+    retr = w.retrieval(0)
+    cache.compress_seq(0, 0, K[0], V[0], 100, retr, 20)
+    with pytest.raises(rz.RazorError) as e:
+        cache.decode(0, q)
+    assert e.value.status == -6                                   # sequence 1 still missing
+    with pytest.raises(rz.RazorError) as e:
+        cache.compress_seq(0, 1, K[1], V[1], 50, 1 - retr, 20)    # retrieval set must match the layer's
+    assert e.value.status == -1
+    cache.compress_seq(0, 1, K[1], V[1], 50, retr, 20)
+    cache.decode(0, q, out)
+    cache.append(0, k_new, v_new)
+    cache.append(0, k_new, v_new)
+    with pytest.raises(rz.RazorError) as e:
+        cache.append(0, k_new, v_new)                             # max_new_tokens = 2
+    assert e.value.status == -5
+    with pytest.raises(rz.RazorError) as e:
+        rz.razor_compress(cache.handle, 0, K, V, K.stride(0), K.stride(1), K.stride(2), [101, 50], retr, 4, [20, 20])
+    assert e.value.status == -5                                   # beyond max_ctx_len
+    with pytest.raises(rz.RazorError) as e:
+        rz.razor_compress(cache.handle, 0, K, V, K.stride(0), K.stride(1), K.stride(2), w.ctx_len, retr, 3, w.window)
+    assert e.value.status == -1                                   # n_sink differs from the config
+    with pytest.raises(rz.RazorError) as e:
+        rz.razor_compress(cache.handle, 0, K.data_ptr() + 2, V, K.stride(0), K.stride(1), K.stride(2), w.ctx_len,
+                          retr, 4, w.window)
+    assert e.value.status == -8
+    with pytest.raises(rz.RazorError) as e:
+        rz.razor_compress(cache.handle, 5, K, V, K.stride(0), K.stride(1), K.stride(2), w.ctx_len, retr, 4, w.window)
+    assert e.value.status == -1
+    # the pool holds every layer once; asking for a bigger plan than the pool has left fails cleanly
+    cache.compress(1, K, V, w.ctx_len, w.retrieval(1), w.window)
+    big = synth.Workload("err2", 2, 2, 2, 2, 64, "bf16", [100, 100], [90, 90], 4, 2, 2, 5)
+    with pytest.raises(rz.RazorError) as e:
+        cache.compress(1, K, V, [100, 100], np.ones(2, dtype=np.uint8), [90, 90])
+    assert e.value.status == -4
+    # the context is still healthy
+    cache.decode(0, q, out)
+    torch.cuda.synchronize()
+    assert torch.isfinite(out).all()
+    cache.close()
+
+
+def test_recompress_reuses_pages_and_reset_frees_them():
+    w = synth.workload("cfg2", 1 / 32)
+    w.decode_steps = 2
+    cache = make_cache(w)
+    K, V = synth.make_dense_kv(w, 0, DEV)
+    q = synth.make_queries(w, 0, 0, DEV)
+    outs = []
+    for _ in range(3):                                            # same plan: fits in the same pages
+        cache.compress(0, K, V, w.ctx_len, w.retrieval(0), w.window)
+        outs.append(cache.decode(0, q).clone())
+    assert (bits(outs[0]) == bits(outs[1])).all() and (bits(outs[1]) == bits(outs[2])).all()
+    rz.razor_cache_reset(cache.handle)
+    with pytest.raises(rz.RazorError):
+        cache.decode(0, q)
+    cache.compress(0, K, V, w.ctx_len, w.retrieval(0), w.window)
+    assert (bits(cache.decode(0, q)) == bits(outs[0])).all()
+    cache.close()
+
+
+def test_strided_dense_input_and_schedule_query():
+    """K/V taken as views of a larger buffer (row stride > D, padded context)."""
+    w = synth.Workload("strided", 2, 1, 4, 4, 128, "bf16", [500, 260], [100, 100], 4, 1, 1, 31)
+    Kc, Vc = synth.make_dense_kv(w, 0, DEV)
+    big_k = torch.zeros((2, 4, 520, 256), dtype=torch.bfloat16, device=DEV)
+    big_v = torch.zeros_like(big_k)
+    big_k[:, :, :500, 64:192] = Kc
+    big_v[:, :, :500, 64:192] = Vc
+    Kv, Vv = big_k[:, :, :, 64:192], big_v[:, :, :, 64:192]
+    cache = make_cache(w)
+    cache.compress(0, Kv, Vv, w.ctx_len, w.retrieval(0), w.window)
+    q = synth.make_queries(w, 0, 0, DEV)
+    a = cache.decode(0, q).clone()
+    items = rz.razor_schedule_query(cache.handle, 0)
+    assert set(items[:, 0].tolist()) == set(range(8))
+    cache.compress(0, Kc, Vc, w.ctx_len, w.retrieval(0), w.window)
+    b = cache.decode(0, q)
+    assert (bits(a) == bits(b)).all()
+    cache.close()
