@@ -1,0 +1,468 @@
+#!/usr/bin/env python
+"""Benchmark of the RazorAttention hot path on B200: compress -> (append, decode attention) x steps.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg3] [--impl reference]
+
+One "step" is one pass of the whole hot path over one synthetic batch of the workload:
+prefill-end compression of every layer (from a dense layer buffer resident in HBM), then the
+workload's decode steps, each a razor_append + razor_decode_attention on every layer.
+
+metric/value: compressed-cache decode attention GB/s = compressed K+V bytes the pass's decode calls
+attend over, divided by the time of the WHOLE pass (compression and appends included).
+`decode` in the JSON line isolates the decode-attention kernel; `roofline` is that kernel against
+the measured HBM copy bandwidth.  Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "compressed_cache_decode_attention_GBps"
+UNIT = "GB/s"
+NOMINAL_HBM_GBS = 8000.0        # the "~8 TB/s" the target is quoted against
+FALLBACK_HBM_GBS = 6650.0       # used only when MEASURED_PEAKS.json is absent
+# DRAM traffic of the decode kernel per algorithmic byte, from the ncu capture summarised in
+# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over the algorithmic bytes of the launch).
+DECODE_TRAFFIC_PER_ALG_BYTE = None
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="razor", choices=["razor", "reference"])
+    ap.add_argument("--workload", default="cfg3", choices=["cfg2", "cfg3", "cfg4", "cfg5"])
+    ap.add_argument("--layers", type=int, default=0, help="use only the first LAYERS layers (profiling; not a valid bench number)")
+    ap.add_argument("--decode-steps", type=int, default=0, help="override the workload's decode steps (profiling)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-dense", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.idx, self.proc, self.lines = gpu_index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.idx)], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, mx, pw, reasons = [], [], [], set()
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2])); pw.append(float(f[3]))
+            except ValueError:
+                continue
+            for name, val in zip(["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"], f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "power_w_max": max(pw), "samples": len(sm),
+                "reasons": sorted(reasons)}
+
+
+# ---------------------------------------------------------------------------------------------- oracle leg
+def oracle_sample(w, budget_s=12.0):
+    """Times the CPU oracle, as it stands, on a bounded sample of the workload: layer 0, sequence 0,
+    KV heads taken in order until the budget is spent (at least one retrieval and one other head);
+    per head one compression and the workload's decode steps (one query each, no appends: the oracle
+    would recompress the whole history at every append).
+    Returns (GB/s = compressed K+V bytes attended / (compress + decode time), description, threads, raw)."""
+    import numpy as np
+    from oracle import razor_oracle as orc
+    from paper_2407_15891_b200 import synth
+    try:
+        from threadpoolctl import threadpool_info
+        threads = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+    except Exception:
+        threads = 1
+    retr = w.retrieval(0)
+    order = [g for g in range(w.n_kv_heads) if retr[g]][:1] + [g for g in range(w.n_kv_heads) if not retr[g]][:1]
+    order += [g for g in range(w.n_kv_heads) if g not in order]
+    b = 0
+    n, win, T = w.ctx_len[b], w.window[b], w.decode_steps
+    qs = [synth.make_queries(w, 0, t).double().numpy() for t in range(T)]
+    scale = 1.0 / math.sqrt(w.head_dim)
+    t_comp = t_dec = 0.0
+    bytes_attended = 0
+    heads = n_retr = 0
+    t_start = time.perf_counter()
+    for g in order:
+        K, V = synth.make_dense_head(w, 0, b, g)
+        K, V = K.double().numpy()[:n], V.double().numpy()[:n]
+        t0 = time.perf_counter()
+        hc = orc.compress_head(K, V, n, w.n_sink, win, bool(retr[g]))
+        t1 = time.perf_counter()
+        for t in range(T):
+            for j in range(w.group):
+                orc.decode_head(qs[t][b, g * w.group + j], hc, scale)
+        t2 = time.perf_counter()
+        t_comp += t1 - t0
+        t_dec += t2 - t1
+        bytes_attended += T * len(hc.kept_pos) * 2 * w.head_dim * w.esz()
+        heads += 1
+        n_retr += int(retr[g])
+        if time.perf_counter() - t_start > budget_s and heads >= 2:
+            break
+    desc = (f"layer 0, sequence 0, {heads} of {w.n_kv_heads} KV heads ({n_retr} retrieval): one compression + {T} "
+            f"decode steps each (no appends); compress {t_comp:.3f}s, decode {t_dec:.3f}s "
+            f"(decode alone: {bytes_attended / t_dec / 1e9:.2f} GB/s); inputs generated per head outside the timing")
+    return bytes_attended / (t_comp + t_dec) / 1e9, desc, threads, dict(decode_s=t_dec, compress_s=t_comp, heads=heads)
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle timed on the host cores, same metric / unit / config."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2407_15891_b200 import synth
+    w = synth.workload(args.workload)
+    vals, times = [], []
+    desc, threads = "", 1
+    budget = max(2.0, min(12.0, 90.0 / max(1, args.steps + args.warmup)))
+    for i in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        v, desc, threads, _ = oracle_sample(w, budget_s=budget)
+        if i >= args.warmup:
+            vals.append(v)
+            times.append(time.perf_counter() - t0)
+    value = statistics.mean(vals)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * statistics.mean(times), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(w, args),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def workload_config(w, args):
+    return {"workload": f"{w.name}: batch {w.batch}, {w.n_layers} layers, {w.n_q_heads}/{w.n_kv_heads} heads, "
+                        f"head_dim {w.head_dim}, context {min(w.ctx_len)}..{max(w.ctx_len)}, {w.dtype} K/V, "
+                        f"{w.n_retrieval_kv} retrieval KV heads per layer, n_sink {w.n_sink}, window "
+                        f"{min(w.window)}..{max(w.window)}, {w.decode_steps} decode steps per pass",
+            "step": "compress all layers + decode_steps x layers x (append + decode attention)",
+            "l2": "inputs larger than L2 (every launch streams > 126 MB of distinct cache pages)",
+            "dense_input": "one seeded dense layer buffer resident in HBM, reused for every layer"}
+
+
+# ---------------------------------------------------------------------------------------------- GPU legs
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import numpy as np
+    import torch
+    from paper_2407_15891_b200 import binding as rz
+    from paper_2407_15891_b200 import build as rz_build
+    from paper_2407_15891_b200 import synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        rz_build.build()
+    if dist is not None:
+        dist.barrier()
+    rz.load()
+
+    w = synth.workload(args.workload)
+    if args.layers:
+        w.n_layers = min(w.n_layers, args.layers)
+    if args.decode_steps:
+        w.decode_steps = args.decode_steps
+    L, T = w.n_layers, w.decode_steps
+    tdt = synth.torch_dtype(w)
+    per_seq = w.name == "cfg5"
+
+    retr = [w.retrieval(l) for l in range(L)]
+    cfg = rz.make_config(w.batch, L, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, w.n_sink, max(w.ctx_len), T)
+    cache = rz.RazorCache(cfg, w.ctx_len, w.window, np.stack(retr), device=dev)
+
+    # inputs, resident in HBM before the timed region
+    if per_seq:
+        dense = []
+        for b in range(w.batch):
+            wb = synth.Workload(w.name, 1, 1, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, [w.ctx_len[b]],
+                                [w.window[b]], w.n_sink, w.n_retrieval_kv, T, w.seed * 131 + b)
+            K, V = synth.make_dense_kv(wb, 0, dev)
+            dense.append((K[0], V[0]))
+    else:
+        w0 = synth.Workload(w.name, w.batch, 1, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, w.ctx_len, w.window,
+                            w.n_sink, w.n_retrieval_kv, T, w.seed)
+        Kd, Vd = synth.make_dense_kv(w0, 0, dev)
+    n_q = 4   # distinct per-step inputs, cycled
+    qs = [synth.make_queries(w, 0, i, dev) for i in range(n_q)]
+    kvs = [synth.make_new_kv(w, 0, i, dev) for i in range(n_q)]
+    out = torch.empty((w.batch, w.n_q_heads, w.head_dim), dtype=torch.float32, device=dev)
+    torch.cuda.synchronize()
+
+    launches = {"n": 0}
+
+    def compress_all():
+        for l in range(L):
+            if per_seq:
+                for b in range(w.batch):
+                    cache.compress_seq(l, b, dense[b][0], dense[b][1], w.ctx_len[b], retr[l], w.window[b])
+                    launches["n"] += 2
+            else:
+                cache.compress(l, Kd, Vd, w.ctx_len, retr[l], w.window)
+                launches["n"] += 2
+
+    def one_pass(ev=None):
+        compress_all()
+        if ev is not None:
+            ev["compress_end"].record()
+        for t in range(T):
+            k_new, v_new = kvs[t % n_q]
+            q = qs[t % n_q]
+            for l in range(L):
+                cache.append(l, k_new, v_new)
+                sample = ev is not None and ((l + t) % ev["every"] == 0)
+                if sample:
+                    e0 = torch.cuda.Event(enable_timing=True); e0.record()
+                cache.decode(l, q, out)
+                if sample:
+                    e1 = torch.cuda.Event(enable_timing=True); e1.record()
+                    ev["decode"].append((e0, e1, l, t))
+                launches["n"] += 2
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    # algorithmic bytes of the pass
+    def decode_alg_bytes(l, t):
+        kv = w.compressed_bytes(l, extra=t + 1)
+        n_nonretr = int((1 - retr[l]).sum()) * w.batch
+        small = w.batch * w.n_q_heads * w.head_dim * (w.esz() + 4) + n_nonretr * 2 * w.head_dim * 4
+        return kv, kv + small
+    attended = sum(decode_alg_bytes(l, t)[0] for l in range(L) for t in range(T))
+    compress_read = w.dense_bytes() * L
+    compress_write = sum(w.compressed_bytes(l) for l in range(L))
+
+    for _ in range(args.warmup):
+        one_pass()
+    sync_all()
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    ev = {"decode": [], "every": 4 if L * T >= 16 else 1,
+          "compress_end": torch.cuda.Event(enable_timing=True)}
+    starts, ends, comp_ends = [], [], []
+    launches["n"] = 0
+    sync_all()
+    for _ in range(args.steps):
+        s = torch.cuda.Event(enable_timing=True); e = torch.cuda.Event(enable_timing=True)
+        ev["compress_end"] = torch.cuda.Event(enable_timing=True)
+        s.record()
+        one_pass(ev)
+        e.record()
+        starts.append(s); ends.append(e); comp_ends.append(ev["compress_end"])
+    sync_all()
+    clocks = sampler.stop()
+    n_launches = launches["n"]
+
+    total_ms = starts[0].elapsed_time(ends[-1])
+    if dist is not None:
+        tt = torch.tensor([total_ms], device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms = float(tt.item())
+    ms_per_step = total_ms / args.steps
+    value = world * attended / (ms_per_step * 1e-3) / 1e9
+
+    comp_ms = statistics.mean(s.elapsed_time(c) for s, c in zip(starts, comp_ends))
+    dec_phase_ms = statistics.mean(c.elapsed_time(e) for c, e in zip(comp_ends, ends))
+    dec_us = [a.elapsed_time(b) * 1e3 for a, b, _, _ in ev["decode"]]
+    dec_alg = [decode_alg_bytes(l, t)[1] for _, _, l, t in ev["decode"]]
+    dec_gbs = sum(dec_alg) / (sum(dec_us) * 1e-6) / 1e9
+    peak, peak_kind = measured_peak()
+    alg_per_launch = statistics.mean(dec_alg)
+    roofline = {"bound": "hbm", "kernel": "decode_kernel", "achieved": dec_gbs, "peak": peak, "unit": "GB/s",
+                "frac": dec_gbs / peak, "peak_kind": f"of {peak_kind} (sustained copy bandwidth)",
+                "frac_of_nominal_8TBs": dec_gbs / NOMINAL_HBM_GBS,
+                "alg_bytes_per_launch": alg_per_launch, "us_per_launch": statistics.mean(dec_us),
+                "launches_timed": len(dec_us),
+                "traffic": (DECODE_TRAFFIC_PER_ALG_BYTE * alg_per_launch) if DECODE_TRAFFIC_PER_ALG_BYTE else None}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": w.dtype if w.dtype != "bf16" else "bf16", "data": "synthetic", "config": workload_config(w, args),
+        "clocks": clocks, "gpu_launches": n_launches, "roofline": roofline,
+        "decode": {"gbs_kernel": dec_gbs, "us_per_layer": statistics.mean(dec_us),
+                   "us_per_decode_step": dec_phase_ms * 1e3 / T,
+                   "gbs_phase_incl_append": attended / (dec_phase_ms * 1e-3) / 1e9,
+                   "compressed_gb_per_decode_step": attended / T / 1e9},
+        "compress": {"ms_per_pass": comp_ms, "gbs": (compress_read + compress_write) / (comp_ms * 1e-3) / 1e9,
+                     "read_gb": compress_read / 1e9, "write_gb": compress_write / 1e9},
+    }
+
+    # ------------------------------------------------------------------ dense full-cache decode, same GPU
+    if not args.no_dense and rank == 0 and not per_seq:
+        try:
+            cfg_d = rz.make_config(w.batch, 1, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, w.n_sink,
+                                   max(w.ctx_len), 1)
+            all_r = np.ones(w.n_kv_heads, dtype=np.uint8)
+            dcache = rz.RazorCache(cfg_d, w.ctx_len, w.window, all_r, device=dev)
+            dcache.compress(0, Kd, Vd, w.ctx_len, all_r, w.window)
+            for _ in range(3):
+                dcache.decode(0, qs[0], out)
+            torch.cuda.synchronize()
+            reps = 5
+            a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+            a.record()
+            for i in range(reps):
+                dcache.decode(0, qs[i % n_q], out)
+            b.record()
+            torch.cuda.synchronize()
+            d_us = a.elapsed_time(b) * 1e3 / reps
+            line["dense_decode"] = {"us_per_layer": d_us, "gbs": w.dense_bytes() / (d_us * 1e-6) / 1e9,
+                                    "us_per_decode_step": d_us * L,
+                                    "speedup_compressed_vs_dense": d_us / statistics.mean(dec_us)}
+            dcache.close()
+            del dcache
+        except Exception as ex:   # e.g. not enough memory for a dense layer beside the compressed stack
+            line["dense_decode"] = {"unavailable": str(ex)[:200]}
+
+    # ------------------------------------------------------------------ end to end with HOST buffers
+    if not args.no_e2e:
+        e2e_steps = max(1, min(args.steps, 2))
+        if per_seq:
+            host_dense = None
+        else:
+            host_dense = (torch.empty(Kd.shape, dtype=tdt, pin_memory=True), torch.empty(Vd.shape, dtype=tdt, pin_memory=True))
+            host_dense[0].copy_(Kd); host_dense[1].copy_(Vd)
+        h_q = [x.cpu().pin_memory() for x in qs]
+        h_kv = [(a.cpu().pin_memory(), b.cpu().pin_memory()) for a, b in kvs]
+        h_out = torch.empty(out.shape, dtype=torch.float32, pin_memory=True)
+        d_q = torch.empty_like(qs[0]); d_k = torch.empty_like(kvs[0][0]); d_v = torch.empty_like(kvs[0][1])
+        h2d = d2h = 0
+
+        def e2e_pass(count=False):
+            nonlocal h2d, d2h
+            for l in range(L):
+                if per_seq:
+                    for b in range(w.batch):
+                        cache.compress_seq(l, b, dense[b][0], dense[b][1], w.ctx_len[b], retr[l], w.window[b])
+                else:
+                    Kd.copy_(host_dense[0], non_blocking=True)
+                    Vd.copy_(host_dense[1], non_blocking=True)
+                    if count:
+                        h2d += 2 * Kd.numel() * Kd.element_size()
+                    cache.compress(l, Kd, Vd, w.ctx_len, retr[l], w.window)
+            for t in range(T):
+                for l in range(L):
+                    d_q.copy_(h_q[t % n_q], non_blocking=True)
+                    d_k.copy_(h_kv[t % n_q][0], non_blocking=True)
+                    d_v.copy_(h_kv[t % n_q][1], non_blocking=True)
+                    cache.append(l, d_k, d_v)
+                    cache.decode(l, d_q, out)
+                    h_out.copy_(out, non_blocking=True)
+                    if count:
+                        h2d += (d_q.numel() + 2 * d_k.numel()) * d_q.element_size()
+                        d2h += out.numel() * 4
+            torch.cuda.current_stream().synchronize()
+
+        e2e_pass()
+        sync_all()
+        t0 = time.perf_counter()
+        a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+        a.record()
+        for i in range(e2e_steps):
+            e2e_pass(count=(i == 0))
+        b.record()
+        sync_all()
+        e_ms = a.elapsed_time(b) / e2e_steps
+        if dist is not None:
+            tt = torch.tensor([e_ms], device=dev)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            e_ms = float(tt.item())
+        line["e2e"] = {"value": world * attended / (e_ms * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                       "d2h_bytes_per_step": d2h, "ms_per_step": e_ms, "steps": e2e_steps,
+                       "note": "host-pinned dense K/V, q, k_new, v_new copied in and out[] copied back inside the "
+                               "timed region" + ("; cfg5 dense K/V stay on the device (75 GB of host staging "
+                                                 "does not fit the time budget)" if per_seq else "")}
+        del host_dense
+
+    # ------------------------------------------------------------------ CPU oracle on the host cores
+    if not args.no_cpu_baseline and rank == 0:
+        v, desc, threads, _ = oracle_sample(synth.workload(args.workload))
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc}
+
+    cache.close()
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
