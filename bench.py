@@ -46,6 +46,7 @@ def parse_args():
     ap.add_argument("--workload", default="cfg3", choices=["cfg2", "cfg3", "cfg4", "cfg5"])
     ap.add_argument("--layers", type=int, default=0, help="use only the first LAYERS layers (profiling; not a valid bench number)")
     ap.add_argument("--decode-steps", type=int, default=0, help="override the workload's decode steps (profiling)")
+    ap.add_argument("--scale", type=float, default=1.0, help="shrink contexts and windows (profiling captures; not a valid bench number)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-dense", action="store_true")
@@ -191,6 +192,13 @@ def run_reference(args):
 
 
 def workload_config(w, args):
+    cfg = _workload_config(w, args)
+    if args.layers or args.decode_steps or args.scale != 1.0:
+        cfg["reduced_for_profiling"] = True      # not the benchmark workload: numbers are not bench values
+    return cfg
+
+
+def _workload_config(w, args):
     return {"workload": f"{w.name}: batch {w.batch}, {w.n_layers} layers, {w.n_q_heads}/{w.n_kv_heads} heads, "
                         f"head_dim {w.head_dim}, context {min(w.ctx_len)}..{max(w.ctx_len)}, {w.dtype} K/V, "
                         f"{w.n_retrieval_kv} retrieval KV heads per layer, n_sink {w.n_sink}, window "
@@ -230,7 +238,7 @@ def main():
         dist.barrier()
     rz.load()
 
-    w = synth.workload(args.workload)
+    w = synth.workload(args.workload, args.scale)
     if args.layers:
         w.n_layers = min(w.n_layers, args.layers)
     if args.decode_steps:
