@@ -163,19 +163,43 @@ RAZOR_API int razor_cache_stats(const razor_cache_t* cache, int32_t layer, size_
 
 /*
  * The decode work schedule (host only; no device is touched).  Every (sequence, KV head) token
- * stream is cut into page ranges of near-equal size so that one launch is balanced over the SMs
- * whatever the mix of full-length and short heads; ranges are ordered longest first.
+ * stream is cut into page ranges of near-equal size (work items) so that one launch is balanced over
+ * the SMs whatever the mix of full-length and short heads.  A range is at most
+ * max(min_chunk_pages, ceil(total_pages / target_items)) pages; heads cut into the most parts come
+ * first, longer ranges before shorter ones.
  *   razor_schedule_plan   plans for given stream lengths: tokens host int32[n_heads] (tokens stored
- *                         per head), target_items = how many ranges to aim for (>= 1).
+ *                         per head), target_items >= 1, min_chunk_pages >= 1.
  *   razor_schedule_query  the plan the next razor_decode_attention of `layer` would use.
- * items: host int32[max_items][4] = {head index b*Hkv + kv_head, first_page, end_page,
- * parts_of_this_head}, may be NULL; n_items receives the count.  A page is 16 tokens.
+ * items: host int32[max_items][4] = {head index b*Hkv + kv_head, first_page, end_page (-1: to the
+ * end of the stream), parts_of_this_head}, may be NULL; n_items receives the count.  A page is 16 tokens.
  * Errors: NULL_PTR, INVALID_ARG (also when max_items is too small), NOT_COMPRESSED.
  */
-RAZOR_API int razor_schedule_plan(const int32_t* tokens, int32_t n_heads, int32_t target_items, int32_t* items,
-                        int32_t max_items, int32_t* n_items);
+RAZOR_API int razor_schedule_plan(const int32_t* tokens, int32_t n_heads, int32_t target_items,
+                        int32_t min_chunk_pages, int32_t* items, int32_t max_items, int32_t* n_items);
 RAZOR_API int razor_schedule_query(razor_cache_t* cache, int32_t layer, int32_t* items, int32_t max_items,
                          int32_t* n_items);
+
+/*
+ * Decode tuning knobs; the defaults suit long-context caches on a B200.  A change takes effect at the
+ * next razor_decode_attention.  Errors: NULL_PTR, INVALID_ARG (unknown option or value out of range).
+ */
+enum {
+  RAZOR_OPT_DECODE_ITEMS_PER_SM = 1,    /* work items aimed for per SM (1..1024; default 24)              */
+  RAZOR_OPT_DECODE_MIN_CHUNK_PAGES = 2, /* smallest work item in pages (default 8)                        */
+  RAZOR_OPT_DECODE_RING_KB = 3,         /* shared-memory page ring per CTA in KiB; 0 = as large as fits   */
+  RAZOR_OPT_DECODE_CONSUMER_WARPS = 4   /* 0 = default; 8, 12 or 16 (bf16, group <= 2 only)               */
+};
+RAZOR_API int razor_cache_set_option(razor_cache_t* cache, int32_t option, int32_t value);
+
+/*
+ * Device-side health of the cache's kernels.  Every wait inside the decode kernel is bounded; a wait
+ * that runs out makes the kernel stop early and set a bit of a sticky status word instead of hanging.
+ * This call synchronises `stream`, stores the word in *status (0 = healthy) and, when it is non-zero,
+ * clears it together with the kernel's work counters so that the cache can be used again; outputs of
+ * the affected launch are undefined.  Bits: 1 producer wait, 2 consumer wait, 4 reducer wait, 8 copies
+ * still in flight at exit.  Errors: NULL_PTR, CUDA.
+ */
+RAZOR_API int razor_cache_device_status(razor_cache_t* cache, int32_t* status, void* stream);
 
 /* Forget every compressed layer and give all pages back (the handle and buffers stay usable). */
 RAZOR_API int razor_cache_reset(razor_cache_t* cache);

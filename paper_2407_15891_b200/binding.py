@@ -27,7 +27,7 @@ STATUS = {
 SYMBOLS = [
     "razor_query_bytes", "razor_cache_create", "razor_compress", "razor_compress_seq", "razor_append",
     "razor_decode_attention", "razor_cache_export", "razor_cache_stats", "razor_schedule_plan",
-    "razor_schedule_query", "razor_cache_reset", "razor_cache_destroy", "razor_status_string",
+    "razor_schedule_query", "razor_cache_set_option", "razor_cache_device_status", "razor_cache_reset", "razor_cache_destroy", "razor_status_string",
     "razor_last_cuda_error", "razor_version",
 ]
 
@@ -73,7 +73,9 @@ def load() -> C.CDLL:
     lib.razor_cache_export.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, C.POINTER(i32),
                                        C.POINTER(i32), vp]
     lib.razor_cache_stats.argtypes = [vp, i32, C.POINTER(sz), C.POINTER(sz)]
-    lib.razor_schedule_plan.argtypes = [vp, i32, i32, vp, i32, C.POINTER(i32)]
+    lib.razor_schedule_plan.argtypes = [vp, i32, i32, i32, vp, i32, C.POINTER(i32)]
+    lib.razor_cache_set_option.argtypes = [vp, i32, i32]
+    lib.razor_cache_device_status.argtypes = [vp, C.POINTER(i32), vp]
     lib.razor_schedule_query.argtypes = [vp, i32, vp, i32, C.POINTER(i32)]
     lib.razor_cache_reset.argtypes = [vp]
     lib.razor_cache_destroy.argtypes = [vp]
@@ -191,16 +193,31 @@ def razor_cache_stats(cache: int, layer: int) -> Tuple[int, int]:
     return k.value, d.value
 
 
-def razor_schedule_plan(tokens, target_items: int) -> np.ndarray:
+def razor_schedule_plan(tokens, target_items: int, min_chunk_pages: int = 1) -> np.ndarray:
     """Host-only: -> int32 [n_items, 4] = (head, first_page, end_page (-1: open), parts_of_head)."""
     t = _i32(tokens)
     n = C.c_int32(0)
     lib = load()
-    _check(lib.razor_schedule_plan(t.ctypes.data, len(t), target_items, None, 0, C.byref(n)), "razor_schedule_plan")
-    items = np.zeros((n.value, 4), dtype=np.int32)
-    _check(lib.razor_schedule_plan(t.ctypes.data, len(t), target_items, items.ctypes.data, n.value, C.byref(n)),
+    _check(lib.razor_schedule_plan(t.ctypes.data, len(t), target_items, min_chunk_pages, None, 0, C.byref(n)),
            "razor_schedule_plan")
+    items = np.zeros((n.value, 4), dtype=np.int32)
+    _check(lib.razor_schedule_plan(t.ctypes.data, len(t), target_items, min_chunk_pages, items.ctypes.data, n.value,
+                                   C.byref(n)), "razor_schedule_plan")
     return items
+
+
+OPT_DECODE_ITEMS_PER_SM, OPT_DECODE_MIN_CHUNK_PAGES, OPT_DECODE_RING_KB, OPT_DECODE_CONSUMER_WARPS = 1, 2, 3, 4
+
+
+def razor_cache_set_option(cache: int, option: int, value: int) -> None:
+    _check(load().razor_cache_set_option(cache, option, value), "razor_cache_set_option")
+
+
+def razor_cache_device_status(cache: int, stream=None) -> int:
+    """Synchronises the stream; -> the device status word (0 = healthy), cleared when non-zero."""
+    st = C.c_int32(0)
+    _check(load().razor_cache_device_status(cache, C.byref(st), _stream(stream)), "razor_cache_device_status")
+    return st.value
 
 
 def razor_schedule_query(cache: int, layer: int) -> np.ndarray:
@@ -273,6 +290,12 @@ class RazorCache:
         razor_cache_export(self.handle, layer, b, kv_head, kp, K, V, f[0], f[1], f[2], f[3])
         return dict(kept_pos=kp[:n_kept], K=K[:n_kept], V=V[:n_kept], mean_k=f[0], mean_v=f[1], sum_k=f[2],
                     sum_v=f[3], n_drop=n_drop)
+
+    def set_option(self, option: int, value: int) -> None:
+        razor_cache_set_option(self.handle, option, value)
+
+    def device_status(self) -> int:
+        return razor_cache_device_status(self.handle)
 
     def stats(self, layer: int):
         return razor_cache_stats(self.handle, layer)

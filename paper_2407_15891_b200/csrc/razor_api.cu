@@ -33,8 +33,8 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 inline int ceil_div(long long a, long long b) { return (int)((a + b - 1) / b); }
 
 struct Layout {
-  size_t state, comp_sum, comp_mean, page_table, items, partials, tickets, queue, scratch, seq_desc, total;
-  int max_pages, max_items;
+  size_t state, comp_sum, comp_mean, page_table, items, rec_ml, rec_o, tickets, queue, scratch, seq_desc, total;
+  int max_pages, max_items, max_recs, max_tickets;
 };
 
 int check_config(const razor_config_t* c) {
@@ -63,6 +63,9 @@ Layout make_layout(const razor_config_t& c) {
   const int g = c.n_q_heads / c.n_kv_heads;
   l.max_pages = std::max(1, ceil_div((long long)c.max_ctx_len + c.max_new_tokens, kPageTokens));
   l.max_items = (int)nh + kItemBudget;
+  // Level-0 records plus the inner nodes of the combine trees (fan-in kMergeFanIn), with slack per head.
+  l.max_recs = l.max_items + l.max_items / (kMergeFanIn - 1) + kMaxTreeLevels * (int)nh;
+  l.max_tickets = l.max_items / (kMergeFanIn - 1) + kMaxTreeLevels * (int)nh;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
   l.state = take(L * nh * sizeof(HeadState));
@@ -70,9 +73,10 @@ Layout make_layout(const razor_config_t& c) {
   l.comp_mean = take(L * nh * 2 * D * sizeof(float));
   l.page_table = take(L * nh * (size_t)l.max_pages * sizeof(int32_t));
   l.items = take(L * (size_t)l.max_items * sizeof(WorkItem));
-  l.partials = take((size_t)l.max_items * g * (kPartialPad + D) * sizeof(float));
-  l.tickets = take(nh * sizeof(int32_t));
-  l.queue = take(4 * sizeof(int32_t));
+  l.rec_ml = take((size_t)l.max_recs * g * sizeof(float2));
+  l.rec_o = take((size_t)l.max_recs * g * D * sizeof(float));
+  l.tickets = take((size_t)l.max_tickets * sizeof(int32_t));
+  l.queue = take(8 * sizeof(int32_t));   // queue[0..3], then the status word
   l.scratch = take(nh * kCompressMaxSlices * 2 * D * sizeof(float));
   l.seq_desc = take((size_t)c.batch * sizeof(SeqDesc));
   l.total = off;
@@ -115,6 +119,7 @@ struct razor_cache {
   DeviceView dv;
   long long pool_pages = 0, next_page = 0;
   int n_sms = 148;
+  DecodeTuning tune{24, 8, 0, 0};
   std::vector<LayerHost> layers;
   WorkItem* pinned_items = nullptr;   // [L][max_items]
 };
@@ -192,15 +197,19 @@ int razor_cache_create(razor_cache_t** out, const razor_config_t* cfg, void* poo
   dv.comp_mean = (float*)(ws + lay.comp_mean);
   dv.page_table = (int32_t*)(ws + lay.page_table);
   dv.items = (WorkItem*)(ws + lay.items);
-  dv.partials = (float*)(ws + lay.partials);
+  dv.rec_ml = (float2*)(ws + lay.rec_ml);
+  dv.rec_o = (float*)(ws + lay.rec_o);
   dv.tickets = (int32_t*)(ws + lay.tickets);
   dv.queue = (int32_t*)(ws + lay.queue);
+  dv.status = dv.queue + 4;
   dv.compress_scratch = (float*)(ws + lay.scratch);
   dv.seq_desc = (SeqDesc*)(ws + lay.seq_desc);
   dv.n_heads = cfg->batch * cfg->n_kv_heads;
   dv.n_kv_heads = cfg->n_kv_heads;
   dv.max_pages = lay.max_pages;
   dv.max_items = lay.max_items;
+  dv.max_recs = lay.max_recs;
+  dv.max_tickets = lay.max_tickets;
   dv.head_dim = cfg->head_dim;
   dv.n_sink = cfg->n_sink;
   dv.group = cfg->n_q_heads / cfg->n_kv_heads;
@@ -387,8 +396,8 @@ int ensure_schedule(razor_cache* c, int layer, cudaStream_t stream, bool upload)
   std::vector<int32_t> pages(nh);
   for (int h = 0; h < nh; ++h) pages[h] = ceil_div(L.hs[h].len, kPageTokens);
   if (L.upload_done) RZ_CUDA(cudaEventSynchronize(L.upload_done));   // previous upload has left the staging area
-  const int warps = c->n_sms * (c->dv.group == 1 ? 16 : 8);
-  const int n = build_schedule(pages.data(), nh, warps * 4, c->lay.max_items, L.items, &L.chunk_pages);
+  const int n = build_schedule(pages.data(), nh, c->n_sms * c->tune.items_per_sm, c->tune.min_chunk_pages,
+                               c->lay.max_items, c->lay.max_recs, c->lay.max_tickets, L.items, &L.chunk_pages);
   if (n < 0) return RAZOR_E_INVALID_ARG;
   L.n_items = n;
   L.growth_tokens = 0;
@@ -491,7 +500,7 @@ int razor_decode_attention(razor_cache_t* c, int32_t layer, const void* q, float
   if (((uintptr_t)q | (uintptr_t)out) & 15) return RAZOR_E_MISALIGNED;
   rc = ensure_schedule(c, layer, (cudaStream_t)stream, true);
   if (rc) return rc;
-  RZ_CUDA(launch_decode(c->dv, c->cfg.dtype, layer, c->layers[layer].n_items, q, out, c->n_sms,
+  RZ_CUDA(launch_decode(c->dv, c->cfg.dtype, layer, c->layers[layer].n_items, q, out, c->n_sms, c->tune,
                         (cudaStream_t)stream));
   return RAZOR_OK;
 }
@@ -532,10 +541,10 @@ int razor_cache_stats(const razor_cache_t* c, int32_t layer, size_t* kept_bytes,
   return RAZOR_OK;
 }
 
-int razor_schedule_plan(const int32_t* tokens, int32_t n_heads, int32_t target_items, int32_t* items,
-                        int32_t max_items, int32_t* n_items) {
+int razor_schedule_plan(const int32_t* tokens, int32_t n_heads, int32_t target_items, int32_t min_chunk_pages,
+                        int32_t* items, int32_t max_items, int32_t* n_items) {
   if (!tokens || !n_items) return RAZOR_E_NULL_PTR;
-  if (n_heads < 1 || target_items < 1) return RAZOR_E_INVALID_ARG;
+  if (n_heads < 1 || target_items < 1 || min_chunk_pages < 1) return RAZOR_E_INVALID_ARG;
   std::vector<int32_t> pages(n_heads);
   for (int h = 0; h < n_heads; ++h) {
     if (tokens[h] < 0) return RAZOR_E_INVALID_ARG;
@@ -544,9 +553,51 @@ int razor_schedule_plan(const int32_t* tokens, int32_t n_heads, int32_t target_i
   const int cap = n_heads + kItemBudget;
   std::vector<WorkItem> w(cap);
   int chunk = 0;
-  const int n = build_schedule(pages.data(), n_heads, target_items, cap, w.data(), &chunk);
+  const int n = build_schedule(pages.data(), n_heads, target_items, min_chunk_pages, cap, 2 * cap + kMaxTreeLevels * n_heads,
+                               cap + kMaxTreeLevels * n_heads, w.data(), &chunk);
   if (n < 0) return RAZOR_E_INVALID_ARG;
   return emit_items(w.data(), n, items, max_items, n_items);
+}
+
+int razor_cache_set_option(razor_cache_t* c, int32_t option, int32_t value) {
+  if (!c) return RAZOR_E_NULL_PTR;
+  switch (option) {
+    case RAZOR_OPT_DECODE_ITEMS_PER_SM:
+      if (value < 1 || value > 1024) return RAZOR_E_INVALID_ARG;
+      c->tune.items_per_sm = value;
+      break;
+    case RAZOR_OPT_DECODE_MIN_CHUNK_PAGES:
+      if (value < 1 || value > (1 << 20)) return RAZOR_E_INVALID_ARG;
+      c->tune.min_chunk_pages = value;
+      break;
+    case RAZOR_OPT_DECODE_RING_KB:
+      if (value < 0 || value > 227) return RAZOR_E_INVALID_ARG;
+      c->tune.ring_kb = value;
+      break;
+    case RAZOR_OPT_DECODE_CONSUMER_WARPS:
+      if (value != 0 && value != 8 && value != 12 && value != 16) return RAZOR_E_INVALID_ARG;
+      c->tune.consumer_warps = value;
+      break;
+    default:
+      return RAZOR_E_INVALID_ARG;
+  }
+  for (LayerHost& L : c->layers) L.sched_valid = false;   // the next decode re-plans
+  return RAZOR_OK;
+}
+
+int razor_cache_device_status(razor_cache_t* c, int32_t* status, void* stream) {
+  if (!c || !status) return RAZOR_E_NULL_PTR;
+  int32_t host = 0;
+  RZ_CUDA(cudaMemcpyAsync(&host, c->dv.status, sizeof(host), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+  RZ_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+  *status = host;
+  if (host != 0) {
+    // A kernel gave up part-way: its queue and ticket counters may be left non-zero.  Put them back.
+    RZ_CUDA(cudaMemsetAsync(c->dv.queue, 0, 8 * sizeof(int32_t), (cudaStream_t)stream));
+    RZ_CUDA(cudaMemsetAsync(c->dv.tickets, 0, (size_t)c->lay.max_tickets * sizeof(int32_t), (cudaStream_t)stream));
+    RZ_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+  }
+  return RAZOR_OK;
 }
 
 int razor_schedule_query(razor_cache_t* c, int32_t layer, int32_t* items, int32_t max_items, int32_t* n_items) {

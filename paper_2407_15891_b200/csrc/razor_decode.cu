@@ -1,22 +1,145 @@
-// Decode attention over the compressed cache (Eq. 5; Algorithm 1 line 5): split-K flash decoding.
+// Decode attention over the compressed cache (Eq. 5; Algorithm 1 line 5): split-K flash decoding as a
+// persistent producer / consumer kernel, one CTA per SM.
 //
-// One launch covers every (sequence, KV head) of a layer, full-length retrieval heads and short
-// heads alike.  The host cuts the token streams into page ranges of near-equal size (work items);
-// warps pull items from a queue.  A warp streams its pages once, keeps an online softmax state
-// (m, l, o) per query head of the group in registers, and either writes the output directly (head
-// not split) or writes a partial record and takes a ticket; the warp that draws the head's last
-// ticket merges the partials, so there is no second launch and no spin-wait anywhere.
+// One launch covers every (sequence, KV head) of a layer, full-length retrieval heads and short heads
+// alike.  The host cuts the token streams into page ranges of near-equal size (work items) that the
+// CTAs pull from a queue.  Inside a CTA
+//   * the PRODUCER warp pops items, publishes each item's descriptor, query rows and compensation
+//     token in a small shared-memory slot, and streams the item's pages (one contiguous K|V block
+//     each) into a shared-memory ring with bulk asynchronous copies that complete on mbarriers.  It
+//     runs ahead across item boundaries, so the ring never drains;
+//   * NC CONSUMER warps take the ring's pages round-robin; each keeps an online-softmax state
+//     (m, l, o) per query head of the group in registers and hands it over at the end of the item;
+//   * the REDUCER warp merges the NC states of an item into one partial record, and closes the nodes
+//     of the head's combine tree whose last input it delivered (ticket counters; no second launch).
 //
 // The compensation token of a non-retrieval head is folded into the online softmax as the initial
 // state of the head's first part: m = s_c + log2(N_d), l = 1, o = v_hat, which is the term
 // N_d * exp(s_c) * v_hat of Eq. 5 with the count moved onto the logit.
 //
 // Logits live in the log2 domain: q is pre-multiplied by sm_scale * log2(e) and exp is ex2.
+//
+// Every wait on an mbarrier is bounded in time.  A wait that runs out sets a CTA-wide abort flag and a
+// bit of the device status word; the other warps see the flag in their own waits and leave, and the
+// producer waits (again bounded) for its copies in flight before the CTA exits.
 #include <math_constants.h>
+
+#include <algorithm>
 
 #include "razor_common.cuh"
 
 namespace razor {
+
+namespace {
+
+constexpr int kItemSlots = 4;            // item descriptors in flight between producer and consumers
+constexpr int kMergeBufs = 2;            // consumer -> reducer hand-over buffers
+constexpr int kMaxStages = 64;           // ring stages (pages in flight per CTA)
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s: far beyond any healthy wait
+
+// ------------------------------------------------------------------------------------------ mbarrier
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait for the phase of `bar` with the given parity.  False: the CTA is aborting (this wait ran
+// out of time, or another warp's did).
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = global_ns();
+  for (;;) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (global_ns() - t0 > kWaitLimitNs) {
+      *abort_flag = 1;
+      return false;
+    }
+  }
+}
+// Bounded wait that ignores the abort flag (used on the abort path itself).
+__device__ __forceinline__ bool mbar_wait_drain(uint64_t* bar, uint32_t parity) {
+  const unsigned long long t0 = global_ns();
+  for (;;) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (global_ns() - t0 > kWaitLimitNs) return false;
+  }
+}
+// Bulk asynchronous copy global -> shared; completion is counted in bytes on `bar`.
+// dst, src 16-byte aligned, bytes a multiple of 16.
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   smem_u32(dst)),
+               "l"(src), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+
+// ------------------------------------------------------------------------------------------ shared layout
+struct ItemDesc {
+  int32_t head;        // < 0: no more items
+  int32_t page_begin;
+  int32_t n_pages;
+  int32_t len;         // tokens the head holds (masks the tail of its last page)
+  int32_t part_idx;
+  int32_t n_parts;
+  int32_t rec_base;
+  int32_t ticket_base;
+  int32_t seed;        // 1: this part starts from the compensation token
+  int32_t n_drop;
+  int32_t pad0, pad1;
+};
+
+template <typename T, int D, int G>
+struct alignas(16) ItemSlot {
+  ItemDesc desc;
+  alignas(16) T q[G][D];
+  alignas(16) float mean[2][D];   // k_hat, v_hat
+};
+
+struct Barriers {
+  uint64_t full[kMaxStages];
+  uint64_t empty[kMaxStages];
+  uint64_t item_full[kItemSlots];
+  uint64_t item_empty[kItemSlots];
+  uint64_t merge_full[kMergeBufs];
+  uint64_t merge_free[kMergeBufs];
+};
+
+// Hand-over buffer: the descriptor of the item, then per consumer warp and query head (m, l) and o[D].
+template <int D, int G, int NC>
+struct alignas(16) MergeBuf {
+  ItemDesc desc;
+  float2 ml[NC][G];
+  alignas(16) float o[NC][G][D];
+};
+
+// Dynamic shared memory: the hand-over buffers, then the page ring (1 KiB aligned).
+template <typename T, int D, int G, int NC>
+constexpr size_t decode_ring_offset() {
+  return (sizeof(MergeBuf<D, G, NC>) * kMergeBufs + 1023) & ~(size_t)1023;
+}
 
 template <int G, int EPL>
 struct SoftmaxState {
@@ -45,254 +168,535 @@ __device__ __forceinline__ void merge_state(float& m, float& l, float (&o)[EPL],
   m = mm;
 }
 
+// One page (16 tokens) from shared memory into the running state of a consumer warp.
+// kp points at this lane's first 16-byte fragment of the page (row group rg, fragment lir).
 template <typename T, int D, int G>
-__global__ void __launch_bounds__(128, (G == 1 ? 4 : 2))
-decode_kernel(DeviceView dv, int layer, int n_items, const T* __restrict__ q, float* __restrict__ out) {
+__device__ __forceinline__ void consume_page(const uint4* kp, int valid, int rg,
+                                             const float (&qf)[G][Elem<T>::kEpl], SoftmaxState<G, Elem<T>::kEpl>& S) {
   using Geo = RowGeom<T, D>;
   constexpr int LPR = Geo::kLpr, EPL = Geo::kEpl, RG = Geo::kRg, RPG = Geo::kRowsPerGroup;
-  constexpr int REC = kPartialPad + D;   // floats per partial record
-  const int lane = threadIdx.x & 31;
-  const int lir = lane % LPR, rg = lane / LPR;
-  const int n_q_heads = dv.n_kv_heads * G;
-  const WorkItem* items = dv.items + (size_t)layer * dv.max_items;
-  const int total_warps = gridDim.x * (blockDim.x >> 5);
+  uint4 kf[RPG], vf[RPG];
+#pragma unroll
+  for (int i = 0; i < RPG; ++i) kf[i] = kp[i * 32];
+#pragma unroll
+  for (int i = 0; i < RPG; ++i) vf[i] = kp[kPageTokens * LPR + i * 32];
 
-  for (;;) {
-    int it = 0;
-    if (lane == 0) it = atomicAdd(dv.queue, 1);
-    it = __shfl_sync(0xffffffffu, it, 0);
-    if (it >= n_items) break;
-
-    const WorkItem w = items[it];
-    const size_t hs = (size_t)layer * dv.n_heads + w.head;
-    const HeadState st = dv.state[hs];
-    const int n_pages = (st.len + kPageTokens - 1) / kPageTokens;
-    const int page_end = w.page_end < 0 ? n_pages : min(w.page_end, n_pages);
-    const int b = w.head / dv.n_kv_heads, g = w.head % dv.n_kv_heads;
-    const size_t q_row = (size_t)b * n_q_heads + (size_t)g * G;
-
-    float qf[G][EPL];
+  float s[G][RPG];
+#pragma unroll
+  for (int i = 0; i < RPG; ++i) {
+    float a[EPL];
+    Elem<T>::unpack(kf[i], a);
 #pragma unroll
     for (int j = 0; j < G; ++j) {
-      const uint4 u = ((const uint4*)(q + (q_row + j) * D))[lir];
-      Elem<T>::unpack(u, qf[j]);
+      float acc = 0.f;
 #pragma unroll
-      for (int e = 0; e < EPL; ++e) qf[j][e] *= dv.scale_log2;
+      for (int e = 0; e < EPL; ++e) acc += a[e] * qf[j][e];
+      s[j][i] = acc;
     }
-
-    SoftmaxState<G, EPL> S;
-    S.clear();
-
-    // Compensation token (Eq. 4, Eq. 5) seeds the first part of a head that dropped tokens.
-    if (w.part_idx == 0 && dv.use_comp && st.n_drop > 0 && st.window >= 0) {
-      const float* mean = dv.comp_mean + hs * 2 * D + lir * EPL;
-      float kh[EPL], vh[EPL];
+  }
 #pragma unroll
-      for (int e = 0; e < EPL; ++e) { kh[e] = mean[e]; vh[e] = mean[D + e]; }
-      const float log_cnt = log2f((float)st.n_drop);
+  for (int j = 0; j < G; ++j)
+#pragma unroll
+    for (int i = 0; i < RPG; ++i) s[j][i] = row_sum<LPR>(s[j][i]);
+
+  if (valid < kPageTokens) {   // rows of this page beyond the head's length
+#pragma unroll
+    for (int i = 0; i < RPG; ++i) {
+      if (i * RG + rg >= valid) {
+#pragma unroll
+        for (int j = 0; j < G; ++j) s[j][i] = -CUDART_INF_F;
+        vf[i] = make_uint4(0u, 0u, 0u, 0u);   // unused slots may hold anything, NaN patterns included
+      }
+    }
+  }
+
+#pragma unroll
+  for (int j = 0; j < G; ++j) {
+    float mx = s[j][0];
+#pragma unroll
+    for (int i = 1; i < RPG; ++i) mx = fmaxf(mx, s[j][i]);
+    const float m_new = fmaxf(S.m[j], mx);
+    const float m_use = (m_new == -CUDART_INF_F) ? 0.f : m_new;
+    const float corr = fast_exp2(S.m[j] - m_use);
+    float psum = 0.f;
+#pragma unroll
+    for (int i = 0; i < RPG; ++i) {
+      s[j][i] = fast_exp2(s[j][i] - m_use);
+      psum += s[j][i];
+    }
+    S.l[j] = S.l[j] * corr + psum;
+    S.m[j] = m_new;
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) S.o[j][e] *= corr;
+  }
+#pragma unroll
+  for (int i = 0; i < RPG; ++i) {
+    float v[EPL];
+    Elem<T>::unpack(vf[i], v);
+#pragma unroll
+    for (int j = 0; j < G; ++j)
+#pragma unroll
+      for (int e = 0; e < EPL; ++e) S.o[j][e] += s[j][i] * v[e];
+  }
+}
+
+// Reducer-side vector of D/32 consecutive floats per lane.
+template <int D>
+struct LaneVec;
+template <>
+struct LaneVec<128> {
+  float4 v;
+  __device__ __forceinline__ void zero() { v = make_float4(0.f, 0.f, 0.f, 0.f); }
+  __device__ __forceinline__ void fma(float c, const LaneVec& o) {
+    v.x += c * o.v.x; v.y += c * o.v.y; v.z += c * o.v.z; v.w += c * o.v.w;
+  }
+  __device__ __forceinline__ void scale(float c) { v.x *= c; v.y *= c; v.z *= c; v.w *= c; }
+  __device__ __forceinline__ void load_shared(const float* row, int lane) { v = *(const float4*)(row + lane * 4); }
+  __device__ __forceinline__ void load_l2(const float* row, int lane) { v = __ldcg((const float4*)(row + lane * 4)); }
+  __device__ __forceinline__ void store(float* row, int lane) const { *(float4*)(row + lane * 4) = v; }
+};
+template <>
+struct LaneVec<64> {
+  float2 v;
+  __device__ __forceinline__ void zero() { v = make_float2(0.f, 0.f); }
+  __device__ __forceinline__ void fma(float c, const LaneVec& o) { v.x += c * o.v.x; v.y += c * o.v.y; }
+  __device__ __forceinline__ void scale(float c) { v.x *= c; v.y *= c; }
+  __device__ __forceinline__ void load_shared(const float* row, int lane) { v = *(const float2*)(row + lane * 2); }
+  __device__ __forceinline__ void load_l2(const float* row, int lane) { v = __ldcg((const float2*)(row + lane * 2)); }
+  __device__ __forceinline__ void store(float* row, int lane) const { *(float2*)(row + lane * 2) = v; }
+};
+
+// ------------------------------------------------------------------------------------------ the kernel
+template <typename T, int D, int G, int NC>
+__global__ void __launch_bounds__((NC + 2) * 32, 1)
+decode_kernel(DeviceView dv, int layer, int n_items, const T* __restrict__ q, float* __restrict__ out, int n_stages) {
+  using Geo = RowGeom<T, D>;
+  constexpr int LPR = Geo::kLpr, EPL = Geo::kEpl;
+  constexpr uint32_t PB = Geo::kPageBytes;
+  constexpr int F = kMergeFanIn;
+  using Slot = ItemSlot<T, D, G>;
+  using MBuf = MergeBuf<D, G, NC>;
+
+  extern __shared__ __align__(1024) uint8_t dyn_smem[];
+  __shared__ Barriers bars;
+  __shared__ Slot slots[kItemSlots];
+  __shared__ int abort_flag_s;
+  volatile int* abort_flag = &abort_flag_s;
+
+  MBuf* mbufs = (MBuf*)dyn_smem;
+  uint8_t* ring = dyn_smem + decode_ring_offset<T, D, G, NC>();
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    abort_flag_s = 0;
+    for (int s = 0; s < n_stages; ++s) {
+      mbar_init(&bars.full[s], 1);
+      mbar_init(&bars.empty[s], 1);
+    }
+    for (int s = 0; s < kItemSlots; ++s) {
+      mbar_init(&bars.item_full[s], 1);
+      mbar_init(&bars.item_empty[s], NC);
+    }
+    for (int s = 0; s < kMergeBufs; ++s) {
+      mbar_init(&bars.merge_full[s], NC);
+      mbar_init(&bars.merge_free[s], 1);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  __syncthreads();
+
+  const WorkItem* items = dv.items + (size_t)layer * dv.max_items;
+  const int n_q_heads = dv.n_kv_heads * G;
+  // Warp-uniform bounded wait: false for every lane if any lane's wait failed.
+  auto warp_wait = [&](uint64_t* bar, uint32_t parity) -> bool {
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
+  };
+
+  if (warp == NC) {
+    // ======================================================================== producer
+    const unsigned ns = (unsigned)n_stages;
+    const int batch = n_stages < 32 ? n_stages : 32;   // pages issued per round: never more than the ring holds
+    unsigned c = 0;                                      // ring positions issued so far by this CTA (exact)
+    unsigned seq_issued = 0;                             // item slots whose copies were issued
+    int marker_slot = -1;                                // slot that received the end marker
+    bool ok = true;
+    for (unsigned seq = 0; ok; ++seq) {
+      const int slot = seq % kItemSlots;
+      int it = 0;
+      if (lane == 0) it = atomicAdd(dv.queue, 1);
+      it = __shfl_sync(0xffffffffu, it, 0);
+      if (seq >= kItemSlots) ok = warp_wait(&bars.item_empty[slot], ((seq / kItemSlots) - 1) & 1);
+      if (!ok) break;
+      Slot& sl = slots[slot];
+      if (it >= n_items) {
+        if (lane == 0) {
+          sl.desc.head = -1;
+          mbar_arrive(&bars.item_full[slot]);
+        }
+        marker_slot = slot;
+        break;
+      }
+      const WorkItem w = items[it];
+      const size_t hs = (size_t)layer * dv.n_heads + w.head;
+      const HeadState st = dv.state[hs];
+      const int head_pages = (st.len + kPageTokens - 1) / kPageTokens;
+      const int page_end = w.page_end < 0 ? head_pages : min(w.page_end, head_pages);
+      const int n = max(0, page_end - w.page_begin);
+      const bool seed = w.part_idx == 0 && dv.use_comp && st.n_drop > 0 && st.window >= 0;
+      if (lane == 0) {
+        ItemDesc d;
+        d.head = w.head; d.page_begin = w.page_begin; d.n_pages = n; d.len = st.len;
+        d.part_idx = w.part_idx; d.n_parts = w.n_parts; d.rec_base = w.rec_base; d.ticket_base = w.ticket_base;
+        d.seed = seed ? 1 : 0; d.n_drop = st.n_drop; d.pad0 = d.pad1 = 0;
+        sl.desc = d;
+        const int b = w.head / dv.n_kv_heads, g = w.head % dv.n_kv_heads;
+        const T* qsrc = q + ((size_t)b * n_q_heads + (size_t)g * G) * D;
+        constexpr uint32_t q_bytes = G * D * sizeof(T), mean_bytes = 2 * D * sizeof(float);
+        mbar_arrive_expect_tx(&bars.item_full[slot], q_bytes + (seed ? mean_bytes : 0u));
+        bulk_load(&sl.q[0][0], qsrc, q_bytes, &bars.item_full[slot]);
+        if (seed) bulk_load(&sl.mean[0][0], dv.comp_mean + hs * 2 * D, mean_bytes, &bars.item_full[slot]);
+      }
+      seq_issued = seq + 1;
+      const int32_t* pt = dv.page_table + hs * dv.max_pages + w.page_begin;
+      // Page i of an item always goes to consumer warp i % NC (so a part's result does not depend on
+      // which CTA streamed it or on what that CTA streamed before): the item starts on a ring position
+      // that is a multiple of NC, and the positions left over in its last round are passed on empty.
+      const int n_pad = (n + NC - 1) / NC * NC;
+      for (int p0 = 0; p0 < n_pad; p0 += batch) {
+        const int in_batch = min(batch, n_pad - p0);
+        const bool mine = lane < in_batch;
+        const bool real = mine && p0 + lane < n;
+        size_t pid = 0;
+        unsigned stage = 0;
+        bool ready = true;
+        if (mine) {
+          if (real) pid = (size_t)pt[p0 + lane];
+          const unsigned cc = c + lane;
+          stage = cc % ns;
+          const unsigned use = cc / ns;
+          if (use > 0) ready = mbar_wait(&bars.empty[stage], (use - 1) & 1, abort_flag);
+        }
+        ok = __all_sync(0xffffffffu, ready);   // all or nothing: `c` stays an exact count of issued positions
+        if (!ok) break;
+        if (real) {
+          mbar_arrive_expect_tx(&bars.full[stage], PB);
+          bulk_load(ring + (size_t)stage * PB, dv.pool + pid * dv.page_bytes, PB, &bars.full[stage]);
+        } else if (mine) {
+          mbar_arrive(&bars.full[stage]);
+        }
+        c += in_batch;
+      }
+    }
+    if (!ok && lane == 0) atomicOr(dv.status, kStatusProducerTimeout);
+    // Wait (bounded) until every copy this warp issued has landed: the CTA's shared memory must not be
+    // released under a copy in flight.  In a healthy run the consumers have waited for all of them already.
+    bool drained = true;
+    for (unsigned s = lane; s < ns && s < c; s += 32) {
+      const unsigned last = s + ns * ((c - 1 - s) / ns);   // latest ring position that used stage s
+      if (!mbar_wait_drain(&bars.full[s], (last / ns) & 1)) drained = false;
+    }
+    // (The slot that took the end marker was first waited free, so its earlier copies have landed; its
+    // barrier has since moved on a phase and must not be asked about the earlier one.)
+    if (lane < kItemSlots && (unsigned)lane < seq_issued && lane != marker_slot) {
+      const unsigned last = lane + kItemSlots * ((seq_issued - 1 - lane) / kItemSlots);
+      if (!mbar_wait_drain(&bars.item_full[lane], (last / kItemSlots) & 1)) drained = false;
+    }
+    if (!__all_sync(0xffffffffu, drained) && lane == 0) atomicOr(dv.status, kStatusDrainTimeout);
+    // Queue reset for the next launch: every CTA has made its last pop before it counts itself done.
+    if (lane == 0) {
+      const int done = atomicAdd(dv.queue + 1, 1);
+      if (done == (int)gridDim.x - 1) {
+        dv.queue[0] = 0;
+        dv.queue[1] = 0;
+      }
+    }
+  } else if (warp < NC) {
+    // ======================================================================== consumers
+    const unsigned ns = (unsigned)n_stages;
+    const int lir = lane % LPR, rg = lane / LPR;
+    unsigned c = 0;   // ring positions of all items so far (the same count in every consumer warp)
+    bool ok = true;
+    for (unsigned seq = 0;; ++seq) {
+      const int slot = seq % kItemSlots;
+      const int mb = seq % kMergeBufs;
+      MBuf& M = mbufs[mb];
+      if (!warp_wait(&bars.item_full[slot], (seq / kItemSlots) & 1)) { ok = false; break; }
+      const Slot& sl = slots[slot];
+      const ItemDesc d = sl.desc;
+      if (d.head < 0) {
+        // pass the end marker on to the reducer
+        if (seq >= kMergeBufs && !warp_wait(&bars.merge_free[mb], ((seq / kMergeBufs) - 1) & 1)) { ok = false; break; }
+        if (warp == 0 && lane == 0) M.desc.head = -1;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars.merge_full[mb]);
+        break;
+      }
+      float qf[G][EPL];
 #pragma unroll
       for (int j = 0; j < G; ++j) {
-        float s = 0.f;
+        const uint4 u = ((const uint4*)&sl.q[j][0])[lir];
+        Elem<T>::unpack(u, qf[j]);
 #pragma unroll
-        for (int e = 0; e < EPL; ++e) s += qf[j][e] * kh[e];
-        s = row_sum<LPR>(s);
-        if (rg == 0) {
-          S.m[j] = s + log_cnt;
-          S.l[j] = 1.f;
-#pragma unroll
-          for (int e = 0; e < EPL; ++e) S.o[j][e] = vh[e];
-        }
+        for (int e = 0; e < EPL; ++e) qf[j][e] *= dv.scale_log2;
       }
-    }
-
-    const int32_t* pt = dv.page_table + hs * dv.max_pages;
-    for (int p = w.page_begin; p < page_end; ++p) {
-      const uint4* kp = (const uint4*)(dv.pool + (size_t)pt[p] * dv.page_bytes) + rg * LPR + lir;
-      uint4 kf[RPG], vf[RPG];
+      SoftmaxState<G, EPL> S;
+      S.clear();
+      const bool first = warp == 0;   // the warp that takes the item's first page also takes its seed
+      // Compensation token (Eq. 4, Eq. 5) seeds the first part of a head that dropped tokens.
+      if (d.seed && first) {
+        float kh[EPL], vh[EPL];
 #pragma unroll
-      for (int i = 0; i < RPG; ++i) kf[i] = ld_stream(kp + i * 32);
-#pragma unroll
-      for (int i = 0; i < RPG; ++i) vf[i] = ld_stream(kp + kPageTokens * LPR + i * 32);
-
-      float s[G][RPG];
-#pragma unroll
-      for (int i = 0; i < RPG; ++i) {
-        float a[EPL];
-        Elem<T>::unpack(kf[i], a);
+        for (int e = 0; e < EPL; ++e) { kh[e] = sl.mean[0][lir * EPL + e]; vh[e] = sl.mean[1][lir * EPL + e]; }
+        const float log_cnt = log2f((float)d.n_drop);
 #pragma unroll
         for (int j = 0; j < G; ++j) {
-          float acc = 0.f;
+          float s = 0.f;
 #pragma unroll
-          for (int e = 0; e < EPL; ++e) acc += a[e] * qf[j][e];
-          s[j][i] = acc;
-        }
-      }
+          for (int e = 0; e < EPL; ++e) s += qf[j][e] * kh[e];
+          s = row_sum<LPR>(s);
+          if (rg == 0) {
+            S.m[j] = s + log_cnt;
+            S.l[j] = 1.f;
 #pragma unroll
-      for (int j = 0; j < G; ++j)
-#pragma unroll
-        for (int i = 0; i < RPG; ++i) s[j][i] = row_sum<LPR>(s[j][i]);
-
-      const int valid = st.len - p * kPageTokens;   // rows of this page that hold tokens
-      if (valid < kPageTokens) {
-#pragma unroll
-        for (int i = 0; i < RPG; ++i) {
-          if (i * RG + rg >= valid) {
-#pragma unroll
-            for (int j = 0; j < G; ++j) s[j][i] = -CUDART_INF_F;
-            vf[i] = make_uint4(0u, 0u, 0u, 0u);   // unused slots may hold anything, NaN patterns included
+            for (int e = 0; e < EPL; ++e) S.o[j][e] = vh[e];
           }
         }
       }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bars.item_empty[slot]);   // this warp holds all it needs from the slot
 
-#pragma unroll
-      for (int j = 0; j < G; ++j) {
-        float mx = s[j][0];
-#pragma unroll
-        for (int i = 1; i < RPG; ++i) mx = fmaxf(mx, s[j][i]);
-        const float m_new = fmaxf(S.m[j], mx);
-        const float m_use = (m_new == -CUDART_INF_F) ? 0.f : m_new;
-        const float corr = fast_exp2(S.m[j] - m_use);
-        float psum = 0.f;
-#pragma unroll
-        for (int i = 0; i < RPG; ++i) {
-          s[j][i] = fast_exp2(s[j][i] - m_use);
-          psum += s[j][i];
+      const int n_pad = (d.n_pages + NC - 1) / NC * NC;
+      for (int i = warp; i < n_pad; i += NC) {
+        const unsigned cc = c + i, stage = cc % ns, use = cc / ns;
+        if (!warp_wait(&bars.full[stage], use & 1)) { ok = false; break; }
+        if (i < d.n_pages) {
+          const uint4* kp = (const uint4*)(ring + (size_t)stage * PB) + rg * LPR + lir;
+          consume_page<T, D, G>(kp, d.len - (d.page_begin + i) * kPageTokens, rg, qf, S);
         }
-        S.l[j] = S.l[j] * corr + psum;
-        S.m[j] = m_new;
-#pragma unroll
-        for (int e = 0; e < EPL; ++e) S.o[j][e] *= corr;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars.empty[stage]);
       }
-#pragma unroll
-      for (int i = 0; i < RPG; ++i) {
-        float v[EPL];
-        Elem<T>::unpack(vf[i], v);
-#pragma unroll
-        for (int j = 0; j < G; ++j)
-#pragma unroll
-          for (int e = 0; e < EPL; ++e) S.o[j][e] += s[j][i] * v[e];
-      }
-    }
+      if (!ok) break;
+      c += n_pad;
 
-    // Row groups of the warp hold disjoint token subsets: merge them.
+      // Row groups of the warp hold disjoint token subsets: merge them.
 #pragma unroll
-    for (int off = LPR; off < 32; off <<= 1) {
+      for (int off = LPR; off < 32; off <<= 1) {
 #pragma unroll
-      for (int j = 0; j < G; ++j) {
-        const float m2 = __shfl_xor_sync(0xffffffffu, S.m[j], off);
-        const float l2 = __shfl_xor_sync(0xffffffffu, S.l[j], off);
-        float o2[EPL];
+        for (int j = 0; j < G; ++j) {
+          const float m2 = __shfl_xor_sync(0xffffffffu, S.m[j], off);
+          const float l2 = __shfl_xor_sync(0xffffffffu, S.l[j], off);
+          float o2[EPL];
 #pragma unroll
-        for (int e = 0; e < EPL; ++e) o2[e] = __shfl_xor_sync(0xffffffffu, S.o[j][e], off);
-        merge_state<EPL>(S.m[j], S.l[j], S.o[j], m2, l2, o2);
+          for (int e = 0; e < EPL; ++e) o2[e] = __shfl_xor_sync(0xffffffffu, S.o[j][e], off);
+          merge_state<EPL>(S.m[j], S.l[j], S.o[j], m2, l2, o2);
+        }
       }
-    }
-
-    if (w.n_parts == 1) {
+      // Hand the state over to the reducer.
+      if (seq >= kMergeBufs && !warp_wait(&bars.merge_free[mb], ((seq / kMergeBufs) - 1) & 1)) { ok = false; break; }
+      if (first && lane == 0) M.desc = d;
       if (rg == 0) {
 #pragma unroll
         for (int j = 0; j < G; ++j) {
-          const float inv = S.l[j] > 0.f ? 1.f / S.l[j] : 0.f;
-          float* dst = out + (q_row + j) * D + lir * EPL;
+          if (lir == 0) M.ml[warp][j] = make_float2(S.m[j], S.l[j]);
 #pragma unroll
           for (int e = 0; e < EPL; e += 4)
-            *(float4*)(dst + e) = make_float4(S.o[j][e] * inv, S.o[j][e + 1] * inv, S.o[j][e + 2] * inv,
-                                              S.o[j][e + 3] * inv);
+            *(float4*)&M.o[warp][j][lir * EPL + e] = make_float4(S.o[j][e], S.o[j][e + 1], S.o[j][e + 2], S.o[j][e + 3]);
         }
       }
-      continue;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bars.merge_full[mb]);
     }
-
-    float* rec0 = dv.partials + (size_t)w.part_base * G * REC;
-    if (rg == 0) {
+    if (!ok && lane == 0) atomicOr(dv.status, kStatusConsumerTimeout);
+  } else {
+    // ======================================================================== reducer
+    bool ok = true;
+    for (unsigned seq = 0;; ++seq) {
+      const int mb = seq % kMergeBufs;
+      if (!warp_wait(&bars.merge_full[mb], (seq / kMergeBufs) & 1)) { ok = false; break; }
+      const MBuf& M = mbufs[mb];
+      const ItemDesc d = M.desc;
+      if (d.head < 0) break;
+      // NC warp states -> one state per query head of the group
+      float m_tot[G], l_tot[G];
+      LaneVec<D> acc[G];
 #pragma unroll
       for (int j = 0; j < G; ++j) {
-        float* rec = rec0 + ((size_t)w.part_idx * G + j) * REC;
-        if (lir == 0) { rec[0] = S.m[j]; rec[1] = S.l[j]; }
+        float mx = -CUDART_INF_F;
 #pragma unroll
-        for (int e = 0; e < EPL; e += 4)
-          *(float4*)(rec + kPartialPad + lir * EPL + e) =
-              make_float4(S.o[j][e], S.o[j][e + 1], S.o[j][e + 2], S.o[j][e + 3]);
+        for (int w = 0; w < NC; ++w) mx = fmaxf(mx, M.ml[w][j].x);
+        const float mu = (mx == -CUDART_INF_F) ? 0.f : mx;
+        float l = 0.f;
+        acc[j].zero();
+#pragma unroll
+        for (int w = 0; w < NC; ++w) {
+          const float2 ml = M.ml[w][j];
+          const float cw = fast_exp2(ml.x - mu);
+          l += ml.y * cw;
+          LaneVec<D> o;
+          o.load_shared(&M.o[w][j][0], lane);
+          acc[j].fma(cw, o);
+        }
+        m_tot[j] = mx;
+        l_tot[j] = l;
       }
-    }
-    __threadfence();
-    __syncwarp();
-    int ticket = 0;
-    if (lane == 0) ticket = atomicAdd(&dv.tickets[w.head], 1);
-    ticket = __shfl_sync(0xffffffffu, ticket, 0);
-    if (ticket != w.n_parts - 1) continue;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bars.merge_free[mb]);
 
-    // Last part of this head to finish: merge all partial records (read through L2).
-    __threadfence();
-    if (lane == 0) dv.tickets[w.head] = 0;
-    if (rg == 0) {
+      const int b = d.head / dv.n_kv_heads, g = d.head % dv.n_kv_heads;
+      float* out_rows = out + ((size_t)b * n_q_heads + (size_t)g * G) * D;
+      if (d.n_parts == 1) {
+#pragma unroll
+        for (int j = 0; j < G; ++j) {
+          acc[j].scale(l_tot[j] > 0.f ? 1.f / l_tot[j] : 0.f);
+          acc[j].store(out_rows + (size_t)j * D, lane);
+        }
+        continue;
+      }
+      // This part's record, then up the head's combine tree for as long as this warp closes the nodes.
+      int idx = d.part_idx, n = d.n_parts, rec_off = d.rec_base, tk_off = d.ticket_base;
+#pragma unroll
+      for (int j = 0; j < G; ++j) {
+        const size_t r = (size_t)(rec_off + idx) * G + j;
+        if (lane == 0) dv.rec_ml[r] = make_float2(m_tot[j], l_tot[j]);
+        acc[j].store(dv.rec_o + r * D, lane);
+      }
+      for (;;) {
+        const int n_next = (n + F - 1) / F, node = idx / F;
+        const int fan = min(F, n - node * F);
+        __threadfence();
+        __syncwarp();
+        int ticket = 0;
+        if (lane == 0) ticket = atomicAdd(&dv.tickets[tk_off + node], 1);
+        ticket = __shfl_sync(0xffffffffu, ticket, 0);
+        if (ticket != fan - 1) break;
+        // Last input of this node: merge its `fan` records (read through L2).
+        __threadfence();
+        if (lane == 0) dv.tickets[tk_off + node] = 0;
+        const int first_rec = rec_off + node * F;
 #pragma unroll 1
-      for (int j = 0; j < G; ++j) {
-        float M = -CUDART_INF_F, L = 0.f, acc[EPL];
+        for (int j = 0; j < G; ++j) {
+          float2 ml = make_float2(-CUDART_INF_F, 0.f);
+          if (lane < fan) ml = __ldcg(&dv.rec_ml[(size_t)(first_rec + lane) * G + j]);
+          float mx = ml.x;
 #pragma unroll
-        for (int e = 0; e < EPL; ++e) acc[e] = 0.f;
-        for (int i = 0; i < w.n_parts; ++i) {
-          const float* rec = rec0 + ((size_t)i * G + j) * REC;
-          const float mi = ld_cg(rec), li = ld_cg(rec + 1);
-          float oi[EPL];
+          for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+          const float mu = (mx == -CUDART_INF_F) ? 0.f : mx;
+          const float cw = fast_exp2(ml.x - mu);
+          float l = ml.y * cw;
 #pragma unroll
-          for (int e = 0; e < EPL; e += 4) {
-            const float4 t = ld_cg4((const float4*)(rec + kPartialPad + lir * EPL + e));
-            oi[e] = t.x; oi[e + 1] = t.y; oi[e + 2] = t.z; oi[e + 3] = t.w;
+          for (int off = 16; off > 0; off >>= 1) l += __shfl_xor_sync(0xffffffffu, l, off);
+          LaneVec<D> sum;
+          sum.zero();
+#pragma unroll
+          for (int r = 0; r < F; ++r) {
+            const float cr = __shfl_sync(0xffffffffu, cw, r);
+            if (r < fan) {
+              LaneVec<D> o;
+              o.load_l2(dv.rec_o + ((size_t)(first_rec + r) * G + j) * D, lane);
+              sum.fma(cr, o);
+            }
           }
-          merge_state<EPL>(M, L, acc, mi, li, oi);
+          if (n_next == 1) {
+            sum.scale(l > 0.f ? 1.f / l : 0.f);
+            sum.store(out_rows + (size_t)j * D, lane);
+          } else {
+            const size_t r = (size_t)(rec_off + n + node) * G + j;
+            if (lane == 0) dv.rec_ml[r] = make_float2(mx, l);
+            sum.store(dv.rec_o + r * D, lane);
+          }
         }
-        const float inv = L > 0.f ? 1.f / L : 0.f;
-        float* dst = out + (q_row + j) * D + lir * EPL;
-#pragma unroll
-        for (int e = 0; e < EPL; e += 4)
-          *(float4*)(dst + e) = make_float4(acc[e] * inv, acc[e + 1] * inv, acc[e + 2] * inv, acc[e + 3] * inv);
+        if (n_next == 1) break;
+        rec_off += n;
+        tk_off += n_next;
+        idx = node;
+        n = n_next;
       }
     }
-  }
-
-  // Queue reset for the next launch: every warp has made its last pop before it counts itself done.
-  if (lane == 0) {
-    const int done = atomicAdd(dv.queue + 1, 1);
-    if (done == total_warps - 1) {
-      dv.queue[0] = 0;
-      dv.queue[1] = 0;
-    }
+    if (!ok && lane == 0) atomicOr(dv.status, kStatusReducerTimeout);
   }
 }
 
-template <typename T, int D, int G>
-static cudaError_t decode_t(const DeviceView& dv, int layer, int n_items, const void* q, float* out, int n_sms,
-                            cudaStream_t s) {
-  const int ctas_per_sm = (G == 1) ? 4 : 2;
-  int grid = n_sms * ctas_per_sm;
-  const int need = (n_items + 3) / 4;
-  if (grid > need) grid = need;
+// ------------------------------------------------------------------------------------------ launch
+constexpr int kSmemOptIn = 232448;   // 227 KiB: the most one CTA may hold on sm_100
+
+template <typename T, int D, int G, int NC>
+cudaError_t decode_launch(const DeviceView& dv, int layer, int n_items, const void* q, float* out, int n_sms,
+                          const DecodeTuning& tune, cudaStream_t s) {
+  auto kern = decode_kernel<T, D, G, NC>;
+  constexpr size_t PB = RowGeom<T, D>::kPageBytes;
+  constexpr size_t ring_off = decode_ring_offset<T, D, G, NC>();
+  static int static_smem = -1;        // per instantiation
+  static bool opted_in[64] = {};
+  cudaError_t e;
+  if (static_smem < 0) {
+    cudaFuncAttributes fa;
+    if ((e = cudaFuncGetAttributes(&fa, kern)) != cudaSuccess) return e;
+    static_smem = (int)fa.sharedSizeBytes;
+  }
+  const long long avail = (long long)kSmemOptIn - static_smem - (long long)ring_off;
+  long long stages = avail / (long long)PB;
+  if (tune.ring_kb > 0) stages = std::min<long long>(stages, (long long)tune.ring_kb * 1024 / (long long)PB);
+  stages = std::min<long long>(stages, kMaxStages);
+  // A stage must always be consumed by the same warp (stage % NC): a warp then never waits on a barrier
+  // that is more than one phase behind it, which a parity wait could not tell from "done".
+  stages = stages / NC * NC;
+  if (stages < NC) return cudaErrorInvalidConfiguration;
+  const size_t dyn = ring_off + (size_t)stages * PB;
+  int dev = 0;
+  if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64 || !opted_in[dev]) {
+    if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                  (int)(kSmemOptIn - static_smem))) != cudaSuccess)
+      return e;
+    if (dev >= 0 && dev < 64) opted_in[dev] = true;
+  }
+  int grid = std::min(n_sms, n_items);
   if (grid < 1) grid = 1;
-  decode_kernel<T, D, G><<<grid, 128, 0, s>>>(dv, layer, n_items, (const T*)q, out);
+  kern<<<grid, (NC + 2) * 32, dyn, s>>>(dv, layer, n_items, (const T*)q, out, (int)stages);
   return cudaGetLastError();
 }
 
+template <typename T, int D, int G>
+cudaError_t decode_nc(const DeviceView& dv, int layer, int n_items, const void* q, float* out, int n_sms,
+                      const DecodeTuning& tune, cudaStream_t s) {
+  // Consumer warps.  The ring holds a multiple of NC pages and (NC + 2) warps share the register file,
+  // so the choice trades pages in flight against registers per thread.
+  if constexpr (sizeof(T) == 2 && G <= 2) {
+    if (tune.consumer_warps == 8) return decode_launch<T, D, G, 8>(dv, layer, n_items, q, out, n_sms, tune, s);
+    if (tune.consumer_warps == 16) return decode_launch<T, D, G, 16>(dv, layer, n_items, q, out, n_sms, tune, s);
+    return decode_launch<T, D, G, 12>(dv, layer, n_items, q, out, n_sms, tune, s);
+  } else if constexpr (sizeof(T) == 2) {
+    return decode_launch<T, D, G, 8>(dv, layer, n_items, q, out, n_sms, tune, s);
+  } else {
+    return decode_launch<T, D, G, 4>(dv, layer, n_items, q, out, n_sms, tune, s);
+  }
+}
+
 template <typename T, int D>
-static cudaError_t decode_g(const DeviceView& dv, int layer, int n_items, const void* q, float* out, int n_sms,
-                            cudaStream_t s) {
+cudaError_t decode_g(const DeviceView& dv, int layer, int n_items, const void* q, float* out, int n_sms,
+                     const DecodeTuning& tune, cudaStream_t s) {
   switch (dv.group) {
-    case 1: return decode_t<T, D, 1>(dv, layer, n_items, q, out, n_sms, s);
-    case 2: return decode_t<T, D, 2>(dv, layer, n_items, q, out, n_sms, s);
-    case 4: return decode_t<T, D, 4>(dv, layer, n_items, q, out, n_sms, s);
-    case 8: return decode_t<T, D, 8>(dv, layer, n_items, q, out, n_sms, s);
+    case 1: return decode_nc<T, D, 1>(dv, layer, n_items, q, out, n_sms, tune, s);
+    case 2: return decode_nc<T, D, 2>(dv, layer, n_items, q, out, n_sms, tune, s);
+    case 4: return decode_nc<T, D, 4>(dv, layer, n_items, q, out, n_sms, tune, s);
+    case 8: return decode_nc<T, D, 8>(dv, layer, n_items, q, out, n_sms, tune, s);
   }
   return cudaErrorInvalidValue;
 }
 
+}  // namespace
+
 cudaError_t launch_decode(const DeviceView& dv, int dtype, int layer, int n_items, const void* q, float* out,
-                          int n_sms, cudaStream_t s) {
+                          int n_sms, const DecodeTuning& tune, cudaStream_t s) {
   if (dtype == RAZOR_BF16) {
-    return dv.head_dim == 128 ? decode_g<__nv_bfloat16, 128>(dv, layer, n_items, q, out, n_sms, s)
-                              : decode_g<__nv_bfloat16, 64>(dv, layer, n_items, q, out, n_sms, s);
+    return dv.head_dim == 128 ? decode_g<__nv_bfloat16, 128>(dv, layer, n_items, q, out, n_sms, tune, s)
+                              : decode_g<__nv_bfloat16, 64>(dv, layer, n_items, q, out, n_sms, tune, s);
   }
-  return dv.head_dim == 128 ? decode_g<float, 128>(dv, layer, n_items, q, out, n_sms, s)
-                            : decode_g<float, 64>(dv, layer, n_items, q, out, n_sms, s);
+  return dv.head_dim == 128 ? decode_g<float, 128>(dv, layer, n_items, q, out, n_sms, tune, s)
+                            : decode_g<float, 64>(dv, layer, n_items, q, out, n_sms, tune, s);
 }
 
 }  // namespace razor

@@ -14,8 +14,8 @@ namespace razor {
 constexpr int kPageTokens = 16;        // tokens per page
 constexpr int kMaxGroup = 8;           // query heads per KV head
 constexpr int kCompressMaxSlices = 64; // row slices per (sequence, KV head) in the compression kernel
-constexpr int kMinChunkPages = 4;      // smallest decode work item
-constexpr int kPartialPad = 4;         // floats before o[] in a partial record: m, l, 2 x pad
+constexpr int kMergeFanIn = 16;        // partial records merged per node of a head's combine tree
+constexpr int kMaxTreeLevels = 6;      // 16^6 parts per head: more than any page count the config allows
 
 // Device-resident state of one (layer, sequence, KV head).  window < 0 marks a head that keeps every
 // token (retrieval head).  Physical slots: [0, n_sink) sinks, then the recent window as a ring whose
@@ -27,16 +27,20 @@ struct HeadState {
   int32_t window;     // recent-window length; < 0: keeps everything
 };
 
-// One decode work item: pages [page_begin, page_end) of one head's token stream.  page_end < 0 means
-// "to the end of the stream as it is now" (the last part of a head grows with appends).
+// One decode work item: pages [page_begin, page_end) of one head's token stream, streamed by one CTA.
+// page_end < 0 means "to the end of the stream as it is now" (the last part of a head grows with
+// appends).  A head cut into n_parts items owns n_parts level-0 partial records starting at rec_base,
+// followed by the records of its combine tree (fan-in kMergeFanIn), and one ticket counter per tree
+// node starting at ticket_base.
 struct WorkItem {
   int32_t head;       // b * Hkv + kv_head
   int32_t page_begin;
   int32_t page_end;
   int32_t part_idx;   // index of this part within its head
   int32_t n_parts;    // parts of this head
-  int32_t part_base;  // first partial-record slot of this head
-  int32_t pad0, pad1;
+  int32_t rec_base;
+  int32_t ticket_base;
+  int32_t pad;
 };
 
 // One sequence handed to the compression kernel.
@@ -51,6 +55,14 @@ struct SeqDesc {
   int32_t pad;
 };
 
+// Bits of the device status word (razor_cache_device_status).
+enum : int32_t {
+  kStatusProducerTimeout = 1,   // the copy-issuing warp gave up waiting for a free ring stage or item slot
+  kStatusConsumerTimeout = 2,   // a streaming warp gave up waiting for a page or an item
+  kStatusReducerTimeout = 4,    // the merging warp gave up waiting for the streaming warps' states
+  kStatusDrainTimeout = 8       // copies were still in flight when the abort path stopped waiting for them
+};
+
 // Pointers into the caller's workspace, plus the dimensions the kernels need.
 struct DeviceView {
   uint8_t* pool;            // pages: [page][K rows | V rows][16][D]
@@ -59,15 +71,19 @@ struct DeviceView {
   float* comp_mean;         // [L][B*Hkv][2][D]
   int32_t* page_table;      // [L][B*Hkv][max_pages]
   WorkItem* items;          // [L][max_items]
-  float* partials;          // [max_items][G][kPartialPad + D]
-  int32_t* tickets;         // [B*Hkv]
-  int32_t* queue;           // [4]: next item, warps done, spare
+  float2* rec_ml;           // [max_recs][G]      running max (log2 domain) and denominator of a partial
+  float* rec_o;             // [max_recs][G][D]   un-normalised numerator of a partial
+  int32_t* tickets;         // [max_tickets]      arrival counters of the combine-tree nodes (zero at rest)
+  int32_t* queue;           // [4]: next item, CTAs done, spare, spare (zero at rest)
+  int32_t* status;          // [1]: kStatus* bits, sticky until razor_cache_device_status clears them
   float* compress_scratch;  // [B*Hkv][kCompressMaxSlices][2][D]
   SeqDesc* seq_desc;        // [B]
   int32_t n_heads;          // B*Hkv
   int32_t n_kv_heads;
   int32_t max_pages;        // page-table row length
   int32_t max_items;
+  int32_t max_recs;
+  int32_t max_tickets;
   int32_t head_dim;
   int32_t n_sink;
   int32_t group;
@@ -76,20 +92,33 @@ struct DeviceView {
   float scale_log2;         // sm_scale * log2(e)
 };
 
+// Decode launch tuning (razor_cache_set_option).
+struct DecodeTuning {
+  int32_t items_per_sm;     // work items aimed for per SM
+  int32_t min_chunk_pages;  // smallest work item
+  int32_t ring_kb;          // shared-memory page ring per CTA, KiB (0: as large as fits)
+  int32_t consumer_warps;   // 0: default for the group size
+};
+
 // Kernel launchers (defined in the .cu files).  Each returns the cudaError_t of the launch.
 cudaError_t launch_compress(const DeviceView& dv, int dtype, int layer, int n_seqs, int n_slices,
                             cudaStream_t stream);
 cudaError_t launch_append(const DeviceView& dv, int dtype, int layer, const void* k_new, const void* v_new,
                           cudaStream_t stream);
 cudaError_t launch_decode(const DeviceView& dv, int dtype, int layer, int n_items, const void* q, float* out,
-                          int n_sms, cudaStream_t stream);
+                          int n_sms, const DecodeTuning& tune, cudaStream_t stream);
 cudaError_t launch_export(const DeviceView& dv, int dtype, int layer, int head, int32_t* kept_pos, void* K, void* V,
                           float* mean_k, float* mean_v, float* sum_k, float* sum_v, cudaStream_t stream);
 
 // Host-only schedule builder (razor_schedule.cpp).  pages[h] = pages of head h's token stream now.
-// Returns the number of items written (<= max_items).
-int build_schedule(const int32_t* pages, int n_heads, int target_items, int max_items, WorkItem* out,
-                   int* chunk_pages_out);
+// Cuts every head into parts of at most chunk pages, chunk = max(min_chunk, total / target_items);
+// lays out each head's partial records and ticket counters.  Returns the number of items written
+// (<= max_items), or -1 when items, records or tickets would not fit.
+int build_schedule(const int32_t* pages, int n_heads, int target_items, int min_chunk, int max_items, int max_recs,
+                   int max_tickets, WorkItem* out, int* chunk_pages_out);
+
+// Records and tickets a head cut into n_parts items needs (n_parts >= 1).
+void tree_sizes(int n_parts, int* n_recs, int* n_tickets);
 
 }  // namespace razor
 #endif

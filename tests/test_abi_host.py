@@ -132,15 +132,16 @@ def _coverage(items, tokens):
     return pages, seen
 
 
-@pytest.mark.parametrize("tokens,target", [
-    ([65536] * 6 + [8196] * 34, 9472),                         # one sequence of the 64K-shaped stack
-    ([131072, 16388, 16388, 16388, 131072, 16388, 16388, 16388], 4736),
-    ([0, 1, 15, 16, 17, 100000, 3], 64),
-    ([5000] * 2048, 9472),
-    ([7], 1),
+@pytest.mark.parametrize("tokens,target,min_chunk", [
+    ([65536] * 6 + [8196] * 34, 148 * 24, 8),                  # one sequence of the 64K-shaped stack
+    ([131072, 16388, 16388, 16388, 131072, 16388, 16388, 16388], 148 * 24, 8),
+    ([0, 1, 15, 16, 17, 100000, 3], 64, 1),
+    ([5000] * 2048, 148 * 24, 8),
+    ([7], 1, 1),
+    ([1 << 20] * 3, 148 * 200, 1),                             # more parts than the item budget: chunk grows
 ])
-def test_schedule_covers_every_page_once_and_is_balanced(tokens, target):
-    items = rz.razor_schedule_plan(tokens, target)
+def test_schedule_covers_every_page_once_and_is_balanced(tokens, target, min_chunk):
+    items = rz.razor_schedule_plan(tokens, target, min_chunk)
     pages, seen = _coverage(items, tokens)
     sizes = []
     for h, parts in seen.items():
@@ -154,18 +155,24 @@ def test_schedule_covers_every_page_once_and_is_balanced(tokens, target):
         assert len(open_ended) == 1                            # the last part grows with appends
         sizes += [p[1] - p[0] for p in parts]
     total = sum(pages)
-    chunk = max(4, -(-total // max(1, min(target, len(items)))))
-    assert max(sizes) <= max(chunk, 4) + 1
-    assert len(items) <= len(tokens) + target + 1
-    # longest first
-    lens = [(pages[h] if p1 < 0 else p1) - p0 for h, p0, p1, _ in items]
-    assert lens == sorted(lens, reverse=True)
+    chunk = max(min_chunk, -(-total // target))
+    if len(tokens) + total // chunk <= 16384:                  # item budget not hit: parts obey the chunk
+        assert max(sizes) <= chunk
+        assert len(items) <= len(tokens) + total // chunk + 1
+    else:                                                      # the chunk grew until the items fit
+        assert len(items) <= len(tokens) + 16384
+        assert max(sizes) - min(sizes) <= 1
+    # heads cut into the most parts first; within equal part counts, longer ranges first
+    keys = [(-parts, -((pages[h] if p1 < 0 else p1) - p0)) for h, p0, p1, parts in items]
+    assert keys == sorted(keys)
 
 
 def test_schedule_splits_only_long_heads():
     tokens = [65536] * 2 + [8196] * 10
-    items = rz.razor_schedule_plan(tokens, 64)
+    items = rz.razor_schedule_plan(tokens, 64, 4)
     parts = {h: n for h, _, _, n in items}
     assert parts[0] > 8 * parts[5] - 8 and parts[5] >= 1
     with pytest.raises(rz.RazorError):
         rz.razor_schedule_plan([-1], 4)
+    with pytest.raises(rz.RazorError):
+        rz.razor_schedule_plan([100], 4, 0)
