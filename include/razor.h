@@ -184,10 +184,13 @@ RAZOR_API int razor_schedule_query(razor_cache_t* cache, int32_t layer, int32_t*
  * next razor_decode_attention.  Errors: NULL_PTR, INVALID_ARG (unknown option or value out of range).
  */
 enum {
-  RAZOR_OPT_DECODE_ITEMS_PER_SM = 1,    /* work items aimed for per SM (1..1024; default 24)              */
+  RAZOR_OPT_DECODE_ITEMS_PER_SM = 1,    /* work items aimed for per SM (1..1024; default 16)              */
   RAZOR_OPT_DECODE_MIN_CHUNK_PAGES = 2, /* smallest work item in pages (default 8)                        */
   RAZOR_OPT_DECODE_RING_KB = 3,         /* shared-memory page ring per CTA in KiB; 0 = as large as fits   */
-  RAZOR_OPT_DECODE_CONSUMER_WARPS = 4   /* 0 = default; 8, 12 or 16 (bf16, group <= 2 only)               */
+  RAZOR_OPT_DECODE_CONSUMER_WARPS = 4,  /* streaming warps per CTA: 0 = default; 4, 8, 12 or 16; a value
+                                           the head shape has no kernel for falls back to the default     */
+  RAZOR_OPT_DECODE_TENSOR_CORES = 5     /* bf16 grouped-query heads: 0 = matrix instructions from group 4
+                                           up (default), 1 = from group 2 up, 2 = never                   */
 };
 RAZOR_API int razor_cache_set_option(razor_cache_t* cache, int32_t option, int32_t value);
 

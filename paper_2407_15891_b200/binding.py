@@ -207,6 +207,7 @@ def razor_schedule_plan(tokens, target_items: int, min_chunk_pages: int = 1) -> 
 
 
 OPT_DECODE_ITEMS_PER_SM, OPT_DECODE_MIN_CHUNK_PAGES, OPT_DECODE_RING_KB, OPT_DECODE_CONSUMER_WARPS = 1, 2, 3, 4
+OPT_DECODE_TENSOR_CORES = 5
 
 
 def razor_cache_set_option(cache: int, option: int, value: int) -> None:

@@ -119,7 +119,7 @@ struct razor_cache {
   DeviceView dv;
   long long pool_pages = 0, next_page = 0;
   int n_sms = 148;
-  DecodeTuning tune{24, 8, 0, 0};
+  DecodeTuning tune{16, 8, 0, 0, 0};
   std::vector<LayerHost> layers;
   WorkItem* pinned_items = nullptr;   // [L][max_items]
 };
@@ -575,8 +575,12 @@ int razor_cache_set_option(razor_cache_t* c, int32_t option, int32_t value) {
       c->tune.ring_kb = value;
       break;
     case RAZOR_OPT_DECODE_CONSUMER_WARPS:
-      if (value != 0 && value != 8 && value != 12 && value != 16) return RAZOR_E_INVALID_ARG;
+      if (value != 0 && value != 4 && value != 8 && value != 12 && value != 16) return RAZOR_E_INVALID_ARG;
       c->tune.consumer_warps = value;
+      break;
+    case RAZOR_OPT_DECODE_TENSOR_CORES:
+      if (value < 0 || value > 2) return RAZOR_E_INVALID_ARG;
+      c->tune.tensor_cores = value;
       break;
     default:
       return RAZOR_E_INVALID_ARG;

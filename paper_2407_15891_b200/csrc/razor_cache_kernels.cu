@@ -61,7 +61,7 @@ __global__ void __launch_bounds__(256) compress_kernel(DeviceView dv, int layer,
       else slot = -1;
       if (slot >= 0) {
         const size_t page = (size_t)pt[slot >> 4];
-        uint4* dst = (uint4*)(dv.pool + page * dv.page_bytes + (size_t)(slot & 15) * Geo::kRowBytes) + lir;
+        uint4* dst = (uint4*)(dv.pool + page * dv.page_bytes + (size_t)(slot & 15) * Geo::kRowBytes) + swz(slot, lir);
         dst[0] = kf[u];
         dst[kPageTokens * LPR] = vf[u];   // V rows follow the 16 K rows of the page
       } else {
@@ -146,7 +146,7 @@ __global__ void __launch_bounds__(128) append_kernel(DeviceView dv, int layer, c
     uint4* krow = nullptr;
     if (slot >= 0) {
       const size_t page = (size_t)dv.page_table[hs * dv.max_pages + (slot >> 4)];
-      krow = (uint4*)(dv.pool + page * dv.page_bytes + (size_t)(slot & 15) * Geo::kRowBytes) + lane;
+      krow = (uint4*)(dv.pool + page * dv.page_bytes + (size_t)(slot & 15) * Geo::kRowBytes) + swz(slot, lane);
     }
     if (evict || fold_new) {
       const uint4 ok = evict ? krow[0] : kf;
@@ -197,7 +197,8 @@ __global__ void __launch_bounds__(256) export_kernel(DeviceView dv, int layer, i
       pos = total - st.window + j;
     }
     const size_t page = (size_t)dv.page_table[hs * dv.max_pages + (slot >> 4)];
-    const uint4* src = (const uint4*)(dv.pool + page * dv.page_bytes + (size_t)(slot & 15) * Geo::kRowBytes) + lir;
+    const uint4* src =
+        (const uint4*)(dv.pool + page * dv.page_bytes + (size_t)(slot & 15) * Geo::kRowBytes) + swz(slot, lir);
     if (K) ((uint4*)(K + (size_t)i * D))[lir] = src[0];
     if (V) ((uint4*)(V + (size_t)i * D))[lir] = src[kPageTokens * LPR];
     if (kept_pos && lir == 0) kept_pos[i] = pos;

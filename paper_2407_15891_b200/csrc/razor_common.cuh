@@ -51,6 +51,13 @@ struct RowGeom {
   static_assert(kLpr == 8 || kLpr == 16 || kLpr == 32, "row must be 128, 256 or 512 bytes");
 };
 
+// In-page placement of 16-byte chunks.  A page is stored as [16 K rows][16 V rows]; chunk c of the row
+// of token t (t = slot & 15) sits at chunk position c ^ (t & 7).  The page travels to shared memory
+// as one flat block, and with this placement eight rows read at the same logical chunk fall into
+// eight different bank groups, which is what the matrix-fragment loads of the grouped-query path
+// need; row-wise readers just permute their lanes.
+__device__ __forceinline__ int swz(int token, int chunk) { return chunk ^ (token & 7); }
+
 // Streaming 16-byte load: the KV cache is read once per step, keep it out of L1.
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
   uint4 v;

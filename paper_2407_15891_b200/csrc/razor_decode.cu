@@ -168,18 +168,18 @@ __device__ __forceinline__ void merge_state(float& m, float& l, float (&o)[EPL],
   m = mm;
 }
 
-// One page (16 tokens) from shared memory into the running state of a consumer warp.
-// kp points at this lane's first 16-byte fragment of the page (row group rg, fragment lir).
+// One page (16 tokens) from shared memory into the running state of a consumer warp (CUDA cores).
+// `page` is the page's first 16-byte chunk; this lane reads logical chunk lir of the rows i*RG + rg.
 template <typename T, int D, int G>
-__device__ __forceinline__ void consume_page(const uint4* kp, int valid, int rg,
+__device__ __forceinline__ void consume_page(const uint4* page, int valid, int rg, int lir,
                                              const float (&qf)[G][Elem<T>::kEpl], SoftmaxState<G, Elem<T>::kEpl>& S) {
   using Geo = RowGeom<T, D>;
   constexpr int LPR = Geo::kLpr, EPL = Geo::kEpl, RG = Geo::kRg, RPG = Geo::kRowsPerGroup;
   uint4 kf[RPG], vf[RPG];
 #pragma unroll
-  for (int i = 0; i < RPG; ++i) kf[i] = kp[i * 32];
+  for (int i = 0; i < RPG; ++i) kf[i] = page[(i * RG + rg) * LPR + swz(i * RG + rg, lir)];
 #pragma unroll
-  for (int i = 0; i < RPG; ++i) vf[i] = kp[kPageTokens * LPR + i * 32];
+  for (int i = 0; i < RPG; ++i) vf[i] = page[(kPageTokens + i * RG + rg) * LPR + swz(i * RG + rg, lir)];
 
   float s[G][RPG];
 #pragma unroll
@@ -240,6 +240,127 @@ __device__ __forceinline__ void consume_page(const uint4* kp, int valid, int rg,
   }
 }
 
+// ------------------------------------------------------------------------------------------ tensor-core path
+// Grouped-query heads (bf16, G >= 2): the G query heads that share a KV head form the rows of a dense
+// tile, so a page is consumed with warp-level matrix instructions (m16n8k16, bf16 in, fp32 out):
+//   S[head][token] = Q[head][:] . K[token][:]      A = Q (rows >= G are zero), B = K rows as they lie
+//   O[head][:]    += P[head][token] * V[token][:]   A = P from the S accumulators, B = V (transposed load)
+// P is split into a bf16 head and a bf16 remainder (two products), so the weights keep fp32-like
+// accuracy.  Lane (g = lane / 4, t = lane % 4) owns head g and tokens {2t, 2t+1, 8+2t, 9+2t} of the page.
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(addr));
+}
+// d += a * b with rows 8..15 of a equal to zero (a1 = a3 = 0).
+__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
+  const uint32_t z = 0u;
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(z), "r"(a2), "r"(z), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);   // .x = lo (low half), .y = hi
+  return *(const uint32_t*)&v;
+}
+
+template <int D>
+struct MmaState {
+  static constexpr int kNT = D / 8;   // 8-wide output tiles along the head dimension
+  float m, l;                          // head g: running max (log2 domain), this lane's share of the denominator
+  float o[kNT][4];                     // o[nt][0..1] = O[g][nt*8 + 2t, +1]; [2..3] belong to the zero rows
+  __device__ __forceinline__ void clear() {
+    m = -CUDART_INF_F;
+    l = 0.f;
+#pragma unroll
+    for (int i = 0; i < kNT; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+  }
+};
+
+// qa[kk][0] = Q[g][kk*16 + 2t, +1], qa[kk][1] = Q[g][kk*16 + 8 + 2t, +1] (bf16 pairs; zero for g >= G).
+template <int D>
+__device__ __forceinline__ void consume_page_mma(uint32_t page_addr, int valid, int lane, float scale_log2,
+                                                 const uint32_t (&qa)[D / 16][2], MmaState<D>& S) {
+  constexpr int ROW = D * 2;          // bytes per row
+  constexpr int KS = D / 16;          // k-steps of the Q.K product
+  constexpr int NT = D / 8;
+  const int r = lane & 7, mi = lane >> 3, t = lane & 3;
+
+  // ---- S = Q K^T: two 8-token tiles, two accumulation chains each
+  float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+  float u0[4] = {0.f, 0.f, 0.f, 0.f}, u1[4] = {0.f, 0.f, 0.f, 0.f};
+  {
+    const int token = ((mi >> 1) << 3) + r;
+    const uint32_t row_addr = page_addr + token * ROW;
+#pragma unroll
+    for (int kk = 0; kk < KS; ++kk) {
+      uint32_t b[4];
+      ldmatrix_x4(b, row_addr + (((2 * kk + (mi & 1)) ^ r) << 4));
+      if (kk & 1) {
+        mma_bf16(u0, qa[kk][0], qa[kk][1], b[0], b[1]);
+        mma_bf16(u1, qa[kk][0], qa[kk][1], b[2], b[3]);
+      } else {
+        mma_bf16(s0, qa[kk][0], qa[kk][1], b[0], b[1]);
+        mma_bf16(s1, qa[kk][0], qa[kk][1], b[2], b[3]);
+      }
+    }
+  }
+  float s[4] = {(s0[0] + u0[0]) * scale_log2, (s0[1] + u0[1]) * scale_log2, (s1[0] + u1[0]) * scale_log2,
+                (s1[1] + u1[1]) * scale_log2};
+  if (valid < kPageTokens) {   // tokens of this page beyond the head's length
+    if (2 * t >= valid) s[0] = -CUDART_INF_F;
+    if (2 * t + 1 >= valid) s[1] = -CUDART_INF_F;
+    if (8 + 2 * t >= valid) s[2] = -CUDART_INF_F;
+    if (9 + 2 * t >= valid) s[3] = -CUDART_INF_F;
+  }
+  // ---- online softmax for head g (the four lanes of a quad share it)
+  float mx = fmaxf(fmaxf(s[0], s[1]), fmaxf(s[2], s[3]));
+  mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+  mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+  const float m_new = fmaxf(S.m, mx);
+  const float m_use = (m_new == -CUDART_INF_F) ? 0.f : m_new;
+  const float corr = fast_exp2(S.m - m_use);
+  float p[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) p[i] = fast_exp2(s[i] - m_use);
+  S.l = S.l * corr + (p[0] + p[1]) + (p[2] + p[3]);
+  S.m = m_new;
+#pragma unroll
+  for (int i = 0; i < NT; ++i) {
+    S.o[i][0] *= corr;
+    S.o[i][1] *= corr;
+  }
+  // P as a bf16 head plus a bf16 remainder
+  float ph[4], pl[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    ph[i] = __bfloat162float(__float2bfloat16_rn(p[i]));
+    pl[i] = p[i] - ph[i];
+  }
+  const uint32_t ah0 = pack_bf16(ph[0], ph[1]), ah2 = pack_bf16(ph[2], ph[3]);
+  const uint32_t al0 = pack_bf16(pl[0], pl[1]), al2 = pack_bf16(pl[2], pl[3]);
+  // ---- O += P V
+  {
+    const int token = ((mi & 1) << 3) + r;
+    const uint32_t row_addr = page_addr + (kPageTokens + token) * ROW;
+#pragma unroll
+    for (int c = 0; c < NT; c += 2) {
+      uint32_t b[4];
+      ldmatrix_x4_trans(b, row_addr + (((c + (mi >> 1)) ^ r) << 4));
+      mma_bf16(S.o[c], ah0, ah2, b[0], b[1]);
+      mma_bf16(S.o[c + 1], ah0, ah2, b[2], b[3]);
+      mma_bf16(S.o[c], al0, al2, b[0], b[1]);
+      mma_bf16(S.o[c + 1], al0, al2, b[2], b[3]);
+    }
+  }
+}
+
 // Reducer-side vector of D/32 consecutive floats per lane.
 template <int D>
 struct LaneVec;
@@ -267,9 +388,10 @@ struct LaneVec<64> {
 };
 
 // ------------------------------------------------------------------------------------------ the kernel
-template <typename T, int D, int G, int NC>
+template <typename T, int D, int G, int NC, bool MMA>
 __global__ void __launch_bounds__((NC + 2) * 32, 1)
 decode_kernel(DeviceView dv, int layer, int n_items, const T* __restrict__ q, float* __restrict__ out, int n_stages) {
+  static_assert(!MMA || (sizeof(T) == 2 && G >= 2), "the tensor-core path is for grouped bf16 heads");
   using Geo = RowGeom<T, D>;
   constexpr int LPR = Geo::kLpr, EPL = Geo::kEpl;
   constexpr uint32_t PB = Geo::kPageBytes;
@@ -433,77 +555,155 @@ decode_kernel(DeviceView dv, int layer, int n_items, const T* __restrict__ q, fl
         if (lane == 0) mbar_arrive(&bars.merge_full[mb]);
         break;
       }
-      float qf[G][EPL];
+      if constexpr (MMA) {
+        // ---------------------------------------------------------------- tensor-core consumer
+        const int g = lane >> 2, t = lane & 3;
+        uint32_t qa[D / 16][2];
 #pragma unroll
-      for (int j = 0; j < G; ++j) {
-        const uint4 u = ((const uint4*)&sl.q[j][0])[lir];
-        Elem<T>::unpack(u, qf[j]);
-#pragma unroll
-        for (int e = 0; e < EPL; ++e) qf[j][e] *= dv.scale_log2;
-      }
-      SoftmaxState<G, EPL> S;
-      S.clear();
-      const bool first = warp == 0;   // the warp that takes the item's first page also takes its seed
-      // Compensation token (Eq. 4, Eq. 5) seeds the first part of a head that dropped tokens.
-      if (d.seed && first) {
-        float kh[EPL], vh[EPL];
-#pragma unroll
-        for (int e = 0; e < EPL; ++e) { kh[e] = sl.mean[0][lir * EPL + e]; vh[e] = sl.mean[1][lir * EPL + e]; }
-        const float log_cnt = log2f((float)d.n_drop);
-#pragma unroll
-        for (int j = 0; j < G; ++j) {
-          float s = 0.f;
-#pragma unroll
-          for (int e = 0; e < EPL; ++e) s += qf[j][e] * kh[e];
-          s = row_sum<LPR>(s);
-          if (rg == 0) {
-            S.m[j] = s + log_cnt;
-            S.l[j] = 1.f;
-#pragma unroll
-            for (int e = 0; e < EPL; ++e) S.o[j][e] = vh[e];
+        for (int kk = 0; kk < D / 16; ++kk) {
+          qa[kk][0] = qa[kk][1] = 0u;
+          if (g < G) {
+            const uint32_t* qrow = (const uint32_t*)&sl.q[g][0];
+            qa[kk][0] = qrow[kk * 8 + t];
+            qa[kk][1] = qrow[kk * 8 + 4 + t];
           }
         }
-      }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&bars.item_empty[slot]);   // this warp holds all it needs from the slot
-
-      const int n_pad = (d.n_pages + NC - 1) / NC * NC;
-      for (int i = warp; i < n_pad; i += NC) {
-        const unsigned cc = c + i, stage = cc % ns, use = cc / ns;
-        if (!warp_wait(&bars.full[stage], use & 1)) { ok = false; break; }
-        if (i < d.n_pages) {
-          const uint4* kp = (const uint4*)(ring + (size_t)stage * PB) + rg * LPR + lir;
-          consume_page<T, D, G>(kp, d.len - (d.page_begin + i) * kPageTokens, rg, qf, S);
+        MmaState<D> S;
+        S.clear();
+        const bool first = warp == 0;
+        // Compensation token (Eq. 4, Eq. 5) seeds the first part of a head that dropped tokens.
+        if (d.seed && first) {
+          constexpr int PER = D / 32;
+          const float log_cnt = log2f((float)d.n_drop);
+#pragma unroll 1
+          for (int j = 0; j < G; ++j) {
+            float sc = 0.f;
+#pragma unroll
+            for (int e = 0; e < PER; ++e)
+              sc += __bfloat162float(sl.q[j][lane * PER + e]) * sl.mean[0][lane * PER + e];
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) sc += __shfl_xor_sync(0xffffffffu, sc, off);
+            if (g == j) {
+              S.m = sc * dv.scale_log2 + log_cnt;
+              S.l = (t == 0) ? 1.f : 0.f;
+#pragma unroll
+              for (int nt = 0; nt < D / 8; ++nt) {
+                S.o[nt][0] = sl.mean[1][nt * 8 + 2 * t];
+                S.o[nt][1] = sl.mean[1][nt * 8 + 2 * t + 1];
+              }
+            }
+          }
         }
         __syncwarp();
-        if (lane == 0) mbar_arrive(&bars.empty[stage]);
-      }
-      if (!ok) break;
-      c += n_pad;
+        if (lane == 0) mbar_arrive(&bars.item_empty[slot]);   // this warp holds all it needs from the slot
 
-      // Row groups of the warp hold disjoint token subsets: merge them.
-#pragma unroll
-      for (int off = LPR; off < 32; off <<= 1) {
-#pragma unroll
-        for (int j = 0; j < G; ++j) {
-          const float m2 = __shfl_xor_sync(0xffffffffu, S.m[j], off);
-          const float l2 = __shfl_xor_sync(0xffffffffu, S.l[j], off);
-          float o2[EPL];
-#pragma unroll
-          for (int e = 0; e < EPL; ++e) o2[e] = __shfl_xor_sync(0xffffffffu, S.o[j][e], off);
-          merge_state<EPL>(S.m[j], S.l[j], S.o[j], m2, l2, o2);
+        const int n_pad = (d.n_pages + NC - 1) / NC * NC;
+        for (int i = warp; i < n_pad; i += NC) {
+          const unsigned cc = c + i, stage = cc % ns, use = cc / ns;
+          if (!warp_wait(&bars.full[stage], use & 1)) { ok = false; break; }
+          if (i < d.n_pages) {
+            uint8_t* page = ring + (size_t)stage * PB;
+            const int valid = d.len - (d.page_begin + i) * kPageTokens;
+            if (valid < kPageTokens) {
+              // V rows beyond the head's length may hold anything; a zero weight times a NaN is a NaN
+              uint4* vrows = (uint4*)page + (kPageTokens + max(valid, 0)) * LPR;
+              for (int idx = lane; idx < (kPageTokens - max(valid, 0)) * LPR; idx += 32)
+                vrows[idx] = make_uint4(0u, 0u, 0u, 0u);
+              __syncwarp();
+            }
+            consume_page_mma<D>(smem_u32(page), valid, lane, dv.scale_log2, qa, S);
+          }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&bars.empty[stage]);
         }
-      }
-      // Hand the state over to the reducer.
-      if (seq >= kMergeBufs && !warp_wait(&bars.merge_free[mb], ((seq / kMergeBufs) - 1) & 1)) { ok = false; break; }
-      if (first && lane == 0) M.desc = d;
-      if (rg == 0) {
+        if (!ok) break;
+        c += n_pad;
+
+        S.l += __shfl_xor_sync(0xffffffffu, S.l, 1);
+        S.l += __shfl_xor_sync(0xffffffffu, S.l, 2);
+        // Hand the state over to the reducer.
+        if (seq >= kMergeBufs && !warp_wait(&bars.merge_free[mb], ((seq / kMergeBufs) - 1) & 1)) { ok = false; break; }
+        if (first && lane == 0) M.desc = d;
+        if (g < G) {
+          if (t == 0) M.ml[warp][g] = make_float2(S.m, S.l);
+#pragma unroll
+          for (int nt = 0; nt < D / 8; ++nt)
+            *(float2*)&M.o[warp][g][nt * 8 + 2 * t] = make_float2(S.o[nt][0], S.o[nt][1]);
+        }
+      } else {
+        // ---------------------------------------------------------------- CUDA-core consumer
+        float qf[G][EPL];
 #pragma unroll
         for (int j = 0; j < G; ++j) {
-          if (lir == 0) M.ml[warp][j] = make_float2(S.m[j], S.l[j]);
+          const uint4 u = ((const uint4*)&sl.q[j][0])[lir];
+          Elem<T>::unpack(u, qf[j]);
 #pragma unroll
-          for (int e = 0; e < EPL; e += 4)
-            *(float4*)&M.o[warp][j][lir * EPL + e] = make_float4(S.o[j][e], S.o[j][e + 1], S.o[j][e + 2], S.o[j][e + 3]);
+          for (int e = 0; e < EPL; ++e) qf[j][e] *= dv.scale_log2;
+        }
+        SoftmaxState<G, EPL> S;
+        S.clear();
+        const bool first = warp == 0;   // the warp that takes the item's first page also takes its seed
+        // Compensation token (Eq. 4, Eq. 5) seeds the first part of a head that dropped tokens.
+        if (d.seed && first) {
+          float kh[EPL], vh[EPL];
+#pragma unroll
+          for (int e = 0; e < EPL; ++e) { kh[e] = sl.mean[0][lir * EPL + e]; vh[e] = sl.mean[1][lir * EPL + e]; }
+          const float log_cnt = log2f((float)d.n_drop);
+#pragma unroll
+          for (int j = 0; j < G; ++j) {
+            float s = 0.f;
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) s += qf[j][e] * kh[e];
+            s = row_sum<LPR>(s);
+            if (rg == 0) {
+              S.m[j] = s + log_cnt;
+              S.l[j] = 1.f;
+#pragma unroll
+              for (int e = 0; e < EPL; ++e) S.o[j][e] = vh[e];
+            }
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bars.item_empty[slot]);   // this warp holds all it needs from the slot
+
+        const int n_pad = (d.n_pages + NC - 1) / NC * NC;
+        for (int i = warp; i < n_pad; i += NC) {
+          const unsigned cc = c + i, stage = cc % ns, use = cc / ns;
+          if (!warp_wait(&bars.full[stage], use & 1)) { ok = false; break; }
+          if (i < d.n_pages) {
+            consume_page<T, D, G>((const uint4*)(ring + (size_t)stage * PB), d.len - (d.page_begin + i) * kPageTokens,
+                                  rg, lir, qf, S);
+          }
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&bars.empty[stage]);
+        }
+        if (!ok) break;
+        c += n_pad;
+
+        // Row groups of the warp hold disjoint token subsets: merge them.
+#pragma unroll
+        for (int off = LPR; off < 32; off <<= 1) {
+#pragma unroll
+          for (int j = 0; j < G; ++j) {
+            const float m2 = __shfl_xor_sync(0xffffffffu, S.m[j], off);
+            const float l2 = __shfl_xor_sync(0xffffffffu, S.l[j], off);
+            float o2[EPL];
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) o2[e] = __shfl_xor_sync(0xffffffffu, S.o[j][e], off);
+            merge_state<EPL>(S.m[j], S.l[j], S.o[j], m2, l2, o2);
+          }
+        }
+        // Hand the state over to the reducer.
+        if (seq >= kMergeBufs && !warp_wait(&bars.merge_free[mb], ((seq / kMergeBufs) - 1) & 1)) { ok = false; break; }
+        if (first && lane == 0) M.desc = d;
+        if (rg == 0) {
+#pragma unroll
+          for (int j = 0; j < G; ++j) {
+            if (lir == 0) M.ml[warp][j] = make_float2(S.m[j], S.l[j]);
+#pragma unroll
+            for (int e = 0; e < EPL; e += 4)
+              *(float4*)&M.o[warp][j][lir * EPL + e] = make_float4(S.o[j][e], S.o[j][e + 1], S.o[j][e + 2], S.o[j][e + 3]);
+          }
         }
       }
       __syncwarp();
@@ -622,10 +822,10 @@ decode_kernel(DeviceView dv, int layer, int n_items, const T* __restrict__ q, fl
 // ------------------------------------------------------------------------------------------ launch
 constexpr int kSmemOptIn = 232448;   // 227 KiB: the most one CTA may hold on sm_100
 
-template <typename T, int D, int G, int NC>
+template <typename T, int D, int G, int NC, bool MMA>
 cudaError_t decode_launch(const DeviceView& dv, int layer, int n_items, const void* q, float* out, int n_sms,
                           const DecodeTuning& tune, cudaStream_t s) {
-  auto kern = decode_kernel<T, D, G, NC>;
+  auto kern = decode_kernel<T, D, G, NC, MMA>;
   constexpr size_t PB = RowGeom<T, D>::kPageBytes;
   constexpr size_t ring_off = decode_ring_offset<T, D, G, NC>();
   static int static_smem = -1;        // per instantiation
@@ -664,14 +864,23 @@ cudaError_t decode_nc(const DeviceView& dv, int layer, int n_items, const void* 
                       const DecodeTuning& tune, cudaStream_t s) {
   // Consumer warps.  The ring holds a multiple of NC pages and (NC + 2) warps share the register file,
   // so the choice trades pages in flight against registers per thread.
-  if constexpr (sizeof(T) == 2 && G <= 2) {
-    if (tune.consumer_warps == 8) return decode_launch<T, D, G, 8>(dv, layer, n_items, q, out, n_sms, tune, s);
-    if (tune.consumer_warps == 16) return decode_launch<T, D, G, 16>(dv, layer, n_items, q, out, n_sms, tune, s);
-    return decode_launch<T, D, G, 12>(dv, layer, n_items, q, out, n_sms, tune, s);
+  const int nc = tune.consumer_warps;
+  if constexpr (sizeof(T) == 2 && G >= 2) {
+    // Grouped heads: the tensor-core consumer unless switched off (default on from group 4 up).
+    const bool mma = tune.tensor_cores == 1 || (tune.tensor_cores == 0 && G >= 4);
+    if (mma) {
+      if (nc == 4) return decode_launch<T, D, G, 4, true>(dv, layer, n_items, q, out, n_sms, tune, s);
+      return decode_launch<T, D, G, 8, true>(dv, layer, n_items, q, out, n_sms, tune, s);
+    }
+  }
+  if constexpr (sizeof(T) == 2 && G == 1) {
+    if (nc == 8) return decode_launch<T, D, G, 8, false>(dv, layer, n_items, q, out, n_sms, tune, s);
+    if (nc == 16) return decode_launch<T, D, G, 16, false>(dv, layer, n_items, q, out, n_sms, tune, s);
+    return decode_launch<T, D, G, 12, false>(dv, layer, n_items, q, out, n_sms, tune, s);
   } else if constexpr (sizeof(T) == 2) {
-    return decode_launch<T, D, G, 8>(dv, layer, n_items, q, out, n_sms, tune, s);
+    return decode_launch<T, D, G, 8, false>(dv, layer, n_items, q, out, n_sms, tune, s);
   } else {
-    return decode_launch<T, D, G, 4>(dv, layer, n_items, q, out, n_sms, tune, s);
+    return decode_launch<T, D, G, 4, false>(dv, layer, n_items, q, out, n_sms, tune, s);
   }
 }
 

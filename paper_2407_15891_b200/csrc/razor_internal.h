@@ -98,6 +98,7 @@ struct DecodeTuning {
   int32_t min_chunk_pages;  // smallest work item
   int32_t ring_kb;          // shared-memory page ring per CTA, KiB (0: as large as fits)
   int32_t consumer_warps;   // 0: default for the group size
+  int32_t tensor_cores;     // grouped bf16 heads: 0 auto (group >= 4), 1 on (group >= 2), 2 off
 };
 
 // Kernel launchers (defined in the .cu files).  Each returns the cudaError_t of the launch.

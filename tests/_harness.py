@@ -45,12 +45,16 @@ def rel_inf(a: np.ndarray, ref: np.ndarray) -> float:
 
 
 def make_cache(w: synth.Workload, layers: Optional[Sequence[int]] = None, max_new: Optional[int] = None,
-               shuffle: int = 0, use_comp: int = 1, sm_scale: float = 0.0, device="cuda:0") -> rz.RazorCache:
+               shuffle: int = 0, use_comp: int = 1, sm_scale: float = 0.0, device="cuda:0",
+               options: Optional[Dict[int, int]] = None) -> rz.RazorCache:
     n_layers = w.n_layers
     cfg = rz.make_config(w.batch, n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, w.n_sink,
                          max(w.ctx_len), w.decode_steps if max_new is None else max_new, use_comp, shuffle, sm_scale)
     retr = np.stack([w.retrieval(l) for l in range(n_layers)])
-    return rz.RazorCache(cfg, w.ctx_len, w.window, retr, device=device)
+    cache = rz.RazorCache(cfg, w.ctx_len, w.window, retr, device=device)
+    for opt, val in (options or {}).items():
+        cache.set_option(opt, val)
+    return cache
 
 
 class HeadRef:
@@ -102,7 +106,8 @@ def sample_heads(w: synth.Workload, layer: int, n_retr: int, n_other: int, batch
 def run_parity(w: synth.Workload, *, layers: Optional[Sequence[int]] = None,
                heads_for: Optional[Dict[int, List[Tuple[int, int]]]] = None, steps: Optional[int] = None,
                shuffle: int = 0, use_comp: int = 1, sm_scale: float = 0.0, per_seq: bool = False,
-               check_layout_every: int = 0, device="cuda:0", stats: Optional[dict] = None) -> dict:
+               check_layout_every: int = 0, device="cuda:0", stats: Optional[dict] = None,
+               options: Optional[Dict[int, int]] = None) -> dict:
     """Compress every layer, then run `steps` x (append, decode) over all layers on the GPU, checking
     the heads listed in heads_for[layer] (default: every head of every layer) against the oracle.
     With steps == 0 one decode is run straight after compression (no append)."""
@@ -115,7 +120,8 @@ def run_parity(w: synth.Workload, *, layers: Optional[Sequence[int]] = None,
     scale = sm_scale if sm_scale else 1.0 / math.sqrt(w.head_dim)
     G = w.group
     tol = TOL_OUT[w.dtype]
-    cache = make_cache(w, max_new=max(steps, 1), shuffle=shuffle, use_comp=use_comp, sm_scale=sm_scale, device=device)
+    cache = make_cache(w, max_new=max(steps, 1), shuffle=shuffle, use_comp=use_comp, sm_scale=sm_scale, device=device,
+                       options=options)
     refs: Dict[Tuple[int, int, int], HeadRef] = {}
     worst = dict(out=0.0, mean=0.0, heads=0, outputs=0)
     try:

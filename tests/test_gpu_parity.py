@@ -119,6 +119,23 @@ def test_small_shape_sweep(dtype, D, group):
         run_parity(w, steps=5 if trial != 3 else 0, shuffle=trial, check_layout_every=1)
 
 
+@pytest.mark.parametrize("group,options", [
+    (2, {rz.OPT_DECODE_TENSOR_CORES: 1}),                                   # matrix instructions from group 2
+    (2, {rz.OPT_DECODE_TENSOR_CORES: 1, rz.OPT_DECODE_CONSUMER_WARPS: 4}),
+    (4, {rz.OPT_DECODE_TENSOR_CORES: 2}),                                   # grouped heads on the CUDA cores
+    (4, {rz.OPT_DECODE_CONSUMER_WARPS: 4, rz.OPT_DECODE_ITEMS_PER_SM: 64, rz.OPT_DECODE_MIN_CHUNK_PAGES: 1}),
+    (8, {rz.OPT_DECODE_RING_KB: 64}),
+    (1, {rz.OPT_DECODE_CONSUMER_WARPS: 16, rz.OPT_DECODE_RING_KB: 128}),
+    (1, {rz.OPT_DECODE_CONSUMER_WARPS: 8, rz.OPT_DECODE_ITEMS_PER_SM: 200, rz.OPT_DECODE_MIN_CHUNK_PAGES: 1}),
+])
+@pytest.mark.parametrize("D", [64, 128])
+def test_decode_kernel_variants(group, options, D):
+    """Every decode kernel variant the options can select, on a ragged batch whose long head is cut into
+    enough parts for a two-level combine tree."""
+    w = synth.Workload("variants", 3, 1, 2 * group, 2, D, "bf16", [9000, 37, 700], [300, 300, 100], 4, 1, 3, 2024 + group)
+    run_parity(w, steps=3, shuffle=7, options=options, check_layout_every=2)
+
+
 def test_append_many_tokens_crosses_pages_evicts_and_rebuilds_schedule():
     w = synth.Workload("long_append", 2, 1, 4, 4, 128, "bf16", [700, 90], [64, 200], 4, 1, 300, 4242)
     run_parity(w, steps=300, check_layout_every=37)
