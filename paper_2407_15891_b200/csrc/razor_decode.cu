@@ -125,6 +125,7 @@ struct Barriers {
   uint64_t item_empty[kItemSlots];
   uint64_t merge_full[kMergeBufs];
   uint64_t merge_free[kMergeBufs];
+  uint64_t land;   // landing zone of the combine-tree merges
 };
 
 // Hand-over buffer: the descriptor of the item, then per consumer warp and query head (m, l) and o[D].
@@ -135,10 +136,16 @@ struct alignas(16) MergeBuf {
   alignas(16) float o[NC][G][D];
 };
 
-// Dynamic shared memory: the hand-over buffers, then the page ring (1 KiB aligned).
+// Dynamic shared memory: the hand-over buffers, the landing zone of the combine-tree merges
+// (kMergeFanIn records x up to 4 heads x D floats), then the page ring (1 KiB aligned).
+template <typename T, int D, int G, int NC>
+constexpr size_t decode_land_offset() {
+  return (sizeof(MergeBuf<D, G, NC>) * kMergeBufs + 127) & ~(size_t)127;
+}
 template <typename T, int D, int G, int NC>
 constexpr size_t decode_ring_offset() {
-  return (sizeof(MergeBuf<D, G, NC>) * kMergeBufs + 1023) & ~(size_t)1023;
+  return (decode_land_offset<T, D, G, NC>() + (size_t)kMergeFanIn * (G < 4 ? G : 4) * D * sizeof(float) + 1023) &
+         ~(size_t)1023;
 }
 
 template <int G, int EPL>
@@ -241,12 +248,15 @@ __device__ __forceinline__ void consume_page(const uint4* page, int valid, int r
 }
 
 // ------------------------------------------------------------------------------------------ tensor-core path
-// Grouped-query heads (bf16, G >= 2): the G query heads that share a KV head form the rows of a dense
-// tile, so a page is consumed with warp-level matrix instructions (m16n8k16, bf16 in, fp32 out):
-//   S[head][token] = Q[head][:] . K[token][:]      A = Q (rows >= G are zero), B = K rows as they lie
-//   O[head][:]    += P[head][token] * V[token][:]   A = P from the S accumulators, B = V (transposed load)
-// P is split into a bf16 head and a bf16 remainder (two products), so the weights keep fp32-like
-// accuracy.  Lane (g = lane / 4, t = lane % 4) owns head g and tokens {2t, 2t+1, 8+2t, 9+2t} of the page.
+// Grouped-query heads (bf16, G >= 2): the query heads that share a KV head make a dense tile with the
+// page's 16 tokens, so a page is consumed with warp-level matrix instructions (m16n8k16, bf16 in,
+// fp32 accumulate):
+//   S[token][head]  = K[token][:] . Q[head][:]       A = K rows as they lie, B = Q (heads >= G are zero)
+//   O^T[d][head]   += V^T[d][token] * P[token][head]  A = V through a transposing load, B = P
+// P goes from the accumulator layout of S to the B layout through an 8x8 register transpose, and is
+// split into a bf16 head and a bf16 remainder (two products), so the weights keep fp32-like accuracy.
+// Lane (g = lane / 4, t = lane % 4) owns query heads 2t, 2t+1: tokens g, g+8 of S and rows g, g+8 of
+// every 16-row tile of O^T.
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
@@ -257,13 +267,17 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t add
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
                : "r"(addr));
 }
-// d += a * b with rows 8..15 of a equal to zero (a1 = a3 = 0).
-__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
-  const uint32_t z = 0u;
+// Transpose of an 8x8 matrix of 16-bit elements held one row-pair per lane.
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t x) {
+  uint32_t y;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(y) : "r"(x));
+  return y;
+}
+__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
   asm volatile(
       "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-      : "r"(a0), "r"(z), "r"(a2), "r"(z), "r"(b0), "r"(b1));
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);   // .x = lo (low half), .y = hi
@@ -272,91 +286,86 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 
 template <int D>
 struct MmaState {
-  static constexpr int kNT = D / 8;   // 8-wide output tiles along the head dimension
-  float m, l;                          // head g: running max (log2 domain), this lane's share of the denominator
-  float o[kNT][4];                     // o[nt][0..1] = O[g][nt*8 + 2t, +1]; [2..3] belong to the zero rows
+  static constexpr int kMT = D / 16;   // 16-row tiles of O^T along the head dimension
+  float m[2], l[2];                     // heads 2t, 2t+1: running max (log2 domain), this lane's share of the denominator
+  float o[kMT][4];                      // o[mt] = O^T[mt*16 + {g, g, g+8, g+8}][head {2t, 2t+1, 2t, 2t+1}]
   __device__ __forceinline__ void clear() {
-    m = -CUDART_INF_F;
-    l = 0.f;
+    m[0] = m[1] = -CUDART_INF_F;
+    l[0] = l[1] = 0.f;
 #pragma unroll
-    for (int i = 0; i < kNT; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+    for (int i = 0; i < kMT; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
   }
 };
 
-// qa[kk][0] = Q[g][kk*16 + 2t, +1], qa[kk][1] = Q[g][kk*16 + 8 + 2t, +1] (bf16 pairs; zero for g >= G).
+// qb[kk][0] = Q[head g][kk*16 + 2t, +1], qb[kk][1] = Q[head g][kk*16 + 8 + 2t, +1] (bf16 pairs; zero for g >= G).
 template <int D>
 __device__ __forceinline__ void consume_page_mma(uint32_t page_addr, int valid, int lane, float scale_log2,
-                                                 const uint32_t (&qa)[D / 16][2], MmaState<D>& S) {
+                                                 const uint32_t (&qb)[D / 16][2], MmaState<D>& S) {
   constexpr int ROW = D * 2;          // bytes per row
-  constexpr int KS = D / 16;          // k-steps of the Q.K product
-  constexpr int NT = D / 8;
-  const int r = lane & 7, mi = lane >> 3, t = lane & 3;
+  constexpr int KS = D / 16;          // k-steps of the K.Q product
+  constexpr int MT = D / 16;
+  const int r = lane & 7, mi = lane >> 3, g = lane >> 2;
 
-  // ---- S = Q K^T: two 8-token tiles, two accumulation chains each
+  // ---- S = K Q^T, two accumulation chains
   float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
-  float u0[4] = {0.f, 0.f, 0.f, 0.f}, u1[4] = {0.f, 0.f, 0.f, 0.f};
   {
-    const int token = ((mi >> 1) << 3) + r;
-    const uint32_t row_addr = page_addr + token * ROW;
+    // matrices of one load: (tokens 0-7, chunk 2kk), (tokens 8-15, 2kk), (tokens 0-7, 2kk+1), (tokens 8-15, 2kk+1)
+    const uint32_t row_addr = page_addr + (((mi & 1) << 3) + r) * ROW;
 #pragma unroll
     for (int kk = 0; kk < KS; ++kk) {
-      uint32_t b[4];
-      ldmatrix_x4(b, row_addr + (((2 * kk + (mi & 1)) ^ r) << 4));
-      if (kk & 1) {
-        mma_bf16(u0, qa[kk][0], qa[kk][1], b[0], b[1]);
-        mma_bf16(u1, qa[kk][0], qa[kk][1], b[2], b[3]);
-      } else {
-        mma_bf16(s0, qa[kk][0], qa[kk][1], b[0], b[1]);
-        mma_bf16(s1, qa[kk][0], qa[kk][1], b[2], b[3]);
-      }
+      uint32_t a[4];
+      ldmatrix_x4(a, row_addr + (((2 * kk + (mi >> 1)) ^ r) << 4));
+      if (kk & 1) mma_bf16(s1, a, qb[kk][0], qb[kk][1]);
+      else mma_bf16(s0, a, qb[kk][0], qb[kk][1]);
     }
   }
-  float s[4] = {(s0[0] + u0[0]) * scale_log2, (s0[1] + u0[1]) * scale_log2, (s1[0] + u1[0]) * scale_log2,
-                (s1[1] + u1[1]) * scale_log2};
+  // s[0], s[1]: token g, heads 2t, 2t+1;  s[2], s[3]: token g+8
+  float s[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) s[i] = (s0[i] + s1[i]) * scale_log2;
   if (valid < kPageTokens) {   // tokens of this page beyond the head's length
-    if (2 * t >= valid) s[0] = -CUDART_INF_F;
-    if (2 * t + 1 >= valid) s[1] = -CUDART_INF_F;
-    if (8 + 2 * t >= valid) s[2] = -CUDART_INF_F;
-    if (9 + 2 * t >= valid) s[3] = -CUDART_INF_F;
+    if (g >= valid) s[0] = s[1] = -CUDART_INF_F;
+    if (g + 8 >= valid) s[2] = s[3] = -CUDART_INF_F;
   }
-  // ---- online softmax for head g (the four lanes of a quad share it)
-  float mx = fmaxf(fmaxf(s[0], s[1]), fmaxf(s[2], s[3]));
-  mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-  mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-  const float m_new = fmaxf(S.m, mx);
-  const float m_use = (m_new == -CUDART_INF_F) ? 0.f : m_new;
-  const float corr = fast_exp2(S.m - m_use);
-  float p[4];
+  // ---- online softmax of heads 2t, 2t+1 (the eight lanes with the same t share them)
+  float mx0 = fmaxf(s[0], s[2]), mx1 = fmaxf(s[1], s[3]);
 #pragma unroll
-  for (int i = 0; i < 4; ++i) p[i] = fast_exp2(s[i] - m_use);
-  S.l = S.l * corr + (p[0] + p[1]) + (p[2] + p[3]);
-  S.m = m_new;
-#pragma unroll
-  for (int i = 0; i < NT; ++i) {
-    S.o[i][0] *= corr;
-    S.o[i][1] *= corr;
+  for (int off = 4; off < 32; off <<= 1) {
+    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
+    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
   }
-  // P as a bf16 head plus a bf16 remainder
-  float ph[4], pl[4];
+  const float mn0 = fmaxf(S.m[0], mx0), mn1 = fmaxf(S.m[1], mx1);
+  const float mu0 = (mn0 == -CUDART_INF_F) ? 0.f : mn0, mu1 = (mn1 == -CUDART_INF_F) ? 0.f : mn1;
+  const float corr0 = fast_exp2(S.m[0] - mu0), corr1 = fast_exp2(S.m[1] - mu1);
+  const float p0 = fast_exp2(s[0] - mu0), p1 = fast_exp2(s[1] - mu1);
+  const float p2 = fast_exp2(s[2] - mu0), p3 = fast_exp2(s[3] - mu1);
+  S.l[0] = S.l[0] * corr0 + (p0 + p2);
+  S.l[1] = S.l[1] * corr1 + (p1 + p3);
+  S.m[0] = mn0;
+  S.m[1] = mn1;
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    ph[i] = __bfloat162float(__float2bfloat16_rn(p[i]));
-    pl[i] = p[i] - ph[i];
+  for (int i = 0; i < MT; ++i) {
+    S.o[i][0] *= corr0;
+    S.o[i][1] *= corr1;
+    S.o[i][2] *= corr0;
+    S.o[i][3] *= corr1;
   }
-  const uint32_t ah0 = pack_bf16(ph[0], ph[1]), ah2 = pack_bf16(ph[2], ph[3]);
-  const uint32_t al0 = pack_bf16(pl[0], pl[1]), al2 = pack_bf16(pl[2], pl[3]);
-  // ---- O += P V
+  // P as a bf16 head plus a bf16 remainder, transposed into the B layout:
+  // b0 = P[tokens 2t, 2t+1][head g], b1 = P[tokens 8+2t, 9+2t][head g]
+  const float h0 = __bfloat162float(__float2bfloat16_rn(p0)), h1 = __bfloat162float(__float2bfloat16_rn(p1));
+  const float h2 = __bfloat162float(__float2bfloat16_rn(p2)), h3 = __bfloat162float(__float2bfloat16_rn(p3));
+  const uint32_t bh0 = movmatrix_trans(pack_bf16(h0, h1)), bh1 = movmatrix_trans(pack_bf16(h2, h3));
+  const uint32_t bl0 = movmatrix_trans(pack_bf16(p0 - h0, p1 - h1)), bl1 = movmatrix_trans(pack_bf16(p2 - h2, p3 - h3));
+  // ---- O^T += V^T P
   {
-    const int token = ((mi & 1) << 3) + r;
-    const uint32_t row_addr = page_addr + (kPageTokens + token) * ROW;
+    // matrices of one load: (tokens 0-7, chunk 2mt), (tokens 0-7, 2mt+1), (tokens 8-15, 2mt), (tokens 8-15, 2mt+1)
+    const uint32_t row_addr = page_addr + (kPageTokens + ((mi >> 1) << 3) + r) * ROW;
 #pragma unroll
-    for (int c = 0; c < NT; c += 2) {
-      uint32_t b[4];
-      ldmatrix_x4_trans(b, row_addr + (((c + (mi >> 1)) ^ r) << 4));
-      mma_bf16(S.o[c], ah0, ah2, b[0], b[1]);
-      mma_bf16(S.o[c + 1], ah0, ah2, b[2], b[3]);
-      mma_bf16(S.o[c], al0, al2, b[0], b[1]);
-      mma_bf16(S.o[c + 1], al0, al2, b[2], b[3]);
+    for (int mt = 0; mt < MT; ++mt) {
+      uint32_t a[4];
+      ldmatrix_x4_trans(a, row_addr + (((2 * mt + (mi & 1)) ^ r) << 4));
+      mma_bf16(S.o[mt], a, bh0, bh1);
+      mma_bf16(S.o[mt], a, bl0, bl1);
     }
   }
 }
@@ -424,6 +433,7 @@ decode_kernel(DeviceView dv, int layer, int n_items, const T* __restrict__ q, fl
       mbar_init(&bars.merge_full[s], NC);
       mbar_init(&bars.merge_free[s], 1);
     }
+    mbar_init(&bars.land, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
@@ -444,11 +454,24 @@ decode_kernel(DeviceView dv, int layer, int n_items, const T* __restrict__ q, fl
     unsigned seq_issued = 0;                             // item slots whose copies were issued
     int marker_slot = -1;                                // slot that received the end marker
     bool ok = true;
+    // Look-ahead of one item: the next item's queue pop, its descriptor, its head state and its first
+    // page ids are requested while the current item's pages are being issued, so that the ring is not
+    // left to drain over a chain of dependent global loads at every item boundary.
+    const WorkItem no_item = {0, 0, 0, 0, 1, 0, 0, 0};
+    auto row_of = [&](const WorkItem& w) { return (size_t)layer * dv.n_heads + w.head; };
+    auto first_pids = [&](const WorkItem& w) {
+      return dv.page_table[row_of(w) * dv.max_pages + min(w.page_begin + lane, dv.max_pages - 1)];
+    };
+    int it = 0;
+    if (lane == 0) it = atomicAdd(dv.queue, 1);
+    it = __shfl_sync(0xffffffffu, it, 0);
+    WorkItem w = it < n_items ? items[it] : no_item;
+    HeadState st = dv.state[row_of(w)];
+    int32_t pid_first = first_pids(w);
     for (unsigned seq = 0; ok; ++seq) {
       const int slot = seq % kItemSlots;
-      int it = 0;
-      if (lane == 0) it = atomicAdd(dv.queue, 1);
-      it = __shfl_sync(0xffffffffu, it, 0);
+      int next_raw = n_items;
+      if (lane == 0 && it < n_items) next_raw = atomicAdd(dv.queue, 1);   // result is picked up below
       if (seq >= kItemSlots) ok = warp_wait(&bars.item_empty[slot], ((seq / kItemSlots) - 1) & 1);
       if (!ok) break;
       Slot& sl = slots[slot];
@@ -460,9 +483,7 @@ decode_kernel(DeviceView dv, int layer, int n_items, const T* __restrict__ q, fl
         marker_slot = slot;
         break;
       }
-      const WorkItem w = items[it];
-      const size_t hs = (size_t)layer * dv.n_heads + w.head;
-      const HeadState st = dv.state[hs];
+      const size_t hs = row_of(w);
       const int head_pages = (st.len + kPageTokens - 1) / kPageTokens;
       const int page_end = w.page_end < 0 ? head_pages : min(w.page_end, head_pages);
       const int n = max(0, page_end - w.page_begin);
@@ -486,15 +507,18 @@ decode_kernel(DeviceView dv, int layer, int n_items, const T* __restrict__ q, fl
       // which CTA streamed it or on what that CTA streamed before): the item starts on a ring position
       // that is a multiple of NC, and the positions left over in its last round are passed on empty.
       const int n_pad = (n + NC - 1) / NC * NC;
+      int it_next = n_items;
+      WorkItem w_next = no_item;
+      bool have_next = false;
+      int32_t pid_cur = pid_first;
       for (int p0 = 0; p0 < n_pad; p0 += batch) {
         const int in_batch = min(batch, n_pad - p0);
         const bool mine = lane < in_batch;
         const bool real = mine && p0 + lane < n;
-        size_t pid = 0;
+        const int32_t pid_after = (p0 + batch + lane < n) ? pt[p0 + batch + lane] : 0;   // ids of the next round
         unsigned stage = 0;
         bool ready = true;
         if (mine) {
-          if (real) pid = (size_t)pt[p0 + lane];
           const unsigned cc = c + lane;
           stage = cc % ns;
           const unsigned use = cc / ns;
@@ -504,12 +528,27 @@ decode_kernel(DeviceView dv, int layer, int n_items, const T* __restrict__ q, fl
         if (!ok) break;
         if (real) {
           mbar_arrive_expect_tx(&bars.full[stage], PB);
-          bulk_load(ring + (size_t)stage * PB, dv.pool + pid * dv.page_bytes, PB, &bars.full[stage]);
+          bulk_load(ring + (size_t)stage * PB, dv.pool + (size_t)pid_cur * dv.page_bytes, PB, &bars.full[stage]);
         } else if (mine) {
           mbar_arrive(&bars.full[stage]);
         }
         c += in_batch;
+        pid_cur = pid_after;
+        if (!have_next) {   // the pop issued above has had a round of copies to come back
+          it_next = __shfl_sync(0xffffffffu, next_raw, 0);
+          w_next = it_next < n_items ? items[it_next] : no_item;
+          have_next = true;
+        }
       }
+      if (!ok) break;
+      if (!have_next) {
+        it_next = __shfl_sync(0xffffffffu, next_raw, 0);
+        w_next = it_next < n_items ? items[it_next] : no_item;
+      }
+      it = it_next;
+      w = w_next;
+      st = dv.state[row_of(w)];
+      pid_first = first_pids(w);
     }
     if (!ok && lane == 0) atomicOr(dv.status, kStatusProducerTimeout);
     // Wait (bounded) until every copy this warp issued has landed: the CTA's shared memory must not be
@@ -558,7 +597,7 @@ decode_kernel(DeviceView dv, int layer, int n_items, const T* __restrict__ q, fl
       if constexpr (MMA) {
         // ---------------------------------------------------------------- tensor-core consumer
         const int g = lane >> 2, t = lane & 3;
-        uint32_t qa[D / 16][2];
+        uint32_t qa[D / 16][2];   // B fragments of Q: head g
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
           qa[kk][0] = qa[kk][1] = 0u;
@@ -575,7 +614,7 @@ decode_kernel(DeviceView dv, int layer, int n_items, const T* __restrict__ q, fl
         if (d.seed && first) {
           constexpr int PER = D / 32;
           const float log_cnt = log2f((float)d.n_drop);
-#pragma unroll 1
+#pragma unroll
           for (int j = 0; j < G; ++j) {
             float sc = 0.f;
 #pragma unroll
@@ -583,13 +622,13 @@ decode_kernel(DeviceView dv, int layer, int n_items, const T* __restrict__ q, fl
               sc += __bfloat162float(sl.q[j][lane * PER + e]) * sl.mean[0][lane * PER + e];
 #pragma unroll
             for (int off = 16; off > 0; off >>= 1) sc += __shfl_xor_sync(0xffffffffu, sc, off);
-            if (g == j) {
-              S.m = sc * dv.scale_log2 + log_cnt;
-              S.l = (t == 0) ? 1.f : 0.f;
+            if (t == (j >> 1)) {   // head j lives in slot j & 1 of the lanes with t = j / 2
+              S.m[j & 1] = sc * dv.scale_log2 + log_cnt;
+              S.l[j & 1] = (g == 0) ? 1.f : 0.f;
 #pragma unroll
-              for (int nt = 0; nt < D / 8; ++nt) {
-                S.o[nt][0] = sl.mean[1][nt * 8 + 2 * t];
-                S.o[nt][1] = sl.mean[1][nt * 8 + 2 * t + 1];
+              for (int mt = 0; mt < D / 16; ++mt) {
+                S.o[mt][j & 1] = sl.mean[1][mt * 16 + g];
+                S.o[mt][2 + (j & 1)] = sl.mean[1][mt * 16 + 8 + g];
               }
             }
           }
@@ -619,16 +658,25 @@ decode_kernel(DeviceView dv, int layer, int n_items, const T* __restrict__ q, fl
         if (!ok) break;
         c += n_pad;
 
-        S.l += __shfl_xor_sync(0xffffffffu, S.l, 1);
-        S.l += __shfl_xor_sync(0xffffffffu, S.l, 2);
+#pragma unroll
+        for (int off = 4; off < 32; off <<= 1) {
+          S.l[0] += __shfl_xor_sync(0xffffffffu, S.l[0], off);
+          S.l[1] += __shfl_xor_sync(0xffffffffu, S.l[1], off);
+        }
         // Hand the state over to the reducer.
         if (seq >= kMergeBufs && !warp_wait(&bars.merge_free[mb], ((seq / kMergeBufs) - 1) & 1)) { ok = false; break; }
         if (first && lane == 0) M.desc = d;
-        if (g < G) {
-          if (t == 0) M.ml[warp][g] = make_float2(S.m, S.l);
 #pragma unroll
-          for (int nt = 0; nt < D / 8; ++nt)
-            *(float2*)&M.o[warp][g][nt * 8 + 2 * t] = make_float2(S.o[nt][0], S.o[nt][1]);
+        for (int e = 0; e < 2; ++e) {
+          const int h = 2 * t + e;
+          if (h < G) {
+            if (g == 0) M.ml[warp][h] = make_float2(S.m[e], S.l[e]);
+#pragma unroll
+            for (int mt = 0; mt < D / 16; ++mt) {
+              M.o[warp][h][mt * 16 + g] = S.o[mt][e];
+              M.o[warp][h][mt * 16 + 8 + g] = S.o[mt][2 + e];
+            }
+          }
         }
       } else {
         // ---------------------------------------------------------------- CUDA-core consumer
@@ -713,7 +761,101 @@ decode_kernel(DeviceView dv, int layer, int n_items, const T* __restrict__ q, fl
   } else {
     // ======================================================================== reducer
     bool ok = true;
-    for (unsigned seq = 0;; ++seq) {
+    unsigned land_uses = 0;
+    float* land = (float*)(dyn_smem + decode_land_offset<T, D, G, NC>());
+    constexpr int GB = G < 4 ? G : 4;   // query heads whose rows land together
+
+    // A part's record has been written and its arrival counted (`ticket` is the count before it).  Walk up
+    // the head's combine tree for as long as this warp delivers the last input of a node.
+    auto climb = [&](int ticket, int idx, int n, int rec_off, int tk_off, float* out_rows) {
+      for (;;) {
+        const int n_next = (n + F - 1) / F, node = idx / F;
+        const int fan = min(F, n - node * F);
+        if (ticket != fan - 1) return;
+        // Last input of this node: merge its `fan` records.
+        __threadfence();
+        if (lane == 0) dv.tickets[tk_off + node] = 0;
+        const int first_rec = rec_off + node * F;
+#pragma unroll 1
+        for (int jh = 0; jh < G; jh += GB) {
+          // The rows of GB heads of every record travel to shared memory as one bulk copy per record
+          // (a single round trip for the whole node); (m, l) come by ordinary loads meanwhile.
+          asm volatile("fence.proxy.async;" ::: "memory");
+          if (lane == 0) mbar_arrive_expect_tx(&bars.land, (uint32_t)fan * GB * D * sizeof(float));
+          __syncwarp();
+          if (lane < fan)
+            bulk_load(land + (size_t)lane * GB * D, dv.rec_o + ((size_t)(first_rec + lane) * G + jh) * D,
+                      GB * D * sizeof(float), &bars.land);
+          float mx[GB], l[GB], cw[GB];
+#pragma unroll
+          for (int jj = 0; jj < GB; ++jj) {
+            float2 ml = make_float2(-CUDART_INF_F, 0.f);
+            if (lane < fan) ml = __ldcg(&dv.rec_ml[(size_t)(first_rec + lane) * G + jh + jj]);
+            mx[jj] = ml.x;
+            l[jj] = ml.y;
+            cw[jj] = ml.x;
+          }
+#pragma unroll
+          for (int jj = 0; jj < GB; ++jj) {
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) mx[jj] = fmaxf(mx[jj], __shfl_xor_sync(0xffffffffu, mx[jj], off));
+            const float mu = (mx[jj] == -CUDART_INF_F) ? 0.f : mx[jj];
+            cw[jj] = fast_exp2(cw[jj] - mu);
+            l[jj] *= cw[jj];
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) l[jj] += __shfl_xor_sync(0xffffffffu, l[jj], off);
+          }
+          if (!warp_wait(&bars.land, land_uses & 1)) { ok = false; return; }
+          ++land_uses;
+#pragma unroll
+          for (int jj = 0; jj < GB; ++jj) {
+            LaneVec<D> sum;
+            sum.zero();
+#pragma unroll
+            for (int r = 0; r < F; ++r) {
+              const float cr = __shfl_sync(0xffffffffu, cw[jj], r);
+              if (r < fan) {
+                LaneVec<D> o;
+                o.load_shared(land + ((size_t)r * GB + jj) * D, lane);
+                sum.fma(cr, o);
+              }
+            }
+            if (n_next == 1) {
+              sum.scale(l[jj] > 0.f ? 1.f / l[jj] : 0.f);
+              sum.store(out_rows + (size_t)(jh + jj) * D, lane);
+            } else {
+              const size_t r = (size_t)(rec_off + n + node) * G + jh + jj;
+              if (lane == 0) dv.rec_ml[r] = make_float2(mx[jj], l[jj]);
+              sum.store(dv.rec_o + r * D, lane);
+            }
+          }
+          __syncwarp();   // every lane is done with the landing zone before the next copies are issued
+        }
+        if (n_next == 1) return;
+        rec_off += n;
+        tk_off += n_next;
+        idx = node;
+        n = n_next;
+        __threadfence();
+        __syncwarp();
+        ticket = 0;
+        if (lane == 0) ticket = atomicAdd(&dv.tickets[tk_off + idx / F], 1);
+        ticket = __shfl_sync(0xffffffffu, ticket, 0);
+      }
+    };
+
+    // The arrival count of a part's record is asked for right after the record is written, but looked at
+    // only after the next item has been reduced, so its round trip overlaps useful work.
+    bool pend = false;
+    int pend_ticket = 0, pend_idx = 0, pend_n = 0, pend_rec = 0, pend_tk = 0;
+    float* pend_out = nullptr;
+    auto resolve = [&]() {
+      if (!pend) return;
+      pend = false;
+      climb(__shfl_sync(0xffffffffu, pend_ticket, 0), pend_idx, pend_n, pend_rec, pend_tk, pend_out);
+    };
+
+    for (unsigned seq = 0; ok; ++seq) {
       const int mb = seq % kMergeBufs;
       if (!warp_wait(&bars.merge_full[mb], (seq / kMergeBufs) & 1)) { ok = false; break; }
       const MBuf& M = mbufs[mb];
@@ -753,68 +895,27 @@ decode_kernel(DeviceView dv, int layer, int n_items, const T* __restrict__ q, fl
           acc[j].scale(l_tot[j] > 0.f ? 1.f / l_tot[j] : 0.f);
           acc[j].store(out_rows + (size_t)j * D, lane);
         }
+        resolve();
         continue;
       }
-      // This part's record, then up the head's combine tree for as long as this warp closes the nodes.
-      int idx = d.part_idx, n = d.n_parts, rec_off = d.rec_base, tk_off = d.ticket_base;
+      // This part's record and its arrival at the level-0 node.
 #pragma unroll
       for (int j = 0; j < G; ++j) {
-        const size_t r = (size_t)(rec_off + idx) * G + j;
+        const size_t r = (size_t)(d.rec_base + d.part_idx) * G + j;
         if (lane == 0) dv.rec_ml[r] = make_float2(m_tot[j], l_tot[j]);
         acc[j].store(dv.rec_o + r * D, lane);
       }
-      for (;;) {
-        const int n_next = (n + F - 1) / F, node = idx / F;
-        const int fan = min(F, n - node * F);
-        __threadfence();
-        __syncwarp();
-        int ticket = 0;
-        if (lane == 0) ticket = atomicAdd(&dv.tickets[tk_off + node], 1);
-        ticket = __shfl_sync(0xffffffffu, ticket, 0);
-        if (ticket != fan - 1) break;
-        // Last input of this node: merge its `fan` records (read through L2).
-        __threadfence();
-        if (lane == 0) dv.tickets[tk_off + node] = 0;
-        const int first_rec = rec_off + node * F;
-#pragma unroll 1
-        for (int j = 0; j < G; ++j) {
-          float2 ml = make_float2(-CUDART_INF_F, 0.f);
-          if (lane < fan) ml = __ldcg(&dv.rec_ml[(size_t)(first_rec + lane) * G + j]);
-          float mx = ml.x;
-#pragma unroll
-          for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
-          const float mu = (mx == -CUDART_INF_F) ? 0.f : mx;
-          const float cw = fast_exp2(ml.x - mu);
-          float l = ml.y * cw;
-#pragma unroll
-          for (int off = 16; off > 0; off >>= 1) l += __shfl_xor_sync(0xffffffffu, l, off);
-          LaneVec<D> sum;
-          sum.zero();
-#pragma unroll
-          for (int r = 0; r < F; ++r) {
-            const float cr = __shfl_sync(0xffffffffu, cw, r);
-            if (r < fan) {
-              LaneVec<D> o;
-              o.load_l2(dv.rec_o + ((size_t)(first_rec + r) * G + j) * D, lane);
-              sum.fma(cr, o);
-            }
-          }
-          if (n_next == 1) {
-            sum.scale(l > 0.f ? 1.f / l : 0.f);
-            sum.store(out_rows + (size_t)j * D, lane);
-          } else {
-            const size_t r = (size_t)(rec_off + n + node) * G + j;
-            if (lane == 0) dv.rec_ml[r] = make_float2(mx, l);
-            sum.store(dv.rec_o + r * D, lane);
-          }
-        }
-        if (n_next == 1) break;
-        rec_off += n;
-        tk_off += n_next;
-        idx = node;
-        n = n_next;
-      }
+      __threadfence();
+      __syncwarp();
+      int ticket_raw = 0;
+      if (lane == 0) ticket_raw = atomicAdd(&dv.tickets[d.ticket_base + d.part_idx / F], 1);
+      resolve();   // the previous part's count has had this item's time to arrive
+      pend = true;
+      pend_ticket = ticket_raw;
+      pend_idx = d.part_idx; pend_n = d.n_parts; pend_rec = d.rec_base; pend_tk = d.ticket_base;
+      pend_out = out_rows;
     }
+    if (ok) resolve();
     if (!ok && lane == 0) atomicOr(dv.status, kStatusReducerTimeout);
   }
 }
