@@ -204,6 +204,35 @@ RAZOR_API int razor_cache_set_option(razor_cache_t* cache, int32_t option, int32
  */
 RAZOR_API int razor_cache_device_status(razor_cache_t* cache, int32_t* status, void* stream);
 
+/*
+ * The compensation token of the KV heads of ONE sequence without a cache, a pool or a workspace.
+ * (The paper has no counterpart to this call; it computes the same means as Eq. 4.)
+ *
+ * For callers that cannot allocate device memory: a plugin inside an application that owns the
+ * allocator and passes in only input and output tensors, code running while a stream is being
+ * captured, a process whose memory was fixed at start-up.  They cannot set up razor_cache_create's
+ * buffers, yet the means of the dropped rows need a cross-block reduction and so some scratch.  Here
+ * that scratch is a fixed 2 MiB array inside the library itself (each GPU that loads the library
+ * holds it until the process ends); the call allocates nothing and frees nothing.
+ *
+ *   K, V       device, [n_kv_heads, >= ctx_len, head_dim] with element strides stride_h / stride_n,
+ *              16-byte aligned like razor_compress's inputs; dtype RAZOR_F32 or RAZOR_BF16
+ *   mean_k/v   device fp32 [n_kv_heads, head_dim]: means over rows [n_sink, ctx_len - window);
+ *              zeros when ctx_len <= n_sink + window
+ *   n_drop     host, may be NULL: number of rows averaged
+ * Limits: n_kv_heads <= 64 (RAZOR_E_CAPACITY beyond that: split the heads over several calls),
+ * head_dim 64 or 128.
+ * The first call on a device looks up the array's device address; make that call outside any stream
+ * capture.  All calls on a device share the array, so two calls whose kernels could run at the same
+ * time (different streams, no ordering between them) corrupt each other: keep them stream-ordered.
+ * Nothing in the array needs clearing between calls.
+ * Errors: NULL_PTR, INVALID_ARG, CAPACITY, UNSUPPORTED_DIM, MISALIGNED, CUDA.
+ */
+RAZOR_API int razor_compensation_mean_static(const void* K, const void* V, int64_t stride_h, int64_t stride_n,
+                                   int32_t n_kv_heads, int32_t head_dim, int32_t dtype, int32_t ctx_len,
+                                   int32_t n_sink, int32_t window, float* mean_k, float* mean_v, int32_t* n_drop,
+                                   void* stream);
+
 /* Forget every compressed layer and give all pages back (the handle and buffers stay usable). */
 RAZOR_API int razor_cache_reset(razor_cache_t* cache);
 

@@ -27,7 +27,8 @@ STATUS = {
 SYMBOLS = [
     "razor_query_bytes", "razor_cache_create", "razor_compress", "razor_compress_seq", "razor_append",
     "razor_decode_attention", "razor_cache_export", "razor_cache_stats", "razor_schedule_plan",
-    "razor_schedule_query", "razor_cache_set_option", "razor_cache_device_status", "razor_cache_reset", "razor_cache_destroy", "razor_status_string",
+    "razor_schedule_query", "razor_cache_set_option", "razor_cache_device_status", "razor_compensation_mean_static",
+    "razor_cache_reset", "razor_cache_destroy", "razor_status_string",
     "razor_last_cuda_error", "razor_version",
 ]
 
@@ -77,6 +78,8 @@ def load() -> C.CDLL:
     lib.razor_cache_set_option.argtypes = [vp, i32, i32]
     lib.razor_cache_device_status.argtypes = [vp, C.POINTER(i32), vp]
     lib.razor_schedule_query.argtypes = [vp, i32, vp, i32, C.POINTER(i32)]
+    lib.razor_compensation_mean_static.argtypes = [vp, vp, i64, i64, i32, i32, i32, i32, i32, i32, vp, vp,
+                                                   C.POINTER(i32), vp]
     lib.razor_cache_reset.argtypes = [vp]
     lib.razor_cache_destroy.argtypes = [vp]
     lib.razor_status_string.argtypes = [C.c_int]
@@ -228,6 +231,17 @@ def razor_schedule_query(cache: int, layer: int) -> np.ndarray:
     items = np.zeros((n.value, 4), dtype=np.int32)
     _check(lib.razor_schedule_query(cache, layer, items.ctypes.data, n.value, C.byref(n)), "razor_schedule_query")
     return items
+
+
+def razor_compensation_mean_static(K, V, stride_h: int, stride_n: int, n_kv_heads: int, head_dim: int, dtype: int,
+                                   ctx_len: int, n_sink: int, window: int, mean_k, mean_v, stream=None) -> int:
+    """Means of the dropped K and V rows of one sequence's heads, using only the library's built-in
+    scratch array (no pool, no workspace, no allocation).  -> number of rows averaged."""
+    nd = C.c_int32(0)
+    _check(load().razor_compensation_mean_static(_ptr(K), _ptr(V), stride_h, stride_n, n_kv_heads, head_dim, dtype,
+                                                 ctx_len, n_sink, window, _ptr(mean_k), _ptr(mean_v), C.byref(nd),
+                                                 _stream(stream)), "razor_compensation_mean_static")
+    return nd.value
 
 
 def razor_cache_reset(cache: int) -> None:
