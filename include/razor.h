@@ -162,20 +162,23 @@ RAZOR_API int razor_cache_export(razor_cache_t* cache, int32_t layer, int32_t b,
 RAZOR_API int razor_cache_stats(const razor_cache_t* cache, int32_t layer, size_t* kept_bytes, size_t* dense_bytes);
 
 /*
- * The decode work schedule (host only; no device is touched).  Every (sequence, KV head) token
- * stream is cut into page ranges of near-equal size (work items) so that one launch is balanced over
- * the SMs whatever the mix of full-length and short heads.  A range is at most
- * max(min_chunk_pages, ceil(total_pages / target_items)) pages; heads cut into the most parts come
- * first, longer ranges before shorter ones.
+ * The decode work schedule (host only; no device is touched).  The page streams of all (sequence,
+ * KV head) pairs are laid end to end, longest first.  The first static_percent of the pages is cut
+ * into one equal span per CTA (a span that crosses a head boundary becomes several work items, one
+ * per head); the rest is cut into small tail items, about tail_items_per_cta per CTA, which the CTAs
+ * pull one by one when their span is done.  A job is what a CTA pulls: a span or one tail item.
  *   razor_schedule_plan   plans for given stream lengths: tokens host int32[n_heads] (tokens stored
- *                         per head), target_items >= 1, min_chunk_pages >= 1.
+ *                         per head), n_ctas >= 1 (the SM count), 0 <= static_percent <= 100,
+ *                         tail_items_per_cta >= 1, min_chunk_pages >= 1 (smallest span / tail item).
  *   razor_schedule_query  the plan the next razor_decode_attention of `layer` would use.
- * items: host int32[max_items][4] = {head index b*Hkv + kv_head, first_page, end_page (-1: to the
- * end of the stream), parts_of_this_head}, may be NULL; n_items receives the count.  A page is 16 tokens.
+ * items: host int32[max_items][5] = {head index b*Hkv + kv_head, first_page, end_page (-1: to the
+ * end of the stream), parts_of_this_head, job}, in job order, may be NULL; n_items receives the
+ * count, n_spans (may be NULL) how many of the jobs are spans.  A page is 16 tokens.
  * Errors: NULL_PTR, INVALID_ARG (also when max_items is too small), NOT_COMPRESSED.
  */
-RAZOR_API int razor_schedule_plan(const int32_t* tokens, int32_t n_heads, int32_t target_items,
-                        int32_t min_chunk_pages, int32_t* items, int32_t max_items, int32_t* n_items);
+RAZOR_API int razor_schedule_plan(const int32_t* tokens, int32_t n_heads, int32_t n_ctas, int32_t static_percent,
+                        int32_t tail_items_per_cta, int32_t min_chunk_pages, int32_t* items, int32_t max_items,
+                        int32_t* n_items, int32_t* n_spans);
 RAZOR_API int razor_schedule_query(razor_cache_t* cache, int32_t layer, int32_t* items, int32_t max_items,
                          int32_t* n_items);
 
@@ -184,13 +187,15 @@ RAZOR_API int razor_schedule_query(razor_cache_t* cache, int32_t layer, int32_t*
  * next razor_decode_attention.  Errors: NULL_PTR, INVALID_ARG (unknown option or value out of range).
  */
 enum {
-  RAZOR_OPT_DECODE_ITEMS_PER_SM = 1,    /* work items aimed for per SM (1..1024; default 16)              */
-  RAZOR_OPT_DECODE_MIN_CHUNK_PAGES = 2, /* smallest work item in pages (default 8)                        */
+  RAZOR_OPT_DECODE_TAIL_ITEMS_PER_SM = 1, /* tail items aimed for per SM (1..1024; default 4)             */
+  RAZOR_OPT_DECODE_MIN_CHUNK_PAGES = 2, /* smallest span or tail item in pages (default 8)                */
   RAZOR_OPT_DECODE_RING_KB = 3,         /* shared-memory page ring per CTA in KiB; 0 = as large as fits   */
   RAZOR_OPT_DECODE_CONSUMER_WARPS = 4,  /* streaming warps per CTA: 0 = default; 4, 8, 12 or 16; a value
                                            the head shape has no kernel for falls back to the default     */
-  RAZOR_OPT_DECODE_TENSOR_CORES = 5     /* bf16 grouped-query heads: 0 = matrix instructions from group 4
+  RAZOR_OPT_DECODE_TENSOR_CORES = 5,    /* bf16 grouped-query heads: 0 = matrix instructions from group 4
                                            up (default), 1 = from group 2 up, 2 = never                   */
+  RAZOR_OPT_DECODE_STATIC_PERCENT = 6   /* share of the pages handed out as per-CTA spans (0..100;
+                                           default 85); 0 makes every job a tail item                     */
 };
 RAZOR_API int razor_cache_set_option(razor_cache_t* cache, int32_t option, int32_t value);
 

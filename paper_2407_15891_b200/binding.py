@@ -74,7 +74,7 @@ def load() -> C.CDLL:
     lib.razor_cache_export.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, C.POINTER(i32),
                                        C.POINTER(i32), vp]
     lib.razor_cache_stats.argtypes = [vp, i32, C.POINTER(sz), C.POINTER(sz)]
-    lib.razor_schedule_plan.argtypes = [vp, i32, i32, i32, vp, i32, C.POINTER(i32)]
+    lib.razor_schedule_plan.argtypes = [vp, i32, i32, i32, i32, i32, vp, i32, C.POINTER(i32), C.POINTER(i32)]
     lib.razor_cache_set_option.argtypes = [vp, i32, i32]
     lib.razor_cache_device_status.argtypes = [vp, C.POINTER(i32), vp]
     lib.razor_schedule_query.argtypes = [vp, i32, vp, i32, C.POINTER(i32)]
@@ -196,21 +196,22 @@ def razor_cache_stats(cache: int, layer: int) -> Tuple[int, int]:
     return k.value, d.value
 
 
-def razor_schedule_plan(tokens, target_items: int, min_chunk_pages: int = 1) -> np.ndarray:
-    """Host-only: -> int32 [n_items, 4] = (head, first_page, end_page (-1: open), parts_of_head)."""
+def razor_schedule_plan(tokens, n_ctas: int = 148, static_percent: int = 85, tail_items_per_cta: int = 4,
+                        min_chunk_pages: int = 8, with_spans: bool = False):
+    """Host-only: -> int32 [n_items, 5] = (head, first_page, end_page (-1: open), parts_of_head, job) in job
+    order (and the number of span jobs when with_spans is set)."""
     t = _i32(tokens)
-    n = C.c_int32(0)
+    n, ns = C.c_int32(0), C.c_int32(0)
     lib = load()
-    _check(lib.razor_schedule_plan(t.ctypes.data, len(t), target_items, min_chunk_pages, None, 0, C.byref(n)),
-           "razor_schedule_plan")
-    items = np.zeros((n.value, 4), dtype=np.int32)
-    _check(lib.razor_schedule_plan(t.ctypes.data, len(t), target_items, min_chunk_pages, items.ctypes.data, n.value,
-                                   C.byref(n)), "razor_schedule_plan")
-    return items
+    args = (t.ctypes.data, len(t), n_ctas, static_percent, tail_items_per_cta, min_chunk_pages)
+    _check(lib.razor_schedule_plan(*args, None, 0, C.byref(n), C.byref(ns)), "razor_schedule_plan")
+    items = np.zeros((n.value, 5), dtype=np.int32)
+    _check(lib.razor_schedule_plan(*args, items.ctypes.data, n.value, C.byref(n), C.byref(ns)), "razor_schedule_plan")
+    return (items, ns.value) if with_spans else items
 
 
-OPT_DECODE_ITEMS_PER_SM, OPT_DECODE_MIN_CHUNK_PAGES, OPT_DECODE_RING_KB, OPT_DECODE_CONSUMER_WARPS = 1, 2, 3, 4
-OPT_DECODE_TENSOR_CORES = 5
+OPT_DECODE_TAIL_ITEMS_PER_SM, OPT_DECODE_MIN_CHUNK_PAGES, OPT_DECODE_RING_KB, OPT_DECODE_CONSUMER_WARPS = 1, 2, 3, 4
+OPT_DECODE_TENSOR_CORES, OPT_DECODE_STATIC_PERCENT = 5, 6
 
 
 def razor_cache_set_option(cache: int, option: int, value: int) -> None:
@@ -228,7 +229,7 @@ def razor_schedule_query(cache: int, layer: int) -> np.ndarray:
     n = C.c_int32(0)
     lib = load()
     _check(lib.razor_schedule_query(cache, layer, None, 0, C.byref(n)), "razor_schedule_query")
-    items = np.zeros((n.value, 4), dtype=np.int32)
+    items = np.zeros((n.value, 5), dtype=np.int32)
     _check(lib.razor_schedule_query(cache, layer, items.ctypes.data, n.value, C.byref(n)), "razor_schedule_query")
     return items
 

@@ -33,7 +33,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 inline int ceil_div(long long a, long long b) { return (int)((a + b - 1) / b); }
 
 struct Layout {
-  size_t state, comp_sum, comp_mean, page_table, items, rec_ml, rec_o, tickets, queue, scratch, seq_desc, total;
+  size_t state, comp_sum, comp_mean, page_table, items, jobs, rec_ml, rec_o, tickets, queue, scratch, seq_desc, total;
   int max_pages, max_items, max_recs, max_tickets;
 };
 
@@ -73,6 +73,7 @@ Layout make_layout(const razor_config_t& c) {
   l.comp_mean = take(L * nh * 2 * D * sizeof(float));
   l.page_table = take(L * nh * (size_t)l.max_pages * sizeof(int32_t));
   l.items = take(L * (size_t)l.max_items * sizeof(WorkItem));
+  l.jobs = take(L * ((size_t)l.max_items + 1) * sizeof(int32_t));
   l.rec_ml = take((size_t)l.max_recs * g * sizeof(float2));
   l.rec_o = take((size_t)l.max_recs * g * D * sizeof(float));
   l.tickets = take((size_t)l.max_tickets * sizeof(int32_t));
@@ -99,8 +100,9 @@ struct LayerHost {
   int appended = 0;
   // decode schedule
   bool sched_valid = false;
-  int n_items = 0, chunk_pages = 0, growth_tokens = 0;
+  int n_items = 0, n_jobs = 0, n_spans = 0, chunk_pages = 0, growth_tokens = 0;
   WorkItem* items = nullptr;        // pinned host, [max_items]
+  int32_t* jobs = nullptr;          // pinned host, [max_items + 1]
   cudaEvent_t upload_done = nullptr;
 };
 
@@ -119,9 +121,10 @@ struct razor_cache {
   DeviceView dv;
   long long pool_pages = 0, next_page = 0;
   int n_sms = 148;
-  DecodeTuning tune{16, 8, 0, 0, 0};
+  DecodeTuning tune{4, 85, 8, 0, 0, 0};
   std::vector<LayerHost> layers;
   WorkItem* pinned_items = nullptr;   // [L][max_items]
+  int32_t* pinned_jobs = nullptr;     // [L][max_items + 1]
 };
 
 extern "C" {
@@ -197,6 +200,7 @@ int razor_cache_create(razor_cache_t** out, const razor_config_t* cfg, void* poo
   dv.comp_mean = (float*)(ws + lay.comp_mean);
   dv.page_table = (int32_t*)(ws + lay.page_table);
   dv.items = (WorkItem*)(ws + lay.items);
+  dv.jobs = (int32_t*)(ws + lay.jobs);
   dv.rec_ml = (float2*)(ws + lay.rec_ml);
   dv.rec_o = (float*)(ws + lay.rec_o);
   dv.tickets = (int32_t*)(ws + lay.tickets);
@@ -221,9 +225,14 @@ int razor_cache_create(razor_cache_t** out, const razor_config_t* cfg, void* poo
   if (e == cudaSuccess)
     e = cudaHostAlloc((void**)&c->pinned_items, (size_t)cfg->n_layers * lay.max_items * sizeof(WorkItem),
                       cudaHostAllocDefault);
+  if (e == cudaSuccess)
+    e = cudaHostAlloc((void**)&c->pinned_jobs, (size_t)cfg->n_layers * (lay.max_items + 1) * sizeof(int32_t),
+                      cudaHostAllocDefault);
   if (e != cudaSuccess) {
     g_last_cuda_error = (int)e;
     (void)cudaGetLastError();
+    if (c->pinned_items) cudaFreeHost(c->pinned_items);
+  if (c->pinned_jobs) cudaFreeHost(c->pinned_jobs);
     delete c;
     return RAZOR_E_CUDA;
   }
@@ -236,6 +245,7 @@ int razor_cache_create(razor_cache_t** out, const razor_config_t* cfg, void* poo
     L.region_start.assign(cfg->batch, 0);
     L.region_count.assign(cfg->batch, 0);
     L.items = c->pinned_items + (size_t)l * lay.max_items;
+    L.jobs = c->pinned_jobs + (size_t)l * (lay.max_items + 1);
   }
   *out = c;
   return RAZOR_OK;
@@ -261,6 +271,7 @@ int razor_cache_destroy(razor_cache_t* c) {
   for (LayerHost& L : c->layers)
     if (L.upload_done) cudaEventDestroy(L.upload_done);
   if (c->pinned_items) cudaFreeHost(c->pinned_items);
+  if (c->pinned_jobs) cudaFreeHost(c->pinned_jobs);
   delete c;
   return RAZOR_OK;
 }
@@ -396,15 +407,22 @@ int ensure_schedule(razor_cache* c, int layer, cudaStream_t stream, bool upload)
   std::vector<int32_t> pages(nh);
   for (int h = 0; h < nh; ++h) pages[h] = ceil_div(L.hs[h].len, kPageTokens);
   if (L.upload_done) RZ_CUDA(cudaEventSynchronize(L.upload_done));   // previous upload has left the staging area
-  const int n = build_schedule(pages.data(), nh, c->n_sms * c->tune.items_per_sm, c->tune.min_chunk_pages,
-                               c->lay.max_items, c->lay.max_recs, c->lay.max_tickets, L.items, &L.chunk_pages);
+  const SchedParams sp{c->n_sms, c->tune.static_pct, c->tune.tail_items_per_sm, c->tune.min_chunk_pages};
+  SchedInfo info{};
+  const int n = build_schedule(pages.data(), nh, sp, c->lay.max_items, c->lay.max_recs, c->lay.max_tickets, L.items,
+                               L.jobs, &info);
   if (n < 0) return RAZOR_E_INVALID_ARG;
   L.n_items = n;
+  L.n_jobs = info.n_jobs;
+  L.n_spans = info.n_spans;
+  L.chunk_pages = info.chunk_pages;
   L.growth_tokens = 0;
   if (upload) {
     if (!L.upload_done) RZ_CUDA(cudaEventCreateWithFlags(&L.upload_done, cudaEventDisableTiming));
     RZ_CUDA(cudaMemcpyAsync(c->dv.items + (size_t)layer * c->lay.max_items, L.items, (size_t)n * sizeof(WorkItem),
                             cudaMemcpyHostToDevice, stream));
+    RZ_CUDA(cudaMemcpyAsync(c->dv.jobs + (size_t)layer * (c->lay.max_items + 1), L.jobs,
+                            (size_t)(L.n_jobs + 1) * sizeof(int32_t), cudaMemcpyHostToDevice, stream));
     RZ_CUDA(cudaEventRecord(L.upload_done, stream));
     L.sched_valid = true;
   } else {
@@ -420,15 +438,19 @@ inline int layer_ready(const razor_cache* c, int layer) {
   return RAZOR_OK;
 }
 
-int emit_items(const WorkItem* w, int n, int32_t* items, int32_t max_items, int32_t* n_items) {
+int emit_items(const WorkItem* w, int n, const int32_t* jobs, int n_jobs, int32_t* items, int32_t max_items,
+               int32_t* n_items) {
   *n_items = n;
   if (!items) return RAZOR_OK;
   if (max_items < n) return RAZOR_E_INVALID_ARG;
+  int job = 0;
   for (int i = 0; i < n; ++i) {
-    items[4 * i + 0] = w[i].head;
-    items[4 * i + 1] = w[i].page_begin;
-    items[4 * i + 2] = w[i].page_end;
-    items[4 * i + 3] = w[i].n_parts;
+    while (job + 1 < n_jobs && jobs[job + 1] <= i) ++job;
+    items[5 * i + 0] = w[i].head;
+    items[5 * i + 1] = w[i].page_begin;
+    items[5 * i + 2] = w[i].page_end;
+    items[5 * i + 3] = w[i].n_parts;
+    items[5 * i + 4] = job;
   }
   return RAZOR_OK;
 }
@@ -500,7 +522,9 @@ int razor_decode_attention(razor_cache_t* c, int32_t layer, const void* q, float
   if (((uintptr_t)q | (uintptr_t)out) & 15) return RAZOR_E_MISALIGNED;
   rc = ensure_schedule(c, layer, (cudaStream_t)stream, true);
   if (rc) return rc;
-  RZ_CUDA(launch_decode(c->dv, c->cfg.dtype, layer, c->layers[layer].n_items, q, out, c->n_sms, c->tune,
+  const LayerHost& L = c->layers[layer];
+  const DecodeJobs jb{L.n_items, L.n_jobs, L.n_spans, L.jobs[L.n_spans]};
+  RZ_CUDA(launch_decode(c->dv, c->cfg.dtype, layer, jb, q, out, c->n_sms, c->tune,
                         (cudaStream_t)stream));
   return RAZOR_OK;
 }
@@ -541,10 +565,13 @@ int razor_cache_stats(const razor_cache_t* c, int32_t layer, size_t* kept_bytes,
   return RAZOR_OK;
 }
 
-int razor_schedule_plan(const int32_t* tokens, int32_t n_heads, int32_t target_items, int32_t min_chunk_pages,
-                        int32_t* items, int32_t max_items, int32_t* n_items) {
+int razor_schedule_plan(const int32_t* tokens, int32_t n_heads, int32_t n_ctas, int32_t static_percent,
+                        int32_t tail_items_per_cta, int32_t min_chunk_pages, int32_t* items, int32_t max_items,
+                        int32_t* n_items, int32_t* n_spans) {
   if (!tokens || !n_items) return RAZOR_E_NULL_PTR;
-  if (n_heads < 1 || target_items < 1 || min_chunk_pages < 1) return RAZOR_E_INVALID_ARG;
+  if (n_heads < 1 || n_ctas < 1 || static_percent < 0 || static_percent > 100 || tail_items_per_cta < 1 ||
+      min_chunk_pages < 1)
+    return RAZOR_E_INVALID_ARG;
   std::vector<int32_t> pages(n_heads);
   for (int h = 0; h < n_heads; ++h) {
     if (tokens[h] < 0) return RAZOR_E_INVALID_ARG;
@@ -552,19 +579,26 @@ int razor_schedule_plan(const int32_t* tokens, int32_t n_heads, int32_t target_i
   }
   const int cap = n_heads + kItemBudget;
   std::vector<WorkItem> w(cap);
-  int chunk = 0;
-  const int n = build_schedule(pages.data(), n_heads, target_items, min_chunk_pages, cap, 2 * cap + kMaxTreeLevels * n_heads,
-                               cap + kMaxTreeLevels * n_heads, w.data(), &chunk);
+  std::vector<int32_t> jobs(cap + 1);
+  const SchedParams sp{n_ctas, static_percent, tail_items_per_cta, min_chunk_pages};
+  SchedInfo info{};
+  const int n = build_schedule(pages.data(), n_heads, sp, cap, 2 * cap + kMaxTreeLevels * n_heads,
+                               cap + kMaxTreeLevels * n_heads, w.data(), jobs.data(), &info);
   if (n < 0) return RAZOR_E_INVALID_ARG;
-  return emit_items(w.data(), n, items, max_items, n_items);
+  if (n_spans) *n_spans = info.n_spans;
+  return emit_items(w.data(), n, jobs.data(), info.n_jobs, items, max_items, n_items);
 }
 
 int razor_cache_set_option(razor_cache_t* c, int32_t option, int32_t value) {
   if (!c) return RAZOR_E_NULL_PTR;
   switch (option) {
-    case RAZOR_OPT_DECODE_ITEMS_PER_SM:
+    case RAZOR_OPT_DECODE_TAIL_ITEMS_PER_SM:
       if (value < 1 || value > 1024) return RAZOR_E_INVALID_ARG;
-      c->tune.items_per_sm = value;
+      c->tune.tail_items_per_sm = value;
+      break;
+    case RAZOR_OPT_DECODE_STATIC_PERCENT:
+      if (value < 0 || value > 100) return RAZOR_E_INVALID_ARG;
+      c->tune.static_pct = value;
       break;
     case RAZOR_OPT_DECODE_MIN_CHUNK_PAGES:
       if (value < 1 || value > (1 << 20)) return RAZOR_E_INVALID_ARG;
@@ -610,7 +644,8 @@ int razor_schedule_query(razor_cache_t* c, int32_t layer, int32_t* items, int32_
   if (rc) return rc;
   rc = ensure_schedule(c, layer, nullptr, false);
   if (rc) return rc;
-  return emit_items(c->layers[layer].items, c->layers[layer].n_items, items, max_items, n_items);
+  const LayerHost& L = c->layers[layer];
+  return emit_items(L.items, L.n_items, L.jobs, L.n_jobs, items, max_items, n_items);
 }
 
 }  // extern "C"

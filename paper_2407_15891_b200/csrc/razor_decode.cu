@@ -32,8 +32,12 @@ namespace razor {
 
 namespace {
 
-constexpr int kItemSlots = 4;            // item descriptors in flight between producer and consumers
-constexpr int kMergeBufs = 2;            // consumer -> reducer hand-over buffers
+constexpr int kItemSlots = 2;            // item descriptors in flight between producer and consumers
+constexpr int kMaxMergeBufs = 2;         // consumer -> reducer hand-over buffers (one where they are large)
+template <int G>
+constexpr int merge_bufs() { return G >= 4 ? 1 : 2; }
+template <int G>
+constexpr int land_heads() { return G < 2 ? G : 2; }   // query heads whose rows land together in a merge
 constexpr int kMaxStages = 64;           // ring stages (pages in flight per CTA)
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s: far beyond any healthy wait
 
@@ -96,6 +100,19 @@ __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t b
                : "memory");
 }
 
+// Ring position -> (stage, use).  Position p is always consumed by warp p % NC, and a stage must always
+// be consumed by the same warp: a warp then never waits on a barrier that is more than one phase behind
+// it, which a parity wait could not tell from "done".  So the ring is NC interleaved sub-rings: warp w
+// owns stages w, w + NC, w + 2 NC, ... below n_stages (the sub-rings differ in length by at most one
+// when n_stages is not a multiple of NC) and walks them round-robin.
+template <int NC>
+__device__ __forceinline__ void ring_slot(unsigned pos, unsigned n_stages, unsigned& stage, unsigned& use) {
+  const unsigned w = pos % NC, k = pos / NC;
+  const unsigned cnt = (n_stages - w + NC - 1) / NC;   // stages of warp w's sub-ring (n_stages >= NC)
+  stage = w + NC * (k % cnt);
+  use = k / cnt;
+}
+
 // ------------------------------------------------------------------------------------------ shared layout
 struct ItemDesc {
   int32_t head;        // < 0: no more items
@@ -123,8 +140,8 @@ struct Barriers {
   uint64_t empty[kMaxStages];
   uint64_t item_full[kItemSlots];
   uint64_t item_empty[kItemSlots];
-  uint64_t merge_full[kMergeBufs];
-  uint64_t merge_free[kMergeBufs];
+  uint64_t merge_full[kMaxMergeBufs];
+  uint64_t merge_free[kMaxMergeBufs];
   uint64_t land;   // landing zone of the combine-tree merges
 };
 
@@ -137,14 +154,14 @@ struct alignas(16) MergeBuf {
 };
 
 // Dynamic shared memory: the hand-over buffers, the landing zone of the combine-tree merges
-// (kMergeFanIn records x up to 4 heads x D floats), then the page ring (1 KiB aligned).
+// (kMergeFanIn records x up to 2 heads x D floats), then the page ring (1 KiB aligned).
 template <typename T, int D, int G, int NC>
 constexpr size_t decode_land_offset() {
-  return (sizeof(MergeBuf<D, G, NC>) * kMergeBufs + 127) & ~(size_t)127;
+  return (sizeof(MergeBuf<D, G, NC>) * merge_bufs<G>() + 127) & ~(size_t)127;
 }
 template <typename T, int D, int G, int NC>
 constexpr size_t decode_ring_offset() {
-  return (decode_land_offset<T, D, G, NC>() + (size_t)kMergeFanIn * (G < 4 ? G : 4) * D * sizeof(float) + 1023) &
+  return (decode_land_offset<T, D, G, NC>() + (size_t)kMergeFanIn * land_heads<G>() * D * sizeof(float) + 1023) &
          ~(size_t)1023;
 }
 
@@ -399,7 +416,7 @@ struct LaneVec<64> {
 // ------------------------------------------------------------------------------------------ the kernel
 template <typename T, int D, int G, int NC, bool MMA>
 __global__ void __launch_bounds__((NC + 2) * 32, 1)
-decode_kernel(DeviceView dv, int layer, int n_items, const T* __restrict__ q, float* __restrict__ out, int n_stages) {
+decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, float* __restrict__ out, int n_stages) {
   static_assert(!MMA || (sizeof(T) == 2 && G >= 2), "the tensor-core path is for grouped bf16 heads");
   using Geo = RowGeom<T, D>;
   constexpr int LPR = Geo::kLpr, EPL = Geo::kEpl;
@@ -407,6 +424,7 @@ decode_kernel(DeviceView dv, int layer, int n_items, const T* __restrict__ q, fl
   constexpr int F = kMergeFanIn;
   using Slot = ItemSlot<T, D, G>;
   using MBuf = MergeBuf<D, G, NC>;
+  constexpr int kMergeBufs = merge_bufs<G>();
 
   extern __shared__ __align__(1024) uint8_t dyn_smem[];
   __shared__ Barriers bars;
@@ -440,6 +458,8 @@ decode_kernel(DeviceView dv, int layer, int n_items, const T* __restrict__ q, fl
   __syncthreads();
 
   const WorkItem* items = dv.items + (size_t)layer * dv.max_items;
+  const int32_t* jobs = dv.jobs + (size_t)layer * (dv.max_items + 1);
+  const int n_items = jb.n_items;
   const int n_q_heads = dv.n_kv_heads * G;
   // Warp-uniform bounded wait: false for every lane if any lane's wait failed.
   auto warp_wait = [&](uint64_t* bar, uint32_t parity) -> bool {
@@ -449,7 +469,9 @@ decode_kernel(DeviceView dv, int layer, int n_items, const T* __restrict__ q, fl
   if (warp == NC) {
     // ======================================================================== producer
     const unsigned ns = (unsigned)n_stages;
-    const int batch = n_stages < 32 ? n_stages : 32;   // pages issued per round: never more than the ring holds
+    // positions issued per round: never more than one lap of the shortest sub-ring, so that no lane of
+    // a round waits for a stage that another lane of the same round is about to fill
+    const int batch = min(32, NC * (n_stages / NC));
     unsigned c = 0;                                      // ring positions issued so far by this CTA (exact)
     unsigned seq_issued = 0;                             // item slots whose copies were issued
     int marker_slot = -1;                                // slot that received the end marker
@@ -462,16 +484,33 @@ decode_kernel(DeviceView dv, int layer, int n_items, const T* __restrict__ q, fl
     auto first_pids = [&](const WorkItem& w) {
       return dv.page_table[row_of(w) * dv.max_pages + min(w.page_begin + lane, dv.max_pages - 1)];
     };
-    int it = 0;
-    if (lane == 0) it = atomicAdd(dv.queue, 1);
-    it = __shfl_sync(0xffffffffu, it, 0);
+    // A job is a run of consecutive items: a span (looked up in jobs[]) or a single tail item (tail
+    // jobs follow the spans and map to consecutive items, so they need no lookup).
+    auto job_range = [&](int j, int& first, int& end) {
+      if (j >= jb.n_jobs) {
+        first = end = n_items;
+      } else if (j >= jb.n_spans) {
+        first = jb.tail_first + (j - jb.n_spans);
+        end = first + 1;
+      } else {
+        first = jobs[j];
+        end = jobs[j + 1];
+      }
+    };
+    int it = 0, job_end = 0;
+    {
+      int j = 0;
+      if (lane == 0) j = atomicAdd(dv.queue, 1);
+      job_range(__shfl_sync(0xffffffffu, j, 0), it, job_end);
+    }
     WorkItem w = it < n_items ? items[it] : no_item;
     HeadState st = dv.state[row_of(w)];
     int32_t pid_first = first_pids(w);
     for (unsigned seq = 0; ok; ++seq) {
       const int slot = seq % kItemSlots;
-      int next_raw = n_items;
-      if (lane == 0 && it < n_items) next_raw = atomicAdd(dv.queue, 1);   // result is picked up below
+      const bool need_pop = it < n_items && it + 1 >= job_end;   // the job ends with this item
+      int next_raw = jb.n_jobs;
+      if (lane == 0 && need_pop) next_raw = atomicAdd(dv.queue, 1);   // result is picked up below
       if (seq >= kItemSlots) ok = warp_wait(&bars.item_empty[slot], ((seq / kItemSlots) - 1) & 1);
       if (!ok) break;
       Slot& sl = slots[slot];
@@ -507,7 +546,7 @@ decode_kernel(DeviceView dv, int layer, int n_items, const T* __restrict__ q, fl
       // which CTA streamed it or on what that CTA streamed before): the item starts on a ring position
       // that is a multiple of NC, and the positions left over in its last round are passed on empty.
       const int n_pad = (n + NC - 1) / NC * NC;
-      int it_next = n_items;
+      int it_next = it + 1, end_next = job_end;   // the next item of this job, unless the job ends here
       WorkItem w_next = no_item;
       bool have_next = false;
       int32_t pid_cur = pid_first;
@@ -519,9 +558,8 @@ decode_kernel(DeviceView dv, int layer, int n_items, const T* __restrict__ q, fl
         unsigned stage = 0;
         bool ready = true;
         if (mine) {
-          const unsigned cc = c + lane;
-          stage = cc % ns;
-          const unsigned use = cc / ns;
+          unsigned use;
+          ring_slot<NC>(c + lane, ns, stage, use);
           if (use > 0) ready = mbar_wait(&bars.empty[stage], (use - 1) & 1, abort_flag);
         }
         ok = __all_sync(0xffffffffu, ready);   // all or nothing: `c` stays an exact count of issued positions
@@ -535,17 +573,18 @@ decode_kernel(DeviceView dv, int layer, int n_items, const T* __restrict__ q, fl
         c += in_batch;
         pid_cur = pid_after;
         if (!have_next) {   // the pop issued above has had a round of copies to come back
-          it_next = __shfl_sync(0xffffffffu, next_raw, 0);
+          if (need_pop) job_range(__shfl_sync(0xffffffffu, next_raw, 0), it_next, end_next);
           w_next = it_next < n_items ? items[it_next] : no_item;
           have_next = true;
         }
       }
       if (!ok) break;
       if (!have_next) {
-        it_next = __shfl_sync(0xffffffffu, next_raw, 0);
+        if (need_pop) job_range(__shfl_sync(0xffffffffu, next_raw, 0), it_next, end_next);
         w_next = it_next < n_items ? items[it_next] : no_item;
       }
       it = it_next;
+      job_end = end_next;
       w = w_next;
       st = dv.state[row_of(w)];
       pid_first = first_pids(w);
@@ -554,9 +593,13 @@ decode_kernel(DeviceView dv, int layer, int n_items, const T* __restrict__ q, fl
     // Wait (bounded) until every copy this warp issued has landed: the CTA's shared memory must not be
     // released under a copy in flight.  In a healthy run the consumers have waited for all of them already.
     bool drained = true;
-    for (unsigned s = lane; s < ns && s < c; s += 32) {
-      const unsigned last = s + ns * ((c - 1 - s) / ns);   // latest ring position that used stage s
-      if (!mbar_wait_drain(&bars.full[s], (last / ns) & 1)) drained = false;
+    for (unsigned s = lane; s < ns; s += 32) {
+      const unsigned w = s % NC, j = s / NC, cnt = (ns - w + NC - 1) / NC;
+      const unsigned kw = c > w ? (c - w + NC - 1) / NC : 0;   // positions issued so far on warp w's sub-ring
+      if (kw > j) {
+        const unsigned k_last = j + cnt * ((kw - 1 - j) / cnt);   // latest of them that used stage s
+        if (!mbar_wait_drain(&bars.full[s], (k_last / cnt) & 1)) drained = false;
+      }
     }
     // (The slot that took the end marker was first waited free, so its earlier copies have landed; its
     // barrier has since moved on a phase and must not be asked about the earlier one.)
@@ -638,7 +681,8 @@ decode_kernel(DeviceView dv, int layer, int n_items, const T* __restrict__ q, fl
 
         const int n_pad = (d.n_pages + NC - 1) / NC * NC;
         for (int i = warp; i < n_pad; i += NC) {
-          const unsigned cc = c + i, stage = cc % ns, use = cc / ns;
+          unsigned stage, use;
+          ring_slot<NC>(c + i, ns, stage, use);
           if (!warp_wait(&bars.full[stage], use & 1)) { ok = false; break; }
           if (i < d.n_pages) {
             uint8_t* page = ring + (size_t)stage * PB;
@@ -716,7 +760,8 @@ decode_kernel(DeviceView dv, int layer, int n_items, const T* __restrict__ q, fl
 
         const int n_pad = (d.n_pages + NC - 1) / NC * NC;
         for (int i = warp; i < n_pad; i += NC) {
-          const unsigned cc = c + i, stage = cc % ns, use = cc / ns;
+          unsigned stage, use;
+          ring_slot<NC>(c + i, ns, stage, use);
           if (!warp_wait(&bars.full[stage], use & 1)) { ok = false; break; }
           if (i < d.n_pages) {
             consume_page<T, D, G>((const uint4*)(ring + (size_t)stage * PB), d.len - (d.page_begin + i) * kPageTokens,
@@ -763,7 +808,7 @@ decode_kernel(DeviceView dv, int layer, int n_items, const T* __restrict__ q, fl
     bool ok = true;
     unsigned land_uses = 0;
     float* land = (float*)(dyn_smem + decode_land_offset<T, D, G, NC>());
-    constexpr int GB = G < 4 ? G : 4;   // query heads whose rows land together
+    constexpr int GB = land_heads<G>();   // query heads whose rows land together
 
     // A part's record has been written and its arrival counted (`ticket` is the count before it).  Walk up
     // the head's combine tree for as long as this warp delivers the last input of a node.
@@ -924,7 +969,7 @@ decode_kernel(DeviceView dv, int layer, int n_items, const T* __restrict__ q, fl
 constexpr int kSmemOptIn = 232448;   // 227 KiB: the most one CTA may hold on sm_100
 
 template <typename T, int D, int G, int NC, bool MMA>
-cudaError_t decode_launch(const DeviceView& dv, int layer, int n_items, const void* q, float* out, int n_sms,
+cudaError_t decode_launch(const DeviceView& dv, int layer, const DecodeJobs& jb, const void* q, float* out, int n_sms,
                           const DecodeTuning& tune, cudaStream_t s) {
   auto kern = decode_kernel<T, D, G, NC, MMA>;
   constexpr size_t PB = RowGeom<T, D>::kPageBytes;
@@ -941,10 +986,7 @@ cudaError_t decode_launch(const DeviceView& dv, int layer, int n_items, const vo
   long long stages = avail / (long long)PB;
   if (tune.ring_kb > 0) stages = std::min<long long>(stages, (long long)tune.ring_kb * 1024 / (long long)PB);
   stages = std::min<long long>(stages, kMaxStages);
-  // A stage must always be consumed by the same warp (stage % NC): a warp then never waits on a barrier
-  // that is more than one phase behind it, which a parity wait could not tell from "done".
-  stages = stages / NC * NC;
-  if (stages < NC) return cudaErrorInvalidConfiguration;
+  if (stages < NC) return cudaErrorInvalidConfiguration;   // every consumer warp owns at least one stage
   const size_t dyn = ring_off + (size_t)stages * PB;
   int dev = 0;
   if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
@@ -954,14 +996,14 @@ cudaError_t decode_launch(const DeviceView& dv, int layer, int n_items, const vo
       return e;
     if (dev >= 0 && dev < 64) opted_in[dev] = true;
   }
-  int grid = std::min(n_sms, n_items);
+  int grid = std::min(n_sms, (int)jb.n_jobs);
   if (grid < 1) grid = 1;
-  kern<<<grid, (NC + 2) * 32, dyn, s>>>(dv, layer, n_items, (const T*)q, out, (int)stages);
+  kern<<<grid, (NC + 2) * 32, dyn, s>>>(dv, layer, jb, (const T*)q, out, (int)stages);
   return cudaGetLastError();
 }
 
 template <typename T, int D, int G>
-cudaError_t decode_nc(const DeviceView& dv, int layer, int n_items, const void* q, float* out, int n_sms,
+cudaError_t decode_nc(const DeviceView& dv, int layer, const DecodeJobs& jb, const void* q, float* out, int n_sms,
                       const DecodeTuning& tune, cudaStream_t s) {
   // Consumer warps.  The ring holds a multiple of NC pages and (NC + 2) warps share the register file,
   // so the choice trades pages in flight against registers per thread.
@@ -970,43 +1012,43 @@ cudaError_t decode_nc(const DeviceView& dv, int layer, int n_items, const void* 
     // Grouped heads: the tensor-core consumer unless switched off (default on from group 4 up).
     const bool mma = tune.tensor_cores == 1 || (tune.tensor_cores == 0 && G >= 4);
     if (mma) {
-      if (nc == 4) return decode_launch<T, D, G, 4, true>(dv, layer, n_items, q, out, n_sms, tune, s);
-      return decode_launch<T, D, G, 8, true>(dv, layer, n_items, q, out, n_sms, tune, s);
+      if (nc == 4) return decode_launch<T, D, G, 4, true>(dv, layer, jb, q, out, n_sms, tune, s);
+      return decode_launch<T, D, G, 8, true>(dv, layer, jb, q, out, n_sms, tune, s);
     }
   }
   if constexpr (sizeof(T) == 2 && G == 1) {
-    if (nc == 8) return decode_launch<T, D, G, 8, false>(dv, layer, n_items, q, out, n_sms, tune, s);
-    if (nc == 16) return decode_launch<T, D, G, 16, false>(dv, layer, n_items, q, out, n_sms, tune, s);
-    return decode_launch<T, D, G, 12, false>(dv, layer, n_items, q, out, n_sms, tune, s);
+    if (nc == 8) return decode_launch<T, D, G, 8, false>(dv, layer, jb, q, out, n_sms, tune, s);
+    if (nc == 16) return decode_launch<T, D, G, 16, false>(dv, layer, jb, q, out, n_sms, tune, s);
+    return decode_launch<T, D, G, 12, false>(dv, layer, jb, q, out, n_sms, tune, s);
   } else if constexpr (sizeof(T) == 2) {
-    return decode_launch<T, D, G, 8, false>(dv, layer, n_items, q, out, n_sms, tune, s);
+    return decode_launch<T, D, G, 8, false>(dv, layer, jb, q, out, n_sms, tune, s);
   } else {
-    return decode_launch<T, D, G, 4, false>(dv, layer, n_items, q, out, n_sms, tune, s);
+    return decode_launch<T, D, G, 4, false>(dv, layer, jb, q, out, n_sms, tune, s);
   }
 }
 
 template <typename T, int D>
-cudaError_t decode_g(const DeviceView& dv, int layer, int n_items, const void* q, float* out, int n_sms,
+cudaError_t decode_g(const DeviceView& dv, int layer, const DecodeJobs& jb, const void* q, float* out, int n_sms,
                      const DecodeTuning& tune, cudaStream_t s) {
   switch (dv.group) {
-    case 1: return decode_nc<T, D, 1>(dv, layer, n_items, q, out, n_sms, tune, s);
-    case 2: return decode_nc<T, D, 2>(dv, layer, n_items, q, out, n_sms, tune, s);
-    case 4: return decode_nc<T, D, 4>(dv, layer, n_items, q, out, n_sms, tune, s);
-    case 8: return decode_nc<T, D, 8>(dv, layer, n_items, q, out, n_sms, tune, s);
+    case 1: return decode_nc<T, D, 1>(dv, layer, jb, q, out, n_sms, tune, s);
+    case 2: return decode_nc<T, D, 2>(dv, layer, jb, q, out, n_sms, tune, s);
+    case 4: return decode_nc<T, D, 4>(dv, layer, jb, q, out, n_sms, tune, s);
+    case 8: return decode_nc<T, D, 8>(dv, layer, jb, q, out, n_sms, tune, s);
   }
   return cudaErrorInvalidValue;
 }
 
 }  // namespace
 
-cudaError_t launch_decode(const DeviceView& dv, int dtype, int layer, int n_items, const void* q, float* out,
+cudaError_t launch_decode(const DeviceView& dv, int dtype, int layer, const DecodeJobs& jb, const void* q, float* out,
                           int n_sms, const DecodeTuning& tune, cudaStream_t s) {
   if (dtype == RAZOR_BF16) {
-    return dv.head_dim == 128 ? decode_g<__nv_bfloat16, 128>(dv, layer, n_items, q, out, n_sms, tune, s)
-                              : decode_g<__nv_bfloat16, 64>(dv, layer, n_items, q, out, n_sms, tune, s);
+    return dv.head_dim == 128 ? decode_g<__nv_bfloat16, 128>(dv, layer, jb, q, out, n_sms, tune, s)
+                              : decode_g<__nv_bfloat16, 64>(dv, layer, jb, q, out, n_sms, tune, s);
   }
-  return dv.head_dim == 128 ? decode_g<float, 128>(dv, layer, n_items, q, out, n_sms, tune, s)
-                            : decode_g<float, 64>(dv, layer, n_items, q, out, n_sms, tune, s);
+  return dv.head_dim == 128 ? decode_g<float, 128>(dv, layer, jb, q, out, n_sms, tune, s)
+                            : decode_g<float, 64>(dv, layer, jb, q, out, n_sms, tune, s);
 }
 
 }  // namespace razor

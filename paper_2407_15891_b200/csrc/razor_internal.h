@@ -14,8 +14,8 @@ namespace razor {
 constexpr int kPageTokens = 16;        // tokens per page
 constexpr int kMaxGroup = 8;           // query heads per KV head
 constexpr int kCompressMaxSlices = 64; // row slices per (sequence, KV head) in the compression kernel
-constexpr int kMergeFanIn = 16;        // partial records merged per node of a head's combine tree
-constexpr int kMaxTreeLevels = 6;      // 16^6 parts per head: more than any page count the config allows
+constexpr int kMergeFanIn = 32;        // partial records merged per node of a head's combine tree
+constexpr int kMaxTreeLevels = 5;      // 32^5 parts per head: more than any page count the config allows
 
 // Device-resident state of one (layer, sequence, KV head).  window < 0 marks a head that keeps every
 // token (retrieval head).  Physical slots: [0, n_sink) sinks, then the recent window as a ring whose
@@ -71,6 +71,7 @@ struct DeviceView {
   float* comp_mean;         // [L][B*Hkv][2][D]
   int32_t* page_table;      // [L][B*Hkv][max_pages]
   WorkItem* items;          // [L][max_items]
+  int32_t* jobs;            // [L][max_items + 1]  first item of every job (a span or one tail item), then n_items
   float2* rec_ml;           // [max_recs][G]      running max (log2 domain) and denominator of a partial
   float* rec_o;             // [max_recs][G][D]   un-normalised numerator of a partial
   int32_t* tickets;         // [max_tickets]      arrival counters of the combine-tree nodes (zero at rest)
@@ -94,8 +95,9 @@ struct DeviceView {
 
 // Decode launch tuning (razor_cache_set_option).
 struct DecodeTuning {
-  int32_t items_per_sm;     // work items aimed for per SM
-  int32_t min_chunk_pages;  // smallest work item
+  int32_t tail_items_per_sm;  // small items per SM that the dynamic tail of the schedule is cut into
+  int32_t static_pct;         // percent of the pages handed out as one equal span per CTA
+  int32_t min_chunk_pages;    // smallest span / tail item
   int32_t ring_kb;          // shared-memory page ring per CTA, KiB (0: as large as fits)
   int32_t consumer_warps;   // 0: default for the group size
   int32_t tensor_cores;     // grouped bf16 heads: 0 auto (group >= 4), 1 on (group >= 2), 2 off
@@ -106,17 +108,33 @@ cudaError_t launch_compress(const DeviceView& dv, int dtype, int layer, int n_se
                             cudaStream_t stream);
 cudaError_t launch_append(const DeviceView& dv, int dtype, int layer, const void* k_new, const void* v_new,
                           cudaStream_t stream);
-cudaError_t launch_decode(const DeviceView& dv, int dtype, int layer, int n_items, const void* q, float* out,
-                          int n_sms, const DecodeTuning& tune, cudaStream_t stream);
+// What a decode launch pulls from the queue: n_jobs jobs, the first n_spans of them spans (item
+// ranges jobs[j]..jobs[j+1]), the others single items starting at tail_first.
+struct DecodeJobs {
+  int32_t n_items, n_jobs, n_spans, tail_first;
+};
+cudaError_t launch_decode(const DeviceView& dv, int dtype, int layer, const DecodeJobs& jobs, const void* q,
+                          float* out, int n_sms, const DecodeTuning& tune, cudaStream_t stream);
 cudaError_t launch_export(const DeviceView& dv, int dtype, int layer, int head, int32_t* kept_pos, void* K, void* V,
                           float* mean_k, float* mean_v, float* sum_k, float* sum_v, cudaStream_t stream);
 
-// Host-only schedule builder (razor_schedule.cpp).  pages[h] = pages of head h's token stream now.
-// Cuts every head into parts of at most chunk pages, chunk = max(min_chunk, total / target_items);
-// lays out each head's partial records and ticket counters.  Returns the number of items written
-// (<= max_items), or -1 when items, records or tickets would not fit.
-int build_schedule(const int32_t* pages, int n_heads, int target_items, int min_chunk, int max_items, int max_recs,
-                   int max_tickets, WorkItem* out, int* chunk_pages_out);
+// Host-only schedule builder (razor_schedule.cpp).
+struct SchedParams {
+  int n_ctas;              // CTAs of the launch (one per SM)
+  int static_pct;          // 0..100
+  int tail_items_per_cta;  // >= 1
+  int min_chunk_pages;     // >= 1
+};
+struct SchedInfo {
+  int n_items, n_jobs, n_spans;   // the first n_spans jobs are spans
+  int span_pages, chunk_pages;    // size of a span, largest tail item
+};
+// pages[h] = pages of head h's token stream now.  Writes the work items in job order to out[] and the
+// first item of each job to jobs[] (n_jobs + 1 entries); lays out each head's partial records and
+// ticket counters.  Returns the number of items (<= max_items), or -1 when items, records or tickets
+// would not fit.
+int build_schedule(const int32_t* pages, int n_heads, const SchedParams& sp, int max_items, int max_recs,
+                   int max_tickets, WorkItem* out, int32_t* jobs, SchedInfo* info);
 
 // Records and tickets a head cut into n_parts items needs (n_parts >= 1).
 void tree_sizes(int n_parts, int* n_recs, int* n_tickets);

@@ -2,13 +2,20 @@
 //
 // The compressed cache is head-heterogeneous: a retrieval head holds the whole context, every other
 // head holds sinks + window only (Algorithm 1), and a serving batch mixes context lengths.  One
-// launch covers them all, so the token streams are cut into page ranges of near-equal size (work
-// items); the kernel's CTAs pull items from a queue and each streams its item with all of its warps.
-// A head cut into several parts produces one partial (m, l, o) record per part; records are merged
-// by a tree of fan-in kMergeFanIn whose nodes are closed by whichever CTA delivers a node's last
-// input, so no merge is longer than kMergeFanIn records however long the head is.
+// launch covers them all.  The heads' page streams are laid end to end (longest head first) and cut
+// in two regions:
+//   * the first `static_pct` percent is cut into one equal SPAN per CTA.  A span crosses head
+//     boundaries where it must, so it is a short run of work items (one per head it touches), and
+//     the long heads end up in few, large parts;
+//   * the rest is cut into small TAIL items (`tail_items_per_cta` per CTA) that the CTAs pull one at
+//     a time as they finish their spans, which evens out whatever difference in speed there was.
+// A job is what a CTA pops from the queue: a span (several consecutive items) or one tail item.
+// A head cut into several parts produces one partial (m, l, o) record per part; records are merged by
+// a tree of fan-in kMergeFanIn whose nodes are closed by whichever CTA delivers a node's last input.
 #include <algorithm>
 #include <cstdint>
+#include <numeric>
+#include <vector>
 
 #include "razor_internal.h"
 
@@ -29,56 +36,110 @@ void tree_sizes(int n_parts, int* n_recs, int* n_tickets) {
   *n_tickets = tickets;
 }
 
-int build_schedule(const int32_t* pages, int n_heads, int target_items, int min_chunk, int max_items, int max_recs,
-                   int max_tickets, WorkItem* out, int* chunk_pages_out) {
+namespace {
+
+struct Piece {
+  int head, begin, end;   // pages [begin, end) of the head
+  int job;                // span index, or n_spans + running index for tail pieces
+};
+
+}  // namespace
+
+int build_schedule(const int32_t* pages, int n_heads, const SchedParams& sp, int max_items, int max_recs,
+                   int max_tickets, WorkItem* out, int32_t* jobs, SchedInfo* info) {
+  const int n_ctas = std::max(1, sp.n_ctas);
+  const int min_chunk = std::max(1, sp.min_chunk_pages);
+  const int static_pct = std::min(100, std::max(0, sp.static_pct));
+  const int tail_per_cta = std::max(1, sp.tail_items_per_cta);
+
+  std::vector<int> order(n_heads);
+  std::iota(order.begin(), order.end(), 0);
+  std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return pages[a] > pages[b]; });
   long long total = 0;
   for (int h = 0; h < n_heads; ++h) total += pages[h];
-  if (target_items < 1) target_items = 1;
-  if (min_chunk < 1) min_chunk = 1;
-  long long chunk = (total + target_items - 1) / target_items;
+
+  // Spans: equal, at least min_chunk pages, at most one per CTA.
+  const long long static_pages = total * static_pct / 100;
+  long long span = (static_pages + n_ctas - 1) / n_ctas;
+  if (span < min_chunk) span = min_chunk;
+  const long long n_spans = std::min<long long>(n_ctas, static_pages / span);
+  const long long static_end = n_spans * span;
+  const long long tail_pages = total - static_end;
+  long long chunk = (tail_pages + (long long)n_ctas * tail_per_cta - 1) / ((long long)n_ctas * tail_per_cta);
   if (chunk < min_chunk) chunk = min_chunk;
-  // Every head costs one item at least; grow the chunk until the items fit.
-  for (;;) {
-    long long n = 0;
-    for (int h = 0; h < n_heads; ++h) n += std::max<long long>(1, (pages[h] + chunk - 1) / chunk);
-    if (n <= max_items) break;
+
+  std::vector<Piece> pieces;
+  for (;;) {   // grow the tail chunk until the items fit
+    pieces.clear();
+    long long pos = 0;
+    int tail_jobs = 0;
+    for (int oi = 0; oi < n_heads; ++oi) {
+      const int h = order[oi];
+      const int p = pages[h];
+      int at = 0;
+      while (at < p && pos + at < static_end) {   // static region: cut at span boundaries
+        const long long k = (pos + at) / span;
+        const int stop = (int)std::min<long long>(p, (k + 1) * span - pos);
+        pieces.push_back({h, at, stop, (int)k});
+        at = stop;
+      }
+      if (at < p || p == 0) {   // dynamic region: equal parts of at most `chunk` pages; an empty head gets one empty item
+        const int len = p - at;
+        const int parts = std::max(1, (int)((len + chunk - 1) / chunk));
+        for (int i = 0; i < parts; ++i) {
+          const int b = at + (int)((long long)len * i / parts), e = at + (int)((long long)len * (i + 1) / parts);
+          pieces.push_back({h, b, e, (int)n_spans + tail_jobs++});
+        }
+      }
+      pos += p;
+    }
+    if ((long long)pieces.size() <= max_items) break;
     if (chunk > total) return -1;
     chunk += (chunk + 3) / 4;
   }
-  if (chunk_pages_out) *chunk_pages_out = (int)chunk;
 
-  int n = 0, rec = 0, ticket = 0;
+  // Per head: lay out records and tickets.
+  std::vector<int> n_parts(n_heads, 0), rec_base(n_heads, 0), ticket_base(n_heads, 0), next_part(n_heads, 0);
+  for (const Piece& pc : pieces) n_parts[pc.head] += 1;
+  int rec = 0, ticket = 0;
   for (int h = 0; h < n_heads; ++h) {
-    const int p = pages[h];
-    int parts = (int)((p + chunk - 1) / chunk);
-    if (parts < 1) parts = 1;
-    int n_recs, n_tickets;
-    tree_sizes(parts, &n_recs, &n_tickets);
-    if (rec + n_recs > max_recs || ticket + n_tickets > max_tickets) return -1;
-    for (int i = 0; i < parts; ++i) {
-      WorkItem w;
-      w.head = h;
-      w.page_begin = (int)((long long)p * i / parts);
-      w.page_end = (i == parts - 1) ? -1 : (int)((long long)p * (i + 1) / parts);
-      w.part_idx = i;
-      w.n_parts = parts;
-      w.rec_base = rec;
-      w.ticket_base = ticket;
-      w.pad = 0;
-      out[n++] = w;
-    }
-    rec += n_recs;
-    ticket += n_tickets;
+    int nr, nt;
+    tree_sizes(n_parts[h], &nr, &nt);
+    if (rec + nr > max_recs || ticket + nt > max_tickets) return -1;
+    rec_base[h] = rec;
+    ticket_base[h] = ticket;
+    rec += nr;
+    ticket += nt;
   }
-  // Heads with the deepest combine trees first (their merges then overlap the streaming of the
-  // rest), longer parts before shorter ones within equal depth: the queue ends on short items of
-  // heads whose final merge is a single node.
-  std::stable_sort(out, out + n, [&](const WorkItem& a, const WorkItem& b) {
-    if (a.n_parts != b.n_parts) return a.n_parts > b.n_parts;
-    const int la = (a.page_end < 0 ? pages[a.head] : a.page_end) - a.page_begin;
-    const int lb = (b.page_end < 0 ? pages[b.head] : b.page_end) - b.page_begin;
-    return la > lb;
-  });
+  // Job order: spans in stream order, then the tail items.  Jobs are numbered along the stream, so the
+  // pieces of one head stay in page order and part indices can be handed out as the pieces come.
+  std::stable_sort(pieces.begin(), pieces.end(), [](const Piece& a, const Piece& b) { return a.job < b.job; });
+  int n = 0, n_jobs = 0, last_job = -1, first_tail_job = -1;
+  for (const Piece& pc : pieces) {
+    if (pc.job != last_job) {
+      if (pc.job >= n_spans && first_tail_job < 0) first_tail_job = n_jobs;
+      jobs[n_jobs++] = n;
+      last_job = pc.job;
+    }
+    WorkItem w;
+    w.head = pc.head;
+    w.page_begin = pc.begin;
+    w.page_end = (pc.end == pages[pc.head]) ? -1 : pc.end;   // the head's last part grows with appends
+    w.part_idx = next_part[pc.head]++;
+    w.n_parts = n_parts[pc.head];
+    w.rec_base = rec_base[pc.head];
+    w.ticket_base = ticket_base[pc.head];
+    w.pad = 0;
+    out[n++] = w;
+  }
+  jobs[n_jobs] = n;
+  if (info) {
+    info->n_items = n;
+    info->n_jobs = n_jobs;
+    info->n_spans = first_tail_job < 0 ? n_jobs : first_tail_job;
+    info->span_pages = (int)span;
+    info->chunk_pages = (int)chunk;
+  }
   return n;
 }
 

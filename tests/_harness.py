@@ -158,7 +158,8 @@ def run_parity(w: synth.Workload, *, layers: Optional[Sequence[int]] = None,
                 q = synth.make_queries(w, l, t, dev)
                 out = cache.decode(l, q)
                 if t == 0 and l == all_layers[0]:
-                    assert cache.device_status() == 0, "a bounded wait inside the decode kernel ran out"
+                    status = cache.device_status()
+                    assert status == 0, f"a bounded wait inside the decode kernel ran out (status bits {status})"
                 if l not in heads_for:
                     continue
                 out_h = to_f64(out)
@@ -181,7 +182,8 @@ def run_parity(w: synth.Workload, *, layers: Optional[Sequence[int]] = None,
                         worst["out"] = max(worst["out"], err)
                         worst["outputs"] += 1
                         assert err <= tol, f"out max-abs {err:.3e} > {tol} at layer {l} b {b} head {g * G + j} step {t}"
-        assert cache.device_status() == 0, "a bounded wait inside the decode kernel ran out"
+        status = cache.device_status()
+        assert status == 0, f"a bounded wait inside the decode kernel ran out (status bits {status})"
         if stats is not None:
             stats.update(worst)
             stats["kept_bytes"], stats["dense_bytes"] = cache.stats(0)

@@ -125,54 +125,68 @@ def test_create_fails_loudly_without_a_gpu():
 
 # ------------------------------------------------------------------ decode schedule (host only)
 def _coverage(items, tokens):
-    pages = [(t + 15) // 16 for t in tokens]
+    pages = [-(-t // 16) for t in tokens]
     seen = {h: [] for h in range(len(tokens))}
-    for head, p0, p1, parts in items:
-        seen[head].append((p0, pages[head] if p1 < 0 else p1, parts))
+    for head, p0, p1, parts, job in items:
+        seen[head].append((p0, pages[head] if p1 < 0 else p1, parts, job))
     return pages, seen
 
 
-@pytest.mark.parametrize("tokens,target,min_chunk", [
-    ([65536] * 6 + [8196] * 34, 148 * 24, 8),                  # one sequence of the 64K-shaped stack
-    ([131072, 16388, 16388, 16388, 131072, 16388, 16388, 16388], 148 * 24, 8),
-    ([0, 1, 15, 16, 17, 100000, 3], 64, 1),
-    ([5000] * 2048, 148 * 24, 8),
-    ([7], 1, 1),
-    ([1 << 20] * 3, 148 * 200, 1),                             # more parts than the item budget: chunk grows
+@pytest.mark.parametrize("tokens,n_ctas,pct,tail,min_chunk", [
+    ([65536] * 24 + [8196] * 136, 148, 85, 4, 8),              # one layer of the 64K-shaped stack
+    ([131072, 16388, 16388, 16388, 131072, 16388, 16388, 16388] * 2, 148, 85, 4, 8),
+    ([0, 1, 15, 16, 17, 100000, 3], 148, 85, 4, 1),
+    ([5000] * 2048, 148, 85, 4, 8),
+    ([7], 148, 85, 4, 8),
+    ([1 << 20] * 3, 148, 0, 1000, 1),                          # more tail items than the item budget: chunk grows
+    ([9000, 37, 700, 9000, 37, 700], 5, 50, 2, 1),
+    ([4000] * 10, 148, 100, 1, 1),
 ])
-def test_schedule_covers_every_page_once_and_is_balanced(tokens, target, min_chunk):
-    items = rz.razor_schedule_plan(tokens, target, min_chunk)
+def test_schedule_covers_every_page_once_and_is_balanced(tokens, n_ctas, pct, tail, min_chunk):
+    items, n_spans = rz.razor_schedule_plan(tokens, n_ctas, pct, tail, min_chunk, with_spans=True)
     pages, seen = _coverage(items, tokens)
-    sizes = []
     for h, parts in seen.items():
         assert len(parts) >= 1                                 # every head gets at least one item (even empty)
-        parts.sort()
+        assert parts == sorted(parts)                          # parts of a head come in page order within the job order
         assert parts[0][0] == 0 and parts[-1][1] == pages[h]
         assert all(p[2] == len(parts) for p in parts)
         for a, b in zip(parts, parts[1:]):
             assert a[1] == b[0]                                # contiguous, no overlap
         open_ended = [it for it in items if it[0] == h and it[2] < 0]
         assert len(open_ended) == 1                            # the last part grows with appends
-        sizes += [p[1] - p[0] for p in parts]
     total = sum(pages)
-    chunk = max(min_chunk, -(-total // target))
-    if len(tokens) + total // chunk <= 16384:                  # item budget not hit: parts obey the chunk
-        assert max(sizes) <= chunk
-        assert len(items) <= len(tokens) + total // chunk + 1
-    else:                                                      # the chunk grew until the items fit
-        assert len(items) <= len(tokens) + 16384
-        assert max(sizes) - min(sizes) <= 1
-    # heads cut into the most parts first; within equal part counts, longer ranges first
-    keys = [(-parts, -((pages[h] if p1 < 0 else p1) - p0)) for h, p0, p1, parts in items]
-    assert keys == sorted(keys)
+    jobs = items[:, 4]
+    assert (np.diff(jobs) >= 0).all() and jobs[0] == 0         # job order, jobs numbered from 0
+    n_jobs = int(jobs[-1]) + 1
+    assert 0 <= n_spans <= min(n_ctas, n_jobs)
+    size = np.array([(pages[h] if p1 < 0 else p1) - p0 for h, p0, p1, _, _ in items])
+    job_pages = np.bincount(jobs, weights=size, minlength=n_jobs)
+    if n_spans:
+        span = job_pages[0]
+        assert (job_pages[:n_spans] == span).all()             # spans are equal
+        assert span >= min_chunk
+        assert n_spans * span <= total * pct / 100 + 1e-9
+        assert n_spans == n_ctas or (n_spans + 1) * span > total * pct // 100
+    tail_sizes = job_pages[n_spans:]
+    assert (np.bincount(jobs)[n_spans:] == 1).all()            # a tail job is one item
+    if len(tail_sizes):
+        tail_total = int(tail_sizes.sum())
+        chunk = max(min_chunk, -(-tail_total // (n_ctas * tail)))
+        if len(tokens) + n_spans + tail_total // chunk <= 16384:
+            assert tail_sizes.max() <= chunk
+        else:                                                  # the chunk grew until the items fit the budget
+            assert tail_sizes.max() - tail_sizes[tail_sizes > 0].min() <= 1
+    assert len(items) <= len(tokens) + 16384
 
 
-def test_schedule_splits_only_long_heads():
-    tokens = [65536] * 2 + [8196] * 10
-    items = rz.razor_schedule_plan(tokens, 64, 4)
-    parts = {h: n for h, _, _, n in items}
-    assert parts[0] > 8 * parts[5] - 8 and parts[5] >= 1
+def test_schedule_gives_long_heads_few_parts():
+    tokens = [65536] * 24 + [8196] * 136                       # 6 retrieval heads x 4 sequences, 40 heads each
+    items = rz.razor_schedule_plan(tokens)
+    parts = {h: n for h, _, _, n, _ in items}
+    assert max(parts[h] for h in range(24)) <= 8               # a full-length head spans about four CTAs' shares
     with pytest.raises(rz.RazorError):
-        rz.razor_schedule_plan([-1], 4)
+        rz.razor_schedule_plan([-1])
     with pytest.raises(rz.RazorError):
-        rz.razor_schedule_plan([100], 4, 0)
+        rz.razor_schedule_plan([100], 148, 85, 4, 0)
+    with pytest.raises(rz.RazorError):
+        rz.razor_schedule_plan([100], 148, 101, 4, 1)

@@ -123,10 +123,13 @@ def test_small_shape_sweep(dtype, D, group):
     (2, {rz.OPT_DECODE_TENSOR_CORES: 1}),                                   # matrix instructions from group 2
     (2, {rz.OPT_DECODE_TENSOR_CORES: 1, rz.OPT_DECODE_CONSUMER_WARPS: 4}),
     (4, {rz.OPT_DECODE_TENSOR_CORES: 2}),                                   # grouped heads on the CUDA cores
-    (4, {rz.OPT_DECODE_CONSUMER_WARPS: 4, rz.OPT_DECODE_ITEMS_PER_SM: 64, rz.OPT_DECODE_MIN_CHUNK_PAGES: 1}),
+    (4, {rz.OPT_DECODE_CONSUMER_WARPS: 4, rz.OPT_DECODE_TAIL_ITEMS_PER_SM: 64, rz.OPT_DECODE_MIN_CHUNK_PAGES: 1}),
+    (4, {rz.OPT_DECODE_STATIC_PERCENT: 0, rz.OPT_DECODE_TAIL_ITEMS_PER_SM: 2, rz.OPT_DECODE_MIN_CHUNK_PAGES: 1}),
+    (1, {rz.OPT_DECODE_STATIC_PERCENT: 100, rz.OPT_DECODE_MIN_CHUNK_PAGES: 1}),
     (8, {rz.OPT_DECODE_RING_KB: 64}),
     (1, {rz.OPT_DECODE_CONSUMER_WARPS: 16, rz.OPT_DECODE_RING_KB: 128}),
-    (1, {rz.OPT_DECODE_CONSUMER_WARPS: 8, rz.OPT_DECODE_ITEMS_PER_SM: 200, rz.OPT_DECODE_MIN_CHUNK_PAGES: 1}),
+    (1, {rz.OPT_DECODE_CONSUMER_WARPS: 8, rz.OPT_DECODE_STATIC_PERCENT: 30, rz.OPT_DECODE_TAIL_ITEMS_PER_SM: 200,
+         rz.OPT_DECODE_MIN_CHUNK_PAGES: 1}),
 ])
 @pytest.mark.parametrize("D", [64, 128])
 def test_decode_kernel_variants(group, options, D):
