@@ -33,8 +33,8 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 inline int ceil_div(long long a, long long b) { return (int)((a + b - 1) / b); }
 
 struct Layout {
-  size_t state, comp_sum, comp_mean, page_table, items, jobs, rec_ml, rec_o, tickets, queue, scratch, seq_desc, total;
-  int max_pages, max_items, max_recs, max_tickets;
+  size_t state, comp_sum, comp_mean, page_table, items, jobs, multi, rec_ml, rec_o, queue, scratch, seq_desc, total;
+  int max_pages, max_items;
 };
 
 int check_config(const razor_config_t* c) {
@@ -63,9 +63,6 @@ Layout make_layout(const razor_config_t& c) {
   const int g = c.n_q_heads / c.n_kv_heads;
   l.max_pages = std::max(1, ceil_div((long long)c.max_ctx_len + c.max_new_tokens, kPageTokens));
   l.max_items = (int)nh + kItemBudget;
-  // Level-0 records plus the inner nodes of the combine trees (fan-in kMergeFanIn), with slack per head.
-  l.max_recs = l.max_items + l.max_items / (kMergeFanIn - 1) + kMaxTreeLevels * (int)nh;
-  l.max_tickets = l.max_items / (kMergeFanIn - 1) + kMaxTreeLevels * (int)nh;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
   l.state = take(L * nh * sizeof(HeadState));
@@ -74,9 +71,9 @@ Layout make_layout(const razor_config_t& c) {
   l.page_table = take(L * nh * (size_t)l.max_pages * sizeof(int32_t));
   l.items = take(L * (size_t)l.max_items * sizeof(WorkItem));
   l.jobs = take(L * ((size_t)l.max_items + 1) * sizeof(int32_t));
-  l.rec_ml = take((size_t)l.max_recs * g * sizeof(float2));
-  l.rec_o = take((size_t)l.max_recs * g * D * sizeof(float));
-  l.tickets = take((size_t)l.max_tickets * sizeof(int32_t));
+  l.multi = take(L * nh * sizeof(MultiHead));
+  l.rec_ml = take((size_t)l.max_items * g * sizeof(float2));
+  l.rec_o = take((size_t)l.max_items * g * D * sizeof(float));
   l.queue = take(8 * sizeof(int32_t));   // queue[0..3], then the status word
   l.scratch = take(nh * kCompressMaxSlices * 2 * D * sizeof(float));
   l.seq_desc = take((size_t)c.batch * sizeof(SeqDesc));
@@ -100,9 +97,10 @@ struct LayerHost {
   int appended = 0;
   // decode schedule
   bool sched_valid = false;
-  int n_items = 0, n_jobs = 0, n_spans = 0, chunk_pages = 0, growth_tokens = 0;
+  int n_items = 0, n_jobs = 0, n_spans = 0, n_multi = 0, chunk_pages = 0, growth_tokens = 0;
   WorkItem* items = nullptr;        // pinned host, [max_items]
   int32_t* jobs = nullptr;          // pinned host, [max_items + 1]
+  MultiHead* multi = nullptr;       // pinned host, [B*Hkv]
   cudaEvent_t upload_done = nullptr;
 };
 
@@ -125,6 +123,7 @@ struct razor_cache {
   std::vector<LayerHost> layers;
   WorkItem* pinned_items = nullptr;   // [L][max_items]
   int32_t* pinned_jobs = nullptr;     // [L][max_items + 1]
+  MultiHead* pinned_multi = nullptr;  // [L][B*Hkv]
 };
 
 extern "C" {
@@ -203,7 +202,7 @@ int razor_cache_create(razor_cache_t** out, const razor_config_t* cfg, void* poo
   dv.jobs = (int32_t*)(ws + lay.jobs);
   dv.rec_ml = (float2*)(ws + lay.rec_ml);
   dv.rec_o = (float*)(ws + lay.rec_o);
-  dv.tickets = (int32_t*)(ws + lay.tickets);
+  dv.multi = (MultiHead*)(ws + lay.multi);
   dv.queue = (int32_t*)(ws + lay.queue);
   dv.status = dv.queue + 4;
   dv.compress_scratch = (float*)(ws + lay.scratch);
@@ -212,8 +211,6 @@ int razor_cache_create(razor_cache_t** out, const razor_config_t* cfg, void* poo
   dv.n_kv_heads = cfg->n_kv_heads;
   dv.max_pages = lay.max_pages;
   dv.max_items = lay.max_items;
-  dv.max_recs = lay.max_recs;
-  dv.max_tickets = lay.max_tickets;
   dv.head_dim = cfg->head_dim;
   dv.n_sink = cfg->n_sink;
   dv.group = cfg->n_q_heads / cfg->n_kv_heads;
@@ -228,11 +225,14 @@ int razor_cache_create(razor_cache_t** out, const razor_config_t* cfg, void* poo
   if (e == cudaSuccess)
     e = cudaHostAlloc((void**)&c->pinned_jobs, (size_t)cfg->n_layers * (lay.max_items + 1) * sizeof(int32_t),
                       cudaHostAllocDefault);
+  if (e == cudaSuccess)
+    e = cudaHostAlloc((void**)&c->pinned_multi, (size_t)cfg->n_layers * dv.n_heads * sizeof(MultiHead),
+                      cudaHostAllocDefault);
   if (e != cudaSuccess) {
     g_last_cuda_error = (int)e;
     (void)cudaGetLastError();
     if (c->pinned_items) cudaFreeHost(c->pinned_items);
-  if (c->pinned_jobs) cudaFreeHost(c->pinned_jobs);
+    if (c->pinned_jobs) cudaFreeHost(c->pinned_jobs);
     delete c;
     return RAZOR_E_CUDA;
   }
@@ -246,6 +246,7 @@ int razor_cache_create(razor_cache_t** out, const razor_config_t* cfg, void* poo
     L.region_count.assign(cfg->batch, 0);
     L.items = c->pinned_items + (size_t)l * lay.max_items;
     L.jobs = c->pinned_jobs + (size_t)l * (lay.max_items + 1);
+    L.multi = c->pinned_multi + (size_t)l * dv.n_heads;
   }
   *out = c;
   return RAZOR_OK;
@@ -272,6 +273,7 @@ int razor_cache_destroy(razor_cache_t* c) {
     if (L.upload_done) cudaEventDestroy(L.upload_done);
   if (c->pinned_items) cudaFreeHost(c->pinned_items);
   if (c->pinned_jobs) cudaFreeHost(c->pinned_jobs);
+  if (c->pinned_multi) cudaFreeHost(c->pinned_multi);
   delete c;
   return RAZOR_OK;
 }
@@ -409,12 +411,12 @@ int ensure_schedule(razor_cache* c, int layer, cudaStream_t stream, bool upload)
   if (L.upload_done) RZ_CUDA(cudaEventSynchronize(L.upload_done));   // previous upload has left the staging area
   const SchedParams sp{c->n_sms, c->tune.static_pct, c->tune.tail_items_per_sm, c->tune.min_chunk_pages};
   SchedInfo info{};
-  const int n = build_schedule(pages.data(), nh, sp, c->lay.max_items, c->lay.max_recs, c->lay.max_tickets, L.items,
-                               L.jobs, &info);
+  const int n = build_schedule(pages.data(), nh, sp, c->lay.max_items, L.items, L.jobs, L.multi, &info);
   if (n < 0) return RAZOR_E_INVALID_ARG;
   L.n_items = n;
   L.n_jobs = info.n_jobs;
   L.n_spans = info.n_spans;
+  L.n_multi = info.n_multi;
   L.chunk_pages = info.chunk_pages;
   L.growth_tokens = 0;
   if (upload) {
@@ -423,6 +425,9 @@ int ensure_schedule(razor_cache* c, int layer, cudaStream_t stream, bool upload)
                             cudaMemcpyHostToDevice, stream));
     RZ_CUDA(cudaMemcpyAsync(c->dv.jobs + (size_t)layer * (c->lay.max_items + 1), L.jobs,
                             (size_t)(L.n_jobs + 1) * sizeof(int32_t), cudaMemcpyHostToDevice, stream));
+    if (L.n_multi)
+      RZ_CUDA(cudaMemcpyAsync(c->dv.multi + (size_t)layer * nh, L.multi, (size_t)L.n_multi * sizeof(MultiHead),
+                              cudaMemcpyHostToDevice, stream));
     RZ_CUDA(cudaEventRecord(L.upload_done, stream));
     L.sched_valid = true;
   } else {
@@ -523,7 +528,7 @@ int razor_decode_attention(razor_cache_t* c, int32_t layer, const void* q, float
   rc = ensure_schedule(c, layer, (cudaStream_t)stream, true);
   if (rc) return rc;
   const LayerHost& L = c->layers[layer];
-  const DecodeJobs jb{L.n_items, L.n_jobs, L.n_spans, L.jobs[L.n_spans]};
+  const DecodeJobs jb{L.n_items, L.n_jobs, L.n_spans, L.jobs[L.n_spans], L.n_multi};
   RZ_CUDA(launch_decode(c->dv, c->cfg.dtype, layer, jb, q, out, c->n_sms, c->tune,
                         (cudaStream_t)stream));
   return RAZOR_OK;
@@ -580,10 +585,10 @@ int razor_schedule_plan(const int32_t* tokens, int32_t n_heads, int32_t n_ctas, 
   const int cap = n_heads + kItemBudget;
   std::vector<WorkItem> w(cap);
   std::vector<int32_t> jobs(cap + 1);
+  std::vector<MultiHead> multi(n_heads);
   const SchedParams sp{n_ctas, static_percent, tail_items_per_cta, min_chunk_pages};
   SchedInfo info{};
-  const int n = build_schedule(pages.data(), n_heads, sp, cap, 2 * cap + kMaxTreeLevels * n_heads,
-                               cap + kMaxTreeLevels * n_heads, w.data(), jobs.data(), &info);
+  const int n = build_schedule(pages.data(), n_heads, sp, cap, w.data(), jobs.data(), multi.data(), &info);
   if (n < 0) return RAZOR_E_INVALID_ARG;
   if (n_spans) *n_spans = info.n_spans;
   return emit_items(w.data(), n, jobs.data(), info.n_jobs, items, max_items, n_items);
@@ -630,9 +635,8 @@ int razor_cache_device_status(razor_cache_t* c, int32_t* status, void* stream) {
   RZ_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
   *status = host;
   if (host != 0) {
-    // A kernel gave up part-way: its queue and ticket counters may be left non-zero.  Put them back.
+    // A kernel gave up part-way: its job queue may be left non-zero.  Put it back.
     RZ_CUDA(cudaMemsetAsync(c->dv.queue, 0, 8 * sizeof(int32_t), (cudaStream_t)stream));
-    RZ_CUDA(cudaMemsetAsync(c->dv.tickets, 0, (size_t)c->lay.max_tickets * sizeof(int32_t), (cudaStream_t)stream));
     RZ_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
   }
   return RAZOR_OK;

@@ -2,16 +2,18 @@
 // persistent producer / consumer kernel, one CTA per SM.
 //
 // One launch covers every (sequence, KV head) of a layer, full-length retrieval heads and short heads
-// alike.  The host cuts the token streams into page ranges of near-equal size (work items) that the
-// CTAs pull from a queue.  Inside a CTA
+// alike.  The host lays the heads' page streams end to end and cuts them into one equal span per CTA
+// plus a tail of small items; a CTA pulls its span, then tail items, from a queue.  Inside a CTA
 //   * the PRODUCER warp pops items, publishes each item's descriptor, query rows and compensation
 //     token in a small shared-memory slot, and streams the item's pages (one contiguous K|V block
 //     each) into a shared-memory ring with bulk asynchronous copies that complete on mbarriers.  It
 //     runs ahead across item boundaries, so the ring never drains;
 //   * NC CONSUMER warps take the ring's pages round-robin; each keeps an online-softmax state
 //     (m, l, o) per query head of the group in registers and hands it over at the end of the item;
-//   * the REDUCER warp merges the NC states of an item into one partial record, and closes the nodes
-//     of the head's combine tree whose last input it delivered (ticket counters; no second launch).
+//   * the REDUCER warp merges the NC states of an item into one state and writes it out: as the head's
+//     output when the head is in one part, else as a partial record.
+// Heads cut into several parts are finished by combine_kernel, a small dependent launch that merges
+// their records (one CTA per head) as soon as the streaming kernel has drained.
 //
 // The compensation token of a non-retrieval head is folded into the online softmax as the initial
 // state of the head's first part: m = s_c + log2(N_d), l = 1, o = v_hat, which is the term
@@ -36,8 +38,6 @@ constexpr int kItemSlots = 2;            // item descriptors in flight between p
 constexpr int kMaxMergeBufs = 2;         // consumer -> reducer hand-over buffers (one where they are large)
 template <int G>
 constexpr int merge_bufs() { return G >= 4 ? 1 : 2; }
-template <int G>
-constexpr int land_heads() { return G < 2 ? G : 2; }   // query heads whose rows land together in a merge
 constexpr int kMaxStages = 64;           // ring stages (pages in flight per CTA)
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s: far beyond any healthy wait
 
@@ -122,7 +122,7 @@ struct ItemDesc {
   int32_t part_idx;
   int32_t n_parts;
   int32_t rec_base;
-  int32_t ticket_base;
+  int32_t pad2;
   int32_t seed;        // 1: this part starts from the compensation token
   int32_t n_drop;
   int32_t pad0, pad1;
@@ -142,7 +142,6 @@ struct Barriers {
   uint64_t item_empty[kItemSlots];
   uint64_t merge_full[kMaxMergeBufs];
   uint64_t merge_free[kMaxMergeBufs];
-  uint64_t land;   // landing zone of the combine-tree merges
 };
 
 // Hand-over buffer: the descriptor of the item, then per consumer warp and query head (m, l) and o[D].
@@ -153,16 +152,10 @@ struct alignas(16) MergeBuf {
   alignas(16) float o[NC][G][D];
 };
 
-// Dynamic shared memory: the hand-over buffers, the landing zone of the combine-tree merges
-// (kMergeFanIn records x up to 2 heads x D floats), then the page ring (1 KiB aligned).
-template <typename T, int D, int G, int NC>
-constexpr size_t decode_land_offset() {
-  return (sizeof(MergeBuf<D, G, NC>) * merge_bufs<G>() + 127) & ~(size_t)127;
-}
+// Dynamic shared memory: the hand-over buffers, then the page ring (1 KiB aligned).
 template <typename T, int D, int G, int NC>
 constexpr size_t decode_ring_offset() {
-  return (decode_land_offset<T, D, G, NC>() + (size_t)kMergeFanIn * land_heads<G>() * D * sizeof(float) + 1023) &
-         ~(size_t)1023;
+  return (sizeof(MergeBuf<D, G, NC>) * merge_bufs<G>() + 1023) & ~(size_t)1023;
 }
 
 template <int G, int EPL>
@@ -421,7 +414,6 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
   using Geo = RowGeom<T, D>;
   constexpr int LPR = Geo::kLpr, EPL = Geo::kEpl;
   constexpr uint32_t PB = Geo::kPageBytes;
-  constexpr int F = kMergeFanIn;
   using Slot = ItemSlot<T, D, G>;
   using MBuf = MergeBuf<D, G, NC>;
   constexpr int kMergeBufs = merge_bufs<G>();
@@ -451,11 +443,13 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
       mbar_init(&bars.merge_full[s], NC);
       mbar_init(&bars.merge_free[s], 1);
     }
-    mbar_init(&bars.land, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   __syncthreads();
+  // The combine kernel that follows may be made resident as soon as SMs free up; it waits for this whole
+  // grid to finish before it reads anything this grid writes.
+  cudaTriggerProgrammaticLaunchCompletion();
 
   const WorkItem* items = dv.items + (size_t)layer * dv.max_items;
   const int32_t* jobs = dv.jobs + (size_t)layer * (dv.max_items + 1);
@@ -530,7 +524,7 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
       if (lane == 0) {
         ItemDesc d;
         d.head = w.head; d.page_begin = w.page_begin; d.n_pages = n; d.len = st.len;
-        d.part_idx = w.part_idx; d.n_parts = w.n_parts; d.rec_base = w.rec_base; d.ticket_base = w.ticket_base;
+        d.part_idx = w.part_idx; d.n_parts = w.n_parts; d.rec_base = w.rec_base; d.pad2 = 0;
         d.seed = seed ? 1 : 0; d.n_drop = st.n_drop; d.pad0 = d.pad1 = 0;
         sl.desc = d;
         const int b = w.head / dv.n_kv_heads, g = w.head % dv.n_kv_heads;
@@ -555,20 +549,28 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
         const bool mine = lane < in_batch;
         const bool real = mine && p0 + lane < n;
         const int32_t pid_after = (p0 + batch + lane < n) ? pt[p0 + batch + lane] : 0;   // ids of the next round
-        unsigned stage = 0;
+        unsigned stage = 0, use_cur = 0;
         bool ready = true;
         if (mine) {
-          unsigned use;
-          ring_slot<NC>(c + lane, ns, stage, use);
-          if (use > 0) ready = mbar_wait(&bars.empty[stage], (use - 1) & 1, abort_flag);
+          // Each lane waits for its own stage and issues at once, inside the same divergent region: a freed
+          // stage is refilled whatever the other stages of the round are doing.
+          ring_slot<NC>(c + lane, ns, stage, use_cur);
+          if (use_cur > 0) ready = mbar_wait(&bars.empty[stage], (use_cur - 1) & 1, abort_flag);
+          if (ready) {
+            if (real) {
+              mbar_arrive_expect_tx(&bars.full[stage], PB);
+              bulk_load(ring + (size_t)stage * PB, dv.pool + (size_t)pid_cur * dv.page_bytes, PB, &bars.full[stage]);
+            } else {
+              mbar_arrive(&bars.full[stage]);
+            }
+          }
         }
-        ok = __all_sync(0xffffffffu, ready);   // all or nothing: `c` stays an exact count of issued positions
-        if (!ok) break;
-        if (real) {
-          mbar_arrive_expect_tx(&bars.full[stage], PB);
-          bulk_load(ring + (size_t)stage * PB, dv.pool + (size_t)pid_cur * dv.page_bytes, PB, &bars.full[stage]);
-        } else if (mine) {
-          mbar_arrive(&bars.full[stage]);
+        ok = __all_sync(0xffffffffu, ready);
+        if (!ok) {
+          // Some lane gave up, so `c` no longer says exactly which positions were issued: the lanes that
+          // did issue a copy in this round wait (bounded) for it here, before the common exit path.
+          if (ready && real && !mbar_wait_drain(&bars.full[stage], use_cur & 1)) atomicOr(dv.status, kStatusDrainTimeout);
+          break;
         }
         c += in_batch;
         pid_cur = pid_after;
@@ -806,101 +808,7 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
   } else {
     // ======================================================================== reducer
     bool ok = true;
-    unsigned land_uses = 0;
-    float* land = (float*)(dyn_smem + decode_land_offset<T, D, G, NC>());
-    constexpr int GB = land_heads<G>();   // query heads whose rows land together
-
-    // A part's record has been written and its arrival counted (`ticket` is the count before it).  Walk up
-    // the head's combine tree for as long as this warp delivers the last input of a node.
-    auto climb = [&](int ticket, int idx, int n, int rec_off, int tk_off, float* out_rows) {
-      for (;;) {
-        const int n_next = (n + F - 1) / F, node = idx / F;
-        const int fan = min(F, n - node * F);
-        if (ticket != fan - 1) return;
-        // Last input of this node: merge its `fan` records.
-        __threadfence();
-        if (lane == 0) dv.tickets[tk_off + node] = 0;
-        const int first_rec = rec_off + node * F;
-#pragma unroll 1
-        for (int jh = 0; jh < G; jh += GB) {
-          // The rows of GB heads of every record travel to shared memory as one bulk copy per record
-          // (a single round trip for the whole node); (m, l) come by ordinary loads meanwhile.
-          asm volatile("fence.proxy.async;" ::: "memory");
-          if (lane == 0) mbar_arrive_expect_tx(&bars.land, (uint32_t)fan * GB * D * sizeof(float));
-          __syncwarp();
-          if (lane < fan)
-            bulk_load(land + (size_t)lane * GB * D, dv.rec_o + ((size_t)(first_rec + lane) * G + jh) * D,
-                      GB * D * sizeof(float), &bars.land);
-          float mx[GB], l[GB], cw[GB];
-#pragma unroll
-          for (int jj = 0; jj < GB; ++jj) {
-            float2 ml = make_float2(-CUDART_INF_F, 0.f);
-            if (lane < fan) ml = __ldcg(&dv.rec_ml[(size_t)(first_rec + lane) * G + jh + jj]);
-            mx[jj] = ml.x;
-            l[jj] = ml.y;
-            cw[jj] = ml.x;
-          }
-#pragma unroll
-          for (int jj = 0; jj < GB; ++jj) {
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) mx[jj] = fmaxf(mx[jj], __shfl_xor_sync(0xffffffffu, mx[jj], off));
-            const float mu = (mx[jj] == -CUDART_INF_F) ? 0.f : mx[jj];
-            cw[jj] = fast_exp2(cw[jj] - mu);
-            l[jj] *= cw[jj];
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) l[jj] += __shfl_xor_sync(0xffffffffu, l[jj], off);
-          }
-          if (!warp_wait(&bars.land, land_uses & 1)) { ok = false; return; }
-          ++land_uses;
-#pragma unroll
-          for (int jj = 0; jj < GB; ++jj) {
-            LaneVec<D> sum;
-            sum.zero();
-#pragma unroll
-            for (int r = 0; r < F; ++r) {
-              const float cr = __shfl_sync(0xffffffffu, cw[jj], r);
-              if (r < fan) {
-                LaneVec<D> o;
-                o.load_shared(land + ((size_t)r * GB + jj) * D, lane);
-                sum.fma(cr, o);
-              }
-            }
-            if (n_next == 1) {
-              sum.scale(l[jj] > 0.f ? 1.f / l[jj] : 0.f);
-              sum.store(out_rows + (size_t)(jh + jj) * D, lane);
-            } else {
-              const size_t r = (size_t)(rec_off + n + node) * G + jh + jj;
-              if (lane == 0) dv.rec_ml[r] = make_float2(mx[jj], l[jj]);
-              sum.store(dv.rec_o + r * D, lane);
-            }
-          }
-          __syncwarp();   // every lane is done with the landing zone before the next copies are issued
-        }
-        if (n_next == 1) return;
-        rec_off += n;
-        tk_off += n_next;
-        idx = node;
-        n = n_next;
-        __threadfence();
-        __syncwarp();
-        ticket = 0;
-        if (lane == 0) ticket = atomicAdd(&dv.tickets[tk_off + idx / F], 1);
-        ticket = __shfl_sync(0xffffffffu, ticket, 0);
-      }
-    };
-
-    // The arrival count of a part's record is asked for right after the record is written, but looked at
-    // only after the next item has been reduced, so its round trip overlaps useful work.
-    bool pend = false;
-    int pend_ticket = 0, pend_idx = 0, pend_n = 0, pend_rec = 0, pend_tk = 0;
-    float* pend_out = nullptr;
-    auto resolve = [&]() {
-      if (!pend) return;
-      pend = false;
-      climb(__shfl_sync(0xffffffffu, pend_ticket, 0), pend_idx, pend_n, pend_rec, pend_tk, pend_out);
-    };
-
-    for (unsigned seq = 0; ok; ++seq) {
+    for (unsigned seq = 0;; ++seq) {
       const int mb = seq % kMergeBufs;
       if (!warp_wait(&bars.merge_full[mb], (seq / kMergeBufs) & 1)) { ok = false; break; }
       const MBuf& M = mbufs[mb];
@@ -932,37 +840,110 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
       __syncwarp();
       if (lane == 0) mbar_arrive(&bars.merge_free[mb]);
 
-      const int b = d.head / dv.n_kv_heads, g = d.head % dv.n_kv_heads;
-      float* out_rows = out + ((size_t)b * n_q_heads + (size_t)g * G) * D;
-      if (d.n_parts == 1) {
+      if (d.n_parts == 1) {   // the head's only part: this is its output
+        const int b = d.head / dv.n_kv_heads, g = d.head % dv.n_kv_heads;
+        float* out_rows = out + ((size_t)b * n_q_heads + (size_t)g * G) * D;
 #pragma unroll
         for (int j = 0; j < G; ++j) {
           acc[j].scale(l_tot[j] > 0.f ? 1.f / l_tot[j] : 0.f);
           acc[j].store(out_rows + (size_t)j * D, lane);
         }
-        resolve();
-        continue;
-      }
-      // This part's record and its arrival at the level-0 node.
+      } else {                // one of several parts: its record, for the combine kernel
 #pragma unroll
-      for (int j = 0; j < G; ++j) {
-        const size_t r = (size_t)(d.rec_base + d.part_idx) * G + j;
-        if (lane == 0) dv.rec_ml[r] = make_float2(m_tot[j], l_tot[j]);
-        acc[j].store(dv.rec_o + r * D, lane);
+        for (int j = 0; j < G; ++j) {
+          const size_t r = (size_t)(d.rec_base + d.part_idx) * G + j;
+          if (lane == 0) dv.rec_ml[r] = make_float2(m_tot[j], l_tot[j]);
+          acc[j].store(dv.rec_o + r * D, lane);
+        }
       }
-      __threadfence();
-      __syncwarp();
-      int ticket_raw = 0;
-      if (lane == 0) ticket_raw = atomicAdd(&dv.tickets[d.ticket_base + d.part_idx / F], 1);
-      resolve();   // the previous part's count has had this item's time to arrive
-      pend = true;
-      pend_ticket = ticket_raw;
-      pend_idx = d.part_idx; pend_n = d.n_parts; pend_rec = d.rec_base; pend_tk = d.ticket_base;
-      pend_out = out_rows;
     }
-    if (ok) resolve();
     if (!ok && lane == 0) atomicOr(dv.status, kStatusReducerTimeout);
   }
+}
+
+// ------------------------------------------------------------------------------------------ combine
+// Merges the partial records of the heads that were cut into several parts (Eq. 5 regrouped: sums of
+// exponentials under a common maximum).  One CTA per (such head, query head of its group); warp w folds
+// records w, w + 8, ... in that order and the eight warp states are folded in warp order, so the result
+// does not depend on timing.  Launched as a programmatic dependent of the streaming kernel: its CTAs
+// may become resident while that kernel drains, and wait for all of its writes at
+// cudaGridDependencySynchronize().
+constexpr int kCombineWarps = 8;
+
+template <int D>
+__global__ void __launch_bounds__(kCombineWarps * 32) combine_kernel(DeviceView dv, int layer, float* __restrict__ out) {
+  __shared__ float2 s_ml[kCombineWarps];
+  __shared__ __align__(16) float s_o[kCombineWarps][D];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int G = dv.group, j = blockIdx.y;
+  const MultiHead mh = dv.multi[(size_t)layer * dv.n_heads + blockIdx.x];   // uploaded before either kernel
+  cudaGridDependencySynchronize();   // the streaming kernel's records are complete and visible from here on
+  float m = -CUDART_INF_F, l = 0.f;
+  LaneVec<D> acc;
+  acc.zero();
+  constexpr int U = 8;   // records in flight per warp
+  for (int r0 = warp; r0 < mh.n_parts; r0 += kCombineWarps * U) {
+    float2 ml[U];
+    LaneVec<D> rows[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int r = min(r0 + u * kCombineWarps, mh.n_parts - 1);   // beyond the end: re-read the last one, unused
+      const size_t idx = (size_t)(mh.rec_base + r) * G + j;
+      ml[u] = __ldcg(&dv.rec_ml[idx]);
+      rows[u].load_l2(dv.rec_o + idx * D, lane);
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      if (r0 + u * kCombineWarps < mh.n_parts) {
+        const float mn = fmaxf(m, ml[u].x);
+        const float mu = (mn == -CUDART_INF_F) ? 0.f : mn;
+        const float c_old = fast_exp2(m - mu), c_new = fast_exp2(ml[u].x - mu);
+        l = l * c_old + ml[u].y * c_new;
+        acc.scale(c_old);
+        acc.fma(c_new, rows[u]);
+        m = mn;
+      }
+    }
+  }
+  if (lane == 0) s_ml[warp] = make_float2(m, l);
+  acc.store(&s_o[warp][0], lane);
+  __syncthreads();
+  if (warp == 0) {
+    float mx = -CUDART_INF_F;
+#pragma unroll
+    for (int w = 0; w < kCombineWarps; ++w) mx = fmaxf(mx, s_ml[w].x);
+    const float mu = (mx == -CUDART_INF_F) ? 0.f : mx;
+    float lt = 0.f;
+    LaneVec<D> sum;
+    sum.zero();
+#pragma unroll
+    for (int w = 0; w < kCombineWarps; ++w) {
+      const float cw = fast_exp2(s_ml[w].x - mu);
+      lt += s_ml[w].y * cw;
+      LaneVec<D> o;
+      o.load_shared(&s_o[w][0], lane);
+      sum.fma(cw, o);
+    }
+    sum.scale(lt > 0.f ? 1.f / lt : 0.f);
+    const int b = mh.head / dv.n_kv_heads, g = mh.head % dv.n_kv_heads;
+    sum.store(out + (((size_t)b * dv.n_kv_heads + g) * G + j) * D, lane);
+  }
+}
+
+template <int D>
+cudaError_t combine_launch(const DeviceView& dv, int layer, int n_multi, float* out, cudaStream_t s) {
+  if (n_multi <= 0) return cudaSuccess;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(n_multi, dv.group);
+  cfg.blockDim = dim3(kCombineWarps * 32);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, combine_kernel<D>, dv, layer, out);
 }
 
 // ------------------------------------------------------------------------------------------ launch
@@ -999,7 +980,8 @@ cudaError_t decode_launch(const DeviceView& dv, int layer, const DecodeJobs& jb,
   int grid = std::min(n_sms, (int)jb.n_jobs);
   if (grid < 1) grid = 1;
   kern<<<grid, (NC + 2) * 32, dyn, s>>>(dv, layer, jb, (const T*)q, out, (int)stages);
-  return cudaGetLastError();
+  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  return combine_launch<D>(dv, layer, jb.n_multi, out, s);
 }
 
 template <typename T, int D, int G>

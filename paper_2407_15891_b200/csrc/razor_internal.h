@@ -14,8 +14,6 @@ namespace razor {
 constexpr int kPageTokens = 16;        // tokens per page
 constexpr int kMaxGroup = 8;           // query heads per KV head
 constexpr int kCompressMaxSlices = 64; // row slices per (sequence, KV head) in the compression kernel
-constexpr int kMergeFanIn = 32;        // partial records merged per node of a head's combine tree
-constexpr int kMaxTreeLevels = 5;      // 32^5 parts per head: more than any page count the config allows
 
 // Device-resident state of one (layer, sequence, KV head).  window < 0 marks a head that keeps every
 // token (retrieval head).  Physical slots: [0, n_sink) sinks, then the recent window as a ring whose
@@ -29,9 +27,8 @@ struct HeadState {
 
 // One decode work item: pages [page_begin, page_end) of one head's token stream, streamed by one CTA.
 // page_end < 0 means "to the end of the stream as it is now" (the last part of a head grows with
-// appends).  A head cut into n_parts items owns n_parts level-0 partial records starting at rec_base,
-// followed by the records of its combine tree (fan-in kMergeFanIn), and one ticket counter per tree
-// node starting at ticket_base.
+// appends).  A head cut into n_parts > 1 items owns n_parts partial records starting at rec_base, which
+// the combine kernel merges; a head in one part writes its output directly.
 struct WorkItem {
   int32_t head;       // b * Hkv + kv_head
   int32_t page_begin;
@@ -39,7 +36,14 @@ struct WorkItem {
   int32_t part_idx;   // index of this part within its head
   int32_t n_parts;    // parts of this head
   int32_t rec_base;
-  int32_t ticket_base;
+  int32_t pad0, pad1;
+};
+
+// A head whose stream was cut into several parts: one entry of the combine kernel's work list.
+struct MultiHead {
+  int32_t head;       // b * Hkv + kv_head
+  int32_t rec_base;
+  int32_t n_parts;
   int32_t pad;
 };
 
@@ -72,9 +76,9 @@ struct DeviceView {
   int32_t* page_table;      // [L][B*Hkv][max_pages]
   WorkItem* items;          // [L][max_items]
   int32_t* jobs;            // [L][max_items + 1]  first item of every job (a span or one tail item), then n_items
-  float2* rec_ml;           // [max_recs][G]      running max (log2 domain) and denominator of a partial
-  float* rec_o;             // [max_recs][G][D]   un-normalised numerator of a partial
-  int32_t* tickets;         // [max_tickets]      arrival counters of the combine-tree nodes (zero at rest)
+  MultiHead* multi;         // [L][B*Hkv]          heads in several parts (combine kernel's work list)
+  float2* rec_ml;           // [max_items][G]      running max (log2 domain) and denominator of a partial
+  float* rec_o;             // [max_items][G][D]   un-normalised numerator of a partial
   int32_t* queue;           // [4]: next item, CTAs done, spare, spare (zero at rest)
   int32_t* status;          // [1]: kStatus* bits, sticky until razor_cache_device_status clears them
   float* compress_scratch;  // [B*Hkv][kCompressMaxSlices][2][D]
@@ -83,8 +87,6 @@ struct DeviceView {
   int32_t n_kv_heads;
   int32_t max_pages;        // page-table row length
   int32_t max_items;
-  int32_t max_recs;
-  int32_t max_tickets;
   int32_t head_dim;
   int32_t n_sink;
   int32_t group;
@@ -112,6 +114,7 @@ cudaError_t launch_append(const DeviceView& dv, int dtype, int layer, const void
 // ranges jobs[j]..jobs[j+1]), the others single items starting at tail_first.
 struct DecodeJobs {
   int32_t n_items, n_jobs, n_spans, tail_first;
+  int32_t n_multi;   // heads in several parts
 };
 cudaError_t launch_decode(const DeviceView& dv, int dtype, int layer, const DecodeJobs& jobs, const void* q,
                           float* out, int n_sms, const DecodeTuning& tune, cudaStream_t stream);
@@ -128,16 +131,14 @@ struct SchedParams {
 struct SchedInfo {
   int n_items, n_jobs, n_spans;   // the first n_spans jobs are spans
   int span_pages, chunk_pages;    // size of a span, largest tail item
+  int n_multi;                    // entries written to multi[]
 };
 // pages[h] = pages of head h's token stream now.  Writes the work items in job order to out[] and the
-// first item of each job to jobs[] (n_jobs + 1 entries); lays out each head's partial records and
-// ticket counters.  Returns the number of items (<= max_items), or -1 when items, records or tickets
-// would not fit.
-int build_schedule(const int32_t* pages, int n_heads, const SchedParams& sp, int max_items, int max_recs,
-                   int max_tickets, WorkItem* out, int32_t* jobs, SchedInfo* info);
-
-// Records and tickets a head cut into n_parts items needs (n_parts >= 1).
-void tree_sizes(int n_parts, int* n_recs, int* n_tickets);
+// first item of each job to jobs[] (n_jobs + 1 entries); lays out the partial records of the heads cut
+// into several parts and lists those heads in multi[] (at most n_heads entries).  Returns the number of
+// items (<= max_items), or -1 when they would not fit.
+int build_schedule(const int32_t* pages, int n_heads, const SchedParams& sp, int max_items, WorkItem* out,
+                   int32_t* jobs, MultiHead* multi, SchedInfo* info);
 
 }  // namespace razor
 #endif

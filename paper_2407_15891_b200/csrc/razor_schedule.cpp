@@ -10,8 +10,8 @@
 //   * the rest is cut into small TAIL items (`tail_items_per_cta` per CTA) that the CTAs pull one at
 //     a time as they finish their spans, which evens out whatever difference in speed there was.
 // A job is what a CTA pops from the queue: a span (several consecutive items) or one tail item.
-// A head cut into several parts produces one partial (m, l, o) record per part; records are merged by
-// a tree of fan-in kMergeFanIn whose nodes are closed by whichever CTA delivers a node's last input.
+// A head cut into several parts produces one partial (m, l, o) record per part; a small combine kernel
+// that follows the streaming kernel merges them, one CTA per such head.
 #include <algorithm>
 #include <cstdint>
 #include <numeric>
@@ -20,21 +20,6 @@
 #include "razor_internal.h"
 
 namespace razor {
-
-void tree_sizes(int n_parts, int* n_recs, int* n_tickets) {
-  int recs = 0, tickets = 0;
-  if (n_parts > 1) {
-    int n = n_parts;
-    recs = n;
-    while (n > 1) {
-      n = (n + kMergeFanIn - 1) / kMergeFanIn;
-      tickets += n;          // one counter per node of this level
-      if (n > 1) recs += n;  // the root writes the output, not a record
-    }
-  }
-  *n_recs = recs;
-  *n_tickets = tickets;
-}
 
 namespace {
 
@@ -45,8 +30,8 @@ struct Piece {
 
 }  // namespace
 
-int build_schedule(const int32_t* pages, int n_heads, const SchedParams& sp, int max_items, int max_recs,
-                   int max_tickets, WorkItem* out, int32_t* jobs, SchedInfo* info) {
+int build_schedule(const int32_t* pages, int n_heads, const SchedParams& sp, int max_items, WorkItem* out,
+                   int32_t* jobs, MultiHead* multi, SchedInfo* info) {
   const int n_ctas = std::max(1, sp.n_ctas);
   const int min_chunk = std::max(1, sp.min_chunk_pages);
   const int static_pct = std::min(100, std::max(0, sp.static_pct));
@@ -98,18 +83,16 @@ int build_schedule(const int32_t* pages, int n_heads, const SchedParams& sp, int
     chunk += (chunk + 3) / 4;
   }
 
-  // Per head: lay out records and tickets.
-  std::vector<int> n_parts(n_heads, 0), rec_base(n_heads, 0), ticket_base(n_heads, 0), next_part(n_heads, 0);
+  // Per head: partial records for the heads in several parts (never more records than items).
+  std::vector<int> n_parts(n_heads, 0), rec_base(n_heads, 0), next_part(n_heads, 0);
   for (const Piece& pc : pieces) n_parts[pc.head] += 1;
-  int rec = 0, ticket = 0;
-  for (int h = 0; h < n_heads; ++h) {
-    int nr, nt;
-    tree_sizes(n_parts[h], &nr, &nt);
-    if (rec + nr > max_recs || ticket + nt > max_tickets) return -1;
+  int rec = 0, n_multi = 0;
+  for (int oi = 0; oi < n_heads; ++oi) {   // longest heads first: they have the most parts to merge
+    const int h = order[oi];
+    if (n_parts[h] < 2) continue;
     rec_base[h] = rec;
-    ticket_base[h] = ticket;
-    rec += nr;
-    ticket += nt;
+    multi[n_multi++] = MultiHead{h, rec, n_parts[h], 0};
+    rec += n_parts[h];
   }
   // Job order: spans in stream order, then the tail items.  Jobs are numbered along the stream, so the
   // pieces of one head stay in page order and part indices can be handed out as the pieces come.
@@ -128,8 +111,7 @@ int build_schedule(const int32_t* pages, int n_heads, const SchedParams& sp, int
     w.part_idx = next_part[pc.head]++;
     w.n_parts = n_parts[pc.head];
     w.rec_base = rec_base[pc.head];
-    w.ticket_base = ticket_base[pc.head];
-    w.pad = 0;
+    w.pad0 = w.pad1 = 0;
     out[n++] = w;
   }
   jobs[n_jobs] = n;
@@ -139,6 +121,7 @@ int build_schedule(const int32_t* pages, int n_heads, const SchedParams& sp, int
     info->n_spans = first_tail_job < 0 ? n_jobs : first_tail_job;
     info->span_pages = (int)span;
     info->chunk_pages = (int)chunk;
+    info->n_multi = n_multi;
   }
   return n;
 }
