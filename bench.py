@@ -53,6 +53,21 @@ def parse_args():
     return ap.parse_args()
 
 
+def max_over_ranks(ms: float, dist, device) -> float:
+    """The slowest rank's time (every rank runs an independent replica; the job is as slow as that one)."""
+    if dist is None:
+        return ms
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replica_throughput(world: int, bytes_per_rank: float, ms: float) -> float:
+    """Whole-job GB/s of `world` replicas that each moved bytes_per_rank in ms (the max over ranks)."""
+    return world * bytes_per_rank / (ms * 1e-3) / 1e9
+
+
 def measured_peak():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -376,13 +391,9 @@ def main():
     clocks = sampler.stop()
     n_launches = launches["n"]
 
-    total_ms = starts[0].elapsed_time(ends[-1])
-    if dist is not None:
-        tt = torch.tensor([total_ms], device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms = float(tt.item())
+    total_ms = max_over_ranks(starts[0].elapsed_time(ends[-1]), dist, dev)
     ms_per_step = total_ms / args.steps
-    value = world * attended / (ms_per_step * 1e-3) / 1e9
+    value = replica_throughput(world, attended, ms_per_step)
 
     comp_ms = statistics.mean(s.elapsed_time(c) for s, c in zip(starts, comp_ends))
     dec_phase_ms = statistics.mean(c.elapsed_time(e) for c, e in zip(comp_ends, ends))
@@ -494,12 +505,8 @@ def main():
             e2e_pass(count=(i == 0))
         b.record()
         sync_all()
-        e_ms = a.elapsed_time(b) / e2e_steps
-        if dist is not None:
-            tt = torch.tensor([e_ms], device=dev)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            e_ms = float(tt.item())
-        line["e2e"] = {"value": world * attended / (e_ms * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d,
+        e_ms = max_over_ranks(a.elapsed_time(b) / e2e_steps, dist, dev)
+        line["e2e"] = {"value": replica_throughput(world, attended, e_ms), "unit": UNIT, "h2d_bytes_per_step": h2d,
                        "d2h_bytes_per_step": d2h, "ms_per_step": e_ms, "steps": e2e_steps,
                        "note": "host-pinned dense K/V, q, k_new, v_new copied in and out[] copied back inside the "
                                "timed region" + ("; cfg5 dense K/V stay on the device (75 GB of host staging "
