@@ -165,8 +165,10 @@ RAZOR_API int razor_cache_stats(const razor_cache_t* cache, int32_t layer, size_
  * The decode work schedule (host only; no device is touched).  The page streams of all (sequence,
  * KV head) pairs are laid end to end, longest first.  The first static_percent of the pages is cut
  * into one equal span per CTA (a span that crosses a head boundary becomes several work items, one
- * per head); the rest is cut into small tail items, about tail_items_per_cta per CTA, which the CTAs
- * pull one by one when their span is done.  A job is what a CTA pulls: a span or one tail item.
+ * per head); the rest is cut into tail items which the CTAs pull one by one when their span is done.
+ * Tail items shrink along the stream: each is 1 / tail_items_per_cta of an equal share of the tail
+ * still left, but at least min_chunk_pages (and never across a head boundary).  A job is what a CTA
+ * pulls: a span or one tail item.
  *   razor_schedule_plan   plans for given stream lengths: tokens host int32[n_heads] (tokens stored
  *                         per head), n_ctas >= 1 (the SM count), 0 <= static_percent <= 100,
  *                         tail_items_per_cta >= 1, min_chunk_pages >= 1 (smallest span / tail item).
@@ -187,15 +189,16 @@ RAZOR_API int razor_schedule_query(razor_cache_t* cache, int32_t layer, int32_t*
  * next razor_decode_attention.  Errors: NULL_PTR, INVALID_ARG (unknown option or value out of range).
  */
 enum {
-  RAZOR_OPT_DECODE_TAIL_ITEMS_PER_SM = 1, /* tail items aimed for per SM (1..1024; default 4)             */
-  RAZOR_OPT_DECODE_MIN_CHUNK_PAGES = 2, /* smallest span or tail item in pages (default 8)                */
+  RAZOR_OPT_DECODE_TAIL_ITEMS_PER_SM = 1, /* a tail item is 1/k of an SM's share of the remaining tail
+                                             (k = 1..1024; default 3)                                      */
+  RAZOR_OPT_DECODE_MIN_CHUNK_PAGES = 2, /* smallest span or tail item in pages (default 16)               */
   RAZOR_OPT_DECODE_RING_KB = 3,         /* shared-memory page ring per CTA in KiB; 0 = as large as fits   */
   RAZOR_OPT_DECODE_CONSUMER_WARPS = 4,  /* streaming warps per CTA: 0 = default; 4, 8, 12 or 16; a value
                                            the head shape has no kernel for falls back to the default     */
   RAZOR_OPT_DECODE_TENSOR_CORES = 5,    /* bf16 grouped-query heads: 0 = matrix instructions from group 4
                                            up (default), 1 = from group 2 up, 2 = never                   */
   RAZOR_OPT_DECODE_STATIC_PERCENT = 6   /* share of the pages handed out as per-CTA spans (0..100;
-                                           default 85); 0 makes every job a tail item                     */
+                                           default 80); 0 makes every job a tail item                     */
 };
 RAZOR_API int razor_cache_set_option(razor_cache_t* cache, int32_t option, int32_t value);
 

@@ -196,8 +196,8 @@ def razor_cache_stats(cache: int, layer: int) -> Tuple[int, int]:
     return k.value, d.value
 
 
-def razor_schedule_plan(tokens, n_ctas: int = 148, static_percent: int = 85, tail_items_per_cta: int = 4,
-                        min_chunk_pages: int = 8, with_spans: bool = False):
+def razor_schedule_plan(tokens, n_ctas: int = 148, static_percent: int = 80, tail_items_per_cta: int = 3,
+                        min_chunk_pages: int = 16, with_spans: bool = False):
     """Host-only: -> int32 [n_items, 5] = (head, first_page, end_page (-1: open), parts_of_head, job) in job
     order (and the number of span jobs when with_spans is set)."""
     t = _i32(tokens)

@@ -119,7 +119,7 @@ struct razor_cache {
   DeviceView dv;
   long long pool_pages = 0, next_page = 0;
   int n_sms = 148;
-  DecodeTuning tune{4, 85, 8, 0, 0, 0};
+  DecodeTuning tune{3, 80, 16, 0, 0, 0};
   std::vector<LayerHost> layers;
   WorkItem* pinned_items = nullptr;   // [L][max_items]
   int32_t* pinned_jobs = nullptr;     // [L][max_items + 1]

@@ -118,6 +118,7 @@ __global__ void __launch_bounds__(128) append_kernel(DeviceView dv, int layer, c
   constexpr int LPR = Geo::kLpr, EPL = Geo::kEpl;
   const int lane = threadIdx.x & 31;
   const int head = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  cudaTriggerProgrammaticLaunchCompletion();   // the decode kernel queued behind the append may set itself up
   if (head >= dv.n_heads) return;
   const size_t hs = (size_t)layer * dv.n_heads + head;
   HeadState st = dv.state[hs];

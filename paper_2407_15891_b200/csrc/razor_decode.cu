@@ -447,6 +447,10 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   __syncthreads();
+  // This kernel is launched as a programmatic dependent of whatever precedes it on the stream (the
+  // append or an earlier combine), so everything above overlaps that kernel's tail; nothing that kernel
+  // wrote is touched before this point.
+  cudaGridDependencySynchronize();
   // The combine kernel that follows may be made resident as soon as SMs free up; it waits for this whole
   // grid to finish before it reads anything this grid writes.
   cudaTriggerProgrammaticLaunchCompletion();
@@ -864,11 +868,11 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
 // ------------------------------------------------------------------------------------------ combine
 // Merges the partial records of the heads that were cut into several parts (Eq. 5 regrouped: sums of
 // exponentials under a common maximum).  One CTA per (such head, query head of its group); warp w folds
-// records w, w + 8, ... in that order and the eight warp states are folded in warp order, so the result
+// records w, w + 16, ... in that order and the warp states are folded in warp order, so the result
 // does not depend on timing.  Launched as a programmatic dependent of the streaming kernel: its CTAs
 // may become resident while that kernel drains, and wait for all of its writes at
 // cudaGridDependencySynchronize().
-constexpr int kCombineWarps = 8;
+constexpr int kCombineWarps = 16;
 
 template <int D>
 __global__ void __launch_bounds__(kCombineWarps * 32) combine_kernel(DeviceView dv, int layer, float* __restrict__ out) {
@@ -877,6 +881,7 @@ __global__ void __launch_bounds__(kCombineWarps * 32) combine_kernel(DeviceView 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = dv.group, j = blockIdx.y;
   const MultiHead mh = dv.multi[(size_t)layer * dv.n_heads + blockIdx.x];   // uploaded before either kernel
+  cudaTriggerProgrammaticLaunchCompletion();   // a decode kernel queued behind this one may set itself up
   cudaGridDependencySynchronize();   // the streaming kernel's records are complete and visible from here on
   float m = -CUDART_INF_F, l = 0.f;
   LaneVec<D> acc;
@@ -979,8 +984,17 @@ cudaError_t decode_launch(const DeviceView& dv, int layer, const DecodeJobs& jb,
   }
   int grid = std::min(n_sms, (int)jb.n_jobs);
   if (grid < 1) grid = 1;
-  kern<<<grid, (NC + 2) * 32, dyn, s>>>(dv, layer, jb, (const T*)q, out, (int)stages);
-  if ((e = cudaGetLastError()) != cudaSuccess) return e;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3((NC + 2) * 32);
+  cfg.dynamicSmemBytes = dyn;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if ((e = cudaLaunchKernelEx(&cfg, kern, dv, layer, jb, (const T*)q, out, (int)stages)) != cudaSuccess) return e;
   return combine_launch<D>(dv, layer, jb.n_multi, out, s);
 }
 

@@ -7,8 +7,10 @@
 //   * the first `static_pct` percent is cut into one equal SPAN per CTA.  A span crosses head
 //     boundaries where it must, so it is a short run of work items (one per head it touches), and
 //     the long heads end up in few, large parts;
-//   * the rest is cut into small TAIL items (`tail_items_per_cta` per CTA) that the CTAs pull one at
-//     a time as they finish their spans, which evens out whatever difference in speed there was.
+//   * the rest is cut into TAIL items that the CTAs pull one at a time as they finish their spans, which
+//     evens out whatever difference in speed there was.  Their sizes shrink along the stream (guided
+//     self-scheduling): each is 1 / tail_items_per_cta of an equal share of the tail that is left, but
+//     not less than min_chunk pages, so the queue ends on small items without starting on them.
 // A job is what a CTA pops from the queue: a span (several consecutive items) or one tail item.
 // A head cut into several parts produces one partial (m, l, o) record per part; a small combine kernel
 // that follows the streaming kernel merges them, one CTA per such head.
@@ -50,14 +52,15 @@ int build_schedule(const int32_t* pages, int n_heads, const SchedParams& sp, int
   const long long n_spans = std::min<long long>(n_ctas, static_pages / span);
   const long long static_end = n_spans * span;
   const long long tail_pages = total - static_end;
-  long long chunk = (tail_pages + (long long)n_ctas * tail_per_cta - 1) / ((long long)n_ctas * tail_per_cta);
-  if (chunk < min_chunk) chunk = min_chunk;
+  long long floor_chunk = min_chunk;   // smallest tail item; grows only if the items would not fit
+  long long first_chunk = 0;
 
   std::vector<Piece> pieces;
-  for (;;) {   // grow the tail chunk until the items fit
+  for (;;) {   // grow the smallest tail item until the items fit
     pieces.clear();
-    long long pos = 0;
+    long long pos = 0, tail_left = tail_pages;
     int tail_jobs = 0;
+    first_chunk = 0;
     for (int oi = 0; oi < n_heads; ++oi) {
       const int h = order[oi];
       const int p = pages[h];
@@ -68,19 +71,22 @@ int build_schedule(const int32_t* pages, int n_heads, const SchedParams& sp, int
         pieces.push_back({h, at, stop, (int)k});
         at = stop;
       }
-      if (at < p || p == 0) {   // dynamic region: equal parts of at most `chunk` pages; an empty head gets one empty item
-        const int len = p - at;
-        const int parts = std::max(1, (int)((len + chunk - 1) / chunk));
-        for (int i = 0; i < parts; ++i) {
-          const int b = at + (int)((long long)len * i / parts), e = at + (int)((long long)len * (i + 1) / parts);
-          pieces.push_back({h, b, e, (int)n_spans + tail_jobs++});
-        }
+      if (p == 0) pieces.push_back({h, 0, 0, (int)n_spans + tail_jobs++});   // an empty head gets one empty item
+      while (at < p) {   // dynamic region: guided sizes, cut at the head's end
+        long long chunk = (tail_left + (long long)n_ctas * tail_per_cta - 1) / ((long long)n_ctas * tail_per_cta);
+        if (chunk < floor_chunk) chunk = floor_chunk;
+        if (first_chunk == 0) first_chunk = chunk;
+        int stop = (int)std::min<long long>(p, at + chunk);
+        if (p - stop < floor_chunk / 2) stop = p;   // no crumbs at the end of a head
+        pieces.push_back({h, at, stop, (int)n_spans + tail_jobs++});
+        tail_left -= stop - at;
+        at = stop;
       }
       pos += p;
     }
     if ((long long)pieces.size() <= max_items) break;
-    if (chunk > total) return -1;
-    chunk += (chunk + 3) / 4;
+    if (floor_chunk > total) return -1;
+    floor_chunk += (floor_chunk + 3) / 4;
   }
 
   // Per head: partial records for the heads in several parts (never more records than items).
@@ -120,7 +126,7 @@ int build_schedule(const int32_t* pages, int n_heads, const SchedParams& sp, int
     info->n_jobs = n_jobs;
     info->n_spans = first_tail_job < 0 ? n_jobs : first_tail_job;
     info->span_pages = (int)span;
-    info->chunk_pages = (int)chunk;
+    info->chunk_pages = (int)floor_chunk;
     info->n_multi = n_multi;
   }
   return n;

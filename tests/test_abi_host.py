@@ -171,11 +171,16 @@ def test_schedule_covers_every_page_once_and_is_balanced(tokens, n_ctas, pct, ta
     assert (np.bincount(jobs)[n_spans:] == 1).all()            # a tail job is one item
     if len(tail_sizes):
         tail_total = int(tail_sizes.sum())
-        chunk = max(min_chunk, -(-tail_total // (n_ctas * tail)))
-        if len(tokens) + n_spans + tail_total // chunk <= 16384:
-            assert tail_sizes.max() <= chunk
-        else:                                                  # the chunk grew until the items fit the budget
-            assert tail_sizes.max() - tail_sizes[tail_sizes > 0].min() <= 1
+        first = max(min_chunk, -(-tail_total // (n_ctas * tail)))
+        if len(tokens) + n_spans + 4 * n_ctas * tail + tail_total // max(min_chunk, 1) <= 16384:
+            # guided sizes: nothing larger than the first chunk (plus the crumb a head's end may add),
+            # and the sizes never grow along the stream except where a head ended early
+            assert tail_sizes.max() <= first + min_chunk // 2
+            left = tail_total
+            for sz in tail_sizes:
+                bound = max(min_chunk, -(-left // (n_ctas * tail)))
+                assert sz <= bound + min_chunk // 2
+                left -= int(sz)
     assert len(items) <= len(tokens) + 16384
 
 
