@@ -446,6 +446,40 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
+  const WorkItem* items = dv.items + (size_t)layer * dv.max_items;
+  const int32_t* jobs = dv.jobs + (size_t)layer * (dv.max_items + 1);
+  const int n_items = jb.n_items;
+  const WorkItem no_item = {0, 0, 0, 0, 1, 0, 0, 0};
+  auto row_of = [&](const WorkItem& w) { return (size_t)layer * dv.n_heads + w.head; };
+  auto first_pids = [&](const WorkItem& w) {
+    return dv.page_table[row_of(w) * dv.max_pages + min(w.page_begin + lane, dv.max_pages - 1)];
+  };
+  // A job is a run of consecutive items: a span (looked up in jobs[]) or a single tail item (tail
+  // jobs follow the spans and map to consecutive items, so they need no lookup).
+  auto job_range = [&](int j, int& first, int& end) {
+    if (j >= jb.n_jobs) {
+      first = end = n_items;
+    } else if (j >= jb.n_spans) {
+      first = jb.tail_first + (j - jb.n_spans);
+      end = first + 1;
+    } else {
+      first = jobs[j];
+      end = jobs[j + 1];
+    }
+  };
+  // The spans are handed out by CTA index and the queue counts tail jobs only, so the producer can look
+  // up its span, the span's first item and that item's first page ids right here: the schedule and the
+  // page table are written by host copies only, never by a kernel, and may be read before the
+  // dependency below is resolved.
+  int it0 = n_items, job_end0 = n_items;
+  WorkItem w0 = no_item;
+  int32_t pid0 = 0;
+  const bool has_span = (int)blockIdx.x < jb.n_spans;
+  if (warp == NC && has_span) {
+    job_range((int)blockIdx.x, it0, job_end0);
+    w0 = it0 < n_items ? items[it0] : no_item;
+    pid0 = first_pids(w0);
+  }
   __syncthreads();
   // This kernel is launched as a programmatic dependent of whatever precedes it on the stream (the
   // append or an earlier combine), so everything above overlaps that kernel's tail; nothing that kernel
@@ -455,9 +489,6 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
   // grid to finish before it reads anything this grid writes.
   cudaTriggerProgrammaticLaunchCompletion();
 
-  const WorkItem* items = dv.items + (size_t)layer * dv.max_items;
-  const int32_t* jobs = dv.jobs + (size_t)layer * (dv.max_items + 1);
-  const int n_items = jb.n_items;
   const int n_q_heads = dv.n_kv_heads * G;
   // Warp-uniform bounded wait: false for every lane if any lane's wait failed.
   auto warp_wait = [&](uint64_t* bar, uint32_t parity) -> bool {
@@ -477,33 +508,17 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
     // Look-ahead of one item: the next item's queue pop, its descriptor, its head state and its first
     // page ids are requested while the current item's pages are being issued, so that the ring is not
     // left to drain over a chain of dependent global loads at every item boundary.
-    const WorkItem no_item = {0, 0, 0, 0, 1, 0, 0, 0};
-    auto row_of = [&](const WorkItem& w) { return (size_t)layer * dv.n_heads + w.head; };
-    auto first_pids = [&](const WorkItem& w) {
-      return dv.page_table[row_of(w) * dv.max_pages + min(w.page_begin + lane, dv.max_pages - 1)];
-    };
-    // A job is a run of consecutive items: a span (looked up in jobs[]) or a single tail item (tail
-    // jobs follow the spans and map to consecutive items, so they need no lookup).
-    auto job_range = [&](int j, int& first, int& end) {
-      if (j >= jb.n_jobs) {
-        first = end = n_items;
-      } else if (j >= jb.n_spans) {
-        first = jb.tail_first + (j - jb.n_spans);
-        end = first + 1;
-      } else {
-        first = jobs[j];
-        end = jobs[j + 1];
-      }
-    };
-    int it = 0, job_end = 0;
-    {
+    int it = it0, job_end = job_end0;
+    WorkItem w = w0;
+    int32_t pid_first = pid0;
+    if (!has_span) {   // more CTAs than spans: start on the tail
       int j = 0;
       if (lane == 0) j = atomicAdd(dv.queue, 1);
-      job_range(__shfl_sync(0xffffffffu, j, 0), it, job_end);
+      job_range(jb.n_spans + __shfl_sync(0xffffffffu, j, 0), it, job_end);
+      w = it < n_items ? items[it] : no_item;
+      pid_first = first_pids(w);
     }
-    WorkItem w = it < n_items ? items[it] : no_item;
     HeadState st = dv.state[row_of(w)];
-    int32_t pid_first = first_pids(w);
     for (unsigned seq = 0; ok; ++seq) {
       const int slot = seq % kItemSlots;
       const bool need_pop = it < n_items && it + 1 >= job_end;   // the job ends with this item
@@ -579,14 +594,14 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
         c += in_batch;
         pid_cur = pid_after;
         if (!have_next) {   // the pop issued above has had a round of copies to come back
-          if (need_pop) job_range(__shfl_sync(0xffffffffu, next_raw, 0), it_next, end_next);
+          if (need_pop) job_range(jb.n_spans + __shfl_sync(0xffffffffu, next_raw, 0), it_next, end_next);
           w_next = it_next < n_items ? items[it_next] : no_item;
           have_next = true;
         }
       }
       if (!ok) break;
       if (!have_next) {
-        if (need_pop) job_range(__shfl_sync(0xffffffffu, next_raw, 0), it_next, end_next);
+        if (need_pop) job_range(jb.n_spans + __shfl_sync(0xffffffffu, next_raw, 0), it_next, end_next);
         w_next = it_next < n_items ? items[it_next] : no_item;
       }
       it = it_next;
