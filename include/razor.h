@@ -208,9 +208,18 @@ RAZOR_API int razor_cache_set_option(razor_cache_t* cache, int32_t option, int32
  * This call synchronises `stream`, stores the word in *status (0 = healthy) and, when it is non-zero,
  * clears it together with the kernel's work counters so that the cache can be used again; outputs of
  * the affected launch are undefined.  Bits: 1 producer wait, 2 consumer wait, 4 reducer wait, 8 copies
- * still in flight at exit.  Errors: NULL_PTR, CUDA.
+ * still in flight at exit, 16 the self-test below.  Errors: NULL_PTR, CUDA.
  */
 RAZOR_API int razor_cache_device_status(razor_cache_t* cache, int32_t* status, void* stream);
+
+/*
+ * Self-test of the bounded waits.  Enqueues a one-warp kernel that waits, with the decode kernel's own
+ * wait routine and a limit of limit_ns (1 us .. 1 s), on a barrier nothing ever arrives on.  The wait
+ * has to give up by itself; razor_cache_device_status then reports bit 16 (and clears it), and the
+ * cache stays usable.  Nothing faults, traps or spins without bound.
+ * Errors: NULL_PTR, INVALID_ARG, CUDA.
+ */
+RAZOR_API int razor_cache_wait_selftest(razor_cache_t* cache, int64_t limit_ns, void* stream);
 
 /*
  * The compensation token of the KV heads of ONE sequence without a cache, a pool or a workspace.

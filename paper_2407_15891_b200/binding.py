@@ -27,7 +27,7 @@ STATUS = {
 SYMBOLS = [
     "razor_query_bytes", "razor_cache_create", "razor_compress", "razor_compress_seq", "razor_append",
     "razor_decode_attention", "razor_cache_export", "razor_cache_stats", "razor_schedule_plan",
-    "razor_schedule_query", "razor_cache_set_option", "razor_cache_device_status", "razor_compensation_mean_static",
+    "razor_schedule_query", "razor_cache_set_option", "razor_cache_device_status", "razor_cache_wait_selftest", "razor_compensation_mean_static",
     "razor_cache_reset", "razor_cache_destroy", "razor_status_string",
     "razor_last_cuda_error", "razor_version",
 ]
@@ -80,6 +80,7 @@ def load() -> C.CDLL:
     lib.razor_schedule_query.argtypes = [vp, i32, vp, i32, C.POINTER(i32)]
     lib.razor_compensation_mean_static.argtypes = [vp, vp, i64, i64, i32, i32, i32, i32, i32, i32, vp, vp,
                                                    C.POINTER(i32), vp]
+    lib.razor_cache_wait_selftest.argtypes = [vp, i64, vp]
     lib.razor_cache_reset.argtypes = [vp]
     lib.razor_cache_destroy.argtypes = [vp]
     lib.razor_status_string.argtypes = [C.c_int]
@@ -232,6 +233,11 @@ def razor_schedule_query(cache: int, layer: int) -> np.ndarray:
     items = np.zeros((n.value, 5), dtype=np.int32)
     _check(lib.razor_schedule_query(cache, layer, items.ctypes.data, n.value, C.byref(n)), "razor_schedule_query")
     return items
+
+
+def razor_cache_wait_selftest(cache: int, limit_ns: int, stream=None) -> None:
+    """Enqueue the kernel whose (bounded) wait nothing answers; razor_cache_device_status then shows bit 16."""
+    _check(load().razor_cache_wait_selftest(cache, limit_ns, _stream(stream)), "razor_cache_wait_selftest")
 
 
 def razor_compensation_mean_static(K, V, stride_h: int, stride_n: int, n_kv_heads: int, head_dim: int, dtype: int,

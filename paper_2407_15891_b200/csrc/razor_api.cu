@@ -642,6 +642,13 @@ int razor_cache_device_status(razor_cache_t* c, int32_t* status, void* stream) {
   return RAZOR_OK;
 }
 
+int razor_cache_wait_selftest(razor_cache_t* c, int64_t limit_ns, void* stream) {
+  if (!c) return RAZOR_E_NULL_PTR;
+  if (limit_ns < 1000 || limit_ns > 1000000000ll) return RAZOR_E_INVALID_ARG;
+  RZ_CUDA(launch_wait_selftest(c->dv, (unsigned long long)limit_ns, (cudaStream_t)stream));
+  return RAZOR_OK;
+}
+
 int razor_schedule_query(razor_cache_t* c, int32_t layer, int32_t* items, int32_t max_items, int32_t* n_items) {
   if (!c || !n_items) return RAZOR_E_NULL_PTR;
   int rc = layer_ready(c, layer);

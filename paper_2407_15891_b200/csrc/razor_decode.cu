@@ -71,13 +71,14 @@ __device__ __forceinline__ unsigned long long global_ns() {
 }
 // Bounded wait for the phase of `bar` with the given parity.  False: the CTA is aborting (this wait ran
 // out of time, or another warp's did).
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                          unsigned long long limit_ns = kWaitLimitNs) {
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = global_ns();
   for (;;) {
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (global_ns() - t0 > kWaitLimitNs) {
+    if (global_ns() - t0 > limit_ns) {
       *abort_flag = 1;
       return false;
     }
@@ -1050,7 +1051,28 @@ cudaError_t decode_g(const DeviceView& dv, int layer, const DecodeJobs& jb, cons
   return cudaErrorInvalidValue;
 }
 
+// One warp waits, with the decode kernel's own bounded wait, on a barrier that nothing will ever arrive
+// on.  The wait must give up after limit_ns, raise the abort flag and report through the status word:
+// a check that the safety net under every wait of the decode kernel works, without hanging anything.
+__global__ void wait_selftest_kernel(DeviceView dv, unsigned long long limit_ns) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag_s;
+  if (threadIdx.x == 0) {
+    abort_flag_s = 0;
+    mbar_init(&bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  const bool ok = mbar_wait(&bar, 0, &abort_flag_s, limit_ns);
+  if (!ok && threadIdx.x == 0) atomicOr(dv.status, kStatusSelfTest);
+}
+
 }  // namespace
+
+cudaError_t launch_wait_selftest(const DeviceView& dv, unsigned long long limit_ns, cudaStream_t s) {
+  wait_selftest_kernel<<<1, 32, 0, s>>>(dv, limit_ns);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_decode(const DeviceView& dv, int dtype, int layer, const DecodeJobs& jb, const void* q, float* out,
                           int n_sms, const DecodeTuning& tune, cudaStream_t s) {

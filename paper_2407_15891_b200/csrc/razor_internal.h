@@ -64,7 +64,8 @@ enum : int32_t {
   kStatusProducerTimeout = 1,   // the copy-issuing warp gave up waiting for a free ring stage or item slot
   kStatusConsumerTimeout = 2,   // a streaming warp gave up waiting for a page or an item
   kStatusReducerTimeout = 4,    // the merging warp gave up waiting for the streaming warps' states
-  kStatusDrainTimeout = 8       // copies were still in flight when the abort path stopped waiting for them
+  kStatusDrainTimeout = 8,      // copies were still in flight when the abort path stopped waiting for them
+  kStatusSelfTest = 16          // razor_cache_wait_selftest: the deliberately unanswered wait gave up, as it must
 };
 
 // Pointers into the caller's workspace, plus the dimensions the kernels need.
@@ -118,6 +119,7 @@ struct DecodeJobs {
 };
 cudaError_t launch_decode(const DeviceView& dv, int dtype, int layer, const DecodeJobs& jobs, const void* q,
                           float* out, int n_sms, const DecodeTuning& tune, cudaStream_t stream);
+cudaError_t launch_wait_selftest(const DeviceView& dv, unsigned long long limit_ns, cudaStream_t stream);
 cudaError_t launch_export(const DeviceView& dv, int dtype, int layer, int head, int32_t* kept_pos, void* K, void* V,
                           float* mean_k, float* mean_v, float* sum_k, float* sum_v, cudaStream_t stream);
 

@@ -220,6 +220,29 @@ def test_error_codes_on_a_live_cache():
     cache.close()
 
 
+def test_a_wait_that_nothing_answers_gives_up_and_reports():
+    """Failure detection without a fault: the decode kernel's wait routine, pointed at a barrier nobody
+    arrives on, returns after its limit, the status word says so, and the cache goes on working."""
+    import time
+    w = synth.workload("cfg2", 1 / 32)
+    cache = make_cache(w)
+    K, V = synth.make_dense_kv(w, 0, DEV)
+    q = synth.make_queries(w, 0, 0, DEV)
+    cache.compress(0, K, V, w.ctx_len, w.retrieval(0), w.window)
+    before = cache.decode(0, q).clone()
+    assert cache.device_status() == 0
+    t0 = time.perf_counter()
+    rz.razor_cache_wait_selftest(cache.handle, 2_000_000)           # 2 ms
+    status = cache.device_status()                                  # synchronises
+    assert time.perf_counter() - t0 < 1.0
+    assert status == 16
+    assert cache.device_status() == 0                               # reading it cleared it
+    assert (bits(cache.decode(0, q)) == bits(before)).all()         # the context and the cache are healthy
+    with pytest.raises(rz.RazorError):
+        rz.razor_cache_wait_selftest(cache.handle, 10)              # limit out of range
+    cache.close()
+
+
 def test_recompress_reuses_pages_and_reset_frees_them():
     w = synth.workload("cfg2", 1 / 32)
     w.decode_steps = 2
