@@ -34,7 +34,7 @@ NOMINAL_HBM_GBS = 8000.0        # the "~8 TB/s" the target is quoted against
 FALLBACK_HBM_GBS = 6650.0       # used only when MEASURED_PEAKS.json is absent
 # DRAM traffic of the decode kernel per algorithmic byte, from the ncu capture summarised in
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over the algorithmic bytes of the launch).
-DECODE_TRAFFIC_PER_ALG_BYTE = None
+DECODE_TRAFFIC_PER_ALG_BYTE = 1.008
 
 
 def parse_args():
