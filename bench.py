@@ -32,8 +32,10 @@ METRIC = "compressed_cache_decode_attention_GBps"
 UNIT = "GB/s"
 NOMINAL_HBM_GBS = 8000.0        # the "~8 TB/s" the target is quoted against
 FALLBACK_HBM_GBS = 6650.0       # used only when MEASURED_PEAKS.json is absent
-# DRAM traffic of the decode kernel per algorithmic byte, from the ncu capture summarised in
-# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over the algorithmic bytes of the launch).
+# DRAM traffic of the decode kernel per algorithmic byte: (dram__bytes_read.sum + dram__bytes_write.sum) of one launch
+# over the kept K+V bytes of that launch, from the ncu capture summarised in
+# profiles/decode_kernel_cfg3_half_scale_and_cfg4_ncu_full.md (taken on the half-scale case; traffic grows in
+# proportion to the kept tokens, so the ratio carries over to the full-size launch).  Set to None when the kernel changes.
 DECODE_TRAFFIC_PER_ALG_BYTE = 1.008
 
 
