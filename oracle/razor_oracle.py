@@ -217,3 +217,32 @@ def compression_ratio(n_ctx: int, n_heads: int, n_retrieval: int, n_sink: int, s
     cached = n_retrieval * kept_token_count(n_ctx, n_sink, w, True) \
         + (n_heads - n_retrieval) * kept_token_count(n_ctx, n_sink, w, False)
     return n_heads * n_ctx / cached
+
+
+# --------------------------------------------------------------------------- several new tokens at once
+def multi_query_attention(qs: np.ndarray, K_all: np.ndarray, V_all: np.ndarray, n_sink: int, window: int,
+                          is_retrieval: bool, scale: float, use_compensation: bool = True) -> np.ndarray:
+    """Attention of the LAST T tokens of a sequence, all against the cache as it stands after the T-th one.
+
+    The paper runs Algorithm 1 once on the prompt and is silent on rounds that add several tokens at
+    once (a second prompt, a verify step).  Reading taken: the cache holds the compression of the whole
+    (N + T)-token history with the window fixed (as for single appends); query t = 0..T-1 sits at
+    position N + t and attends, by causality (Section 3.1: n <= m), to the kept tokens at positions
+    <= N + t, plus the compensation token of Eq. 4 over every dropped token with its count N_d (Eq. 5).
+    All dropped tokens precede every query as long as window >= T, which callers must ensure.
+
+    qs: [T, D]; K_all, V_all: [N + T, D] dense history of one KV head.  Returns [T, D].
+    """
+    qs = np.asarray(qs, dtype=np.float64)
+    T = qs.shape[0]
+    total = int(np.asarray(K_all).shape[0])
+    hc = compress_head(K_all, V_all, total, n_sink, window, is_retrieval)
+    if hc.n_drop > 0:
+        assert window >= T, "a query would see the mean of tokens that come after it"
+    out = np.zeros((T, qs.shape[1]), dtype=np.float64)
+    for t in range(T):
+        q_pos = total - T + t
+        vis = hc.kept_pos <= q_pos
+        n_d = hc.n_drop if use_compensation else 0
+        out[t] = compensated_attention(qs[t], np.asarray(hc.K)[vis], np.asarray(hc.V)[vis], hc.k_hat, hc.v_hat, n_d, scale)
+    return out

@@ -355,3 +355,49 @@ def test_needle_is_recalled_only_by_the_retrieval_head():
     assert err0 < 0.05
     for h in (1, 2, 3):
         assert np.abs(out[0, h] - V[0, h, 200]).max() > 0.5
+
+
+# ------------------------------------------------------------------ several new tokens at once (verify step)
+def test_multi_query_single_token_is_the_decode_step():
+    rng = _rng(70)
+    K, V, q = rng.standard_normal((90, 16)), rng.standard_normal((90, 16)), rng.standard_normal((1, 16))
+    for retr in (False, True):
+        a = orc.multi_query_attention(q, K, V, 4, 20, retr, 0.3)[0]
+        b = orc.decode_head(q[0], orc.compress_head(K, V, 90, 4, 20, retr), 0.3)
+        assert np.allclose(a, b, rtol=0, atol=1e-14)
+
+
+def test_multi_query_on_a_full_cache_is_causal_full_attention():
+    """Retrieval head, or a window covering everything: query t equals brute-force attention over the
+    first N + t + 1 tokens, and tokens after a query do not influence it."""
+    rng = _rng(71)
+    n, T, d = 37, 5, 8
+    K, V, qs = rng.standard_normal((n + T, d)), rng.standard_normal((n + T, d)), rng.standard_normal((T, d))
+    for retr, win in ((True, 3), (False, 100)):
+        out = orc.multi_query_attention(qs, K, V, 2, max(win, T), retr, 0.5)
+        for t in range(T):
+            ref = brute_full_attention(qs[t], K[: n + t + 1], V[: n + t + 1], 0.5)
+            assert np.allclose(out[t], ref, rtol=0, atol=1e-12)
+    K2, V2 = K.copy(), V.copy()
+    K2[n + 2:], V2[n + 2:] = 7.0, -3.0                        # change what comes after query 1
+    a = orc.multi_query_attention(qs, K, V, 2, 10, False, 0.5)
+    b = orc.multi_query_attention(qs, K2, V2, 2, 10, False, 0.5)
+    assert np.allclose(a[:2], b[:2], rtol=0, atol=1e-14) and not np.allclose(a[2:], b[2:])
+
+
+def test_multi_query_equals_eq5_with_replicated_compensation_token_and_causal_mask():
+    rng = _rng(72)
+    n, T, d, n0, w = 60, 4, 8, 3, 9
+    K, V, qs = rng.standard_normal((n + T, d)), rng.standard_normal((n + T, d)), rng.standard_normal((T, d))
+    out = orc.multi_query_attention(qs, K, V, n0, w, False, 0.4)
+    total = n + T
+    drop = np.arange(n0, total - w)
+    k_hat, v_hat = K[drop].mean(0), V[drop].mean(0)
+    for t in range(T):
+        kept = [p for p in range(total) if (p < n0 or p >= total - w) and p <= n + t]
+        Kx = np.concatenate([K[kept], np.repeat(k_hat[None], len(drop), 0)])
+        Vx = np.concatenate([V[kept], np.repeat(v_hat[None], len(drop), 0)])
+        ref = scipy_softmax(0.4 * Kx @ qs[t]) @ Vx
+        assert np.allclose(out[t], ref, rtol=0, atol=1e-12)
+    with pytest.raises(AssertionError):
+        orc.multi_query_attention(qs, K, V, n0, T - 1, False, 0.4)   # window shorter than the round
