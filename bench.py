@@ -226,7 +226,7 @@ def _workload_config(w, args):
 
 
 # ---------------------------------------------------------------------------------------------- GPU legs
-def decode_only(rz, synth, name, n_layers, dev, peak, reps=60):
+def decode_only(rz, synth, name, n_layers, dev, peak, reps=60, n_tok=1):
     """Decode attention alone on the first n_layers layers of another workload (each layer compressed from
     one seeded dense buffer): back-to-back razor_decode_attention calls cycling over the layers, so that
     every call streams pages that the L2 no longer holds."""
@@ -235,7 +235,8 @@ def decode_only(rz, synth, name, n_layers, dev, peak, reps=60):
     w = synth.workload(name)
     w.n_layers = n_layers
     retr = [w.retrieval(l) for l in range(n_layers)]
-    cfg = rz.make_config(w.batch, n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, w.n_sink, max(w.ctx_len), 1)
+    cfg = rz.make_config(w.batch, n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, w.n_sink, max(w.ctx_len),
+                         max(1, n_tok))
     cache = rz.RazorCache(cfg, w.ctx_len, w.window, np.stack(retr), device=dev)
     w0 = synth.Workload(w.name, w.batch, 1, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, w.ctx_len, w.window,
                         w.n_sink, w.n_retrieval_kv, 1, w.seed)
@@ -243,26 +244,38 @@ def decode_only(rz, synth, name, n_layers, dev, peak, reps=60):
     for l in range(n_layers):
         cache.compress(l, K, V, w.ctx_len, retr[l], w.window)
     del K, V
-    q = synth.make_queries(w, 0, 0, dev)
-    out = torch.empty((w.batch, w.n_q_heads, w.head_dim), dtype=torch.float32, device=dev)
+    if n_tok > 1:     # a round of n_tok new tokens per sequence: bulk append, then all their queries in one call
+        kv_shape = (w.batch, n_tok, w.n_kv_heads, w.head_dim)
+        k_new = synth.normal_bf16(w.seed, synth.TAG_KNEW, kv_shape, dev, sub=77)
+        v_new = synth.normal_bf16(w.seed, synth.TAG_VNEW, kv_shape, dev, sub=77)
+        q = synth.normal_bf16(w.seed, synth.TAG_Q, (w.batch, n_tok, w.n_q_heads, w.head_dim), dev, sub=77)
+        out = torch.empty(q.shape, dtype=torch.float32, device=dev)
+        for l in range(n_layers):
+            cache.append_many(l, k_new, v_new)
+        call = cache.decode_multi
+    else:
+        q = synth.make_queries(w, 0, 0, dev)
+        out = torch.empty((w.batch, w.n_q_heads, w.head_dim), dtype=torch.float32, device=dev)
+        call = cache.decode
     for l in range(n_layers):
-        cache.decode(l, q, out)
+        call(l, q, out)
     torch.cuda.synchronize()
     a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
     a.record()
     for i in range(reps):
-        cache.decode(i % n_layers, q, out)
+        call(i % n_layers, q, out)
     b.record()
     torch.cuda.synchronize()
     us = a.elapsed_time(b) * 1e3 / reps
-    kept = w.compressed_bytes(0)
+    kept = w.compressed_bytes(0, extra=n_tok if n_tok > 1 else 0)
     status = cache.device_status()
     cache.close()
     gbs = kept / (us * 1e-6) / 1e9
     return {"workload": f"{name}: batch {w.batch}, {w.n_q_heads}/{w.n_kv_heads} heads, context {max(w.ctx_len)}, "
                         f"{n_layers} layers cycled ({n_layers * kept / 1e9:.2f} GB of pages)",
             "us_per_layer": us, "gbs": gbs, "frac_of_measured": gbs / peak, "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS,
-            "compressed_mb_per_layer": kept / 1e6, "launches_timed": reps, "device_status": status}
+            "compressed_mb_per_layer": kept / 1e6, "launches_timed": reps, "device_status": status,
+            "query_tokens_per_call": n_tok}
 
 
 def main():
@@ -458,6 +471,10 @@ def main():
             line["decode_128k_gqa"] = decode_only(rz, synth, "cfg4", 6, dev, peak)
         except Exception as ex:
             line["decode_128k_gqa"] = {"unavailable": str(ex)[:200]}
+        try:   # a 4-token round (verify step) on the 32K MHA shape: same pages streamed, four queries per head
+            line["round_of_4_tokens_32k"] = decode_only(rz, synth, "cfg2", 3, dev, peak, n_tok=4)
+        except Exception as ex:
+            line["round_of_4_tokens_32k"] = {"unavailable": str(ex)[:200]}
 
     # ------------------------------------------------------------------ end to end with HOST buffers
     if not args.no_e2e:

@@ -148,6 +148,28 @@ RAZOR_API int razor_append(razor_cache_t* cache, int32_t layer, const void* k_ne
 RAZOR_API int razor_decode_attention(razor_cache_t* cache, int32_t layer, const void* q, float* out, void* stream);
 
 /*
+ * A round of several new tokens per sequence (a second prompt chunk, a speculative-decoding verify
+ * step).  The paper runs Algorithm 1 once on the prompt and says nothing about such rounds; the
+ * reading taken extends the single-token rule.
+ *   razor_append_many             adds n_tokens tokens per sequence, k_new, v_new device
+ *                                 [B, n_tokens, Hkv, D] contiguous: exactly what n_tokens razor_append
+ *                                 calls would leave (window fixed, evicted tokens folded into Eq. 4).
+ *   razor_decode_attention_multi  q device [B, n_tokens, Hq, D], out device fp32 [B, n_tokens, Hq, D]:
+ *                                 query t is the token at position (tokens seen) - n_tokens + t and
+ *                                 attends to the kept tokens at positions <= its own (Section 3.1:
+ *                                 n <= m) plus the compensation token with its count N_d (Eq. 5).
+ *                                 n_tokens = 1 is razor_decode_attention.
+ * Limits of the multi-token call: bf16, (Hq / Hkv) * n_tokens in {2, 4, 8} (the rows of one KV head's
+ * tile run on matrix instructions), at least n_tokens tokens cached, and every head that has dropped
+ * tokens must have a window >= n_tokens (otherwise its mean would hold tokens that come after a query).
+ * Errors: NULL_PTR, INVALID_ARG, UNSUPPORTED_DIM, NOT_COMPRESSED, CAPACITY (append), MISALIGNED, CUDA.
+ */
+RAZOR_API int razor_append_many(razor_cache_t* cache, int32_t layer, const void* k_new, const void* v_new,
+                      int32_t n_tokens, void* stream);
+RAZOR_API int razor_decode_attention_multi(razor_cache_t* cache, int32_t layer, const void* q, float* out,
+                                 int32_t n_tokens, void* stream);
+
+/*
  * Read back the compressed state of one (layer, sequence, KV head) in LOGICAL order (ascending
  * original position), whatever the physical slot order is.  Device outputs, any of which may be
  * NULL: kept_pos int32[n_kept]; K, V [n_kept, D] in config.dtype; comp_mean_k/v and comp_sum_k/v

@@ -26,7 +26,7 @@ STATUS = {
 # every symbol include/razor.h declares
 SYMBOLS = [
     "razor_query_bytes", "razor_cache_create", "razor_compress", "razor_compress_seq", "razor_append",
-    "razor_decode_attention", "razor_cache_export", "razor_cache_stats", "razor_schedule_plan",
+    "razor_decode_attention", "razor_append_many", "razor_decode_attention_multi", "razor_cache_export", "razor_cache_stats", "razor_schedule_plan",
     "razor_schedule_query", "razor_cache_set_option", "razor_cache_device_status", "razor_cache_wait_selftest", "razor_compensation_mean_static",
     "razor_cache_reset", "razor_cache_destroy", "razor_status_string",
     "razor_last_cuda_error", "razor_version",
@@ -71,6 +71,8 @@ def load() -> C.CDLL:
     lib.razor_compress_seq.argtypes = [vp, i32, i32, vp, vp, i64, i64, i32, vp, i32, i32, vp]
     lib.razor_append.argtypes = [vp, i32, vp, vp, vp]
     lib.razor_decode_attention.argtypes = [vp, i32, vp, vp, vp]
+    lib.razor_append_many.argtypes = [vp, i32, vp, vp, i32, vp]
+    lib.razor_decode_attention_multi.argtypes = [vp, i32, vp, vp, i32, vp]
     lib.razor_cache_export.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, C.POINTER(i32),
                                        C.POINTER(i32), vp]
     lib.razor_cache_stats.argtypes = [vp, i32, C.POINTER(sz), C.POINTER(sz)]
@@ -178,6 +180,16 @@ def razor_append(cache: int, layer: int, k_new, v_new, stream=None) -> None:
 def razor_decode_attention(cache: int, layer: int, q, out, stream=None) -> None:
     _check(load().razor_decode_attention(cache, layer, _ptr(q), _ptr(out), _stream(stream)),
            "razor_decode_attention")
+
+
+def razor_append_many(cache: int, layer: int, k_new, v_new, n_tokens: int, stream=None) -> None:
+    _check(load().razor_append_many(cache, layer, _ptr(k_new), _ptr(v_new), n_tokens, _stream(stream)),
+           "razor_append_many")
+
+
+def razor_decode_attention_multi(cache: int, layer: int, q, out, n_tokens: int, stream=None) -> None:
+    _check(load().razor_decode_attention_multi(cache, layer, _ptr(q), _ptr(out), n_tokens, _stream(stream)),
+           "razor_decode_attention_multi")
 
 
 def razor_cache_export(cache: int, layer: int, b: int, kv_head: int, kept_pos=None, K=None, V=None, comp_mean_k=None,
@@ -298,6 +310,19 @@ class RazorCache:
         if out is None:
             out = torch.empty(q.shape, dtype=torch.float32, device=q.device)
         razor_decode_attention(self.handle, layer, q, out)
+        return out
+
+    def append_many(self, layer: int, k_new: torch.Tensor, v_new: torch.Tensor) -> None:
+        """k_new, v_new: [B, T, Hkv, D]."""
+        assert k_new.is_contiguous() and v_new.is_contiguous()
+        razor_append_many(self.handle, layer, k_new, v_new, k_new.shape[1])
+
+    def decode_multi(self, layer: int, q: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """q: [B, T, Hq, D] -> out fp32 [B, T, Hq, D]."""
+        assert q.is_contiguous()
+        if out is None:
+            out = torch.empty(q.shape, dtype=torch.float32, device=q.device)
+        razor_decode_attention_multi(self.handle, layer, q, out, q.shape[1])
         return out
 
     def export(self, layer: int, b: int, kv_head: int):

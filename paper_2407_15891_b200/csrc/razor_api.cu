@@ -72,8 +72,10 @@ Layout make_layout(const razor_config_t& c) {
   l.items = take(L * (size_t)l.max_items * sizeof(WorkItem));
   l.jobs = take(L * ((size_t)l.max_items + 1) * sizeof(int32_t));
   l.multi = take(L * nh * sizeof(MultiHead));
-  l.rec_ml = take((size_t)l.max_items * g * sizeof(float2));
-  l.rec_o = take((size_t)l.max_items * g * D * sizeof(float));
+  // a partial record holds up to kMaxGroup rows: query heads of the group x query tokens of a round
+  l.rec_ml = take((size_t)l.max_items * kMaxGroup * sizeof(float2));
+  l.rec_o = take((size_t)l.max_items * kMaxGroup * D * sizeof(float));
+  (void)g;
   l.queue = take(8 * sizeof(int32_t));   // queue[0..3], then the status word
   l.scratch = take(nh * kCompressMaxSlices * 2 * D * sizeof(float));
   l.seq_desc = take((size_t)c.batch * sizeof(SeqDesc));
@@ -520,15 +522,66 @@ int razor_append(razor_cache_t* c, int32_t layer, const void* k_new, const void*
   return RAZOR_OK;
 }
 
+int razor_append_many(razor_cache_t* c, int32_t layer, const void* k_new, const void* v_new, int32_t n_tokens,
+                      void* stream) {
+  if (!c || !k_new || !v_new) return RAZOR_E_NULL_PTR;
+  int rc = layer_ready(c, layer);
+  if (rc) return rc;
+  if (n_tokens < 1) return RAZOR_E_INVALID_ARG;
+  if (((uintptr_t)k_new | (uintptr_t)v_new) & 15) return RAZOR_E_MISALIGNED;
+  LayerHost& L = c->layers[layer];
+  if ((long long)L.appended + n_tokens > c->cfg.max_new_tokens) return RAZOR_E_CAPACITY;
+  RZ_CUDA(launch_append_many(c->dv, c->cfg.dtype, layer, k_new, v_new, n_tokens, (cudaStream_t)stream));
+  const int n_sink = c->cfg.n_sink;
+  for (int t = 0; t < n_tokens; ++t)   // host mirror of the kernel's state update
+    for (HeadState& h : L.hs) {
+      if (h.window < 0 || h.len < n_sink + h.window) {
+        h.len += 1;
+      } else if (h.window == 0) {
+        h.n_drop += 1;
+      } else {
+        h.n_drop += 1;
+        h.ring_head = (h.ring_head + 1 == h.window) ? 0 : h.ring_head + 1;
+      }
+    }
+  L.appended += n_tokens;
+  L.growth_tokens += n_tokens;
+  return RAZOR_OK;
+}
+
+static int decode_impl(razor_cache_t* c, int32_t layer, const void* q, float* out, int32_t n_tokens, void* stream);
+
+int razor_decode_attention_multi(razor_cache_t* c, int32_t layer, const void* q, float* out, int32_t n_tokens,
+                                 void* stream) {
+  if (!c || !q || !out) return RAZOR_E_NULL_PTR;
+  int rc = layer_ready(c, layer);
+  if (rc) return rc;
+  if (n_tokens < 1) return RAZOR_E_INVALID_ARG;
+  if (n_tokens > 1) {
+    const int rows = (c->cfg.n_q_heads / c->cfg.n_kv_heads) * n_tokens;
+    if (c->cfg.dtype != RAZOR_BF16 || (rows != 2 && rows != 4 && rows != 8)) return RAZOR_E_UNSUPPORTED_DIM;
+    for (const HeadState& h : c->layers[layer].hs) {
+      if (h.len + h.n_drop < n_tokens) return RAZOR_E_INVALID_ARG;          // fewer tokens cached than queries
+      if (h.n_drop > 0 && h.window < n_tokens) return RAZOR_E_INVALID_ARG;  // the mean would hold tokens after a query
+    }
+  }
+  return decode_impl(c, layer, q, out, n_tokens, stream);
+}
+
 int razor_decode_attention(razor_cache_t* c, int32_t layer, const void* q, float* out, void* stream) {
   if (!c || !q || !out) return RAZOR_E_NULL_PTR;
   int rc = layer_ready(c, layer);
   if (rc) return rc;
+  return decode_impl(c, layer, q, out, 1, stream);
+}
+
+static int decode_impl(razor_cache_t* c, int32_t layer, const void* q, float* out, int32_t n_tokens, void* stream) {
+  int rc;
   if (((uintptr_t)q | (uintptr_t)out) & 15) return RAZOR_E_MISALIGNED;
   rc = ensure_schedule(c, layer, (cudaStream_t)stream, true);
   if (rc) return rc;
   const LayerHost& L = c->layers[layer];
-  const DecodeJobs jb{L.n_items, L.n_jobs, L.n_spans, L.jobs[L.n_spans], L.n_multi};
+  const DecodeJobs jb{L.n_items, L.n_jobs, L.n_spans, L.jobs[L.n_spans], L.n_multi, n_tokens};
   RZ_CUDA(launch_decode(c->dv, c->cfg.dtype, layer, jb, q, out, c->n_sms, c->tune,
                         (cudaStream_t)stream));
   return RAZOR_OK;

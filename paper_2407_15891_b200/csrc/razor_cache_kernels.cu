@@ -177,6 +177,77 @@ __global__ void __launch_bounds__(128) append_kernel(DeviceView dv, int layer, c
 }
 
 // ---------------------------------------------------------------------------------------------
+// Append of a round of n_tok tokens per sequence (a second prompt, a verify step): one warp per
+// (sequence, KV head) applies the single-token rule n_tok times in order, so the state afterwards is
+// what n_tok razor_append calls would leave.  k_new, v_new: [B, n_tok, Hkv, D].
+template <typename T, int D>
+__global__ void __launch_bounds__(128) append_many_kernel(DeviceView dv, int layer, const T* __restrict__ k_new,
+                                                          const T* __restrict__ v_new, int n_tok) {
+  using Geo = RowGeom<T, D>;
+  constexpr int LPR = Geo::kLpr, EPL = Geo::kEpl;
+  const int lane = threadIdx.x & 31;
+  const int head = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  cudaTriggerProgrammaticLaunchCompletion();
+  if (head >= dv.n_heads) return;
+  const size_t hs = (size_t)layer * dv.n_heads + head;
+  HeadState st = dv.state[hs];
+  __syncwarp();
+  const int n_sink = dv.n_sink;
+  const bool keeps_all = st.window < 0;
+  const int b = head / dv.n_kv_heads, g = head % dv.n_kv_heads;
+  float* sum = dv.comp_sum + hs * 2 * D + lane * EPL;
+  float* mean = dv.comp_mean + hs * 2 * D + lane * EPL;
+  for (int t = 0; t < n_tok; ++t) {
+    int slot = -1;
+    bool evict = false, fold_new = false;
+    if (keeps_all || st.len < n_sink + st.window) {
+      slot = st.len;
+      st.len += 1;
+    } else if (st.window == 0) {
+      fold_new = true;
+      st.n_drop += 1;
+    } else {
+      slot = n_sink + st.ring_head;
+      evict = true;
+      st.n_drop += 1;
+      st.ring_head = (st.ring_head + 1 == st.window) ? 0 : st.ring_head + 1;
+    }
+    if (lane < LPR) {
+      const size_t row = (((size_t)b * n_tok + t) * dv.n_kv_heads + g) * D;
+      const uint4 kf = ((const uint4*)(k_new + row))[lane];
+      const uint4 vf = ((const uint4*)(v_new + row))[lane];
+      uint4* krow = nullptr;
+      if (slot >= 0) {
+        const size_t page = (size_t)dv.page_table[hs * dv.max_pages + (slot >> 4)];
+        krow = (uint4*)(dv.pool + page * dv.page_bytes + (size_t)(slot & 15) * Geo::kRowBytes) + swz(slot, lane);
+      }
+      if (evict || fold_new) {
+        const uint4 ok = evict ? krow[0] : kf;
+        const uint4 ov = evict ? krow[kPageTokens * LPR] : vf;
+        float a[EPL], c[EPL];
+        Elem<T>::unpack(ok, a);
+        Elem<T>::unpack(ov, c);
+        const float cnt = (float)st.n_drop;
+#pragma unroll
+        for (int i = 0; i < EPL; ++i) {
+          const float sk = sum[i] + a[i], sv = sum[D + i] + c[i];
+          sum[i] = sk;
+          sum[D + i] = sv;
+          mean[i] = __fdiv_rn(sk, cnt);
+          mean[D + i] = __fdiv_rn(sv, cnt);
+        }
+      }
+      if (slot >= 0) {
+        krow[0] = kf;
+        krow[kPageTokens * LPR] = vf;
+      }
+    }
+    __syncwarp();   // a later token of the round may evict a row this one just stored
+  }
+  if (lane == 0) dv.state[hs] = st;
+}
+
+// ---------------------------------------------------------------------------------------------
 // Export in logical order (ascending original position).  With T = len + n_drop tokens seen so far:
 // logical index i < N0 (or any i while nothing has been dropped) is position i in slot i; otherwise
 // j = i - N0 is the j-th oldest recent token: slot N0 + (ring_head + j) mod W, position T - W + j.
@@ -247,6 +318,24 @@ cudaError_t launch_append(const DeviceView& dv, int dtype, int layer, const void
                               : append_t<__nv_bfloat16, 64>(dv, layer, k, v, s);
   }
   return dv.head_dim == 128 ? append_t<float, 128>(dv, layer, k, v, s) : append_t<float, 64>(dv, layer, k, v, s);
+}
+
+template <typename T, int D>
+static cudaError_t append_many_t(const DeviceView& dv, int layer, const void* k, const void* v, int n_tok, cudaStream_t s) {
+  const int warps = 4;
+  append_many_kernel<T, D><<<(dv.n_heads + warps - 1) / warps, warps * 32, 0, s>>>(dv, layer, (const T*)k, (const T*)v,
+                                                                                  n_tok);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_append_many(const DeviceView& dv, int dtype, int layer, const void* k, const void* v, int n_tok,
+                               cudaStream_t s) {
+  if (dtype == RAZOR_BF16) {
+    return dv.head_dim == 128 ? append_many_t<__nv_bfloat16, 128>(dv, layer, k, v, n_tok, s)
+                              : append_many_t<__nv_bfloat16, 64>(dv, layer, k, v, n_tok, s);
+  }
+  return dv.head_dim == 128 ? append_many_t<float, 128>(dv, layer, k, v, n_tok, s)
+                            : append_many_t<float, 64>(dv, layer, k, v, n_tok, s);
 }
 
 template <typename T, int D>

@@ -123,10 +123,11 @@ struct ItemDesc {
   int32_t part_idx;
   int32_t n_parts;
   int32_t rec_base;
-  int32_t pad2;
+  int32_t ring_head;   // ring index of the oldest recent token (slot -> position, multi-token rounds)
   int32_t seed;        // 1: this part starts from the compensation token
   int32_t n_drop;
-  int32_t pad0, pad1;
+  int32_t window;      // recent-window length, < 0: the head keeps everything
+  int32_t pad1;
 };
 
 template <typename T, int D, int G>
@@ -309,9 +310,25 @@ struct MmaState {
 };
 
 // qb[kk][0] = Q[head g][kk*16 + 2t, +1], qb[kk][1] = Q[head g][kk*16 + 8 + 2t, +1] (bf16 pairs; zero for g >= G).
+// What a consumer needs to apply causality inside a round of several query tokens: the position of a
+// slot's token and the position of each query row.
+struct RoundMask {
+  int n_tok, g_real;            // query tokens of the round; query heads per KV head
+  int total;                    // tokens the head has seen (len + n_drop): query t sits at total - n_tok + t
+  int n_sink, ring_head, window, n_drop;
+  int slot0;                    // slot of the page's first token
+  // position of the token in slot s (Algorithm 1 line 3 keeps sinks + a ring of the recent tokens)
+  __device__ __forceinline__ int pos(int s) const {
+    if (window < 0 || n_drop == 0 || s < n_sink) return s;
+    int j = s - n_sink - ring_head;
+    if (j < 0) j += window;
+    return total - window + j;
+  }
+};
+
 template <int D>
 __device__ __forceinline__ void consume_page_mma(uint32_t page_addr, int valid, int lane, float scale_log2,
-                                                 const uint32_t (&qb)[D / 16][2], MmaState<D>& S) {
+                                                 const uint32_t (&qb)[D / 16][2], MmaState<D>& S, const RoundMask& mk) {
   constexpr int ROW = D * 2;          // bytes per row
   constexpr int KS = D / 16;          // k-steps of the K.Q product
   constexpr int MT = D / 16;
@@ -337,6 +354,15 @@ __device__ __forceinline__ void consume_page_mma(uint32_t page_addr, int valid, 
   if (valid < kPageTokens) {   // tokens of this page beyond the head's length
     if (g >= valid) s[0] = s[1] = -CUDART_INF_F;
     if (g + 8 >= valid) s[2] = s[3] = -CUDART_INF_F;
+  }
+  if (mk.n_tok > 1) {          // causality inside the round: a query does not see the tokens after it
+    const int t2 = (lane & 3) * 2;
+    const int qp0 = mk.total - mk.n_tok + t2 / mk.g_real, qp1 = mk.total - mk.n_tok + (t2 + 1) / mk.g_real;
+    const int p0 = mk.pos(mk.slot0 + g), p1 = mk.pos(mk.slot0 + g + 8);
+    if (p0 > qp0) s[0] = -CUDART_INF_F;
+    if (p0 > qp1) s[1] = -CUDART_INF_F;
+    if (p1 > qp0) s[2] = -CUDART_INF_F;
+    if (p1 > qp1) s[3] = -CUDART_INF_F;
   }
   // ---- online softmax of heads 2t, 2t+1 (the eight lanes with the same t share them)
   float mx0 = fmaxf(s[0], s[2]), mx1 = fmaxf(s[1], s[3]);
@@ -490,7 +516,13 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
   // grid to finish before it reads anything this grid writes.
   cudaTriggerProgrammaticLaunchCompletion();
 
-  const int n_q_heads = dv.n_kv_heads * G;
+  // Row r of a KV head's tile is query token r / g_real, query head r % g_real of the group (one token
+  // per sequence: g_real = G).  Offset, in elements, of that row in q and in out ([B, n_tok, Hq, D]).
+  const int g_real = G / jb.n_tok;
+  auto row_offset = [&](int head, int r) {
+    const int b = head / dv.n_kv_heads, g = head % dv.n_kv_heads;
+    return (((size_t)b * jb.n_tok + r / g_real) * ((size_t)dv.n_kv_heads * g_real) + (size_t)g * g_real + r % g_real) * D;
+  };
   // Warp-uniform bounded wait: false for every lane if any lane's wait failed.
   auto warp_wait = [&](uint64_t* bar, uint32_t parity) -> bool {
     return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
@@ -544,14 +576,13 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
       if (lane == 0) {
         ItemDesc d;
         d.head = w.head; d.page_begin = w.page_begin; d.n_pages = n; d.len = st.len;
-        d.part_idx = w.part_idx; d.n_parts = w.n_parts; d.rec_base = w.rec_base; d.pad2 = 0;
-        d.seed = seed ? 1 : 0; d.n_drop = st.n_drop; d.pad0 = d.pad1 = 0;
+        d.part_idx = w.part_idx; d.n_parts = w.n_parts; d.rec_base = w.rec_base; d.ring_head = st.ring_head;
+        d.seed = seed ? 1 : 0; d.n_drop = st.n_drop; d.window = st.window; d.pad1 = 0;
         sl.desc = d;
-        const int b = w.head / dv.n_kv_heads, g = w.head % dv.n_kv_heads;
-        const T* qsrc = q + ((size_t)b * n_q_heads + (size_t)g * G) * D;
         constexpr uint32_t q_bytes = G * D * sizeof(T), mean_bytes = 2 * D * sizeof(float);
         mbar_arrive_expect_tx(&bars.item_full[slot], q_bytes + (seed ? mean_bytes : 0u));
-        bulk_load(&sl.q[0][0], qsrc, q_bytes, &bars.item_full[slot]);
+        for (int t = 0; t < jb.n_tok; ++t)   // the g_real rows of one query token are contiguous
+          bulk_load(&sl.q[t * g_real][0], q + row_offset(w.head, t * g_real), q_bytes / jb.n_tok, &bars.item_full[slot]);
         if (seed) bulk_load(&sl.mean[0][0], dv.comp_mean + hs * 2 * D, mean_bytes, &bars.item_full[slot]);
       }
       seq_issued = seq + 1;
@@ -716,7 +747,9 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
                 vrows[idx] = make_uint4(0u, 0u, 0u, 0u);
               __syncwarp();
             }
-            consume_page_mma<D>(smem_u32(page), valid, lane, dv.scale_log2, qa, S);
+            const RoundMask mk{jb.n_tok, g_real, d.len + d.n_drop, dv.n_sink, d.ring_head, d.window, d.n_drop,
+                               (d.page_begin + i) * kPageTokens};
+            consume_page_mma<D>(smem_u32(page), valid, lane, dv.scale_log2, qa, S, mk);
           }
           __syncwarp();
           if (lane == 0) mbar_arrive(&bars.empty[stage]);
@@ -861,12 +894,10 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
       if (lane == 0) mbar_arrive(&bars.merge_free[mb]);
 
       if (d.n_parts == 1) {   // the head's only part: this is its output
-        const int b = d.head / dv.n_kv_heads, g = d.head % dv.n_kv_heads;
-        float* out_rows = out + ((size_t)b * n_q_heads + (size_t)g * G) * D;
 #pragma unroll
         for (int j = 0; j < G; ++j) {
           acc[j].scale(l_tot[j] > 0.f ? 1.f / l_tot[j] : 0.f);
-          acc[j].store(out_rows + (size_t)j * D, lane);
+          acc[j].store(out + row_offset(d.head, j), lane);
         }
       } else {                // one of several parts: its record, for the combine kernel
 #pragma unroll
@@ -891,11 +922,12 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
 constexpr int kCombineWarps = 16;
 
 template <int D>
-__global__ void __launch_bounds__(kCombineWarps * 32) combine_kernel(DeviceView dv, int layer, float* __restrict__ out) {
+__global__ void __launch_bounds__(kCombineWarps * 32) combine_kernel(DeviceView dv, int layer, int n_tok,
+                                                                     float* __restrict__ out) {
   __shared__ float2 s_ml[kCombineWarps];
   __shared__ __align__(16) float s_o[kCombineWarps][D];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int G = dv.group, j = blockIdx.y;
+  const int G = dv.group * n_tok, j = blockIdx.y;   // rows per KV head: query tokens x query heads of the group
   const MultiHead mh = dv.multi[(size_t)layer * dv.n_heads + blockIdx.x];   // uploaded before either kernel
   cudaTriggerProgrammaticLaunchCompletion();   // a decode kernel queued behind this one may set itself up
   cudaGridDependencySynchronize();   // the streaming kernel's records are complete and visible from here on
@@ -946,16 +978,16 @@ __global__ void __launch_bounds__(kCombineWarps * 32) combine_kernel(DeviceView 
       sum.fma(cw, o);
     }
     sum.scale(lt > 0.f ? 1.f / lt : 0.f);
-    const int b = mh.head / dv.n_kv_heads, g = mh.head % dv.n_kv_heads;
-    sum.store(out + (((size_t)b * dv.n_kv_heads + g) * G + j) * D, lane);
+    const int b = mh.head / dv.n_kv_heads, g = mh.head % dv.n_kv_heads, gr = dv.group;
+    sum.store(out + (((size_t)b * n_tok + j / gr) * ((size_t)dv.n_kv_heads * gr) + (size_t)g * gr + j % gr) * D, lane);
   }
 }
 
 template <int D>
-cudaError_t combine_launch(const DeviceView& dv, int layer, int n_multi, float* out, cudaStream_t s) {
+cudaError_t combine_launch(const DeviceView& dv, int layer, int n_multi, int n_tok, float* out, cudaStream_t s) {
   if (n_multi <= 0) return cudaSuccess;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(n_multi, dv.group);
+  cfg.gridDim = dim3(n_multi, dv.group * n_tok);
   cfg.blockDim = dim3(kCombineWarps * 32);
   cfg.dynamicSmemBytes = 0;
   cfg.stream = s;
@@ -964,7 +996,7 @@ cudaError_t combine_launch(const DeviceView& dv, int layer, int n_multi, float* 
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, combine_kernel<D>, dv, layer, out);
+  return cudaLaunchKernelEx(&cfg, combine_kernel<D>, dv, layer, n_tok, out);
 }
 
 // ------------------------------------------------------------------------------------------ launch
@@ -1011,7 +1043,7 @@ cudaError_t decode_launch(const DeviceView& dv, int layer, const DecodeJobs& jb,
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   if ((e = cudaLaunchKernelEx(&cfg, kern, dv, layer, jb, (const T*)q, out, (int)stages)) != cudaSuccess) return e;
-  return combine_launch<D>(dv, layer, jb.n_multi, out, s);
+  return combine_launch<D>(dv, layer, jb.n_multi, jb.n_tok, out, s);
 }
 
 template <typename T, int D, int G>
@@ -1022,7 +1054,8 @@ cudaError_t decode_nc(const DeviceView& dv, int layer, const DecodeJobs& jb, con
   const int nc = tune.consumer_warps;
   if constexpr (sizeof(T) == 2 && G >= 2) {
     // Grouped heads: the tensor-core consumer unless switched off (default on from group 4 up).
-    const bool mma = tune.tensor_cores == 1 || (tune.tensor_cores == 0 && G >= 4);
+    // (rounds of several query tokens always take it: only that consumer applies their causal mask)
+    const bool mma = jb.n_tok > 1 || tune.tensor_cores == 1 || (tune.tensor_cores == 0 && G >= 4);
     if (mma) {
       if (nc == 4) return decode_launch<T, D, G, 4, true>(dv, layer, jb, q, out, n_sms, tune, s);
       return decode_launch<T, D, G, 8, true>(dv, layer, jb, q, out, n_sms, tune, s);
@@ -1042,7 +1075,7 @@ cudaError_t decode_nc(const DeviceView& dv, int layer, const DecodeJobs& jb, con
 template <typename T, int D>
 cudaError_t decode_g(const DeviceView& dv, int layer, const DecodeJobs& jb, const void* q, float* out, int n_sms,
                      const DecodeTuning& tune, cudaStream_t s) {
-  switch (dv.group) {
+  switch (dv.group * jb.n_tok) {   // rows of a KV head's tile
     case 1: return decode_nc<T, D, 1>(dv, layer, jb, q, out, n_sms, tune, s);
     case 2: return decode_nc<T, D, 2>(dv, layer, jb, q, out, n_sms, tune, s);
     case 4: return decode_nc<T, D, 4>(dv, layer, jb, q, out, n_sms, tune, s);

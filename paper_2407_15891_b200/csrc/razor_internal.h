@@ -111,11 +111,14 @@ cudaError_t launch_compress(const DeviceView& dv, int dtype, int layer, int n_se
                             cudaStream_t stream);
 cudaError_t launch_append(const DeviceView& dv, int dtype, int layer, const void* k_new, const void* v_new,
                           cudaStream_t stream);
+cudaError_t launch_append_many(const DeviceView& dv, int dtype, int layer, const void* k_new, const void* v_new,
+                               int n_tok, cudaStream_t stream);
 // What a decode launch pulls from the queue: n_jobs jobs, the first n_spans of them spans (item
 // ranges jobs[j]..jobs[j+1]), the others single items starting at tail_first.
 struct DecodeJobs {
   int32_t n_items, n_jobs, n_spans, tail_first;
   int32_t n_multi;   // heads in several parts
+  int32_t n_tok;     // query tokens per sequence in this call (1 for a decode step)
 };
 cudaError_t launch_decode(const DeviceView& dv, int dtype, int layer, const DecodeJobs& jobs, const void* q,
                           float* out, int n_sms, const DecodeTuning& tune, cudaStream_t stream);
