@@ -246,3 +246,34 @@ def multi_query_attention(qs: np.ndarray, K_all: np.ndarray, V_all: np.ndarray, 
         n_d = hc.n_drop if use_compensation else 0
         out[t] = compensated_attention(qs[t], np.asarray(hc.K)[vis], np.asarray(hc.V)[vis], hc.k_hat, hc.v_hat, n_d, scale)
     return out
+
+
+# --------------------------------------------------------------------------- ALiBi heads (Section 3.1)
+def alibi_attention(q: np.ndarray, K: np.ndarray, V: np.ndarray, positions: np.ndarray, q_pos: int,
+                    slope: float, scale: float) -> np.ndarray:
+    """Eq. 1: score of the query at position m = q_pos to the key at position n is q.k - l_h (m - n);
+    softmax over the given keys (all at positions <= q_pos).  `scale` multiplies q.k only (Eq. 1 prints
+    none); the distance penalty is not scaled."""
+    q = np.asarray(q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    V = np.asarray(V, dtype=np.float64)
+    pos = np.asarray(positions, dtype=np.float64)
+    s = scale * (K @ q) - slope * (float(q_pos) - pos)
+    w = np.exp(s - s.max())
+    return (w @ V) / w.sum()
+
+
+def alibi_decode_head(qs: np.ndarray, K_all: np.ndarray, V_all: np.ndarray, window: int, slope: float,
+                      scale: float, n_sink: int = 0) -> np.ndarray:
+    """Section 3.1: an ALiBi head keeps only its most recent L_h = `window` tokens (window < 0: all of
+    them); the last T tokens of the history are the queries (T = 1: a decode step), each attending with
+    Eq. 1 to the kept tokens at positions <= its own.  qs [T, D]; K_all, V_all [N + T, D]."""
+    qs = np.asarray(qs, dtype=np.float64)
+    T, total = qs.shape[0], int(np.asarray(K_all).shape[0])
+    kept = kept_positions(total, n_sink, window if window >= 0 else total, window < 0)
+    out = np.zeros_like(qs)
+    for t in range(T):
+        q_pos = total - T + t
+        vis = kept[kept <= q_pos]
+        out[t] = alibi_attention(qs[t], np.asarray(K_all)[vis], np.asarray(V_all)[vis], vis, q_pos, slope, scale)
+    return out

@@ -401,3 +401,56 @@ def test_multi_query_equals_eq5_with_replicated_compensation_token_and_causal_ma
         assert np.allclose(out[t], ref, rtol=0, atol=1e-12)
     with pytest.raises(AssertionError):
         orc.multi_query_attention(qs, K, V, n0, T - 1, False, 0.4)   # window shorter than the round
+
+
+# ------------------------------------------------------------------ ALiBi heads (Section 3.1, Eq. 1, Theorem 1)
+def test_alibi_matches_scalar_brute_force_and_reduces_to_plain_attention():
+    rng = _rng(80)
+    n, d = 23, 6
+    K, V, q = rng.standard_normal((n, d)), rng.standard_normal((n, d)), rng.standard_normal(d)
+    pos = np.arange(n)
+    slope, scale = 0.37, 0.8
+    logits = [scale * sum(q[i] * K[t][i] for i in range(d)) - slope * ((n - 1) - t) for t in range(n)]
+    w = [math.exp(x - max(logits)) for x in logits]
+    ref = np.array([sum(w[t] * V[t][i] for t in range(n)) / sum(w) for i in range(d)])
+    assert np.allclose(orc.alibi_attention(q, K, V, pos, n - 1, slope, scale), ref, rtol=0, atol=1e-13)
+    # slope 0: ordinary attention; shifting every position by a constant changes nothing
+    assert np.allclose(orc.alibi_attention(q, K, V, pos, n - 1, 0.0, scale), orc.full_attention(q, K, V, scale), atol=1e-14)
+    assert np.allclose(orc.alibi_attention(q, K, V, pos + 1000, n + 999, slope, scale), ref, rtol=0, atol=1e-12)
+
+
+def test_alibi_far_tokens_weigh_less_than_epsilon_beyond_the_vision_scope():
+    """Theorem 1 with the bound on |q.k| taken from the data: if |scale q.k_n| <= B for every n, the weight
+    of a key at distance > (2B - ln eps) / l_h is below eps, so truncating there changes the output by
+    at most about eps * (number of far tokens) * max|v|."""
+    rng = _rng(81)
+    n, d, slope, scale, eps = 400, 8, 0.25, 0.5, 1e-3
+    K, V, q = rng.standard_normal((n, d)), rng.standard_normal((n, d)), rng.standard_normal(d)
+    B = np.abs(scale * K @ q).max()
+    L_h = int(math.ceil((2 * B - math.log(eps)) / slope))
+    assert L_h < n
+    s = scale * (K @ q) - slope * ((n - 1) - np.arange(n))
+    wts = np.exp(s - s.max()); wts /= wts.sum()
+    assert wts[: n - 1 - L_h].max() <= eps
+    full = orc.alibi_decode_head(q[None], K, V, -1, slope, scale)[0]
+    cut = orc.alibi_decode_head(q[None], K, V, L_h + 1, slope, scale)[0]
+    assert np.abs(full - cut).max() <= 2 * wts[: n - 1 - L_h].sum() * np.abs(V).max()
+    assert np.abs(full - cut).max() < 1e-2
+
+
+def test_alibi_decode_head_keeps_the_recent_window_and_is_causal():
+    rng = _rng(82)
+    n, T, d, win = 50, 3, 8, 12
+    K, V, qs = rng.standard_normal((n + T, d)), rng.standard_normal((n + T, d)), rng.standard_normal((T, d))
+    out = orc.alibi_decode_head(qs, K, V, win, 0.1, 0.6)
+    total = n + T
+    for t in range(T):
+        vis = [p for p in range(total - win, total) if p <= n + t]
+        ref = orc.alibi_attention(qs[t], K[vis], V[vis], np.array(vis), n + t, 0.1, 0.6)
+        assert np.allclose(out[t], ref, rtol=0, atol=1e-13)
+    K2 = K.copy(); K2[: total - win] += 5.0                  # tokens outside the window do not matter
+    assert np.allclose(orc.alibi_decode_head(qs, K2, V, win, 0.1, 0.6), out, atol=1e-14)
+    # slope 0 and a window: plain truncation (the Table 1 scheme) of the decode oracle
+    hc = orc.compress_head(K[: n + 1], V[: n + 1], n + 1, 0, win, False)
+    assert np.allclose(orc.alibi_decode_head(qs[:1], K[: n + 1], V[: n + 1], win, 0.0, 0.6)[0],
+                       orc.decode_head(qs[0], hc, 0.6, use_compensation=False), atol=1e-13)
