@@ -226,7 +226,7 @@ def _workload_config(w, args):
 
 
 # ---------------------------------------------------------------------------------------------- GPU legs
-def decode_only(rz, synth, name, n_layers, dev, peak, reps=60, n_tok=1):
+def decode_only(rz, synth, name, n_layers, dev, peak, reps=60, n_tok=1, alibi=False):
     """Decode attention alone on the first n_layers layers of another workload (each layer compressed from
     one seeded dense buffer): back-to-back razor_decode_attention calls cycling over the layers, so that
     every call streams pages that the L2 no longer holds."""
@@ -235,9 +235,14 @@ def decode_only(rz, synth, name, n_layers, dev, peak, reps=60, n_tok=1):
     w = synth.workload(name)
     w.n_layers = n_layers
     retr = [w.retrieval(l) for l in range(n_layers)]
-    cfg = rz.make_config(w.batch, n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, w.n_sink, max(w.ctx_len),
-                         max(1, n_tok))
+    cfg = rz.make_config(w.batch, n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, 0 if alibi else w.n_sink,
+                         max(w.ctx_len), max(1, n_tok), use_compensation=0 if alibi else 1)
     cache = rz.RazorCache(cfg, w.ctx_len, w.window, np.stack(retr), device=dev)
+    if alibi:   # the ALiBi variant: distance penalty on every logit, recent tokens only, no compensation token
+        slopes = np.array([2.0 ** (-8.0 * (i + 1) / w.n_q_heads) for i in range(w.n_q_heads)], dtype=np.float32)
+        rz.razor_cache_set_alibi(cache.handle, np.tile(slopes, n_layers))
+        w = synth.Workload(w.name, w.batch, w.n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, w.ctx_len,
+                           w.window, 0, w.n_retrieval_kv, w.decode_steps, w.seed)
     w0 = synth.Workload(w.name, w.batch, 1, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, w.ctx_len, w.window,
                         w.n_sink, w.n_retrieval_kv, 1, w.seed)
     K, V = synth.make_dense_kv(w0, 0, dev)
@@ -275,7 +280,7 @@ def decode_only(rz, synth, name, n_layers, dev, peak, reps=60, n_tok=1):
                         f"{n_layers} layers cycled ({n_layers * kept / 1e9:.2f} GB of pages)",
             "us_per_layer": us, "gbs": gbs, "frac_of_measured": gbs / peak, "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS,
             "compressed_mb_per_layer": kept / 1e6, "launches_timed": reps, "device_status": status,
-            "query_tokens_per_call": n_tok}
+            "query_tokens_per_call": n_tok, "alibi": bool(alibi)}
 
 
 def main():
@@ -471,6 +476,10 @@ def main():
             line["decode_128k_gqa"] = decode_only(rz, synth, "cfg4", 6, dev, peak)
         except Exception as ex:
             line["decode_128k_gqa"] = {"unavailable": str(ex)[:200]}
+        try:   # the ALiBi variant on the 32K MHA shape
+            line["alibi_32k"] = decode_only(rz, synth, "cfg2", 3, dev, peak, alibi=True)
+        except Exception as ex:
+            line["alibi_32k"] = {"unavailable": str(ex)[:200]}
         try:   # a 4-token round (verify step) on the 32K MHA shape: same pages streamed, four queries per head
             line["round_of_4_tokens_32k"] = decode_only(rz, synth, "cfg2", 3, dev, peak, n_tok=4)
         except Exception as ex:

@@ -235,6 +235,28 @@ RAZOR_API int razor_cache_set_option(razor_cache_t* cache, int32_t option, int32
 RAZOR_API int razor_cache_device_status(razor_cache_t* cache, int32_t* status, void* stream);
 
 /*
+ * ALiBi models (Section 3.1).  Their head h scores a key at distance m - n with q.k - l_h (m - n)
+ * (Eq. 1) and keeps only its most recent L_h tokens, L_h being the head's vision scope (Theorem 1;
+ * computing it needs the model's weights, so it is an input here).
+ *   razor_cache_set_alibi         slopes host fp32 [L * Hq], l_h >= 0 of every query head; from the next
+ *                                 decode call on, every logit gets - l_h * (query position - key
+ *                                 position); sm_scale multiplies q.k only.  NULL switches it off.
+ *                                 Needs config.use_compensation = 0 (a mean of dropped tokens has no
+ *                                 position; the paper uses none for ALiBi heads); n_sink = 0 gives the
+ *                                 paper's recent-tokens-only cache.  The query of a decode step is the
+ *                                 newest cached token (append first); in a multi-token round query t
+ *                                 sits at its own position.
+ *   razor_cache_set_head_windows  window_h host int32 [Hkv] for one layer: from the next razor_compress
+ *                                 of that layer on, KV head g keeps min(window[b], window_h[g]) recent
+ *                                 tokens (heads flagged in head_is_retrieval still keep everything).
+ *                                 NULL removes the caps.  Pool sizing stays razor_query_bytes' with
+ *                                 window[b] (an upper bound).
+ * Errors: NULL_PTR, INVALID_ARG, CUDA.
+ */
+RAZOR_API int razor_cache_set_alibi(razor_cache_t* cache, const float* slopes, void* stream);
+RAZOR_API int razor_cache_set_head_windows(razor_cache_t* cache, int32_t layer, const int32_t* window_h);
+
+/*
  * Self-test of the bounded waits.  Enqueues a one-warp kernel that waits, with the decode kernel's own
  * wait routine and a limit of limit_ns (1 us .. 1 s), on a barrier nothing ever arrives on.  The wait
  * has to give up by itself; razor_cache_device_status then reports bit 16 (and clears it), and the

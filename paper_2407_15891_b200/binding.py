@@ -27,7 +27,8 @@ STATUS = {
 SYMBOLS = [
     "razor_query_bytes", "razor_cache_create", "razor_compress", "razor_compress_seq", "razor_append",
     "razor_decode_attention", "razor_append_many", "razor_decode_attention_multi", "razor_cache_export", "razor_cache_stats", "razor_schedule_plan",
-    "razor_schedule_query", "razor_cache_set_option", "razor_cache_device_status", "razor_cache_wait_selftest", "razor_compensation_mean_static",
+    "razor_schedule_query", "razor_cache_set_option", "razor_cache_device_status", "razor_cache_wait_selftest", "razor_cache_set_alibi", "razor_cache_set_head_windows",
+    "razor_compensation_mean_static",
     "razor_cache_reset", "razor_cache_destroy", "razor_status_string",
     "razor_last_cuda_error", "razor_version",
 ]
@@ -83,6 +84,8 @@ def load() -> C.CDLL:
     lib.razor_compensation_mean_static.argtypes = [vp, vp, i64, i64, i32, i32, i32, i32, i32, i32, vp, vp,
                                                    C.POINTER(i32), vp]
     lib.razor_cache_wait_selftest.argtypes = [vp, i64, vp]
+    lib.razor_cache_set_alibi.argtypes = [vp, vp, vp]
+    lib.razor_cache_set_head_windows.argtypes = [vp, i32, vp]
     lib.razor_cache_reset.argtypes = [vp]
     lib.razor_cache_destroy.argtypes = [vp]
     lib.razor_status_string.argtypes = [C.c_int]
@@ -245,6 +248,24 @@ def razor_schedule_query(cache: int, layer: int) -> np.ndarray:
     items = np.zeros((n.value, 5), dtype=np.int32)
     _check(lib.razor_schedule_query(cache, layer, items.ctypes.data, n.value, C.byref(n)), "razor_schedule_query")
     return items
+
+
+def razor_cache_set_alibi(cache: int, slopes, stream=None) -> None:
+    """slopes: [L * Hq] (or [L, Hq]) ALiBi slopes l_h; None switches the distance penalty off."""
+    if slopes is None:
+        _check(load().razor_cache_set_alibi(cache, None, _stream(stream)), "razor_cache_set_alibi")
+        return
+    a = np.ascontiguousarray(np.asarray(slopes, dtype=np.float32).reshape(-1))
+    _check(load().razor_cache_set_alibi(cache, a.ctypes.data, _stream(stream)), "razor_cache_set_alibi")
+
+
+def razor_cache_set_head_windows(cache: int, layer: int, window_h) -> None:
+    """window_h: [Hkv] per-head caps on the recent window for later compressions of `layer`; None removes them."""
+    if window_h is None:
+        _check(load().razor_cache_set_head_windows(cache, layer, None), "razor_cache_set_head_windows")
+        return
+    a = _i32(window_h)
+    _check(load().razor_cache_set_head_windows(cache, layer, a.ctypes.data), "razor_cache_set_head_windows")
 
 
 def razor_cache_wait_selftest(cache: int, limit_ns: int, stream=None) -> None:

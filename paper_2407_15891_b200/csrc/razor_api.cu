@@ -33,7 +33,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 inline int ceil_div(long long a, long long b) { return (int)((a + b - 1) / b); }
 
 struct Layout {
-  size_t state, comp_sum, comp_mean, page_table, items, jobs, multi, rec_ml, rec_o, queue, scratch, seq_desc, total;
+  size_t state, comp_sum, comp_mean, page_table, items, jobs, multi, rec_ml, rec_o, queue, scratch, seq_desc, slopes, total;
   int max_pages, max_items;
 };
 
@@ -79,6 +79,7 @@ Layout make_layout(const razor_config_t& c) {
   l.queue = take(8 * sizeof(int32_t));   // queue[0..3], then the status word
   l.scratch = take(nh * kCompressMaxSlices * 2 * D * sizeof(float));
   l.seq_desc = take((size_t)c.batch * sizeof(SeqDesc));
+  l.slopes = take(L * (size_t)c.n_q_heads * sizeof(float));
   l.total = off;
   return l;
 }
@@ -93,6 +94,7 @@ struct LayerHost {
   bool any = false;
   int n_done = 0;
   std::vector<uint8_t> retr;        // [Hkv]
+  std::vector<int32_t> head_window; // [Hkv] per-head cap on the recent window (razor_cache_set_head_windows); empty: none
   std::vector<uint8_t> seq_done;    // [B]
   std::vector<HeadState> hs;        // [B*Hkv] mirror of the device state
   std::vector<long long> region_start, region_count;   // pages owned by (layer, b)
@@ -209,6 +211,8 @@ int razor_cache_create(razor_cache_t** out, const razor_config_t* cfg, void* poo
   dv.status = dv.queue + 4;
   dv.compress_scratch = (float*)(ws + lay.scratch);
   dv.seq_desc = (SeqDesc*)(ws + lay.seq_desc);
+  dv.alibi_slopes = (float*)(ws + lay.slopes);
+  dv.alibi = 0;
   dv.n_heads = cfg->batch * cfg->n_kv_heads;
   dv.n_kv_heads = cfg->n_kv_heads;
   dv.max_pages = lay.max_pages;
@@ -327,6 +331,11 @@ int compress_impl(razor_cache* c, int layer, const std::vector<SeqIn>& seqs, con
     n_max = std::max(n_max, s.n_ctx);
   }
 
+  // A head's recent window: the sequence's, capped by the head's own when per-head windows are set
+  // (ALiBi heads each have their own vision scope, Section 3.1).
+  auto eff_window = [&](int seq_window, int g) {
+    return L.head_window.empty() ? seq_window : std::min(seq_window, L.head_window[g]);
+  };
   // Page plan per sequence; allocate (or reuse) the sequence's region, all-or-nothing.
   std::vector<long long> need(seqs.size());
   long long next = c->next_page;
@@ -334,7 +343,8 @@ int compress_impl(razor_cache* c, int layer, const std::vector<SeqIn>& seqs, con
   for (size_t i = 0; i < seqs.size(); ++i) {
     long long pages = 0;
     for (int g = 0; g < H; ++g)
-      pages += ceil_div(head_capacity_tokens(cfg, seqs[i].n_ctx, seqs[i].window, flags[g] != 0), kPageTokens);
+      pages += ceil_div(head_capacity_tokens(cfg, seqs[i].n_ctx, eff_window(seqs[i].window, g), flags[g] != 0),
+                        kPageTokens);
     need[i] = pages;
     if (pages > L.region_count[seqs[i].b]) {
       if (next + pages > c->pool_pages) return RAZOR_E_POOL_TOO_SMALL;
@@ -367,14 +377,15 @@ int compress_impl(razor_cache* c, int layer, const std::vector<SeqIn>& seqs, con
     size_t cursor = 0;
     for (int g = 0; g < H; ++g) {
       const bool r = flags[g] != 0;
-      const int cap_pages = ceil_div(head_capacity_tokens(cfg, s.n_ctx, s.window, r), kPageTokens);
+      const int wg = eff_window(s.window, g);
+      const int cap_pages = ceil_div(head_capacity_tokens(cfg, s.n_ctx, wg, r), kPageTokens);
       for (int k = 0; k < cap_pages; ++k) rows[(size_t)g * c->lay.max_pages + k] = ids[cursor++];
-      const bool keep_all = r || s.n_ctx <= cfg.n_sink + s.window;
+      const bool keep_all = r || s.n_ctx <= cfg.n_sink + wg;
       HeadState h;
-      h.len = keep_all ? s.n_ctx : cfg.n_sink + s.window;
-      h.n_drop = keep_all ? 0 : s.n_ctx - cfg.n_sink - s.window;
+      h.len = keep_all ? s.n_ctx : cfg.n_sink + wg;
+      h.n_drop = keep_all ? 0 : s.n_ctx - cfg.n_sink - wg;
       h.ring_head = 0;
-      h.window = r ? -1 : s.window;
+      h.window = r ? -1 : wg;
       states[g] = h;
       L.hs[(size_t)s.b * H + g] = h;
     }
@@ -692,6 +703,39 @@ int razor_cache_device_status(razor_cache_t* c, int32_t* status, void* stream) {
     RZ_CUDA(cudaMemsetAsync(c->dv.queue, 0, 8 * sizeof(int32_t), (cudaStream_t)stream));
     RZ_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
   }
+  return RAZOR_OK;
+}
+
+int razor_cache_set_alibi(razor_cache_t* c, const float* slopes, void* stream) {
+  if (!c) return RAZOR_E_NULL_PTR;
+  if (!slopes) {
+    c->dv.alibi = 0;
+    return RAZOR_OK;
+  }
+  if (c->cfg.use_compensation) return RAZOR_E_INVALID_ARG;   // the compensation token has no position to penalise
+  const size_t n = (size_t)c->cfg.n_layers * c->cfg.n_q_heads;
+  std::vector<float> scaled(n);
+  for (size_t i = 0; i < n; ++i) {
+    if (!(slopes[i] >= 0.f) || std::isinf(slopes[i])) return RAZOR_E_INVALID_ARG;
+    scaled[i] = slopes[i] * 1.4426950408889634f;   // the kernels work in the log2 domain
+  }
+  RZ_CUDA(cudaMemcpyAsync(c->dv.alibi_slopes, scaled.data(), n * sizeof(float), cudaMemcpyHostToDevice,
+                          (cudaStream_t)stream));   // pageable source: staged before the call returns
+  c->dv.alibi = 1;
+  return RAZOR_OK;
+}
+
+int razor_cache_set_head_windows(razor_cache_t* c, int32_t layer, const int32_t* window_h) {
+  if (!c) return RAZOR_E_NULL_PTR;
+  if (layer < 0 || layer >= c->cfg.n_layers) return RAZOR_E_INVALID_ARG;
+  LayerHost& L = c->layers[layer];
+  if (!window_h) {
+    L.head_window.clear();
+    return RAZOR_OK;
+  }
+  for (int g = 0; g < c->cfg.n_kv_heads; ++g)
+    if (window_h[g] < 0) return RAZOR_E_INVALID_ARG;
+  L.head_window.assign(window_h, window_h + c->cfg.n_kv_heads);
   return RAZOR_OK;
 }
 

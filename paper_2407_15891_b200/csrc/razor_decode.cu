@@ -187,11 +187,29 @@ __device__ __forceinline__ void merge_state(float& m, float& l, float (&o)[EPL],
   m = mm;
 }
 
+// What a consumer needs to apply causality inside a round of several query tokens, or the distance
+// penalty of ALiBi heads (Eq. 1): the position of a slot's token and the position of each query row.
+struct RoundMask {
+  int n_tok, g_real;            // query tokens of the round; query heads per KV head
+  int alibi;                    // 1: add the ALiBi distance penalty
+  int total;                    // tokens the head has seen (len + n_drop): query t sits at total - n_tok + t
+  int n_sink, ring_head, window, n_drop;
+  int slot0;                    // slot of the page's first token
+  // position of the token in slot s (Algorithm 1 line 3 keeps sinks + a ring of the recent tokens)
+  __device__ __forceinline__ int pos(int s) const {
+    if (window < 0 || n_drop == 0 || s < n_sink) return s;
+    int j = s - n_sink - ring_head;
+    if (j < 0) j += window;
+    return total - window + j;
+  }
+};
+
 // One page (16 tokens) from shared memory into the running state of a consumer warp (CUDA cores).
 // `page` is the page's first 16-byte chunk; this lane reads logical chunk lir of the rows i*RG + rg.
 template <typename T, int D, int G>
 __device__ __forceinline__ void consume_page(const uint4* page, int valid, int rg, int lir,
-                                             const float (&qf)[G][Elem<T>::kEpl], SoftmaxState<G, Elem<T>::kEpl>& S) {
+                                             const float (&qf)[G][Elem<T>::kEpl], SoftmaxState<G, Elem<T>::kEpl>& S,
+                                             bool alibi, const RoundMask& mk, const float (&slope)[G]) {
   using Geo = RowGeom<T, D>;
   constexpr int LPR = Geo::kLpr, EPL = Geo::kEpl, RG = Geo::kRg, RPG = Geo::kRowsPerGroup;
   uint4 kf[RPG], vf[RPG];
@@ -218,6 +236,15 @@ __device__ __forceinline__ void consume_page(const uint4* page, int valid, int r
 #pragma unroll
     for (int i = 0; i < RPG; ++i) s[j][i] = row_sum<LPR>(s[j][i]);
 
+  if (alibi) {   // Eq. 1: - l_h (m - n), slopes already in the log2 domain; one query token on this path
+    const int q_pos = mk.total - 1;
+#pragma unroll
+    for (int i = 0; i < RPG; ++i) {
+      const float dist = (float)(mk.pos(mk.slot0 + i * RG + rg) - q_pos);
+#pragma unroll
+      for (int j = 0; j < G; ++j) s[j][i] += slope[j] * dist;
+    }
+  }
   if (valid < kPageTokens) {   // rows of this page beyond the head's length
 #pragma unroll
     for (int i = 0; i < RPG; ++i) {
@@ -310,25 +337,10 @@ struct MmaState {
 };
 
 // qb[kk][0] = Q[head g][kk*16 + 2t, +1], qb[kk][1] = Q[head g][kk*16 + 8 + 2t, +1] (bf16 pairs; zero for g >= G).
-// What a consumer needs to apply causality inside a round of several query tokens: the position of a
-// slot's token and the position of each query row.
-struct RoundMask {
-  int n_tok, g_real;            // query tokens of the round; query heads per KV head
-  int total;                    // tokens the head has seen (len + n_drop): query t sits at total - n_tok + t
-  int n_sink, ring_head, window, n_drop;
-  int slot0;                    // slot of the page's first token
-  // position of the token in slot s (Algorithm 1 line 3 keeps sinks + a ring of the recent tokens)
-  __device__ __forceinline__ int pos(int s) const {
-    if (window < 0 || n_drop == 0 || s < n_sink) return s;
-    int j = s - n_sink - ring_head;
-    if (j < 0) j += window;
-    return total - window + j;
-  }
-};
-
 template <int D>
 __device__ __forceinline__ void consume_page_mma(uint32_t page_addr, int valid, int lane, float scale_log2,
-                                                 const uint32_t (&qb)[D / 16][2], MmaState<D>& S, const RoundMask& mk) {
+                                                 const uint32_t (&qb)[D / 16][2], MmaState<D>& S, const RoundMask& mk,
+                                                 float slope0, float slope1) {
   constexpr int ROW = D * 2;          // bytes per row
   constexpr int KS = D / 16;          // k-steps of the K.Q product
   constexpr int MT = D / 16;
@@ -355,10 +367,17 @@ __device__ __forceinline__ void consume_page_mma(uint32_t page_addr, int valid, 
     if (g >= valid) s[0] = s[1] = -CUDART_INF_F;
     if (g + 8 >= valid) s[2] = s[3] = -CUDART_INF_F;
   }
-  if (mk.n_tok > 1) {          // causality inside the round: a query does not see the tokens after it
+  if (mk.n_tok > 1 || mk.alibi) {
     const int t2 = (lane & 3) * 2;
     const int qp0 = mk.total - mk.n_tok + t2 / mk.g_real, qp1 = mk.total - mk.n_tok + (t2 + 1) / mk.g_real;
     const int p0 = mk.pos(mk.slot0 + g), p1 = mk.pos(mk.slot0 + g + 8);
+    if (mk.alibi) {            // Eq. 1: - l_h (m - n); slope0/1 belong to this lane's two rows, log2 domain
+      s[0] += slope0 * (float)(p0 - qp0);
+      s[1] += slope1 * (float)(p0 - qp1);
+      s[2] += slope0 * (float)(p1 - qp0);
+      s[3] += slope1 * (float)(p1 - qp1);
+    }
+    // causality inside the round: a query does not see the tokens after it
     if (p0 > qp0) s[0] = -CUDART_INF_F;
     if (p0 > qp1) s[1] = -CUDART_INF_F;
     if (p1 > qp0) s[2] = -CUDART_INF_F;
@@ -703,6 +722,12 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
             qa[kk][1] = qrow[kk * 8 + 4 + t];
           }
         }
+        float slope0 = 0.f, slope1 = 0.f;   // ALiBi slopes of this lane's rows 2t, 2t+1 (query head = row % g_real)
+        if (dv.alibi) {
+          const float* sl_h = dv.alibi_slopes + (size_t)layer * dv.n_kv_heads * g_real + (size_t)(d.head % dv.n_kv_heads) * g_real;
+          slope0 = sl_h[(2 * t) % g_real];
+          slope1 = sl_h[(2 * t + 1) % g_real];
+        }
         MmaState<D> S;
         S.clear();
         const bool first = warp == 0;
@@ -747,9 +772,9 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
                 vrows[idx] = make_uint4(0u, 0u, 0u, 0u);
               __syncwarp();
             }
-            const RoundMask mk{jb.n_tok, g_real, d.len + d.n_drop, dv.n_sink, d.ring_head, d.window, d.n_drop,
+            const RoundMask mk{jb.n_tok, g_real, dv.alibi, d.len + d.n_drop, dv.n_sink, d.ring_head, d.window, d.n_drop,
                                (d.page_begin + i) * kPageTokens};
-            consume_page_mma<D>(smem_u32(page), valid, lane, dv.scale_log2, qa, S, mk);
+            consume_page_mma<D>(smem_u32(page), valid, lane, dv.scale_log2, qa, S, mk, slope0, slope1);
           }
           __syncwarp();
           if (lane == 0) mbar_arrive(&bars.empty[stage]);
@@ -787,6 +812,10 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
 #pragma unroll
           for (int e = 0; e < EPL; ++e) qf[j][e] *= dv.scale_log2;
         }
+        float slope[G];   // ALiBi slopes of the group's query heads (log2 domain); zero when ALiBi is off
+#pragma unroll
+        for (int j = 0; j < G; ++j)
+          slope[j] = dv.alibi ? dv.alibi_slopes[(size_t)layer * dv.n_kv_heads * G + (size_t)(d.head % dv.n_kv_heads) * G + j] : 0.f;
         SoftmaxState<G, EPL> S;
         S.clear();
         const bool first = warp == 0;   // the warp that takes the item's first page also takes its seed
@@ -819,8 +848,10 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
           ring_slot<NC>(c + i, ns, stage, use);
           if (!warp_wait(&bars.full[stage], use & 1)) { ok = false; break; }
           if (i < d.n_pages) {
+            const RoundMask mk{1, G, dv.alibi, d.len + d.n_drop, dv.n_sink, d.ring_head, d.window, d.n_drop,
+                               (d.page_begin + i) * kPageTokens};
             consume_page<T, D, G>((const uint4*)(ring + (size_t)stage * PB), d.len - (d.page_begin + i) * kPageTokens,
-                                  rg, lir, qf, S);
+                                  rg, lir, qf, S, dv.alibi != 0, mk, slope);
           }
           __syncwarp();
           if (lane == 0) mbar_arrive(&bars.empty[stage]);

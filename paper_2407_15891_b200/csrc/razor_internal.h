@@ -84,6 +84,8 @@ struct DeviceView {
   int32_t* status;          // [1]: kStatus* bits, sticky until razor_cache_device_status clears them
   float* compress_scratch;  // [B*Hkv][kCompressMaxSlices][2][D]
   SeqDesc* seq_desc;        // [B]
+  float* alibi_slopes;      // [L][Hq]  ALiBi slopes l_h times log2(e); read only when alibi != 0
+  int32_t alibi;            // 1: logits get - l_h (m - n) (Eq. 1), from razor_cache_set_alibi
   int32_t n_heads;          // B*Hkv
   int32_t n_kv_heads;
   int32_t max_pages;        // page-table row length
