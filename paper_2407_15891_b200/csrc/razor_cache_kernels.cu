@@ -118,6 +118,7 @@ __global__ void __launch_bounds__(128) append_kernel(DeviceView dv, int layer, c
   constexpr int LPR = Geo::kLpr, EPL = Geo::kEpl;
   const int lane = threadIdx.x & 31;
   const int head = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  cudaGridDependencySynchronize();             // launched as a programmatic dependent of the kernel before it
   cudaTriggerProgrammaticLaunchCompletion();   // the decode kernel queued behind the append may set itself up
   if (head >= dv.n_heads) return;
   const size_t hs = (size_t)layer * dv.n_heads + head;
@@ -187,6 +188,7 @@ __global__ void __launch_bounds__(128) append_many_kernel(DeviceView dv, int lay
   constexpr int LPR = Geo::kLpr, EPL = Geo::kEpl;
   const int lane = threadIdx.x & 31;
   const int head = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  cudaGridDependencySynchronize();
   cudaTriggerProgrammaticLaunchCompletion();
   if (head >= dv.n_heads) return;
   const size_t hs = (size_t)layer * dv.n_heads + head;
@@ -286,6 +288,24 @@ __global__ void __launch_bounds__(256) export_kernel(DeviceView dv, int layer, i
 }
 
 // ---------------------------------------------------------------------------------------------
+// Launch as a programmatic dependent of the preceding kernel on the stream: the launch latency and the
+// kernel's first instructions overlap that kernel's tail; the kernel itself waits at
+// cudaGridDependencySynchronize() before it touches memory.
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_dependent(void (*kernel)(KArgs...), int grid, int block, cudaStream_t s, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(block);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 template <typename T, int D>
 static cudaError_t compress_t(const DeviceView& dv, int layer, int n_seqs, int n_slices, cudaStream_t s) {
   dim3 grid(n_slices, dv.n_kv_heads, n_seqs);
@@ -308,8 +328,8 @@ cudaError_t launch_compress(const DeviceView& dv, int dtype, int layer, int n_se
 template <typename T, int D>
 static cudaError_t append_t(const DeviceView& dv, int layer, const void* k, const void* v, cudaStream_t s) {
   const int warps = 4;
-  append_kernel<T, D><<<(dv.n_heads + warps - 1) / warps, warps * 32, 0, s>>>(dv, layer, (const T*)k, (const T*)v);
-  return cudaGetLastError();
+  return launch_dependent(append_kernel<T, D>, (dv.n_heads + warps - 1) / warps, warps * 32, s, dv, layer, (const T*)k,
+                          (const T*)v);
 }
 
 cudaError_t launch_append(const DeviceView& dv, int dtype, int layer, const void* k, const void* v, cudaStream_t s) {
@@ -323,9 +343,8 @@ cudaError_t launch_append(const DeviceView& dv, int dtype, int layer, const void
 template <typename T, int D>
 static cudaError_t append_many_t(const DeviceView& dv, int layer, const void* k, const void* v, int n_tok, cudaStream_t s) {
   const int warps = 4;
-  append_many_kernel<T, D><<<(dv.n_heads + warps - 1) / warps, warps * 32, 0, s>>>(dv, layer, (const T*)k, (const T*)v,
-                                                                                  n_tok);
-  return cudaGetLastError();
+  return launch_dependent(append_many_kernel<T, D>, (dv.n_heads + warps - 1) / warps, warps * 32, s, dv, layer,
+                          (const T*)k, (const T*)v, n_tok);
 }
 
 cudaError_t launch_append_many(const DeviceView& dv, int dtype, int layer, const void* k, const void* v, int n_tok,
