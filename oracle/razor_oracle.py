@@ -277,3 +277,44 @@ def alibi_decode_head(qs: np.ndarray, K_all: np.ndarray, V_all: np.ndarray, wind
         vis = kept[kept <= q_pos]
         out[t] = alibi_attention(qs[t], np.asarray(K_all)[vis], np.asarray(V_all)[vis], vis, q_pos, slope, scale)
     return out
+
+
+# --------------------------------------------------------------------------- retrieval-head identification (Section 3.3)
+def echo_induction_scores(Q: np.ndarray, K: np.ndarray, period: int, scale: float) -> Tuple[float, float]:
+    """Section 3.3 for one head.  The input is `period` random tokens repeated several times; Q, K [N, D] are
+    the head's (post-rotary) queries and keys on it.  For the query at position m >= period, the echo
+    tokens are the earlier copies of the current token, at m - j*period, and the induction tokens are the
+    ones right after them, at m - j*period + 1 (j = 1, 2, ... while the position is >= 0).  The echo
+    (induction) score of the head is the causal-softmax attention weight the query puts on its echo
+    (induction) tokens, summed over j and averaged over all m >= period."""
+    Q = np.asarray(Q, dtype=np.float64)
+    K = np.asarray(K, dtype=np.float64)
+    n = Q.shape[0]
+    echo = induction = 0.0
+    for m in range(period, n):
+        s = scale * (K[: m + 1] @ Q[m])
+        w = np.exp(s - s.max())
+        w /= w.sum()
+        j = 1
+        while m - j * period >= 0:
+            echo += w[m - j * period]
+            induction += w[m - j * period + 1]
+            j += 1
+    cnt = max(1, n - period)
+    return echo / cnt, induction / cnt
+
+
+def select_retrieval_heads(echo: Sequence[float], induction: Sequence[float], frac_induction: float = 0.14,
+                           frac_echo: float = 0.01) -> np.ndarray:
+    """Section 3.3 / Table 2: the retrieval heads are the top 14 % of all heads by induction score plus the
+    top 1 % by echo score (counts rounded to the nearest integer, at least one each; ties broken by the
+    lower head index).  Returns a uint8 mask over the heads."""
+    echo = np.asarray(echo, dtype=np.float64).reshape(-1)
+    induction = np.asarray(induction, dtype=np.float64).reshape(-1)
+    n = echo.size
+    k_i = max(1, int(round(frac_induction * n)))
+    k_e = max(1, int(round(frac_echo * n)))
+    mask = np.zeros(n, dtype=np.uint8)
+    mask[np.argsort(-induction, kind="stable")[:k_i]] = 1
+    mask[np.argsort(-echo, kind="stable")[:k_e]] = 1
+    return mask

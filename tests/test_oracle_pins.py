@@ -454,3 +454,44 @@ def test_alibi_decode_head_keeps_the_recent_window_and_is_causal():
     hc = orc.compress_head(K[: n + 1], V[: n + 1], n + 1, 0, win, False)
     assert np.allclose(orc.alibi_decode_head(qs[:1], K[: n + 1], V[: n + 1], win, 0.0, 0.6)[0],
                        orc.decode_head(qs[0], hc, 0.6, use_compensation=False), atol=1e-13)
+
+
+# ------------------------------------------------------------------ retrieval-head identification (Section 3.3)
+def test_scores_of_a_head_with_uniform_attention_have_a_closed_form():
+    """q = 0: every causal weight is 1 / (m + 1), so both scores are mean_m (number of earlier copies) / (m + 1)."""
+    n, P, d = 40, 10, 4
+    K = _rng(90).standard_normal((n, d))
+    e, i = orc.echo_induction_scores(np.zeros((n, d)), K, P, 1.0)
+    ref = np.mean([(m // P) / (m + 1) for m in range(P, n)])
+    assert abs(e - ref) < 1e-14 and abs(i - ref) < 1e-14
+
+
+def test_scores_single_out_echo_and_induction_heads():
+    """Keys that are one-hot in the token identity: a query that looks for its own token is an echo head, a
+    query that looks for the token BEFORE a key's position is an induction head (it lands on the successor)."""
+    P, reps, beta = 12, 4, 30.0
+    n = P * reps
+    ids = np.arange(n) % P
+    K = np.eye(P)[ids]                                         # key n encodes token id(n)
+    q_echo = beta * np.eye(P)[ids]                             # looks for the same token
+    K_prev = np.eye(P)[np.roll(ids, 1)]                        # key n encodes the token before n
+    e1, i1 = orc.echo_induction_scores(q_echo, K, P, 1.0)
+    e2, i2 = orc.echo_induction_scores(q_echo, K_prev, P, 1.0) # same query against "previous token" keys
+    # the echo head also sees itself (position m holds the same token), so its echo mass is below 1 but large
+    assert e1 > 0.6 and i1 < 1e-6
+    assert i2 > 0.6 and e2 < 1e-6
+    # brute force of one query
+    m = n - 1
+    s = np.array([float(q_echo[m] @ K[t]) for t in range(m + 1)])
+    w = np.exp(s - s.max()); w /= w.sum()
+    assert abs(sum(w[m - j * P] for j in range(1, reps)) - (reps - 1) / reps) < 1e-9
+
+
+def test_selection_takes_top_induction_and_top_echo_heads():
+    ind = np.linspace(0, 1, 100)                               # head 99 has the largest induction score
+    echo = np.zeros(100); echo[7] = 0.9; echo[99] = 0.5
+    mask = orc.select_retrieval_heads(echo, ind)               # 14 + 1
+    assert mask.sum() == 15 and mask[86:].all() and mask[7] == 1 and mask[85] == 0
+    assert orc.select_retrieval_heads(np.zeros(8), np.arange(8.0)).sum() == 2    # round(1.12)=1 by induction, 1 by echo (head 0)
+    g = _golden()
+    assert g["induction_head_fraction"] == 0.14 and g["echo_head_fraction"] == 0.01
