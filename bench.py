@@ -283,6 +283,35 @@ def decode_only(rz, synth, name, n_layers, dev, peak, reps=60, n_tok=1, alibi=Fa
             "query_tokens_per_call": n_tok, "alibi": bool(alibi)}
 
 
+def head_scores_leg(rz, synth, dev, reps=5):
+    """Section 3.3's score reduction on its own input shape: 2500 random tokens repeated 4 times, 32 heads of
+    dimension 128 (one layer of a 7B-class model).  A dense contraction (causal Q.K^T), so it is reported
+    against the tensor peak; it runs once per model, offline."""
+    import torch
+    H, period, D = 32, 2500, 128
+    n = 4 * period
+    Q = synth.normal_bf16(7, synth.TAG_Q, (H, n, D), dev)
+    K = synth.normal_bf16(7, synth.TAG_K, (H, n, D), dev)
+    rz.razor_head_scores(Q, K, period)
+    torch.cuda.synchronize()
+    a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(reps):
+        rz.razor_head_scores(Q, K, period)
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / reps
+    flops = H * 2.0 * D * (n * (n + 64) / 2.0)          # causal score tiles actually computed (64-query tiles)
+    try:
+        peak = float(json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))["bf16_tflops"])
+        kind = "measured (cuBLAS bf16 burst)"
+    except Exception:
+        peak, kind = 1590.0, "fallback"
+    return {"workload": f"{H} heads x {n} tokens x {D}, period {period}", "ms": ms, "tflops": flops / (ms * 1e-3) / 1e12,
+            "bound": "tensor", "peak_tflops": peak, "peak_kind": kind, "frac": flops / (ms * 1e-3) / 1e12 / peak,
+            "note": "warp-level mma.sync path; an offline, once-per-model step"}
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
@@ -476,6 +505,10 @@ def main():
             line["decode_128k_gqa"] = decode_only(rz, synth, "cfg4", 6, dev, peak)
         except Exception as ex:
             line["decode_128k_gqa"] = {"unavailable": str(ex)[:200]}
+        try:   # retrieval-head identification scores (Section 3.3)
+            line["head_scores"] = head_scores_leg(rz, synth, dev)
+        except Exception as ex:
+            line["head_scores"] = {"unavailable": str(ex)[:200]}
         try:   # the ALiBi variant on the 32K MHA shape
             line["alibi_32k"] = decode_only(rz, synth, "cfg2", 3, dev, peak, alibi=True)
         except Exception as ex:

@@ -257,6 +257,30 @@ RAZOR_API int razor_cache_set_alibi(razor_cache_t* cache, const float* slopes, v
 RAZOR_API int razor_cache_set_head_windows(razor_cache_t* cache, int32_t layer, const int32_t* window_h);
 
 /*
+ * Retrieval-head identification, the arithmetic of Section 3.3.  The model is run (by the caller) on
+ * `period` random tokens repeated several times; for one layer's heads this call takes their
+ * post-rotary queries and keys on that input and returns, per head, the echo score (causal-softmax
+ * attention weight on the earlier copies of the current token, positions m - j*period) and the
+ * induction score (weight on the tokens right after those, m - j*period + 1), each summed over j and
+ * averaged over the queries m >= period.
+ *   Q, K       device bf16 [n_heads, n_tokens, head_dim] contiguous (a grouped-query model passes each
+ *              query head with its KV head's keys); head_dim 64 or 128; 2 <= period < n_tokens
+ *   sm_scale   multiplies q.k; 0 means 1/sqrt(head_dim)
+ *   echo, induction   device fp32 [n_heads]
+ *   scratch    device, razor_head_scores_scratch_bytes(n_heads, n_tokens) bytes, caller-owned
+ * razor_select_retrieval_heads (host only) then marks the top frac_induction of the heads by
+ * induction score and the top frac_echo by echo score (Table 2: 0.14 and 0.01; counts rounded to the
+ * nearest integer, at least one each, ties to the lower index): mask[h] = 1 for a retrieval head.
+ * Errors: NULL_PTR, INVALID_ARG, UNSUPPORTED_DIM, MISALIGNED, POOL_TOO_SMALL (scratch), CUDA.
+ */
+RAZOR_API int razor_head_scores_scratch_bytes(int32_t n_heads, int32_t n_tokens, size_t* bytes);
+RAZOR_API int razor_head_scores(const void* Q, const void* K, int32_t n_heads, int32_t n_tokens, int32_t head_dim,
+                      int32_t dtype, int32_t period, float sm_scale, float* echo, float* induction, void* scratch,
+                      size_t scratch_bytes, void* stream);
+RAZOR_API int razor_select_retrieval_heads(const float* echo, const float* induction, int32_t n_heads,
+                                 float frac_induction, float frac_echo, uint8_t* mask);
+
+/*
  * Self-test of the bounded waits.  Enqueues a one-warp kernel that waits, with the decode kernel's own
  * wait routine and a limit of limit_ns (1 us .. 1 s), on a barrier nothing ever arrives on.  The wait
  * has to give up by itself; razor_cache_device_status then reports bit 16 (and clears it), and the

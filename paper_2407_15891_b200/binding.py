@@ -28,8 +28,8 @@ SYMBOLS = [
     "razor_query_bytes", "razor_cache_create", "razor_compress", "razor_compress_seq", "razor_append",
     "razor_decode_attention", "razor_append_many", "razor_decode_attention_multi", "razor_cache_export", "razor_cache_stats", "razor_schedule_plan",
     "razor_schedule_query", "razor_cache_set_option", "razor_cache_device_status", "razor_cache_wait_selftest", "razor_cache_set_alibi", "razor_cache_set_head_windows",
-    "razor_compensation_mean_static",
-    "razor_cache_reset", "razor_cache_destroy", "razor_status_string",
+    "razor_compensation_mean_static", "razor_head_scores_scratch_bytes", "razor_head_scores",
+    "razor_select_retrieval_heads", "razor_cache_reset", "razor_cache_destroy", "razor_status_string",
     "razor_last_cuda_error", "razor_version",
 ]
 
@@ -86,6 +86,9 @@ def load() -> C.CDLL:
     lib.razor_cache_wait_selftest.argtypes = [vp, i64, vp]
     lib.razor_cache_set_alibi.argtypes = [vp, vp, vp]
     lib.razor_cache_set_head_windows.argtypes = [vp, i32, vp]
+    lib.razor_head_scores_scratch_bytes.argtypes = [i32, i32, C.POINTER(sz)]
+    lib.razor_head_scores.argtypes = [vp, vp, i32, i32, i32, i32, i32, C.c_float, vp, vp, vp, sz, vp]
+    lib.razor_select_retrieval_heads.argtypes = [vp, vp, i32, C.c_float, C.c_float, vp]
     lib.razor_cache_reset.argtypes = [vp]
     lib.razor_cache_destroy.argtypes = [vp]
     lib.razor_status_string.argtypes = [C.c_int]
@@ -282,6 +285,30 @@ def razor_compensation_mean_static(K, V, stride_h: int, stride_n: int, n_kv_head
                                                  ctx_len, n_sink, window, _ptr(mean_k), _ptr(mean_v), C.byref(nd),
                                                  _stream(stream)), "razor_compensation_mean_static")
     return nd.value
+
+
+def razor_head_scores(Q: torch.Tensor, K: torch.Tensor, period: int, sm_scale: float = 0.0, stream=None):
+    """Q, K: bf16 device tensors [H, N, D].  -> (echo, induction) fp32 device tensors [H]."""
+    assert Q.is_contiguous() and K.is_contiguous() and Q.shape == K.shape and Q.dtype == torch.bfloat16
+    H, N, D = Q.shape
+    need = C.c_size_t(0)
+    _check(load().razor_head_scores_scratch_bytes(H, N, C.byref(need)), "razor_head_scores_scratch_bytes")
+    scratch = torch.empty(need.value, dtype=torch.uint8, device=Q.device)
+    echo = torch.empty(H, dtype=torch.float32, device=Q.device)
+    induction = torch.empty(H, dtype=torch.float32, device=Q.device)
+    _check(load().razor_head_scores(_ptr(Q), _ptr(K), H, N, D, RAZOR_BF16, period, sm_scale, _ptr(echo),
+                                    _ptr(induction), _ptr(scratch), need.value, _stream(stream)), "razor_head_scores")
+    return echo, induction
+
+
+def razor_select_retrieval_heads(echo, induction, frac_induction: float = 0.14, frac_echo: float = 0.01) -> np.ndarray:
+    """Host-only: uint8 mask over the heads (1 = retrieval head)."""
+    e = np.ascontiguousarray(np.asarray(echo, dtype=np.float32).reshape(-1))
+    i = np.ascontiguousarray(np.asarray(induction, dtype=np.float32).reshape(-1))
+    mask = np.zeros(e.size, dtype=np.uint8)
+    _check(load().razor_select_retrieval_heads(e.ctypes.data, i.ctypes.data, e.size, frac_induction, frac_echo,
+                                               mask.ctypes.data), "razor_select_retrieval_heads")
+    return mask
 
 
 def razor_cache_reset(cache: int) -> None:
