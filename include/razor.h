@@ -267,7 +267,10 @@ RAZOR_API int razor_cache_set_head_windows(razor_cache_t* cache, int32_t layer, 
  *              query head with its KV head's keys); head_dim 64 or 128; 2 <= period < n_tokens
  *   sm_scale   multiplies q.k; 0 means 1/sqrt(head_dim)
  *   echo, induction   device fp32 [n_heads]
- *   scratch    device, razor_head_scores_scratch_bytes(n_heads, n_tokens) bytes, caller-owned
+ *   scratch    device, 16-byte aligned, razor_head_scores_scratch_bytes(n_heads, n_tokens) bytes,
+ *              caller-owned; its content on entry does not matter
+ * The kernel's internal waits are bounded in time; should one ever run out, every score of the call is
+ * NaN (nothing else is touched, the context stays usable).
  * razor_select_retrieval_heads (host only) then marks the top frac_induction of the heads by
  * induction score and the top frac_echo by echo score (Table 2: 0.14 and 0.01; counts rounded to the
  * nearest integer, at least one each, ties to the lower index): mask[h] = 1 for a retrieval head.
