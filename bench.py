@@ -52,6 +52,8 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-dense", action="store_true")
+    ap.add_argument("--only-head-scores", type=int, default=0, metavar="HEADS",
+                    help="run only the head-score leg on HEADS heads and print its line (profiling; not the bench line)")
     return ap.parse_args()
 
 
@@ -283,12 +285,12 @@ def decode_only(rz, synth, name, n_layers, dev, peak, reps=60, n_tok=1, alibi=Fa
             "query_tokens_per_call": n_tok, "alibi": bool(alibi)}
 
 
-def head_scores_leg(rz, synth, dev, reps=5):
+def head_scores_leg(rz, synth, dev, reps=5, heads=32):
     """Section 3.3's score reduction on its own input shape: 2500 random tokens repeated 4 times, 32 heads of
     dimension 128 (one layer of a 7B-class model).  A dense contraction (causal Q.K^T), so it is reported
     against the tensor peak; it runs once per model, offline."""
     import torch
-    H, period, D = 32, 2500, 128
+    H, period, D = heads, 2500, 128
     n = 4 * period
     Q = synth.normal_bf16(7, synth.TAG_Q, (H, n, D), dev)
     K = synth.normal_bf16(7, synth.TAG_K, (H, n, D), dev)
@@ -301,7 +303,8 @@ def head_scores_leg(rz, synth, dev, reps=5):
     b.record()
     torch.cuda.synchronize()
     ms = a.elapsed_time(b) / reps
-    flops = H * 2.0 * D * (n * (n + 64) / 2.0)          # causal score tiles actually computed (64-query tiles)
+    tiles = sum(t + 1 for t in range((n + 127) // 128) if (t + 1) * 128 > period)   # 128 x 128 score tiles computed
+    flops = H * tiles * 2.0 * 128 * 128 * D
     try:
         peak = float(json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))["bf16_tflops"])
         kind = "measured (cuBLAS bf16 burst)"
@@ -309,7 +312,7 @@ def head_scores_leg(rz, synth, dev, reps=5):
         peak, kind = 1590.0, "fallback"
     return {"workload": f"{H} heads x {n} tokens x {D}, period {period}", "ms": ms, "tflops": flops / (ms * 1e-3) / 1e12,
             "bound": "tensor", "peak_tflops": peak, "peak_kind": kind, "frac": flops / (ms * 1e-3) / 1e12 / peak,
-            "note": "warp-level mma.sync path; an offline, once-per-model step"}
+            "note": "tcgen05 score tiles in tensor memory, exp-bound (one ex2 per score); an offline, once-per-model step"}
 
 
 def main():
@@ -331,6 +334,10 @@ def main():
         raise SystemExit("bench.py needs a CUDA device: the product has no CPU path")
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
+    if args.only_head_scores > 0:
+        if rank == 0:
+            print(json.dumps(head_scores_leg(rz, synth, dev, reps=max(1, args.steps), heads=args.only_head_scores)))
+        return
     dist = None
     if world > 1:
         import torch.distributed as dist

@@ -9,18 +9,24 @@
 //
 // A CTA owns 128 queries of one head (the rows of the accumulator, one per tensor-memory lane) and walks
 // the key tiles up to its own diagonal.  Three roles, connected by mbarriers:
-//   * four LOADER warps copy the next 128 keys into one of two shared-memory stages, in the layout the
-//     matrix unit reads (rows of 128 bytes, eight rows to a 1 KB group, 16-byte chunks XOR-swizzled
-//     by the row number within the group; a row of D = 128 elements is two such half rows);
-//   * one thread of the MMA warp issues the D / 16 instructions of a tile (K = 16 each) into one of two
+//   * one thread issues the TMA copies: the query tile once, then 128 keys at a time into one of two
+//     shared-memory stages.  The tensor map's 128-byte swizzle puts them in the layout the matrix unit
+//     reads (rows of 128 bytes, eight rows to a 1 KB group, 16-byte chunks XOR-swizzled by the row
+//     number within the group; a row of D = 128 elements is two such half rows, one box each), and
+//     rows beyond the sequence arrive as zeros;
+//   * one thread issues the D / 16 matrix instructions of a tile (K = 16 each) into one of two
 //     accumulator buffers and commits them onto the barriers that free the stage and publish the tile;
-//   * four SOFTMAX warps read the tile out of tensor memory, a thread per query: it sees its whole row,
-//     so the running max and sum need no shuffles.  Only the diagonal tile needs the causal mask.
-// The handful of target logits per query are then plain dot products.  Per-CTA partial sums go to
-// caller-provided scratch and are added in a fixed order (reproducible).
+//   * eight SOFTMAX warps read the tile out of tensor memory: warps w and w + 4 share lanes
+//     32 (w % 4) .. + 31, i.e. 32 queries, and take one half of the 128 columns each, so a thread sees
+//     half a row of its query and keeps a running max and sum without shuffles; the two halves are
+//     merged once at the end.  Only the diagonal tile needs the causal mask.
+// The denominators go to scratch; a second, small kernel computes the handful of target logits per query
+// as plain dot products and sums the weights per block; the blocks are added in a fixed order (reproducible).
 //
 // Every barrier wait is bounded in time; a wait that runs out makes the CTA leave through the common
-// exit (tensor memory is always released) and sets a flag in scratch, which turns the scores into NaN.
+// exit (copies in flight are waited for, tensor memory is always released) and sets a flag in scratch,
+// which turns the scores into NaN.
+#include <cuda.h>
 #include <math_constants.h>
 
 #include "razor_common.cuh"
@@ -32,9 +38,9 @@ namespace {
 constexpr int kQTile = 128;         // queries per CTA = accumulator rows = tensor-memory lanes
 constexpr int kKTile = 128;         // keys per tile = accumulator columns
 constexpr int kStages = 2;          // key stages in shared memory and accumulator buffers in tensor memory
-constexpr int kSoftmaxWarps = 4;    // warp w reads tensor-memory lanes 32 w .. 32 w + 31
-constexpr int kLoaderWarps = 4;
-constexpr int kScoreWarps = kSoftmaxWarps + kLoaderWarps + 1;
+constexpr int kSoftmaxWarps = 8;    // warp w: lanes 32 (w % 4) .. + 31, columns 64 (w / 4) .. + 63
+constexpr int kCopyWarp = kSoftmaxWarps, kMmaWarp = kSoftmaxWarps + 1;
+constexpr int kScoreWarps = kSoftmaxWarps + 2;
 constexpr int kScoreThreads = kScoreWarps * 32;
 constexpr uint32_t kTmemCols = kStages * kKTile;   // a power of two >= 32
 constexpr int kHalfRowBytes = 128;                 // one swizzle row: 64 bf16
@@ -42,15 +48,15 @@ constexpr int kHalfTileBytes = 128 * kHalfRowBytes;
 
 // Barriers and small exchange areas behind the tiles.
 struct ScoreCtl {
-  uint64_t k_full[kStages];    // loaders -> MMA: the stage holds its keys
-  uint64_t k_empty[kStages];   // MMA (commit) -> loaders: the stage has been read
+  uint64_t q_full;             // copy -> MMA: the query tile has landed
+  uint64_t k_full[kStages];    // copy -> MMA: the stage holds its keys
+  uint64_t k_empty[kStages];   // MMA (commit) -> copy: the stage has been read
   uint64_t t_full[kStages];    // MMA (commit) -> softmax: the accumulator buffer holds a tile
   uint64_t t_empty[kStages];   // softmax -> MMA: the buffer has been read out
   uint64_t drain;              // abort path: MMAs in flight have finished
   uint32_t tmem_base;
   int abort_flag;
-  float lse[kQTile];           // log2 of each query's softmax denominator
-  float red[kScoreWarps][2];
+  float2 half_ml[kQTile];      // (max, sum) of the upper column half, for the merge
 };
 
 template <int D>
@@ -88,15 +94,13 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-// 32 consecutive columns of this thread's lane, complete on return.
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+// Issues the load of 32 consecutive columns of this thread's lane; the registers are valid after tmem_ld_wait().
+__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t* v) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
       "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
-      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n\t"
-      "tcgen05.wait::ld.sync.aligned;"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
       : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
         "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
         "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
@@ -104,28 +108,36 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
       : "r"(taddr)
       : "memory");
 }
-
-// Rows [row0, row0 + 128) of X[n_tokens][D] into a tile in the matrix unit's layout; rows beyond the
-// sequence are zero.  Called by `n_thr` threads with ranks `t`.
-template <int D>
-__device__ __forceinline__ void stage_tile(uint8_t* tile, const __nv_bfloat16* __restrict__ X, int row0, int n_tokens,
-                                           int t, int n_thr) {
-  constexpr int CH = D / 8;   // 16-byte chunks per row
-  for (int idx = t; idx < 128 * CH; idx += n_thr) {
-    const int r = idx / CH, c = idx % CH;
-    uint4 v = make_uint4(0u, 0u, 0u, 0u);
-    if (row0 + r < n_tokens) v = ((const uint4*)(X + (size_t)(row0 + r) * D))[c];
-    *(uint4*)(tile + (c >> 3) * kHalfTileBytes + r * kHalfRowBytes + (((c & 7) ^ (r & 7)) << 4)) = v;
-  }
+// Completes the loads issued so far.  The registers pass through the statement so that no use of them
+// can be scheduled ahead of it.
+__device__ __forceinline__ void tmem_ld_wait(uint32_t (&v)[64]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int j = 0; j < 64; ++j) asm volatile("" : "+r"(v[j]));
 }
 
-// grid = (query tiles, heads), block = kScoreThreads.
-// scratch[(head * n_tiles + tile) * 2 + {0: echo, 1: induction}]; *fault is set when a wait gave up.
+// One box of the [heads][tokens][D] tensor (64 elements x 128 rows of one head) into shared memory;
+// completion is counted in bytes on `bar`.  x is a multiple of 64 elements, i.e. of 128 bytes.
+__device__ __forceinline__ void tma_load_box(void* dst, const CUtensorMap* map, int x, int row, int head, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::
+          "r"(smem_u32(dst)),
+      "l"(map), "r"(x), "r"(row), "r"(head), "r"(smem_u32(bar))
+      : "memory");
+}
 template <int D>
-__global__ void __launch_bounds__(kScoreThreads, 2) head_scores_kernel(const __nv_bfloat16* __restrict__ Q,
-                                                                       const __nv_bfloat16* __restrict__ K,
-                                                                       int n_tokens, int period, float scale_log2,
-                                                                       float* __restrict__ scratch, int* fault) {
+__device__ __forceinline__ void tma_load_tile(uint8_t* tile, const CUtensorMap* map, int row0, int head, uint64_t* bar) {
+  mbar_arrive_expect_tx(bar, (uint32_t)score_tile_bytes<D>());
+#pragma unroll
+  for (int h = 0; h < D / 64; ++h) tma_load_box(tile + h * kHalfTileBytes, map, h * 64, row0, head, bar);
+}
+
+// grid = (query tiles, heads), block = kScoreThreads.  Writes lse[head][m], the log2 of the causal softmax
+// denominator of query m (scaled logits in the log2 domain); *fault is set when a wait gave up.
+template <int D>
+__global__ void __launch_bounds__(kScoreThreads, 2)
+    head_lse_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k, int n_tokens,
+                    int period, float scale_log2, float* __restrict__ lse, int* fault) {
   constexpr int TB = score_tile_bytes<D>();
   extern __shared__ uint8_t smem_raw[];
   uint8_t* base = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
@@ -137,17 +149,12 @@ __global__ void __launch_bounds__(kScoreThreads, 2) head_scores_kernel(const __n
   const int tile = n_tiles - 1 - (int)blockIdx.x;   // the long rows of the triangle first
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int q0 = tile * kQTile;
-  const __nv_bfloat16* Qh = Q + (size_t)head * n_tokens * D;
-  const __nv_bfloat16* Kh = K + (size_t)head * n_tokens * D;
-  float* dst = scratch + ((size_t)head * n_tiles + tile) * 2;
-  if (q0 + kQTile <= period) {   // none of these queries has an earlier copy of its token
-    if (threadIdx.x == 0) dst[0] = dst[1] = 0.f;
-    return;
-  }
+  if (q0 + kQTile <= period) return;   // none of these queries has an earlier copy of its token
   volatile int* abort_flag = &ctl->abort_flag;
   if (threadIdx.x == 0) {
+    mbar_init(&ctl->q_full, 1);
     for (int s = 0; s < kStages; ++s) {
-      mbar_init(&ctl->k_full[s], kLoaderWarps * 32);
+      mbar_init(&ctl->k_full[s], 1);
       mbar_init(&ctl->k_empty[s], 1);
       mbar_init(&ctl->t_full[s], 1);
       mbar_init(&ctl->t_empty[s], kSoftmaxWarps * 32);
@@ -156,14 +163,12 @@ __global__ void __launch_bounds__(kScoreThreads, 2) head_scores_kernel(const __n
     ctl->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == kScoreWarps - 1) {   // the MMA warp owns the tensor-memory allocation
+  if (warp == kMmaWarp) {   // the MMA warp owns the tensor-memory allocation
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)),
                  "r"(kTmemCols)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  stage_tile<D>(qtile, Qh, q0, n_tokens, threadIdx.x, kScoreThreads);
-  fence_async_smem();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -171,58 +176,67 @@ __global__ void __launch_bounds__(kScoreThreads, 2) head_scores_kernel(const __n
   const int n_kt = tile + 1;   // key tiles up to and including the diagonal
 
   if (warp < kSoftmaxWarps) {
-    // ---- softmax: thread = query q0 + threadIdx.x, lane threadIdx.x of the accumulator
-    const int row = threadIdx.x;
+    // ---- softmax: query q0 + row, columns [col0, col0 + 64) of every tile
+    const int row = (warp & 3) * 32 + lane, col0 = (warp >> 2) * 64;
     float m_run = -CUDART_INF_F, l_run = 0.f;
-    const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+    const uint32_t lane_addr = tmem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)col0;
     for (int kt = 0; kt < n_kt; ++kt) {
       const int b = kt & 1;
       if (!__all_sync(0xffffffffu, mbar_wait(&ctl->t_full[b], (kt >> 1) & 1, abort_flag))) break;
       tc_fence_after();
-      const bool diag = kt == tile;
-#pragma unroll 1
-      for (int c4 = 0; c4 < kKTile / 32; ++c4) {
-        uint32_t v[32];
-        tmem_ld32(lane_addr + (uint32_t)(b * kKTile + c4 * 32), v);
-        if (c4 == kKTile / 32 - 1) {   // the buffer is in registers: hand it back
-          tc_fence_before();
-          mbar_arrive(&ctl->t_empty[b]);
-        }
-        float x[32];
-        float mx = -CUDART_INF_F;
+      uint32_t v[64];
+      tmem_ld32_issue(lane_addr + (uint32_t)(b * kKTile), v);
+      tmem_ld32_issue(lane_addr + (uint32_t)(b * kKTile + 32), v + 32);
+      tmem_ld_wait(v);
+      tc_fence_before();
+      mbar_arrive(&ctl->t_empty[b]);   // the buffer is in registers: hand it back
+      float mx[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
+      if (kt == tile) {   // causality: key q0 + column against query q0 + row
 #pragma unroll
-        for (int j = 0; j < 32; ++j) x[j] = __uint_as_float(v[j]) * scale_log2;
-        if (diag) {   // causality: key q0 + column against query q0 + row
+        for (int j = 0; j < 64; ++j)
+          if (col0 + j > row) v[j] = 0xff800000u;   // -inf
+      }
 #pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (c4 * 32 + j > row) x[j] = -CUDART_INF_F;
-        }
+      for (int j = 0; j < 64; ++j) mx[j & 3] = fmaxf(mx[j & 3], __uint_as_float(v[j]));
+      // the scale is positive, so the max of the scaled logits is the scaled max
+      const float tile_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale_log2;
+      const float mn = fmaxf(m_run, tile_max);
+      const float mu = (mn == -CUDART_INF_F) ? 0.f : mn;   // a fully masked half row so far
+      float sum[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-        for (int j = 0; j < 32; ++j) mx = fmaxf(mx, x[j]);
-        const float mn = fmaxf(m_run, mx);   // finite: column 0 of tile 0 is never masked
-        float sum = 0.f;
-#pragma unroll
-        for (int j = 0; j < 32; ++j) sum += fast_exp2(x[j] - mn);
-        l_run = l_run * fast_exp2(m_run - mn) + sum;
-        m_run = mn;
+      for (int j = 0; j < 64; ++j) sum[j & 3] += fast_exp2(fmaf(__uint_as_float(v[j]), scale_log2, -mu));
+      l_run = l_run * fast_exp2(m_run - mu) + ((sum[0] + sum[1]) + (sum[2] + sum[3]));
+      m_run = mn;
+    }
+    if (col0) ctl->half_ml[row] = make_float2(m_run, l_run);
+    asm volatile("bar.sync 1, %0;" ::"n"(kSoftmaxWarps * 32) : "memory");   // the softmax warps only
+    if (!col0 && q0 + row < n_tokens) {
+      const float2 o = ctl->half_ml[row];
+      const float mn = fmaxf(m_run, o.x);   // finite: column 0 of tile 0 is never masked
+      const float l = l_run * fast_exp2(m_run - mn) + o.y * fast_exp2(o.x - mn);
+      lse[(size_t)head * n_tokens + q0 + row] = mn + log2f(l);
+    }
+  } else if (warp == kCopyWarp) {
+    // ---- TMA issue: one thread
+    if (lane == 0) {
+      tma_load_tile<D>(qtile, &map_q, q0, head, &ctl->q_full);
+      int issued = 0;
+      for (int kt = 0; kt < n_kt; ++kt) {
+        const int s = kt & 1;
+        if (kt >= kStages && !mbar_wait(&ctl->k_empty[s], ((kt >> 1) - 1) & 1, abort_flag)) break;
+        tma_load_tile<D>(ktile + s * TB, &map_k, kt * kKTile, head, &ctl->k_full[s]);
+        issued = kt + 1;
+      }
+      if (*abort_flag) {   // leaving early: the copies in flight must land before the CTA may exit
+        (void)mbar_wait_drain(&ctl->q_full, 0);
+        for (int kt = max(0, issued - kStages); kt < issued; ++kt) (void)mbar_wait_drain(&ctl->k_full[kt & 1], (kt >> 1) & 1);
       }
     }
-    ctl->lse[row] = m_run + log2f(l_run);
-  } else if (warp < kSoftmaxWarps + kLoaderWarps) {
-    // ---- loaders
-    const int t = threadIdx.x - kSoftmaxWarps * 32;
-    for (int kt = 0; kt < n_kt; ++kt) {
-      const int s = kt & 1;
-      if (kt >= kStages && !__all_sync(0xffffffffu, mbar_wait(&ctl->k_empty[s], ((kt >> 1) - 1) & 1, abort_flag)))
-        break;
-      stage_tile<D>(ktile + s * TB, Kh, kt * kKTile, n_tokens, t, kLoaderWarps * 32);
-      fence_async_smem();
-      mbar_arrive(&ctl->k_full[s]);
-    }
+    __syncwarp();
   } else {
     // ---- MMA issue: one thread
     if (lane == 0) {
-      bool ok = true;
+      bool ok = mbar_wait(&ctl->q_full, 0, abort_flag);
       for (int kt = 0; kt < n_kt && ok; ++kt) {
         const int s = kt & 1;
         ok = mbar_wait(&ctl->k_full[s], (kt >> 1) & 1, abort_flag);
@@ -247,83 +261,165 @@ __global__ void __launch_bounds__(kScoreThreads, 2) head_scores_kernel(const __n
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == kScoreWarps - 1) {
+  if (warp == kMmaWarp) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
   }
-  if (*abort_flag) {
-    if (threadIdx.x == 0) {
-      atomicOr(fault, 1);
-      dst[0] = dst[1] = 0.f;
-    }
-    return;
+  if (*abort_flag && threadIdx.x == 0) atomicOr(fault, 1);
+}
+
+// E = 4 or 8 consecutive bf16 (8 or 16 bytes, aligned) as floats.
+template <int E>
+__device__ __forceinline__ void load_bf16(const __nv_bfloat16* p, float (&f)[E]) {
+  static_assert(E == 4 || E == 8, "one 8- or 16-byte load");
+  uint32_t w[E / 2];
+  if constexpr (E == 8) {
+    const uint4 u = __ldg((const uint4*)p);
+    w[0] = u.x; w[1] = u.y; w[2] = u.z; w[3] = u.w;
+  } else {
+    const uint2 u = __ldg((const uint2*)p);
+    w[0] = u.x; w[1] = u.y;
   }
-  // ---- the target logits: a few plain dot products per query, lanes splitting the head dimension
-  constexpr int PER = D / 32;
-  float echo = 0.f, induction = 0.f;
-  for (int qi = warp; qi < kQTile; qi += kScoreWarps) {
-    const int m = q0 + qi;
-    if (m < period || m >= n_tokens) continue;   // warp-uniform
-    const float lse = ctl->lse[qi];
-    float qv[PER];
 #pragma unroll
-    for (int e = 0; e < PER; ++e) qv[e] = __bfloat162float(Qh[(size_t)m * D + lane * PER + e]);
-    for (int n = m - period; n >= 0; n -= period) {
-      float de = 0.f, di = 0.f;
-#pragma unroll
-      for (int e = 0; e < PER; ++e) {
-        de += qv[e] * __bfloat162float(Kh[(size_t)n * D + lane * PER + e]);
-        di += qv[e] * __bfloat162float(Kh[(size_t)(n + 1) * D + lane * PER + e]);
-      }
-#pragma unroll
-      for (int off = 16; off > 0; off >>= 1) {
-        de += __shfl_xor_sync(0xffffffffu, de, off);
-        di += __shfl_xor_sync(0xffffffffu, di, off);
-      }
-      echo += fast_exp2(de * scale_log2 - lse);
-      induction += fast_exp2(di * scale_log2 - lse);
-    }
-  }
-  if (lane == 0) {
-    ctl->red[warp][0] = echo;
-    ctl->red[warp][1] = induction;
-  }
-  __syncthreads();
-  if (threadIdx.x < 2) {
-    float sum = 0.f;
-    for (int w = 0; w < kScoreWarps; ++w) sum += ctl->red[w][threadIdx.x];
-    dst[threadIdx.x] = sum;
+  for (int i = 0; i < E / 2; ++i) {   // bf16 -> fp32 is a 16-bit shift
+    f[2 * i] = __uint_as_float(w[i] << 16);
+    f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
   }
 }
 
-// grid = heads, block = 32: tiles added in order, then the mean over the queries m >= period.
+constexpr int kTargetQueries = 64;   // queries per CTA of the target kernel (8 warps x 8 queries)
+
+// The handful of target logits per query, as plain dot products, turned into attention weights with the
+// denominators from head_lse_kernel.  A warp takes a query and one earlier copy of its token at a time:
+// its lower 16 lanes hold the copy's key (echo), its upper 16 lanes the key after it (induction), each
+// lane D / 16 elements.  grid = (ceil(n_tokens / 64), heads), block = 256;
+// partial[(head * n_blocks + block) * 2 + {0: echo, 1: induction}] = the block's sums of weights.
+template <int D>
+__global__ void __launch_bounds__(256) head_targets_kernel(const __nv_bfloat16* __restrict__ Q,
+                                                           const __nv_bfloat16* __restrict__ K,
+                                                           const float* __restrict__ lse, int n_tokens, int period,
+                                                           float scale_log2, float* __restrict__ partial) {
+  constexpr int E = D / 16;   // elements per lane
+  __shared__ float red[8][2];
+  const int head = blockIdx.y, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int kind = lane >> 4, l16 = lane & 15;
+  const __nv_bfloat16* Qh = Q + (size_t)head * n_tokens * D;
+  const __nv_bfloat16* Kh = K + (size_t)head * n_tokens * D;
+  // The warp's 8 queries are consecutive, so are their targets in every earlier period: one batch of 8
+  // independent row loads per period.
+  const int m0 = (int)blockIdx.x * kTargetQueries + warp * 8;
+  float qf[8][E], lse_m[8];
+#pragma unroll
+  for (int qi = 0; qi < 8; ++qi) {
+    const int m = min(m0 + qi, n_tokens - 1);
+    load_bf16<E>(Qh + (size_t)m * D + l16 * E, qf[qi]);
+    lse_m[qi] = lse[(size_t)head * n_tokens + m];
+  }
+  float acc = 0.f;
+  for (int c0 = m0 - period; c0 + 7 >= 0; c0 -= period) {   // c0 + qi: the copy of query m0 + qi's token
+    float dot[8];
+#pragma unroll
+    for (int qi = 0; qi < 8; ++qi) {
+      const int c = max(c0 + qi, 0);   // clamped rows are discarded below; c + kind <= m - period + 1
+      float kf[E];
+      load_bf16<E>(Kh + (size_t)(c + kind) * D + l16 * E, kf);
+      dot[qi] = 0.f;
+#pragma unroll
+      for (int e = 0; e < E; ++e) dot[qi] = fmaf(qf[qi][e], kf[e], dot[qi]);
+    }
+#pragma unroll
+    for (int off = 8; off > 0; off >>= 1)
+#pragma unroll
+      for (int qi = 0; qi < 8; ++qi) dot[qi] += __shfl_xor_sync(0xffffffffu, dot[qi], off);
+#pragma unroll
+    for (int qi = 0; qi < 8; ++qi)
+      if (c0 + qi >= 0 && m0 + qi < n_tokens) acc += fast_exp2(dot[qi] * scale_log2 - lse_m[qi]);
+  }
+  if (l16 == 0) red[warp][kind] = acc;
+  __syncthreads();
+  if (threadIdx.x < 2) {
+    float sum = 0.f;
+    for (int w = 0; w < 8; ++w) sum += red[w][threadIdx.x];
+    partial[((size_t)head * gridDim.x + blockIdx.x) * 2 + threadIdx.x] = sum;
+  }
+}
+
+// grid = heads, block = 32: the blocks' sums added, then the mean over the queries m >= period.
 // A launch in which some wait gave up has no valid partial sums: its scores are NaN.
 __global__ void head_scores_finalize_kernel(const float* __restrict__ scratch, const int* __restrict__ fault,
-                                            int n_tiles, int n_queries, float* __restrict__ echo,
+                                            int n_blocks, int n_queries, float* __restrict__ echo,
                                             float* __restrict__ induction) {
-  if (threadIdx.x >= 2) return;
-  const float* src = scratch + (size_t)blockIdx.x * n_tiles * 2 + threadIdx.x;
-  float s = 0.f;
-  for (int i = 0; i < n_tiles; ++i) s += src[(size_t)i * 2];
-  float mean = n_queries > 0 ? s / (float)n_queries : 0.f;
-  if (*fault) mean = CUDART_NAN_F;
-  (threadIdx.x == 0 ? echo : induction)[blockIdx.x] = mean;
+  const int lane = threadIdx.x;
+  const float* src = scratch + (size_t)blockIdx.x * n_blocks * 2;
+  float e = 0.f, i = 0.f;
+  for (int b = lane; b < n_blocks; b += 32) {   // lane-strided, then a fixed tree: the same order every run
+    e += src[2 * b];
+    i += src[2 * b + 1];
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    e += __shfl_xor_sync(0xffffffffu, e, off);
+    i += __shfl_xor_sync(0xffffffffu, i, off);
+  }
+  if (lane == 0) {
+    const bool bad = *fault != 0;
+    echo[blockIdx.x] = bad ? CUDART_NAN_F : (n_queries > 0 ? e / (float)n_queries : 0.f);
+    induction[blockIdx.x] = bad ? CUDART_NAN_F : (n_queries > 0 ? i / (float)n_queries : 0.f);
+  }
+}
+
+// cuTensorMapEncodeTiled, looked up through the runtime (the library does not link against the driver).
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q = cudaDriverEntryPointSymbolNotFound;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+      p = nullptr;
+    return (EncodeTiledFn)p;
+  }();
+  return fn;
+}
+
+// Tensor map of X[n_heads][n_tokens][D] bf16 with boxes of 64 elements x 128 rows of one head, written
+// to shared memory with the 128-byte swizzle; rows beyond n_tokens read as zeros.
+template <int D>
+bool make_tile_map(CUtensorMap* map, const void* X, int n_heads, int n_tokens) {
+  const EncodeTiledFn encode = encode_tiled_fn();
+  if (!encode) return false;
+  const cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)n_tokens, (cuuint64_t)n_heads};
+  const cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)n_tokens * D * 2};   // bytes, dimensions 1 and 2
+  const cuuint32_t box[3] = {64, 128, 1};
+  const cuuint32_t elem_strides[3] = {1, 1, 1};
+  return encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(X), dims, strides, box, elem_strides,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 template <int D>
 cudaError_t run_head_scores(const void* Q, const void* K, int n_heads, int n_tokens, int period, float scale_log2,
-                            float* echo, float* induction, float* partial, int* fault, cudaStream_t s) {
-  const int tiles = (n_tokens + kQTile - 1) / kQTile;
-  cudaError_t e = cudaFuncSetAttribute(head_scores_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                            float* echo, float* induction, float* partial, float* lse, int* fault, cudaStream_t s) {
+  const int tiles = (n_tokens + kQTile - 1) / kQTile, blocks = (n_tokens + kTargetQueries - 1) / kTargetQueries;
+  CUtensorMap map_q, map_k;
+  if (!make_tile_map<D>(&map_q, Q, n_heads, n_tokens) || !make_tile_map<D>(&map_k, K, n_heads, n_tokens))
+    return cudaErrorInvalidValue;
+  cudaError_t e = cudaFuncSetAttribute(head_lse_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        (int)score_smem_bytes<D>());
   if (e != cudaSuccess) return e;
   e = cudaMemsetAsync(fault, 0, sizeof(int), s);
   if (e != cudaSuccess) return e;
-  head_scores_kernel<D><<<dim3(tiles, n_heads), kScoreThreads, score_smem_bytes<D>(), s>>>(
-      (const __nv_bfloat16*)Q, (const __nv_bfloat16*)K, n_tokens, period, scale_log2, partial, fault);
+  head_lse_kernel<D><<<dim3(tiles, n_heads), kScoreThreads, score_smem_bytes<D>(), s>>>(map_q, map_k, n_tokens, period,
+                                                                                        scale_log2, lse, fault);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  head_scores_finalize_kernel<<<n_heads, 32, 0, s>>>(partial, fault, tiles, n_tokens - period, echo, induction);
+  head_targets_kernel<D><<<dim3(blocks, n_heads), 256, 0, s>>>((const __nv_bfloat16*)Q, (const __nv_bfloat16*)K, lse,
+                                                              n_tokens, period, scale_log2, partial);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  head_scores_finalize_kernel<<<n_heads, 32, 0, s>>>(partial, fault, blocks, n_tokens - period, echo, induction);
   return cudaGetLastError();
 }
 
@@ -331,16 +427,20 @@ cudaError_t run_head_scores(const void* Q, const void* K, int n_heads, int n_tok
 }  // namespace razor
 
 namespace {
+// Scratch layout: per-block partial sums | lse[n_heads][n_tokens] | fault word.
 size_t partial_bytes(int n_heads, int n_tokens) {
-  const size_t tiles = ((size_t)n_tokens + razor::kQTile - 1) / razor::kQTile;
-  return ((size_t)n_heads * tiles * 2 * sizeof(float) + 255) / 256 * 256;
+  const size_t blocks = ((size_t)n_tokens + razor::kTargetQueries - 1) / razor::kTargetQueries;
+  return ((size_t)n_heads * blocks * 2 * sizeof(float) + 255) / 256 * 256;
+}
+size_t lse_bytes(int n_heads, int n_tokens) {
+  return ((size_t)n_heads * (size_t)n_tokens * sizeof(float) + 255) / 256 * 256;
 }
 }  // namespace
 
 extern "C" int razor_head_scores_scratch_bytes(int32_t n_heads, int32_t n_tokens, size_t* bytes) {
   if (!bytes) return RAZOR_E_NULL_PTR;
   if (n_heads < 1 || n_tokens < 1) return RAZOR_E_INVALID_ARG;
-  *bytes = partial_bytes(n_heads, n_tokens) + 256;   // per-tile partial sums, then the fault word
+  *bytes = partial_bytes(n_heads, n_tokens) + lse_bytes(n_heads, n_tokens) + 256;
   return RAZOR_OK;
 }
 
@@ -359,11 +459,12 @@ extern "C" int razor_head_scores(const void* Q, const void* K, int32_t n_heads, 
   const float scale = sm_scale == 0.f ? 1.0f / sqrtf((float)head_dim) : sm_scale;
   const float scale_log2 = scale * 1.4426950408889634f;
   float* partial = (float*)scratch;
-  int* fault = (int*)((uint8_t*)scratch + partial_bytes(n_heads, n_tokens));
+  float* lse = (float*)((uint8_t*)scratch + partial_bytes(n_heads, n_tokens));
+  int* fault = (int*)((uint8_t*)lse + lse_bytes(n_heads, n_tokens));
   cudaStream_t s = (cudaStream_t)stream;
   const cudaError_t e =
-      head_dim == 128 ? run_head_scores<128>(Q, K, n_heads, n_tokens, period, scale_log2, echo, induction, partial, fault, s)
-                      : run_head_scores<64>(Q, K, n_heads, n_tokens, period, scale_log2, echo, induction, partial, fault, s);
+      head_dim == 128 ? run_head_scores<128>(Q, K, n_heads, n_tokens, period, scale_log2, echo, induction, partial, lse, fault, s)
+                      : run_head_scores<64>(Q, K, n_heads, n_tokens, period, scale_log2, echo, induction, partial, lse, fault, s);
   if (e != cudaSuccess) {
     (void)cudaGetLastError();
     return RAZOR_E_CUDA;
