@@ -2,10 +2,10 @@
  * razor.h - C ABI of the B200 (sm_100a) RazorAttention hot path.
  *
  * RazorAttention (arXiv 2407.15891) keeps the whole KV cache only for "retrieval" heads.  Every
- * other head keeps its first N0 attention-sink tokens and its most recent L tokens (Algorithm 1,
- * lines 2-3) and folds all dropped tokens into one compensation token, the mean of the dropped
+ * other head keeps its first N0 attention-sink tokens and its most recent L tokens (Algorithm 1)
+ * and folds all dropped tokens into one compensation token, the mean of the dropped
  * keys and values (Eq. 4).  At decode time that token enters the softmax with weight N_d, the
- * number of dropped tokens (Eq. 5); retrieval heads use ordinary attention (Algorithm 1, line 5).
+ * number of dropped tokens (Eq. 5); retrieval heads use ordinary attention (Algorithm 1).
  *
  * This library builds that head-heterogeneous cache at the end of prefill (razor_compress), adds
  * decode tokens to it (razor_append) and runs decode attention over it (razor_decode_attention).
@@ -76,7 +76,7 @@ typedef struct {
 } razor_config_t;
 
 /*
- * Sizes of the two caller-owned device buffers (Algorithm 1, line 2 fixes how many tokens each
+ * Sizes of the two caller-owned device buffers (Algorithm 1 fixes how many tokens each
  * head keeps).  ctx_len[B], window[B]: host; head_is_retrieval[L*Hkv]: host, 1 = the KV head keeps
  * every token (for grouped-query models the caller ORs the flags of the group's query heads,
  * Section 4.1).  pool_bytes covers every layer compressed once, with room for max_new_tokens
@@ -94,7 +94,7 @@ RAZOR_API int razor_cache_create(razor_cache_t** out, const razor_config_t* cfg,
                        void* workspace_dev, size_t workspace_bytes, void* stream);
 
 /*
- * Prefill-end compression of one layer (Algorithm 1 lines 1-4, Eq. 4).
+ * Prefill-end compression of one layer (Algorithm 1, Eq. 4).
  *   K, V     device, [B, Hkv, N, D] with element strides stride_b / stride_h / stride_n (innermost
  *            dimension contiguous); rows at or beyond ctx_len[b] are never read.  Base pointers
  *            16-byte aligned, strides multiples of 16 bytes.
@@ -102,7 +102,7 @@ RAZOR_API int razor_cache_create(razor_cache_t** out, const razor_config_t* cfg,
  *   head_is_retrieval  host [Hkv] for this layer
  *   n_sink   must equal config.n_sink
  *   window   host [B]: recent-window length L_h of each sequence (>= 0); the caller evaluates
- *            max(S0, N/C) of Algorithm 1 line 2
+ *            max(S0, N/C) of Algorithm 1
  * A retrieval head, and any head with ctx_len <= n_sink + window, keeps positions [0, N).  Any
  * other head keeps [0, n_sink) and [N - window, N); positions [n_sink, N - window) are summed in
  * fp32 into its compensation sums, and the means and the count N_d are stored.  Kept rows are
@@ -136,8 +136,8 @@ RAZOR_API int razor_compress_seq(razor_cache_t* cache, int32_t layer, int32_t b,
 RAZOR_API int razor_append(razor_cache_t* cache, int32_t layer, const void* k_new, const void* v_new, void* stream);
 
 /*
- * Decode attention of one query token per sequence over the compressed layer (Eq. 5; Algorithm 1
- * line 5).  q: device [B, Hq, D] contiguous, config.dtype.  out: device [B, Hq, D] fp32.
+ * Decode attention of one query token per sequence over the compressed layer (Eq. 5; Algorithm 1).
+ * q: device [B, Hq, D] contiguous, config.dtype.  out: device [B, Hq, D] fp32.
  * Query head j reads KV head j / group.  For a head with N_d > 0 dropped tokens
  *   out = (N_d e^{s_c} v_hat + sum_kept e^{s_n} v_n) / (N_d e^{s_c} + sum_kept e^{s_n}),
  *   s_n = sm_scale q.k_n,  s_c = sm_scale q.k_hat;

@@ -35,14 +35,14 @@ from typing import List, Optional, Sequence, Tuple
 import numpy as np
 
 
-# --------------------------------------------------------------------------- Algorithm 1, lines 2-3
+# --------------------------------------------------------------------------- Algorithm 1
 def buffer_length(n_ctx: int, s0: int, c: int) -> int:
-    """Algorithm 1 line 2 / Table 2: L_h = max(S0, N / C), N / C floored."""
+    """Algorithm 1 / Table 2: L_h = max(S0, N / C), N / C floored."""
     return max(int(s0), int(n_ctx) // int(c))
 
 
 def kept_positions(n_ctx: int, n_sink: int, window: int, is_retrieval: bool) -> np.ndarray:
-    """Algorithm 1 line 3: positions kept by one head, ascending.
+    """Algorithm 1: positions kept by one head, ascending.
 
     Retrieval heads keep every token.  Any other head keeps the first `n_sink`
     positions and the most recent `window` positions; everything between is dropped.
@@ -56,7 +56,7 @@ def kept_positions(n_ctx: int, n_sink: int, window: int, is_retrieval: bool) -> 
 
 
 def dropped_positions(n_ctx: int, n_sink: int, window: int, is_retrieval: bool) -> np.ndarray:
-    """Algorithm 1 line 3: the set {D} of dropped positions (complement of the kept set)."""
+    """Algorithm 1: the set {D} of dropped positions (complement of the kept set)."""
     keep = np.zeros(int(n_ctx), dtype=bool)
     keep[kept_positions(n_ctx, n_sink, window, is_retrieval)] = True
     return np.nonzero(~keep)[0].astype(np.int64)
@@ -86,7 +86,7 @@ def compensation_token(K: np.ndarray, V: np.ndarray, dropped: np.ndarray) -> Tup
 
 # --------------------------------------------------------------------------- original attention
 def full_attention(q: np.ndarray, K: np.ndarray, V: np.ndarray, scale: float) -> np.ndarray:
-    """Softmax attention of one query over all rows of K, V (retrieval heads, Algorithm 1 line 5)."""
+    """Softmax attention of one query over all rows of K, V (retrieval heads, Algorithm 1)."""
     q = np.asarray(q, dtype=np.float64)
     K = np.asarray(K, dtype=np.float64)
     V = np.asarray(V, dtype=np.float64)
@@ -138,7 +138,7 @@ class HeadCache:
 
 def compress_head(K: np.ndarray, V: np.ndarray, n_ctx: int, n_sink: int, window: int,
                   is_retrieval: bool) -> HeadCache:
-    """Algorithm 1 lines 2-3 and Eq. 4 for one head.  K, V: [>= n_ctx, D]; rows >= n_ctx ignored."""
+    """Algorithm 1 and Eq. 4 for one head.  K, V: [>= n_ctx, D]; rows >= n_ctx ignored."""
     K = np.asarray(K)[:n_ctx]
     V = np.asarray(V)[:n_ctx]
     kept = kept_positions(n_ctx, n_sink, window, is_retrieval)
@@ -148,7 +148,7 @@ def compress_head(K: np.ndarray, V: np.ndarray, n_ctx: int, n_sink: int, window:
 
 
 def decode_head(q: np.ndarray, hc: HeadCache, scale: float, use_compensation: bool = True) -> np.ndarray:
-    """Algorithm 1 line 5 for one query head: Eq. 5 (or plain attention when nothing was dropped).
+    """Algorithm 1 for one query head: Eq. 5 (or plain attention when nothing was dropped).
 
     use_compensation=False gives plain truncation (the scheme of Table 1: recent tokens only).
     """

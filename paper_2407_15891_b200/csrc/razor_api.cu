@@ -1,5 +1,5 @@
 // Host side of the C ABI declared in include/razor.h: argument checks, the per-head plan
-// (Algorithm 1 line 2: how many tokens each head keeps), page allocation, host mirrors of the
+// (Algorithm 1: how many tokens each head keeps), page allocation, host mirrors of the
 // per-head lengths (they are deterministic, so no device->host read is ever needed), the cached
 // decode schedule, and the kernel launches.
 #include <algorithm>
@@ -84,7 +84,7 @@ Layout make_layout(const razor_config_t& c) {
   return l;
 }
 
-// Tokens a head can ever hold (Algorithm 1 line 3 plus room for appended decode tokens).
+// Tokens a head can ever hold (Algorithm 1 plus room for appended decode tokens).
 inline long long head_capacity_tokens(const razor_config_t& c, int n_ctx, int window, bool retrieval) {
   const long long grown = (long long)n_ctx + c.max_new_tokens;
   return retrieval ? grown : std::min(grown, (long long)c.n_sink + window);

@@ -1,4 +1,4 @@
-// Cache-building kernels: prefill-end compression (Algorithm 1 lines 2-3, Eq. 4), decode-token
+// Cache-building kernels: prefill-end compression (Algorithm 1, Eq. 4), decode-token
 // append with fold-on-evict, and the logical-order export used for snapshots and parity checks.
 #include "razor_common.cuh"
 

@@ -1,4 +1,4 @@
-// Decode attention over the compressed cache (Eq. 5; Algorithm 1 line 5): split-K flash decoding as a
+// Decode attention over the compressed cache (Eq. 5; Algorithm 1): split-K flash decoding as a
 // persistent producer / consumer kernel, one CTA per SM.
 //
 // One launch covers every (sequence, KV head) of a layer, full-length retrieval heads and short heads
@@ -143,7 +143,7 @@ struct RoundMask {
   int total;                    // tokens the head has seen (len + n_drop): query t sits at total - n_tok + t
   int n_sink, ring_head, window, n_drop;
   int slot0;                    // slot of the page's first token
-  // position of the token in slot s (Algorithm 1 line 3 keeps sinks + a ring of the recent tokens)
+  // position of the token in slot s (Algorithm 1 keeps sinks + a ring of the recent tokens)
   __device__ __forceinline__ int pos(int s) const {
     if (window < 0 || n_drop == 0 || s < n_sink) return s;
     int j = s - n_sink - ring_head;

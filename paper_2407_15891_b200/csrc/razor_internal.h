@@ -17,7 +17,7 @@ constexpr int kCompressMaxSlices = 64; // row slices per (sequence, KV head) in 
 
 // Device-resident state of one (layer, sequence, KV head).  window < 0 marks a head that keeps every
 // token (retrieval head).  Physical slots: [0, n_sink) sinks, then the recent window as a ring whose
-// oldest element sits at ring index ring_head (Algorithm 1 line 3 keeps sinks + recent tokens).
+// oldest element sits at ring index ring_head (Algorithm 1 keeps sinks + recent tokens).
 struct HeadState {
   int32_t len;        // tokens stored (physical slots in use)
   int32_t n_drop;     // N_d of Eq. 4: tokens folded into the compensation sums so far

@@ -1,5 +1,5 @@
 """CPU-side tests of the C-ABI library: it loads, exports every symbol include/razor.h declares,
-validates arguments, sizes its buffers as Algorithm 1 line 2-3 dictates, and plans balanced decode
+validates arguments, sizes its buffers as Algorithm 1 dictates, and plans balanced decode
 schedules.  No compute call is made here (there is no GPU on this machine)."""
 import ctypes as C
 import os

@@ -37,7 +37,7 @@ def brute_full_attention(q, K, V, scale):
     return np.array([sum(w[t] * float(V[t][i]) for t in range(n)) / z for i in range(len(V[0]))])
 
 
-# ------------------------------------------------------------------ kept set (Algorithm 1 lines 2-3)
+# ------------------------------------------------------------------ kept set (Algorithm 1)
 def test_kept_set_matches_per_position_rule_exhaustively():
     for n in range(0, 41):
         for n0 in range(0, 6):
