@@ -33,7 +33,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 inline int ceil_div(long long a, long long b) { return (int)((a + b - 1) / b); }
 
 struct Layout {
-  size_t state, comp_sum, comp_mean, page_table, items, jobs, multi, rec_ml, rec_o, queue, scratch, seq_desc, slopes, total;
+  size_t state, comp_sum, comp_mean, page_table, items, jobs, multi, rec_ml, rec_o, queue, scratch, plan, slopes, total;
   int max_pages, max_items;
 };
 
@@ -78,7 +78,7 @@ Layout make_layout(const razor_config_t& c) {
   (void)g;
   l.queue = take(8 * sizeof(int32_t));   // queue[0..3], then the status word
   l.scratch = take(nh * kCompressMaxSlices * 2 * D * sizeof(float));
-  l.seq_desc = take((size_t)c.batch * sizeof(SeqDesc));
+  l.plan = take(nh * sizeof(HeadPlan) + (size_t)c.batch * sizeof(SeqDesc));   // plan[], then seq_desc[]
   l.slopes = take(L * (size_t)c.n_q_heads * sizeof(float));
   l.total = off;
   return l;
@@ -106,6 +106,9 @@ struct LayerHost {
   int32_t* jobs = nullptr;          // pinned host, [max_items + 1]
   MultiHead* multi = nullptr;       // pinned host, [B*Hkv]
   cudaEvent_t upload_done = nullptr;
+  // compression plan staging: HeadPlan[B*Hkv] then SeqDesc[B], the image of the device's plan region
+  uint8_t* plan = nullptr;          // pinned host
+  cudaEvent_t plan_done = nullptr;
 };
 
 uint64_t mix64(uint64_t x) {
@@ -128,6 +131,8 @@ struct razor_cache {
   WorkItem* pinned_items = nullptr;   // [L][max_items]
   int32_t* pinned_jobs = nullptr;     // [L][max_items + 1]
   MultiHead* pinned_multi = nullptr;  // [L][B*Hkv]
+  uint8_t* pinned_plan = nullptr;     // [L][plan_bytes]
+  size_t plan_bytes = 0;
 };
 
 extern "C" {
@@ -210,7 +215,8 @@ int razor_cache_create(razor_cache_t** out, const razor_config_t* cfg, void* poo
   dv.queue = (int32_t*)(ws + lay.queue);
   dv.status = dv.queue + 4;
   dv.compress_scratch = (float*)(ws + lay.scratch);
-  dv.seq_desc = (SeqDesc*)(ws + lay.seq_desc);
+  dv.plan = (HeadPlan*)(ws + lay.plan);
+  dv.seq_desc = (SeqDesc*)(ws + lay.plan + (size_t)cfg->batch * cfg->n_kv_heads * sizeof(HeadPlan));
   dv.alibi_slopes = (float*)(ws + lay.slopes);
   dv.alibi = 0;
   dv.n_heads = cfg->batch * cfg->n_kv_heads;
@@ -234,11 +240,16 @@ int razor_cache_create(razor_cache_t** out, const razor_config_t* cfg, void* poo
   if (e == cudaSuccess)
     e = cudaHostAlloc((void**)&c->pinned_multi, (size_t)cfg->n_layers * dv.n_heads * sizeof(MultiHead),
                       cudaHostAllocDefault);
+  c->plan_bytes = (size_t)dv.n_heads * sizeof(HeadPlan) + (size_t)cfg->batch * sizeof(SeqDesc);
+  if (e == cudaSuccess)
+    e = cudaHostAlloc((void**)&c->pinned_plan, (size_t)cfg->n_layers * c->plan_bytes, cudaHostAllocDefault);
   if (e != cudaSuccess) {
     g_last_cuda_error = (int)e;
     (void)cudaGetLastError();
     if (c->pinned_items) cudaFreeHost(c->pinned_items);
     if (c->pinned_jobs) cudaFreeHost(c->pinned_jobs);
+    if (c->pinned_multi) cudaFreeHost(c->pinned_multi);
+  if (c->pinned_plan) cudaFreeHost(c->pinned_plan);
     delete c;
     return RAZOR_E_CUDA;
   }
@@ -253,6 +264,7 @@ int razor_cache_create(razor_cache_t** out, const razor_config_t* cfg, void* poo
     L.items = c->pinned_items + (size_t)l * lay.max_items;
     L.jobs = c->pinned_jobs + (size_t)l * (lay.max_items + 1);
     L.multi = c->pinned_multi + (size_t)l * dv.n_heads;
+    L.plan = c->pinned_plan + (size_t)l * c->plan_bytes;
   }
   *out = c;
   return RAZOR_OK;
@@ -275,11 +287,14 @@ int razor_cache_reset(razor_cache_t* c) {
 
 int razor_cache_destroy(razor_cache_t* c) {
   if (!c) return RAZOR_E_NULL_PTR;
-  for (LayerHost& L : c->layers)
+  for (LayerHost& L : c->layers) {
     if (L.upload_done) cudaEventDestroy(L.upload_done);
+    if (L.plan_done) cudaEventDestroy(L.plan_done);
+  }
   if (c->pinned_items) cudaFreeHost(c->pinned_items);
   if (c->pinned_jobs) cudaFreeHost(c->pinned_jobs);
   if (c->pinned_multi) cudaFreeHost(c->pinned_multi);
+  if (c->pinned_plan) cudaFreeHost(c->pinned_plan);
   delete c;
   return RAZOR_OK;
 }
@@ -354,63 +369,78 @@ int compress_impl(razor_cache* c, int layer, const std::vector<SeqIn>& seqs, con
   }
   c->next_page = next;
 
-  std::vector<int32_t> rows((size_t)H * c->lay.max_pages);
-  std::vector<HeadState> states(H);
-  std::vector<SeqDesc> descs(seqs.size());
+  // The plan goes to the device in one copy from pinned memory: per head its state after the call and the
+  // run of pool pages behind its page-table row (compress_plan_kernel writes both), then the sequences.
+  if (L.plan_done) RZ_CUDA(cudaEventSynchronize(L.plan_done));   // the previous plan has left the staging area
+  HeadPlan* plan = (HeadPlan*)L.plan;
+  SeqDesc* descs = (SeqDesc*)(L.plan + (size_t)c->dv.n_heads * sizeof(HeadPlan));
+  int n_plan = 0;
+  std::vector<int32_t> rows;   // only for permuted page ids
   for (size_t i = 0; i < seqs.size(); ++i) {
     const SeqIn& s = seqs[i];
     if (new_start[i] >= 0) {
       L.region_start[s.b] = new_start[i];
       L.region_count[s.b] = need[i];
     }
-    // page ids of the region, optionally permuted
-    std::vector<int32_t> ids((size_t)need[i]);
-    for (long long k = 0; k < need[i]; ++k) ids[(size_t)k] = (int32_t)(L.region_start[s.b] + k);
-    if (cfg.page_shuffle_seed) {
+    const bool shuffled = cfg.page_shuffle_seed != 0;
+    std::vector<int32_t> ids;
+    if (shuffled) {   // page ids of the region, permuted: the rows are written from the host
+      ids.resize((size_t)need[i]);
+      for (long long k = 0; k < need[i]; ++k) ids[(size_t)k] = (int32_t)(L.region_start[s.b] + k);
       uint64_t st = mix64((uint64_t)cfg.page_shuffle_seed * 1315423911ull + (uint64_t)layer * 2654435761ull + s.b);
       for (long long k = need[i] - 1; k > 0; --k) {
         st = mix64(st);
         std::swap(ids[(size_t)k], ids[(size_t)(st % (uint64_t)(k + 1))]);
       }
+      rows.assign((size_t)H * c->lay.max_pages, 0);
     }
-    std::fill(rows.begin(), rows.end(), 0);
-    size_t cursor = 0;
+    long long cursor = 0;
     for (int g = 0; g < H; ++g) {
       const bool r = flags[g] != 0;
       const int wg = eff_window(s.window, g);
       const int cap_pages = ceil_div(head_capacity_tokens(cfg, s.n_ctx, wg, r), kPageTokens);
-      for (int k = 0; k < cap_pages; ++k) rows[(size_t)g * c->lay.max_pages + k] = ids[cursor++];
       const bool keep_all = r || s.n_ctx <= cfg.n_sink + wg;
       HeadState h;
       h.len = keep_all ? s.n_ctx : cfg.n_sink + wg;
       h.n_drop = keep_all ? 0 : s.n_ctx - cfg.n_sink - wg;
       h.ring_head = 0;
       h.window = r ? -1 : wg;
-      states[g] = h;
       L.hs[(size_t)s.b * H + g] = h;
+      HeadPlan& pl = plan[n_plan++];
+      pl.head = s.b * H + g;
+      pl.first_page = (int32_t)(L.region_start[s.b] + cursor);
+      pl.n_pages = shuffled ? 0 : cap_pages;
+      pl.len = h.len;
+      pl.n_drop = h.n_drop;
+      pl.window = h.window;
+      if (shuffled)
+        for (int k = 0; k < cap_pages; ++k) rows[(size_t)g * c->lay.max_pages + k] = ids[(size_t)(cursor + k)];
+      cursor += cap_pages;
     }
-    const size_t head0 = (size_t)layer * c->dv.n_heads + (size_t)s.b * H;
-    RZ_CUDA(cudaMemcpyAsync(c->dv.page_table + head0 * c->lay.max_pages, rows.data(), rows.size() * sizeof(int32_t),
-                            cudaMemcpyHostToDevice, stream));
-    RZ_CUDA(cudaMemcpyAsync(c->dv.state + head0, states.data(), states.size() * sizeof(HeadState),
-                            cudaMemcpyHostToDevice, stream));
+    if (shuffled) {
+      const size_t head0 = (size_t)layer * c->dv.n_heads + (size_t)s.b * H;
+      RZ_CUDA(cudaMemcpyAsync(c->dv.page_table + head0 * c->lay.max_pages, rows.data(), rows.size() * sizeof(int32_t),
+                              cudaMemcpyHostToDevice, stream));   // pageable source: staged before the call returns
+    }
     SeqDesc d;
     d.K = s.K; d.V = s.V; d.stride_h = s.stride_h; d.stride_n = s.stride_n;
     d.n_ctx = s.n_ctx; d.window = s.window; d.b = s.b; d.pad = 0;
     descs[i] = d;
     if (!L.seq_done[s.b]) { L.seq_done[s.b] = 1; L.n_done += 1; }
   }
-  RZ_CUDA(cudaMemcpyAsync(c->dv.seq_desc, descs.data(), descs.size() * sizeof(SeqDesc), cudaMemcpyHostToDevice,
-                          stream));
+  // one copy covers plan[0 .. n_plan) and, behind the full plan array, the sequence descriptors
+  RZ_CUDA(cudaMemcpyAsync(c->dv.plan, L.plan, c->plan_bytes, cudaMemcpyHostToDevice, stream));
+  if (!L.plan_done) RZ_CUDA(cudaEventCreateWithFlags(&L.plan_done, cudaEventDisableTiming));
+  RZ_CUDA(cudaEventRecord(L.plan_done, stream));
   L.retr = flags;
   L.any = true;
   L.appended = 0;
   L.sched_valid = false;
 
   // Slices per head: enough CTAs to fill the machine, slices no shorter than 64 rows.
-  int slices = ceil_div((long long)c->n_sms * 8, (long long)seqs.size() * H);
+  int slices = ceil_div((long long)c->n_sms * 24, (long long)seqs.size() * H);
   slices = std::max(1, std::min({slices, kCompressMaxSlices, std::max(1, n_max / 64)}));
-  RZ_CUDA(launch_compress(c->dv, cfg.dtype, layer, (int)seqs.size(), slices, stream));
+  RZ_CUDA(launch_compress(c->dv, cfg.dtype, layer, (int)seqs.size(), slices, n_plan, stream));
   return RAZOR_OK;
 }
 

@@ -1,6 +1,7 @@
 // Cache-building kernels: prefill-end compression (Algorithm 1, Eq. 4), decode-token
 // append with fold-on-evict, and the logical-order export used for snapshots and parity checks.
 #include "razor_common.cuh"
+#include "razor_sync.cuh"
 
 namespace razor {
 
@@ -12,11 +13,35 @@ namespace razor {
 // (Eq. 4) is reproducible from run to run.
 // Slot of a kept position p (ascending position order): retrieval head or N <= N0 + W: slot = p;
 // otherwise sinks p < N0 keep slot p and recent tokens p >= N - W go to N0 + (p - (N - W)).
+//
+// The rows come in through the bulk-copy engine: a producer warp copies blocks of 16 rows (their K
+// rows, then their V rows: one copy each when the rows are contiguous in the source, one per row
+// otherwise) into a ring of shared-memory stages that complete on mbarriers, and kCompressWarps
+// consumer warps take the blocks round-robin, 16 bytes of a row per lane.  Block i always goes to warp
+// i % kCompressWarps and the ring length is a multiple of that, so the sums are added in the same
+// order every run.  All waits are bounded (status bits as in the decode kernel).
+constexpr int kCompressWarps = 4;
+constexpr int kCompressThreads = (kCompressWarps + 1) * 32;
+constexpr int kCompressRingBytes = 64 * 1024;
+
 template <typename T, int D>
-__global__ void __launch_bounds__(256) compress_kernel(DeviceView dv, int layer, int n_slices) {
+struct CompressSmem {
+  static constexpr int kBlockBytes = 2 * kPageTokens * RowGeom<T, D>::kRowBytes;   // 16 K rows + 16 V rows
+  static constexpr int kStages = kCompressRingBytes / kBlockBytes;
+  static_assert(kStages >= kCompressWarps && kStages % kCompressWarps == 0, "a stage belongs to one warp");
+  alignas(128) uint8_t ring[kStages][kBlockBytes];
+  float red[kCompressWarps][RowGeom<T, D>::kRg][2][D];   // [warp][row within a pass][K | V][D]
+  uint64_t full[kStages], empty[kStages];
+  int abort_flag;
+};
+
+template <typename T, int D>
+__global__ void __launch_bounds__(kCompressThreads) compress_kernel(DeviceView dv, int layer, int n_slices) {
   using Geo = RowGeom<T, D>;
-  constexpr int LPR = Geo::kLpr, EPL = Geo::kEpl, NGRP = 256 / LPR;
-  __shared__ float red[NGRP][2][D];
+  using Smem = CompressSmem<T, D>;
+  constexpr int LPR = Geo::kLpr, RG = Geo::kRg, EPL = Geo::kEpl, RB = Geo::kRowBytes, S = Smem::kStages;
+  extern __shared__ __align__(128) uint8_t compress_smem_raw[];
+  Smem& sm = *reinterpret_cast<Smem*>(compress_smem_raw);
 
   const SeqDesc sd = dv.seq_desc[blockIdx.z];
   const int g = blockIdx.y;
@@ -29,64 +54,136 @@ __global__ void __launch_bounds__(256) compress_kernel(DeviceView dv, int layer,
   const int rows_per_slice = (((N + n_slices - 1) / n_slices) + 15) & ~15;
   const int r0 = blockIdx.x * rows_per_slice;
   const int r1 = min(N, r0 + rows_per_slice);
-  const int lir = threadIdx.x % LPR, grp = threadIdx.x / LPR;
+  const int n_blocks = r1 > r0 ? (r1 - r0 + kPageTokens - 1) / kPageTokens : 0;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   const char* Kb = (const char*)sd.K + (size_t)g * sd.stride_h * sizeof(T);
   const char* Vb = (const char*)sd.V + (size_t)g * sd.stride_h * sizeof(T);
   const size_t row_stride = (size_t)sd.stride_n * sizeof(T);
-  const int32_t* pt = dv.page_table + ((size_t)layer * dv.n_heads + head) * dv.max_pages;
+  volatile int* abort_flag = &sm.abort_flag;
 
-  float accK[EPL], accV[EPL];
-#pragma unroll
-  for (int i = 0; i < EPL; ++i) accK[i] = accV[i] = 0.f;
-
-  constexpr int UNROLL = 4;
-  for (int p0 = r0 + grp; p0 < r1; p0 += NGRP * UNROLL) {
-    uint4 kf[UNROLL], vf[UNROLL];
-#pragma unroll
-    for (int u = 0; u < UNROLL; ++u) {
-      const int p = p0 + u * NGRP;
-      if (p < r1) {
-        kf[u] = ld_stream((const uint4*)(Kb + (size_t)p * row_stride) + lir);
-        vf[u] = ld_stream((const uint4*)(Vb + (size_t)p * row_stride) + lir);
-      }
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S; ++s) {
+      mbar_init(&sm.full[s], 1);
+      mbar_init(&sm.empty[s], 1);
     }
-#pragma unroll
-    for (int u = 0; u < UNROLL; ++u) {
-      const int p = p0 + u * NGRP;
-      if (p >= r1) continue;
-      int slot;
-      if (keep_all || p < n_sink) slot = p;
-      else if (p >= recent0) slot = n_sink + (p - recent0);
-      else slot = -1;
-      if (slot >= 0) {
-        const size_t page = (size_t)pt[slot >> 4];
-        uint4* dst = (uint4*)(dv.pool + page * dv.page_bytes + (size_t)(slot & 15) * Geo::kRowBytes) + swz(slot, lir);
-        dst[0] = kf[u];
-        dst[kPageTokens * LPR] = vf[u];   // V rows follow the 16 K rows of the page
-      } else {
-        float a[EPL], b[EPL];
-        Elem<T>::unpack(kf[u], a);
-        Elem<T>::unpack(vf[u], b);
-#pragma unroll
-        for (int i = 0; i < EPL; ++i) { accK[i] += a[i]; accV[i] += b[i]; }
-      }
-    }
+    sm.abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  __syncthreads();
 
+  if (warp == kCompressWarps) {
+    // ---- producer
+    if (lane == 0) {
+      const bool contiguous = row_stride == (size_t)RB;
+      int issued = 0;
+      for (int i = 0; i < n_blocks; ++i) {
+        const int s = i % S, use = i / S;
+        if (use > 0 && !mbar_wait(&sm.empty[s], (use - 1) & 1, abort_flag)) {
+          atomicOr(dv.status, kStatusProducerTimeout);
+          break;
+        }
+        const int p = r0 + i * kPageTokens, rows = min(kPageTokens, r1 - p);
+        mbar_arrive_expect_tx(&sm.full[s], (uint32_t)(2 * rows * RB));
+        uint8_t* dstK = sm.ring[s];
+        uint8_t* dstV = dstK + kPageTokens * RB;
+        if (contiguous) {
+          bulk_load(dstK, Kb + (size_t)p * row_stride, (uint32_t)(rows * RB), &sm.full[s]);
+          bulk_load(dstV, Vb + (size_t)p * row_stride, (uint32_t)(rows * RB), &sm.full[s]);
+        } else {
+          for (int t = 0; t < rows; ++t) {
+            bulk_load(dstK + t * RB, Kb + (size_t)(p + t) * row_stride, RB, &sm.full[s]);
+            bulk_load(dstV + t * RB, Vb + (size_t)(p + t) * row_stride, RB, &sm.full[s]);
+          }
+        }
+        issued = i + 1;
+      }
+      if (*abort_flag) {   // the copies in flight must land before the CTA may exit
+        for (int i = max(0, issued - S); i < issued; ++i)
+          if (!mbar_wait_drain(&sm.full[i % S], (i / S) & 1)) atomicOr(dv.status, kStatusDrainTimeout);
+      }
+    }
+  } else {
+    // ---- consumers: LPR lanes per row, so a warp takes RG rows of a block per pass
+    const int lir = lane % LPR, par = lane / LPR;
+    const int32_t* pt = dv.page_table + ((size_t)layer * dv.n_heads + head) * dv.max_pages;
+    float accK[EPL], accV[EPL];
 #pragma unroll
-  for (int i = 0; i < EPL; ++i) {
-    red[grp][0][lir * EPL + i] = accK[i];
-    red[grp][1][lir * EPL + i] = accV[i];
+    for (int i = 0; i < EPL; ++i) accK[i] = accV[i] = 0.f;
+    for (int i = warp; i < n_blocks; i += kCompressWarps) {
+      const int s = i % S, use = i / S;
+      if (!__all_sync(0xffffffffu, mbar_wait(&sm.full[s], use & 1, abort_flag))) {
+        if (lane == 0) atomicOr(dv.status, kStatusConsumerTimeout);
+        break;
+      }
+      const int p0 = r0 + i * kPageTokens;
+      const uint4* rowsK = (const uint4*)sm.ring[s];
+      const uint4* rowsV = rowsK + kPageTokens * LPR;
+      // The block goes to registers (eight passes at a time) and the stage back to the producer before
+      // the rows are looked at, so that a stage is held only for the time of a few shared-memory loads.
+      constexpr int PASSES = kPageTokens / RG, CH = PASSES < 8 ? PASSES : 8;
+#pragma unroll
+      for (int c = 0; c < PASSES / CH; ++c) {
+        uint4 kf[CH], vf[CH];
+#pragma unroll
+        for (int it = 0; it < CH; ++it) {
+          const int t = RG * (c * CH + it) + par;
+          kf[it] = rowsK[t * LPR + lir];
+          vf[it] = rowsV[t * LPR + lir];
+        }
+        if (c == PASSES / CH - 1) {
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&sm.empty[s]);
+        }
+#pragma unroll
+        for (int it = 0; it < CH; ++it) {
+          const int t = RG * (c * CH + it) + par, p = p0 + t;
+          if (p >= r1) continue;
+          int slot;
+          if (keep_all || p < n_sink) slot = p;
+          else if (p >= recent0) slot = n_sink + (p - recent0);
+          else slot = -1;
+          if (slot >= 0) {
+            const size_t page = (size_t)pt[slot >> 4];
+            uint4* dst = (uint4*)(dv.pool + page * dv.page_bytes + (size_t)(slot & 15) * RB) + swz(slot, lir);
+            dst[0] = kf[it];
+            dst[kPageTokens * LPR] = vf[it];   // V rows follow the 16 K rows of the page
+          } else {
+            float a[EPL], b[EPL];
+            Elem<T>::unpack(kf[it], a);
+            Elem<T>::unpack(vf[it], b);
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) { accK[e] += a[e]; accV[e] += b[e]; }
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) {
+      sm.red[warp][par][0][lir * EPL + e] = accK[e];
+      sm.red[warp][par][1][lir * EPL + e] = accV[e];
+    }
   }
   __syncthreads();
   float* scratch = dv.compress_scratch + ((size_t)head * kCompressMaxSlices + blockIdx.x) * 2 * D;
-  for (int e = threadIdx.x; e < 2 * D; e += 256) {
-    float s = 0.f;
+  for (int e = threadIdx.x; e < 2 * D; e += kCompressThreads) {
+    float sum = 0.f;
 #pragma unroll
-    for (int r = 0; r < NGRP; ++r) s += (&red[r][0][0])[e];
-    scratch[e] = s;
+    for (int w = 0; w < kCompressWarps; ++w)
+#pragma unroll
+      for (int r = 0; r < RG; ++r) sum += sm.red[w][r][e / D][e % D];
+    scratch[e] = sum;
   }
+}
+
+// grid = planned heads, block = 256: the head's state and its page-table row (consecutive pool pages), so
+// that a compression call sends a few bytes per head to the device instead of whole page-table rows.
+__global__ void __launch_bounds__(256) compress_plan_kernel(DeviceView dv, int layer) {
+  const HeadPlan pl = dv.plan[blockIdx.x];
+  const size_t hs = (size_t)layer * dv.n_heads + pl.head;
+  int32_t* row = dv.page_table + hs * dv.max_pages;
+  for (int k = threadIdx.x; k < pl.n_pages; k += 256) row[k] = pl.first_page + k;
+  if (threadIdx.x == 0) dv.state[hs] = HeadState{pl.len, pl.n_drop, 0, pl.window};
 }
 
 // grid = (Hkv, sequences), block = 2*D threads: fixed-order sum of the slice partials, then the
@@ -307,22 +404,31 @@ static cudaError_t launch_dependent(void (*kernel)(KArgs...), int grid, int bloc
 }
 
 template <typename T, int D>
-static cudaError_t compress_t(const DeviceView& dv, int layer, int n_seqs, int n_slices, cudaStream_t s) {
+static cudaError_t compress_t(const DeviceView& dv, int layer, int n_seqs, int n_slices, int n_plan, cudaStream_t s) {
   dim3 grid(n_slices, dv.n_kv_heads, n_seqs);
-  compress_kernel<T, D><<<grid, 256, 0, s>>>(dv, layer, n_slices);
-  cudaError_t e = cudaGetLastError();
+  const size_t smem = sizeof(CompressSmem<T, D>);
+  cudaError_t e = cudaFuncSetAttribute(compress_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  if (n_plan > 0) {
+    compress_plan_kernel<<<n_plan, 256, 0, s>>>(dv, layer);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+  }
+  compress_kernel<T, D><<<grid, kCompressThreads, smem, s>>>(dv, layer, n_slices);
+  e = cudaGetLastError();
   if (e != cudaSuccess) return e;
   compress_finalize_kernel<D><<<dim3(dv.n_kv_heads, n_seqs), 2 * D, 0, s>>>(dv, layer, n_slices);
   return cudaGetLastError();
 }
 
-cudaError_t launch_compress(const DeviceView& dv, int dtype, int layer, int n_seqs, int n_slices, cudaStream_t s) {
+cudaError_t launch_compress(const DeviceView& dv, int dtype, int layer, int n_seqs, int n_slices, int n_plan,
+                            cudaStream_t s) {
   if (dtype == RAZOR_BF16) {
-    return dv.head_dim == 128 ? compress_t<__nv_bfloat16, 128>(dv, layer, n_seqs, n_slices, s)
-                              : compress_t<__nv_bfloat16, 64>(dv, layer, n_seqs, n_slices, s);
+    return dv.head_dim == 128 ? compress_t<__nv_bfloat16, 128>(dv, layer, n_seqs, n_slices, n_plan, s)
+                              : compress_t<__nv_bfloat16, 64>(dv, layer, n_seqs, n_slices, n_plan, s);
   }
-  return dv.head_dim == 128 ? compress_t<float, 128>(dv, layer, n_seqs, n_slices, s)
-                            : compress_t<float, 64>(dv, layer, n_seqs, n_slices, s);
+  return dv.head_dim == 128 ? compress_t<float, 128>(dv, layer, n_seqs, n_slices, n_plan, s)
+                            : compress_t<float, 64>(dv, layer, n_seqs, n_slices, n_plan, s);
 }
 
 template <typename T, int D>

@@ -40,15 +40,6 @@ constexpr int kMaxMergeBufs = 2;         // consumer -> reducer hand-over buffer
 template <int G>
 constexpr int merge_bufs() { return G >= 4 ? 1 : 2; }
 constexpr int kMaxStages = 64;           // ring stages (pages in flight per CTA)
-// Bulk asynchronous copy global -> shared; completion is counted in bytes on `bar`.
-// dst, src 16-byte aligned, bytes a multiple of 16.
-__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                   smem_u32(dst)),
-               "l"(src), "r"(bytes), "r"(smem_u32(bar))
-               : "memory");
-}
-
 // Ring position -> (stage, use).  Position p is always consumed by warp p % NC, and a stage must always
 // be consumed by the same warp: a warp then never waits on a barrier that is more than one phase behind
 // it, which a parity wait could not tell from "done".  So the ring is NC interleaved sub-rings: warp w

@@ -59,6 +59,16 @@ struct SeqDesc {
   int32_t pad;
 };
 
+// One (sequence, KV head) of a compression call, as planned on the host: the head's state after the
+// call and the run of consecutive pool pages that backs its page-table row.  n_pages = 0 leaves the row
+// alone (the host has written it itself, e.g. in a permuted order).
+struct HeadPlan {
+  int32_t head;        // b * Hkv + kv_head
+  int32_t first_page;
+  int32_t n_pages;
+  int32_t len, n_drop, window;   // HeadState after compression (ring_head = 0)
+};
+
 // Bits of the device status word (razor_cache_device_status).
 enum : int32_t {
   kStatusProducerTimeout = 1,   // the copy-issuing warp gave up waiting for a free ring stage or item slot
@@ -83,7 +93,8 @@ struct DeviceView {
   int32_t* queue;           // [4]: next item, CTAs done, spare, spare (zero at rest)
   int32_t* status;          // [1]: kStatus* bits, sticky until razor_cache_device_status clears them
   float* compress_scratch;  // [B*Hkv][kCompressMaxSlices][2][D]
-  SeqDesc* seq_desc;        // [B]
+  HeadPlan* plan;           // [B*Hkv]  heads of the compression call in flight
+  SeqDesc* seq_desc;        // [B]      directly behind plan[]: both arrive in one copy
   float* alibi_slopes;      // [L][Hq]  ALiBi slopes l_h times log2(e); read only when alibi != 0
   int32_t alibi;            // 1: logits get - l_h (m - n) (Eq. 1), from razor_cache_set_alibi
   int32_t n_heads;          // B*Hkv
@@ -109,7 +120,8 @@ struct DecodeTuning {
 };
 
 // Kernel launchers (defined in the .cu files).  Each returns the cudaError_t of the launch.
-cudaError_t launch_compress(const DeviceView& dv, int dtype, int layer, int n_seqs, int n_slices,
+// n_plan: entries of dv.plan to apply (state and page-table rows) before the rows are streamed.
+cudaError_t launch_compress(const DeviceView& dv, int dtype, int layer, int n_seqs, int n_slices, int n_plan,
                             cudaStream_t stream);
 cudaError_t launch_append(const DeviceView& dv, int dtype, int layer, const void* k_new, const void* v_new,
                           cudaStream_t stream);
