@@ -386,10 +386,10 @@ def main():
             if per_seq:
                 for b in range(w.batch):
                     cache.compress_seq(l, b, dense[b][0], dense[b][1], w.ctx_len[b], retr[l], w.window[b])
-                    launches["n"] += 2
+                    launches["n"] += 3    # plan, streaming compression kernel, finalize
             else:
                 cache.compress(l, Kd, Vd, w.ctx_len, retr[l], w.window)
-                launches["n"] += 2
+                launches["n"] += 3
 
     def one_pass(ev=None):
         compress_all()
