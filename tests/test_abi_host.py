@@ -195,3 +195,17 @@ def test_schedule_gives_long_heads_few_parts():
         rz.razor_schedule_plan([100], 148, 85, 4, 0)
     with pytest.raises(rz.RazorError):
         rz.razor_schedule_plan([100], 148, 101, 4, 1)
+
+
+def test_header_is_plain_c():
+    """The public header must compile as C99 on its own: no C++ constructs, no CUDA or torch types."""
+    import shutil
+    import subprocess
+    gcc = shutil.which("gcc")
+    if gcc is None:
+        pytest.skip("no C compiler")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    src = '#include "razor.h"\nint main(void) { razor_config_t c; (void)c; return razor_version() == 0; }\n'
+    r = subprocess.run([gcc, "-std=c99", "-Wall", "-Werror", "-pedantic", "-fsyntax-only", "-I", os.path.join(root, "include"),
+                        "-x", "c", "-"], input=src, text=True, capture_output=True)
+    assert r.returncode == 0, r.stderr
