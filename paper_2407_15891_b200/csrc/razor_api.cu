@@ -77,7 +77,7 @@ Layout make_layout(const razor_config_t& c) {
   l.rec_o = take((size_t)l.max_items * kMaxGroup * D * sizeof(float));
   (void)g;
   l.queue = take(8 * sizeof(int32_t));   // queue[0..3], then the status word
-  l.scratch = take(nh * kCompressMaxSlices * 2 * D * sizeof(float));
+  l.scratch = take(((size_t)kCompressSliceBudget + nh) * 2 * D * sizeof(float));
   l.plan = take(nh * sizeof(HeadPlan) + (size_t)c.batch * sizeof(SeqDesc));   // plan[], then seq_desc[]
   l.slopes = take(L * (size_t)c.n_q_heads * sizeof(float));
   l.total = off;
@@ -437,10 +437,13 @@ int compress_impl(razor_cache* c, int layer, const std::vector<SeqIn>& seqs, con
   L.appended = 0;
   L.sched_valid = false;
 
-  // Slices per head: enough CTAs to fill the machine, slices no shorter than 64 rows.
-  int slices = ceil_div((long long)c->n_sms * 24, (long long)seqs.size() * H);
-  slices = std::max(1, std::min({slices, kCompressMaxSlices, std::max(1, n_max / 64)}));
-  RZ_CUDA(launch_compress(c->dv, cfg.dtype, layer, (int)seqs.size(), slices, n_plan, stream));
+  // Slices per head: about 24 CTAs per SM in all (eight rounds of the three a SM holds), slices no shorter
+  // than 64 rows, and no more slice sums than the scratch has room for.
+  const long long heads_in_call = (long long)seqs.size() * H;
+  const long long room = ((long long)kCompressSliceBudget + c->dv.n_heads) / heads_in_call;
+  long long slices = ceil_div((long long)c->n_sms * 24, heads_in_call);
+  slices = std::max(1LL, std::min({slices, (long long)kCompressMaxSlices, room, (long long)std::max(1, n_max / 64)}));
+  RZ_CUDA(launch_compress(c->dv, cfg.dtype, layer, (int)seqs.size(), (int)slices, n_plan, stream));
   return RAZOR_OK;
 }
 

@@ -165,7 +165,8 @@ __global__ void __launch_bounds__(kCompressThreads) compress_kernel(DeviceView d
     }
   }
   __syncthreads();
-  float* scratch = dv.compress_scratch + ((size_t)head * kCompressMaxSlices + blockIdx.x) * 2 * D;
+  float* scratch =
+      dv.compress_scratch + (((size_t)blockIdx.z * dv.n_kv_heads + g) * n_slices + blockIdx.x) * 2 * D;
   for (int e = threadIdx.x; e < 2 * D; e += kCompressThreads) {
     float sum = 0.f;
 #pragma unroll
@@ -194,7 +195,7 @@ __global__ void compress_finalize_kernel(DeviceView dv, int layer, int n_slices)
   const int head = sd.b * dv.n_kv_heads + blockIdx.x;
   const size_t hs = (size_t)layer * dv.n_heads + head;
   const int n_drop = dv.state[hs].n_drop;
-  const float* scratch = dv.compress_scratch + (size_t)head * kCompressMaxSlices * 2 * D;
+  const float* scratch = dv.compress_scratch + ((size_t)blockIdx.y * dv.n_kv_heads + blockIdx.x) * n_slices * 2 * D;
   const int e = threadIdx.x;
   float s = 0.f;
   for (int i = 0; i < n_slices; ++i) s += scratch[(size_t)i * 2 * D + e];

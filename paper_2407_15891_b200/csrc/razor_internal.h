@@ -13,7 +13,8 @@ namespace razor {
 
 constexpr int kPageTokens = 16;        // tokens per page
 constexpr int kMaxGroup = 8;           // query heads per KV head
-constexpr int kCompressMaxSlices = 64; // row slices per (sequence, KV head) in the compression kernel
+constexpr int kCompressMaxSlices = 512;    // row slices per (sequence, KV head) in the compression kernel
+constexpr int kCompressSliceBudget = 8192; // slice sums a call may produce beyond one per head (sizes the scratch)
 
 // Device-resident state of one (layer, sequence, KV head).  window < 0 marks a head that keeps every
 // token (retrieval head).  Physical slots: [0, n_sink) sinks, then the recent window as a ring whose
@@ -92,7 +93,7 @@ struct DeviceView {
   float* rec_o;             // [max_items][G][D]   un-normalised numerator of a partial
   int32_t* queue;           // [4]: next item, CTAs done, spare, spare (zero at rest)
   int32_t* status;          // [1]: kStatus* bits, sticky until razor_cache_device_status clears them
-  float* compress_scratch;  // [B*Hkv][kCompressMaxSlices][2][D]
+  float* compress_scratch;  // [kCompressSliceBudget + B*Hkv][2][D]: slice s of head h of a call at h_in_call * n_slices + s
   HeadPlan* plan;           // [B*Hkv]  heads of the compression call in flight
   SeqDesc* seq_desc;        // [B]      directly behind plan[]: both arrive in one copy
   float* alibi_slopes;      // [L][Hq]  ALiBi slopes l_h times log2(e); read only when alibi != 0
