@@ -43,7 +43,7 @@ def _heads(n_heads, n, period, D, seed, dev):
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("D,n,period,heads", [(128, 384, 96, 5), (64, 300, 70, 4), (128, 1000, 333, 3), (64, 130, 64, 2), (64, 1500, 400, 2)])
+@pytest.mark.parametrize("D,n,period,heads", [(128, 384, 96, 5), (64, 300, 70, 4), (128, 1000, 333, 3), (64, 130, 64, 2), (64, 1500, 400, 2), (128, 100, 30, 2), (64, 40, 7, 3)])
 def test_scores_match_the_oracle_on_small_inputs(D, n, period, heads):
     Q, K = _heads(heads, n, period, D, 4000 + D + n, DEV)
     echo, ind = rz.razor_head_scores(Q, K, period)
