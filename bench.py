@@ -285,6 +285,52 @@ def decode_only(rz, synth, name, n_layers, dev, peak, reps=60, n_tok=1, alibi=Fa
             "query_tokens_per_call": n_tok, "alibi": bool(alibi)}
 
 
+def chunked_prefill_leg(rz, synth, dev, peak, chunk=8192, reps=3):
+    """One cfg3-shaped layer (batch 4, 40 heads, 65536 tokens) built chunk by chunk from an empty layer with
+    razor_append_many, as a chunked prefill hands its K/V over: no dense cache of the whole context exists.
+    Bytes: every chunk row is read once; a row that stays is written once; an evicted row is read once more."""
+    import numpy as np
+    import torch
+    w = synth.workload("cfg3")
+    N = max(w.ctx_len)
+    retr = w.retrieval(0)
+    cfg = rz.make_config(w.batch, 1, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, w.n_sink, 0, N)
+    cache = rz.RazorCache(cfg, [0] * w.batch, w.window, np.stack([retr]), device=dev)
+    shp = (w.batch, chunk, w.n_kv_heads, w.head_dim)
+    k = synth.normal_bf16(w.seed, synth.TAG_KNEW, shp, dev, sub=5)
+    v = synth.normal_bf16(w.seed, synth.TAG_VNEW, shp, dev, sub=6)
+    n_chunks = N // chunk
+
+    def build():
+        cache.start_empty(0, retr, w.window)
+        for _ in range(n_chunks):
+            cache.append_many(0, k, v)
+
+    build()
+    torch.cuda.synchronize()
+    a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(reps):
+        build()
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / reps
+    row = w.head_dim * 2 * 2                                    # K and V row, bf16
+    n_retr = int(np.sum(retr))
+    read = w.batch * w.n_kv_heads * N * row
+    kept_short = w.n_sink + w.window[0]
+    # with chunk <= window every row is stored once, and every row that ends up dropped is read back once
+    written = w.batch * row * w.n_kv_heads * N
+    evicted = w.batch * row * (w.n_kv_heads - n_retr) * max(0, N - kept_short)
+    status = cache.device_status()
+    cache.close()
+    total = read + written + evicted
+    return {"workload": f"cfg3 layer: {n_chunks} chunks of {chunk} tokens, batch {w.batch}, {w.n_kv_heads} heads",
+            "ms_per_layer": ms, "us_per_chunk": ms * 1e3 / n_chunks, "gbs": total / (ms * 1e-3) / 1e9,
+            "frac_of_measured": total / (ms * 1e-3) / 1e9 / peak, "read_gb": (read + evicted) / 1e9,
+            "write_gb": written / 1e9, "device_status": status}
+
+
 def head_scores_leg(rz, synth, dev, reps=5, heads=32):
     """Section 3.3's score reduction on its own input shape: 2500 random tokens repeated 4 times, 32 heads of
     dimension 128 (one layer of a 7B-class model).  A dense contraction (causal Q.K^T), so it is reported

@@ -342,6 +342,12 @@ class RazorCache:
         razor_compress(self.handle, layer, K, V, K.stride(0), K.stride(1), K.stride(2), ctx_len, head_is_retrieval,
                        self.cfg.n_sink, window)
 
+    def start_empty(self, layer: int, head_is_retrieval, window) -> None:
+        """A layer with no tokens yet, its retrieval set and windows fixed: the start of a chunked prefill, whose
+        chunks then arrive through append_many."""
+        razor_compress(self.handle, layer, None, None, 0, 0, 0, [0] * self.cfg.batch, head_is_retrieval,
+                       self.cfg.n_sink, window)
+
     def compress_seq(self, layer: int, b: int, K: torch.Tensor, V: torch.Tensor, ctx_len: int, head_is_retrieval,
                      window: int) -> None:
         """K, V: [Hkv, N, D] device tensors of one sequence."""

@@ -303,6 +303,8 @@ int razor_cache_destroy(razor_cache_t* c) {
 
 namespace {
 
+constexpr int kAppendChunkMin = 64;   // razor_append_many: runs this long are appended in parallel over the tokens
+
 struct SeqIn {
   int b;
   const void* K;
@@ -575,19 +577,26 @@ int razor_append_many(razor_cache_t* c, int32_t layer, const void* k_new, const 
   if (((uintptr_t)k_new | (uintptr_t)v_new) & 15) return RAZOR_E_MISALIGNED;
   LayerHost& L = c->layers[layer];
   if ((long long)L.appended + n_tokens > c->cfg.max_new_tokens) return RAZOR_E_CAPACITY;
-  RZ_CUDA(launch_append_many(c->dv, c->cfg.dtype, layer, k_new, v_new, n_tokens, (cudaStream_t)stream));
+  // Long runs go to the kernel that is parallel over the tokens: about eight CTAs per SM in all, slices of
+  // at least 32 tokens, no more slice sums than the scratch holds.
+  int slices = 0;
+  if (n_tokens >= kAppendChunkMin) {
+    const long long nh = c->dv.n_heads;
+    const long long room = ((long long)kCompressSliceBudget + nh) / nh;
+    slices = (int)std::max(1LL, std::min({(long long)ceil_div((long long)c->n_sms * 8, nh), room,
+                                           (long long)(n_tokens / 32)}));
+  }
+  RZ_CUDA(launch_append_many(c->dv, c->cfg.dtype, layer, k_new, v_new, n_tokens, slices, (cudaStream_t)stream));
   const int n_sink = c->cfg.n_sink;
-  for (int t = 0; t < n_tokens; ++t)   // host mirror of the kernel's state update
-    for (HeadState& h : L.hs) {
-      if (h.window < 0 || h.len < n_sink + h.window) {
-        h.len += 1;
-      } else if (h.window == 0) {
-        h.n_drop += 1;
-      } else {
-        h.n_drop += 1;
-        h.ring_head = (h.ring_head + 1 == h.window) ? 0 : h.ring_head + 1;
-      }
-    }
+  for (HeadState& h : L.hs) {   // host mirror of the kernels' state update, in closed form
+    const bool keeps_all = h.window < 0;
+    const int cap = keeps_all ? 0 : n_sink + h.window;
+    const int f = keeps_all ? n_tokens : std::min(n_tokens, std::max(0, cap - h.len));
+    const int E = n_tokens - f;
+    h.len += f;
+    h.n_drop += E;
+    h.ring_head = h.window > 0 ? (int)(((long long)h.ring_head + E) % h.window) : 0;
+  }
   L.appended += n_tokens;
   L.growth_tokens += n_tokens;
   return RAZOR_OK;

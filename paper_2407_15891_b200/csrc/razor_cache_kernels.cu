@@ -348,6 +348,122 @@ __global__ void __launch_bounds__(128) append_many_kernel(DeviceView dv, int lay
 }
 
 // ---------------------------------------------------------------------------------------------
+// Append of a long run of tokens (a prompt chunk of a chunked prefill, a long second prompt), in
+// parallel over the tokens.  The state afterwards is what n_tok single appends would leave; what n_tok
+// single appends do one after the other is decided here per token in closed form.  With len0, ring_head0
+// the state before the call, cap = N0 + W, f = tokens that still fit (all of them for a head that keeps
+// everything) and E = n_tok - f tokens that each evict the oldest recent token:
+//   * token a < f goes to slot len0 + a; it is overwritten again within the call when its ring index
+//     r = len0 + a - N0 is below E (the ring starts at index 0 while it fills);
+//   * evicting token j = a - f goes to ring index (ring_head0 + j) mod W and stays iff j >= E - W;
+//   * a token that does not stay is added to the compensation sums straight from the input; a token that
+//     stays in a ring slot that held a token from before the call adds that old row to the sums first.
+// Every slot is written by exactly one thread group, after it has read the old row, so there is no order
+// between CTAs to keep.  grid = (slices, heads); per-slice sums go to the compression scratch and
+// append_chunk_finalize_kernel adds them to the running sums (Eq. 4 over everything dropped so far).
+template <typename T, int D>
+__global__ void __launch_bounds__(256) append_chunk_kernel(DeviceView dv, int layer, const T* __restrict__ k_new,
+                                                           const T* __restrict__ v_new, int n_tok, int n_slices) {
+  using Geo = RowGeom<T, D>;
+  constexpr int LPR = Geo::kLpr, EPL = Geo::kEpl, NGRP = 256 / LPR;
+  __shared__ float red[NGRP][2][D];
+  const int head = blockIdx.y;
+  const size_t hs = (size_t)layer * dv.n_heads + head;
+  const HeadState st = dv.state[hs];
+  const int n_sink = dv.n_sink, W = st.window;
+  const bool keeps_all = W < 0;
+  const int cap = keeps_all ? 0 : n_sink + W;
+  const int f = keeps_all ? n_tok : min(n_tok, max(0, cap - st.len));
+  const int E = n_tok - f;
+  const int ring0 = max(0, st.len - n_sink);   // ring tokens from before the call
+  const int b = head / dv.n_kv_heads, g = head % dv.n_kv_heads;
+  const int32_t* pt = dv.page_table + hs * dv.max_pages;
+  const int per = (n_tok + n_slices - 1) / n_slices;
+  const int a0 = min(n_tok, (int)blockIdx.x * per), a1 = min(n_tok, a0 + per);
+  const int lir = threadIdx.x % LPR, grp = threadIdx.x / LPR;
+
+  float accK[EPL], accV[EPL];
+#pragma unroll
+  for (int i = 0; i < EPL; ++i) accK[i] = accV[i] = 0.f;
+  for (int a = a0 + grp; a < a1; a += NGRP) {
+    const size_t row = (((size_t)b * n_tok + a) * dv.n_kv_heads + g) * D;
+    const uint4 kf = ld_stream((const uint4*)(k_new + row) + lir);
+    const uint4 vf = ld_stream((const uint4*)(v_new + row) + lir);
+    int slot;
+    bool stays, had_old = false;
+    if (a < f) {
+      slot = st.len + a;
+      stays = keeps_all || slot < n_sink || slot - n_sink >= E;
+    } else {
+      const int j = a - f;
+      stays = j >= E - W;   // never when W == 0
+      const int r = stays ? (int)(((long long)st.ring_head + j) % W) : 0;
+      slot = n_sink + r;
+      had_old = stays && r < ring0;
+    }
+    float a_k[EPL], a_v[EPL];
+    if (stays) {
+      const size_t page = (size_t)pt[slot >> 4];
+      uint4* dst = (uint4*)(dv.pool + page * dv.page_bytes + (size_t)(slot & 15) * Geo::kRowBytes) + swz(slot, lir);
+      if (had_old) {
+        Elem<T>::unpack(dst[0], a_k);
+        Elem<T>::unpack(dst[kPageTokens * LPR], a_v);
+#pragma unroll
+        for (int i = 0; i < EPL; ++i) { accK[i] += a_k[i]; accV[i] += a_v[i]; }
+      }
+      dst[0] = kf;
+      dst[kPageTokens * LPR] = vf;
+    } else {
+      Elem<T>::unpack(kf, a_k);
+      Elem<T>::unpack(vf, a_v);
+#pragma unroll
+      for (int i = 0; i < EPL; ++i) { accK[i] += a_k[i]; accV[i] += a_v[i]; }
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < EPL; ++i) {
+    red[grp][0][lir * EPL + i] = accK[i];
+    red[grp][1][lir * EPL + i] = accV[i];
+  }
+  __syncthreads();
+  float* scratch = dv.compress_scratch + ((size_t)head * n_slices + blockIdx.x) * 2 * D;
+  for (int e = threadIdx.x; e < 2 * D; e += 256) {
+    float sum = 0.f;
+#pragma unroll
+    for (int r = 0; r < NGRP; ++r) sum += (&red[r][0][0])[e];
+    scratch[e] = sum;
+  }
+}
+
+// grid = heads, block = 2*D: slice sums added in a fixed order onto the running sums, means recomputed,
+// state advanced by n_tok appends.
+template <int D>
+__global__ void append_chunk_finalize_kernel(DeviceView dv, int layer, int n_tok, int n_slices) {
+  const int head = blockIdx.x, e = threadIdx.x;
+  const size_t hs = (size_t)layer * dv.n_heads + head;
+  const HeadState st = dv.state[hs];
+  const bool keeps_all = st.window < 0;
+  const int cap = keeps_all ? 0 : dv.n_sink + st.window;
+  const int f = keeps_all ? n_tok : min(n_tok, max(0, cap - st.len));
+  const int E = n_tok - f;
+  if (E > 0) {
+    const float* scratch = dv.compress_scratch + (size_t)head * n_slices * 2 * D;
+    float s = dv.comp_sum[hs * 2 * D + e];
+    for (int i = 0; i < n_slices; ++i) s += scratch[(size_t)i * 2 * D + e];
+    dv.comp_sum[hs * 2 * D + e] = s;
+    dv.comp_mean[hs * 2 * D + e] = __fdiv_rn(s, (float)(st.n_drop + E));
+  }
+  __syncthreads();   // every thread has read the old state
+  if (e == 0) {
+    HeadState nx = st;
+    nx.len = st.len + f;
+    nx.n_drop = st.n_drop + E;
+    nx.ring_head = st.window > 0 ? (int)(((long long)st.ring_head + E) % st.window) : 0;
+    dv.state[hs] = nx;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
 // Export in logical order (ascending original position).  With T = len + n_drop tokens seen so far:
 // logical index i < N0 (or any i while nothing has been dropped) is position i in slot i; otherwise
 // j = i - N0 is the j-th oldest recent token: slot N0 + (ring_head + j) mod W, position T - W + j.
@@ -448,20 +564,29 @@ cudaError_t launch_append(const DeviceView& dv, int dtype, int layer, const void
 }
 
 template <typename T, int D>
-static cudaError_t append_many_t(const DeviceView& dv, int layer, const void* k, const void* v, int n_tok, cudaStream_t s) {
+static cudaError_t append_many_t(const DeviceView& dv, int layer, const void* k, const void* v, int n_tok, int n_slices,
+                                 cudaStream_t s) {
+  if (n_slices > 0) {   // a long run: parallel over the tokens
+    append_chunk_kernel<T, D><<<dim3(n_slices, dv.n_heads), 256, 0, s>>>(dv, layer, (const T*)k, (const T*)v, n_tok,
+                                                                         n_slices);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    append_chunk_finalize_kernel<D><<<dv.n_heads, 2 * D, 0, s>>>(dv, layer, n_tok, n_slices);
+    return cudaGetLastError();
+  }
   const int warps = 4;
   return launch_dependent(append_many_kernel<T, D>, (dv.n_heads + warps - 1) / warps, warps * 32, s, dv, layer,
                           (const T*)k, (const T*)v, n_tok);
 }
 
 cudaError_t launch_append_many(const DeviceView& dv, int dtype, int layer, const void* k, const void* v, int n_tok,
-                               cudaStream_t s) {
+                               int n_slices, cudaStream_t s) {
   if (dtype == RAZOR_BF16) {
-    return dv.head_dim == 128 ? append_many_t<__nv_bfloat16, 128>(dv, layer, k, v, n_tok, s)
-                              : append_many_t<__nv_bfloat16, 64>(dv, layer, k, v, n_tok, s);
+    return dv.head_dim == 128 ? append_many_t<__nv_bfloat16, 128>(dv, layer, k, v, n_tok, n_slices, s)
+                              : append_many_t<__nv_bfloat16, 64>(dv, layer, k, v, n_tok, n_slices, s);
   }
-  return dv.head_dim == 128 ? append_many_t<float, 128>(dv, layer, k, v, n_tok, s)
-                            : append_many_t<float, 64>(dv, layer, k, v, n_tok, s);
+  return dv.head_dim == 128 ? append_many_t<float, 128>(dv, layer, k, v, n_tok, n_slices, s)
+                            : append_many_t<float, 64>(dv, layer, k, v, n_tok, n_slices, s);
 }
 
 template <typename T, int D>

@@ -126,8 +126,10 @@ cudaError_t launch_compress(const DeviceView& dv, int dtype, int layer, int n_se
                             cudaStream_t stream);
 cudaError_t launch_append(const DeviceView& dv, int dtype, int layer, const void* k_new, const void* v_new,
                           cudaStream_t stream);
+// n_slices > 0: the run is long, use the kernel that is parallel over the tokens with that many slices per
+// head (n_heads * n_slices slice sums must fit the compression scratch); 0: one warp per head, token by token.
 cudaError_t launch_append_many(const DeviceView& dv, int dtype, int layer, const void* k_new, const void* v_new,
-                               int n_tok, cudaStream_t stream);
+                               int n_tok, int n_slices, cudaStream_t stream);
 // What a decode launch pulls from the queue: n_jobs jobs, the first n_spans of them spans (item
 // ranges jobs[j]..jobs[j+1]), the others single items starting at tail_first.
 struct DecodeJobs {
