@@ -525,6 +525,20 @@ def main():
                      "read_gb": compress_read / 1e9, "write_gb": compress_write / 1e9},
     }
 
+    # ------------------------------------------------------------------ append alone: latency-bound, reported in us
+    compress_all()
+    sync_all()
+    a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+    a.record()
+    for t in range(T):
+        k_new, v_new = kvs[t % n_q]
+        for l in range(L):
+            cache.append(l, k_new, v_new)
+    b.record()
+    sync_all()
+    line["append"] = {"us_per_layer": a.elapsed_time(b) * 1e3 / (T * L), "launches_timed": T * L,
+                      "note": "razor_append calls back to back, one token per (sequence, KV head)"}
+
     # ------------------------------------------------------------------ dense full-cache decode, same GPU
     if not args.no_dense and rank == 0 and not per_seq:
         try:

@@ -95,6 +95,23 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
+// 2^t for t <= 0 on the FMA and integer pipes, relative error below 5e-5: t = n + f with n the nearest
+// integer (read off the low mantissa bits of t + 1.5 * 2^23) and |f| <= 1/2, 2^f as a degree-4 polynomial,
+// n added onto the exponent field.  The transcendental unit is the busiest pipe of this kernel (one ex2 per
+// score), so every kPolyEvery-th exponential takes this route instead.
+constexpr int kPolyEvery = 4;
+__device__ __forceinline__ float exp2_fma(float t) {
+  t = fmaxf(t, -125.f);                       // keeps the result a normal number; 2^-125 stands for zero
+  const float r = t + 12582912.f;
+  const float f = t - (r - 12582912.f);
+  float p = 0.0096181291f;
+  p = fmaf(p, f, 0.0555041087f);
+  p = fmaf(p, f, 0.2402265070f);
+  p = fmaf(p, f, 0.6931471806f);
+  p = fmaf(p, f, 1.0f);
+  return __int_as_float(__float_as_int(p) + (__float_as_int(r) << 23));
+}
+
 // Issues the load of 32 consecutive columns of this thread's lane; the registers are valid after tmem_ld_wait().
 __device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t* v) {
   asm volatile(
@@ -204,7 +221,10 @@ __global__ void __launch_bounds__(kScoreThreads, 2)
       const float mu = (mn == -CUDART_INF_F) ? 0.f : mn;   // a fully masked half row so far
       float sum[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int j = 0; j < 64; ++j) sum[j & 3] += fast_exp2(fmaf(__uint_as_float(v[j]), scale_log2, -mu));
+      for (int j = 0; j < 64; ++j) {
+        const float t = fmaf(__uint_as_float(v[j]), scale_log2, -mu);
+        sum[j & 3] += (j % kPolyEvery == kPolyEvery - 1) ? exp2_fma(t) : fast_exp2(t);
+      }
       l_run = l_run * fast_exp2(m_run - mu) + ((sum[0] + sum[1]) + (sum[2] + sum[3]));
       m_run = mn;
     }
