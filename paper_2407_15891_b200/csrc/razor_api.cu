@@ -90,6 +90,8 @@ inline long long head_capacity_tokens(const razor_config_t& c, int n_ctx, int wi
   return retrieval ? grown : std::min(grown, (long long)c.n_sink + window);
 }
 
+constexpr int kPlanSlots = 16;   // compression plans that may be on their way to the device at once
+
 struct LayerHost {
   bool any = false;
   int n_done = 0;
@@ -106,9 +108,6 @@ struct LayerHost {
   int32_t* jobs = nullptr;          // pinned host, [max_items + 1]
   MultiHead* multi = nullptr;       // pinned host, [B*Hkv]
   cudaEvent_t upload_done = nullptr;
-  // compression plan staging: HeadPlan[B*Hkv] then SeqDesc[B], the image of the device's plan region
-  uint8_t* plan = nullptr;          // pinned host
-  cudaEvent_t plan_done = nullptr;
 };
 
 uint64_t mix64(uint64_t x) {
@@ -131,8 +130,12 @@ struct razor_cache {
   WorkItem* pinned_items = nullptr;   // [L][max_items]
   int32_t* pinned_jobs = nullptr;     // [L][max_items + 1]
   MultiHead* pinned_multi = nullptr;  // [L][B*Hkv]
-  uint8_t* pinned_plan = nullptr;     // [L][plan_bytes]
+  // Compression plan staging: a ring of images of the device's plan region (HeadPlan[B*Hkv], then SeqDesc[B]),
+  // so that a run of compression calls does not wait for each upload before preparing the next.
+  uint8_t* pinned_plan = nullptr;     // [kPlanSlots][plan_bytes]
   size_t plan_bytes = 0;
+  cudaEvent_t plan_done[kPlanSlots] = {};
+  int plan_next = 0;
 };
 
 extern "C" {
@@ -242,7 +245,7 @@ int razor_cache_create(razor_cache_t** out, const razor_config_t* cfg, void* poo
                       cudaHostAllocDefault);
   c->plan_bytes = (size_t)dv.n_heads * sizeof(HeadPlan) + (size_t)cfg->batch * sizeof(SeqDesc);
   if (e == cudaSuccess)
-    e = cudaHostAlloc((void**)&c->pinned_plan, (size_t)cfg->n_layers * c->plan_bytes, cudaHostAllocDefault);
+    e = cudaHostAlloc((void**)&c->pinned_plan, (size_t)kPlanSlots * c->plan_bytes, cudaHostAllocDefault);
   if (e != cudaSuccess) {
     g_last_cuda_error = (int)e;
     (void)cudaGetLastError();
@@ -264,7 +267,6 @@ int razor_cache_create(razor_cache_t** out, const razor_config_t* cfg, void* poo
     L.items = c->pinned_items + (size_t)l * lay.max_items;
     L.jobs = c->pinned_jobs + (size_t)l * (lay.max_items + 1);
     L.multi = c->pinned_multi + (size_t)l * dv.n_heads;
-    L.plan = c->pinned_plan + (size_t)l * c->plan_bytes;
   }
   *out = c;
   return RAZOR_OK;
@@ -289,12 +291,13 @@ int razor_cache_destroy(razor_cache_t* c) {
   if (!c) return RAZOR_E_NULL_PTR;
   for (LayerHost& L : c->layers) {
     if (L.upload_done) cudaEventDestroy(L.upload_done);
-    if (L.plan_done) cudaEventDestroy(L.plan_done);
   }
   if (c->pinned_items) cudaFreeHost(c->pinned_items);
   if (c->pinned_jobs) cudaFreeHost(c->pinned_jobs);
   if (c->pinned_multi) cudaFreeHost(c->pinned_multi);
   if (c->pinned_plan) cudaFreeHost(c->pinned_plan);
+  for (cudaEvent_t ev : c->plan_done)
+    if (ev) cudaEventDestroy(ev);
   delete c;
   return RAZOR_OK;
 }
@@ -373,9 +376,12 @@ int compress_impl(razor_cache* c, int layer, const std::vector<SeqIn>& seqs, con
 
   // The plan goes to the device in one copy from pinned memory: per head its state after the call and the
   // run of pool pages behind its page-table row (compress_plan_kernel writes both), then the sequences.
-  if (L.plan_done) RZ_CUDA(cudaEventSynchronize(L.plan_done));   // the previous plan has left the staging area
-  HeadPlan* plan = (HeadPlan*)L.plan;
-  SeqDesc* descs = (SeqDesc*)(L.plan + (size_t)c->dv.n_heads * sizeof(HeadPlan));
+  const int slot = c->plan_next;
+  c->plan_next = (slot + 1) % kPlanSlots;
+  if (c->plan_done[slot]) RZ_CUDA(cudaEventSynchronize(c->plan_done[slot]));   // its last upload has left the slot
+  uint8_t* staging = c->pinned_plan + (size_t)slot * c->plan_bytes;
+  HeadPlan* plan = (HeadPlan*)staging;
+  SeqDesc* descs = (SeqDesc*)(staging + (size_t)c->dv.n_heads * sizeof(HeadPlan));
   int n_plan = 0;
   std::vector<int32_t> rows;   // only for permuted page ids
   for (size_t i = 0; i < seqs.size(); ++i) {
@@ -431,9 +437,9 @@ int compress_impl(razor_cache* c, int layer, const std::vector<SeqIn>& seqs, con
     if (!L.seq_done[s.b]) { L.seq_done[s.b] = 1; L.n_done += 1; }
   }
   // one copy covers plan[0 .. n_plan) and, behind the full plan array, the sequence descriptors
-  RZ_CUDA(cudaMemcpyAsync(c->dv.plan, L.plan, c->plan_bytes, cudaMemcpyHostToDevice, stream));
-  if (!L.plan_done) RZ_CUDA(cudaEventCreateWithFlags(&L.plan_done, cudaEventDisableTiming));
-  RZ_CUDA(cudaEventRecord(L.plan_done, stream));
+  RZ_CUDA(cudaMemcpyAsync(c->dv.plan, staging, c->plan_bytes, cudaMemcpyHostToDevice, stream));
+  if (!c->plan_done[slot]) RZ_CUDA(cudaEventCreateWithFlags(&c->plan_done[slot], cudaEventDisableTiming));
+  RZ_CUDA(cudaEventRecord(c->plan_done[slot], stream));
   L.retr = flags;
   L.any = true;
   L.appended = 0;
