@@ -165,9 +165,11 @@ RAZOR_API int razor_decode_attention(razor_cache_t* cache, int32_t layer, const 
  *                                 attends to the kept tokens at positions <= its own (Section 3.1:
  *                                 n <= m) plus the compensation token with its count N_d (Eq. 5).
  *                                 n_tokens = 1 is razor_decode_attention.
- * Limits of the multi-token call: bf16, (Hq / Hkv) * n_tokens in {2, 4, 8} (the rows of one KV head's
- * tile run on matrix instructions), at least n_tokens tokens cached, and every head that has dropped
+ * Limits of the multi-token call: bf16; at least n_tokens tokens cached; every head that has dropped
  * tokens must have a window >= n_tokens (otherwise its mean would hold tokens that come after a query).
+ * One launch takes a tile of 2, 4 or 8 rows per KV head (query heads of the group x query tokens, on
+ * matrix instructions); a longer round runs as several launches, block by block, each streaming the
+ * cache once and masking the round's tokens that come after its block.
  * Errors: NULL_PTR, INVALID_ARG, UNSUPPORTED_DIM, NOT_COMPRESSED, CAPACITY (append), MISALIGNED, CUDA.
  */
 RAZOR_API int razor_append_many(razor_cache_t* cache, int32_t layer, const void* k_new, const void* v_new,

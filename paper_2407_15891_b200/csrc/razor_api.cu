@@ -608,7 +608,8 @@ int razor_append_many(razor_cache_t* c, int32_t layer, const void* k_new, const 
   return RAZOR_OK;
 }
 
-static int decode_impl(razor_cache_t* c, int32_t layer, const void* q, float* out, int32_t n_tokens, void* stream);
+static int decode_impl(razor_cache_t* c, int32_t layer, const void* q, float* out, int32_t n_tokens,
+                       int32_t tok_stride, int32_t q_after, void* stream);
 
 int razor_decode_attention_multi(razor_cache_t* c, int32_t layer, const void* q, float* out, int32_t n_tokens,
                                  void* stream) {
@@ -616,31 +617,44 @@ int razor_decode_attention_multi(razor_cache_t* c, int32_t layer, const void* q,
   int rc = layer_ready(c, layer);
   if (rc) return rc;
   if (n_tokens < 1) return RAZOR_E_INVALID_ARG;
-  if (n_tokens > 1) {
-    const int rows = (c->cfg.n_q_heads / c->cfg.n_kv_heads) * n_tokens;
-    if (c->cfg.dtype != RAZOR_BF16 || (rows != 2 && rows != 4 && rows != 8)) return RAZOR_E_UNSUPPORTED_DIM;
-    for (const HeadState& h : c->layers[layer].hs) {
-      if (h.len + h.n_drop < n_tokens) return RAZOR_E_INVALID_ARG;          // fewer tokens cached than queries
-      if (h.n_drop > 0 && h.window < n_tokens) return RAZOR_E_INVALID_ARG;  // the mean would hold tokens after a query
-    }
+  if (n_tokens == 1) return decode_impl(c, layer, q, out, 1, 1, 0, stream);
+  if (c->cfg.dtype != RAZOR_BF16) return RAZOR_E_UNSUPPORTED_DIM;
+  for (const HeadState& h : c->layers[layer].hs) {
+    if (h.len + h.n_drop < n_tokens) return RAZOR_E_INVALID_ARG;          // fewer tokens cached than queries
+    if (h.n_drop > 0 && h.window < n_tokens) return RAZOR_E_INVALID_ARG;  // the mean would hold tokens after a query
   }
-  return decode_impl(c, layer, q, out, n_tokens, stream);
+  // One launch takes a tile of 2, 4 or 8 rows per KV head (query heads of the group x query tokens).  A
+  // longer round runs block by block, the largest block that fits; when the round is not a multiple of
+  // the block, the last block is moved back to end with the round and recomputes a few tokens.
+  const int group = c->cfg.n_q_heads / c->cfg.n_kv_heads;
+  int block = 0;
+  for (int rows = 8; rows >= 2 && !block; rows >>= 1)
+    if (rows % group == 0 && rows / group <= n_tokens) block = rows / group;
+  if (!block) return RAZOR_E_UNSUPPORTED_DIM;
+  const size_t row_elems = (size_t)c->cfg.n_q_heads * c->cfg.head_dim;
+  for (int start = 0;; start += block) {
+    if (start + block > n_tokens) start = n_tokens - block;
+    rc = decode_impl(c, layer, (const char*)q + (size_t)start * row_elems * esz(c->cfg), out + (size_t)start * row_elems,
+                     block, n_tokens, n_tokens - start - block, stream);
+    if (rc || start + block >= n_tokens) return rc;
+  }
 }
 
 int razor_decode_attention(razor_cache_t* c, int32_t layer, const void* q, float* out, void* stream) {
   if (!c || !q || !out) return RAZOR_E_NULL_PTR;
   int rc = layer_ready(c, layer);
   if (rc) return rc;
-  return decode_impl(c, layer, q, out, 1, stream);
+  return decode_impl(c, layer, q, out, 1, 1, 0, stream);
 }
 
-static int decode_impl(razor_cache_t* c, int32_t layer, const void* q, float* out, int32_t n_tokens, void* stream) {
+static int decode_impl(razor_cache_t* c, int32_t layer, const void* q, float* out, int32_t n_tokens,
+                       int32_t tok_stride, int32_t q_after, void* stream) {
   int rc;
   if (((uintptr_t)q | (uintptr_t)out) & 15) return RAZOR_E_MISALIGNED;
   rc = ensure_schedule(c, layer, (cudaStream_t)stream, true);
   if (rc) return rc;
   const LayerHost& L = c->layers[layer];
-  const DecodeJobs jb{L.n_items, L.n_jobs, L.n_spans, L.jobs[L.n_spans], L.n_multi, n_tokens};
+  const DecodeJobs jb{L.n_items, L.n_jobs, L.n_spans, L.jobs[L.n_spans], L.n_multi, n_tokens, tok_stride, q_after};
   RZ_CUDA(launch_decode(c->dv, c->cfg.dtype, layer, jb, q, out, c->n_sms, c->tune,
                         (cudaStream_t)stream));
   return RAZOR_OK;

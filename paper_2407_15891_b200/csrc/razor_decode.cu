@@ -131,7 +131,8 @@ __device__ __forceinline__ void merge_state(float& m, float& l, float (&o)[EPL],
 struct RoundMask {
   int n_tok, g_real;            // query tokens of the round; query heads per KV head
   int alibi;                    // 1: add the ALiBi distance penalty
-  int total;                    // tokens the head has seen (len + n_drop): query t sits at total - n_tok + t
+  int total;                    // tokens the head has seen (len + n_drop)
+  int q_after;                  // tokens of the round after this launch's block: query t sits at total - q_after - n_tok + t
   int n_sink, ring_head, window, n_drop;
   int slot0;                    // slot of the page's first token
   // position of the token in slot s (Algorithm 1 keeps sinks + a ring of the recent tokens)
@@ -306,9 +307,9 @@ __device__ __forceinline__ void consume_page_mma(uint32_t page_addr, int valid, 
     if (g >= valid) s[0] = s[1] = -CUDART_INF_F;
     if (g + 8 >= valid) s[2] = s[3] = -CUDART_INF_F;
   }
-  if (mk.n_tok > 1 || mk.alibi) {
-    const int t2 = (lane & 3) * 2;
-    const int qp0 = mk.total - mk.n_tok + t2 / mk.g_real, qp1 = mk.total - mk.n_tok + (t2 + 1) / mk.g_real;
+  if (mk.n_tok > 1 || mk.alibi || mk.q_after > 0) {
+    const int t2 = (lane & 3) * 2, q_first = mk.total - mk.q_after - mk.n_tok;
+    const int qp0 = q_first + t2 / mk.g_real, qp1 = q_first + (t2 + 1) / mk.g_real;
     const int p0 = mk.pos(mk.slot0 + g), p1 = mk.pos(mk.slot0 + g + 8);
     if (mk.alibi) {            // Eq. 1: - l_h (m - n); slope0/1 belong to this lane's two rows, log2 domain
       s[0] += slope0 * (float)(p0 - qp0);
@@ -479,7 +480,7 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
   const int g_real = G / jb.n_tok;
   auto row_offset = [&](int head, int r) {
     const int b = head / dv.n_kv_heads, g = head % dv.n_kv_heads;
-    return (((size_t)b * jb.n_tok + r / g_real) * ((size_t)dv.n_kv_heads * g_real) + (size_t)g * g_real + r % g_real) * D;
+    return (((size_t)b * jb.tok_stride + r / g_real) * ((size_t)dv.n_kv_heads * g_real) + (size_t)g * g_real + r % g_real) * D;
   };
   // Warp-uniform bounded wait: false for every lane if any lane's wait failed.
   auto warp_wait = [&](uint64_t* bar, uint32_t parity) -> bool {
@@ -711,8 +712,8 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
                 vrows[idx] = make_uint4(0u, 0u, 0u, 0u);
               __syncwarp();
             }
-            const RoundMask mk{jb.n_tok, g_real, dv.alibi, d.len + d.n_drop, dv.n_sink, d.ring_head, d.window, d.n_drop,
-                               (d.page_begin + i) * kPageTokens};
+            const RoundMask mk{jb.n_tok, g_real, dv.alibi, d.len + d.n_drop, jb.q_after, dv.n_sink, d.ring_head, d.window,
+                               d.n_drop, (d.page_begin + i) * kPageTokens};
             consume_page_mma<D>(smem_u32(page), valid, lane, dv.scale_log2, qa, S, mk, slope0, slope1);
           }
           __syncwarp();
@@ -787,7 +788,7 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
           ring_slot<NC>(c + i, ns, stage, use);
           if (!warp_wait(&bars.full[stage], use & 1)) { ok = false; break; }
           if (i < d.n_pages) {
-            const RoundMask mk{1, G, dv.alibi, d.len + d.n_drop, dv.n_sink, d.ring_head, d.window, d.n_drop,
+            const RoundMask mk{1, G, dv.alibi, d.len + d.n_drop, 0, dv.n_sink, d.ring_head, d.window, d.n_drop,
                                (d.page_begin + i) * kPageTokens};
             consume_page<T, D, G>((const uint4*)(ring + (size_t)stage * PB), d.len - (d.page_begin + i) * kPageTokens,
                                   rg, lir, qf, S, dv.alibi != 0, mk, slope);
@@ -893,7 +894,7 @@ constexpr int kCombineWarps = 16;
 
 template <int D>
 __global__ void __launch_bounds__(kCombineWarps * 32) combine_kernel(DeviceView dv, int layer, int n_tok,
-                                                                     float* __restrict__ out) {
+                                                                     int tok_stride, float* __restrict__ out) {
   __shared__ float2 s_ml[kCombineWarps];
   __shared__ __align__(16) float s_o[kCombineWarps][D];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -949,12 +950,13 @@ __global__ void __launch_bounds__(kCombineWarps * 32) combine_kernel(DeviceView 
     }
     sum.scale(lt > 0.f ? 1.f / lt : 0.f);
     const int b = mh.head / dv.n_kv_heads, g = mh.head % dv.n_kv_heads, gr = dv.group;
-    sum.store(out + (((size_t)b * n_tok + j / gr) * ((size_t)dv.n_kv_heads * gr) + (size_t)g * gr + j % gr) * D, lane);
+    sum.store(out + (((size_t)b * tok_stride + j / gr) * ((size_t)dv.n_kv_heads * gr) + (size_t)g * gr + j % gr) * D, lane);
   }
 }
 
 template <int D>
-cudaError_t combine_launch(const DeviceView& dv, int layer, int n_multi, int n_tok, float* out, cudaStream_t s) {
+cudaError_t combine_launch(const DeviceView& dv, int layer, int n_multi, int n_tok, int tok_stride, float* out,
+                           cudaStream_t s) {
   if (n_multi <= 0) return cudaSuccess;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(n_multi, dv.group * n_tok);
@@ -966,7 +968,7 @@ cudaError_t combine_launch(const DeviceView& dv, int layer, int n_multi, int n_t
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, combine_kernel<D>, dv, layer, n_tok, out);
+  return cudaLaunchKernelEx(&cfg, combine_kernel<D>, dv, layer, n_tok, tok_stride, out);
 }
 
 // ------------------------------------------------------------------------------------------ launch
@@ -1013,7 +1015,7 @@ cudaError_t decode_launch(const DeviceView& dv, int layer, const DecodeJobs& jb,
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   if ((e = cudaLaunchKernelEx(&cfg, kern, dv, layer, jb, (const T*)q, out, (int)stages)) != cudaSuccess) return e;
-  return combine_launch<D>(dv, layer, jb.n_multi, jb.n_tok, out, s);
+  return combine_launch<D>(dv, layer, jb.n_multi, jb.n_tok, jb.tok_stride, out, s);
 }
 
 template <typename T, int D, int G>
@@ -1025,7 +1027,7 @@ cudaError_t decode_nc(const DeviceView& dv, int layer, const DecodeJobs& jb, con
   if constexpr (sizeof(T) == 2 && G >= 2) {
     // Grouped heads: the tensor-core consumer unless switched off (default on from group 4 up).
     // (rounds of several query tokens always take it: only that consumer applies their causal mask)
-    const bool mma = jb.n_tok > 1 || tune.tensor_cores == 1 || (tune.tensor_cores == 0 && G >= 4);
+    const bool mma = jb.n_tok > 1 || jb.q_after > 0 || tune.tensor_cores == 1 || (tune.tensor_cores == 0 && G >= 4);
     if (mma) {
       if (nc == 4) return decode_launch<T, D, G, 4, true>(dv, layer, jb, q, out, n_sms, tune, s);
       return decode_launch<T, D, G, 8, true>(dv, layer, jb, q, out, n_sms, tune, s);

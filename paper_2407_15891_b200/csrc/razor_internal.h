@@ -135,7 +135,12 @@ cudaError_t launch_append_many(const DeviceView& dv, int dtype, int layer, const
 struct DecodeJobs {
   int32_t n_items, n_jobs, n_spans, tail_first;
   int32_t n_multi;   // heads in several parts
-  int32_t n_tok;     // query tokens per sequence in this call (1 for a decode step)
+  int32_t n_tok;     // query tokens per sequence in this launch (1 for a decode step)
+  // A round longer than one launch can take is run block by block: q and out point at the block's first
+  // token, tok_stride is the round's length (tokens per sequence in q and out), q_after the number of
+  // tokens of the round that come after the block (they are cached already, and masked).
+  int32_t tok_stride;
+  int32_t q_after;
 };
 cudaError_t launch_decode(const DeviceView& dv, int dtype, int layer, const DecodeJobs& jobs, const void* q,
                           float* out, int n_sms, const DecodeTuning& tune, cudaStream_t stream);

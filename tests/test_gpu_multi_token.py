@@ -78,6 +78,34 @@ def test_round_on_a_long_context_with_split_heads():
     cache.close()
 
 
+@pytest.mark.parametrize("group,T,D", [(1, 16, 128), (1, 9, 128), (1, 3, 64), (2, 5, 128), (4, 3, 128), (8, 2, 64), (1, 29, 128)])
+def test_round_longer_than_one_launch_runs_block_by_block(group, T, D):
+    """Rounds that do not fit one tile of 2, 4 or 8 rows: blocks of the largest size that fits, the last one moved
+    back to end with the round; every block masks the round's tokens that come after it."""
+    Hkv = 2
+    w = synth.Workload("long_round", 2, 1, Hkv * group, Hkv, D, "bf16", [700, 90], [120, 40], 4, 1, T, 777 + T + group)
+    cache = make_cache(w, max_new=T)
+    K, V = synth.make_dense_kv(w, 0, DEV)
+    retr = w.retrieval(0)
+    cache.compress(0, K, V, w.ctx_len, retr, w.window)
+    refs = {(b, g): HeadRef(0, b, g, K[b, g], V[b, g], w.ctx_len[b], T) for b in range(w.batch) for g in range(Hkv)}
+    k, v, q = _round_inputs(w, T, 3)
+    cache.append_many(0, k, v)
+    out = to_f64(cache.decode_multi(0, q))
+    assert cache.device_status() == 0
+    kh, vh, qh = k.cpu(), v.cpu(), to_f64(q)
+    scale = 1.0 / math.sqrt(D)
+    for (b, g), ref in refs.items():
+        for t in range(T):
+            ref.append(kh[b, t, g], vh[b, t, g])
+        for j in range(group):
+            expect = orc.multi_query_attention(qh[b, :, g * group + j], ref.K[:ref.n], ref.V[:ref.n], w.n_sink,
+                                               w.window[b], bool(retr[g]), scale)
+            err = float(np.abs(out[b, :, g * group + j] - expect).max())
+            assert err <= TOL_OUT["bf16"], (err, b, g, j)
+    cache.close()
+
+
 def test_round_limits_are_reported():
     w = synth.Workload("round_err", 1, 1, 2, 2, 64, "bf16", [100], [3], 4, 0, 8, 1)
     cache = make_cache(w, max_new=8)
@@ -88,10 +116,6 @@ def test_round_limits_are_reported():
     with pytest.raises(rz.RazorError) as e:
         cache.decode_multi(0, q)                               # window 3 < 4 tokens of the round
     assert e.value.status == -1
-    k3, v3, q3 = _round_inputs(w, 3, 1)
-    with pytest.raises(rz.RazorError) as e:
-        cache.decode_multi(0, q3)                              # 1 x 3 rows: not a tile shape
-    assert e.value.status == -3
     with pytest.raises(rz.RazorError) as e:
         rz.razor_append_many(cache.handle, 0, k, v, 5)         # beyond max_new_tokens
     assert e.value.status == -5
