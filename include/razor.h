@@ -174,6 +174,19 @@ RAZOR_API int razor_decode_attention(razor_cache_t* cache, int32_t layer, const 
  */
 RAZOR_API int razor_append_many(razor_cache_t* cache, int32_t layer, const void* k_new, const void* v_new,
                       int32_t n_tokens, void* stream);
+
+/*
+ * Host only: what a run of n_tokens appends does to ONE head whose state is (len, n_drop, ring_head,
+ * window; window < 0: the head keeps everything), in closed form - the rule the parallel append kernel
+ * and the library's host mirror apply.  slot[a] (host, [n_tokens] or NULL): physical slot token a ends up
+ * in, -1 when the run itself evicts it again (it is then folded into the compensation sums directly);
+ * evicts_old[a] (host or NULL): 1 when that slot held a token from before the run, which is folded into
+ * the sums first.  The state after the run goes to the three out-pointers (each may be NULL).
+ * Errors: INVALID_ARG (a state no sequence of appends can produce).
+ */
+RAZOR_API int razor_append_plan(int32_t len, int32_t n_drop, int32_t ring_head, int32_t window, int32_t n_sink,
+                                int32_t n_tokens, int32_t* slot, uint8_t* evicts_old, int32_t* len_after,
+                                int32_t* n_drop_after, int32_t* ring_head_after);
 RAZOR_API int razor_decode_attention_multi(razor_cache_t* cache, int32_t layer, const void* q, float* out,
                                  int32_t n_tokens, void* stream);
 

@@ -26,7 +26,7 @@ STATUS = {
 # every symbol include/razor.h declares
 SYMBOLS = [
     "razor_query_bytes", "razor_cache_create", "razor_compress", "razor_compress_seq", "razor_append",
-    "razor_decode_attention", "razor_append_many", "razor_decode_attention_multi", "razor_cache_export", "razor_cache_stats", "razor_schedule_plan",
+    "razor_decode_attention", "razor_append_many", "razor_append_plan", "razor_decode_attention_multi", "razor_cache_export", "razor_cache_stats", "razor_schedule_plan",
     "razor_schedule_query", "razor_cache_set_option", "razor_cache_device_status", "razor_cache_wait_selftest", "razor_cache_set_alibi", "razor_cache_set_head_windows",
     "razor_compensation_mean_static", "razor_head_scores_scratch_bytes", "razor_head_scores",
     "razor_select_retrieval_heads", "razor_cache_reset", "razor_cache_destroy", "razor_status_string",
@@ -73,6 +73,7 @@ def load() -> C.CDLL:
     lib.razor_append.argtypes = [vp, i32, vp, vp, vp]
     lib.razor_decode_attention.argtypes = [vp, i32, vp, vp, vp]
     lib.razor_append_many.argtypes = [vp, i32, vp, vp, i32, vp]
+    lib.razor_append_plan.argtypes = [i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp]
     lib.razor_decode_attention_multi.argtypes = [vp, i32, vp, vp, i32, vp]
     lib.razor_cache_export.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, C.POINTER(i32),
                                        C.POINTER(i32), vp]
@@ -191,6 +192,17 @@ def razor_decode_attention(cache: int, layer: int, q, out, stream=None) -> None:
 def razor_append_many(cache: int, layer: int, k_new, v_new, n_tokens: int, stream=None) -> None:
     _check(load().razor_append_many(cache, layer, _ptr(k_new), _ptr(v_new), n_tokens, _stream(stream)),
            "razor_append_many")
+
+
+def razor_append_plan(len_: int, n_drop: int, ring_head: int, window: int, n_sink: int, n_tokens: int):
+    """Host only.  -> (slot[n_tokens] int32, evicts_old[n_tokens] uint8, (len, n_drop, ring_head) after the run)."""
+    slot = np.empty(max(1, n_tokens), dtype=np.int32)
+    old = np.empty(max(1, n_tokens), dtype=np.uint8)
+    after = np.zeros(3, dtype=np.int32)
+    _check(load().razor_append_plan(len_, n_drop, ring_head, window, n_sink, n_tokens, slot.ctypes.data, old.ctypes.data,
+                                    after[0:].ctypes.data, after[1:].ctypes.data, after[2:].ctypes.data),
+           "razor_append_plan")
+    return slot[:n_tokens], old[:n_tokens], tuple(int(x) for x in after)
 
 
 def razor_decode_attention_multi(cache: int, layer: int, q, out, n_tokens: int, stream=None) -> None:

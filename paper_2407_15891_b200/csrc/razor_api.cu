@@ -594,17 +594,29 @@ int razor_append_many(razor_cache_t* c, int32_t layer, const void* k_new, const 
   }
   RZ_CUDA(launch_append_many(c->dv, c->cfg.dtype, layer, k_new, v_new, n_tokens, slices, (cudaStream_t)stream));
   const int n_sink = c->cfg.n_sink;
-  for (HeadState& h : L.hs) {   // host mirror of the kernels' state update, in closed form
-    const bool keeps_all = h.window < 0;
-    const int cap = keeps_all ? 0 : n_sink + h.window;
-    const int f = keeps_all ? n_tokens : std::min(n_tokens, std::max(0, cap - h.len));
-    const int E = n_tokens - f;
-    h.len += f;
-    h.n_drop += E;
-    h.ring_head = h.window > 0 ? (int)(((long long)h.ring_head + E) % h.window) : 0;
-  }
+  for (HeadState& h : L.hs) h = state_after_run(h, n_sink, n_tokens);   // host mirror of the kernels' state update
   L.appended += n_tokens;
   L.growth_tokens += n_tokens;
+  return RAZOR_OK;
+}
+
+int razor_append_plan(int32_t len, int32_t n_drop, int32_t ring_head, int32_t window, int32_t n_sink, int32_t n_tokens,
+                      int32_t* slot, uint8_t* evicts_old, int32_t* len_after, int32_t* n_drop_after,
+                      int32_t* ring_head_after) {
+  if (len < 0 || n_drop < 0 || n_sink < 0 || n_tokens < 0) return RAZOR_E_INVALID_ARG;
+  if (window >= 0 && (len > n_sink + window || ring_head < 0 || (window > 0 && ring_head >= window)))
+    return RAZOR_E_INVALID_ARG;
+  if (window >= 0 && len < n_sink + window && ring_head != 0) return RAZOR_E_INVALID_ARG;   // a ring that fills starts at 0
+  const HeadState st{len, n_drop, ring_head, window};
+  for (int a = 0; a < n_tokens; ++a) {
+    const AppendFate f = append_fate(st, n_sink, n_tokens, a);
+    if (slot) slot[a] = f.slot;
+    if (evicts_old) evicts_old[a] = f.evicts_old ? 1 : 0;
+  }
+  const HeadState nx = state_after_run(st, n_sink, n_tokens);
+  if (len_after) *len_after = nx.len;
+  if (n_drop_after) *n_drop_after = nx.n_drop;
+  if (ring_head_after) *ring_head_after = nx.ring_head;
   return RAZOR_OK;
 }
 

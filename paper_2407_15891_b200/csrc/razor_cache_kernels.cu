@@ -349,18 +349,13 @@ __global__ void __launch_bounds__(128) append_many_kernel(DeviceView dv, int lay
 
 // ---------------------------------------------------------------------------------------------
 // Append of a long run of tokens (a prompt chunk of a chunked prefill, a long second prompt), in
-// parallel over the tokens.  The state afterwards is what n_tok single appends would leave; what n_tok
-// single appends do one after the other is decided here per token in closed form.  With len0, ring_head0
-// the state before the call, cap = N0 + W, f = tokens that still fit (all of them for a head that keeps
-// everything) and E = n_tok - f tokens that each evict the oldest recent token:
-//   * token a < f goes to slot len0 + a; it is overwritten again within the call when its ring index
-//     r = len0 + a - N0 is below E (the ring starts at index 0 while it fills);
-//   * evicting token j = a - f goes to ring index (ring_head0 + j) mod W and stays iff j >= E - W;
-//   * a token that does not stay is added to the compensation sums straight from the input; a token that
-//     stays in a ring slot that held a token from before the call adds that old row to the sums first.
-// Every slot is written by exactly one thread group, after it has read the old row, so there is no order
-// between CTAs to keep.  grid = (slices, heads); per-slice sums go to the compression scratch and
-// append_chunk_finalize_kernel adds them to the running sums (Eq. 4 over everything dropped so far).
+// parallel over the tokens.  The state afterwards is what n_tok single appends would leave; append_fate()
+// decides per token, in closed form, where it ends up.  A token that does not stay is added to the
+// compensation sums straight from the input; a token that stays in a ring slot that held a token from
+// before the call adds that old row to the sums first.  Every slot is written by exactly one thread group,
+// after it has read the old row, so there is no order between CTAs to keep.  grid = (slices, heads);
+// per-slice sums go to the compression scratch and append_chunk_finalize_kernel adds them to the running
+// sums (Eq. 4 over everything dropped so far).
 template <typename T, int D>
 __global__ void __launch_bounds__(256) append_chunk_kernel(DeviceView dv, int layer, const T* __restrict__ k_new,
                                                            const T* __restrict__ v_new, int n_tok, int n_slices) {
@@ -370,12 +365,7 @@ __global__ void __launch_bounds__(256) append_chunk_kernel(DeviceView dv, int la
   const int head = blockIdx.y;
   const size_t hs = (size_t)layer * dv.n_heads + head;
   const HeadState st = dv.state[hs];
-  const int n_sink = dv.n_sink, W = st.window;
-  const bool keeps_all = W < 0;
-  const int cap = keeps_all ? 0 : n_sink + W;
-  const int f = keeps_all ? n_tok : min(n_tok, max(0, cap - st.len));
-  const int E = n_tok - f;
-  const int ring0 = max(0, st.len - n_sink);   // ring tokens from before the call
+  const int n_sink = dv.n_sink;
   const int b = head / dv.n_kv_heads, g = head % dv.n_kv_heads;
   const int32_t* pt = dv.page_table + hs * dv.max_pages;
   const int per = (n_tok + n_slices - 1) / n_slices;
@@ -389,18 +379,9 @@ __global__ void __launch_bounds__(256) append_chunk_kernel(DeviceView dv, int la
     const size_t row = (((size_t)b * n_tok + a) * dv.n_kv_heads + g) * D;
     const uint4 kf = ld_stream((const uint4*)(k_new + row) + lir);
     const uint4 vf = ld_stream((const uint4*)(v_new + row) + lir);
-    int slot;
-    bool stays, had_old = false;
-    if (a < f) {
-      slot = st.len + a;
-      stays = keeps_all || slot < n_sink || slot - n_sink >= E;
-    } else {
-      const int j = a - f;
-      stays = j >= E - W;   // never when W == 0
-      const int r = stays ? (int)(((long long)st.ring_head + j) % W) : 0;
-      slot = n_sink + r;
-      had_old = stays && r < ring0;
-    }
+    const AppendFate fate = append_fate(st, n_sink, n_tok, a);
+    const int slot = fate.slot;
+    const bool stays = slot >= 0, had_old = fate.evicts_old;
     float a_k[EPL], a_v[EPL];
     if (stays) {
       const size_t page = (size_t)pt[slot >> 4];
@@ -442,10 +423,7 @@ __global__ void append_chunk_finalize_kernel(DeviceView dv, int layer, int n_tok
   const int head = blockIdx.x, e = threadIdx.x;
   const size_t hs = (size_t)layer * dv.n_heads + head;
   const HeadState st = dv.state[hs];
-  const bool keeps_all = st.window < 0;
-  const int cap = keeps_all ? 0 : dv.n_sink + st.window;
-  const int f = keeps_all ? n_tok : min(n_tok, max(0, cap - st.len));
-  const int E = n_tok - f;
+  const int E = n_tok - append_run_fits(st, dv.n_sink, n_tok);
   if (E > 0) {
     const float* scratch = dv.compress_scratch + (size_t)head * n_slices * 2 * D;
     float s = dv.comp_sum[hs * 2 * D + e];
@@ -454,13 +432,7 @@ __global__ void append_chunk_finalize_kernel(DeviceView dv, int layer, int n_tok
     dv.comp_mean[hs * 2 * D + e] = __fdiv_rn(s, (float)(st.n_drop + E));
   }
   __syncthreads();   // every thread has read the old state
-  if (e == 0) {
-    HeadState nx = st;
-    nx.len = st.len + f;
-    nx.n_drop = st.n_drop + E;
-    nx.ring_head = st.window > 0 ? (int)(((long long)st.ring_head + E) % st.window) : 0;
-    dv.state[hs] = nx;
-  }
+  if (e == 0) dv.state[hs] = state_after_run(st, dv.n_sink, n_tok);
 }
 
 // ---------------------------------------------------------------------------------------------

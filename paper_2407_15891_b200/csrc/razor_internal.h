@@ -26,6 +26,54 @@ struct HeadState {
   int32_t window;     // recent-window length; < 0: keeps everything
 };
 
+// A run of n_tok appended tokens, decided per token in closed form (what n_tok single appends do one after
+// the other).  With cap = N0 + W: the first f tokens still fit (all of them for a head that keeps everything),
+// the other E = n_tok - f each evict the oldest recent token.  Token a < f goes to slot len + a and is overwritten
+// again within the run when its ring index len + a - N0 is below E (the ring starts at index 0 while it fills);
+// evicting token j = a - f goes to ring index (ring_head + j) mod W and stays iff j >= E - W.  A token that stays
+// in a ring slot which held a token from before the run (ring index below the old ring fill) evicts that old
+// row: it has to be added to the compensation sums before it is overwritten.  A token that does not stay is
+// added to the sums itself.
+struct AppendFate {
+  int32_t slot;     // physical slot the token ends up in, -1 when it does not stay
+  bool evicts_old;  // the slot held a token from before the run
+};
+#if defined(__CUDACC__)
+#define RAZOR_HD __host__ __device__
+#else
+#define RAZOR_HD
+#endif
+RAZOR_HD inline int append_run_fits(const HeadState& st, int n_sink, int n_tok) {
+  if (st.window < 0) return n_tok;
+  const int room = n_sink + st.window - st.len;
+  return room <= 0 ? 0 : (room < n_tok ? room : n_tok);
+}
+RAZOR_HD inline AppendFate append_fate(const HeadState& st, int n_sink, int n_tok, int a) {
+  const int f = append_run_fits(st, n_sink, n_tok), E = n_tok - f, W = st.window;
+  AppendFate r{-1, false};
+  if (a < f) {
+    const int slot = st.len + a;
+    if (W < 0 || slot < n_sink || slot - n_sink >= E) r.slot = slot;
+  } else {
+    const int j = a - f;
+    if (j >= E - W) {   // never when W == 0
+      const int ring = (int)(((long long)st.ring_head + j) % W);
+      const int ring_fill = st.len > n_sink ? st.len - n_sink : 0;   // ring tokens from before the run
+      r.slot = n_sink + ring;
+      r.evicts_old = ring < ring_fill;
+    }
+  }
+  return r;
+}
+RAZOR_HD inline HeadState state_after_run(const HeadState& st, int n_sink, int n_tok) {
+  const int f = append_run_fits(st, n_sink, n_tok), E = n_tok - f;
+  HeadState nx = st;
+  nx.len = st.len + f;
+  nx.n_drop = st.n_drop + E;
+  nx.ring_head = st.window > 0 ? (int)(((long long)st.ring_head + E) % st.window) : 0;
+  return nx;
+}
+
 // One decode work item: pages [page_begin, page_end) of one head's token stream, streamed by one CTA.
 // page_end < 0 means "to the end of the stream as it is now" (the last part of a head grows with
 // appends).  A head cut into n_parts > 1 items owns n_parts partial records starting at rec_base, which

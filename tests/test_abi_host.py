@@ -209,3 +209,57 @@ def test_header_is_plain_c():
     r = subprocess.run([gcc, "-std=c99", "-Wall", "-Werror", "-pedantic", "-fsyntax-only", "-I", os.path.join(root, "include"),
                         "-x", "c", "-"], input=src, text=True, capture_output=True)
     assert r.returncode == 0, r.stderr
+
+
+def _sequential_appends(len0, n_drop0, ring_head0, window, n_sink, n_tokens):
+    """The single-token rule applied n_tokens times on a model cache: slots hold token ids (old tokens are
+    negative, new token a is a), `folded` collects what went into the compensation sums."""
+    slots = {s: -(s + 1) for s in range(len0)}
+    length, n_drop, head, folded = len0, n_drop0, ring_head0, []
+    for a in range(n_tokens):
+        if window < 0 or length < n_sink + window:
+            slots[length] = a
+            length += 1
+        elif window == 0:
+            folded.append(a)
+            n_drop += 1
+        else:
+            s = n_sink + head
+            folded.append(slots[s])
+            slots[s] = a
+            n_drop += 1
+            head = (head + 1) % window
+    return slots, folded, (length, n_drop, head)
+
+
+def test_append_run_in_closed_form_equals_single_appends():
+    """razor_append_plan (the rule of the parallel append kernel and of the host mirror) against the single-token
+    rule applied token by token, for every small state: same final slot contents, same set of folded tokens, same
+    state."""
+    checked = 0
+    for n_sink in (0, 1, 3):
+        for window in (-1, 0, 1, 2, 5, 8):
+            cap = n_sink + max(window, 0)
+            for len0 in range(0, (cap if window >= 0 else 12) + 1):
+                full = window > 0 and len0 == cap
+                for ring_head0 in (range(window) if full else [0]):
+                    for n_tokens in (0, 1, 2, 3, 7, 8, 9, 20):
+                        want_slots, want_folded, want_state = _sequential_appends(len0, 4, ring_head0, window, n_sink, n_tokens)
+                        slot, old, state = rz.razor_append_plan(len0, 4, ring_head0, window, n_sink, n_tokens)
+                        assert state == want_state
+                        got_slots = {s: -(s + 1) for s in range(len0)}
+                        got_folded = []
+                        for a in range(n_tokens):
+                            if slot[a] < 0:
+                                got_folded.append(a)
+                                continue
+                            if old[a]:
+                                got_folded.append(-(int(slot[a]) + 1))          # the old token of that slot
+                            got_slots[int(slot[a])] = a
+                        assert got_slots == want_slots
+                        assert sorted(got_folded) == sorted(want_folded)
+                        assert len(set(int(s) for s in slot if s >= 0)) == int((slot >= 0).sum())   # one writer per slot
+                        checked += 1
+    assert checked > 1000
+    with pytest.raises(rz.RazorError):
+        rz.razor_append_plan(3, 0, 1, 8, 2, 3)                  # a ring that is still filling starts at index 0
