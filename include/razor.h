@@ -238,8 +238,9 @@ enum {
   RAZOR_OPT_DECODE_RING_KB = 3,         /* shared-memory page ring per CTA in KiB; 0 = as large as fits   */
   RAZOR_OPT_DECODE_CONSUMER_WARPS = 4,  /* streaming warps per CTA: 0 = default; 4, 8, 12 or 16; a value
                                            the head shape has no kernel for falls back to the default     */
-  RAZOR_OPT_DECODE_TENSOR_CORES = 5,    /* bf16 grouped-query heads: 0 = matrix instructions from group 4
-                                           up (default), 1 = from group 2 up, 2 = never                   */
+  RAZOR_OPT_DECODE_TENSOR_CORES = 5,    /* bf16 heads: 0 = matrix instructions from group 4 up (default),
+                                           1 = for every group size (a single head fills one row of the
+                                           tile), 2 = never                                               */
   RAZOR_OPT_DECODE_STATIC_PERCENT = 6   /* share of the pages handed out as per-CTA spans (0..100;
                                            default 80); 0 makes every job a tail item                     */
 };

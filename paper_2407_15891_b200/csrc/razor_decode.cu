@@ -396,7 +396,7 @@ struct LaneVec<64> {
 template <typename T, int D, int G, int NC, bool MMA>
 __global__ void __launch_bounds__((NC + 2) * 32, 1)
 decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, float* __restrict__ out, int n_stages) {
-  static_assert(!MMA || (sizeof(T) == 2 && G >= 2), "the tensor-core path is for grouped bf16 heads");
+  static_assert(!MMA || sizeof(T) == 2, "the tensor-core path is for bf16 heads");
   using Geo = RowGeom<T, D>;
   constexpr int LPR = Geo::kLpr, EPL = Geo::kEpl;
   constexpr uint32_t PB = Geo::kPageBytes;
@@ -1034,6 +1034,7 @@ cudaError_t decode_nc(const DeviceView& dv, int layer, const DecodeJobs& jb, con
     }
   }
   if constexpr (sizeof(T) == 2 && G == 1) {
+    if (tune.tensor_cores == 1) return decode_launch<T, D, G, 8, true>(dv, layer, jb, q, out, n_sms, tune, s);
     if (nc == 8) return decode_launch<T, D, G, 8, false>(dv, layer, jb, q, out, n_sms, tune, s);
     if (nc == 16) return decode_launch<T, D, G, 16, false>(dv, layer, jb, q, out, n_sms, tune, s);
     return decode_launch<T, D, G, 12, false>(dv, layer, jb, q, out, n_sms, tune, s);

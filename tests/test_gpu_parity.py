@@ -121,6 +121,7 @@ def test_small_shape_sweep(dtype, D, group):
 
 @pytest.mark.parametrize("group,options", [
     (2, {rz.OPT_DECODE_TENSOR_CORES: 1}),                                   # matrix instructions from group 2
+    (1, {rz.OPT_DECODE_TENSOR_CORES: 1}),                                   # ... and for single heads (one row of the tile)
     (2, {rz.OPT_DECODE_TENSOR_CORES: 1, rz.OPT_DECODE_CONSUMER_WARPS: 4}),
     (4, {rz.OPT_DECODE_TENSOR_CORES: 2}),                                   # grouped heads on the CUDA cores
     (4, {rz.OPT_DECODE_CONSUMER_WARPS: 4, rz.OPT_DECODE_TAIL_ITEMS_PER_SM: 64, rz.OPT_DECODE_MIN_CHUNK_PAGES: 1}),
