@@ -149,7 +149,7 @@ __device__ __forceinline__ void tma_load_tile(uint8_t* tile, const CUtensorMap* 
   for (int h = 0; h < D / 64; ++h) tma_load_box(tile + h * kHalfTileBytes, map, h * 64, row0, head, bar);
 }
 
-// grid = (query tiles, heads), block = kScoreThreads.  Writes lse[head][m], the log2 of the causal softmax
+// grid = (heads, query tiles), block = kScoreThreads.  Writes lse[head][m], the log2 of the causal softmax
 // denominator of query m (scaled logits in the log2 domain); *fault is set when a wait gave up.
 template <int D>
 __global__ void __launch_bounds__(kScoreThreads, 2)
@@ -162,8 +162,10 @@ __global__ void __launch_bounds__(kScoreThreads, 2)
   uint8_t* ktile = base + TB;
   ScoreCtl* ctl = (ScoreCtl*)(base + (1 + kStages) * TB);
 
-  const int head = blockIdx.y, n_tiles = gridDim.x;
-  const int tile = n_tiles - 1 - (int)blockIdx.x;   // the long rows of the triangle first
+  // Heads vary fastest in the launch order: the longest row of the triangle of every head first, then the next
+  // one of every head, so that the grid ends on the short rows.
+  const int head = blockIdx.x, n_tiles = gridDim.y;
+  const int tile = n_tiles - 1 - (int)blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int q0 = tile * kQTile;
   if (q0 + kQTile <= period) return;   // none of these queries has an earlier copy of its token
@@ -431,7 +433,7 @@ cudaError_t run_head_scores(const void* Q, const void* K, int n_heads, int n_tok
   if (e != cudaSuccess) return e;
   e = cudaMemsetAsync(fault, 0, sizeof(int), s);
   if (e != cudaSuccess) return e;
-  head_lse_kernel<D><<<dim3(tiles, n_heads), kScoreThreads, score_smem_bytes<D>(), s>>>(map_q, map_k, n_tokens, period,
+  head_lse_kernel<D><<<dim3(n_heads, tiles), kScoreThreads, score_smem_bytes<D>(), s>>>(map_q, map_k, n_tokens, period,
                                                                                         scale_log2, lse, fault);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
@@ -470,6 +472,7 @@ extern "C" int razor_head_scores(const void* Q, const void* K, int32_t n_heads, 
   using namespace razor;
   if (!Q || !K || !echo || !induction || !scratch) return RAZOR_E_NULL_PTR;
   if (n_heads < 1 || n_heads > 65535 || n_tokens < 2 || period < 2 || period >= n_tokens) return RAZOR_E_INVALID_ARG;
+  if (n_tokens > 65535 * razor::kQTile) return RAZOR_E_CAPACITY;   // query tiles are a grid y dimension
   if (!(sm_scale >= 0.f)) return RAZOR_E_INVALID_ARG;
   if (dtype != RAZOR_BF16 || (head_dim != 64 && head_dim != 128)) return RAZOR_E_UNSUPPORTED_DIM;
   if (((uintptr_t)Q | (uintptr_t)K | (uintptr_t)scratch) & 15) return RAZOR_E_MISALIGNED;
