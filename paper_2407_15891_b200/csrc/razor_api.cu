@@ -136,6 +136,9 @@ struct razor_cache {
   size_t plan_bytes = 0;
   cudaEvent_t plan_done[kPlanSlots] = {};
   int plan_next = 0;
+  // Layer whose pages, state or sums the last kernel launched for this cache wrote (-1: it wrote none, a decode).
+  // An append of another layer may read before it waits for that kernel.
+  int last_writer_layer = -1;
 };
 
 extern "C" {
@@ -452,6 +455,7 @@ int compress_impl(razor_cache* c, int layer, const std::vector<SeqIn>& seqs, con
   long long slices = ceil_div((long long)c->n_sms * 24, heads_in_call);
   slices = std::max(1LL, std::min({slices, (long long)kCompressMaxSlices, room, (long long)std::max(1, n_max / 64)}));
   RZ_CUDA(launch_compress(c->dv, cfg.dtype, layer, (int)seqs.size(), (int)slices, n_plan, stream));
+  c->last_writer_layer = layer;
   return RAZOR_OK;
 }
 
@@ -556,7 +560,9 @@ int razor_append(razor_cache_t* c, int32_t layer, const void* k_new, const void*
   if (((uintptr_t)k_new | (uintptr_t)v_new) & 15) return RAZOR_E_MISALIGNED;
   LayerHost& L = c->layers[layer];
   if (L.appended >= c->cfg.max_new_tokens) return RAZOR_E_CAPACITY;
-  RZ_CUDA(launch_append(c->dv, c->cfg.dtype, layer, k_new, v_new, (cudaStream_t)stream));
+  const int early_reads = c->last_writer_layer != layer;
+  RZ_CUDA(launch_append(c->dv, c->cfg.dtype, layer, k_new, v_new, early_reads, (cudaStream_t)stream));
+  c->last_writer_layer = layer;
   // Host mirror of the kernel's state update.
   const int n_sink = c->cfg.n_sink;
   for (HeadState& h : L.hs) {
@@ -593,6 +599,7 @@ int razor_append_many(razor_cache_t* c, int32_t layer, const void* k_new, const 
                                            (long long)(n_tokens / 32)}));
   }
   RZ_CUDA(launch_append_many(c->dv, c->cfg.dtype, layer, k_new, v_new, n_tokens, slices, (cudaStream_t)stream));
+  c->last_writer_layer = layer;
   const int n_sink = c->cfg.n_sink;
   for (HeadState& h : L.hs) h = state_after_run(h, n_sink, n_tokens);   // host mirror of the kernels' state update
   L.appended += n_tokens;
@@ -669,6 +676,7 @@ static int decode_impl(razor_cache_t* c, int32_t layer, const void* q, float* ou
   const DecodeJobs jb{L.n_items, L.n_jobs, L.n_spans, L.jobs[L.n_spans], L.n_multi, n_tokens, tok_stride, q_after};
   RZ_CUDA(launch_decode(c->dv, c->cfg.dtype, layer, jb, q, out, c->n_sms, c->tune,
                         (cudaStream_t)stream));
+  c->last_writer_layer = -1;
   return RAZOR_OK;
 }
 

@@ -211,17 +211,20 @@ __global__ void compress_finalize_kernel(DeviceView dv, int layer, int n_slices)
 // recomputed (Eq. 4 over every token dropped so far) and the new row takes that slot.
 template <typename T, int D>
 __global__ void __launch_bounds__(128) append_kernel(DeviceView dv, int layer, const T* __restrict__ k_new,
-                                                     const T* __restrict__ v_new) {
+                                                     const T* __restrict__ v_new, int early_reads) {
   using Geo = RowGeom<T, D>;
   constexpr int LPR = Geo::kLpr, EPL = Geo::kEpl;
   const int lane = threadIdx.x & 31;
   const int head = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  cudaGridDependencySynchronize();             // launched as a programmatic dependent of the kernel before it
-  cudaTriggerProgrammaticLaunchCompletion();   // the decode kernel queued behind the append may set itself up
-  if (head >= dv.n_heads) return;
-  const size_t hs = (size_t)layer * dv.n_heads + head;
+  // Launched as a programmatic dependent of the kernel before it.  Everything this kernel READS belongs to
+  // its own layer and was last written by that layer's compression or previous append; unless that append
+  // is the kernel directly before this one (early_reads = 0), those writes are complete, so the reads and
+  // the arithmetic may run while the kernel before (another layer's decode or combine) is still finishing.
+  // The WRITES wait for it in every case, which also keeps completion in stream order.
+  if (!early_reads) cudaGridDependencySynchronize();
+  const bool active = head < dv.n_heads;
+  const size_t hs = (size_t)layer * dv.n_heads + (active ? head : 0);
   HeadState st = dv.state[hs];
-  __syncwarp();
   const int n_sink = dv.n_sink;
   const bool keeps_all = st.window < 0;
 
@@ -240,10 +243,13 @@ __global__ void __launch_bounds__(128) append_kernel(DeviceView dv, int layer, c
     st.ring_head = (st.ring_head + 1 == st.window) ? 0 : st.ring_head + 1;
   }
 
-  if (lane < LPR) {
-    const uint4 kf = ((const uint4*)(k_new + (size_t)head * D))[lane];
-    const uint4 vf = ((const uint4*)(v_new + (size_t)head * D))[lane];
-    uint4* krow = nullptr;
+  const bool row_lane = active && lane < LPR;
+  uint4 kf = make_uint4(0u, 0u, 0u, 0u), vf = kf;
+  uint4* krow = nullptr;
+  float new_sum[2][EPL], new_mean[2][EPL];
+  if (row_lane) {
+    kf = ((const uint4*)(k_new + (size_t)head * D))[lane];
+    vf = ((const uint4*)(v_new + (size_t)head * D))[lane];
     if (slot >= 0) {
       const size_t page = (size_t)dv.page_table[hs * dv.max_pages + (slot >> 4)];
       krow = (uint4*)(dv.pool + page * dv.page_bytes + (size_t)(slot & 15) * Geo::kRowBytes) + swz(slot, lane);
@@ -254,16 +260,29 @@ __global__ void __launch_bounds__(128) append_kernel(DeviceView dv, int layer, c
       float a[EPL], b[EPL];
       Elem<T>::unpack(ok, a);
       Elem<T>::unpack(ov, b);
-      float* sum = dv.comp_sum + hs * 2 * D + lane * EPL;
-      float* mean = dv.comp_mean + hs * 2 * D + lane * EPL;
+      const float* sum = dv.comp_sum + hs * 2 * D + lane * EPL;
       const float cnt = (float)st.n_drop;
 #pragma unroll
       for (int i = 0; i < EPL; ++i) {
-        const float sk = sum[i] + a[i], sv = sum[D + i] + b[i];
-        sum[i] = sk;
-        sum[D + i] = sv;
-        mean[i] = __fdiv_rn(sk, cnt);
-        mean[D + i] = __fdiv_rn(sv, cnt);
+        new_sum[0][i] = sum[i] + a[i];
+        new_sum[1][i] = sum[D + i] + b[i];
+        new_mean[0][i] = __fdiv_rn(new_sum[0][i], cnt);
+        new_mean[1][i] = __fdiv_rn(new_sum[1][i], cnt);
+      }
+    }
+  }
+  if (early_reads) cudaGridDependencySynchronize();
+  cudaTriggerProgrammaticLaunchCompletion();   // the decode kernel queued behind the append may set itself up
+  if (row_lane) {
+    if (evict || fold_new) {
+      float* sum = dv.comp_sum + hs * 2 * D + lane * EPL;
+      float* mean = dv.comp_mean + hs * 2 * D + lane * EPL;
+#pragma unroll
+      for (int i = 0; i < EPL; ++i) {
+        sum[i] = new_sum[0][i];
+        sum[D + i] = new_sum[1][i];
+        mean[i] = new_mean[0][i];
+        mean[D + i] = new_mean[1][i];
       }
     }
     if (slot >= 0) {
@@ -271,8 +290,7 @@ __global__ void __launch_bounds__(128) append_kernel(DeviceView dv, int layer, c
       krow[kPageTokens * LPR] = vf;
     }
   }
-  __syncwarp();
-  if (lane == 0) dv.state[hs] = st;
+  if (active && lane == 0) dv.state[hs] = st;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -521,18 +539,21 @@ cudaError_t launch_compress(const DeviceView& dv, int dtype, int layer, int n_se
 }
 
 template <typename T, int D>
-static cudaError_t append_t(const DeviceView& dv, int layer, const void* k, const void* v, cudaStream_t s) {
+static cudaError_t append_t(const DeviceView& dv, int layer, const void* k, const void* v, int early_reads,
+                            cudaStream_t s) {
   const int warps = 4;
   return launch_dependent(append_kernel<T, D>, (dv.n_heads + warps - 1) / warps, warps * 32, s, dv, layer, (const T*)k,
-                          (const T*)v);
+                          (const T*)v, early_reads);
 }
 
-cudaError_t launch_append(const DeviceView& dv, int dtype, int layer, const void* k, const void* v, cudaStream_t s) {
+cudaError_t launch_append(const DeviceView& dv, int dtype, int layer, const void* k, const void* v, int early_reads,
+                          cudaStream_t s) {
   if (dtype == RAZOR_BF16) {
-    return dv.head_dim == 128 ? append_t<__nv_bfloat16, 128>(dv, layer, k, v, s)
-                              : append_t<__nv_bfloat16, 64>(dv, layer, k, v, s);
+    return dv.head_dim == 128 ? append_t<__nv_bfloat16, 128>(dv, layer, k, v, early_reads, s)
+                              : append_t<__nv_bfloat16, 64>(dv, layer, k, v, early_reads, s);
   }
-  return dv.head_dim == 128 ? append_t<float, 128>(dv, layer, k, v, s) : append_t<float, 64>(dv, layer, k, v, s);
+  return dv.head_dim == 128 ? append_t<float, 128>(dv, layer, k, v, early_reads, s)
+                            : append_t<float, 64>(dv, layer, k, v, early_reads, s);
 }
 
 template <typename T, int D>

@@ -172,8 +172,10 @@ struct DecodeTuning {
 // n_plan: entries of dv.plan to apply (state and page-table rows) before the rows are streamed.
 cudaError_t launch_compress(const DeviceView& dv, int dtype, int layer, int n_seqs, int n_slices, int n_plan,
                             cudaStream_t stream);
+// early_reads: the last kernel the library launched that WROTE this layer's pages, state or sums is not the one
+// directly before this append in the stream, so the append may read before it waits for that kernel.
 cudaError_t launch_append(const DeviceView& dv, int dtype, int layer, const void* k_new, const void* v_new,
-                          cudaStream_t stream);
+                          int early_reads, cudaStream_t stream);
 // n_slices > 0: the run is long, use the kernel that is parallel over the tokens with that many slices per
 // head (n_heads * n_slices slice sums must fit the compression scratch); 0: one warp per head, token by token.
 cudaError_t launch_append_many(const DeviceView& dv, int dtype, int layer, const void* k_new, const void* v_new,
