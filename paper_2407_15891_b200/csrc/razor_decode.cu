@@ -454,9 +454,9 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
     }
   };
   // The spans are handed out by CTA index and the queue counts tail jobs only, so the producer can look
-  // up its span, the span's first item and that item's first page ids right here: the schedule and the
-  // page table are written by host copies only, never by a kernel, and may be read before the
-  // dependency below is resolved.
+  // up its span, the span's first item and that item's first page ids right here: the schedule is written
+  // by host copies only and the page table by host copies or the compression's plan kernel, which lies
+  // whole kernels back in the stream, so both may be read before the dependency below is resolved.
   int it0 = n_items, job_end0 = n_items;
   WorkItem w0 = no_item;
   int32_t pid0 = 0;
