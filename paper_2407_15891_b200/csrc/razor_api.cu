@@ -448,12 +448,15 @@ int compress_impl(razor_cache* c, int layer, const std::vector<SeqIn>& seqs, con
   L.appended = 0;
   L.sched_valid = false;
 
-  // Slices per head: about 24 CTAs per SM in all (eight rounds of the three a SM holds), slices no shorter
-  // than 64 rows, and no more slice sums than the scratch has room for.
+  // Slices per head: about 48 CTAs per SM in all (sixteen rounds of the three a SM holds: short CTAs keep the
+  // end of the grid even, whichever heads come last), slices no shorter than 512 rows where the context allows
+  // (a CTA that streams less pays more for its start than it evens out) and never shorter than 64, and no more
+  // slice sums than the scratch has room for.
   const long long heads_in_call = (long long)seqs.size() * H;
   const long long room = ((long long)kCompressSliceBudget + c->dv.n_heads) / heads_in_call;
-  long long slices = ceil_div((long long)c->n_sms * 24, heads_in_call);
-  slices = std::max(1LL, std::min({slices, (long long)kCompressMaxSlices, room, (long long)std::max(1, n_max / 64)}));
+  long long slices = ceil_div((long long)c->n_sms * 48, heads_in_call);
+  const long long by_rows = n_max >= 8 * 512 ? n_max / 512 : std::max(1, n_max / 64);
+  slices = std::max(1LL, std::min({slices, (long long)kCompressMaxSlices, room, by_rows}));
   RZ_CUDA(launch_compress(c->dv, cfg.dtype, layer, (int)seqs.size(), (int)slices, n_plan, stream));
   c->last_writer_layer = layer;
   return RAZOR_OK;
