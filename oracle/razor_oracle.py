@@ -21,7 +21,9 @@ Readings taken where the paper is silent (each is also a pinned test):
     token leaving the window joins the dropped set, so the state after t appended
     tokens is, by definition, the compression of the (N + t)-token context;
   * grouped-query attention: a KV head is kept in full when any query head of its
-    group is a retrieval head (Section 4.1 on Llama-3-8B).
+    group is a retrieval head (Section 4.1 on Llama-3-8B);
+  * a head that holds no token at all (an empty sequence before its first append) has
+    nothing to attend to: both sums of Eq. 5 are empty and the output is defined as zeros.
 
 Parity pins: every function below is pinned by tests/test_oracle_pins.py (brute
 force, closed forms, library special cases, the paper's 3.125x figure); none is
@@ -108,6 +110,8 @@ def compensated_attention(q: np.ndarray, K_kept: np.ndarray, V_kept: np.ndarray,
     q = np.asarray(q, dtype=np.float64)
     K_kept = np.asarray(K_kept, dtype=np.float64)
     V_kept = np.asarray(V_kept, dtype=np.float64)
+    if K_kept.shape[0] == 0 and n_d == 0:
+        return np.zeros(V_kept.shape[1])         # nothing to attend to: both sums of Eq. 5 are empty (reading: zeros)
     s = scale * (K_kept @ q)
     if n_d > 0:
         s_c = scale * float(np.dot(q, np.asarray(k_hat, dtype=np.float64)))

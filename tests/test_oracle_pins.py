@@ -495,3 +495,21 @@ def test_selection_takes_top_induction_and_top_echo_heads():
     assert orc.select_retrieval_heads(np.zeros(8), np.arange(8.0)).sum() == 2    # round(1.12)=1 by induction, 1 by echo (head 0)
     g = _golden()
     assert g["induction_head_fraction"] == 0.14 and g["echo_head_fraction"] == 0.01
+
+
+def test_attention_over_no_tokens_is_defined_as_zeros():
+    """Eq. 5 with an empty kept set and nothing dropped: numerator and denominator are empty sums.  A scalar-loop
+    evaluation gives num = 0 and den = 0; the reading taken is out = num (zeros), never 0/0."""
+    D = 8
+    q = np.arange(D, dtype=np.float64)
+    num, den = np.zeros(D), 0.0
+    for _ in range(0):                                   # the sums of Eq. 5 over zero kept tokens
+        pass
+    assert den == 0.0
+    hc = orc.compress_head(np.zeros((0, D)), np.zeros((0, D)), 0, 4, 16, False)
+    assert len(hc.kept_pos) == 0 and hc.n_drop == 0
+    out = orc.decode_head(q, hc, 0.5)
+    assert out.shape == (D,) and (out == num).all()
+    # one token: attention returns that token's value, whatever the logit
+    K1, V1 = np.ones((1, D)), np.arange(D, dtype=np.float64)[None] * 3.0
+    assert np.allclose(orc.decode_head(q, orc.compress_head(K1, V1, 1, 4, 16, False), 0.5), V1[0])
