@@ -131,6 +131,12 @@ RAZOR_API int razor_compress_seq(razor_cache_t* cache, int32_t layer, int32_t b,
  * that slot; the window length stays what it was at compression (the paper does not say how the
  * cache grows while decoding).  Hence t appends leave exactly the state that compressing the
  * (N + t)-token context with the same window would.
+ * Ordering: the kernel is launched so that it may start while the kernel before it on the stream is
+ * still finishing.  In that early phase it reads only the library's own state of this layer (written
+ * by earlier razor calls on the same stream).  k_new and v_new are read, and everything is written,
+ * only after the preceding kernel has completed and its writes are visible, so the kernel that produces
+ * k_new / v_new may be the one directly before this call.  None of the caller's memory is ever read
+ * before the preceding kernel has finished; the same holds for q of razor_decode_attention.
  * Errors: NULL_PTR, INVALID_ARG, NOT_COMPRESSED, CAPACITY (more than max_new_tokens appends), CUDA.
  */
 RAZOR_API int razor_append(razor_cache_t* cache, int32_t layer, const void* k_new, const void* v_new, void* stream);
@@ -141,7 +147,8 @@ RAZOR_API int razor_append(razor_cache_t* cache, int32_t layer, const void* k_ne
  * Query head j reads KV head j / group.  For a head with N_d > 0 dropped tokens
  *   out = (N_d e^{s_c} v_hat + sum_kept e^{s_n} v_n) / (N_d e^{s_c} + sum_kept e^{s_n}),
  *   s_n = sm_scale q.k_n,  s_c = sm_scale q.k_hat;
- * other heads get softmax attention over all their tokens.  A sequence with no tokens gives zeros.
+ * other heads get softmax attention over all their tokens.  A sequence with no tokens gives zeros
+ * (both sums are empty).
  * Call razor_append first when the query token should attend to itself.
  * Errors: NULL_PTR, INVALID_ARG, NOT_COMPRESSED, CUDA.
  */

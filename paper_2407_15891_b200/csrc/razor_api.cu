@@ -20,8 +20,7 @@ thread_local int g_last_cuda_error = 0;
   do {                                         \
     cudaError_t e__ = (call);                  \
     if (e__ != cudaSuccess) {                  \
-      g_last_cuda_error = (int)e__;            \
-      (void)cudaGetLastError();                \
+      razor::note_cuda_error(e__);             \
       return RAZOR_E_CUDA;                     \
     }                                          \
   } while (0)
@@ -118,6 +117,11 @@ uint64_t mix64(uint64_t x) {
 }
 
 }  // namespace
+
+void razor::note_cuda_error(cudaError_t e) {
+  g_last_cuda_error = (int)e;
+  (void)cudaGetLastError();
+}
 
 struct razor_cache {
   razor_config_t cfg;
@@ -250,12 +254,11 @@ int razor_cache_create(razor_cache_t** out, const razor_config_t* cfg, void* poo
   if (e == cudaSuccess)
     e = cudaHostAlloc((void**)&c->pinned_plan, (size_t)kPlanSlots * c->plan_bytes, cudaHostAllocDefault);
   if (e != cudaSuccess) {
-    g_last_cuda_error = (int)e;
-    (void)cudaGetLastError();
+    note_cuda_error(e);
     if (c->pinned_items) cudaFreeHost(c->pinned_items);
     if (c->pinned_jobs) cudaFreeHost(c->pinned_jobs);
     if (c->pinned_multi) cudaFreeHost(c->pinned_multi);
-  if (c->pinned_plan) cudaFreeHost(c->pinned_plan);
+    if (c->pinned_plan) cudaFreeHost(c->pinned_plan);
     delete c;
     return RAZOR_E_CUDA;
   }
@@ -375,12 +378,25 @@ int compress_impl(razor_cache* c, int layer, const std::vector<SeqIn>& seqs, con
       next += pages;
     }
   }
-  c->next_page = next;
+  // Nothing of the host mirror (page cursor, regions, head states, "compressed" marks) is touched until every
+  // CUDA call of this function has succeeded: after a failure the layer is left as it was, so a later call
+  // cannot run on lengths the device never received.
+  std::vector<HeadState> new_hs(seqs.size() * (size_t)H);
+  std::vector<long long> region_start(seqs.size());
+  // Once something has been enqueued the device copy of these sequences may have changed (page-table rows, the
+  // plan): after a failure from there on they count as not compressed until a compression of them succeeds.
+  auto fail_enqueued = [&](cudaError_t e) {
+    for (const SeqIn& s : seqs)
+      if (L.seq_done[s.b]) { L.seq_done[s.b] = 0; L.n_done -= 1; }
+    L.sched_valid = false;
+    note_cuda_error(e);
+    return (int)RAZOR_E_CUDA;
+  };
+  cudaError_t ce;
 
   // The plan goes to the device in one copy from pinned memory: per head its state after the call and the
   // run of pool pages behind its page-table row (compress_plan_kernel writes both), then the sequences.
   const int slot = c->plan_next;
-  c->plan_next = (slot + 1) % kPlanSlots;
   if (c->plan_done[slot]) RZ_CUDA(cudaEventSynchronize(c->plan_done[slot]));   // its last upload has left the slot
   uint8_t* staging = c->pinned_plan + (size_t)slot * c->plan_bytes;
   HeadPlan* plan = (HeadPlan*)staging;
@@ -389,15 +405,12 @@ int compress_impl(razor_cache* c, int layer, const std::vector<SeqIn>& seqs, con
   std::vector<int32_t> rows;   // only for permuted page ids
   for (size_t i = 0; i < seqs.size(); ++i) {
     const SeqIn& s = seqs[i];
-    if (new_start[i] >= 0) {
-      L.region_start[s.b] = new_start[i];
-      L.region_count[s.b] = need[i];
-    }
+    region_start[i] = new_start[i] >= 0 ? new_start[i] : L.region_start[s.b];
     const bool shuffled = cfg.page_shuffle_seed != 0;
     std::vector<int32_t> ids;
     if (shuffled) {   // page ids of the region, permuted: the rows are written from the host
       ids.resize((size_t)need[i]);
-      for (long long k = 0; k < need[i]; ++k) ids[(size_t)k] = (int32_t)(L.region_start[s.b] + k);
+      for (long long k = 0; k < need[i]; ++k) ids[(size_t)k] = (int32_t)(region_start[i] + k);
       uint64_t st = mix64((uint64_t)cfg.page_shuffle_seed * 1315423911ull + (uint64_t)layer * 2654435761ull + s.b);
       for (long long k = need[i] - 1; k > 0; --k) {
         st = mix64(st);
@@ -416,10 +429,10 @@ int compress_impl(razor_cache* c, int layer, const std::vector<SeqIn>& seqs, con
       h.n_drop = keep_all ? 0 : s.n_ctx - cfg.n_sink - wg;
       h.ring_head = 0;
       h.window = r ? -1 : wg;
-      L.hs[(size_t)s.b * H + g] = h;
+      new_hs[i * (size_t)H + g] = h;
       HeadPlan& pl = plan[n_plan++];
       pl.head = s.b * H + g;
-      pl.first_page = (int32_t)(L.region_start[s.b] + cursor);
+      pl.first_page = (int32_t)(region_start[i] + cursor);
       pl.n_pages = shuffled ? 0 : cap_pages;
       pl.len = h.len;
       pl.n_drop = h.n_drop;
@@ -430,23 +443,23 @@ int compress_impl(razor_cache* c, int layer, const std::vector<SeqIn>& seqs, con
     }
     if (shuffled) {
       const size_t head0 = (size_t)layer * c->dv.n_heads + (size_t)s.b * H;
-      RZ_CUDA(cudaMemcpyAsync(c->dv.page_table + head0 * c->lay.max_pages, rows.data(), rows.size() * sizeof(int32_t),
-                              cudaMemcpyHostToDevice, stream));   // pageable source: staged before the call returns
+      ce = cudaMemcpyAsync(c->dv.page_table + head0 * c->lay.max_pages, rows.data(), rows.size() * sizeof(int32_t),
+                           cudaMemcpyHostToDevice, stream);   // pageable source: staged before the call returns
+      if (ce != cudaSuccess) return fail_enqueued(ce);
     }
     SeqDesc d;
     d.K = s.K; d.V = s.V; d.stride_h = s.stride_h; d.stride_n = s.stride_n;
     d.n_ctx = s.n_ctx; d.window = s.window; d.b = s.b; d.pad = 0;
     descs[i] = d;
-    if (!L.seq_done[s.b]) { L.seq_done[s.b] = 1; L.n_done += 1; }
   }
   // one copy covers plan[0 .. n_plan) and, behind the full plan array, the sequence descriptors
-  RZ_CUDA(cudaMemcpyAsync(c->dv.plan, staging, c->plan_bytes, cudaMemcpyHostToDevice, stream));
-  if (!c->plan_done[slot]) RZ_CUDA(cudaEventCreateWithFlags(&c->plan_done[slot], cudaEventDisableTiming));
-  RZ_CUDA(cudaEventRecord(c->plan_done[slot], stream));
-  L.retr = flags;
-  L.any = true;
-  L.appended = 0;
-  L.sched_valid = false;
+  if (!c->plan_done[slot] &&
+      (ce = cudaEventCreateWithFlags(&c->plan_done[slot], cudaEventDisableTiming)) != cudaSuccess)
+    return fail_enqueued(ce);
+  if ((ce = cudaMemcpyAsync(c->dv.plan, staging, c->plan_bytes, cudaMemcpyHostToDevice, stream)) != cudaSuccess)
+    return fail_enqueued(ce);
+  c->plan_next = (slot + 1) % kPlanSlots;   // the slot is in use from here on, whatever happens next
+  if ((ce = cudaEventRecord(c->plan_done[slot], stream)) != cudaSuccess) return fail_enqueued(ce);
 
   // Slices per head: about 48 CTAs per SM in all (sixteen rounds of the three a SM holds: short CTAs keep the
   // end of the grid even, whichever heads come last), slices no shorter than 512 rows where the context allows
@@ -457,8 +470,24 @@ int compress_impl(razor_cache* c, int layer, const std::vector<SeqIn>& seqs, con
   long long slices = ceil_div((long long)c->n_sms * 48, heads_in_call);
   const long long by_rows = n_max >= 8 * 512 ? n_max / 512 : std::max(1, n_max / 64);
   slices = std::max(1LL, std::min({slices, (long long)kCompressMaxSlices, room, by_rows}));
-  RZ_CUDA(launch_compress(c->dv, cfg.dtype, layer, (int)seqs.size(), (int)slices, n_plan, stream));
   c->last_writer_layer = layer;
+  ce = launch_compress(c->dv, cfg.dtype, layer, (int)seqs.size(), (int)slices, n_plan, stream);
+  if (ce != cudaSuccess) return fail_enqueued(ce);
+  // ---- commit
+  c->next_page = next;
+  for (size_t i = 0; i < seqs.size(); ++i) {
+    const int b = seqs[i].b;
+    if (new_start[i] >= 0) {
+      L.region_start[b] = new_start[i];
+      L.region_count[b] = need[i];
+    }
+    for (int g = 0; g < H; ++g) L.hs[(size_t)b * H + g] = new_hs[i * (size_t)H + g];
+    if (!L.seq_done[b]) { L.seq_done[b] = 1; L.n_done += 1; }
+  }
+  L.retr = flags;
+  L.any = true;
+  L.appended = 0;
+  L.sched_valid = false;
   return RAZOR_OK;
 }
 

@@ -216,11 +216,15 @@ __global__ void __launch_bounds__(128) append_kernel(DeviceView dv, int layer, c
   constexpr int LPR = Geo::kLpr, EPL = Geo::kEpl;
   const int lane = threadIdx.x & 31;
   const int head = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  // Launched as a programmatic dependent of the kernel before it.  Everything this kernel READS belongs to
-  // its own layer and was last written by that layer's compression or previous append; unless that append
-  // is the kernel directly before this one (early_reads = 0), those writes are complete, so the reads and
-  // the arithmetic may run while the kernel before (another layer's decode or combine) is still finishing.
-  // The WRITES wait for it in every case, which also keeps completion in stream order.
+  // Launched as a programmatic dependent of the kernel before it on the stream, which may still be running
+  // when this kernel starts.  Two kinds of memory are read here:
+  //   * the library's own state of this layer (head state, page id, the row about to be evicted, the
+  //     compensation sums), last written by this layer's compression or previous append.  Unless that writer
+  //     is the kernel directly before this one (early_reads = 0) it finished long ago, so these reads and the
+  //     arithmetic on them may run ahead of the dependency wait;
+  //   * the caller's k_new / v_new.  Whatever produced them (in a model: the K/V projection, the kernel
+  //     directly before this one) is not known to the library, so they are read only after the wait.
+  // Every write comes after the wait as well, which keeps completion in stream order.
   if (!early_reads) cudaGridDependencySynchronize();
   const bool active = head < dv.n_heads;
   const size_t hs = (size_t)layer * dv.n_heads + (active ? head : 0);
@@ -244,45 +248,43 @@ __global__ void __launch_bounds__(128) append_kernel(DeviceView dv, int layer, c
   }
 
   const bool row_lane = active && lane < LPR;
-  uint4 kf = make_uint4(0u, 0u, 0u, 0u), vf = kf;
   uint4* krow = nullptr;
-  float new_sum[2][EPL], new_mean[2][EPL];
+  float fold[2][EPL], old_sum[2][EPL];   // the row that joins the dropped set (K, V) and the sums so far
   if (row_lane) {
-    kf = ((const uint4*)(k_new + (size_t)head * D))[lane];
-    vf = ((const uint4*)(v_new + (size_t)head * D))[lane];
     if (slot >= 0) {
       const size_t page = (size_t)dv.page_table[hs * dv.max_pages + (slot >> 4)];
       krow = (uint4*)(dv.pool + page * dv.page_bytes + (size_t)(slot & 15) * Geo::kRowBytes) + swz(slot, lane);
     }
     if (evict || fold_new) {
-      const uint4 ok = evict ? krow[0] : kf;
-      const uint4 ov = evict ? krow[kPageTokens * LPR] : vf;
-      float a[EPL], b[EPL];
-      Elem<T>::unpack(ok, a);
-      Elem<T>::unpack(ov, b);
       const float* sum = dv.comp_sum + hs * 2 * D + lane * EPL;
-      const float cnt = (float)st.n_drop;
 #pragma unroll
-      for (int i = 0; i < EPL; ++i) {
-        new_sum[0][i] = sum[i] + a[i];
-        new_sum[1][i] = sum[D + i] + b[i];
-        new_mean[0][i] = __fdiv_rn(new_sum[0][i], cnt);
-        new_mean[1][i] = __fdiv_rn(new_sum[1][i], cnt);
-      }
+      for (int i = 0; i < EPL; ++i) { old_sum[0][i] = sum[i]; old_sum[1][i] = sum[D + i]; }
+    }
+    if (evict) {
+      Elem<T>::unpack(krow[0], fold[0]);
+      Elem<T>::unpack(krow[kPageTokens * LPR], fold[1]);
     }
   }
   if (early_reads) cudaGridDependencySynchronize();
   cudaTriggerProgrammaticLaunchCompletion();   // the decode kernel queued behind the append may set itself up
   if (row_lane) {
+    const uint4 kf = ((const uint4*)(k_new + (size_t)head * D))[lane];
+    const uint4 vf = ((const uint4*)(v_new + (size_t)head * D))[lane];
+    if (fold_new) {
+      Elem<T>::unpack(kf, fold[0]);
+      Elem<T>::unpack(vf, fold[1]);
+    }
     if (evict || fold_new) {
       float* sum = dv.comp_sum + hs * 2 * D + lane * EPL;
       float* mean = dv.comp_mean + hs * 2 * D + lane * EPL;
+      const float cnt = (float)st.n_drop;
 #pragma unroll
       for (int i = 0; i < EPL; ++i) {
-        sum[i] = new_sum[0][i];
-        sum[D + i] = new_sum[1][i];
-        mean[i] = new_mean[0][i];
-        mean[D + i] = new_mean[1][i];
+        const float sk = old_sum[0][i] + fold[0][i], sv = old_sum[1][i] + fold[1][i];
+        sum[i] = sk;
+        sum[D + i] = sv;
+        mean[i] = __fdiv_rn(sk, cnt);
+        mean[D + i] = __fdiv_rn(sv, cnt);
       }
     }
     if (slot >= 0) {
@@ -493,8 +495,9 @@ __global__ void __launch_bounds__(256) export_kernel(DeviceView dv, int layer, i
 
 // ---------------------------------------------------------------------------------------------
 // Launch as a programmatic dependent of the preceding kernel on the stream: the launch latency and the
-// kernel's first instructions overlap that kernel's tail; the kernel itself waits at
-// cudaGridDependencySynchronize() before it touches memory.
+// kernel's first instructions overlap that kernel's tail.  Before its cudaGridDependencySynchronize() such a
+// kernel touches at most memory that the library itself wrote whole kernels earlier; the caller's buffers
+// are read, and everything is written, only after that wait.
 template <typename... KArgs, typename... Args>
 static cudaError_t launch_dependent(void (*kernel)(KArgs...), int grid, int block, cudaStream_t s, Args... args) {
   cudaLaunchConfig_t cfg = {};

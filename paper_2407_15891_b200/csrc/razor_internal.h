@@ -168,6 +168,10 @@ struct DecodeTuning {
   int32_t tensor_cores;     // grouped bf16 heads: 0 auto (group >= 4), 1 on (group >= 2), 2 off
 };
 
+// Records the code razor_last_cuda_error() reports (per thread) and clears the runtime's sticky-free error state.
+// Every entry point that returns RAZOR_E_CUDA goes through it, whichever source file it lives in.
+void note_cuda_error(cudaError_t e);
+
 // Kernel launchers (defined in the .cu files).  Each returns the cudaError_t of the launch.
 // n_plan: entries of dv.plan to apply (state and page-table rows) before the rows are streamed.
 cudaError_t launch_compress(const DeviceView& dv, int dtype, int layer, int n_seqs, int n_slices, int n_plan,

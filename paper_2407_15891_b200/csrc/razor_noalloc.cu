@@ -89,7 +89,9 @@ cudaError_t run_static(const void* K, const void* V, int64_t stride_h, int64_t s
 }
 
 // Device address of the scratch array, looked up once per device (the array's name is only a
-// host-side handle in host code; kernels must be given the address the runtime reports).
+// host-side handle in host code; kernels must be given the address the runtime reports).  The address
+// is remembered per device ordinal for the life of the process: it assumes the device's primary context
+// is not destroyed (cudaDeviceReset) while the library stays loaded.
 cudaError_t scratch_address(float** out) {
   static float* cached[64] = {};
   int dev = 0;
@@ -142,7 +144,7 @@ extern "C" int razor_compensation_mean_static(const void* K, const void* V, int6
                           : run_static<float, 64>(K, V, stride_h, stride_n, n_kv_heads, first, last, scratch, mean_k, mean_v, s);
   }
   if (e != cudaSuccess) {
-    (void)cudaGetLastError();
+    note_cuda_error(e);   // razor_last_cuda_error() reports it
     return RAZOR_E_CUDA;
   }
   if (n_drop) *n_drop = last - first;

@@ -489,7 +489,7 @@ extern "C" int razor_head_scores(const void* Q, const void* K, int32_t n_heads, 
       head_dim == 128 ? run_head_scores<128>(Q, K, n_heads, n_tokens, period, scale_log2, echo, induction, partial, lse, fault, s)
                       : run_head_scores<64>(Q, K, n_heads, n_tokens, period, scale_log2, echo, induction, partial, lse, fault, s);
   if (e != cudaSuccess) {
-    (void)cudaGetLastError();
+    razor::note_cuda_error(e);   // razor_last_cuda_error() reports it
     return RAZOR_E_CUDA;
   }
   return RAZOR_OK;
