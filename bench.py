@@ -39,6 +39,29 @@ FALLBACK_HBM_GBS = 6650.0       # used only when MEASURED_PEAKS.json is absent
 DECODE_TRAFFIC_PER_ALG_BYTE = 1.008
 
 
+# ---------------------------------------------------------------------------------------------- byte accounting
+def kept_tokens(w, layer: int, extra: int = 0) -> int:
+    """Tokens the compressed cache of one layer holds, summed over (sequence, KV head), after `extra` appended
+    tokens: a retrieval head holds its whole context, any other head at most n_sink + window tokens."""
+    r = w.retrieval(layer)
+    n_retr, n_other = int(r.sum()), int((1 - r).sum())
+    tot = 0
+    for b in range(w.batch):
+        n = w.ctx_len[b] + extra
+        tot += n_retr * n + n_other * min(n, w.n_sink + w.window[b])
+    return tot
+
+
+def compressed_bytes(w, layer: int, extra: int = 0) -> int:
+    """Algorithmic bytes of one decode launch: every kept K and V row once."""
+    return kept_tokens(w, layer, extra) * 2 * w.head_dim * w.esz()
+
+
+def dense_bytes(w, extra: int = 0) -> int:
+    """K + V bytes of one layer's uncompressed cache."""
+    return sum(n + extra for n in w.ctx_len) * w.n_kv_heads * 2 * w.head_dim * w.esz()
+
+
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -274,7 +297,7 @@ def decode_only(rz, synth, name, n_layers, dev, peak, reps=60, n_tok=1, alibi=Fa
     b.record()
     torch.cuda.synchronize()
     us = a.elapsed_time(b) * 1e3 / reps
-    kept = w.compressed_bytes(0, extra=n_tok if n_tok > 1 else 0)
+    kept = compressed_bytes(w, 0, extra=n_tok if n_tok > 1 else 0)
     status = cache.device_status()
     cache.close()
     gbs = kept / (us * 1e-6) / 1e9
@@ -463,13 +486,13 @@ def main():
 
     # algorithmic bytes of the pass
     def decode_alg_bytes(l, t):
-        kv = w.compressed_bytes(l, extra=t + 1)
+        kv = compressed_bytes(w, l, extra=t + 1)
         n_nonretr = int((1 - retr[l]).sum()) * w.batch
         small = w.batch * w.n_q_heads * w.head_dim * (w.esz() + 4) + n_nonretr * 2 * w.head_dim * 4
         return kv, kv + small
     attended = sum(decode_alg_bytes(l, t)[0] for l in range(L) for t in range(T))
-    compress_read = w.dense_bytes() * L
-    compress_write = sum(w.compressed_bytes(l) for l in range(L))
+    compress_read = dense_bytes(w) * L
+    compress_write = sum(compressed_bytes(w, l) for l in range(L))
 
     for _ in range(args.warmup):
         one_pass()
@@ -561,7 +584,7 @@ def main():
             b.record()
             torch.cuda.synchronize()
             d_us = a.elapsed_time(b) * 1e3 / reps
-            line["dense_decode"] = {"us_per_layer": d_us, "gbs": w.dense_bytes() / (d_us * 1e-6) / 1e9,
+            line["dense_decode"] = {"us_per_layer": d_us, "gbs": dense_bytes(w) / (d_us * 1e-6) / 1e9,
                                     "us_per_decode_step": d_us * L,
                                     "speedup_compressed_vs_dense": d_us / statistics.mean(dec_us)}
             dcache.close()

@@ -132,11 +132,6 @@ def retrieval_mask(seed: int, layer: int, n_heads: int, n_retrieval: int) -> np.
     return m
 
 
-def buffer_length(n_ctx: int, s0: int = 4000, c: int = 5) -> int:
-    """Recent-window length from the paper's hyper-parameter table: max(S0, N/C), floor division."""
-    return max(s0, n_ctx // c)
-
-
 @dataclass
 class Workload:
     """Shape of one synthetic workload (one of the five configurations)."""
@@ -173,24 +168,8 @@ class Workload:
             return m
         return retrieval_mask(self.seed, layer, self.n_kv_heads, self.n_retrieval_kv)
 
-    def kept_tokens(self, layer: int, extra: int = 0) -> int:
-        """Sum over (b, kv head) of kept tokens after `extra` appended tokens."""
-        r = self.retrieval(layer)
-        tot = 0
-        for b in range(self.batch):
-            n = self.ctx_len[b] + extra
-            short = min(n, self.n_sink + self.window[b])
-            tot += int(r.sum()) * n + int((1 - r).sum()) * short
-        return tot
-
     def esz(self) -> int:
         return 2 if self.dtype == "bf16" else 4
-
-    def compressed_bytes(self, layer: int, extra: int = 0) -> int:
-        return self.kept_tokens(layer, extra) * 2 * self.head_dim * self.esz()
-
-    def dense_bytes(self, extra: int = 0) -> int:
-        return sum(n + extra for n in self.ctx_len) * self.n_kv_heads * 2 * self.head_dim * self.esz()
 
 
 def workload(name: str, scale: float = 1.0) -> Workload:

@@ -9,6 +9,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import razor_oracle as orc
 from paper_2407_15891_b200 import binding as rz
 from paper_2407_15891_b200 import build as rz_build
 from paper_2407_15891_b200 import synth
@@ -74,9 +75,11 @@ def test_pool_size_tracks_the_compressed_bytes_of_the_paper_shaped_configs(name)
                          max(w.ctx_len), 0)
     retr = np.stack([w.retrieval(l) for l in range(w.n_layers)])
     pool, _ = rz.razor_query_bytes(cfg, w.ctx_len, w.window, retr)
-    kept = sum(w.compressed_bytes(l) for l in range(w.n_layers))
+    row = 2 * w.head_dim * w.esz()                # one K row + one V row
+    kept = row * sum(len(orc.kept_positions(n, w.n_sink, win, bool(r)))
+                     for l in range(w.n_layers) for r in w.retrieval(l) for n, win in zip(w.ctx_len, w.window))
     assert kept <= pool < kept * 1.002            # only page rounding on top
-    dense = w.dense_bytes() * w.n_layers
+    dense = row * sum(w.ctx_len) * w.n_kv_heads * w.n_layers
     ratio = dense / kept
     expect = {"cfg2": 3.08, "cfg3": 3.90, "cfg4": 2.91}[name]
     assert abs(ratio - expect) < 0.01
