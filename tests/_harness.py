@@ -94,15 +94,6 @@ def check_head_state(cache: rz.RazorCache, ref: HeadRef, n_sink: int, window: in
     return hc
 
 
-def sample_heads(w: synth.Workload, layer: int, n_retr: int, n_other: int, batches: Sequence[int]) -> List[Tuple[int, int]]:
-    r = w.retrieval(layer)
-    ret = [g for g in range(w.n_kv_heads) if r[g]][:n_retr]
-    oth = [g for g in range(w.n_kv_heads) if not r[g]]
-    step = max(1, len(oth) // max(1, n_other))
-    oth = oth[::step][:n_other]
-    return [(b, g) for b in batches for g in ret + oth]
-
-
 def run_parity(w: synth.Workload, *, layers: Optional[Sequence[int]] = None,
                heads_for: Optional[Dict[int, List[Tuple[int, int]]]] = None, steps: Optional[int] = None,
                shuffle: int = 0, use_comp: int = 1, sm_scale: float = 0.0, per_seq: bool = False,
@@ -202,3 +193,187 @@ def _single_seq_view(w: synth.Workload, b: int) -> synth.Workload:
     wb.window = [w.window[b]]
     wb.seed = w.seed * 131 + b
     return wb
+
+
+# ------------------------------------------------------------------------------------------------------------
+# Full-size parity.  The GPU runs the workload exactly as the benchmark does (compress every layer, then
+# decode steps x layers x (append, decode)) and what it produced is recorded: every output, a snapshot of the
+# checked heads' exported state in the middle of the run, and the live state at the end.  The oracle then
+# replays one group (a layer, or a sequence of the ragged batch) at a time from the regenerated inputs, so
+# that only one group's dense fp64 history is ever held on the host, with the heads of the group spread over
+# a thread pool (the oracle itself stays single-threaded numpy).
+def oracle_threads() -> int:
+    import os
+    try:
+        n = len(os.sched_getaffinity(0))
+    except AttributeError:
+        n = os.cpu_count() or 1
+    return max(1, min(32, n))
+
+
+def export_to_host(cache: rz.RazorCache, l: int, b: int, g: int) -> dict:
+    ex = cache.export(l, b, g)
+    return {k: (v.cpu() if isinstance(v, torch.Tensor) else v) for k, v in ex.items()}
+
+
+def check_export(ex: dict, ref: HeadRef, n_sink: int, window: int, is_retr: bool) -> orc.HeadCache:
+    """Layout (bit-exact) and compensation means (1e-3 relative) of an exported head against the oracle."""
+    hc = orc.compress_head(ref.K, ref.V, ref.n, n_sink, window, is_retr)
+    where = (ref.layer, ref.b, ref.g, ref.n)
+    kept = ex["kept_pos"].cpu().numpy().astype(np.int64)
+    assert kept.shape == hc.kept_pos.shape and (kept == hc.kept_pos).all(), f"kept positions differ at {where}"
+    assert ex["n_drop"] == hc.n_drop, where
+    assert (bits(ex["K"]) == ref.K_bits[hc.kept_pos]).all(), f"K rows not bit-exact at {where}"
+    assert (bits(ex["V"]) == ref.V_bits[hc.kept_pos]).all(), f"V rows not bit-exact at {where}"
+    mk, mv = to_f64(ex["mean_k"]), to_f64(ex["mean_v"])
+    if hc.n_drop > 0:
+        assert rel_inf(mk, hc.k_hat) <= TOL_MEAN_REL, (rel_inf(mk, hc.k_hat), where)
+        assert rel_inf(mv, hc.v_hat) <= TOL_MEAN_REL, (rel_inf(mv, hc.v_hat), where)
+    else:
+        assert not mk.any() and not mv.any(), where
+    return hc
+
+
+def run_parity_recorded(w: synth.Workload, *, heads_for: Dict[int, List[Tuple[int, int]]], steps: int,
+                        per_seq: bool = False, device="cuda:0", options: Optional[Dict[int, int]] = None) -> dict:
+    """heads_for[layer] = [(b, kv head)] to check.  steps >= 1: that many (append, decode) rounds over all
+    layers; steps == 0: one decode straight after compression.  Layout is checked right after compression,
+    after the middle step and after the last one; outputs at every step.  Returns counts and worst errors."""
+    from concurrent.futures import ThreadPoolExecutor
+    from threadpoolctl import threadpool_limits
+
+    dev = torch.device(device)
+    L, G = w.n_layers, w.group
+    scale = 1.0 / math.sqrt(w.head_dim)
+    tol = TOL_OUT[w.dtype]
+    n_rounds = max(steps, 1)
+    mid = (steps // 2 - 1) if steps >= 4 else -1                       # snapshot after this step's appends
+    cache = make_cache(w, max_new=max(steps, 1), device=device, options=options)
+    pool = ThreadPoolExecutor(oracle_threads())
+    res = dict(out=0.0, mean=0.0, heads=0, outputs=0, layouts=0)
+
+    def groups():
+        """(layer, sequences) units whose dense inputs are generated together."""
+        for l in range(L):
+            if per_seq:
+                for b in sorted({b for (b, _) in heads_for.get(l, [])}):
+                    yield l, [b]
+            else:
+                yield l, None
+
+    def dense_of(l, seqs):
+        """Dense K, V [B', Hkv, N, D] on the device and the sequences they belong to."""
+        if seqs is None:
+            K, V = synth.make_dense_kv(w, l, dev)
+            return K, V, list(range(w.batch))
+        K, V = synth.make_dense_kv(_single_seq_view(w, seqs[0]), l, dev)
+        return K, V, seqs
+
+    def build_refs(l, K, V, seqs):
+        todo = [(b, g) for (b, g) in heads_for.get(l, []) if b in seqs]
+        host = {(b, g): (K[seqs.index(b), g].cpu(), V[seqs.index(b), g].cpu()) for (b, g) in todo}
+        make = lambda bg: HeadRef(l, bg[0], bg[1], host[bg][0], host[bg][1], w.ctx_len[bg[0]], steps)
+        return dict(zip(todo, pool.map(make, todo)))
+
+    try:
+        with threadpool_limits(limits=1):
+            # ---- phase 1: compression in the benchmark's order; layout of the checked heads right after it
+            for l in range(L):
+                retr = w.retrieval(l)
+                if per_seq:
+                    for b in range(w.batch):
+                        K, V, seqs = dense_of(l, [b])
+                        cache.compress_seq(l, b, K[0], V[0], w.ctx_len[b], retr, w.window[b])
+                        refs = build_refs(l, K, V, seqs)
+                        exs = {bg: export_to_host(cache, l, *bg) for bg in refs}
+                        list(pool.map(lambda bg: check_export(exs[bg], refs[bg], w.n_sink, w.window[bg[0]], bool(retr[bg[1]])), refs))
+                        res["layouts"] += len(refs)
+                        torch.cuda.synchronize()
+                        del K, V, refs, exs
+                else:
+                    K, V, seqs = dense_of(l, None)
+                    cache.compress(l, K, V, w.ctx_len, retr, w.window)
+                    refs = build_refs(l, K, V, seqs)
+                    exs = {bg: export_to_host(cache, l, *bg) for bg in refs}
+                    list(pool.map(lambda bg: check_export(exs[bg], refs[bg], w.n_sink, w.window[bg[0]], bool(retr[bg[1]])), refs))
+                    res["layouts"] += len(refs)
+                    torch.cuda.synchronize()
+                    del K, V, refs, exs
+            # ---- phase 2: the decode steps, step-major over the layers as the benchmark runs them
+            outs = {}
+            snap = {}
+            for t in range(n_rounds):
+                for l in range(L):
+                    if steps > 0:
+                        k_new, v_new = synth.make_new_kv(w, l, t, dev)
+                        cache.append(l, k_new, v_new)
+                    out = cache.decode(l, synth.make_queries(w, l, t, dev))
+                    if l in heads_for:
+                        outs[(l, t)] = out.cpu()
+                        if t == mid:
+                            for bg in heads_for[l]:
+                                snap[(l,) + bg] = cache.export(l, *bg)          # stays on the device until replayed
+            status = cache.device_status()
+            assert status == 0, f"a bounded wait inside the decode kernel ran out (status bits {status})"
+
+            # ---- phase 3: the oracle replays one group at a time
+            def replay(l, bg, ref, ex_mid, ex_last):
+                b, g = bg
+                is_retr = bool(w.retrieval(l)[g])
+                worst, n_out, n_lay = 0.0, 0, 0
+                for t in range(n_rounds):
+                    if steps > 0:
+                        k_new, v_new = synth.make_new_kv(w, l, t)              # regenerated on the host
+                        ref.append(k_new[b, g], v_new[b, g])
+                    if t == mid:
+                        hc = check_export(ex_mid, ref, w.n_sink, w.window[b], is_retr); n_lay += 1
+                    elif t == n_rounds - 1 and steps > 0:
+                        hc = check_export(ex_last, ref, w.n_sink, w.window[b], is_retr); n_lay += 1
+                    else:
+                        hc = None
+                    q = to_f64(synth.make_queries(w, l, t))
+                    out = to_f64(outs[(l, t)])
+                    for j in range(G):
+                        h = g * G + j
+                        if is_retr and hc is None:       # Algorithm 1: a retrieval head is ordinary attention over every token
+                            expect = orc.full_attention(q[b, h], ref.K[:ref.n], ref.V[:ref.n], scale)
+                        else:
+                            if hc is None:
+                                hc = orc.compress_head(ref.K, ref.V, ref.n, w.n_sink, w.window[b], is_retr)
+                            expect = orc.decode_head(q[b, h], hc, scale)
+                        err = float(np.abs(out[b, h] - expect).max())
+                        assert err <= tol, f"out max-abs {err:.3e} > {tol} at layer {l} b {b} head {h} step {t}"
+                        worst = max(worst, err)
+                        n_out += 1
+                return worst, n_out, n_lay
+
+            for l, seqs in groups():
+                if not heads_for.get(l):
+                    continue
+                K, V, seqs = dense_of(l, seqs)
+                refs = build_refs(l, K, V, seqs)
+                del K, V
+                ex_mid = {bg: {k: (v.cpu() if isinstance(v, torch.Tensor) else v) for k, v in snap.pop((l,) + bg).items()}
+                          for bg in refs} if mid >= 0 else {bg: None for bg in refs}
+                ex_last = {bg: export_to_host(cache, l, *bg) for bg in refs} if steps > 0 else {bg: None for bg in refs}
+                for worst, n_out, n_lay in pool.map(lambda bg: replay(l, bg, refs[bg], ex_mid[bg], ex_last[bg]), list(refs)):
+                    res["out"] = max(res["out"], worst)
+                    res["outputs"] += n_out
+                    res["layouts"] += n_lay
+                res["heads"] += len(refs)
+                del refs, ex_mid, ex_last
+    finally:
+        pool.shutdown(wait=True, cancel_futures=True)
+        cache.close()
+    return res
+
+
+def floor_heads(w: synth.Workload, layer: int, batches: Sequence[int], frac_other: float = 0.10) -> List[Tuple[int, int]]:
+    """Every retrieval KV head of the layer plus a seeded tenth (rounded up) of the others, for the given sequences."""
+    r = w.retrieval(layer)
+    ret = [g for g in range(w.n_kv_heads) if r[g]]
+    oth = [g for g in range(w.n_kv_heads) if not r[g]]
+    n_oth = min(len(oth), max(1, math.ceil(frac_other * len(oth)))) if oth else 0
+    perm = synth.seeded_permutation(w.seed * 31 + layer, len(oth))
+    pick = sorted(oth[i] for i in perm[:n_oth])
+    return [(b, g) for b in batches for g in ret + pick]

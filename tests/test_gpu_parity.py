@@ -11,7 +11,7 @@ from oracle import razor_oracle as orc
 from paper_2407_15891_b200 import binding as rz
 from paper_2407_15891_b200 import synth
 
-from _harness import TOL_OUT, bits, make_cache, run_parity, sample_heads, to_f64
+from _harness import HeadRef, TOL_OUT, bits, check_head_state, floor_heads, make_cache, run_parity, run_parity_recorded, to_f64
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
@@ -53,33 +53,44 @@ def test_cfg2_llama2_7b_shaped_32k_every_head():
     st = {}
     r = run_parity(w, steps=0, stats=st)
     assert r["heads"] == 8 * 32
-    assert st["kept_bytes"] == w.compressed_bytes(0) and st["dense_bytes"] == w.dense_bytes()
+    row = 2 * w.head_dim * w.esz()
+    kept = row * sum(len(orc.kept_positions(n, w.n_sink, win, bool(f))) for f in w.retrieval(0)
+                     for n, win in zip(w.ctx_len, w.window))
+    assert st["kept_bytes"] == kept and st["dense_bytes"] == row * sum(w.ctx_len) * w.n_kv_heads
 
 
-def test_cfg3_llama2_13b_64k_full_stack_16_steps_sampled():
+# The three large configurations run on the GPU exactly as the benchmark runs them (all layers compressed, then
+# the decode steps step-major over the layers); checked against the oracle are, in EVERY layer and for every
+# sequence listed, every retrieval KV head plus a seeded tenth of the others: layout bit-exact and means right
+# after compression, after the middle step and after the last one, outputs at every step.
+def test_cfg3_llama2_13b_64k_full_stack_16_steps_every_layer():
     w = synth.workload("cfg3")
-    layers = [0, 13, 26, 39]
-    heads = {l: sample_heads(w, l, 2, 3, range(w.batch)) for l in layers}
-    r = run_parity(w, layers=layers, heads_for=heads, steps=16, check_layout_every=5)
-    assert r["outputs"] == 4 * 4 * 5 * 16
+    heads = {l: floor_heads(w, l, range(w.batch)) for l in range(w.n_layers)}
+    assert all(len(heads[l]) == 4 * (6 + 4) for l in heads)                     # 6 retrieval + 4 of the other 34, x 4 sequences
+    r = run_parity_recorded(w, heads_for=heads, steps=16)
+    assert r["heads"] == 40 * 40 and r["outputs"] == 40 * 40 * 16 and r["layouts"] == 3 * 40 * 40
 
 
-def test_cfg4_gqa_llama3_8b_shaped_128k_sampled():
+def test_cfg4_gqa_llama3_8b_shaped_128k_every_layer():
     w = synth.workload("cfg4")
-    layers = [0, 15, 31]
-    heads = {l: sample_heads(w, l, 2, 3, range(w.batch)) for l in layers}
-    r = run_parity(w, layers=layers, heads_for=heads, steps=0)
-    assert r["outputs"] == 3 * 2 * 5 * 4
-    r = run_parity(w, layers=layers, heads_for={l: heads[l][:3] for l in layers}, steps=2)
+    heads = {l: floor_heads(w, l, range(w.batch)) for l in range(w.n_layers)}
+    assert all(len(heads[l]) == 2 * (2 + 1) for l in heads)                     # 2 retrieval + 1 of the other 6 KV heads, x 2
+    r = run_parity_recorded(w, heads_for=heads, steps=0)                        # the configuration: compression + one decode
+    assert r["heads"] == 32 * 6 and r["outputs"] == 32 * 6 * 4 and r["layouts"] == 32 * 6
+    few = {l: heads[l] for l in (0, 15, 31)}
+    r = run_parity_recorded(w, heads_for=few, steps=4)                          # and with appended tokens
+    assert r["outputs"] == 3 * 6 * 4 * 4 and r["layouts"] == 3 * 3 * 6
 
 
-def test_cfg5_ragged_serving_mix_64_steps_sampled():
+def test_cfg5_ragged_serving_mix_64_steps_shortest_median_longest():
     w = synth.workload("cfg5")
-    order = np.argsort(w.ctx_len)
-    bs = [int(order[0]), int(order[len(order) // 2]), int(order[-1])]      # shortest, median, longest
-    heads = {0: sample_heads(w, 0, 1, 2, bs)}
-    r = run_parity(w, layers=[0], heads_for=heads, steps=64, per_seq=True, check_layout_every=16)
-    assert r["outputs"] == 3 * 3 * 64
+    order = [int(i) for i in np.argsort(w.ctx_len)]
+    bs = sorted(set(order[:8] + order[28:36] + order[-8:]))                    # the 8 shortest, 8 around the median, 8 longest
+    assert len(bs) == 24
+    heads = {0: floor_heads(w, 0, bs)}
+    assert len(heads[0]) == 24 * (5 + 3)                                        # 5 retrieval + 3 of the other 27
+    r = run_parity_recorded(w, heads_for=heads, steps=64, per_seq=True)
+    assert r["heads"] == 24 * 8 and r["outputs"] == 24 * 8 * 64 and r["layouts"] == 3 * 24 * 8
 
 
 # ------------------------------------------------------------------ scaled copies, every head, paged
@@ -163,6 +174,62 @@ def test_invariants_on_gpu_window_covers_context_equals_full_attention():
     for h in range(2):
         ref = orc.full_attention(to_f64(q[0, h]), to_f64(K[0, h]), to_f64(V[0, h]), 1 / math.sqrt(128))
         assert np.abs(out[0, h] - ref).max() <= 3e-3
+    cache.close()
+
+
+def test_append_directly_behind_the_kernel_that_produces_its_rows():
+    """In a decoder the K/V projection is the kernel right before razor_append and writes k_new / v_new into
+    the same buffers every step.  Here a small elementwise kernel refills one pair of buffers immediately
+    before each of 200 appends (no synchronisation in between); the cache must hold exactly the rows of each
+    step: layout bit-exact against the oracle's recompression of the whole history, means within 1e-3."""
+    steps = 200
+    w = synth.Workload("producer", 3, 2, 4, 4, 128, "bf16", [300, 40, 77], [48, 90, 20], 4, 1, steps, 555)
+    cache = make_cache(w, max_new=steps)
+    refs = {}
+    for l in range(w.n_layers):
+        K, V = synth.make_dense_kv(w, l, DEV)
+        cache.compress(l, K, V, w.ctx_len, w.retrieval(l), w.window)
+        for b in range(w.batch):
+            for g in range(w.n_kv_heads):
+                refs[(l, b, g)] = HeadRef(l, b, g, K[b, g], V[b, g], w.ctx_len[b], steps)
+    rows = [[synth.make_new_kv(w, l, t, DEV) for t in range(steps)] for l in range(w.n_layers)]
+    k_buf = torch.empty_like(rows[0][0][0])
+    v_buf = torch.empty_like(k_buf)
+    q = synth.make_queries(w, 0, 0, DEV)
+    out = torch.empty((w.batch, w.n_q_heads, w.head_dim), dtype=torch.float32, device=DEV)
+    one = torch.ones((), dtype=torch.bfloat16, device=DEV)
+    torch.cuda.synchronize()
+    for t in range(steps):
+        for l in range(w.n_layers):
+            torch.mul(rows[l][t][0], one, out=k_buf)            # the "projection": an elementwise kernel, not a copy
+            torch.mul(rows[l][t][1], one, out=v_buf)
+            cache.append(l, k_buf, v_buf)
+            cache.decode(l, q, out)                              # keeps the append's programmatic launch chain as in a pass
+    torch.cuda.synchronize()
+    for (l, b, g), ref in refs.items():
+        for t in range(steps):
+            ref.append(rows[l][t][0][b, g].cpu(), rows[l][t][1][b, g].cpu())
+        check_head_state(cache, ref, w.n_sink, w.window[b], bool(w.retrieval(l)[g]))
+    assert cache.device_status() == 0
+    cache.close()
+
+
+def test_a_sequence_without_tokens_attends_to_nothing_and_gives_zeros():
+    """A head that holds no token has both sums of Eq. 5 empty; library and oracle define the output as zeros."""
+    w = synth.Workload("empty", 2, 1, 4, 2, 64, "bf16", [0, 50], [16, 16], 4, 1, 2, 99)
+    cache = make_cache(w, max_new=2)
+    K, V = synth.make_dense_kv(w, 0, DEV)
+    cache.compress(0, K, V, w.ctx_len, w.retrieval(0), w.window)
+    q = synth.make_queries(w, 0, 0, DEV)
+    out = to_f64(cache.decode(0, q))
+    qh = to_f64(q)
+    for b in range(2):
+        for g in range(2):
+            hc = orc.compress_head(to_f64(K[b, g]), to_f64(V[b, g]), w.ctx_len[b], w.n_sink, w.window[b], bool(w.retrieval(0)[g]))
+            for j in range(2):
+                expect = orc.decode_head(qh[b, g * 2 + j], hc, 1 / math.sqrt(64))
+                assert np.abs(out[b, g * 2 + j] - expect).max() <= 3e-3
+    assert not out[0].any()                                       # the empty sequence: exact zeros
     cache.close()
 
 
