@@ -32,11 +32,37 @@ METRIC = "compressed_cache_decode_attention_GBps"
 UNIT = "GB/s"
 NOMINAL_HBM_GBS = 8000.0        # the "~8 TB/s" the target is quoted against
 FALLBACK_HBM_GBS = 6650.0       # used only when MEASURED_PEAKS.json is absent
-# DRAM traffic of the decode kernel per algorithmic byte: (dram__bytes_read.sum + dram__bytes_write.sum) of one launch
-# over the kept K+V bytes of that launch, from the ncu capture summarised in
-# profiles/decode_kernel_cfg3_half_scale_and_cfg4_ncu_full.md (taken on the half-scale case; traffic grows in
-# proportion to the kept tokens, so the ratio carries over to the full-size launch).  Set to None when the kernel changes.
-DECODE_TRAFFIC_PER_ALG_BYTE = 1.008
+# DRAM traffic of the decode kernel per algorithmic byte comes from an ncu capture summarised under profiles/.
+# The summary names the sources it was taken on by their SHA-256; the ratio is used only while those
+# sources are unchanged, otherwise roofline.traffic is null.
+DECODE_TRAFFIC_PROFILE = os.path.join("profiles", "decode_kernel_cfg3_half_scale_and_cfg4_ncu_full.md")
+DECODE_SOURCES = ["razor_decode.cu", "razor_sync.cuh", "razor_common.cuh", "razor_internal.h"]
+
+
+def decode_sources_sha256() -> str:
+    import hashlib
+    h = hashlib.sha256()
+    for name in DECODE_SOURCES:
+        with open(os.path.join(ROOT, "paper_2407_15891_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def decode_traffic_per_alg_byte():
+    """(ratio, where it comes from) or (None, why not)."""
+    import re
+    path = os.path.join(ROOT, DECODE_TRAFFIC_PROFILE)
+    try:
+        text = open(path).read()
+    except OSError:
+        return None, "no capture summary"
+    sha = re.search(r"decode_sources_sha256:\s*([0-9a-f]{64})", text)
+    ratio = re.search(r"dram_bytes_per_algorithmic_byte:\s*([0-9.]+)", text)
+    if not sha or not ratio:
+        return None, "capture summary carries no source hash"
+    if sha.group(1) != decode_sources_sha256():
+        return None, "the decode kernel's sources changed since the capture in " + DECODE_TRAFFIC_PROFILE
+    return float(ratio.group(1)), DECODE_TRAFFIC_PROFILE
 
 
 # ---------------------------------------------------------------------------------------------- byte accounting
@@ -166,10 +192,15 @@ def oracle_sample(w, budget_s=12.0):
     from oracle import razor_oracle as orc
     from paper_2407_15891_b200 import synth
     try:
+        cores = len(os.sched_getaffinity(0))        # host cores this process may run on
+    except AttributeError:
+        cores = os.cpu_count() or 1
+    try:
         from threadpoolctl import threadpool_info
-        threads = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+        blas = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
     except Exception:
-        threads = 1
+        blas = 1
+    threads = cores
     retr = w.retrieval(0)
     order = [g for g in range(w.n_kv_heads) if retr[g]][:1] + [g for g in range(w.n_kv_heads) if not retr[g]][:1]
     order += [g for g in range(w.n_kv_heads) if g not in order]
@@ -200,7 +231,9 @@ def oracle_sample(w, budget_s=12.0):
             break
     desc = (f"layer 0, sequence 0, {heads} of {w.n_kv_heads} KV heads ({n_retr} retrieval): one compression + {T} "
             f"decode steps each (no appends); compress {t_comp:.3f}s, decode {t_dec:.3f}s "
-            f"(decode alone: {bytes_attended / t_dec / 1e9:.2f} GB/s); inputs generated per head outside the timing")
+            f"(decode alone: {bytes_attended / t_dec / 1e9:.2f} GB/s); inputs generated per head outside the timing; "
+            f"plain numpy fp64: the compression (row gather + sum) runs on one thread, the decode's matrix-vector "
+            f"products in a BLAS pool of {blas} threads; {cores} host cores available")
     return bytes_attended / (t_comp + t_dec) / 1e9, desc, threads, dict(decode_s=t_dec, compress_s=t_comp, heads=heads)
 
 
@@ -251,7 +284,7 @@ def _workload_config(w, args):
 
 
 # ---------------------------------------------------------------------------------------------- GPU legs
-def decode_only(rz, synth, name, n_layers, dev, peak, reps=60, n_tok=1, alibi=False):
+def decode_only(rz, synth, name, n_layers, dev, peak, reps=60, n_tok=1, alibi=False, with_append=False):
     """Decode attention alone on the first n_layers layers of another workload (each layer compressed from
     one seeded dense buffer): back-to-back razor_decode_attention calls cycling over the layers, so that
     every call streams pages that the L2 no longer holds."""
@@ -261,7 +294,7 @@ def decode_only(rz, synth, name, n_layers, dev, peak, reps=60, n_tok=1, alibi=Fa
     w.n_layers = n_layers
     retr = [w.retrieval(l) for l in range(n_layers)]
     cfg = rz.make_config(w.batch, n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, 0 if alibi else w.n_sink,
-                         max(w.ctx_len), max(1, n_tok), use_compensation=0 if alibi else 1)
+                         max(w.ctx_len), max(4, n_tok), use_compensation=0 if alibi else 1)
     cache = rz.RazorCache(cfg, w.ctx_len, w.window, np.stack(retr), device=dev)
     if alibi:   # the ALiBi variant: distance penalty on every logit, recent tokens only, no compensation token
         slopes = np.array([2.0 ** (-8.0 * (i + 1) / w.n_q_heads) for i in range(w.n_q_heads)], dtype=np.float32)
@@ -290,6 +323,7 @@ def decode_only(rz, synth, name, n_layers, dev, peak, reps=60, n_tok=1, alibi=Fa
     for l in range(n_layers):
         call(l, q, out)
     torch.cuda.synchronize()
+    reps = max(reps, n_layers)
     a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
     a.record()
     for i in range(reps):
@@ -298,14 +332,37 @@ def decode_only(rz, synth, name, n_layers, dev, peak, reps=60, n_tok=1, alibi=Fa
     torch.cuda.synchronize()
     us = a.elapsed_time(b) * 1e3 / reps
     kept = compressed_bytes(w, 0, extra=n_tok if n_tok > 1 else 0)
-    status = cache.device_status()
-    cache.close()
     gbs = kept / (us * 1e-6) / 1e9
-    return {"workload": f"{name}: batch {w.batch}, {w.n_q_heads}/{w.n_kv_heads} heads, context {max(w.ctx_len)}, "
-                        f"{n_layers} layers cycled ({n_layers * kept / 1e9:.2f} GB of pages)",
-            "us_per_layer": us, "gbs": gbs, "frac_of_measured": gbs / peak, "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS,
-            "compressed_mb_per_layer": kept / 1e6, "launches_timed": reps, "device_status": status,
-            "query_tokens_per_call": n_tok, "alibi": bool(alibi)}
+    res = {"workload": f"{name}: batch {w.batch}, {w.n_q_heads}/{w.n_kv_heads} heads, context {max(w.ctx_len)}, "
+                       f"{n_layers} layers cycled ({n_layers * kept / 1e9:.2f} GB of pages)",
+           "us_per_layer": us, "gbs": gbs, "frac_of_measured": gbs / peak, "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS,
+           "compressed_mb_per_layer": kept / 1e6, "launches_timed": reps,
+           "query_tokens_per_call": n_tok, "alibi": bool(alibi)}
+    if with_append and n_tok == 1:
+        # the workload's decode step as a pass runs it: razor_append + razor_decode_attention on every layer
+        k_new, v_new = synth.make_new_kv(w, 0, 0, dev)
+        steps = 3
+        for l in range(n_layers):                      # (max_new_tokens of this cache is steps + 1)
+            cache.append(l, k_new, v_new); call(l, q, out)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(steps - 1):
+            for l in range(n_layers):
+                cache.append(l, k_new, v_new); call(l, q, out)
+        b.record()
+        torch.cuda.synchronize()
+        us_p = a.elapsed_time(b) * 1e3 / ((steps - 1) * n_layers)
+        kept_p = compressed_bytes(w, 0, extra=2)
+        res["with_append"] = {"us_per_layer": us_p, "us_per_decode_step": us_p * n_layers,
+                              "gbs": kept_p / (us_p * 1e-6) / 1e9,
+                              "frac_of_measured": kept_p / (us_p * 1e-6) / 1e9 / peak,
+                              "frac_of_nominal_8TBs": kept_p / (us_p * 1e-6) / 1e9 / NOMINAL_HBM_GBS,
+                              "launches_timed": (steps - 1) * n_layers,
+                              "note": "per layer: razor_append + razor_decode_attention, all layers of the "
+                                      "configuration, CUDA events at the ends of the run only"}
+    res["device_status"] = cache.device_status()
+    cache.close()
+    return res
 
 
 def chunked_prefill_leg(rz, synth, dev, peak, chunk=8192, reps=3):
@@ -469,13 +526,7 @@ def main():
             q = qs[t % n_q]
             for l in range(L):
                 cache.append(l, k_new, v_new)
-                sample = ev is not None and ((l + t) % ev["every"] == 0)
-                if sample:
-                    e0 = torch.cuda.Event(enable_timing=True); e0.record()
                 cache.decode(l, q, out)
-                if sample:
-                    e1 = torch.cuda.Event(enable_timing=True); e1.record()
-                    ev["decode"].append((e0, e1, l, t))
                 launches["n"] += 3        # append, streaming decode kernel, combine kernel
 
     def sync_all():
@@ -500,8 +551,7 @@ def main():
 
     sampler = ClockSampler(local)
     sampler.start()
-    ev = {"decode": [], "every": 4 if L * T >= 16 else 1,
-          "compress_end": torch.cuda.Event(enable_timing=True)}
+    ev = {"compress_end": torch.cuda.Event(enable_timing=True)}
     starts, ends, comp_ends = [], [], []
     launches["n"] = 0
     sync_all()
@@ -522,25 +572,33 @@ def main():
 
     comp_ms = statistics.mean(s.elapsed_time(c) for s, c in zip(starts, comp_ends))
     dec_phase_ms = statistics.mean(c.elapsed_time(e) for c, e in zip(comp_ends, ends))
-    dec_us = [a.elapsed_time(b) * 1e3 for a, b, _, _ in ev["decode"]]
-    dec_alg = [decode_alg_bytes(l, t)[1] for _, _, l, t in ev["decode"]]
-    dec_gbs = sum(dec_alg) / (sum(dec_us) * 1e-6) / 1e9
+    # The decode launches are timed as they run in the pass: no event sits between two launches (an event record
+    # between an append and its decode kernel would undo the overlap of their programmatic launches), so the
+    # duration of one launch is the decode phase of the pass divided by its launches.  That phase also holds the
+    # append kernels, which makes the figure an upper bound on the decode launch itself.
+    n_dec = T * L
+    us_per_launch = dec_phase_ms * 1e3 / n_dec
+    alg_total = sum(decode_alg_bytes(l, t)[1] for l in range(L) for t in range(T))
+    alg_per_launch = alg_total / n_dec
+    dec_gbs = alg_total / (dec_phase_ms * 1e-3) / 1e9
     peak, peak_kind = measured_peak()
-    alg_per_launch = statistics.mean(dec_alg)
+    ratio, ratio_src = decode_traffic_per_alg_byte()
     roofline = {"bound": "hbm", "kernel": "decode_kernel (+ its dependent combine_kernel): one razor_decode_attention call",
                 "achieved": dec_gbs, "peak": peak, "unit": "GB/s",
                 "frac": dec_gbs / peak, "peak_kind": f"of {peak_kind} (sustained copy bandwidth)",
                 "frac_of_nominal_8TBs": dec_gbs / NOMINAL_HBM_GBS,
-                "alg_bytes_per_launch": alg_per_launch, "us_per_launch": statistics.mean(dec_us),
-                "launches_timed": len(dec_us),
-                "traffic": (DECODE_TRAFFIC_PER_ALG_BYTE * alg_per_launch) if DECODE_TRAFFIC_PER_ALG_BYTE else None}
+                "alg_bytes_per_launch": alg_per_launch, "us_per_launch": us_per_launch,
+                "launches_timed": n_dec * args.steps,
+                "how": "decode phase of the timed passes / its launches, CUDA events at the ends of the phase only; "
+                       "the phase includes the razor_append kernels",
+                "traffic": (ratio * alg_per_launch) if ratio else None, "traffic_source": ratio_src}
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": w.dtype if w.dtype != "bf16" else "bf16", "data": "synthetic", "config": workload_config(w, args),
         "clocks": clocks, "gpu_launches": n_launches, "roofline": roofline,
-        "decode": {"gbs_kernel": dec_gbs, "us_per_layer": statistics.mean(dec_us),
+        "decode": {"gbs_kernel": dec_gbs, "us_per_layer": us_per_launch,
                    "us_per_decode_step": dec_phase_ms * 1e3 / T,
                    "gbs_phase_incl_append": attended / (dec_phase_ms * 1e-3) / 1e9,
                    "compressed_gb_per_decode_step": attended / T / 1e9},
@@ -559,11 +617,27 @@ def main():
             cache.append(l, k_new, v_new)
     b.record()
     sync_all()
-    line["append"] = {"us_per_layer_in_pass": dec_phase_ms * 1e3 / (T * L) - statistics.mean(dec_us),
-                      "us_per_call_back_to_back": a.elapsed_time(b) * 1e3 / (T * L), "launches_timed": T * L,
-                      "note": "in the pass: (append + decode) per layer minus the decode call, the append running as a "
-                              "programmatic dependent; back to back: razor_append calls alone, one token per "
-                              "(sequence, KV head), bound by the host's launch rate"}
+    app_us = a.elapsed_time(b) * 1e3 / (T * L)
+    # decode attention alone, back to back over the layers (every call streams pages the L2 no longer holds)
+    reps = max(1, 80 // L)
+    for l in range(L):
+        cache.decode(l, qs[0], out)
+    sync_all()
+    a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+    a.record()
+    for i in range(reps * L):
+        cache.decode(i % L, qs[i % n_q], out)
+    b.record()
+    sync_all()
+    dec_alone_us = a.elapsed_time(b) * 1e3 / (reps * L)
+    kept_now = statistics.mean(compressed_bytes(w, l, extra=T) for l in range(L))
+    line["decode"]["us_per_layer_back_to_back_no_append"] = dec_alone_us
+    line["decode"]["gbs_back_to_back_no_append"] = kept_now / (dec_alone_us * 1e-6) / 1e9
+    line["append"] = {"us_per_layer_in_pass": us_per_launch - dec_alone_us,
+                      "us_per_call_back_to_back": app_us, "launches_timed": T * L,
+                      "note": "in the pass: (append + decode) per layer minus a decode call timed back to back without "
+                              "appends; back to back: razor_append calls alone, one token per (sequence, KV head), "
+                              "bound by the host's launch rate"}
 
     # ------------------------------------------------------------------ dense full-cache decode, same GPU
     if not args.no_dense and rank == 0 and not per_seq:
@@ -586,7 +660,7 @@ def main():
             d_us = a.elapsed_time(b) * 1e3 / reps
             line["dense_decode"] = {"us_per_layer": d_us, "gbs": dense_bytes(w) / (d_us * 1e-6) / 1e9,
                                     "us_per_decode_step": d_us * L,
-                                    "speedup_compressed_vs_dense": d_us / statistics.mean(dec_us)}
+                                    "speedup_compressed_vs_dense": d_us / us_per_launch}
             dcache.close()
             del dcache
         except Exception as ex:   # e.g. not enough memory for a dense layer beside the compressed stack
@@ -595,7 +669,7 @@ def main():
     # ------------------------------------------------------------------ the 128K grouped-query shape, decode only
     if not args.no_dense and rank == 0 and args.workload == "cfg3" and not args.layers:
         try:
-            line["decode_128k_gqa"] = decode_only(rz, synth, "cfg4", 6, dev, peak)
+            line["decode_128k_gqa"] = decode_only(rz, synth, "cfg4", 32, dev, peak, reps=96, with_append=True)
         except Exception as ex:
             line["decode_128k_gqa"] = {"unavailable": str(ex)[:200]}
         try:   # retrieval-head identification scores (Section 3.3)

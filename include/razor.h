@@ -241,15 +241,20 @@ RAZOR_API int razor_schedule_query(razor_cache_t* cache, int32_t layer, int32_t*
 enum {
   RAZOR_OPT_DECODE_TAIL_ITEMS_PER_SM = 1, /* a tail item is 1/k of an SM's share of the remaining tail
                                              (k = 1..1024; default 3)                                      */
-  RAZOR_OPT_DECODE_MIN_CHUNK_PAGES = 2, /* smallest span or tail item in pages (default 16)               */
+  RAZOR_OPT_DECODE_MIN_CHUNK_PAGES = 2, /* smallest span or tail item in pages (default 32)               */
   RAZOR_OPT_DECODE_RING_KB = 3,         /* shared-memory page ring per CTA in KiB; 0 = as large as fits   */
   RAZOR_OPT_DECODE_CONSUMER_WARPS = 4,  /* streaming warps per CTA: 0 = default; 4, 8, 12 or 16; a value
                                            the head shape has no kernel for falls back to the default     */
   RAZOR_OPT_DECODE_TENSOR_CORES = 5,    /* bf16 heads: 0 = matrix instructions from group 4 up (default),
                                            1 = for every group size (a single head fills one row of the
                                            tile), 2 = never                                               */
-  RAZOR_OPT_DECODE_STATIC_PERCENT = 6   /* share of the pages handed out as per-CTA spans (0..100;
+  RAZOR_OPT_DECODE_STATIC_PERCENT = 6,  /* share of the pages handed out as per-CTA spans (0..100;
                                            default 80); 0 makes every job a tail item                     */
+  RAZOR_OPT_DECODE_EARLY_PREFETCH = 7   /* most pages (0..64; default 12) a CTA copies from the start of its span
+                                           into shared memory before the kernel waits for the launch before it
+                                           on the stream - only pages that no kernel still in flight can be
+                                           writing (the host knows which page a preceding razor_append
+                                           touched); 0: every copy waits                                   */
 };
 RAZOR_API int razor_cache_set_option(razor_cache_t* cache, int32_t option, int32_t value);
 
@@ -259,7 +264,8 @@ RAZOR_API int razor_cache_set_option(razor_cache_t* cache, int32_t option, int32
  * This call synchronises `stream`, stores the word in *status (0 = healthy) and, when it is non-zero,
  * clears it together with the kernel's work counters so that the cache can be used again; outputs of
  * the affected launch are undefined.  Bits: 1 producer wait, 2 consumer wait, 4 reducer wait, 8 copies
- * still in flight at exit, 16 the self-test below.  Errors: NULL_PTR, CUDA.
+ * still in flight at exit, 16 the self-test below, 32 an early-prefetch count that did not match the
+ * device's lengths.  Errors: NULL_PTR, CUDA.
  */
 RAZOR_API int razor_cache_device_status(razor_cache_t* cache, int32_t* status, void* stream);
 

@@ -32,7 +32,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 inline int ceil_div(long long a, long long b) { return (int)((a + b - 1) / b); }
 
 struct Layout {
-  size_t state, comp_sum, comp_mean, page_table, items, jobs, multi, rec_ml, rec_o, queue, scratch, plan, slopes, total;
+  size_t state, comp_sum, comp_mean, page_table, items, jobs, multi, rec_ml, rec_o, queue, tickets, scratch, plan, slopes, total;
   int max_pages, max_items;
 };
 
@@ -76,6 +76,7 @@ Layout make_layout(const razor_config_t& c) {
   l.rec_o = take((size_t)l.max_items * kMaxGroup * D * sizeof(float));
   (void)g;
   l.queue = take(8 * sizeof(int32_t));   // queue[0..3], then the status word
+  l.tickets = take(nh * sizeof(int32_t));
   l.scratch = take(((size_t)kCompressSliceBudget + nh) * 2 * D * sizeof(float));
   l.plan = take(nh * sizeof(HeadPlan) + (size_t)c.batch * sizeof(SeqDesc));   // plan[], then seq_desc[]
   l.slopes = take(L * (size_t)c.n_q_heads * sizeof(float));
@@ -129,7 +130,7 @@ struct razor_cache {
   DeviceView dv;
   long long pool_pages = 0, next_page = 0;
   int n_sms = 148;
-  DecodeTuning tune{3, 80, 16, 0, 0, 0};
+  DecodeTuning tune{3, 80, 32, 0, 0, 0, 12};
   std::vector<LayerHost> layers;
   WorkItem* pinned_items = nullptr;   // [L][max_items]
   int32_t* pinned_jobs = nullptr;     // [L][max_items + 1]
@@ -143,6 +144,17 @@ struct razor_cache {
   // Layer whose pages, state or sums the last kernel launched for this cache wrote (-1: it wrote none, a decode).
   // An append of another layer may read before it waits for that kernel.
   int last_writer_layer = -1;
+  // Kernels launched since the last decode launch that write a layer: (layer, kind).  A decode kernel waits for
+  // everything before it and only then lets its successors start, so these are the only library kernels that
+  // can still be in flight while the NEXT decode kernel runs the part that precedes its own dependency wait.
+  enum { kWriteOneToken = 1, kWriteBulk = 2 };
+  std::vector<std::pair<int, int>> writes_since_decode;
+  bool writes_overflow = false;
+  void note_write(int layer, int kind) {
+    last_writer_layer = layer;
+    if (writes_since_decode.size() < 256) writes_since_decode.emplace_back(layer, kind);
+    else writes_overflow = true;
+  }
 };
 
 extern "C" {
@@ -224,6 +236,7 @@ int razor_cache_create(razor_cache_t** out, const razor_config_t* cfg, void* poo
   dv.multi = (MultiHead*)(ws + lay.multi);
   dv.queue = (int32_t*)(ws + lay.queue);
   dv.status = dv.queue + 4;
+  dv.tickets = (int32_t*)(ws + lay.tickets);
   dv.compress_scratch = (float*)(ws + lay.scratch);
   dv.plan = (HeadPlan*)(ws + lay.plan);
   dv.seq_desc = (SeqDesc*)(ws + lay.plan + (size_t)cfg->batch * cfg->n_kv_heads * sizeof(HeadPlan));
@@ -470,7 +483,7 @@ int compress_impl(razor_cache* c, int layer, const std::vector<SeqIn>& seqs, con
   long long slices = ceil_div((long long)c->n_sms * 48, heads_in_call);
   const long long by_rows = n_max >= 8 * 512 ? n_max / 512 : std::max(1, n_max / 64);
   slices = std::max(1LL, std::min({slices, (long long)kCompressMaxSlices, room, by_rows}));
-  c->last_writer_layer = layer;
+  c->note_write(layer, razor_cache::kWriteBulk);
   ce = launch_compress(c->dv, cfg.dtype, layer, (int)seqs.size(), (int)slices, n_plan, stream);
   if (ce != cudaSuccess) return fail_enqueued(ce);
   // ---- commit
@@ -594,7 +607,7 @@ int razor_append(razor_cache_t* c, int32_t layer, const void* k_new, const void*
   if (L.appended >= c->cfg.max_new_tokens) return RAZOR_E_CAPACITY;
   const int early_reads = c->last_writer_layer != layer;
   RZ_CUDA(launch_append(c->dv, c->cfg.dtype, layer, k_new, v_new, early_reads, (cudaStream_t)stream));
-  c->last_writer_layer = layer;
+  c->note_write(layer, razor_cache::kWriteOneToken);
   // Host mirror of the kernel's state update.
   const int n_sink = c->cfg.n_sink;
   for (HeadState& h : L.hs) {
@@ -631,7 +644,7 @@ int razor_append_many(razor_cache_t* c, int32_t layer, const void* k_new, const 
                                            (long long)(n_tokens / 32)}));
   }
   RZ_CUDA(launch_append_many(c->dv, c->cfg.dtype, layer, k_new, v_new, n_tokens, slices, (cudaStream_t)stream));
-  c->last_writer_layer = layer;
+  c->note_write(layer, razor_cache::kWriteBulk);
   const int n_sink = c->cfg.n_sink;
   for (HeadState& h : L.hs) h = state_after_run(h, n_sink, n_tokens);   // host mirror of the kernels' state update
   L.appended += n_tokens;
@@ -661,6 +674,42 @@ int razor_append_plan(int32_t len, int32_t n_drop, int32_t ring_head, int32_t wi
 
 static int decode_impl(razor_cache_t* c, int32_t layer, const void* q, float* out, int32_t n_tokens,
                        int32_t tok_stride, int32_t q_after, void* stream);
+
+// Which pages a span CTA may copy before the decode kernel waits for the launch it depends on.  While that part
+// of the kernel runs, the library kernels launched since the previous decode may still be writing.  If none of
+// them wrote this layer, every page of it is stable.  If exactly one did and it was a single-token append, the
+// only page of a head it writes is the one holding the appended row, and the host mirror says which: the slot
+// before `len` for a head that grew, the ring slot before ring_head for a head that evicted.  Anything else
+// (a bulk append, a compression, several appends): no early copies.  For CTA i the count covers the leading
+// pages of its span's first work item, cut at the written page and at the item's length as it is now.
+static void plan_early_prefetch(const razor_cache* c, int layer, DecodeJobs& jb) {
+  std::memset(jb.early, 0, sizeof(jb.early));
+  if (!c->tune.early_prefetch || c->writes_overflow) return;
+  int n_writes = 0, kind = 0;
+  for (const auto& wr : c->writes_since_decode)
+    if (wr.first == layer) { n_writes += 1; kind = wr.second; }
+  if (n_writes > 1 || (n_writes == 1 && kind != razor_cache::kWriteOneToken)) return;
+  const LayerHost& L = c->layers[layer];
+  const int n_sink = c->cfg.n_sink;
+  const int n = std::min({L.n_spans, c->n_sms, (int)kEarlyCtas});
+  for (int i = 0; i < n; ++i) {
+    const WorkItem& w = L.items[L.jobs[i]];
+    const HeadState& st = L.hs[w.head];
+    const int head_pages = ceil_div(st.len, kPageTokens);
+    const int page_end = w.page_end < 0 ? head_pages : std::min(w.page_end, head_pages);
+    int e = std::min(c->tune.early_prefetch, std::max(0, page_end - w.page_begin));
+    if (n_writes == 1) {
+      int slot = -1;   // slot the append wrote
+      if (st.window < 0 || st.n_drop == 0) slot = st.len - 1;                                  // the head grew
+      else if (st.window > 0) slot = n_sink + (st.ring_head + st.window - 1) % st.window;       // it evicted
+      if (slot >= 0) {
+        const int tp = slot / kPageTokens - w.page_begin;
+        if (tp >= 0 && tp < e) e = tp;
+      }
+    }
+    jb.early[i] = (uint8_t)e;
+  }
+}
 
 int razor_decode_attention_multi(razor_cache_t* c, int32_t layer, const void* q, float* out, int32_t n_tokens,
                                  void* stream) {
@@ -705,10 +754,13 @@ static int decode_impl(razor_cache_t* c, int32_t layer, const void* q, float* ou
   rc = ensure_schedule(c, layer, (cudaStream_t)stream, true);
   if (rc) return rc;
   const LayerHost& L = c->layers[layer];
-  const DecodeJobs jb{L.n_items, L.n_jobs, L.n_spans, L.jobs[L.n_spans], L.n_multi, n_tokens, tok_stride, q_after};
+  DecodeJobs jb{L.n_items, L.n_jobs, L.n_spans, L.jobs[L.n_spans], L.n_multi, n_tokens, tok_stride, q_after, {}};
+  plan_early_prefetch(c, layer, jb);
   RZ_CUDA(launch_decode(c->dv, c->cfg.dtype, layer, jb, q, out, c->n_sms, c->tune,
                         (cudaStream_t)stream));
   c->last_writer_layer = -1;
+  c->writes_since_decode.clear();
+  c->writes_overflow = false;
   return RAZOR_OK;
 }
 
@@ -799,6 +851,10 @@ int razor_cache_set_option(razor_cache_t* c, int32_t option, int32_t value) {
       if (value < 0 || value > 2) return RAZOR_E_INVALID_ARG;
       c->tune.tensor_cores = value;
       break;
+    case RAZOR_OPT_DECODE_EARLY_PREFETCH:
+      if (value < 0 || value > 64) return RAZOR_E_INVALID_ARG;
+      c->tune.early_prefetch = value;
+      break;
     default:
       return RAZOR_E_INVALID_ARG;
   }
@@ -815,6 +871,7 @@ int razor_cache_device_status(razor_cache_t* c, int32_t* status, void* stream) {
   if (host != 0) {
     // A kernel gave up part-way: its job queue may be left non-zero.  Put it back.
     RZ_CUDA(cudaMemsetAsync(c->dv.queue, 0, 8 * sizeof(int32_t), (cudaStream_t)stream));
+    RZ_CUDA(cudaMemsetAsync(c->dv.tickets, 0, (size_t)c->dv.n_heads * sizeof(int32_t), (cudaStream_t)stream));
     RZ_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
   }
   return RAZOR_OK;

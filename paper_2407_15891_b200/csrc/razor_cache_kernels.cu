@@ -210,7 +210,7 @@ __global__ void compress_finalize_kernel(DeviceView dv, int layer, int n_slices)
 // ring_head) is folded into the fp32 compensation sums, the count grows by one, the means are
 // recomputed (Eq. 4 over every token dropped so far) and the new row takes that slot.
 template <typename T, int D>
-__global__ void __launch_bounds__(128) append_kernel(DeviceView dv, int layer, const T* __restrict__ k_new,
+__global__ void __launch_bounds__(64) append_kernel(DeviceView dv, int layer, const T* __restrict__ k_new,
                                                      const T* __restrict__ v_new, int early_reads) {
   using Geo = RowGeom<T, D>;
   constexpr int LPR = Geo::kLpr, EPL = Geo::kEpl;
@@ -225,6 +225,9 @@ __global__ void __launch_bounds__(128) append_kernel(DeviceView dv, int layer, c
   //   * the caller's k_new / v_new.  Whatever produced them (in a model: the K/V projection, the kernel
   //     directly before this one) is not known to the library, so they are read only after the wait.
   // Every write comes after the wait as well, which keeps completion in stream order.
+  // The kernel queued behind this one (the layer's decode kernel) may start right away: ahead of its own wait
+  // it touches nothing this kernel writes (it is told which page of each head the append stores into).
+  cudaTriggerProgrammaticLaunchCompletion();
   if (!early_reads) cudaGridDependencySynchronize();
   const bool active = head < dv.n_heads;
   const size_t hs = (size_t)layer * dv.n_heads + (active ? head : 0);
@@ -266,7 +269,6 @@ __global__ void __launch_bounds__(128) append_kernel(DeviceView dv, int layer, c
     }
   }
   if (early_reads) cudaGridDependencySynchronize();
-  cudaTriggerProgrammaticLaunchCompletion();   // the decode kernel queued behind the append may set itself up
   if (row_lane) {
     const uint4 kf = ((const uint4*)(k_new + (size_t)head * D))[lane];
     const uint4 vf = ((const uint4*)(v_new + (size_t)head * D))[lane];
@@ -544,7 +546,7 @@ cudaError_t launch_compress(const DeviceView& dv, int dtype, int layer, int n_se
 template <typename T, int D>
 static cudaError_t append_t(const DeviceView& dv, int layer, const void* k, const void* v, int early_reads,
                             cudaStream_t s) {
-  const int warps = 4;
+  const int warps = 2;
   return launch_dependent(append_kernel<T, D>, (dv.n_heads + warps - 1) / warps, warps * 32, s, dv, layer, (const T*)k,
                           (const T*)v, early_reads);
 }

@@ -467,9 +467,27 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
     pid0 = first_pids(w0);
   }
   __syncthreads();
+  // The first pages of the span go into the (still empty) ring right away: the host has named a run of
+  // leading pages of the span's first item that exist and that no kernel still in flight writes (an append
+  // before this launch touches one known page per head).  Positions below the ring length use every stage at
+  // most once, so nothing has to be waited for.  The pages' descriptor, which needs the head's state as the
+  // append leaves it, follows after the dependency wait; the consumers then find these pages already landed.
+  unsigned early_done = 0;
+  if (warp == NC && has_span && blockIdx.x < kEarlyCtas) {
+    const int n_early = min((int)jb.early[blockIdx.x], n_stages);   // the host has applied its own cap already
+    const int32_t* pt0 = dv.page_table + row_of(w0) * dv.max_pages + w0.page_begin;
+    for (int p = lane; p < n_early; p += 32) {
+      unsigned stage, use;
+      ring_slot<NC>((unsigned)p, (unsigned)n_stages, stage, use);
+      mbar_arrive_expect_tx(&bars.full[stage], PB);
+      bulk_load(ring + (size_t)stage * PB, dv.pool + (size_t)pt0[p] * dv.page_bytes, PB, &bars.full[stage]);
+    }
+    early_done = (unsigned)n_early;
+    if (n_early > 0) pid0 = pt0[min(n_early + lane, dv.max_pages - 1 - w0.page_begin)];   // ids of the round that follows
+  }
   // This kernel is launched as a programmatic dependent of whatever precedes it on the stream (the
-  // append or an earlier combine), so everything above overlaps that kernel's tail; nothing that kernel
-  // wrote is touched before this point.
+  // append or an earlier combine), so everything above overlaps that kernel's tail; nothing a kernel
+  // still in flight writes is touched before this point.
   cudaGridDependencySynchronize();
   // The combine kernel that follows may be made resident as soon as SMs free up; it waits for this whole
   // grid to finish before it reads anything this grid writes.
@@ -493,7 +511,7 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
     // positions issued per round: never more than one lap of the shortest sub-ring, so that no lane of
     // a round waits for a stage that another lane of the same round is about to fill
     const int batch = min(32, NC * (n_stages / NC));
-    unsigned c = 0;                                      // ring positions issued so far by this CTA (exact)
+    unsigned c = early_done;                             // ring positions issued so far by this CTA (exact)
     unsigned seq_issued = 0;                             // item slots whose copies were issued
     int marker_slot = -1;                                // slot that received the end marker
     bool ok = true;
@@ -509,6 +527,16 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
       job_range(jb.n_spans + __shfl_sync(0xffffffffu, j, 0), it, job_end);
       w = it < n_items ? items[it] : no_item;
       pid_first = first_pids(w);
+    }
+    // The query rows of the first item do not depend on the head's state: their copy is issued now, next to the
+    // load of that state, instead of behind it.
+    constexpr uint32_t kQBytes = G * D * sizeof(T);
+    bool q_issued = false;
+    if (lane == 0 && it < n_items) {
+      mbar_expect_tx(&bars.item_full[0], kQBytes);
+      for (int t = 0; t < jb.n_tok; ++t)
+        bulk_load(&slots[0].q[t * g_real][0], q + row_offset(w.head, t * g_real), kQBytes / jb.n_tok, &bars.item_full[0]);
+      q_issued = true;
     }
     HeadState st = dv.state[row_of(w)];
     for (unsigned seq = 0; ok; ++seq) {
@@ -531,6 +559,17 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
       const int head_pages = (st.len + kPageTokens - 1) / kPageTokens;
       const int page_end = w.page_end < 0 ? head_pages : min(w.page_end, head_pages);
       const int n = max(0, page_end - w.page_begin);
+      const int p_first = seq == 0 ? (int)early_done : 0;   // pages of this item already on their way
+      if (p_first > n) {   // the host's count and the device's lengths disagree: stop rather than mix items up
+        if (lane == 0) {
+          atomicOr(dv.status, kStatusEarlyMismatch);
+          if (q_issued) mbar_arrive(&bars.item_full[slot]);   // lets the exit path wait for the query copy in flight
+        }
+        if (__shfl_sync(0xffffffffu, (int)q_issued, 0)) seq_issued = seq + 1;
+        *abort_flag = 1;
+        ok = false;
+        break;
+      }
       const bool seed = w.part_idx == 0 && dv.use_comp && st.n_drop > 0 && st.window >= 0;
       if (lane == 0) {
         ItemDesc d;
@@ -538,10 +577,12 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
         d.part_idx = w.part_idx; d.n_parts = w.n_parts; d.rec_base = w.rec_base; d.ring_head = st.ring_head;
         d.seed = seed ? 1 : 0; d.n_drop = st.n_drop; d.window = st.window; d.pad1 = 0;
         sl.desc = d;
-        constexpr uint32_t q_bytes = G * D * sizeof(T), mean_bytes = 2 * D * sizeof(float);
-        mbar_arrive_expect_tx(&bars.item_full[slot], q_bytes + (seed ? mean_bytes : 0u));
-        for (int t = 0; t < jb.n_tok; ++t)   // the g_real rows of one query token are contiguous
-          bulk_load(&sl.q[t * g_real][0], q + row_offset(w.head, t * g_real), q_bytes / jb.n_tok, &bars.item_full[slot]);
+        constexpr uint32_t q_bytes = kQBytes, mean_bytes = 2 * D * sizeof(float);
+        const bool q_now = !(seq == 0 && q_issued);   // the first item's query rows are on their way already
+        mbar_arrive_expect_tx(&bars.item_full[slot], (q_now ? q_bytes : 0u) + (seed ? mean_bytes : 0u));
+        if (q_now)
+          for (int t = 0; t < jb.n_tok; ++t)   // the g_real rows of one query token are contiguous
+            bulk_load(&sl.q[t * g_real][0], q + row_offset(w.head, t * g_real), q_bytes / jb.n_tok, &bars.item_full[slot]);
         if (seed) bulk_load(&sl.mean[0][0], dv.comp_mean + hs * 2 * D, mean_bytes, &bars.item_full[slot]);
       }
       seq_issued = seq + 1;
@@ -554,7 +595,7 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
       WorkItem w_next = no_item;
       bool have_next = false;
       int32_t pid_cur = pid_first;
-      for (int p0 = 0; p0 < n_pad; p0 += batch) {
+      for (int p0 = p_first; p0 < n_pad; p0 += batch) {
         const int in_batch = min(batch, n_pad - p0);
         const bool mine = lane < in_batch;
         const bool real = mine && p0 + lane < n;
@@ -870,12 +911,55 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
           acc[j].scale(l_tot[j] > 0.f ? 1.f / l_tot[j] : 0.f);
           acc[j].store(out + row_offset(d.head, j), lane);
         }
-      } else {                // one of several parts: its record, for the combine kernel
+      } else {                // one of several parts: its record
 #pragma unroll
         for (int j = 0; j < G; ++j) {
           const size_t r = (size_t)(d.rec_base + d.part_idx) * G + j;
           if (lane == 0) dv.rec_ml[r] = make_float2(m_tot[j], l_tot[j]);
           acc[j].store(dv.rec_o + r * D, lane);
+        }
+        if (d.n_parts <= kMergeInKernelMaxParts) {
+          // A head in few parts is finished here, by whichever part is written last: every part publishes its
+          // record (fence), then takes a ticket; the holder of the last ticket sees all records and folds them
+          // in part order, so the result does not depend on who that is.  Nobody waits for anybody.
+          __threadfence();
+          __syncwarp();
+          int ticket = 0;
+          if (lane == 0) ticket = atomicAdd(dv.tickets + d.head, 1);
+          ticket = __shfl_sync(0xffffffffu, ticket, 0);
+          if (ticket == d.n_parts - 1) {
+            if (lane == 0) dv.tickets[d.head] = 0;   // at rest again for the next launch
+            __threadfence();
+#pragma unroll
+            for (int j = 0; j < G; ++j) {
+              float2 ml[kMergeInKernelMaxParts];
+              LaneVec<D> rows[kMergeInKernelMaxParts];
+#pragma unroll
+              for (int p = 0; p < kMergeInKernelMaxParts; ++p) {
+                const size_t r = (size_t)(d.rec_base + min(p, d.n_parts - 1)) * G + j;   // beyond the end: re-read, unused
+                ml[p] = __ldcg(&dv.rec_ml[r]);
+                rows[p].load_l2(dv.rec_o + r * D, lane);
+              }
+              float mx = -CUDART_INF_F;
+#pragma unroll
+              for (int p = 0; p < kMergeInKernelMaxParts; ++p)
+                if (p < d.n_parts) mx = fmaxf(mx, ml[p].x);
+              const float mu = (mx == -CUDART_INF_F) ? 0.f : mx;
+              float lt = 0.f;
+              LaneVec<D> sum;
+              sum.zero();
+#pragma unroll
+              for (int p = 0; p < kMergeInKernelMaxParts; ++p) {
+                if (p < d.n_parts) {
+                  const float cw = fast_exp2(ml[p].x - mu);
+                  lt += ml[p].y * cw;
+                  sum.fma(cw, rows[p]);
+                }
+              }
+              sum.scale(lt > 0.f ? 1.f / lt : 0.f);
+              sum.store(out + row_offset(d.head, j), lane);
+            }
+          }
         }
       }
     }
@@ -885,11 +969,12 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
 
 // ------------------------------------------------------------------------------------------ combine
 // Merges the partial records of the heads that were cut into several parts (Eq. 5 regrouped: sums of
-// exponentials under a common maximum).  One CTA per (such head, query head of its group); warp w folds
+// exponentials under a common maximum).  One CTA per (such head, query row of its tile); warp w folds
 // records w, w + 16, ... in that order and the warp states are folded in warp order, so the result
-// does not depend on timing.  Launched as a programmatic dependent of the streaming kernel: its CTAs
-// may become resident while that kernel drains, and wait for all of its writes at
-// cudaGridDependencySynchronize().
+// does not depend on timing.  Launched as a programmatic dependent of the streaming kernel: its CTAs become
+// resident as that kernel's CTAs leave and wait for all of its writes at cudaGridDependencySynchronize().
+// (CTAs small enough to sit beside a streaming CTA were tried - four warps, 2 KB of shared memory, the same
+// shared-memory split requested: they still only started as streaming CTAs left, and took three times as long.)
 constexpr int kCombineWarps = 16;
 
 template <int D>
@@ -900,7 +985,7 @@ __global__ void __launch_bounds__(kCombineWarps * 32) combine_kernel(DeviceView 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int G = dv.group * n_tok, j = blockIdx.y;   // rows per KV head: query tokens x query heads of the group
   const MultiHead mh = dv.multi[(size_t)layer * dv.n_heads + blockIdx.x];   // uploaded before either kernel
-  cudaTriggerProgrammaticLaunchCompletion();   // a decode kernel queued behind this one may set itself up
+  cudaTriggerProgrammaticLaunchCompletion();   // whatever is queued behind this kernel may set itself up
   cudaGridDependencySynchronize();   // the streaming kernel's records are complete and visible from here on
   float m = -CUDART_INF_F, l = 0.f;
   LaneVec<D> acc;

@@ -13,6 +13,10 @@ namespace razor {
 
 constexpr int kPageTokens = 16;        // tokens per page
 constexpr int kMaxGroup = 8;           // query heads per KV head
+// A head cut into at most this many parts is finished inside the streaming kernel: whichever of its parts is
+// written last (an atomic ticket, nobody waits) folds the head's partial records, in part order.  Heads in more
+// parts are left to the combine kernel that follows.
+constexpr int kMergeInKernelMaxParts = 8;
 constexpr int kCompressMaxSlices = 512;    // row slices per (sequence, KV head) in the compression kernel
 constexpr int kCompressSliceBudget = 8192; // slice sums a call may produce beyond one per head (sizes the scratch)
 
@@ -124,7 +128,8 @@ enum : int32_t {
   kStatusConsumerTimeout = 2,   // a streaming warp gave up waiting for a page or an item
   kStatusReducerTimeout = 4,    // the merging warp gave up waiting for the streaming warps' states
   kStatusDrainTimeout = 8,      // copies were still in flight when the abort path stopped waiting for them
-  kStatusSelfTest = 16          // razor_cache_wait_selftest: the deliberately unanswered wait gave up, as it must
+  kStatusSelfTest = 16,         // razor_cache_wait_selftest: the deliberately unanswered wait gave up, as it must
+  kStatusEarlyMismatch = 32     // a CTA was told to prefetch more pages than its first work item turned out to have
 };
 
 // Pointers into the caller's workspace, plus the dimensions the kernels need.
@@ -140,6 +145,7 @@ struct DeviceView {
   float2* rec_ml;           // [max_items][G]      running max (log2 domain) and denominator of a partial
   float* rec_o;             // [max_items][G][D]   un-normalised numerator of a partial
   int32_t* queue;           // [4]: next item, CTAs done, spare, spare (zero at rest)
+  int32_t* tickets;         // [B*Hkv]: parts of the head written so far in the running decode launch (zero at rest)
   int32_t* status;          // [1]: kStatus* bits, sticky until razor_cache_device_status clears them
   float* compress_scratch;  // [kCompressSliceBudget + B*Hkv][2][D]: slice s of head h of a call at h_in_call * n_slices + s
   HeadPlan* plan;           // [B*Hkv]  heads of the compression call in flight
@@ -166,6 +172,7 @@ struct DecodeTuning {
   int32_t ring_kb;          // shared-memory page ring per CTA, KiB (0: as large as fits)
   int32_t consumer_warps;   // 0: default for the group size
   int32_t tensor_cores;     // grouped bf16 heads: 0 auto (group >= 4), 1 on (group >= 2), 2 off
+  int32_t early_prefetch;   // most pages a span CTA copies ahead of the launch dependency (0: none)
 };
 
 // Records the code razor_last_cuda_error() reports (per thread) and clears the runtime's sticky-free error state.
@@ -186,6 +193,7 @@ cudaError_t launch_append_many(const DeviceView& dv, int dtype, int layer, const
                                int n_tok, int n_slices, cudaStream_t stream);
 // What a decode launch pulls from the queue: n_jobs jobs, the first n_spans of them spans (item
 // ranges jobs[j]..jobs[j+1]), the others single items starting at tail_first.
+constexpr int kEarlyCtas = 160;   // CTAs that can be told how far to prefetch ahead of the launch dependency
 struct DecodeJobs {
   int32_t n_items, n_jobs, n_spans, tail_first;
   int32_t n_multi;   // heads in several parts
@@ -195,6 +203,11 @@ struct DecodeJobs {
   // tokens of the round that come after the block (they are cached already, and masked).
   int32_t tok_stride;
   int32_t q_after;
+  // early[i]: how many of the first pages of CTA i's span (pages of the span's first work item, in order) may
+  // be copied into the ring BEFORE the kernel waits for the launch it depends on.  The host knows every head's
+  // length and which page the preceding append (if any) wrote, so it can name pages that nothing in flight
+  // writes.  0: none.  Only the first kEarlyCtas CTAs take part.
+  uint8_t early[kEarlyCtas];
 };
 cudaError_t launch_decode(const DeviceView& dv, int dtype, int layer, const DecodeJobs& jobs, const void* q,
                           float* out, int n_sms, const DecodeTuning& tune, cudaStream_t stream);

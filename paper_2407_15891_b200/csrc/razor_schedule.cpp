@@ -12,8 +12,9 @@
 //     self-scheduling): each is 1 / tail_items_per_cta of an equal share of the tail that is left, but
 //     not less than min_chunk pages, so the queue ends on small items without starting on them.
 // A job is what a CTA pops from the queue: a span (several consecutive items) or one tail item.
-// A head cut into several parts produces one partial (m, l, o) record per part; a small combine kernel
-// that follows the streaming kernel merges them, one CTA per such head.
+// A head cut into several parts produces one partial (m, l, o) record per part.  Heads in few parts are merged
+// by the streaming kernel itself (the part written last folds them); a small combine kernel that follows it
+// merges the others, one CTA per such head.
 #include <algorithm>
 #include <cstdint>
 #include <numeric>
@@ -97,7 +98,8 @@ int build_schedule(const int32_t* pages, int n_heads, const SchedParams& sp, int
     const int h = order[oi];
     if (n_parts[h] < 2) continue;
     rec_base[h] = rec;
-    multi[n_multi++] = MultiHead{h, rec, n_parts[h], 0};
+    // heads in few parts are folded by the streaming kernel itself; only the others go on the combine kernel's list
+    if (n_parts[h] > kMergeInKernelMaxParts) multi[n_multi++] = MultiHead{h, rec, n_parts[h], 0};
     rec += n_parts[h];
   }
   // Job order: spans in stream order, then the tail items.  Jobs are numbered along the stream, so the
