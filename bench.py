@@ -278,7 +278,7 @@ def _workload_config(w, args):
                         f"head_dim {w.head_dim}, context {min(w.ctx_len)}..{max(w.ctx_len)}, {w.dtype} K/V, "
                         f"{w.n_retrieval_kv} retrieval KV heads per layer, n_sink {w.n_sink}, window "
                         f"{min(w.window)}..{max(w.window)}, {w.decode_steps} decode steps per pass",
-            "step": "compress all layers + decode_steps x layers x (append + decode attention)",
+            "step": "compress all layers + decode_steps x layers x razor_decode_step (append + decode attention in one launch)",
             "l2": "inputs larger than L2 (every launch streams > 126 MB of distinct cache pages)",
             "dense_input": "one seeded dense layer buffer resident in HBM, reused for every layer"}
 
@@ -343,12 +343,12 @@ def decode_only(rz, synth, name, n_layers, dev, peak, reps=60, n_tok=1, alibi=Fa
         k_new, v_new = synth.make_new_kv(w, 0, 0, dev)
         steps = 3
         for l in range(n_layers):                      # (max_new_tokens of this cache is steps + 1)
-            cache.append(l, k_new, v_new); call(l, q, out)
+            cache.decode_step(l, k_new, v_new, q, out)
         torch.cuda.synchronize()
         a.record()
         for _ in range(steps - 1):
             for l in range(n_layers):
-                cache.append(l, k_new, v_new); call(l, q, out)
+                cache.decode_step(l, k_new, v_new, q, out)
         b.record()
         torch.cuda.synchronize()
         us_p = a.elapsed_time(b) * 1e3 / ((steps - 1) * n_layers)
@@ -358,8 +358,8 @@ def decode_only(rz, synth, name, n_layers, dev, peak, reps=60, n_tok=1, alibi=Fa
                               "frac_of_measured": kept_p / (us_p * 1e-6) / 1e9 / peak,
                               "frac_of_nominal_8TBs": kept_p / (us_p * 1e-6) / 1e9 / NOMINAL_HBM_GBS,
                               "launches_timed": (steps - 1) * n_layers,
-                              "note": "per layer: razor_append + razor_decode_attention, all layers of the "
-                                      "configuration, CUDA events at the ends of the run only"}
+                              "note": "per layer: one razor_decode_step call (append + decode attention), all layers "
+                                      "of the configuration, CUDA events at the ends of the run only"}
     res["device_status"] = cache.device_status()
     cache.close()
     return res
@@ -484,7 +484,7 @@ def main():
     per_seq = w.name == "cfg5"
 
     retr = [w.retrieval(l) for l in range(L)]
-    cfg = rz.make_config(w.batch, L, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, w.n_sink, max(w.ctx_len), T)
+    cfg = rz.make_config(w.batch, L, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, w.n_sink, max(w.ctx_len), T + 4)
     cache = rz.RazorCache(cfg, w.ctx_len, w.window, np.stack(retr), device=dev)
 
     # inputs, resident in HBM before the timed region
@@ -525,9 +525,17 @@ def main():
             k_new, v_new = kvs[t % n_q]
             q = qs[t % n_q]
             for l in range(L):
-                cache.append(l, k_new, v_new)
-                cache.decode(l, q, out)
-                launches["n"] += 3        # append, streaming decode kernel, combine kernel
+                cache.decode_step(l, k_new, v_new, q, out)      # append + decode attention, one launch
+                launches["n"] += 1 + combine_launched(l)        # streaming kernel (+ combine kernel for heads in many parts)
+
+    combine_cache = {}
+
+    def combine_launched(l):
+        """1 when the layer's schedule has a head in more parts than the streaming kernel folds itself."""
+        if l not in combine_cache:
+            items = rz.razor_schedule_query(cache.handle, l)
+            combine_cache[l] = int((items[:, 3] > max(1, 16 // w.group)).any())
+        return combine_cache[l]
 
     def sync_all():
         torch.cuda.synchronize()
@@ -589,8 +597,8 @@ def main():
                 "frac_of_nominal_8TBs": dec_gbs / NOMINAL_HBM_GBS,
                 "alg_bytes_per_launch": alg_per_launch, "us_per_launch": us_per_launch,
                 "launches_timed": n_dec * args.steps,
-                "how": "decode phase of the timed passes / its launches, CUDA events at the ends of the phase only; "
-                       "the phase includes the razor_append kernels",
+                "how": "decode phase of the timed passes / its razor_decode_step calls (append + decode attention in one "
+                       "launch), CUDA events at the ends of the phase only",
                 "traffic": (ratio * alg_per_launch) if ratio else None, "traffic_source": ratio_src}
 
     line = {
@@ -633,11 +641,20 @@ def main():
     kept_now = statistics.mean(compressed_bytes(w, l, extra=T) for l in range(L))
     line["decode"]["us_per_layer_back_to_back_no_append"] = dec_alone_us
     line["decode"]["gbs_back_to_back_no_append"] = kept_now / (dec_alone_us * 1e-6) / 1e9
+    # the same step as two calls (razor_append, then razor_decode_attention)
+    a.record()
+    for t in range(2):
+        for l in range(L):
+            cache.append(l, kvs[t % n_q][0], kvs[t % n_q][1])
+            cache.decode(l, qs[t % n_q], out)
+    b.record()
+    sync_all()
+    line["decode"]["us_per_layer_as_two_calls"] = a.elapsed_time(b) * 1e3 / (2 * L)
     line["append"] = {"us_per_layer_in_pass": us_per_launch - dec_alone_us,
                       "us_per_call_back_to_back": app_us, "launches_timed": T * L,
-                      "note": "in the pass: (append + decode) per layer minus a decode call timed back to back without "
-                              "appends; back to back: razor_append calls alone, one token per (sequence, KV head), "
-                              "bound by the host's launch rate"}
+                      "note": "in the pass: a razor_decode_step call minus a razor_decode_attention call timed back to back "
+                              "without appends; back to back: razor_append calls alone, one token per (sequence, KV "
+                              "head), bound by the host's launch rate"}
 
     # ------------------------------------------------------------------ dense full-cache decode, same GPU
     if not args.no_dense and rank == 0 and not per_seq:
@@ -720,8 +737,7 @@ def main():
                     d_q.copy_(h_q[t % n_q], non_blocking=True)
                     d_k.copy_(h_kv[t % n_q][0], non_blocking=True)
                     d_v.copy_(h_kv[t % n_q][1], non_blocking=True)
-                    cache.append(l, d_k, d_v)
-                    cache.decode(l, d_q, out)
+                    cache.decode_step(l, d_k, d_v, d_q, out)
                     h_out.copy_(out, non_blocking=True)
                     if count:
                         h2d += (d_q.numel() + 2 * d_k.numel()) * d_q.element_size()

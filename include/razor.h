@@ -155,6 +155,20 @@ RAZOR_API int razor_append(razor_cache_t* cache, int32_t layer, const void* k_ne
 RAZOR_API int razor_decode_attention(razor_cache_t* cache, int32_t layer, const void* q, float* out, void* stream);
 
 /*
+ * One decode step of a layer in a single launch: razor_append(k_new, v_new) followed by
+ * razor_decode_attention(q, out), with the same arguments, the same result for `out` and the same cache
+ * state afterwards (Algorithm 1 + Eq. 4 for the new token, Eq. 5 for the attention).  The streaming kernel
+ * itself stores the new rows: the part of a head that holds the row's page puts the row into its copy of
+ * the page and into the pool, folds the evicted row into the compensation sums when the window is full,
+ * and the head states advance when the last CTA has finished.  This removes the append kernel, and the
+ * wait for it, from every decode step.  k_new, v_new and q are read only after the kernel before this call
+ * on the stream has completed.
+ * Errors: as razor_append and razor_decode_attention.
+ */
+RAZOR_API int razor_decode_step(razor_cache_t* cache, int32_t layer, const void* k_new, const void* v_new,
+                                const void* q, float* out, void* stream);
+
+/*
  * A round of several new tokens per sequence (a second prompt chunk, a speculative-decoding verify
  * step).  The paper runs Algorithm 1 once on the prompt and says nothing about such rounds; the
  * reading taken extends the single-token rule.

@@ -26,7 +26,7 @@ STATUS = {
 # every symbol include/razor.h declares
 SYMBOLS = [
     "razor_query_bytes", "razor_cache_create", "razor_compress", "razor_compress_seq", "razor_append",
-    "razor_decode_attention", "razor_append_many", "razor_append_plan", "razor_decode_attention_multi", "razor_cache_export", "razor_cache_stats", "razor_schedule_plan",
+    "razor_decode_attention", "razor_decode_step", "razor_append_many", "razor_append_plan", "razor_decode_attention_multi", "razor_cache_export", "razor_cache_stats", "razor_schedule_plan",
     "razor_schedule_query", "razor_cache_set_option", "razor_cache_device_status", "razor_cache_wait_selftest", "razor_cache_set_alibi", "razor_cache_set_head_windows",
     "razor_compensation_mean_static", "razor_head_scores_scratch_bytes", "razor_head_scores",
     "razor_select_retrieval_heads", "razor_cache_reset", "razor_cache_destroy", "razor_status_string",
@@ -72,6 +72,7 @@ def load() -> C.CDLL:
     lib.razor_compress_seq.argtypes = [vp, i32, i32, vp, vp, i64, i64, i32, vp, i32, i32, vp]
     lib.razor_append.argtypes = [vp, i32, vp, vp, vp]
     lib.razor_decode_attention.argtypes = [vp, i32, vp, vp, vp]
+    lib.razor_decode_step.argtypes = [vp, i32, vp, vp, vp, vp, vp]
     lib.razor_append_many.argtypes = [vp, i32, vp, vp, i32, vp]
     lib.razor_append_plan.argtypes = [i32, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp]
     lib.razor_decode_attention_multi.argtypes = [vp, i32, vp, vp, i32, vp]
@@ -187,6 +188,11 @@ def razor_append(cache: int, layer: int, k_new, v_new, stream=None) -> None:
 def razor_decode_attention(cache: int, layer: int, q, out, stream=None) -> None:
     _check(load().razor_decode_attention(cache, layer, _ptr(q), _ptr(out), _stream(stream)),
            "razor_decode_attention")
+
+
+def razor_decode_step(cache: int, layer: int, k_new, v_new, q, out, stream=None) -> None:
+    _check(load().razor_decode_step(cache, layer, _ptr(k_new), _ptr(v_new), _ptr(q), _ptr(out), _stream(stream)),
+           "razor_decode_step")
 
 
 def razor_append_many(cache: int, layer: int, k_new, v_new, n_tokens: int, stream=None) -> None:
@@ -376,6 +382,15 @@ class RazorCache:
         if out is None:
             out = torch.empty(q.shape, dtype=torch.float32, device=q.device)
         razor_decode_attention(self.handle, layer, q, out)
+        return out
+
+    def decode_step(self, layer: int, k_new: torch.Tensor, v_new: torch.Tensor, q: torch.Tensor,
+                    out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """append(k_new, v_new) + decode(q) in one launch."""
+        assert k_new.is_contiguous() and v_new.is_contiguous() and q.is_contiguous()
+        if out is None:
+            out = torch.empty(q.shape, dtype=torch.float32, device=q.device)
+        razor_decode_step(self.handle, layer, k_new, v_new, q, out)
         return out
 
     def append_many(self, layer: int, k_new: torch.Tensor, v_new: torch.Tensor) -> None:

@@ -103,7 +103,7 @@ struct LayerHost {
   int appended = 0;
   // decode schedule
   bool sched_valid = false;
-  int n_items = 0, n_jobs = 0, n_spans = 0, n_multi = 0, chunk_pages = 0, growth_tokens = 0;
+  int n_items = 0, n_jobs = 0, n_spans = 0, n_multi = 0, chunk_pages = 0, growth_tokens = 0, sched_rows = 0;
   WorkItem* items = nullptr;        // pinned host, [max_items]
   int32_t* jobs = nullptr;          // pinned host, [max_items + 1]
   MultiHead* multi = nullptr;       // pinned host, [B*Hkv]
@@ -335,6 +335,8 @@ struct SeqIn {
   int n_ctx, window;
 };
 
+int ensure_schedule(razor_cache* c, int layer, cudaStream_t stream, bool upload, int rows);
+
 // Shared body of razor_compress / razor_compress_seq: the plan (C0), page allocation, uploads, launch.
 int compress_impl(razor_cache* c, int layer, const std::vector<SeqIn>& seqs, const uint8_t* retr, int n_sink,
                   cudaStream_t stream) {
@@ -501,20 +503,27 @@ int compress_impl(razor_cache* c, int layer, const std::vector<SeqIn>& seqs, con
   L.any = true;
   L.appended = 0;
   L.sched_valid = false;
+  // With the layer complete, its decode schedule is planned and sent to the device here, behind the compression
+  // kernels, rather than in front of the layer's first decode launch, where the copies would sit between two
+  // kernels that otherwise overlap.  (A failure here is not an error of the compression: the decode call plans again.)
+  if (L.n_done == cfg.batch) (void)ensure_schedule(c, layer, stream, true, cfg.n_q_heads / cfg.n_kv_heads);
   return RAZOR_OK;
 }
 
-int ensure_schedule(razor_cache* c, int layer, cudaStream_t stream, bool upload) {
+int ensure_schedule(razor_cache* c, int layer, cudaStream_t stream, bool upload, int rows) {
   LayerHost& L = c->layers[layer];
-  const bool stale = !L.sched_valid || (long long)L.growth_tokens * 4 >= (long long)L.chunk_pages * kPageTokens;
+  // (which heads the streaming kernel folds itself depends on the rows of a KV head's tile in this launch)
+  const bool stale = !L.sched_valid || L.sched_rows != rows || (long long)L.growth_tokens * 4 >= (long long)L.chunk_pages * kPageTokens;
   if (!stale) return RAZOR_OK;
   const int nh = c->dv.n_heads;
   std::vector<int32_t> pages(nh);
   for (int h = 0; h < nh; ++h) pages[h] = ceil_div(L.hs[h].len, kPageTokens);
   if (L.upload_done) RZ_CUDA(cudaEventSynchronize(L.upload_done));   // previous upload has left the staging area
-  const SchedParams sp{c->n_sms, c->tune.static_pct, c->tune.tail_items_per_sm, c->tune.min_chunk_pages};
+  const SchedParams sp{c->n_sms, c->tune.static_pct, c->tune.tail_items_per_sm, c->tune.min_chunk_pages,
+                       std::min((int)kMergeInKernelMaxParts, merge_in_kernel_max_parts(rows))};
   SchedInfo info{};
   const int n = build_schedule(pages.data(), nh, sp, c->lay.max_items, L.items, L.jobs, L.multi, &info);
+  L.sched_rows = rows;
   if (n < 0) return RAZOR_E_INVALID_ARG;
   L.n_items = n;
   L.n_jobs = info.n_jobs;
@@ -673,22 +682,30 @@ int razor_append_plan(int32_t len, int32_t n_drop, int32_t ring_head, int32_t wi
 }
 
 static int decode_impl(razor_cache_t* c, int32_t layer, const void* q, float* out, int32_t n_tokens,
-                       int32_t tok_stride, int32_t q_after, void* stream);
+                       int32_t tok_stride, int32_t q_after, void* stream, const void* k_new = nullptr,
+                       const void* v_new = nullptr);
 
 // Which pages a span CTA may copy before the decode kernel waits for the launch it depends on.  While that part
-// of the kernel runs, the library kernels launched since the previous decode may still be writing.  If none of
-// them wrote this layer, every page of it is stable.  If exactly one did and it was a single-token append, the
-// only page of a head it writes is the one holding the appended row, and the host mirror says which: the slot
-// before `len` for a head that grew, the ring slot before ring_head for a head that evicted.  Anything else
-// (a bulk append, a compression, several appends): no early copies.  For CTA i the count covers the leading
-// pages of its span's first work item, cut at the written page and at the item's length as it is now.
+// of the kernel runs, the library kernels launched since the previous decode (and that decode itself, when it
+// appended a token) may still be writing.  If none of them wrote this layer, every page of it is stable.  If the
+// only writes were single-token appends, at most two of them, the only pages they write are the ones holding the
+// rows appended last, and the host mirror says which: the slots before `len` for a head that grew, the ring slots
+// before ring_head for a head that evicted.  Anything else (a bulk append, a compression, more appends): no early
+// copies.  For CTA i the count covers the leading pages of its span's first work item, cut at the first such
+// page and at the item's length as it is now.
 static void plan_early_prefetch(const razor_cache* c, int layer, DecodeJobs& jb) {
   std::memset(jb.early, 0, sizeof(jb.early));
-  if (!c->tune.early_prefetch || c->writes_overflow) return;
-  int n_writes = 0, kind = 0;
-  for (const auto& wr : c->writes_since_decode)
-    if (wr.first == layer) { n_writes += 1; kind = wr.second; }
-  if (n_writes > 1 || (n_writes == 1 && kind != razor_cache::kWriteOneToken)) return;
+  if (c->tune.early_prefetch <= 0 || c->writes_overflow) return;
+  int n_writes = 0;
+  for (const auto& wr : c->writes_since_decode) {
+    if (wr.first != layer) continue;
+    if (wr.second != razor_cache::kWriteOneToken) return;
+    n_writes += 1;
+  }
+  if (n_writes > 2) return;
+  // rows written by appends that may be in flight: the newest n_writes ones; one more is left out for good
+  // measure (in a launch that appends itself the mirror is already one token ahead)
+  const int n_recent = n_writes > 0 || jb.k_new ? n_writes + 1 : 0;
   const LayerHost& L = c->layers[layer];
   const int n_sink = c->cfg.n_sink;
   const int n = std::min({L.n_spans, c->n_sms, (int)kEarlyCtas});
@@ -698,10 +715,15 @@ static void plan_early_prefetch(const razor_cache* c, int layer, DecodeJobs& jb)
     const int head_pages = ceil_div(st.len, kPageTokens);
     const int page_end = w.page_end < 0 ? head_pages : std::min(w.page_end, head_pages);
     int e = std::min(c->tune.early_prefetch, std::max(0, page_end - w.page_begin));
-    if (n_writes == 1) {
-      int slot = -1;   // slot the append wrote
-      if (st.window < 0 || st.n_drop == 0) slot = st.len - 1;                                  // the head grew
-      else if (st.window > 0) slot = n_sink + (st.ring_head + st.window - 1) % st.window;       // it evicted
+    for (int j = 0; j < n_recent && e > 0; ++j) {
+      int slot = -1;   // slot of the (j + 1)-th newest row
+      if (st.window < 0 || st.n_drop == 0) {
+        slot = st.len - 1 - j;                                                   // the head grew
+      } else if (st.window > 0) {
+        if (st.n_drop <= j) { e = 0; break; }                                    // it only just began to evict: leave it
+        const long long r = ((long long)st.ring_head - 1 - j) % st.window;
+        slot = n_sink + (int)(r < 0 ? r + st.window : r);
+      }
       if (slot >= 0) {
         const int tp = slot / kPageTokens - w.page_begin;
         if (tp >= 0 && tp < e) e = tp;
@@ -748,19 +770,62 @@ int razor_decode_attention(razor_cache_t* c, int32_t layer, const void* q, float
 }
 
 static int decode_impl(razor_cache_t* c, int32_t layer, const void* q, float* out, int32_t n_tokens,
-                       int32_t tok_stride, int32_t q_after, void* stream) {
+                       int32_t tok_stride, int32_t q_after, void* stream, const void* k_new, const void* v_new) {
   int rc;
   if (((uintptr_t)q | (uintptr_t)out) & 15) return RAZOR_E_MISALIGNED;
-  rc = ensure_schedule(c, layer, (cudaStream_t)stream, true);
+  rc = ensure_schedule(c, layer, (cudaStream_t)stream, true, (c->cfg.n_q_heads / c->cfg.n_kv_heads) * n_tokens);
   if (rc) return rc;
   const LayerHost& L = c->layers[layer];
-  DecodeJobs jb{L.n_items, L.n_jobs, L.n_spans, L.jobs[L.n_spans], L.n_multi, n_tokens, tok_stride, q_after, {}};
+  DecodeJobs jb{L.n_items, L.n_jobs, L.n_spans, L.jobs[L.n_spans], L.n_multi, n_tokens, tok_stride, q_after, {},
+                k_new, v_new};
   plan_early_prefetch(c, layer, jb);
   RZ_CUDA(launch_decode(c->dv, c->cfg.dtype, layer, jb, q, out, c->n_sms, c->tune,
                         (cudaStream_t)stream));
   c->last_writer_layer = -1;
   c->writes_since_decode.clear();
   c->writes_overflow = false;
+  return RAZOR_OK;
+}
+
+int razor_decode_step(razor_cache_t* c, int32_t layer, const void* k_new, const void* v_new, const void* q, float* out,
+                      void* stream) {
+  if (!c || !k_new || !v_new || !q || !out) return RAZOR_E_NULL_PTR;
+  int rc = layer_ready(c, layer);
+  if (rc) return rc;
+  if (((uintptr_t)k_new | (uintptr_t)v_new) & 15) return RAZOR_E_MISALIGNED;
+  LayerHost& L = c->layers[layer];
+  if (L.appended >= c->cfg.max_new_tokens) return RAZOR_E_CAPACITY;
+  // A head with no recent window at all drops the new token at once (nothing is stored, only the sums change):
+  // that corner stays with the two separate kernels.
+  bool plain = false;
+  for (const HeadState& h : L.hs) plain |= (h.window == 0);
+  if (plain) {
+    rc = razor_append(c, layer, k_new, v_new, stream);
+    return rc ? rc : razor_decode_attention(c, layer, q, out, stream);
+  }
+  // The host mirror moves first (the schedule and the early copies are planned for the lengths the launch
+  // will see) and moves back if the launch fails.
+  const std::vector<HeadState> before = L.hs;
+  const int n_sink = c->cfg.n_sink;
+  for (HeadState& h : L.hs) {
+    if (h.window < 0 || h.len < n_sink + h.window) {
+      h.len += 1;
+    } else {
+      h.n_drop += 1;
+      h.ring_head = (h.ring_head + 1 == h.window) ? 0 : h.ring_head + 1;
+    }
+  }
+  L.appended += 1;
+  L.growth_tokens += 1;
+  rc = decode_impl(c, layer, q, out, 1, 1, 0, stream, k_new, v_new);
+  if (rc) {
+    L.hs = before;
+    L.appended -= 1;
+    L.growth_tokens -= 1;
+    L.sched_valid = false;
+    return rc;
+  }
+  c->note_write(layer, razor_cache::kWriteOneToken);   // the launch stores the new rows late: the next one must leave them alone
   return RAZOR_OK;
 }
 
@@ -816,7 +881,7 @@ int razor_schedule_plan(const int32_t* tokens, int32_t n_heads, int32_t n_ctas, 
   std::vector<WorkItem> w(cap);
   std::vector<int32_t> jobs(cap + 1);
   std::vector<MultiHead> multi(n_heads);
-  const SchedParams sp{n_ctas, static_percent, tail_items_per_cta, min_chunk_pages};
+  const SchedParams sp{n_ctas, static_percent, tail_items_per_cta, min_chunk_pages, kMergeInKernelMaxParts};
   SchedInfo info{};
   const int n = build_schedule(pages.data(), n_heads, sp, cap, w.data(), jobs.data(), multi.data(), &info);
   if (n < 0) return RAZOR_E_INVALID_ARG;
@@ -921,7 +986,7 @@ int razor_schedule_query(razor_cache_t* c, int32_t layer, int32_t* items, int32_
   if (!c || !n_items) return RAZOR_E_NULL_PTR;
   int rc = layer_ready(c, layer);
   if (rc) return rc;
-  rc = ensure_schedule(c, layer, nullptr, false);
+  rc = ensure_schedule(c, layer, nullptr, false, c->cfg.n_q_heads / c->cfg.n_kv_heads);
   if (rc) return rc;
   const LayerHost& L = c->layers[layer];
   return emit_items(L.items, L.n_items, L.jobs, L.n_jobs, items, max_items, n_items);

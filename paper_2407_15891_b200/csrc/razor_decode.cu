@@ -66,14 +66,21 @@ struct ItemDesc {
   int32_t seed;        // 1: this part starts from the compensation token
   int32_t n_drop;
   int32_t window;      // recent-window length, < 0: the head keeps everything
-  int32_t pad1;
+  // a launch that also appends a token: the part that holds the page the new row goes to stores it
+  int32_t tp_index;    // that page, counted from page_begin; -1: not in this part (or nothing is appended)
+  int32_t tp_slot;     // slot of the new row
+  int32_t tp_pid;      // pool page of that slot
+  int32_t fold;        // 1: the slot holds the oldest recent token, which joins the dropped set first (Eq. 4)
+  int32_t merge_here;  // 1: the part that is written last folds the head's records itself
 };
 
 template <typename T, int D, int G>
 struct alignas(16) ItemSlot {
   ItemDesc desc;
   alignas(16) T q[G][D];
-  alignas(16) float mean[2][D];   // k_hat, v_hat
+  alignas(16) float mean[2][D];   // k_hat, v_hat (a part that folds a row receives the sums here and turns them into means)
+  alignas(16) T new_kv[2][D];     // the appended K and V row, for the part that stores it
+  alignas(16) T old_kv[2][D];     // the row it evicts, as it lies in its page (16-byte chunks swizzled)
 };
 
 struct Barriers {
@@ -366,6 +373,45 @@ __device__ __forceinline__ void consume_page_mma(uint32_t page_addr, int valid, 
   }
 }
 
+// The part of a launch-that-appends which evicts a row: sums so far (in mean[]) + the evicted row -> new sums
+// and means (Eq. 4 over every token dropped so far), stored for later launches and left in mean[] for the
+// seed below.  Same arithmetic, in the same order, as the append kernel's.  One warp, D / 32 elements per lane.
+template <typename T, int D>
+__device__ __forceinline__ void fold_evicted_row(float (&mean)[2][D], const T (&old_kv)[2][D], int slot, int n_drop,
+                                                 float* __restrict__ g_sum, float* __restrict__ g_mean, int lane) {
+  constexpr int PER = D / 32, EPC = 16 / (int)sizeof(T);   // elements per lane; elements per 16-byte chunk
+  const float cnt = (float)n_drop;
+#pragma unroll
+  for (int kv = 0; kv < 2; ++kv) {
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+      const int e = lane * PER + i;
+      const int pos = (((e / EPC) ^ (slot & 7)) * EPC) + e % EPC;   // where the page's swizzle put element e
+      const float s = mean[kv][e] + (float)old_kv[kv][pos];
+      const float m = __fdiv_rn(s, cnt);
+      g_sum[kv * D + e] = s;
+      g_mean[kv * D + e] = m;
+      mean[kv][e] = m;
+    }
+  }
+  __syncwarp();
+}
+
+// The appended row into the page that holds its slot: into the copy in shared memory (this launch attends to
+// it) and into the pool (for the launches to come).  Lane c < LPR holds 16-byte chunk c of the K and V row.
+template <int LPR>
+__device__ __forceinline__ void store_new_row(uint8_t* page, uint8_t* pool_page, int slot, const uint4& k, const uint4& v,
+                                              int lane) {
+  if (lane < LPR) {
+    const int t = slot & 15, at = t * LPR + swz(slot, lane);
+    ((uint4*)page)[at] = k;
+    ((uint4*)page)[kPageTokens * LPR + at] = v;
+    ((uint4*)pool_page)[at] = k;
+    ((uint4*)pool_page)[kPageTokens * LPR + at] = v;
+  }
+  __syncwarp();
+}
+
 // Reducer-side vector of D/32 consecutive floats per lane.
 template <int D>
 struct LaneVec;
@@ -432,10 +478,11 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
+  const bool fused = jb.k_new != nullptr;   // this launch also appends a token
   const WorkItem* items = dv.items + (size_t)layer * dv.max_items;
   const int32_t* jobs = dv.jobs + (size_t)layer * (dv.max_items + 1);
   const int n_items = jb.n_items;
-  const WorkItem no_item = {0, 0, 0, 0, 1, 0, 0, 0};
+  const WorkItem no_item = {0, 0, 0, 0, 1, 0, 0, 0};   // (merge_here = 0)
   auto row_of = [&](const WorkItem& w) { return (size_t)layer * dv.n_heads + w.head; };
   auto first_pids = [&](const WorkItem& w) {
     return dv.page_table[row_of(w) * dv.max_pages + min(w.page_begin + lane, dv.max_pages - 1)];
@@ -556,9 +603,26 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
         break;
       }
       const size_t hs = row_of(w);
+      // A launch that appends: `st` becomes the state the append leaves (the stored state stays as it was until
+      // the last CTA of the launch advances every head), tp_slot the slot the new row goes to.
+      int tp_slot = -1;
+      bool evicts = false;
+      if (fused) {
+        if (st.window < 0 || st.len < dv.n_sink + st.window) {
+          tp_slot = st.len;
+          st.len += 1;
+        } else if (st.window > 0) {
+          tp_slot = dv.n_sink + st.ring_head;
+          evicts = true;
+          st.n_drop += 1;
+          st.ring_head = (st.ring_head + 1 == st.window) ? 0 : st.ring_head + 1;
+        }   // (a head with sinks only and no window is not run through this path: the host sees to that)
+      }
       const int head_pages = (st.len + kPageTokens - 1) / kPageTokens;
       const int page_end = w.page_end < 0 ? head_pages : min(w.page_end, head_pages);
       const int n = max(0, page_end - w.page_begin);
+      const int tp_rel = tp_slot >= 0 ? (tp_slot >> 4) - w.page_begin : -1;
+      const bool owns = tp_rel >= 0 && tp_rel < n;   // this part holds the page the new row goes to
       const int p_first = seq == 0 ? (int)early_done : 0;   // pages of this item already on their way
       if (p_first > n) {   // the host's count and the device's lengths disagree: stop rather than mix items up
         if (lane == 0) {
@@ -570,20 +634,37 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
         ok = false;
         break;
       }
-      const bool seed = w.part_idx == 0 && dv.use_comp && st.n_drop > 0 && st.window >= 0;
+      // The compensation token enters the head's first part; in a launch that evicts a row into the sums it
+      // enters the part that holds that row instead, which computes the new mean itself.
+      const bool fold = evicts && owns;
+      const bool seed = dv.use_comp && st.n_drop > 0 && st.window >= 0 && (evicts ? owns : w.part_idx == 0);
       if (lane == 0) {
         ItemDesc d;
         d.head = w.head; d.page_begin = w.page_begin; d.n_pages = n; d.len = st.len;
         d.part_idx = w.part_idx; d.n_parts = w.n_parts; d.rec_base = w.rec_base; d.ring_head = st.ring_head;
-        d.seed = seed ? 1 : 0; d.n_drop = st.n_drop; d.window = st.window; d.pad1 = 0;
+        d.seed = seed ? 1 : 0; d.n_drop = st.n_drop; d.window = st.window; d.merge_here = w.merge_here;
+        d.tp_index = owns ? tp_rel : -1; d.tp_slot = tp_slot; d.fold = fold ? 1 : 0;
+        d.tp_pid = owns ? dv.page_table[hs * dv.max_pages + (tp_slot >> 4)] : 0;
         sl.desc = d;
-        constexpr uint32_t q_bytes = kQBytes, mean_bytes = 2 * D * sizeof(float);
+        constexpr uint32_t q_bytes = kQBytes, mean_bytes = 2 * D * sizeof(float), row_bytes = D * sizeof(T);
         const bool q_now = !(seq == 0 && q_issued);   // the first item's query rows are on their way already
-        mbar_arrive_expect_tx(&bars.item_full[slot], (q_now ? q_bytes : 0u) + (seed ? mean_bytes : 0u));
+        mbar_arrive_expect_tx(&bars.item_full[slot], (q_now ? q_bytes : 0u) + ((seed || fold) ? mean_bytes : 0u) +
+                                                         (owns ? 2 * row_bytes : 0u) + (fold ? 2 * row_bytes : 0u));
         if (q_now)
           for (int t = 0; t < jb.n_tok; ++t)   // the g_real rows of one query token are contiguous
             bulk_load(&sl.q[t * g_real][0], q + row_offset(w.head, t * g_real), q_bytes / jb.n_tok, &bars.item_full[slot]);
-        if (seed) bulk_load(&sl.mean[0][0], dv.comp_mean + hs * 2 * D, mean_bytes, &bars.item_full[slot]);
+        if (fold) {   // the sums so far and the row that leaves the window
+          const uint8_t* old_row = dv.pool + (size_t)d.tp_pid * dv.page_bytes + (size_t)(tp_slot & 15) * row_bytes;
+          bulk_load(&sl.mean[0][0], dv.comp_sum + hs * 2 * D, mean_bytes, &bars.item_full[slot]);
+          bulk_load(&sl.old_kv[0][0], old_row, row_bytes, &bars.item_full[slot]);
+          bulk_load(&sl.old_kv[1][0], old_row + kPageTokens * row_bytes, row_bytes, &bars.item_full[slot]);
+        } else if (seed) {
+          bulk_load(&sl.mean[0][0], dv.comp_mean + hs * 2 * D, mean_bytes, &bars.item_full[slot]);
+        }
+        if (owns) {
+          bulk_load(&sl.new_kv[0][0], (const T*)jb.k_new + (size_t)w.head * D, row_bytes, &bars.item_full[slot]);
+          bulk_load(&sl.new_kv[1][0], (const T*)jb.v_new + (size_t)w.head * D, row_bytes, &bars.item_full[slot]);
+        }
       }
       seq_issued = seq + 1;
       const int32_t* pt = dv.page_table + hs * dv.max_pages + w.page_begin;
@@ -662,11 +743,32 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
     }
     if (!__all_sync(0xffffffffu, drained) && lane == 0) atomicOr(dv.status, kStatusDrainTimeout);
     // Queue reset for the next launch: every CTA has made its last pop before it counts itself done.
+    // In a launch that appends, the stored head states must stay as they were while any CTA still builds
+    // descriptors from them; the CTA that counts itself done last knows that nobody does any more and advances
+    // every head by the append.
+    int done = 0;
     if (lane == 0) {
-      const int done = atomicAdd(dv.queue + 1, 1);
-      if (done == (int)gridDim.x - 1) {
+      __threadfence();
+      done = atomicAdd(dv.queue + 1, 1);
+    }
+    done = __shfl_sync(0xffffffffu, done, 0);
+    if (done == (int)gridDim.x - 1) {
+      if (lane == 0) {
         dv.queue[0] = 0;
         dv.queue[1] = 0;
+      }
+      if (fused) {
+        HeadState* states = dv.state + (size_t)layer * dv.n_heads;
+        for (int h = lane; h < dv.n_heads; h += 32) {
+          HeadState s = states[h];
+          if (s.window < 0 || s.len < dv.n_sink + s.window) {
+            s.len += 1;
+          } else if (s.window > 0) {
+            s.n_drop += 1;
+            s.ring_head = (s.ring_head + 1 == s.window) ? 0 : s.ring_head + 1;
+          }
+          states[h] = s;
+        }
       }
     }
   } else if (warp < NC) {
@@ -680,7 +782,7 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
       const int mb = seq % kMergeBufs;
       MBuf& M = mbufs[mb];
       if (!warp_wait(&bars.item_full[slot], (seq / kItemSlots) & 1)) { ok = false; break; }
-      const Slot& sl = slots[slot];
+      Slot& sl = slots[slot];
       const ItemDesc d = sl.desc;
       if (d.head < 0) {
         // pass the end marker on to the reducer
@@ -712,6 +814,17 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
         MmaState<D> S;
         S.clear();
         const bool first = warp == 0;
+        // a launch that appends: the warp that will meet the new row's page takes the row out of the slot now
+        // (the slot is handed back below), and the first warp folds the evicted row into the sums
+        uint4 new_k = make_uint4(0u, 0u, 0u, 0u), new_v = new_k;
+        if (d.tp_index >= 0 && warp == d.tp_index % NC && lane < LPR) {
+          new_k = ((const uint4*)&sl.new_kv[0][0])[lane];
+          new_v = ((const uint4*)&sl.new_kv[1][0])[lane];
+        }
+        if (d.fold && first) {
+          const size_t hs2 = ((size_t)layer * dv.n_heads + d.head) * 2 * D;
+          fold_evicted_row<T, D>(sl.mean, sl.old_kv, d.tp_slot, d.n_drop, dv.comp_sum + hs2, dv.comp_mean + hs2, lane);
+        }
         // Compensation token (Eq. 4, Eq. 5) seeds the first part of a head that dropped tokens.
         if (d.seed && first) {
           constexpr int PER = D / 32;
@@ -745,6 +858,8 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
           if (!warp_wait(&bars.full[stage], use & 1)) { ok = false; break; }
           if (i < d.n_pages) {
             uint8_t* page = ring + (size_t)stage * PB;
+            if (i == d.tp_index)
+              store_new_row<LPR>(page, dv.pool + (size_t)d.tp_pid * dv.page_bytes, d.tp_slot, new_k, new_v, lane);
             const int valid = d.len - (d.page_begin + i) * kPageTokens;
             if (valid < kPageTokens) {
               // V rows beyond the head's length may hold anything; a zero weight times a NaN is a NaN
@@ -800,6 +915,17 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
         SoftmaxState<G, EPL> S;
         S.clear();
         const bool first = warp == 0;   // the warp that takes the item's first page also takes its seed
+        // a launch that appends: the warp that will meet the new row's page takes the row out of the slot now
+        // (the slot is handed back below), and the first warp folds the evicted row into the sums
+        uint4 new_k = make_uint4(0u, 0u, 0u, 0u), new_v = new_k;
+        if (d.tp_index >= 0 && warp == d.tp_index % NC && lane < LPR) {
+          new_k = ((const uint4*)&sl.new_kv[0][0])[lane];
+          new_v = ((const uint4*)&sl.new_kv[1][0])[lane];
+        }
+        if (d.fold && first) {
+          const size_t hs2 = ((size_t)layer * dv.n_heads + d.head) * 2 * D;
+          fold_evicted_row<T, D>(sl.mean, sl.old_kv, d.tp_slot, d.n_drop, dv.comp_sum + hs2, dv.comp_mean + hs2, lane);
+        }
         // Compensation token (Eq. 4, Eq. 5) seeds the first part of a head that dropped tokens.
         if (d.seed && first) {
           float kh[EPL], vh[EPL];
@@ -829,6 +955,9 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
           ring_slot<NC>(c + i, ns, stage, use);
           if (!warp_wait(&bars.full[stage], use & 1)) { ok = false; break; }
           if (i < d.n_pages) {
+            if (i == d.tp_index)
+              store_new_row<LPR>(ring + (size_t)stage * PB, dv.pool + (size_t)d.tp_pid * dv.page_bytes, d.tp_slot, new_k,
+                                 new_v, lane);
             const RoundMask mk{1, G, dv.alibi, d.len + d.n_drop, 0, dv.n_sink, d.ring_head, d.window, d.n_drop,
                                (d.page_begin + i) * kPageTokens};
             consume_page<T, D, G>((const uint4*)(ring + (size_t)stage * PB), d.len - (d.page_begin + i) * kPageTokens,
@@ -918,7 +1047,7 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
           if (lane == 0) dv.rec_ml[r] = make_float2(m_tot[j], l_tot[j]);
           acc[j].store(dv.rec_o + r * D, lane);
         }
-        if (d.n_parts <= kMergeInKernelMaxParts) {
+        if (d.merge_here) {
           // A head in few parts is finished here, by whichever part is written last: every part publishes its
           // record (fence), then takes a ticket; the holder of the last ticket sees all records and folds them
           // in part order, so the result does not depend on who that is.  Nobody waits for anybody.

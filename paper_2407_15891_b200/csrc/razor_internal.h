@@ -13,10 +13,14 @@ namespace razor {
 
 constexpr int kPageTokens = 16;        // tokens per page
 constexpr int kMaxGroup = 8;           // query heads per KV head
-// A head cut into at most this many parts is finished inside the streaming kernel: whichever of its parts is
-// written last (an atomic ticket, nobody waits) folds the head's partial records, in part order.  Heads in more
-// parts are left to the combine kernel that follows.
-constexpr int kMergeInKernelMaxParts = 8;
+// A head cut into few parts is finished inside the streaming kernel: whichever of its parts is written last (an
+// atomic ticket, nobody waits) folds the head's partial records, in part order.  "Few" is at most
+// kMergeInKernelMaxRows record rows in all (parts x query rows of the KV head's tile), never more than
+// kMergeInKernelMaxParts parts: one warp folds them in about a microsecond.  Heads in more parts are left to the
+// combine kernel that follows.
+constexpr int kMergeInKernelMaxParts = 16;
+constexpr int kMergeInKernelMaxRows = 16;
+inline int merge_in_kernel_max_parts(int rows) { return rows >= kMergeInKernelMaxRows ? 1 : kMergeInKernelMaxRows / rows; }
 constexpr int kCompressMaxSlices = 512;    // row slices per (sequence, KV head) in the compression kernel
 constexpr int kCompressSliceBudget = 8192; // slice sums a call may produce beyond one per head (sizes the scratch)
 
@@ -89,7 +93,8 @@ struct WorkItem {
   int32_t part_idx;   // index of this part within its head
   int32_t n_parts;    // parts of this head
   int32_t rec_base;
-  int32_t pad0, pad1;
+  int32_t merge_here;   // 1: the head's parts are folded by the streaming kernel itself (its last part to arrive)
+  int32_t pad1;
 };
 
 // A head whose stream was cut into several parts: one entry of the combine kernel's work list.
@@ -208,6 +213,10 @@ struct DecodeJobs {
   // length and which page the preceding append (if any) wrote, so it can name pages that nothing in flight
   // writes.  0: none.  Only the first kEarlyCtas CTAs take part.
   uint8_t early[kEarlyCtas];
+  // Not NULL: the launch first adds one token per sequence (k_new, v_new device [B, Hkv, D]) exactly as the
+  // append kernel would, and attends over the cache with that token in it.
+  const void* k_new;
+  const void* v_new;
 };
 cudaError_t launch_decode(const DeviceView& dv, int dtype, int layer, const DecodeJobs& jobs, const void* q,
                           float* out, int n_sms, const DecodeTuning& tune, cudaStream_t stream);
@@ -221,6 +230,7 @@ struct SchedParams {
   int static_pct;          // 0..100
   int tail_items_per_cta;  // >= 1
   int min_chunk_pages;     // >= 1
+  int merge_max_parts;     // heads in at most this many parts are folded inside the streaming kernel
 };
 struct SchedInfo {
   int n_items, n_jobs, n_spans;   // the first n_spans jobs are spans

@@ -99,7 +99,7 @@ int build_schedule(const int32_t* pages, int n_heads, const SchedParams& sp, int
     if (n_parts[h] < 2) continue;
     rec_base[h] = rec;
     // heads in few parts are folded by the streaming kernel itself; only the others go on the combine kernel's list
-    if (n_parts[h] > kMergeInKernelMaxParts) multi[n_multi++] = MultiHead{h, rec, n_parts[h], 0};
+    if (n_parts[h] > sp.merge_max_parts) multi[n_multi++] = MultiHead{h, rec, n_parts[h], 0};
     rec += n_parts[h];
   }
   // Job order: spans in stream order, then the tail items.  Jobs are numbered along the stream, so the
@@ -119,7 +119,8 @@ int build_schedule(const int32_t* pages, int n_heads, const SchedParams& sp, int
     w.part_idx = next_part[pc.head]++;
     w.n_parts = n_parts[pc.head];
     w.rec_base = rec_base[pc.head];
-    w.pad0 = w.pad1 = 0;
+    w.merge_here = (n_parts[pc.head] > 1 && n_parts[pc.head] <= sp.merge_max_parts) ? 1 : 0;
+    w.pad1 = 0;
     out[n++] = w;
   }
   jobs[n_jobs] = n;

@@ -98,10 +98,11 @@ def run_parity(w: synth.Workload, *, layers: Optional[Sequence[int]] = None,
                heads_for: Optional[Dict[int, List[Tuple[int, int]]]] = None, steps: Optional[int] = None,
                shuffle: int = 0, use_comp: int = 1, sm_scale: float = 0.0, per_seq: bool = False,
                check_layout_every: int = 0, device="cuda:0", stats: Optional[dict] = None,
-               options: Optional[Dict[int, int]] = None) -> dict:
+               options: Optional[Dict[int, int]] = None, fused: bool = False) -> dict:
     """Compress every layer, then run `steps` x (append, decode) over all layers on the GPU, checking
     the heads listed in heads_for[layer] (default: every head of every layer) against the oracle.
-    With steps == 0 one decode is run straight after compression (no append)."""
+    With steps == 0 one decode is run straight after compression (no append).  fused: each step is one
+    razor_decode_step call instead of razor_append + razor_decode_attention."""
     dev = torch.device(device)
     all_layers = list(range(w.n_layers))
     check_layers = list(layers) if layers is not None else all_layers
@@ -143,11 +144,16 @@ def run_parity(w: synth.Workload, *, layers: Optional[Sequence[int]] = None,
         n_rounds = max(steps, 1)
         for t in range(n_rounds):
             for l in all_layers:
+                q = synth.make_queries(w, l, t, dev)
                 if steps > 0:
                     k_new, v_new = synth.make_new_kv(w, l, t, dev)
-                    cache.append(l, k_new, v_new)
-                q = synth.make_queries(w, l, t, dev)
-                out = cache.decode(l, q)
+                    if fused:                                   # append + decode in one launch
+                        out = cache.decode_step(l, k_new, v_new, q)
+                    else:
+                        cache.append(l, k_new, v_new)
+                        out = cache.decode(l, q)
+                else:
+                    out = cache.decode(l, q)
                 if t == 0 and l == all_layers[0]:
                     status = cache.device_status()
                     assert status == 0, f"a bounded wait inside the decode kernel ran out (status bits {status})"
@@ -235,7 +241,8 @@ def check_export(ex: dict, ref: HeadRef, n_sink: int, window: int, is_retr: bool
 
 
 def run_parity_recorded(w: synth.Workload, *, heads_for: Dict[int, List[Tuple[int, int]]], steps: int,
-                        per_seq: bool = False, device="cuda:0", options: Optional[Dict[int, int]] = None) -> dict:
+                        per_seq: bool = False, device="cuda:0", options: Optional[Dict[int, int]] = None,
+                        fused: bool = True) -> dict:
     """heads_for[layer] = [(b, kv head)] to check.  steps >= 1: that many (append, decode) rounds over all
     layers; steps == 0: one decode straight after compression.  Layout is checked right after compression,
     after the middle step and after the last one; outputs at every step.  Returns counts and worst errors."""
@@ -304,10 +311,16 @@ def run_parity_recorded(w: synth.Workload, *, heads_for: Dict[int, List[Tuple[in
             snap = {}
             for t in range(n_rounds):
                 for l in range(L):
-                    if steps > 0:
+                    q = synth.make_queries(w, l, t, dev)
+                    if steps > 0 and fused:                  # the benchmark's step: append + decode in one launch
+                        k_new, v_new = synth.make_new_kv(w, l, t, dev)
+                        out = cache.decode_step(l, k_new, v_new, q)
+                    elif steps > 0:
                         k_new, v_new = synth.make_new_kv(w, l, t, dev)
                         cache.append(l, k_new, v_new)
-                    out = cache.decode(l, synth.make_queries(w, l, t, dev))
+                        out = cache.decode(l, q)
+                    else:
+                        out = cache.decode(l, q)
                     if l in heads_for:
                         outs[(l, t)] = out.cpu()
                         if t == mid:

@@ -109,10 +109,11 @@ def test_scaled_configs_every_head_with_shuffled_pages(name, scale):
 
 
 # ------------------------------------------------------------------ property sweep over small shapes
+@pytest.mark.parametrize("fused", [False, True])
 @pytest.mark.parametrize("dtype", ["bf16", "f32"])
 @pytest.mark.parametrize("D", [64, 128])
 @pytest.mark.parametrize("group", [1, 2, 4, 8])
-def test_small_shape_sweep(dtype, D, group):
+def test_small_shape_sweep(dtype, D, group, fused):
     rng = np.random.default_rng(D * 100 + group + (7 if dtype == "f32" else 0))
     for trial in range(6):
         B = int(rng.integers(1, 4))
@@ -127,7 +128,7 @@ def test_small_shape_sweep(dtype, D, group):
         w = synth.Workload(f"sweep{trial}", B, 2, Hkv * group, Hkv, D, dtype, ctx, win, n_sink,
                            n_retrieval_kv=min(1, Hkv - 1) if trial % 2 else 0, decode_steps=5,
                            seed=9000 + trial + D + group)
-        run_parity(w, steps=5 if trial != 3 else 0, shuffle=trial, check_layout_every=1)
+        run_parity(w, steps=5 if trial != 3 else 0, shuffle=trial, check_layout_every=1, fused=fused)
 
 
 @pytest.mark.parametrize("group,options", [
@@ -143,17 +144,61 @@ def test_small_shape_sweep(dtype, D, group):
     (1, {rz.OPT_DECODE_CONSUMER_WARPS: 8, rz.OPT_DECODE_STATIC_PERCENT: 30, rz.OPT_DECODE_TAIL_ITEMS_PER_SM: 200,
          rz.OPT_DECODE_MIN_CHUNK_PAGES: 1}),
 ])
+@pytest.mark.parametrize("fused", [False, True])
 @pytest.mark.parametrize("D", [64, 128])
-def test_decode_kernel_variants(group, options, D):
+def test_decode_kernel_variants(group, options, D, fused):
     """Every decode kernel variant the options can select, on a ragged batch whose long head is cut into
     enough parts for a two-level combine tree."""
     w = synth.Workload("variants", 3, 1, 2 * group, 2, D, "bf16", [9000, 37, 700], [300, 300, 100], 4, 1, 3, 2024 + group)
-    run_parity(w, steps=3, shuffle=7, options=options, check_layout_every=2)
+    run_parity(w, steps=3, shuffle=7, options=options, check_layout_every=2, fused=fused)
 
 
-def test_append_many_tokens_crosses_pages_evicts_and_rebuilds_schedule():
+@pytest.mark.parametrize("fused", [False, True])
+def test_append_many_tokens_crosses_pages_evicts_and_rebuilds_schedule(fused):
     w = synth.Workload("long_append", 2, 1, 4, 4, 128, "bf16", [700, 90], [64, 200], 4, 1, 300, 4242)
-    run_parity(w, steps=300, check_layout_every=37)
+    run_parity(w, steps=300, check_layout_every=37, fused=fused)
+
+
+def test_one_launch_steps_interleaved_with_separate_appends_and_decodes():
+    """razor_decode_step mixed with razor_append / razor_decode_attention on the same layers (one of them a
+    single-layer cache, where consecutive launches touch the same pages), layout checked after every step."""
+    for n_layers in (1, 3):
+        w = synth.Workload("mixed_steps", 3, n_layers, 8, 4, 128, "bf16", [900, 30, 260], [40, 100, 16], 4, 1, 60, 808 + n_layers)
+        cache = make_cache(w, max_new=60)
+        refs = {}
+        for l in range(n_layers):
+            K, V = synth.make_dense_kv(w, l, DEV)
+            cache.compress(l, K, V, w.ctx_len, w.retrieval(l), w.window)
+            for b in range(w.batch):
+                for g in range(w.n_kv_heads):
+                    refs[(l, b, g)] = HeadRef(l, b, g, K[b, g], V[b, g], w.ctx_len[b], 60)
+        rng = np.random.default_rng(5 + n_layers)
+        scale = 1 / math.sqrt(w.head_dim)
+        for t in range(60):
+            for l in range(n_layers):
+                k_new, v_new = synth.make_new_kv(w, l, t, DEV)
+                q = synth.make_queries(w, l, t, DEV)
+                if rng.random() < 0.6:
+                    out = cache.decode_step(l, k_new, v_new, q)
+                else:
+                    cache.append(l, k_new, v_new)
+                    out = cache.decode(l, q)
+                if rng.random() < 0.3:
+                    out = cache.decode(l, q)                      # a second decode of the same layer, no append
+                out_h, q_h = to_f64(out), to_f64(q)
+                for (ll, b, g), ref in refs.items():
+                    if ll != l:
+                        continue
+                    ref.append(k_new[b, g].cpu(), v_new[b, g].cpu())
+                    if t % 7 == 0 or t == 59:
+                        hc = check_head_state(cache, ref, w.n_sink, w.window[b], bool(w.retrieval(l)[g]))
+                    else:
+                        hc = orc.compress_head(ref.K, ref.V, ref.n, w.n_sink, w.window[b], bool(w.retrieval(l)[g]))
+                    for j in range(w.group):
+                        err = np.abs(out_h[b, g * w.group + j] - orc.decode_head(q_h[b, g * w.group + j], hc, scale)).max()
+                        assert err <= 3e-3, (err, l, b, g, j, t)
+        assert cache.device_status() == 0
+        cache.close()
 
 
 def test_plain_truncation_mode_and_literal_scale():
