@@ -365,6 +365,63 @@ def decode_only(rz, synth, name, n_layers, dev, peak, reps=60, n_tok=1, alibi=Fa
     return res
 
 
+def long_round_leg(rz, synth, dev, n_tok=512, n_layers=2, reps=6):
+    """A prompt-sized round on the 32K MHA shape: n_tok new tokens per sequence appended in bulk, then all their
+    queries in one razor_decode_attention_multi call (the query-tiled tensor-core kernel: the cache is streamed
+    once per 128 query rows).  A dense contraction: 4 * D flops per (query row, visible kept token)."""
+    import numpy as np
+    import torch
+    w = synth.workload("cfg2")
+    w.n_layers = n_layers
+    retr = [w.retrieval(l) for l in range(n_layers)]
+    cfg = rz.make_config(w.batch, n_layers, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, w.n_sink, max(w.ctx_len), n_tok)
+    cache = rz.RazorCache(cfg, w.ctx_len, w.window, np.stack(retr), device=dev)
+    w0 = synth.Workload(w.name, w.batch, 1, w.n_q_heads, w.n_kv_heads, w.head_dim, w.dtype, w.ctx_len, w.window,
+                        w.n_sink, w.n_retrieval_kv, 1, w.seed)
+    K, V = synth.make_dense_kv(w0, 0, dev)
+    for l in range(n_layers):
+        cache.compress(l, K, V, w.ctx_len, retr[l], w.window)
+    del K, V
+    kv_shape = (w.batch, n_tok, w.n_kv_heads, w.head_dim)
+    k_new = synth.normal_bf16(w.seed, synth.TAG_KNEW, kv_shape, dev, sub=78)
+    v_new = synth.normal_bf16(w.seed, synth.TAG_VNEW, kv_shape, dev, sub=78)
+    q = synth.normal_bf16(w.seed, synth.TAG_Q, (w.batch, n_tok, w.n_q_heads, w.head_dim), dev, sub=78)
+    out = torch.empty(q.shape, dtype=torch.float32, device=dev)
+    for l in range(n_layers):
+        cache.append_many(l, k_new, v_new)
+        cache.decode_multi(l, q, out)
+    torch.cuda.synchronize()
+    a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+    a.record()
+    for i in range(reps):
+        cache.decode_multi(i % n_layers, q, out)
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / reps
+    # visible (query row, kept token) pairs: every kept token from before the round for every row, the round's own
+    # tokens causally
+    G = w.group
+    pairs = 0
+    for bb in range(w.batch):
+        for g in range(w.n_kv_heads):
+            n = w.ctx_len[bb] + n_tok
+            kept = n if retr[0][g] else min(n, w.n_sink + w.window[bb])
+            pairs += G * (n_tok * (kept - n_tok) + n_tok * (n_tok + 1) // 2)
+    flops = 4.0 * w.head_dim * pairs
+    try:
+        peak = float(json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))["bf16_tflops"])
+        kind = "measured (cuBLAS bf16 burst)"
+    except Exception:
+        peak, kind = 1590.0, "fallback"
+    status = cache.device_status()
+    cache.close()
+    return {"workload": f"cfg2 shape: batch {w.batch}, {w.n_q_heads} heads, context {max(w.ctx_len)}, round of {n_tok} tokens",
+            "ms_per_layer": ms, "tflops": flops / (ms * 1e-3) / 1e12, "bound": "tensor", "peak_tflops": peak,
+            "peak_kind": kind, "frac": flops / (ms * 1e-3) / 1e12 / peak, "device_status": status,
+            "note": "tcgen05 S = Q K^T and O = P V (P as a bf16 head plus a bf16 remainder: three matrix products per "
+                    "block where the flop count above has two), one exponential per score"}
+
+
 def chunked_prefill_leg(rz, synth, dev, peak, chunk=8192, reps=3):
     """One cfg3-shaped layer (batch 4, 40 heads, 65536 tokens) built chunk by chunk from an empty layer with
     razor_append_many, as a chunked prefill hands its K/V over: no dense cache of the whole context exists.
@@ -701,6 +758,10 @@ def main():
             line["alibi_32k"] = decode_only(rz, synth, "cfg2", 3, dev, peak, alibi=True)
         except Exception as ex:
             line["alibi_32k"] = {"unavailable": str(ex)[:200]}
+        try:   # a 512-token round (follow-up prompt) on the 32K MHA shape: the query-tiled kernel
+            line["round_of_512_tokens_32k"] = long_round_leg(rz, synth, dev)
+        except Exception as ex:
+            line["round_of_512_tokens_32k"] = {"unavailable": str(ex)[:200]}
         try:   # a 4-token round (verify step) on the 32K MHA shape: same pages streamed, four queries per head
             line["round_of_4_tokens_32k"] = decode_only(rz, synth, "cfg2", 3, dev, peak, n_tok=4)
         except Exception as ex:

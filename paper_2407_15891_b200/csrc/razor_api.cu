@@ -32,7 +32,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 inline int ceil_div(long long a, long long b) { return (int)((a + b - 1) / b); }
 
 struct Layout {
-  size_t state, comp_sum, comp_mean, page_table, items, jobs, multi, rec_ml, rec_o, queue, tickets, scratch, plan, slopes, total;
+  size_t state, comp_sum, comp_mean, page_table, items, jobs, multi, rec_ml, rec_o, queue, tickets, scratch, plan, slopes, round_items, round_units, total;
   int max_pages, max_items;
 };
 
@@ -80,6 +80,8 @@ Layout make_layout(const razor_config_t& c) {
   l.scratch = take(((size_t)kCompressSliceBudget + nh) * 2 * D * sizeof(float));
   l.plan = take(nh * sizeof(HeadPlan) + (size_t)c.batch * sizeof(SeqDesc));   // plan[], then seq_desc[]
   l.slopes = take(L * (size_t)c.n_q_heads * sizeof(float));
+  l.round_items = take((size_t)kRoundMaxItems * sizeof(RoundItem));
+  l.round_units = take((size_t)kRoundMaxUnits * sizeof(RoundUnit));
   l.total = off;
   return l;
 }
@@ -141,6 +143,9 @@ struct razor_cache {
   size_t plan_bytes = 0;
   cudaEvent_t plan_done[kPlanSlots] = {};
   int plan_next = 0;
+  // Work list of the round kernel (razor_decode_attention_multi on long rounds): pinned staging, one upload in flight.
+  uint8_t* pinned_round = nullptr;   // RoundItem[kRoundMaxItems], then RoundUnit[kRoundMaxUnits]
+  cudaEvent_t round_done = nullptr;
   // Layer whose pages, state or sums the last kernel launched for this cache wrote (-1: it wrote none, a decode).
   // An append of another layer may read before it waits for that kernel.
   int last_writer_layer = -1;
@@ -241,6 +246,8 @@ int razor_cache_create(razor_cache_t** out, const razor_config_t* cfg, void* poo
   dv.plan = (HeadPlan*)(ws + lay.plan);
   dv.seq_desc = (SeqDesc*)(ws + lay.plan + (size_t)cfg->batch * cfg->n_kv_heads * sizeof(HeadPlan));
   dv.alibi_slopes = (float*)(ws + lay.slopes);
+  dv.round_items = (RoundItem*)(ws + lay.round_items);
+  dv.round_units = (RoundUnit*)(ws + lay.round_units);
   dv.alibi = 0;
   dv.n_heads = cfg->batch * cfg->n_kv_heads;
   dv.n_kv_heads = cfg->n_kv_heads;
@@ -266,12 +273,16 @@ int razor_cache_create(razor_cache_t** out, const razor_config_t* cfg, void* poo
   c->plan_bytes = (size_t)dv.n_heads * sizeof(HeadPlan) + (size_t)cfg->batch * sizeof(SeqDesc);
   if (e == cudaSuccess)
     e = cudaHostAlloc((void**)&c->pinned_plan, (size_t)kPlanSlots * c->plan_bytes, cudaHostAllocDefault);
+  if (e == cudaSuccess)
+    e = cudaHostAlloc((void**)&c->pinned_round, (size_t)kRoundMaxItems * sizeof(RoundItem) + (size_t)kRoundMaxUnits * sizeof(RoundUnit),
+                      cudaHostAllocDefault);
   if (e != cudaSuccess) {
     note_cuda_error(e);
     if (c->pinned_items) cudaFreeHost(c->pinned_items);
     if (c->pinned_jobs) cudaFreeHost(c->pinned_jobs);
     if (c->pinned_multi) cudaFreeHost(c->pinned_multi);
     if (c->pinned_plan) cudaFreeHost(c->pinned_plan);
+    if (c->pinned_round) cudaFreeHost(c->pinned_round);
     delete c;
     return RAZOR_E_CUDA;
   }
@@ -315,6 +326,8 @@ int razor_cache_destroy(razor_cache_t* c) {
   if (c->pinned_jobs) cudaFreeHost(c->pinned_jobs);
   if (c->pinned_multi) cudaFreeHost(c->pinned_multi);
   if (c->pinned_plan) cudaFreeHost(c->pinned_plan);
+  if (c->pinned_round) cudaFreeHost(c->pinned_round);
+  if (c->round_done) cudaEventDestroy(c->round_done);
   for (cudaEvent_t ev : c->plan_done)
     if (ev) cudaEventDestroy(ev);
   delete c;
@@ -685,6 +698,85 @@ static int decode_impl(razor_cache_t* c, int32_t layer, const void* q, float* ou
                        int32_t tok_stride, int32_t q_after, void* stream, const void* k_new = nullptr,
                        const void* v_new = nullptr);
 
+// A long round on the query-tiled kernel.  Work items are (KV head, tile of 128 query rows, run of 128-token
+// blocks): every (head, tile) unit is cut into parts of about equal size so that there are a few items per SM,
+// the items are handed out longest first, and units in several parts get partial records (128 rows per part)
+// that a merge kernel folds.  For a head whose slots are in position order (nothing dropped) the blocks that
+// lie wholly after the tile's last query are left out.
+static int round_impl(razor_cache_t* c, int32_t layer, const void* q, float* out, int32_t n_tokens, void* stream) {
+  if (((uintptr_t)q | (uintptr_t)out) & 15) return RAZOR_E_MISALIGNED;
+  const LayerHost& L = c->layers[layer];
+  const int G = c->cfg.n_q_heads / c->cfg.n_kv_heads, nh = c->dv.n_heads;
+  const int tok_per_tile = kRoundTileRows / G;
+  const int n_tiles = ceil_div(n_tokens, tok_per_tile);
+  struct Unit { int head, tile, blocks; };
+  std::vector<Unit> units;
+  units.reserve((size_t)nh * n_tiles);
+  long long total_blocks = 0;
+  for (int h = 0; h < nh; ++h) {
+    const HeadState& st = L.hs[h];
+    const int all_blocks = ceil_div(st.len, kRoundBlockTokens);
+    for (int t = 0; t < n_tiles; ++t) {
+      int blocks = all_blocks;
+      if (st.window < 0 || st.n_drop == 0) {   // slot = position: nothing beyond the tile's last query is visible
+        const int last_q = std::min(n_tokens, (t + 1) * tok_per_tile) - 1;
+        const long long q_pos = (long long)st.len + st.n_drop - n_tokens + last_q;
+        blocks = (int)std::min<long long>(all_blocks, q_pos / kRoundBlockTokens + 1);
+      }
+      units.push_back({h, t, std::max(blocks, 0)});
+      total_blocks += std::max(blocks, 0);
+    }
+  }
+  // parts: about four items per SM, never more than fit the item list or the record rows
+  const long long rec_rows = (long long)c->lay.max_items * kMaxGroup;
+  long long chunk = std::max<long long>(1, ceil_div(total_blocks, (long long)c->n_sms * 4));
+  std::vector<RoundItem> items;
+  std::vector<RoundUnit> multi;
+  for (;;) {
+    items.clear();
+    multi.clear();
+    long long rec = 0;
+    for (const Unit& u : units) {
+      const int parts = std::max(1, ceil_div(u.blocks, chunk));
+      const int per = u.blocks > 0 ? ceil_div(u.blocks, parts) : 0;
+      if (parts > 1) {
+        multi.push_back(RoundUnit{u.head, u.tile, (int32_t)rec, parts});
+      }
+      for (int p = 0; p < parts; ++p) {
+        RoundItem it;
+        it.head = u.head; it.q_tile = u.tile;
+        it.blk_begin = std::min(u.blocks, p * per); it.blk_end = std::min(u.blocks, (p + 1) * per);
+        it.part_idx = p; it.n_parts = parts; it.rec_base = (int32_t)rec; it.pad = 0;
+        items.push_back(it);
+      }
+      if (parts > 1) rec += (long long)parts * kRoundTileRows;
+    }
+    if ((long long)items.size() <= kRoundMaxItems && (long long)multi.size() <= kRoundMaxUnits && rec <= rec_rows) break;
+    if (chunk > total_blocks) return RAZOR_E_CAPACITY;   // even unsplit units do not fit the work list
+    chunk *= 2;
+  }
+  std::stable_sort(items.begin(), items.end(), [](const RoundItem& a, const RoundItem& b) {
+    return a.blk_end - a.blk_begin > b.blk_end - b.blk_begin;
+  });
+  cudaStream_t s = (cudaStream_t)stream;
+  if (c->round_done) RZ_CUDA(cudaEventSynchronize(c->round_done));   // the upload before has left the staging area
+  else RZ_CUDA(cudaEventCreateWithFlags(&c->round_done, cudaEventDisableTiming));
+  RoundItem* st_items = (RoundItem*)c->pinned_round;
+  RoundUnit* st_units = (RoundUnit*)(c->pinned_round + (size_t)kRoundMaxItems * sizeof(RoundItem));
+  std::memcpy(st_items, items.data(), items.size() * sizeof(RoundItem));
+  if (!multi.empty()) std::memcpy(st_units, multi.data(), multi.size() * sizeof(RoundUnit));
+  RZ_CUDA(cudaMemcpyAsync(c->dv.round_items, st_items, items.size() * sizeof(RoundItem), cudaMemcpyHostToDevice, s));
+  if (!multi.empty())
+    RZ_CUDA(cudaMemcpyAsync(c->dv.round_units, st_units, multi.size() * sizeof(RoundUnit), cudaMemcpyHostToDevice, s));
+  RZ_CUDA(cudaEventRecord(c->round_done, s));
+  const RoundJobs jb{(int32_t)items.size(), (int32_t)multi.size(), n_tokens, 0};
+  RZ_CUDA(launch_round(c->dv, c->pool_pages, layer, jb, q, out, c->n_sms, s));
+  c->last_writer_layer = -1;
+  c->writes_since_decode.clear();   // an ordinary launch: everything before it has completed when it starts
+  c->writes_overflow = false;
+  return RAZOR_OK;
+}
+
 // Which pages a span CTA may copy before the decode kernel waits for the launch it depends on.  While that part
 // of the kernel runs, the library kernels launched since the previous decode (and that decode itself, when it
 // appended a token) may still be writing.  If none of them wrote this layer, every page of it is stable.  If the
@@ -745,6 +837,10 @@ int razor_decode_attention_multi(razor_cache_t* c, int32_t layer, const void* q,
     if (h.len + h.n_drop < n_tokens) return RAZOR_E_INVALID_ARG;          // fewer tokens cached than queries
     if (h.n_drop > 0 && h.window < n_tokens) return RAZOR_E_INVALID_ARG;  // the mean would hold tokens after a query
   }
+  const int group0 = c->cfg.n_q_heads / c->cfg.n_kv_heads;
+  // A round with at least 64 query rows per KV head is a dense tile: the query-tiled kernel streams the cache once
+  // per 128 rows (tensor cores).  ALiBi heads stay on the path below.
+  if ((long long)group0 * n_tokens >= kRoundTileRows / 2 && !c->dv.alibi) return round_impl(c, layer, q, out, n_tokens, stream);
   // One launch takes a tile of 2, 4 or 8 rows per KV head (query heads of the group x query tokens).  A
   // longer round runs block by block, the largest block that fits; when the round is not a multiple of
   // the block, the last block is moved back to end with the round and recomputes a few tokens.

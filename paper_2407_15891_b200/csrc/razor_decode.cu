@@ -412,32 +412,6 @@ __device__ __forceinline__ void store_new_row(uint8_t* page, uint8_t* pool_page,
   __syncwarp();
 }
 
-// Reducer-side vector of D/32 consecutive floats per lane.
-template <int D>
-struct LaneVec;
-template <>
-struct LaneVec<128> {
-  float4 v;
-  __device__ __forceinline__ void zero() { v = make_float4(0.f, 0.f, 0.f, 0.f); }
-  __device__ __forceinline__ void fma(float c, const LaneVec& o) {
-    v.x += c * o.v.x; v.y += c * o.v.y; v.z += c * o.v.z; v.w += c * o.v.w;
-  }
-  __device__ __forceinline__ void scale(float c) { v.x *= c; v.y *= c; v.z *= c; v.w *= c; }
-  __device__ __forceinline__ void load_shared(const float* row, int lane) { v = *(const float4*)(row + lane * 4); }
-  __device__ __forceinline__ void load_l2(const float* row, int lane) { v = __ldcg((const float4*)(row + lane * 4)); }
-  __device__ __forceinline__ void store(float* row, int lane) const { *(float4*)(row + lane * 4) = v; }
-};
-template <>
-struct LaneVec<64> {
-  float2 v;
-  __device__ __forceinline__ void zero() { v = make_float2(0.f, 0.f); }
-  __device__ __forceinline__ void fma(float c, const LaneVec& o) { v.x += c * o.v.x; v.y += c * o.v.y; }
-  __device__ __forceinline__ void scale(float c) { v.x *= c; v.y *= c; }
-  __device__ __forceinline__ void load_shared(const float* row, int lane) { v = *(const float2*)(row + lane * 2); }
-  __device__ __forceinline__ void load_l2(const float* row, int lane) { v = __ldcg((const float2*)(row + lane * 2)); }
-  __device__ __forceinline__ void store(float* row, int lane) const { *(float2*)(row + lane * 2) = v; }
-};
-
 // ------------------------------------------------------------------------------------------ the kernel
 template <typename T, int D, int G, int NC, bool MMA>
 __global__ void __launch_bounds__((NC + 2) * 32, 1)

@@ -137,6 +137,8 @@ enum : int32_t {
   kStatusEarlyMismatch = 32     // a CTA was told to prefetch more pages than its first work item turned out to have
 };
 
+struct RoundItem;
+struct RoundUnit;
 // Pointers into the caller's workspace, plus the dimensions the kernels need.
 struct DeviceView {
   uint8_t* pool;            // pages: [page][K rows | V rows][16][D]
@@ -156,6 +158,8 @@ struct DeviceView {
   HeadPlan* plan;           // [B*Hkv]  heads of the compression call in flight
   SeqDesc* seq_desc;        // [B]      directly behind plan[]: both arrive in one copy
   float* alibi_slopes;      // [L][Hq]  ALiBi slopes l_h times log2(e); read only when alibi != 0
+  RoundItem* round_items;   // [kRoundMaxItems]  work list of the round kernel's launch in flight
+  RoundUnit* round_units;   // [kRoundMaxUnits]  its units in several parts
   int32_t alibi;            // 1: logits get - l_h (m - n) (Eq. 1), from razor_cache_set_alibi
   int32_t n_heads;          // B*Hkv
   int32_t n_kv_heads;
@@ -220,6 +224,30 @@ struct DecodeJobs {
 };
 cudaError_t launch_decode(const DeviceView& dv, int dtype, int layer, const DecodeJobs& jobs, const void* q,
                           float* out, int n_sms, const DecodeTuning& tune, cudaStream_t stream);
+// ---- rounds of many query tokens (razor_round.cu): the query rows of a KV head (query tokens x query heads of
+// the group) are tiled kRoundTileRows at a time and the head's slot stream is walked in blocks of kRoundBlockTokens.
+constexpr int kRoundTileRows = 128;
+constexpr int kRoundBlockTokens = 128;
+constexpr int kRoundMaxItems = 8192;
+constexpr int kRoundMaxUnits = 4096;
+struct RoundItem {
+  int32_t head;        // b * Hkv + kv_head
+  int32_t q_tile;      // rows [q_tile * 128, + 128) of the head's query rows
+  int32_t blk_begin;   // 128-token blocks [blk_begin, blk_end) of the head's slots
+  int32_t blk_end;
+  int32_t part_idx;    // index of this part within its (head, q_tile) unit
+  int32_t n_parts;
+  int32_t rec_base;    // first record row of the unit (each part owns kRoundTileRows rows)
+  int32_t pad;
+};
+struct RoundUnit {     // a (head, q_tile) cut into several parts: one entry of the merge kernel's work list
+  int32_t head, q_tile, rec_base, n_parts;
+};
+struct RoundJobs {
+  int32_t n_items, n_units, n_tok, pad;
+};
+cudaError_t launch_round(const DeviceView& dv, long long pool_pages, int layer, const RoundJobs& jb, const void* q,
+                         float* out, int n_sms, cudaStream_t stream);
 cudaError_t launch_wait_selftest(const DeviceView& dv, unsigned long long limit_ns, cudaStream_t stream);
 cudaError_t launch_export(const DeviceView& dv, int dtype, int layer, int head, int32_t* kept_pos, void* K, void* V,
                           float* mean_k, float* mean_v, float* sum_k, float* sum_v, cudaStream_t stream);

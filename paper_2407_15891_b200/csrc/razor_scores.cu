@@ -31,6 +31,7 @@
 
 #include "razor_common.cuh"
 #include "razor_sync.cuh"
+#include "razor_tc.cuh"
 
 namespace razor {
 namespace {
@@ -69,32 +70,13 @@ constexpr size_t score_smem_bytes() {
   return need < 80 * 1024 ? 80 * 1024 : need;
 }
 
-// Shared-memory matrix descriptor of a K-major operand in the 128-byte swizzled layout: start address
-// and strides in 16-byte units; consecutive 8-row groups are 1 KB apart; descriptor version 1.
-__device__ __forceinline__ uint64_t operand_desc(uint32_t addr) {
-  return (uint64_t)((addr >> 4) & 0x3FFFu) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
-}
 // Instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, N / 8 at bit 17, M / 16 at bit 24.
 constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kKTile >> 3) << 17) |
                                 ((uint32_t)(kQTile >> 4) << 24);
 
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      :
-      : "r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(kInstrDesc), "r"(accumulate)
-      : "memory");
+  umma_bf16_desc(tmem_d, desc_a, desc_b, kInstrDesc, accumulate);
 }
-// Arrives on `bar` once every MMA issued so far by this thread has completed.
-__device__ __forceinline__ void umma_commit(uint64_t* bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
-               : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
 // 2^t for t <= 0 on the FMA and integer pipes, relative error below 5e-5: t = n + f with n the nearest
 // integer (read off the low mantissa bits of t + 1.5 * 2^23) and |f| <= 1/2, 2^f as a degree-4 polynomial,
 // n added onto the exponent field.  The transcendental unit is the busiest pipe of this kernel (one ex2 per
@@ -112,19 +94,6 @@ __device__ __forceinline__ float exp2_fma(float t) {
   return __int_as_float(__float_as_int(p) + (__float_as_int(r) << 23));
 }
 
-// Issues the load of 32 consecutive columns of this thread's lane; the registers are valid after tmem_ld_wait().
-__device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t* v) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
-      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-        "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
-        "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
-        "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-      : "r"(taddr)
-      : "memory");
-}
 // Completes the loads issued so far.  The registers pass through the statement so that no use of them
 // can be scheduled ahead of it.
 __device__ __forceinline__ void tmem_ld_wait(uint32_t (&v)[64]) {
@@ -388,22 +357,6 @@ __global__ void head_scores_finalize_kernel(const float* __restrict__ scratch, c
     echo[blockIdx.x] = bad ? CUDART_NAN_F : (n_queries > 0 ? e / (float)n_queries : 0.f);
     induction[blockIdx.x] = bad ? CUDART_NAN_F : (n_queries > 0 ? i / (float)n_queries : 0.f);
   }
-}
-
-// cuTensorMapEncodeTiled, looked up through the runtime (the library does not link against the driver).
-using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-EncodeTiledFn encode_tiled_fn() {
-  static EncodeTiledFn fn = [] {
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult q = cudaDriverEntryPointSymbolNotFound;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
-        q != cudaDriverEntryPointSuccess)
-      p = nullptr;
-    return (EncodeTiledFn)p;
-  }();
-  return fn;
 }
 
 // Tensor map of X[n_heads][n_tokens][D] bf16 with boxes of 64 elements x 128 rows of one head, written

@@ -106,6 +106,65 @@ def test_round_longer_than_one_launch_runs_block_by_block(group, T, D):
     cache.close()
 
 
+@pytest.mark.parametrize("group,T,D", [(1, 64, 128), (1, 200, 128), (4, 40, 128), (2, 300, 64), (8, 16, 128), (1, 512, 64),
+                                        (4, 512, 128)])
+def test_prompt_sized_round_on_the_query_tiled_kernel(group, T, D):
+    """Rounds with at least 64 query rows per KV head run on the query-tiled tensor-core kernel: ragged batch (one
+    sequence shorter than a block, one whose window evicts and wraps during the rounds), two rounds in a row,
+    every row of every head against the oracle, layout bit-exact after the bulk appends."""
+    Hkv = 3
+    win = max(T, 150)
+    w = synth.Workload("tiled_round", 3, 1, Hkv * group, Hkv, D, "bf16", [1500, 70, 700], [win + 60, win, win], 4, 1,
+                       2 * T, 900 + T + group)
+    cache = make_cache(w, max_new=2 * T, shuffle=11)
+    K, V = synth.make_dense_kv(w, 0, DEV)
+    retr = w.retrieval(0)
+    cache.compress(0, K, V, w.ctx_len, retr, w.window)
+    refs = {(b, g): HeadRef(0, b, g, K[b, g], V[b, g], w.ctx_len[b], 2 * T) for b in range(w.batch) for g in range(Hkv)}
+    scale = 1.0 / math.sqrt(D)
+    for rnd in range(2):
+        k, v, q = _round_inputs(w, T, 40 + rnd)
+        cache.append_many(0, k, v)
+        out = to_f64(cache.decode_multi(0, q))
+        assert cache.device_status() == 0
+        kh, vh, qh = k.cpu(), v.cpu(), to_f64(q)
+        for (b, g), ref in refs.items():
+            for t in range(T):
+                ref.append(kh[b, t, g], vh[b, t, g])
+            check_head_state(cache, ref, w.n_sink, w.window[b], bool(retr[g]))
+            for j in range(group):
+                expect = orc.multi_query_attention(qh[b, :, g * group + j], ref.K[:ref.n], ref.V[:ref.n], w.n_sink,
+                                                   w.window[b], bool(retr[g]), scale)
+                err = float(np.abs(out[b, :, g * group + j] - expect).max())
+                assert err <= TOL_OUT["bf16"], (err, rnd, b, g, j)
+    cache.close()
+
+
+def test_prompt_sized_round_on_a_long_context_with_split_units():
+    """8K context, 4 sequences x 32 heads, a 256-token round: the long heads are cut into several parts (partial
+    records of 128 rows each, merged afterwards)."""
+    w = synth.workload("cfg2", 1 / 4)
+    w.batch, w.ctx_len, w.window = 4, w.ctx_len[:4], w.window[:4]
+    T = 256
+    cache = make_cache(w, max_new=T)
+    K, V = synth.make_dense_kv(w, 0, DEV)
+    retr = w.retrieval(0)
+    cache.compress(0, K, V, w.ctx_len, retr, w.window)
+    k, v, q = _round_inputs(w, T, 19)
+    cache.append_many(0, k, v)
+    out = to_f64(cache.decode_multi(0, q))
+    assert cache.device_status() == 0
+    scale = 1.0 / math.sqrt(w.head_dim)
+    heads = [g for g in range(w.n_kv_heads) if retr[g]][:3] + [g for g in range(w.n_kv_heads) if not retr[g]][:4]
+    for b in range(w.batch):
+        for g in heads:
+            Kh = np.concatenate([to_f64(K[b, g]), to_f64(k[b, :, g])])
+            Vh = np.concatenate([to_f64(V[b, g]), to_f64(v[b, :, g])])
+            expect = orc.multi_query_attention(to_f64(q[b, :, g]), Kh, Vh, w.n_sink, w.window[b], bool(retr[g]), scale)
+            assert np.abs(out[b, :, g] - expect).max() <= TOL_OUT["bf16"]
+    cache.close()
+
+
 def test_round_limits_are_reported():
     w = synth.Workload("round_err", 1, 1, 2, 2, 64, "bf16", [100], [3], 4, 0, 8, 1)
     cache = make_cache(w, max_new=8)
