@@ -453,19 +453,20 @@ def chunked_prefill_leg(rz, synth, dev, peak, chunk=8192, reps=3):
     torch.cuda.synchronize()
     ms = a.elapsed_time(b) / reps
     row = w.head_dim * 2 * 2                                    # K and V row, bf16
-    n_retr = int(np.sum(retr))
+    # Algorithmic bytes: every chunk row read once, and written once when it is stored (with chunk <= window every
+    # row is in the cache after its chunk: the cache is usable for attention after every chunk).  With chunks of
+    # at least the window length the evicted rows are not read back (their sum is on record).
     read = w.batch * w.n_kv_heads * N * row
-    kept_short = w.n_sink + w.window[0]
-    # with chunk <= window every row is stored once, and every row that ends up dropped is read back once
     written = w.batch * row * w.n_kv_heads * N
-    evicted = w.batch * row * (w.n_kv_heads - n_retr) * max(0, N - kept_short)
     status = cache.device_status()
     cache.close()
-    total = read + written + evicted
+    total = read + written
     return {"workload": f"cfg3 layer: {n_chunks} chunks of {chunk} tokens, batch {w.batch}, {w.n_kv_heads} heads",
             "ms_per_layer": ms, "us_per_chunk": ms * 1e3 / n_chunks, "gbs": total / (ms * 1e-3) / 1e9,
-            "frac_of_measured": total / (ms * 1e-3) / 1e9 / peak, "read_gb": (read + evicted) / 1e9,
-            "write_gb": written / 1e9, "device_status": status}
+            "frac_of_measured": total / (ms * 1e-3) / 1e9 / peak, "read_gb": read / 1e9,
+            "write_gb": written / 1e9, "device_status": status,
+            "note": "bytes = chunk rows read once + rows stored once" + ("; evicted rows are not read back (chunk >= window)"
+                    if chunk >= max(w.window) else "; chunks shorter than the window read the rows they evict once more")}
 
 
 def head_scores_leg(rz, synth, dev, reps=5, heads=32):

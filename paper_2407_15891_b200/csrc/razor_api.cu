@@ -32,7 +32,7 @@ inline size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
 inline int ceil_div(long long a, long long b) { return (int)((a + b - 1) / b); }
 
 struct Layout {
-  size_t state, comp_sum, comp_mean, page_table, items, jobs, multi, rec_ml, rec_o, queue, tickets, scratch, plan, slopes, round_items, round_units, total;
+  size_t state, comp_sum, comp_mean, ring_sum, ring_valid, page_table, items, jobs, multi, rec_ml, rec_o, queue, tickets, scratch, plan, slopes, round_items, round_units, total;
   int max_pages, max_items;
 };
 
@@ -67,6 +67,8 @@ Layout make_layout(const razor_config_t& c) {
   l.state = take(L * nh * sizeof(HeadState));
   l.comp_sum = take(L * nh * 2 * D * sizeof(float));
   l.comp_mean = take(L * nh * 2 * D * sizeof(float));
+  l.ring_sum = take(L * nh * 2 * D * sizeof(float));
+  l.ring_valid = take(L * nh * sizeof(int32_t));
   l.page_table = take(L * nh * (size_t)l.max_pages * sizeof(int32_t));
   l.items = take(L * (size_t)l.max_items * sizeof(WorkItem));
   l.jobs = take(L * ((size_t)l.max_items + 1) * sizeof(int32_t));
@@ -233,6 +235,8 @@ int razor_cache_create(razor_cache_t** out, const razor_config_t* cfg, void* poo
   dv.state = (HeadState*)(ws + lay.state);
   dv.comp_sum = (float*)(ws + lay.comp_sum);
   dv.comp_mean = (float*)(ws + lay.comp_mean);
+  dv.ring_sum = (float*)(ws + lay.ring_sum);
+  dv.ring_valid = (int32_t*)(ws + lay.ring_valid);
   dv.page_table = (int32_t*)(ws + lay.page_table);
   dv.items = (WorkItem*)(ws + lay.items);
   dv.jobs = (int32_t*)(ws + lay.jobs);
@@ -661,7 +665,7 @@ int razor_append_many(razor_cache_t* c, int32_t layer, const void* k_new, const 
   int slices = 0;
   if (n_tokens >= kAppendChunkMin) {
     const long long nh = c->dv.n_heads;
-    const long long room = ((long long)kCompressSliceBudget + nh) / nh;
+    const long long room = ((long long)kCompressSliceBudget + nh) / (2 * nh);   // two sets of sums per slice
     slices = (int)std::max(1LL, std::min({(long long)ceil_div((long long)c->n_sms * 8, nh), room,
                                            (long long)(n_tokens / 32)}));
   }

@@ -184,7 +184,10 @@ __global__ void __launch_bounds__(256) compress_plan_kernel(DeviceView dv, int l
   const size_t hs = (size_t)layer * dv.n_heads + pl.head;
   int32_t* row = dv.page_table + hs * dv.max_pages;
   for (int k = threadIdx.x; k < pl.n_pages; k += 256) row[k] = pl.first_page + k;
-  if (threadIdx.x == 0) dv.state[hs] = HeadState{pl.len, pl.n_drop, 0, pl.window};
+  if (threadIdx.x == 0) {
+    dv.state[hs] = HeadState{pl.len, pl.n_drop, 0, pl.window};
+    dv.ring_valid[hs] = 0;   // nobody has summed the rows of the new window
+  }
 }
 
 // grid = (Hkv, sequences), block = 2*D threads: fixed-order sum of the slice partials, then the
@@ -294,7 +297,10 @@ __global__ void __launch_bounds__(64) append_kernel(DeviceView dv, int layer, co
       krow[kPageTokens * LPR] = vf;
     }
   }
-  if (active && lane == 0) dv.state[hs] = st;
+  if (active && lane == 0) {
+    dv.state[hs] = st;
+    dv.ring_valid[hs] = 0;   // the window's content changed and its sum was not kept up
+  }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -366,7 +372,10 @@ __global__ void __launch_bounds__(128) append_many_kernel(DeviceView dv, int lay
     }
     __syncwarp();   // a later token of the round may evict a row this one just stored
   }
-  if (lane == 0) dv.state[hs] = st;
+  if (lane == 0) {
+    dv.state[hs] = st;
+    dv.ring_valid[hs] = 0;
+  }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -378,6 +387,10 @@ __global__ void __launch_bounds__(128) append_many_kernel(DeviceView dv, int lay
 // after it has read the old row, so there is no order between CTAs to keep.  grid = (slices, heads);
 // per-slice sums go to the compression scratch and append_chunk_finalize_kernel adds them to the running
 // sums (Eq. 4 over everything dropped so far).
+// Old rows are not read back when the run evicts the whole window and the sum of the window's rows is on
+// record (ring_sum, kept by this kernel: every slice also sums the rows it stores into the window): that sum
+// is then the old rows' share of the dropped set.  A prefill handed over in chunks of at least the window
+// length therefore reads every row once and writes it once.
 template <typename T, int D>
 __global__ void __launch_bounds__(256) append_chunk_kernel(DeviceView dv, int layer, const T* __restrict__ k_new,
                                                            const T* __restrict__ v_new, int n_tok, int n_slices) {
@@ -393,10 +406,14 @@ __global__ void __launch_bounds__(256) append_chunk_kernel(DeviceView dv, int la
   const int per = (n_tok + n_slices - 1) / n_slices;
   const int a0 = min(n_tok, (int)blockIdx.x * per), a1 = min(n_tok, a0 + per);
   const int lir = threadIdx.x % LPR, grp = threadIdx.x / LPR;
+  // the whole old window leaves and its sum is known: no need to read its rows
+  const int ring_fill = st.window >= 0 && st.len > n_sink ? st.len - n_sink : 0;
+  const int n_evict = n_tok - append_run_fits(st, n_sink, n_tok);
+  const bool skip_old = st.window >= 0 && n_evict >= ring_fill && dv.ring_valid[hs] != 0;
 
-  float accK[EPL], accV[EPL];
+  float accK[EPL], accV[EPL], ringK[EPL], ringV[EPL];
 #pragma unroll
-  for (int i = 0; i < EPL; ++i) accK[i] = accV[i] = 0.f;
+  for (int i = 0; i < EPL; ++i) accK[i] = accV[i] = ringK[i] = ringV[i] = 0.f;
   for (int a = a0 + grp; a < a1; a += NGRP) {
     const size_t row = (((size_t)b * n_tok + a) * dv.n_kv_heads + g) * D;
     const uint4 kf = ld_stream((const uint4*)(k_new + row) + lir);
@@ -408,7 +425,7 @@ __global__ void __launch_bounds__(256) append_chunk_kernel(DeviceView dv, int la
     if (stays) {
       const size_t page = (size_t)pt[slot >> 4];
       uint4* dst = (uint4*)(dv.pool + page * dv.page_bytes + (size_t)(slot & 15) * Geo::kRowBytes) + swz(slot, lir);
-      if (had_old) {
+      if (had_old && !skip_old) {
         Elem<T>::unpack(dst[0], a_k);
         Elem<T>::unpack(dst[kPageTokens * LPR], a_v);
 #pragma unroll
@@ -416,6 +433,12 @@ __global__ void __launch_bounds__(256) append_chunk_kernel(DeviceView dv, int la
       }
       dst[0] = kf;
       dst[kPageTokens * LPR] = vf;
+      if (st.window >= 0 && slot >= n_sink) {   // a row of the new window
+        Elem<T>::unpack(kf, a_k);
+        Elem<T>::unpack(vf, a_v);
+#pragma unroll
+        for (int i = 0; i < EPL; ++i) { ringK[i] += a_k[i]; ringV[i] += a_v[i]; }
+      }
     } else {
       Elem<T>::unpack(kf, a_k);
       Elem<T>::unpack(vf, a_v);
@@ -423,18 +446,23 @@ __global__ void __launch_bounds__(256) append_chunk_kernel(DeviceView dv, int la
       for (int i = 0; i < EPL; ++i) { accK[i] += a_k[i]; accV[i] += a_v[i]; }
     }
   }
+  // two sets of sums per slice: rows that join the dropped set, rows stored into the window
+  float* scratch = dv.compress_scratch + ((size_t)head * n_slices + blockIdx.x) * 4 * D;
 #pragma unroll
-  for (int i = 0; i < EPL; ++i) {
-    red[grp][0][lir * EPL + i] = accK[i];
-    red[grp][1][lir * EPL + i] = accV[i];
-  }
-  __syncthreads();
-  float* scratch = dv.compress_scratch + ((size_t)head * n_slices + blockIdx.x) * 2 * D;
-  for (int e = threadIdx.x; e < 2 * D; e += 256) {
-    float sum = 0.f;
+  for (int set = 0; set < 2; ++set) {
+    if (set) __syncthreads();
 #pragma unroll
-    for (int r = 0; r < NGRP; ++r) sum += (&red[r][0][0])[e];
-    scratch[e] = sum;
+    for (int i = 0; i < EPL; ++i) {
+      red[grp][0][lir * EPL + i] = set ? ringK[i] : accK[i];
+      red[grp][1][lir * EPL + i] = set ? ringV[i] : accV[i];
+    }
+    __syncthreads();
+    for (int e = threadIdx.x; e < 2 * D; e += 256) {
+      float sum = 0.f;
+#pragma unroll
+      for (int r = 0; r < NGRP; ++r) sum += (&red[r][0][0])[e];
+      scratch[set * 2 * D + e] = sum;
+    }
   }
 }
 
@@ -446,15 +474,27 @@ __global__ void append_chunk_finalize_kernel(DeviceView dv, int layer, int n_tok
   const size_t hs = (size_t)layer * dv.n_heads + head;
   const HeadState st = dv.state[hs];
   const int E = n_tok - append_run_fits(st, dv.n_sink, n_tok);
+  const int ring_fill = st.window >= 0 && st.len > dv.n_sink ? st.len - dv.n_sink : 0;
+  const bool all_old_gone = st.window >= 0 && E >= ring_fill;        // the window holds rows of this run only
+  const bool skip_old = all_old_gone && dv.ring_valid[hs] != 0;      // (the streaming kernel decided the same)
+  const float* scratch = dv.compress_scratch + (size_t)head * n_slices * 4 * D;
   if (E > 0) {
-    const float* scratch = dv.compress_scratch + (size_t)head * n_slices * 2 * D;
     float s = dv.comp_sum[hs * 2 * D + e];
-    for (int i = 0; i < n_slices; ++i) s += scratch[(size_t)i * 2 * D + e];
+    if (skip_old) s += dv.ring_sum[hs * 2 * D + e];   // the old window's rows, summed when they were stored
+    for (int i = 0; i < n_slices; ++i) s += scratch[(size_t)i * 4 * D + e];
     dv.comp_sum[hs * 2 * D + e] = s;
     dv.comp_mean[hs * 2 * D + e] = __fdiv_rn(s, (float)(st.n_drop + E));
   }
-  __syncthreads();   // every thread has read the old state
-  if (e == 0) dv.state[hs] = state_after_run(st, dv.n_sink, n_tok);
+  if (all_old_gone) {
+    float r = 0.f;
+    for (int i = 0; i < n_slices; ++i) r += scratch[(size_t)i * 4 * D + 2 * D + e];
+    dv.ring_sum[hs * 2 * D + e] = r;
+  }
+  __syncthreads();   // every thread has read the old state and flag
+  if (e == 0) {
+    dv.state[hs] = state_after_run(st, dv.n_sink, n_tok);
+    dv.ring_valid[hs] = all_old_gone ? 1 : 0;
+  }
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -742,6 +742,7 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
             s.ring_head = (s.ring_head + 1 == s.window) ? 0 : s.ring_head + 1;
           }
           states[h] = s;
+          dv.ring_valid[(size_t)layer * dv.n_heads + h] = 0;   // the window's content changed and its sum was not kept up
         }
       }
     }

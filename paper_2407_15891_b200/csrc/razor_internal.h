@@ -145,6 +145,8 @@ struct DeviceView {
   HeadState* state;         // [L][B*Hkv]
   float* comp_sum;          // [L][B*Hkv][2][D]  (K sums then V sums)
   float* comp_mean;         // [L][B*Hkv][2][D]
+  float* ring_sum;          // [L][B*Hkv][2][D]  sum of the K and V rows now in the recent window, valid when ring_valid says so
+  int32_t* ring_valid;      // [L][B*Hkv]        1: ring_sum is up to date (only the bulk append keeps it so)
   int32_t* page_table;      // [L][B*Hkv][max_pages]
   WorkItem* items;          // [L][max_items]
   int32_t* jobs;            // [L][max_items + 1]  first item of every job (a span or one tail item), then n_items

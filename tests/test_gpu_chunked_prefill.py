@@ -60,6 +60,42 @@ def test_cache_built_chunk_by_chunk_from_empty(dtype, D, group):
     cache.close()
 
 
+def test_chunks_of_at_least_the_window_do_not_read_rows_back_and_stay_exact():
+    """Chunk after chunk of the window's length or more: the evicted rows' share of the Eq. 4 sums comes from the
+    recorded sum of the window, not from reading the rows again.  A one-launch decode step in between makes that
+    record stale (the next chunk must read the rows); the chunks after it use the record again."""
+    Hkv, D = 4, 128
+    plan = [256, 256, 300, 256, "step", 256, 256, 256]
+    total = sum(x for x in plan if x != "step") + 1
+    w = synth.Workload("window_chunks", 2, 1, Hkv, Hkv, D, "bf16", [0, 0], [256, 128], 4, 1, total, 7321)
+    cache = make_cache(w, max_new=total)
+    retr = w.retrieval(0)
+    cache.start_empty(0, retr, w.window)
+    dummy = torch.zeros((1, D), dtype=torch.bfloat16)
+    refs = {(b, g): HeadRef(0, b, g, dummy, dummy, 0, total) for b in range(w.batch) for g in range(Hkv)}
+    scale = 1.0 / math.sqrt(D)
+    for i, T in enumerate(plan):
+        q = _gen(w, synth.TAG_Q, (w.batch, w.n_q_heads, D), i)
+        if T == "step":
+            k1, v1 = synth.make_new_kv(w, 0, i, DEV)
+            out = to_f64(cache.decode_step(0, k1, v1, q))
+            kh, vh, n = k1.cpu()[:, None], v1.cpu()[:, None], 1
+        else:
+            k, v = _chunk(w, T, i)
+            cache.append_many(0, k, v)
+            out = to_f64(cache.decode(0, q))
+            kh, vh, n = k.cpu(), v.cpu(), T
+        assert cache.device_status() == 0
+        qh = to_f64(q)
+        for (b, g), ref in refs.items():
+            for t in range(n):
+                ref.append(kh[b, t, g], vh[b, t, g])
+            hc = check_head_state(cache, ref, w.n_sink, w.window[b], bool(retr[g]))
+            err = float(np.abs(out[b, g] - orc.decode_head(qh[b, g], hc, scale)).max())
+            assert err <= TOL_OUT["bf16"], (err, i, b, g)
+    cache.close()
+
+
 def test_chunked_prefill_equals_one_compression():
     """Same tokens, same windows: the exported caches agree bit for bit in layout, and in the means to rounding."""
     Hkv, D, N = 4, 128, 3000
