@@ -101,6 +101,8 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-dense", action="store_true")
+    ap.add_argument("--only-round", type=int, default=0, metavar="TOKENS",
+                    help="run only the long-round leg with TOKENS new tokens per sequence and print its line (profiling; not the bench line)")
     ap.add_argument("--only-head-scores", type=int, default=0, metavar="HEADS",
                     help="run only the head-score leg on HEADS heads and print its line (profiling; not the bench line)")
     return ap.parse_args()
@@ -518,6 +520,10 @@ def main():
         raise SystemExit("bench.py needs a CUDA device: the product has no CPU path")
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
+    if args.only_round > 0:
+        if rank == 0:
+            print(json.dumps(long_round_leg(rz, synth, dev, n_tok=args.only_round, reps=max(1, args.steps))))
+        return
     if args.only_head_scores > 0:
         if rank == 0:
             print(json.dumps(head_scores_leg(rz, synth, dev, reps=max(1, args.steps), heads=args.only_head_scores)))

@@ -18,6 +18,8 @@
 //     reference max and the sum, and writes P (a bf16 head plus a bf16 remainder) into shared memory in operand
 //     layout.  O accumulates in tensor memory over the item's blocks; the reference max may lag the true one by a
 //     factor of 2^8, and only when a row outruns it is the accumulator rescaled in place.
+// (Tried and dropped: two threads per query row, 64 columns each, with the block maxima exchanged through shared
+// memory - no faster: the softmax warps are bound by their instruction count per score, not by their number.)
 // Every wait is bounded in time; a wait that runs out sets the CTA's abort flag and a bit of the device status
 // word, copies and instructions in flight are waited for, tensor memory is released.
 #include <math_constants.h>
