@@ -791,13 +791,17 @@ static int round_impl(razor_cache_t* c, int32_t layer, const void* q, float* out
 // page and at the item's length as it is now.
 static void plan_early_prefetch(const razor_cache* c, int layer, DecodeJobs& jb) {
   std::memset(jb.early, 0, sizeof(jb.early));
+  jb.state_stable = 0;
   if (c->tune.early_prefetch <= 0 || c->writes_overflow) return;
   int n_writes = 0;
+  bool only_appends = true;
   for (const auto& wr : c->writes_since_decode) {
     if (wr.first != layer) continue;
-    if (wr.second != razor_cache::kWriteOneToken) return;
+    only_appends &= wr.second == razor_cache::kWriteOneToken;
     n_writes += 1;
   }
+  jb.state_stable = n_writes == 0 ? 1 : 0;   // nothing in flight writes this layer's head states
+  if (!only_appends) return;
   if (n_writes > 2) return;
   // rows written by appends that may be in flight: the newest n_writes ones; one more is left out for good
   // measure (in a launch that appends itself the mirror is already one token ahead)
@@ -876,7 +880,7 @@ static int decode_impl(razor_cache_t* c, int32_t layer, const void* q, float* ou
   rc = ensure_schedule(c, layer, (cudaStream_t)stream, true, (c->cfg.n_q_heads / c->cfg.n_kv_heads) * n_tokens);
   if (rc) return rc;
   const LayerHost& L = c->layers[layer];
-  DecodeJobs jb{L.n_items, L.n_jobs, L.n_spans, L.jobs[L.n_spans], L.n_multi, n_tokens, tok_stride, q_after, {},
+  DecodeJobs jb{L.n_items, L.n_jobs, L.n_spans, L.jobs[L.n_spans], L.n_multi, n_tokens, tok_stride, q_after, 0, {},
                 k_new, v_new};
   plan_early_prefetch(c, layer, jb);
   RZ_CUDA(launch_decode(c->dv, c->cfg.dtype, layer, jb, q, out, c->n_sms, c->tune,

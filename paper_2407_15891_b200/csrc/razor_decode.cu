@@ -477,15 +477,19 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
   // The spans are handed out by CTA index and the queue counts tail jobs only, so the producer can look
   // up its span, the span's first item and that item's first page ids right here: the schedule is written
   // by host copies only and the page table by host copies or the compression's plan kernel, which lies
-  // whole kernels back in the stream, so both may be read before the dependency below is resolved.
+  // whole kernels back in the stream, so both may be read before the dependency below is resolved.  The head
+  // state of the first item too, when the host says that nothing in flight writes this layer's states.
   int it0 = n_items, job_end0 = n_items;
   WorkItem w0 = no_item;
   int32_t pid0 = 0;
+  HeadState st0 = {0, 0, 0, 0};
   const bool has_span = (int)blockIdx.x < jb.n_spans;
+  const bool state_early = has_span && jb.state_stable != 0;   // the head states of this layer are at rest
   if (warp == NC && has_span) {
     job_range((int)blockIdx.x, it0, job_end0);
     w0 = it0 < n_items ? items[it0] : no_item;
     pid0 = first_pids(w0);
+    if (state_early) st0 = dv.state[row_of(w0)];
   }
   __syncthreads();
   // The first pages of the span go into the (still empty) ring right away: the host has named a run of
@@ -559,7 +563,7 @@ decode_kernel(DeviceView dv, int layer, DecodeJobs jb, const T* __restrict__ q, 
         bulk_load(&slots[0].q[t * g_real][0], q + row_offset(w.head, t * g_real), kQBytes / jb.n_tok, &bars.item_full[0]);
       q_issued = true;
     }
-    HeadState st = dv.state[row_of(w)];
+    HeadState st = state_early ? st0 : dv.state[row_of(w)];
     for (unsigned seq = 0; ok; ++seq) {
       const int slot = seq % kItemSlots;
       const bool need_pop = it < n_items && it + 1 >= job_end;   // the job ends with this item

@@ -214,6 +214,9 @@ struct DecodeJobs {
   // tokens of the round that come after the block (they are cached already, and masked).
   int32_t tok_stride;
   int32_t q_after;
+  // 1: no kernel that can still be in flight when this launch starts writes this layer's head states, so a CTA
+  // may load the state of its first work item ahead of the launch dependency (the host tracks the writers)
+  int32_t state_stable;
   // early[i]: how many of the first pages of CTA i's span (pages of the span's first work item, in order) may
   // be copied into the ring BEFORE the kernel waits for the launch it depends on.  The host knows every head's
   // length and which page the preceding append (if any) wrote, so it can name pages that nothing in flight
