@@ -53,13 +53,12 @@ struct RoundCtl {
   uint64_t o_read;                // softmax -> MMA: the item's output accumulator has been read out of tensor memory
   uint64_t item_ready;            // producer -> everyone: the next item index is in `item`
   uint64_t item_taken;            // MMA warp + softmax threads -> producer: `item` has been read
-  uint64_t blk_sync;              // the softmax threads among themselves, once per block (a bounded wait, unlike bar.sync)
+  uint64_t blk_sync;              // the softmax threads among themselves, once per masked block (a bounded wait, unlike bar.sync)
   uint64_t drain;
   uint32_t tmem_base;
   int abort_flag;
   int item;                       // index of the current work item, -1: no more
-  int32_t col_pos[2][kBlk];       // token position of each column of a block (two blocks may be in progress)
-  int32_t blk_flags[4];           // block g uses slot g % 4: 1 = the block needs masking
+  int32_t col_pos[2][kBlk];       // token position of each column of a masked block (two may be in progress)
 };
 
 template <int D>
@@ -172,7 +171,6 @@ __global__ void __launch_bounds__(kRoundThreads, 1)
     mbar_init(&ctl->blk_sync, kSoftmaxThreads);
     mbar_init(&ctl->drain, 1);
     ctl->abort_flag = 0;
-    for (int i = 0; i < 4; ++i) ctl->blk_flags[i] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {   // the MMA warp owns the tensor-memory allocation
@@ -331,7 +329,7 @@ __global__ void __launch_bounds__(kRoundThreads, 1)
     const int row = sw * 32 + lane;
     const uint32_t lane_addr = tmem + ((uint32_t)(sw * 32) << 16);
     const float scale_log2 = dv.scale_log2;
-    unsigned gb = 0;
+    unsigned gb = 0, n_sync = 0;   // blocks so far; exchanges of column positions so far
     bool ok = true;
     for (unsigned gi = 0; ok; ++gi) {
       ok = mbar_wait(&ctl->item_ready, gi & 1, abort_flag);
@@ -382,30 +380,39 @@ __global__ void __launch_bounds__(kRoundThreads, 1)
         l_run = 1.f;
         w_seed = 1.f;
       }
+      const bool in_order = st.window < 0 || st.n_drop == 0;               // slot = position
+      const int q_pos_min = total - jb.n_tok + w.q_tile * tok_per_tile;    // the tile's earliest query
+      int new_lo = 0, new_hi = 0, new_lo2 = 0, new_hi2 = 0;                // slot ranges [lo, hi) holding the round's tokens
+      if (!in_order) {
+        const int lo = ((st.ring_head - jb.n_tok) % st.window + st.window) % st.window;
+        if (jb.n_tok >= st.window) { new_lo = dv.n_sink; new_hi = dv.n_sink + st.window; }
+        else if (lo < st.ring_head) { new_lo = dv.n_sink + lo; new_hi = dv.n_sink + st.ring_head; }
+        else { new_lo = dv.n_sink + lo; new_hi = dv.n_sink + st.window; new_lo2 = dv.n_sink; new_hi2 = dv.n_sink + st.ring_head; }
+      }
       const int nb = w.blk_end - w.blk_begin;
       for (int i = 0; i < nb && ok; ++i) {
         const unsigned g = gb + i;
         const int sb = g & 1, blk = w.blk_begin + i;
         const int slot0 = blk * kBlk;
-        // does the block need masking: slots beyond the head's length, or tokens of the round that come after
-        // some query of this tile?  A thread looks at its own column; the four warps agree through a flag.
-        int my_pos;
-        {
+        // Does the block need masking?  Slots beyond the head's length, or tokens of the round (the newest n_tok: the
+        // last slots of a head whose slots are in position order, a cyclic run of the ring otherwise) that come
+        // after some query of the tile.  Every thread finds the same answer from the head's state, so the common
+        // case costs no exchange; in a block that does need it each thread works out the position of its own
+        // column and the four warps trade them through shared memory.
+        const int slot1 = slot0 + kBlk;
+        bool masked = slot1 > st.len;
+        if (in_order) masked |= slot1 - 1 > q_pos_min;
+        else masked |= (slot0 < new_hi && new_lo < slot1) || (slot0 < new_hi2 && new_lo2 < slot1);
+        const int32_t* col_pos = ctl->col_pos[n_sync & 1];
+        if (masked) {
           const int s = slot0 + row;   // column `row` of the block
-          my_pos = s < st.len ? slot_pos(s, dv.n_sink, st.ring_head, st.window, st.n_drop, total) : 0x7fffffff;
+          // (double-buffered: a thread may still be reading the positions of the masked block before)
+          ctl->col_pos[n_sync & 1][row] = s < st.len ? slot_pos(s, dv.n_sink, st.ring_head, st.window, st.n_drop, total) : 0x7fffffff;
+          mbar_arrive(&ctl->blk_sync);
+          ok = mbar_wait(&ctl->blk_sync, n_sync & 1, abort_flag);
+          if (!ok) break;
+          n_sync += 1;
         }
-        const int q_pos_min = total - jb.n_tok + w.q_tile * tok_per_tile;   // the tile's earliest query
-        const bool warp_needs = __any_sync(0xffffffffu, my_pos > q_pos_min);
-        // (slot g % 4 of the flags was cleared two blocks ago; col_pos is double-buffered: a thread may still be
-        // reading the block before while another writes this one)
-        ctl->col_pos[sb][row] = my_pos;
-        if (row == 0) ctl->blk_flags[(g + 2) & 3] = 0;
-        if (lane == 0 && warp_needs) atomicOr(&ctl->blk_flags[g & 3], 1);
-        mbar_arrive(&ctl->blk_sync);
-        ok = mbar_wait(&ctl->blk_sync, g & 1, abort_flag);
-        if (!ok) break;
-        const bool masked = ctl->blk_flags[g & 3] != 0;
-        const int32_t* col_pos = ctl->col_pos[sb];
         ok = mbar_wait(&ctl->s_full[sb], (g >> 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
