@@ -148,6 +148,24 @@ int main(void) {
       worst = err > worst ? err : worst;
     }
   }
+  /* the same decode step as ONE call: compress again (same pages), then razor_decode_step */
+  CHECK_RZ(razor_compress(cache, 0, dK, dV, (int64_t)H * N * D, (int64_t)N * D, D, ctx_len, retrieval, NSINK, window,
+                          NULL));
+  CHECK_RZ(razor_decode_step(cache, 0, dk1, dv1, dq, (float*)dout, NULL));
+  CHECK_CUDA(cudaMemcpy(out, dout, sizeof(out), cudaMemcpyDeviceToHost));
+  CHECK_RZ(razor_cache_device_status(cache, &status, NULL));
+  if (status != 0) {
+    fprintf(stderr, "device status %d after razor_decode_step\n", status);
+    return 1;
+  }
+  for (int h = 0; h < H; ++h) {
+    double want[D];
+    expected(h, retrieval[h], 1.0 / sqrt((double)D), want);
+    for (int d = 0; d < D; ++d) {
+      const double err = fabs((double)out[h][d] - want[d]);
+      worst = err > worst ? err : worst;
+    }
+  }
   CHECK_RZ(razor_cache_destroy(cache));
   cudaFree(pool); cudaFree(ws); cudaFree(dK); cudaFree(dV); cudaFree(dq); cudaFree(dk1); cudaFree(dv1); cudaFree(dout);
   if (!(worst <= 1e-5)) {

@@ -80,6 +80,30 @@ def test_static_scratch_with_strided_rows_and_with_the_most_heads_it_takes():
     assert _check_static(w2) == 900 - 4 - 120
 
 
+def test_static_scratch_call_on_a_second_stream_ordered_by_an_event():
+    """The built-in array is shared by every call on the device: a call on another stream is fine as long as
+    it is ordered behind the call before (here by an event), and gives the oracle's means too."""
+    w = synth.Workload("noalloc6", 1, 1, 4, 4, 128, "bf16", [3000], [500], 4, 0, 1, 31342)
+    K, V = synth.make_dense_kv(w, 0, DEV)
+    H, D = w.n_kv_heads, w.head_dim
+    out = [torch.empty((H, D), dtype=torch.float32, device=DEV) for _ in range(4)]
+    rz.razor_compensation_mean_static(K[0], V[0], K.stride(1), K.stride(2), H, D, rz.RAZOR_BF16, 3000, 4, 500, out[0], out[1])
+    done = torch.cuda.Event()
+    done.record()
+    side = torch.cuda.Stream()
+    side.wait_event(done)
+    with torch.cuda.stream(side):
+        nd = rz.razor_compensation_mean_static(K[0], V[0], K.stride(1), K.stride(2), H, D, rz.RAZOR_BF16, 2000, 4, 300,
+                                               out[2], out[3], stream=side.cuda_stream)
+    torch.cuda.synchronize()
+    assert nd == 2000 - 4 - 300
+    for (n, win, mk, mv) in ((3000, 500, out[0], out[1]), (2000, 300, out[2], out[3])):
+        drop = orc.dropped_positions(n, 4, win, False)
+        for g in range(H):
+            k_hat, v_hat, _ = orc.compensation_token(to_f64(K[0, g]), to_f64(V[0, g]), drop)
+            assert rel_inf(to_f64(mk)[g], k_hat) <= TOL_MEAN_REL and rel_inf(to_f64(mv)[g], v_hat) <= TOL_MEAN_REL
+
+
 def test_static_scratch_rejects_what_does_not_fit():
     z = torch.zeros((65, 64), dtype=torch.float32, device=DEV)
     with pytest.raises(rz.RazorError) as e:
