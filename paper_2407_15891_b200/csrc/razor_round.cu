@@ -35,7 +35,7 @@ namespace {
 
 constexpr int kRows = kRoundTileRows;      // query rows per tile = accumulator rows = tensor-memory lanes
 constexpr int kBlk = kRoundBlockTokens;    // tokens per block = columns of S
-constexpr int kKvStages = 2;
+constexpr int kKvStages = 3;
 constexpr int kRoundThreads = 6 * 32;
 constexpr int kSoftmaxThreads = 128;
 constexpr int kHalfBytes = kRows * 128;    // one 64-element half of a 128-row operand tile
@@ -46,10 +46,10 @@ struct RoundCtl {
   uint64_t k_empty[kKvStages];    // MMA (commit of S = Q K^T) -> TMA
   uint64_t v_full[kKvStages];     // the same for V; a V stage is free once O += P V has run
   uint64_t v_empty[kKvStages];
-  uint64_t s_full[2];             // MMA (commit) -> softmax: S buffer holds a block's scores
-  uint64_t s_empty[2];            // softmax -> MMA: S buffer read out
-  uint64_t p_full;                // softmax -> MMA: P of the block is in shared memory
-  uint64_t p_empty;               // MMA (commit) -> softmax: P has been consumed
+  uint64_t s_full;                // MMA (commit) -> softmax: S holds a block's scores
+  uint64_t s_empty;               // softmax -> MMA: S read out into registers
+  uint64_t p_full[2];             // softmax -> MMA: P of the block is in its tensor-memory buffer
+  uint64_t p_empty[2];            // MMA (commit) -> softmax: the product that read the buffer has run
   uint64_t o_read;                // softmax -> MMA: the item's output accumulator has been read out of tensor memory
   uint64_t item_ready;            // producer -> everyone: the next item index is in `item`
   uint64_t item_taken;            // MMA warp + softmax threads -> producer: `item` has been read
@@ -63,8 +63,8 @@ struct RoundCtl {
 
 template <int D>
 constexpr size_t round_smem_bytes() {
-  // 1 KB alignment slack, Q tile, K and V stages, P tile (head and remainder), control block
-  return 1024 + (size_t)kRows * D * 2 + (size_t)kKvStages * 2 * kBlk * D * 2 + 2 * (size_t)kRows * kBlk * 2 + sizeof(RoundCtl);
+  // 1 KB alignment slack, Q tile, K and V stages, control block
+  return 1024 + (size_t)kRows * D * 2 + (size_t)kKvStages * 2 * kBlk * D * 2 + sizeof(RoundCtl);
 }
 
 // One page half: 16 tokens x 64 elements of K or V of pool page `pid` into shared memory (2 KB).
@@ -104,6 +104,16 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* v) {
         "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
       : "memory");
 }
+// The same for 16 columns.
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* v) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+      :
+      : "r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]),
+        "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+      : "memory");
+}
 __device__ __forceinline__ void tmem_st_wait_all() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // 2^t on the FMA and integer pipes, relative error below 5e-5 (t = n + f, n the nearest integer, 2^f as a
@@ -133,19 +143,20 @@ __global__ void __launch_bounds__(kRoundThreads, 1)
     round_kernel(DeviceView dv, const __grid_constant__ CUtensorMap map_pool, int layer, RoundJobs jb,
                  const __nv_bfloat16* __restrict__ q, float* __restrict__ out) {
   constexpr int HALVES = D / 64;
-  constexpr int Q_BYTES = kRows * D * 2, KV_TILE = kBlk * D * 2, P_BYTES = kRows * kBlk * 2;
+  constexpr int Q_BYTES = kRows * D * 2, KV_TILE = kBlk * D * 2;
   constexpr uint32_t kIdescQK = instr_desc_bf16(kRows, kBlk, false);
   constexpr uint32_t kIdescPV = instr_desc_bf16(kRows, D, true);
   constexpr uint32_t kTmemCols = 512;
-  constexpr uint32_t kOCol = 2 * kBlk;   // first column of the output accumulator
+  // tensor memory: S in columns [0, 128), the output accumulator in [128, 128 + D), two buffers of P in [256, 384) and
+  // [384, 512): a row's 128 weights as 64 columns of bf16 pairs (the heads) and 64 more (the remainders)
+  constexpr uint32_t kOCol = kBlk, kPCol = 2 * kBlk, kPBuf = kBlk, kPLo = kBlk / 2;
 
   extern __shared__ uint8_t round_smem_raw[];
   uint8_t* base = round_smem_raw + ((1024u - (smem_u32(round_smem_raw) & 1023u)) & 1023u);
   uint8_t* q_tile = base;
   uint8_t* k_tile = q_tile + Q_BYTES;                    // [stage][half][128 tokens][128 B]
   uint8_t* v_tile = k_tile + kKvStages * KV_TILE;
-  uint8_t* p_tile = v_tile + kKvStages * KV_TILE;        // [head | remainder][half of the tokens][128 rows][128 B]
-  RoundCtl* ctl = (RoundCtl*)(p_tile + 2 * P_BYTES);
+  RoundCtl* ctl = (RoundCtl*)(v_tile + kKvStages * KV_TILE);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   volatile int* abort_flag = &ctl->abort_flag;
@@ -159,12 +170,12 @@ __global__ void __launch_bounds__(kRoundThreads, 1)
       mbar_init(&ctl->v_full[s], 1);
       mbar_init(&ctl->v_empty[s], 1);
     }
+    mbar_init(&ctl->s_full, 1);
+    mbar_init(&ctl->s_empty, kSoftmaxThreads);
     for (int s = 0; s < 2; ++s) {
-      mbar_init(&ctl->s_full[s], 1);
-      mbar_init(&ctl->s_empty[s], kSoftmaxThreads);
+      mbar_init(&ctl->p_full[s], kSoftmaxThreads);
+      mbar_init(&ctl->p_empty[s], 1);
     }
-    mbar_init(&ctl->p_full, kSoftmaxThreads);
-    mbar_init(&ctl->p_empty, 1);
     mbar_init(&ctl->o_read, kSoftmaxThreads);
     mbar_init(&ctl->item_ready, 1);
     mbar_init(&ctl->item_taken, kSoftmaxThreads + 1);
@@ -213,10 +224,11 @@ __global__ void __launch_bounds__(kRoundThreads, 1)
       auto page_of = [&](int blk) { return lane < 8 ? pt[min(blk * 8 + lane, max(head_pages - 1, 0))] : 0; };
       int pid = w.blk_begin < w.blk_end ? page_of(w.blk_begin) : 0;
       for (int blk = w.blk_begin; blk < w.blk_end && ok; ++blk, ++gb) {
-        const int s = gb & 1;
+        const int s = gb % kKvStages;
+        const unsigned use = gb / kKvStages;   // how often the stage has been filled before
         const int pid_next = blk + 1 < w.blk_end ? page_of(blk + 1) : 0;
-        // K of the block: its stage is free as soon as the scores of two blocks ago have been computed
-        if (gb >= kKvStages) ok = __all_sync(0xffffffffu, mbar_wait(&ctl->k_empty[s], ((gb >> 1) - 1) & 1, abort_flag));
+        // K of the block: its stage is free as soon as the scores of three blocks ago have been computed
+        if (gb >= kKvStages) ok = __all_sync(0xffffffffu, mbar_wait(&ctl->k_empty[s], (use - 1) & 1, abort_flag));
         if (!ok) break;
         if (lane == 0) mbar_arrive_expect_tx(&ctl->k_full[s], (uint32_t)KV_TILE);
         __syncwarp();
@@ -227,7 +239,7 @@ __global__ void __launch_bounds__(kRoundThreads, 1)
         }
         issued_k = gb + 1;
         // V of the block: its stage is free once the product of two blocks ago has run
-        if (gb >= kKvStages) ok = __all_sync(0xffffffffu, mbar_wait(&ctl->v_empty[s], ((gb >> 1) - 1) & 1, abort_flag));
+        if (gb >= kKvStages) ok = __all_sync(0xffffffffu, mbar_wait(&ctl->v_empty[s], (use - 1) & 1, abort_flag));
         if (!ok) break;
         if (lane == 0) mbar_arrive_expect_tx(&ctl->v_full[s], (uint32_t)KV_TILE);
         __syncwarp();
@@ -245,9 +257,9 @@ __global__ void __launch_bounds__(kRoundThreads, 1)
       if (lane == 0) {
         atomicOr(dv.status, kStatusProducerTimeout);
         for (unsigned g = issued_k > kKvStages ? issued_k - kKvStages : 0; g < issued_k; ++g)
-          if (!mbar_wait_drain(&ctl->k_full[g & 1], (g >> 1) & 1)) atomicOr(dv.status, kStatusDrainTimeout);
+          if (!mbar_wait_drain(&ctl->k_full[g % kKvStages], (g / kKvStages) & 1)) atomicOr(dv.status, kStatusDrainTimeout);
         for (unsigned g = issued_v > kKvStages ? issued_v - kKvStages : 0; g < issued_v; ++g)
-          if (!mbar_wait_drain(&ctl->v_full[g & 1], (g >> 1) & 1)) atomicOr(dv.status, kStatusDrainTimeout);
+          if (!mbar_wait_drain(&ctl->v_full[g % kKvStages], (g / kKvStages) & 1)) atomicOr(dv.status, kStatusDrainTimeout);
       }
     }
     // queue at rest again for the next launch
@@ -265,26 +277,27 @@ __global__ void __launch_bounds__(kRoundThreads, 1)
     if (lane == 0) {
       unsigned gb = 0;
       bool ok = true;
-      const uint32_t q0 = smem_u32(q_tile), p0 = smem_u32(p_tile);
+      const uint32_t q0 = smem_u32(q_tile);
       // O = sum over the item's blocks of P V, accumulated in tensor memory (the softmax threads rescale it there on
-      // the rare occasions a row's reference maximum moves).
+      // the rare occasions a row's reference maximum moves).  P is read out of tensor memory (operand A), V out of
+      // shared memory.
       auto issue_pv = [&](unsigned g, bool first_of_item, unsigned gi) -> bool {
-        const int s = g & 1;
-        if (!mbar_wait(&ctl->p_full, g & 1, abort_flag)) return false;
-        if (!mbar_wait(&ctl->v_full[s], (g >> 1) & 1, abort_flag)) return false;
+        const int s = g % kKvStages, pb = g & 1;
+        if (!mbar_wait(&ctl->p_full[pb], (g >> 1) & 1, abort_flag)) return false;
+        if (!mbar_wait(&ctl->v_full[s], (g / kKvStages) & 1, abort_flag)) return false;
         // the first product of an item overwrites the accumulator: the item before must have been read out
         if (first_of_item && gi >= 1 && !mbar_wait(&ctl->o_read, (gi - 1) & 1, abort_flag)) return false;
         tc_fence_after();
         const uint32_t v0 = smem_u32(v_tile + s * KV_TILE);
+        const uint32_t p0 = tmem + kPCol + (uint32_t)pb * kPBuf;
 #pragma unroll
-        for (int kk = 0; kk < kBlk / 16; ++kk) {   // 16 tokens per instruction
-          const uint32_t a_off = (uint32_t)((kk >> 2) * kHalfBytes + (kk & 3) * 32);
+        for (int kk = 0; kk < kBlk / 16; ++kk) {   // 16 tokens per instruction: 8 columns of bf16 pairs
           const uint64_t db = operand_desc_mn(v0 + (uint32_t)(kk * 16 * 128), kHalfBytes, 1024);
-          umma_bf16_desc(tmem + kOCol, operand_desc(p0 + a_off), db, kIdescPV, (kk > 0 || !first_of_item) ? 1u : 0u);
-          umma_bf16_desc(tmem + kOCol, operand_desc(p0 + P_BYTES + a_off), db, kIdescPV, 1);
+          umma_bf16_tmem_a(tmem + kOCol, p0 + (uint32_t)(kk * 8), db, kIdescPV, (kk > 0 || !first_of_item) ? 1u : 0u);
+          umma_bf16_tmem_a(tmem + kOCol, p0 + kPLo + (uint32_t)(kk * 8), db, kIdescPV, 1);
         }
         umma_commit(&ctl->v_empty[s]);
-        umma_commit(&ctl->p_empty);
+        umma_commit(&ctl->p_empty[pb]);
         return true;
       };
       for (unsigned gi = 0; ok; ++gi) {
@@ -298,19 +311,20 @@ __global__ void __launch_bounds__(kRoundThreads, 1)
         ok = mbar_wait(&ctl->q_ready, gi & 1, abort_flag);
         for (int i = 0; i < nb && ok; ++i) {
           const unsigned g = gb + i;
-          const int s = g & 1;
-          ok = mbar_wait(&ctl->k_full[s], (g >> 1) & 1, abort_flag);
-          if (ok && g >= 2) ok = mbar_wait(&ctl->s_empty[s], ((g >> 1) - 1) & 1, abort_flag);
+          const int s = g % kKvStages;
+          ok = mbar_wait(&ctl->k_full[s], (g / kKvStages) & 1, abort_flag);
+          // S is overwritten: the softmax threads must have the scores of the block before in registers
+          if (ok && g >= 1) ok = mbar_wait(&ctl->s_empty, (g - 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
           const uint32_t k0 = smem_u32(k_tile + s * KV_TILE);
 #pragma unroll
           for (int kk = 0; kk < D / 16; ++kk) {   // 16 elements = 32 bytes along the swizzled half row
             const uint32_t off = (uint32_t)((kk >> 2) * kHalfBytes + (kk & 3) * 32);
-            umma_bf16_desc(tmem + (uint32_t)(s * kBlk), operand_desc(q0 + off), operand_desc(k0 + off), kIdescQK, kk > 0);
+            umma_bf16_desc(tmem, operand_desc(q0 + off), operand_desc(k0 + off), kIdescQK, kk > 0);
           }
           umma_commit(&ctl->k_empty[s]);
-          umma_commit(&ctl->s_full[s]);
+          umma_commit(&ctl->s_full);
           if (i >= 1) ok = issue_pv(g - 1, i == 1, gi);   // behind the next block's scores, so that its softmax overlaps this product
         }
         if (ok && nb > 0) ok = issue_pv(gb + nb - 1, nb == 1, gi);
@@ -392,7 +406,7 @@ __global__ void __launch_bounds__(kRoundThreads, 1)
       const int nb = w.blk_end - w.blk_begin;
       for (int i = 0; i < nb && ok; ++i) {
         const unsigned g = gb + i;
-        const int sb = g & 1, blk = w.blk_begin + i;
+        const int pb = g & 1, blk = w.blk_begin + i;
         const int slot0 = blk * kBlk;
         // Does the block need masking?  Slots beyond the head's length, or tokens of the round (the newest n_tok: the
         // last slots of a head whose slots are in position order, a cyclic run of the ring otherwise) that come
@@ -413,19 +427,19 @@ __global__ void __launch_bounds__(kRoundThreads, 1)
           if (!ok) break;
           n_sync += 1;
         }
-        ok = mbar_wait(&ctl->s_full[sb], (g >> 1) & 1, abort_flag);
+        ok = mbar_wait(&ctl->s_full, g & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
 
         // ---- this row's 128 scores, in registers
         uint32_t v[kBlk];
 #pragma unroll
-        for (int c = 0; c < kBlk / 32; ++c) tmem_ld32_issue(lane_addr + (uint32_t)(sb * kBlk + c * 32), v + c * 32);
+        for (int c = 0; c < kBlk / 32; ++c) tmem_ld32_issue(lane_addr + (uint32_t)(c * 32), v + c * 32);
         tmem_ld_wait_all();
 #pragma unroll
         for (int e = 0; e < kBlk; ++e) asm volatile("" : "+r"(v[e]));
         tc_fence_before();
-        mbar_arrive(&ctl->s_empty[sb]);
+        mbar_arrive(&ctl->s_empty);
         if (masked) {
 #pragma unroll
           for (int e = 0; e < kBlk; ++e)
@@ -437,15 +451,17 @@ __global__ void __launch_bounds__(kRoundThreads, 1)
         // (the scale is positive: the max of the scaled scores is the scaled max)
         const float m_blk = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale_log2;
 
-        // ---- the product of the block before must be done before P is overwritten (and before O is touched)
-        if (g >= 1) ok = mbar_wait(&ctl->p_empty, (g - 1) & 1, abort_flag);
+        // ---- the product that read this buffer of P (two blocks ago) must have run before it is overwritten
+        if (g >= 2) ok = mbar_wait(&ctl->p_empty[pb], ((g >> 1) - 1) & 1, abort_flag);
         if (!ok) break;
         // ---- move the reference maximum?  Tensor-memory loads and stores are warp-wide, so the warp decides as one.
         const bool want = m_blk > m_ref + kLag || (m_ref == -CUDART_INF_F && m_blk > -CUDART_INF_F);
         if (__any_sync(0xffffffffu, want)) {
           const float m_to = fmaxf(m_ref, m_blk);
           const float f = (m_to == -CUDART_INF_F || m_ref == -CUDART_INF_F) ? 0.f : fast_exp2(m_ref - m_to);   // 1 for a row that stays
-          if (i >= 1) {   // the accumulator holds products of this item: rescale this warp's rows
+          if (i >= 1) {   // the accumulator holds products of this item: rescale this warp's rows, once the last has run
+            ok = mbar_wait(&ctl->p_empty[pb ^ 1], ((g - 1) >> 1) & 1, abort_flag);
+            if (!ok) break;
             tc_fence_after();
 #pragma unroll
             for (int c = 0; c < D / 32; ++c) {
@@ -468,49 +484,52 @@ __global__ void __launch_bounds__(kRoundThreads, 1)
         }
         const float m_use = (m_ref == -CUDART_INF_F) ? 0.f : m_ref;
 
-        // ---- weights, their sum, and P into shared memory (operand layout: 128-byte half rows, chunks swizzled by the row)
+        // ---- weights, their sum, and P into its tensor-memory buffer: column c of the head half holds the bf16 pair of
+        // tokens 2c and 2c + 1 (the operand-A layout of the matrix unit), the remainder half the same
         float psum4[4] = {0.f, 0.f, 0.f, 0.f};
+        const uint32_t p_addr = lane_addr + kPCol + (uint32_t)pb * kPBuf;
 #pragma unroll
-        for (int ch = 0; ch < kBlk / 8; ++ch) {   // 8 tokens = one 16-byte chunk of the row
-          uint32_t hi[4], lo[4];
+        for (int c = 0; c < kBlk / 32; ++c) {   // 32 tokens = 16 columns of pairs
+          uint32_t hi[16], lo[16];
 #pragma unroll
-          for (int e2 = 0; e2 < 4; ++e2) {
-            const int e = ch * 8 + e2 * 2;
+          for (int e2 = 0; e2 < 16; ++e2) {
+            const int e = c * 32 + e2 * 2;
             const float t0 = fmaf(__uint_as_float(v[e]), scale_log2, -m_use), t1 = fmaf(__uint_as_float(v[e + 1]), scale_log2, -m_use);
             // every fourth pair of exponentials on the FMA pipe instead of the transcendental unit
-            const float w0 = (e2 == 3) ? exp2_poly(t0) : fast_exp2(t0);
-            const float w1 = (e2 == 3) ? exp2_poly(t1) : fast_exp2(t1);
-            psum4[e2] += w0 + w1;
+            const float w0 = (e2 & 3) == 3 ? exp2_poly(t0) : fast_exp2(t0);
+            const float w1 = (e2 & 3) == 3 ? exp2_poly(t1) : fast_exp2(t1);
+            psum4[e2 & 3] += w0 + w1;
             // the weight goes into the product as a bf16 head plus a bf16 remainder (two products), so that it
             // keeps fp32-like accuracy: a single bf16 would put 2^-9 of a large weight times its V row into the result
             const __nv_bfloat162 h2 = __floats2bfloat162_rn(w0, w1);
             hi[e2] = *(const uint32_t*)&h2;
             lo[e2] = pack2_bf16(w0 - __low2float(h2), w1 - __high2float(h2));
           }
-          const uint32_t at = (uint32_t)((ch >> 3) * kHalfBytes + row * 128 + (((ch & 7) ^ (row & 7)) << 4));
-          *(uint4*)(p_tile + at) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-          *(uint4*)(p_tile + P_BYTES + at) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+          tmem_st16(p_addr + (uint32_t)(c * 16), hi);
+          tmem_st16(p_addr + kPLo + (uint32_t)(c * 16), lo);
         }
         l_run += (psum4[0] + psum4[1]) + (psum4[2] + psum4[3]);
         // V rows of slots beyond the head's length may hold anything (a zero weight times a NaN is a NaN): zero them
         if (slot0 + kBlk > st.len) {
-          ok = mbar_wait(&ctl->v_full[sb], (g >> 1) & 1, abort_flag);   // the rows must have landed before they are overwritten
+          ok = mbar_wait(&ctl->v_full[g % kKvStages], (g / kKvStages) & 1, abort_flag);   // the rows must have landed before they are overwritten
           if (!ok) break;
           const int first_bad = max(st.len - slot0, 0);
-          uint8_t* vt = v_tile + sb * KV_TILE;
+          uint8_t* vt = v_tile + (g % kKvStages) * KV_TILE;
           for (int idx = first_bad * 8 + row; idx < kBlk * 8; idx += kSoftmaxThreads) {   // 16-byte chunks of the bad rows
 #pragma unroll
             for (int h = 0; h < HALVES; ++h) *(uint4*)(vt + h * kHalfBytes + idx * 16) = make_uint4(0u, 0u, 0u, 0u);
           }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        mbar_arrive(&ctl->p_full);
+        tmem_st_wait_all();
+        tc_fence_before();
+        mbar_arrive(&ctl->p_full[pb]);
       }
       if (!ok) break;
       // ---- the row's result: accumulator out of tensor memory once the last product is done, plus the
       // compensation token's share; the output when the unit is in one part, else a partial record
       if (nb > 0) {
-        ok = mbar_wait(&ctl->p_empty, (gb + nb - 1) & 1, abort_flag);
+        ok = mbar_wait(&ctl->p_empty[(gb + nb - 1) & 1], ((gb + nb - 1) >> 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
       }
