@@ -36,8 +36,8 @@ namespace {
 constexpr int kRows = kRoundTileRows;      // query rows per tile = accumulator rows = tensor-memory lanes
 constexpr int kBlk = kRoundBlockTokens;    // tokens per block = columns of S
 constexpr int kKvStages = 3;
-constexpr int kRoundThreads = 6 * 32;
-constexpr int kSoftmaxThreads = 128;
+constexpr int kRoundThreads = 10 * 32;
+constexpr int kSoftmaxThreads = 256;
 constexpr int kHalfBytes = kRows * 128;    // one 64-element half of a 128-row operand tile
 
 struct RoundCtl {
@@ -91,43 +91,73 @@ __device__ __forceinline__ uint32_t pack2_bf16(float lo, float hi) {
   return *(const uint32_t*)&v;
 }
 
-// 32 consecutive columns of this thread's lane into tensor memory; complete after tmem_st_wait_all().
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* v) {
+// Fragment-shaped accesses: a warp touches 16 lanes (taddr's lane, a multiple of 16, onwards).  Thread t of the warp
+// owns lanes t / 4 and t / 4 + 8 and, in each group of columns, the columns picked by t % 4:
+//   .16x256b (groups of 8 columns): registers 4j .. 4j + 3 of group j are (lane t/4, columns 8j + 2(t%4) and + 1),
+//                                   (lane t/4 + 8, the same two columns);
+//   .16x128b (groups of 4 columns): registers 2j, 2j + 1 of group j are (lane t/4, column 4j + t%4), (lane t/4 + 8,
+//                                   the same column).
+// So the two fp32 values a thread reads from columns 2c, 2c + 1 of S become, as a bf16 pair, its column c of P.
+#define RAZOR_R8(v, o) "r"(v[o]), "r"(v[o + 1]), "r"(v[o + 2]), "r"(v[o + 3]), "r"(v[o + 4]), "r"(v[o + 5]), "r"(v[o + 6]), "r"(v[o + 7])
+#define RAZOR_W8(v, o) "=r"(v[o]), "=r"(v[o + 1]), "=r"(v[o + 2]), "=r"(v[o + 3]), "=r"(v[o + 4]), "=r"(v[o + 5]), "=r"(v[o + 6]), "=r"(v[o + 7])
+// 64 columns (8 groups of 8) of 16 lanes into 32 registers; valid after tmem_ld_wait_all().
+__device__ __forceinline__ void tmem_ld_frag64(uint32_t taddr, uint32_t* v) {
   asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "tcgen05.ld.sync.aligned.16x256b.x8.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : RAZOR_W8(v, 0), RAZOR_W8(v, 8), RAZOR_W8(v, 16), RAZOR_W8(v, 24)
+      : "r"(taddr)
+      : "memory");
+}
+// The store of the same shape; complete after tmem_st_wait_all().
+__device__ __forceinline__ void tmem_st_frag64(uint32_t taddr, const uint32_t* v) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.16x256b.x8.b32 [%0], "
       "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
       "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
       :
-      : "r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]),
-        "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]), "r"(v[16]), "r"(v[17]),
-        "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]), "r"(v[24]), "r"(v[25]), "r"(v[26]),
-        "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
+      : "r"(taddr), RAZOR_R8(v, 0), RAZOR_R8(v, 8), RAZOR_R8(v, 16), RAZOR_R8(v, 24)
       : "memory");
 }
-// The same for 16 columns.
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* v) {
+// 32 columns (8 groups of 4) of 16 lanes out of 16 registers.
+__device__ __forceinline__ void tmem_st_frag32(uint32_t taddr, const uint32_t* v) {
   asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "tcgen05.st.sync.aligned.16x128b.x8.b32 [%0], "
       "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
       :
-      : "r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]),
-        "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+      : "r"(taddr), RAZOR_R8(v, 0), RAZOR_R8(v, 8)
       : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait_all() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
-// 2^t on the FMA and integer pipes, relative error below 5e-5 (t = n + f, n the nearest integer, 2^f as a
-// degree-4 polynomial, n added onto the exponent field); t is clamped to [-125, 125].
-__device__ __forceinline__ float exp2_poly(float t) {
-  t = fminf(fmaxf(t, -125.f), 125.f);
-  const float r = t + 12582912.f;
-  const float f = t - (r - 12582912.f);
-  float p = 0.0096181291f;
-  p = fmaf(p, f, 0.0555041087f);
-  p = fmaf(p, f, 0.2402265070f);
-  p = fmaf(p, f, 0.6931471806f);
-  p = fmaf(p, f, 1.0f);
-  return __int_as_float(__float_as_int(p) + (__float_as_int(r) << 23));
+// Two fp32 values in a 64-bit register pair, and the arithmetic that works on both at once (one instruction slot
+// for two scores); the larger of three values in one instruction.
+__device__ __forceinline__ uint64_t f2_pack(float a, float b) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ void f2_unpack(uint64_t v, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v)); }
+__device__ __forceinline__ uint64_t f2_fma(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+__device__ __forceinline__ uint64_t f2_add(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ uint64_t f2_sub(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
 }
 
 // Position of the token in slot s of a head (Algorithm 1 keeps the sinks and a ring of the recent tokens).
@@ -338,10 +368,15 @@ __global__ void __launch_bounds__(kRoundThreads, 1)
     }
     __syncwarp();
   } else {
-    // ================================================================ softmax and epilogue: a thread per query row
-    const int sw = warp & 3;                     // tensor-memory lane quarter this warp may read
-    const int row = sw * 32 + lane;
-    const uint32_t lane_addr = tmem + ((uint32_t)(sw * 32) << 16);
+    // ================================================================ softmax and epilogue: four threads per query row
+    // A warp works on 16 tensor-memory lanes (query rows) in the fragment layout of the .16x256b loads: thread t has
+    // rows t / 4 and t / 4 + 8 of them and, of every 8 columns, the pair 2 (t % 4), 2 (t % 4) + 1.  Two warps share a
+    // lane quarter (and a scheduler), so one's transcendental and conversion work overlaps the other's arithmetic.
+    const int tid = (int)threadIdx.x - 64;                 // 0 .. 255 among the softmax threads
+    const int lane0 = (warp & 3) * 32 + ((warp - 2) >> 2) * 16;   // first of the warp's 16 lanes (a warp may access the quarter warp % 4)
+    const int cq = lane & 3;
+    const int row0 = lane0 + (lane >> 2);                  // the thread's rows: row0 and row0 + 8
+    const uint32_t lane_addr = tmem + ((uint32_t)lane0 << 16);
     const float scale_log2 = dv.scale_log2;
     unsigned gb = 0, n_sync = 0;   // blocks so far; exchanges of column positions so far
     bool ok = true;
@@ -356,43 +391,74 @@ __global__ void __launch_bounds__(kRoundThreads, 1)
       const HeadState st = dv.state[hs];
       const int b = w.head / dv.n_kv_heads, g_kv = w.head % dv.n_kv_heads;
       const int total = st.len + st.n_drop;
-      // this row: query token t (within the round), query head j of the group
-      const int t = w.q_tile * tok_per_tile + row / G, j = row % G;
-      const bool row_live = t < jb.n_tok;
-      const int q_pos = total - jb.n_tok + t;
-      const size_t row_off = (((size_t)b * jb.n_tok + min(t, jb.n_tok - 1)) * ((size_t)dv.n_kv_heads * G) + (size_t)g_kv * G + j) * D;
+      // row -> query token t (within the round) and query head j of the group
+      auto row_token = [&](int row) { return w.q_tile * tok_per_tile + row / G; };
+      auto row_offset = [&](int row) {
+        const int t = row_token(row), j = row % G;
+        return (((size_t)b * jb.n_tok + min(t, jb.n_tok - 1)) * ((size_t)dv.n_kv_heads * G) + (size_t)g_kv * G + j) * D;
+      };
+      bool row_live[2];
+      int q_pos[2];
+      size_t row_off[2];
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        const int t = row_token(row0 + 8 * r);
+        row_live[r] = t < jb.n_tok;
+        q_pos[r] = total - jb.n_tok + t;
+        row_off[r] = row_offset(row0 + 8 * r);
+      }
 
-      // ---- the query row into shared memory (operand layout: 128-byte half rows, chunks swizzled by the row)
-      const bool seed = w.part_idx == 0 && dv.use_comp && st.n_drop > 0 && st.window >= 0;
-      float s_c = 0.f;
+      // ---- the query tile into shared memory (operand layout: 128-byte half rows, chunks swizzled by the row):
+      // two threads per row, half a row each
       {
-        const uint4* src = (const uint4*)(q + row_off);
-        const float* k_hat = dv.comp_mean + hs * 2 * D;
+        const int qr = tid >> 1;
+        const bool live = row_token(qr) < jb.n_tok;
+        const uint4* src = (const uint4*)(q + row_offset(qr));
 #pragma unroll
-        for (int c = 0; c < D / 8; ++c) {
-          uint4 u = row_live ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);
-          *(uint4*)(q_tile + (c >> 3) * kHalfBytes + row * 128 + (((c & 7) ^ (row & 7)) << 4)) = u;
-          if (seed) {
-            float f[8];
-            Elem<__nv_bfloat16>::unpack(u, f);
-#pragma unroll
-            for (int e = 0; e < 8; ++e) s_c = fmaf(f[e], k_hat[c * 8 + e], s_c);
-          }
+        for (int cc = 0; cc < D / 16; ++cc) {
+          const int c = (tid & 1) * (D / 16) + cc;
+          const uint4 u = live ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);
+          *(uint4*)(q_tile + (c >> 3) * kHalfBytes + qr * 128 + (((c & 7) ^ (qr & 7)) << 4)) = u;
         }
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       mbar_arrive(&ctl->q_ready);
 
+      // ---- the compensation token's score q . k_hat of the thread's two rows: a quarter of the row each, summed
+      // over the four threads
+      const bool seed = w.part_idx == 0 && dv.use_comp && st.n_drop > 0 && st.window >= 0;
+      float s_c[2] = {0.f, 0.f};
+      if (seed) {
+        const float* k_hat = dv.comp_mean + hs * 2 * D;
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+          const uint4* src = (const uint4*)(q + row_off[r]);
+#pragma unroll
+          for (int cc = 0; cc < D / 32; ++cc) {
+            const int c = cq * (D / 32) + cc;
+            const uint4 u = row_live[r] ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);
+            float f[8];
+            Elem<__nv_bfloat16>::unpack(u, f);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) s_c[r] = fmaf(f[e], k_hat[c * 8 + e], s_c[r]);
+          }
+          s_c[r] += __shfl_xor_sync(0xffffffffu, s_c[r], 1);
+          s_c[r] += __shfl_xor_sync(0xffffffffu, s_c[r], 2);
+        }
+      }
+
       // Online softmax against a reference maximum m_ref that is allowed to lag: weights are 2^(s - m_ref), at
       // most 2^kLag, and the accumulator in tensor memory is rescaled only when a row's maximum has outrun the
       // reference by more than kLag (rare after the first blocks).  The compensation token (Eq. 4, Eq. 5: weight
-      // N_d exp(s_c), value v_hat) is carried as a scalar weight w_seed and added at the end.
+      // N_d exp(s_c), value v_hat) is carried as a scalar weight w_seed and added at the end.  A thread keeps the
+      // sum of its own columns' weights; the four partial sums of a row meet at the end.
       constexpr float kLag = 8.f;
-      float m_ref = -CUDART_INF_F, l_run = 0.f, w_seed = 0.f;
-      if (seed) {
-        m_ref = s_c * scale_log2 + log2f((float)st.n_drop);
-        l_run = 1.f;
-        w_seed = 1.f;
+      float m_ref[2], l_part[2], w_seed[2];
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        m_ref[r] = seed ? s_c[r] * scale_log2 + log2f((float)st.n_drop) : -CUDART_INF_F;
+        l_part[r] = (seed && cq == 0) ? 1.f : 0.f;
+        w_seed[r] = seed ? 1.f : 0.f;
       }
       const bool in_order = st.window < 0 || st.n_drop == 0;               // slot = position
       const int q_pos_min = total - jb.n_tok + w.q_tile * tok_per_tile;    // the tile's earliest query
@@ -411,17 +477,19 @@ __global__ void __launch_bounds__(kRoundThreads, 1)
         // Does the block need masking?  Slots beyond the head's length, or tokens of the round (the newest n_tok: the
         // last slots of a head whose slots are in position order, a cyclic run of the ring otherwise) that come
         // after some query of the tile.  Every thread finds the same answer from the head's state, so the common
-        // case costs no exchange; in a block that does need it each thread works out the position of its own
-        // column and the four warps trade them through shared memory.
+        // case costs no exchange; in a block that does need it the position of each column is worked out by one
+        // thread and traded through shared memory.
         const int slot1 = slot0 + kBlk;
         bool masked = slot1 > st.len;
         if (in_order) masked |= slot1 - 1 > q_pos_min;
         else masked |= (slot0 < new_hi && new_lo < slot1) || (slot0 < new_hi2 && new_lo2 < slot1);
         const int32_t* col_pos = ctl->col_pos[n_sync & 1];
         if (masked) {
-          const int s = slot0 + row;   // column `row` of the block
           // (double-buffered: a thread may still be reading the positions of the masked block before)
-          ctl->col_pos[n_sync & 1][row] = s < st.len ? slot_pos(s, dv.n_sink, st.ring_head, st.window, st.n_drop, total) : 0x7fffffff;
+          if (tid < kBlk) {
+            const int s = slot0 + tid;   // column tid of the block
+            ctl->col_pos[n_sync & 1][tid] = s < st.len ? slot_pos(s, dv.n_sink, st.ring_head, st.window, st.n_drop, total) : 0x7fffffff;
+          }
           mbar_arrive(&ctl->blk_sync);
           ok = mbar_wait(&ctl->blk_sync, n_sync & 1, abort_flag);
           if (!ok) break;
@@ -431,91 +499,129 @@ __global__ void __launch_bounds__(kRoundThreads, 1)
         if (!ok) break;
         tc_fence_after();
 
-        // ---- this row's 128 scores, in registers
-        uint32_t v[kBlk];
-#pragma unroll
-        for (int c = 0; c < kBlk / 32; ++c) tmem_ld32_issue(lane_addr + (uint32_t)(c * 32), v + c * 32);
+        // ---- the thread's 2 x 64 scores, in registers: v[4j + 2r + e] is row r, column 8j + 2cq + e
+        uint32_t v[64];
+        tmem_ld_frag64(lane_addr, v);
+        tmem_ld_frag64(lane_addr + 64u, v + 32);
         tmem_ld_wait_all();
 #pragma unroll
-        for (int e = 0; e < kBlk; ++e) asm volatile("" : "+r"(v[e]));
+        for (int e = 0; e < 64; ++e) asm volatile("" : "+r"(v[e]));
         tc_fence_before();
         mbar_arrive(&ctl->s_empty);
         if (masked) {
 #pragma unroll
-          for (int e = 0; e < kBlk; ++e)
-            if (col_pos[e] > q_pos) v[e] = 0xff800000u;   // -inf
-        }
-        float mx4[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
+          for (int j = 0; j < kBlk / 8; ++j)
 #pragma unroll
-        for (int e = 0; e < kBlk; ++e) mx4[e & 3] = fmaxf(mx4[e & 3], __uint_as_float(v[e]));
-        // (the scale is positive: the max of the scaled scores is the scaled max)
-        const float m_blk = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * scale_log2;
+            for (int e = 0; e < 2; ++e) {
+              const int cp = col_pos[8 * j + 2 * cq + e];
+              if (cp > q_pos[0]) v[4 * j + e] = 0xff800000u;   // -inf
+              if (cp > q_pos[1]) v[4 * j + 2 + e] = 0xff800000u;
+            }
+        }
+        // ---- the rows' maxima over the block: own columns, then the four threads of a row
+        float m_blk[2];
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+          float mx0 = -CUDART_INF_F, mx1 = -CUDART_INF_F;
+#pragma unroll
+          for (int j = 0; j < kBlk / 8; j += 2) {
+            mx0 = max3(mx0, __uint_as_float(v[4 * j + 2 * r]), __uint_as_float(v[4 * j + 2 * r + 1]));
+            mx1 = max3(mx1, __uint_as_float(v[4 * j + 4 + 2 * r]), __uint_as_float(v[4 * j + 4 + 2 * r + 1]));
+          }
+          float mx = fmaxf(mx0, mx1);
+          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+          m_blk[r] = mx * scale_log2;   // (the scale is positive: the max of the scaled scores is the scaled max)
+        }
 
         // ---- the product that read this buffer of P (two blocks ago) must have run before it is overwritten
         if (g >= 2) ok = mbar_wait(&ctl->p_empty[pb], ((g >> 1) - 1) & 1, abort_flag);
         if (!ok) break;
-        // ---- move the reference maximum?  Tensor-memory loads and stores are warp-wide, so the warp decides as one.
-        const bool want = m_blk > m_ref + kLag || (m_ref == -CUDART_INF_F && m_blk > -CUDART_INF_F);
+        // ---- move the reference maxima?  Tensor-memory loads and stores are warp-wide, so the warp decides as one.
+        bool want = false;
+#pragma unroll
+        for (int r = 0; r < 2; ++r) want |= m_blk[r] > m_ref[r] + kLag || (m_ref[r] == -CUDART_INF_F && m_blk[r] > -CUDART_INF_F);
         if (__any_sync(0xffffffffu, want)) {
-          const float m_to = fmaxf(m_ref, m_blk);
-          const float f = (m_to == -CUDART_INF_F || m_ref == -CUDART_INF_F) ? 0.f : fast_exp2(m_ref - m_to);   // 1 for a row that stays
+          float f[2];
+#pragma unroll
+          for (int r = 0; r < 2; ++r) {
+            const float m_to = fmaxf(m_ref[r], m_blk[r]);
+            f[r] = (m_to == -CUDART_INF_F || m_ref[r] == -CUDART_INF_F) ? 0.f : fast_exp2(m_ref[r] - m_to);   // 1 for a row that stays
+            l_part[r] *= f[r];
+            w_seed[r] *= f[r];
+            m_ref[r] = m_to;
+          }
           if (i >= 1) {   // the accumulator holds products of this item: rescale this warp's rows, once the last has run
             ok = mbar_wait(&ctl->p_empty[pb ^ 1], ((g - 1) >> 1) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
 #pragma unroll
-            for (int c = 0; c < D / 32; ++c) {
+            for (int c = 0; c < D / 64; ++c) {
               uint32_t o[32];
-              tmem_ld32_issue(lane_addr + kOCol + (uint32_t)(c * 32), o);
+              tmem_ld_frag64(lane_addr + kOCol + (uint32_t)(c * 64), o);
               tmem_ld_wait_all();
 #pragma unroll
               for (int e = 0; e < 32; ++e) {
                 asm volatile("" : "+r"(o[e]));
-                o[e] = __float_as_uint(__uint_as_float(o[e]) * f);
+                o[e] = __float_as_uint(__uint_as_float(o[e]) * f[(e >> 1) & 1]);
               }
-              tmem_st32(lane_addr + kOCol + (uint32_t)(c * 32), o);
+              tmem_st_frag64(lane_addr + kOCol + (uint32_t)(c * 64), o);
             }
             tmem_st_wait_all();
             tc_fence_before();
           }
-          l_run *= f;
-          w_seed *= f;
-          m_ref = m_to;
         }
-        const float m_use = (m_ref == -CUDART_INF_F) ? 0.f : m_ref;
+        float m_use[2];
+#pragma unroll
+        for (int r = 0; r < 2; ++r) m_use[r] = (m_ref[r] == -CUDART_INF_F) ? 0.f : m_ref[r];
 
-        // ---- weights, their sum, and P into its tensor-memory buffer: column c of the head half holds the bf16 pair of
+        // ---- weights, their sums, and P into its tensor-memory buffer: column c of the head half holds the bf16 pair of
         // tokens 2c and 2c + 1 (the operand-A layout of the matrix unit), the remainder half the same
-        float psum4[4] = {0.f, 0.f, 0.f, 0.f};
+        // A weight goes into the product as a bf16 head (its upper 16 bits) plus a bf16 remainder - two products - so
+        // that it keeps fp32-like accuracy: a single bf16 would put 2^-9 of a large weight times its V row into the result.
+        const uint64_t scale2 = f2_pack(scale_log2, scale_log2);
+        uint64_t neg_m2[2], psum2[2][2];
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+          neg_m2[r] = f2_pack(-m_use[r], -m_use[r]);
+          psum2[r][0] = psum2[r][1] = f2_pack(0.f, 0.f);
+        }
         const uint32_t p_addr = lane_addr + kPCol + (uint32_t)pb * kPBuf;
 #pragma unroll
-        for (int c = 0; c < kBlk / 32; ++c) {   // 32 tokens = 16 columns of pairs
+        for (int hh = 0; hh < 2; ++hh) {   // 64 tokens = 32 columns of pairs at a time
           uint32_t hi[16], lo[16];
 #pragma unroll
-          for (int e2 = 0; e2 < 16; ++e2) {
-            const int e = c * 32 + e2 * 2;
-            const float t0 = fmaf(__uint_as_float(v[e]), scale_log2, -m_use), t1 = fmaf(__uint_as_float(v[e + 1]), scale_log2, -m_use);
-            // every fourth pair of exponentials on the FMA pipe instead of the transcendental unit
-            const float w0 = (e2 & 3) == 3 ? exp2_poly(t0) : fast_exp2(t0);
-            const float w1 = (e2 & 3) == 3 ? exp2_poly(t1) : fast_exp2(t1);
-            psum4[e2 & 3] += w0 + w1;
-            // the weight goes into the product as a bf16 head plus a bf16 remainder (two products), so that it
-            // keeps fp32-like accuracy: a single bf16 would put 2^-9 of a large weight times its V row into the result
-            const __nv_bfloat162 h2 = __floats2bfloat162_rn(w0, w1);
-            hi[e2] = *(const uint32_t*)&h2;
-            lo[e2] = pack2_bf16(w0 - __low2float(h2), w1 - __high2float(h2));
+          for (int jj = 0; jj < 8; ++jj) {
+            const int j = hh * 8 + jj;
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+              float t0, t1, l0, l1;
+              f2_unpack(f2_fma(f2_pack(__uint_as_float(v[4 * j + 2 * r]), __uint_as_float(v[4 * j + 2 * r + 1])), scale2, neg_m2[r]), t0, t1);
+              const float w0 = fast_exp2(t0), w1 = fast_exp2(t1);
+              const uint64_t w2 = f2_pack(w0, w1);
+              psum2[r][jj & 1] = f2_add(psum2[r][jj & 1], w2);
+              const uint32_t b0 = __float_as_uint(w0), b1 = __float_as_uint(w1);
+              hi[2 * jj + r] = __byte_perm(b0, b1, 0x7632);
+              f2_unpack(f2_sub(w2, f2_pack(__uint_as_float(b0 & 0xffff0000u), __uint_as_float(b1 & 0xffff0000u))), l0, l1);
+              lo[2 * jj + r] = pack2_bf16(l0, l1);
+            }
           }
-          tmem_st16(p_addr + (uint32_t)(c * 16), hi);
-          tmem_st16(p_addr + kPLo + (uint32_t)(c * 16), lo);
+          tmem_st_frag32(p_addr + (uint32_t)(hh * 32), hi);
+          tmem_st_frag32(p_addr + kPLo + (uint32_t)(hh * 32), lo);
         }
-        l_run += (psum4[0] + psum4[1]) + (psum4[2] + psum4[3]);
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+          float a0, a1;
+          f2_unpack(f2_add(psum2[r][0], psum2[r][1]), a0, a1);
+          l_part[r] += a0 + a1;
+        }
         // V rows of slots beyond the head's length may hold anything (a zero weight times a NaN is a NaN): zero them
         if (slot0 + kBlk > st.len) {
           ok = mbar_wait(&ctl->v_full[g % kKvStages], (g / kKvStages) & 1, abort_flag);   // the rows must have landed before they are overwritten
           if (!ok) break;
           const int first_bad = max(st.len - slot0, 0);
           uint8_t* vt = v_tile + (g % kKvStages) * KV_TILE;
-          for (int idx = first_bad * 8 + row; idx < kBlk * 8; idx += kSoftmaxThreads) {   // 16-byte chunks of the bad rows
+          for (int idx = first_bad * 8 + tid; idx < kBlk * 8; idx += kSoftmaxThreads) {   // 16-byte chunks of the bad rows
 #pragma unroll
             for (int h = 0; h < HALVES; ++h) *(uint4*)(vt + h * kHalfBytes + idx * 16) = make_uint4(0u, 0u, 0u, 0u);
           }
@@ -526,7 +632,7 @@ __global__ void __launch_bounds__(kRoundThreads, 1)
         mbar_arrive(&ctl->p_full[pb]);
       }
       if (!ok) break;
-      // ---- the row's result: accumulator out of tensor memory once the last product is done, plus the
+      // ---- the rows' results: accumulator out of tensor memory once the last product is done, plus the
       // compensation token's share; the output when the unit is in one part, else a partial record
       if (nb > 0) {
         ok = mbar_wait(&ctl->p_empty[(gb + nb - 1) & 1], ((gb + nb - 1) >> 1) & 1, abort_flag);
@@ -535,31 +641,43 @@ __global__ void __launch_bounds__(kRoundThreads, 1)
       }
       gb += nb;
       const bool direct = w.n_parts == 1;
-      const float inv = direct ? (l_run > 0.f ? 1.f / l_run : 0.f) : 1.f;
-      const size_t r = (size_t)w.rec_base + (size_t)w.part_idx * kRows + row;
-      float* dst = direct ? out + row_off : dv.rec_o + r * D;
+      float inv[2];
+      float* dst[2];
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        float l = l_part[r];
+        l += __shfl_xor_sync(0xffffffffu, l, 1);
+        l += __shfl_xor_sync(0xffffffffu, l, 2);
+        l_part[r] = l;
+        inv[r] = direct ? (l > 0.f ? 1.f / l : 0.f) : 1.f;
+        const size_t rr = (size_t)w.rec_base + (size_t)w.part_idx * kRows + (size_t)(row0 + 8 * r);
+        dst[r] = direct ? out + row_off[r] : dv.rec_o + rr * D;
+        if (!direct && cq == 0) dv.rec_ml[rr] = make_float2(m_ref[r], l);
+      }
       const float* v_hat = dv.comp_mean + hs * 2 * D + D;
 #pragma unroll
-      for (int c = 0; c < D / 32; ++c) {
+      for (int c = 0; c < D / 64; ++c) {
         uint32_t o[32];
         if (nb > 0) {
-          tmem_ld32_issue(lane_addr + kOCol + (uint32_t)(c * 32), o);
+          tmem_ld_frag64(lane_addr + kOCol + (uint32_t)(c * 64), o);
           tmem_ld_wait_all();
         }
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          asm volatile("" : "+r"(o[e]));
-          float x = nb > 0 ? __uint_as_float(o[e]) : 0.f;
-          if (seed) x = fmaf(w_seed, v_hat[c * 32 + e], x);
-          o[e] = __float_as_uint(x * inv);
-        }
-        if (direct ? row_live : true) {
+        for (int jj = 0; jj < 8; ++jj) {
+          const int col = c * 64 + 8 * jj + 2 * cq;
 #pragma unroll
-          for (int e = 0; e < 32; e += 4)
-            *(float4*)(dst + c * 32 + e) = make_float4(__uint_as_float(o[e]), __uint_as_float(o[e + 1]), __uint_as_float(o[e + 2]), __uint_as_float(o[e + 3]));
+          for (int r = 0; r < 2; ++r) {
+            asm volatile("" : "+r"(o[4 * jj + 2 * r]), "+r"(o[4 * jj + 2 * r + 1]));
+            float x0 = nb > 0 ? __uint_as_float(o[4 * jj + 2 * r]) : 0.f;
+            float x1 = nb > 0 ? __uint_as_float(o[4 * jj + 2 * r + 1]) : 0.f;
+            if (seed) {
+              x0 = fmaf(w_seed[r], v_hat[col], x0);
+              x1 = fmaf(w_seed[r], v_hat[col + 1], x1);
+            }
+            if (direct ? row_live[r] : true) *(float2*)(dst[r] + col) = make_float2(x0 * inv[r], x1 * inv[r]);
+          }
         }
       }
-      if (!direct) dv.rec_ml[r] = make_float2(m_ref, l_run);
       tc_fence_before();
       mbar_arrive(&ctl->o_read);
     }
