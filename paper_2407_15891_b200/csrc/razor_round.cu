@@ -1,25 +1,33 @@
 // Attention of a long round of new tokens (a follow-up prompt, a prefill chunk) over the compressed cache:
 // the rows of a KV head's queries (query tokens x query heads of the group) are tiled 128 at a time, so
 // the cache is streamed once per 128 query rows and the work is a real dense contraction.  It runs on the
-// 5th-generation tensor cores: S = Q K^T and O = P V as tcgen05.mma with the operands in shared memory
-// and the accumulators in tensor memory.  Same arithmetic as the decode kernel otherwise: causal mask inside
-// the round (Section 3.1), compensation token with its count as the initial softmax state of a head's
-// first part (Eq. 5), split over the tokens with partial records merged afterwards.
+// 5th-generation tensor cores: S = Q K^T with both operands in shared memory, O = P V with P read out of
+// tensor memory and V out of shared memory, accumulators in tensor memory.  Same arithmetic as the decode kernel
+// otherwise: causal mask inside the round (Section 3.1), compensation token with its count as the initial
+// softmax state of a head's first part (Eq. 5), split over the tokens with partial records merged afterwards.
 //
 // A work item is (KV head, tile of 128 query rows, a run of 128-token blocks of the head's slot stream).
-// Persistent CTAs pull items from a queue (longest first).  Four roles in a CTA of six warps:
+// Persistent CTAs pull items from a queue (longest first).  Roles in a CTA of ten warps:
 //   * warp 0, one thread: TMA copies of K and V, one 16-token page at a time.  A page of the pool is
 //     [16 K rows][16 V rows] with the 16-byte chunks of a row XOR-swizzled by the token index; a tensor map
 //     over the pool with a box of (64 elements, 16 tokens) lands each half row at a 128-byte pitch, which is
 //     exactly the 128-byte-swizzled operand layout of the matrix unit: K as a K-major operand of S = Q K^T,
-//     V as an MN-major operand of O = P V.  Two stages of 128 tokens;
+//     V as an MN-major operand of O = P V.  Three stages of 128 tokens each for K and for V;
 //   * warp 1, one thread: issues the matrix instructions and commits them onto the barriers;
-//   * warps 2-5: a thread per query row.  It reads its row of S from tensor memory, scales, masks, keeps a
-//     reference max and the sum, and writes P (a bf16 head plus a bf16 remainder) into shared memory in operand
-//     layout.  O accumulates in tensor memory over the item's blocks; the reference max may lag the true one by a
-//     factor of 2^8, and only when a row outruns it is the accumulator rescaled in place.
-// (Tried and dropped: two threads per query row, 64 columns each, with the block maxima exchanged through shared
-// memory - no faster: the softmax warps are bound by their instruction count per score, not by their number.)
+//   * warps 2-9: softmax.  A warp owns 16 query rows (tensor-memory lanes) in the fragment layout of the 16-lane
+//     loads: four threads per row, each with every fourth pair of columns, so a row's maximum is two shuffles and
+//     two warps share a scheduler.  A thread reads its scores of S from tensor memory, masks, keeps a reference
+//     max and its share of the sum, and writes P - a bf16 head plus a bf16 remainder per weight - into one of two
+//     buffers in tensor memory, in the layout the matrix unit reads operand A in.  Scale, subtraction, sums and
+//     remainders work on two scores per instruction (f32x2).  O accumulates in tensor memory over the item's
+//     blocks; the reference max may lag the true one by a factor of 2^8, and only when a row outruns it is the
+//     accumulator rescaled in place.
+// Tensor memory (512 columns): S in [0, 128), O in [128, 256), P in [256, 384) and [384, 512).
+// (Tried and dropped: P through shared memory - the matrix unit's own operand reads, the TMA writes and the
+// softmax stores then share the shared-memory port; a thread per query row - one warp per scheduler leaves the
+// pipes idle in turn; exponentials partly as a polynomial on the FMA pipe - it costs more issue slots than the
+// transcendental unit saves here; the load of the next block's scores issued ahead of the wait for this block's
+// stores - no faster.)
 // Every wait is bounded in time; a wait that runs out sets the CTA's abort flag and a bit of the device status
 // word, copies and instructions in flight are waited for, tensor memory is released.
 #include <math_constants.h>
