@@ -597,8 +597,7 @@ def main():
     def combine_launched(l):
         """1 when the layer's schedule has a head in more parts than the streaming kernel folds itself."""
         if l not in combine_cache:
-            items = rz.razor_schedule_query(cache.handle, l)
-            combine_cache[l] = int((items[:, 3] > max(1, 16 // w.group)).any())
+            combine_cache[l] = int(len(rz.razor_schedule_combine_heads(cache.handle, l)) > 0)
         return combine_cache[l]
 
     def sync_all():

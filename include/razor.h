@@ -237,6 +237,12 @@ RAZOR_API int razor_cache_stats(const razor_cache_t* cache, int32_t layer, size_
  *                         per head), n_ctas >= 1 (the SM count), 0 <= static_percent <= 100,
  *                         tail_items_per_cta >= 1, min_chunk_pages >= 1 (smallest span / tail item).
  *   razor_schedule_query  the plan the next razor_decode_attention of `layer` would use.
+ *   razor_schedule_combine_heads  which heads of that plan are left to the combine kernel (none: the decode
+ *                         step is one launch).  A head cut into several parts leaves one partial softmax
+ *                         record per part (Eq. 5 regrouped).  The streaming kernel folds the records of a head
+ *                         in few parts itself - the part written last does it; the others are folded by a
+ *                         small kernel launched behind it.  heads: host int32[max_heads] receiving their
+ *                         indices b*Hkv + kv_head, may be NULL; n_heads receives the count.
  * items: host int32[max_items][5] = {head index b*Hkv + kv_head, first_page, end_page (-1: to the
  * end of the stream), parts_of_this_head, job}, in job order, may be NULL; n_items receives the
  * count, n_spans (may be NULL) how many of the jobs are spans.  A page is 16 tokens.
@@ -247,6 +253,8 @@ RAZOR_API int razor_schedule_plan(const int32_t* tokens, int32_t n_heads, int32_
                         int32_t* n_items, int32_t* n_spans);
 RAZOR_API int razor_schedule_query(razor_cache_t* cache, int32_t layer, int32_t* items, int32_t max_items,
                          int32_t* n_items);
+RAZOR_API int razor_schedule_combine_heads(razor_cache_t* cache, int32_t layer, int32_t* heads, int32_t max_heads,
+                                 int32_t* n_heads);
 
 /*
  * Decode tuning knobs; the defaults suit long-context caches on a B200.  A change takes effect at the

@@ -27,7 +27,7 @@ STATUS = {
 SYMBOLS = [
     "razor_query_bytes", "razor_cache_create", "razor_compress", "razor_compress_seq", "razor_append",
     "razor_decode_attention", "razor_decode_step", "razor_append_many", "razor_append_plan", "razor_decode_attention_multi", "razor_cache_export", "razor_cache_stats", "razor_schedule_plan",
-    "razor_schedule_query", "razor_cache_set_option", "razor_cache_device_status", "razor_cache_wait_selftest", "razor_cache_set_alibi", "razor_cache_set_head_windows",
+    "razor_schedule_query", "razor_schedule_combine_heads", "razor_cache_set_option", "razor_cache_device_status", "razor_cache_wait_selftest", "razor_cache_set_alibi", "razor_cache_set_head_windows",
     "razor_compensation_mean_static", "razor_head_scores_scratch_bytes", "razor_head_scores",
     "razor_select_retrieval_heads", "razor_cache_reset", "razor_cache_destroy", "razor_status_string",
     "razor_last_cuda_error", "razor_version",
@@ -83,6 +83,7 @@ def load() -> C.CDLL:
     lib.razor_cache_set_option.argtypes = [vp, i32, i32]
     lib.razor_cache_device_status.argtypes = [vp, C.POINTER(i32), vp]
     lib.razor_schedule_query.argtypes = [vp, i32, vp, i32, C.POINTER(i32)]
+    lib.razor_schedule_combine_heads.argtypes = [vp, i32, vp, i32, C.POINTER(i32)]
     lib.razor_compensation_mean_static.argtypes = [vp, vp, i64, i64, i32, i32, i32, i32, i32, i32, vp, vp,
                                                    C.POINTER(i32), vp]
     lib.razor_cache_wait_selftest.argtypes = [vp, i64, vp]
@@ -269,6 +270,16 @@ def razor_schedule_query(cache: int, layer: int) -> np.ndarray:
     items = np.zeros((n.value, 5), dtype=np.int32)
     _check(lib.razor_schedule_query(cache, layer, items.ctypes.data, n.value, C.byref(n)), "razor_schedule_query")
     return items
+
+
+def razor_schedule_combine_heads(cache: int, layer: int) -> np.ndarray:
+    """Indices (b * Hkv + kv head) of the heads whose partial records the combine kernel folds."""
+    n = C.c_int32(0)
+    lib = load()
+    _check(lib.razor_schedule_combine_heads(cache, layer, None, 0, C.byref(n)), "razor_schedule_combine_heads")
+    heads = np.zeros(n.value, dtype=np.int32)
+    _check(lib.razor_schedule_combine_heads(cache, layer, heads.ctypes.data, n.value, C.byref(n)), "razor_schedule_combine_heads")
+    return heads
 
 
 def razor_cache_set_alibi(cache: int, slopes, stream=None) -> None:

@@ -1096,4 +1096,18 @@ int razor_schedule_query(razor_cache_t* c, int32_t layer, int32_t* items, int32_
   return emit_items(L.items, L.n_items, L.jobs, L.n_jobs, items, max_items, n_items);
 }
 
+int razor_schedule_combine_heads(razor_cache_t* c, int32_t layer, int32_t* heads, int32_t max_heads, int32_t* n_heads) {
+  if (!c || !n_heads) return RAZOR_E_NULL_PTR;
+  int rc = layer_ready(c, layer);
+  if (rc) return rc;
+  rc = ensure_schedule(c, layer, nullptr, false, c->cfg.n_q_heads / c->cfg.n_kv_heads);
+  if (rc) return rc;
+  const LayerHost& L = c->layers[layer];
+  *n_heads = L.n_multi;
+  if (!heads) return RAZOR_OK;
+  if (max_heads < L.n_multi) return RAZOR_E_INVALID_ARG;
+  for (int i = 0; i < L.n_multi; ++i) heads[i] = L.multi[i].head;
+  return RAZOR_OK;
+}
+
 }  // extern "C"

@@ -153,6 +153,22 @@ def test_decode_kernel_variants(group, options, D, fused):
     run_parity(w, steps=3, shuffle=7, options=options, check_layout_every=2, fused=fused)
 
 
+def test_schedule_reports_which_heads_are_left_to_the_combine_kernel():
+    """razor_schedule_combine_heads lists exactly the heads cut into more parts than the streaming kernel folds
+    itself (16 record rows: 16 // group parts), and none when every head is in few parts."""
+    for group, ctx in ((4, [9000, 37, 700]), (1, [700, 40, 300])):
+        w = synth.Workload("combine_list", 3, 1, 2 * group, 2, 128, "bf16", ctx, [300, 300, 100], 4, 1, 1, 99 + group)
+        cache = make_cache(w)
+        K, V = synth.make_dense_kv(w, 0, DEV)
+        cache.compress(0, K, V, w.ctx_len, w.retrieval(0), w.window)
+        items = rz.razor_schedule_query(cache.handle, 0)
+        want = sorted({int(h) for h, _, _, parts, _ in items.tolist() if parts > 16 // group})
+        got = sorted(rz.razor_schedule_combine_heads(cache.handle, 0).tolist())
+        assert got == want
+        assert (len(got) > 0) == (group == 4)
+        cache.close()
+
+
 @pytest.mark.parametrize("fused", [False, True])
 def test_append_many_tokens_crosses_pages_evicts_and_rebuilds_schedule(fused):
     w = synth.Workload("long_append", 2, 1, 4, 4, 128, "bf16", [700, 90], [64, 200], 4, 1, 300, 4242)
