@@ -77,22 +77,9 @@ constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t accumulate) {
   umma_bf16_desc(tmem_d, desc_a, desc_b, kInstrDesc, accumulate);
 }
-// 2^t for t <= 0 on the FMA and integer pipes, relative error below 5e-5: t = n + f with n the nearest
-// integer (read off the low mantissa bits of t + 1.5 * 2^23) and |f| <= 1/2, 2^f as a degree-4 polynomial,
-// n added onto the exponent field.  The transcendental unit is the busiest pipe of this kernel (one ex2 per
-// score), so every kPolyEvery-th exponential takes this route instead.
-constexpr int kPolyEvery = 4;
-__device__ __forceinline__ float exp2_fma(float t) {
-  t = fmaxf(t, -125.f);                       // keeps the result a normal number; 2^-125 stands for zero
-  const float r = t + 12582912.f;
-  const float f = t - (r - 12582912.f);
-  float p = 0.0096181291f;
-  p = fmaf(p, f, 0.0555041087f);
-  p = fmaf(p, f, 0.2402265070f);
-  p = fmaf(p, f, 0.6931471806f);
-  p = fmaf(p, f, 1.0f);
-  return __int_as_float(__float_as_int(p) + (__float_as_int(r) << 23));
-}
+// The transcendental unit is the busiest pipe of this kernel (one ex2 per score), so of every kPolyEvery pairs of
+// exponentials one pair is computed as a polynomial on the FMA and integer pipes instead (f2_exp2_poly).
+constexpr int kPolyEvery = 3;
 
 // Completes the loads issued so far.  The registers pass through the statement so that no use of them
 // can be scheduled ahead of it.
@@ -178,23 +165,42 @@ __global__ void __launch_bounds__(kScoreThreads, 2)
       tmem_ld_wait(v);
       tc_fence_before();
       mbar_arrive(&ctl->t_empty[b]);   // the buffer is in registers: hand it back
-      float mx[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
       if (kt == tile) {   // causality: key q0 + column against query q0 + row
 #pragma unroll
         for (int j = 0; j < 64; ++j)
           if (col0 + j > row) v[j] = 0xff800000u;   // -inf
       }
+      float mx[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};
 #pragma unroll
-      for (int j = 0; j < 64; ++j) mx[j & 3] = fmaxf(mx[j & 3], __uint_as_float(v[j]));
+      for (int j = 0; j < 64; j += 2) mx[(j >> 1) & 3] = max3(mx[(j >> 1) & 3], __uint_as_float(v[j]), __uint_as_float(v[j + 1]));
       // the scale is positive, so the max of the scaled logits is the scaled max
       const float tile_max = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * scale_log2;
       const float mn = fmaxf(m_run, tile_max);
       const float mu = (mn == -CUDART_INF_F) ? 0.f : mn;   // a fully masked half row so far
-      float sum[4] = {0.f, 0.f, 0.f, 0.f};
+      // two scores per instruction: scale and subtract, exponentials, sums
+      const uint64_t scale2 = f2_pack(scale_log2, scale_log2), neg_mu2 = f2_pack(-mu, -mu);
+      uint64_t sum2[4];
 #pragma unroll
-      for (int j = 0; j < 64; ++j) {
-        const float t = fmaf(__uint_as_float(v[j]), scale_log2, -mu);
-        sum[j & 3] += (j % kPolyEvery == kPolyEvery - 1) ? exp2_fma(t) : fast_exp2(t);
+      for (int k = 0; k < 4; ++k) sum2[k] = f2_pack(0.f, 0.f);
+#pragma unroll
+      for (int j = 0; j < 64; j += 2) {
+        const uint64_t t2 = f2_fma(f2_pack(__uint_as_float(v[j]), __uint_as_float(v[j + 1])), scale2, neg_mu2);
+        uint64_t w2;
+        if ((j >> 1) % kPolyEvery == kPolyEvery - 1) {
+          w2 = f2_exp2_poly(t2);
+        } else {
+          float t0, t1;
+          f2_unpack(t2, t0, t1);
+          w2 = f2_pack(fast_exp2(t0), fast_exp2(t1));
+        }
+        sum2[(j >> 1) & 3] = f2_add(sum2[(j >> 1) & 3], w2);
+      }
+      float sum[4];
+      {
+        float a0, a1, b0, b1;
+        f2_unpack(f2_add(sum2[0], sum2[1]), a0, a1);
+        f2_unpack(f2_add(sum2[2], sum2[3]), b0, b1);
+        sum[0] = a0; sum[1] = a1; sum[2] = b0; sum[3] = b1;
       }
       l_run = l_run * fast_exp2(m_run - mu) + ((sum[0] + sum[1]) + (sum[2] + sum[3]));
       m_run = mn;

@@ -76,6 +76,56 @@ __device__ __forceinline__ void tmem_ld32_issue(uint32_t taddr, uint32_t* v) {
 // Completes the tensor-memory loads issued so far.
 __device__ __forceinline__ void tmem_ld_wait_all() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// Two fp32 values in a 64-bit register pair, and the arithmetic that works on both at once (one instruction slot
+// for two scores); the larger of three values in one instruction.
+__device__ __forceinline__ uint64_t f2_pack(float a, float b) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
+}
+__device__ __forceinline__ void f2_unpack(uint64_t v, float& a, float& b) { asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v)); }
+__device__ __forceinline__ uint64_t f2_fma(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+__device__ __forceinline__ uint64_t f2_add(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ uint64_t f2_sub(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+
+// 2^t of two values t <= 0 at once on the FMA and integer pipes, relative error below 5e-5: t = n + f with n the
+// nearest integer (read off the low mantissa bits of t + 1.5 * 2^23) and |f| <= 1/2, 2^f as a degree-4 polynomial,
+// n added onto the exponent field.  Arguments below -125 count as -125 (2^-125 stands for zero).
+__device__ __forceinline__ uint64_t f2_exp2_poly(uint64_t t2) {
+  float t0, t1;
+  f2_unpack(t2, t0, t1);
+  t2 = f2_pack(fmaxf(t0, -125.f), fmaxf(t1, -125.f));
+  const uint64_t magic = f2_pack(12582912.f, 12582912.f);
+  const uint64_t r2 = f2_add(t2, magic);
+  const uint64_t f = f2_sub(t2, f2_sub(r2, magic));
+  uint64_t p = f2_fma(f2_pack(0.0096181291f, 0.0096181291f), f, f2_pack(0.0555041087f, 0.0555041087f));
+  p = f2_fma(p, f, f2_pack(0.2402265070f, 0.2402265070f));
+  p = f2_fma(p, f, f2_pack(0.6931471806f, 0.6931471806f));
+  p = f2_fma(p, f, f2_pack(1.0f, 1.0f));
+  float p0, p1, r0, r1;
+  f2_unpack(p, p0, p1);
+  f2_unpack(r2, r0, r1);
+  return f2_pack(__int_as_float(__float_as_int(p0) + (__float_as_int(r0) << 23)),
+                 __int_as_float(__float_as_int(p1) + (__float_as_int(r1) << 23)));
+}
+
 // cuTensorMapEncodeTiled, looked up through the runtime (the library does not link against the driver).
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
