@@ -6,28 +6,27 @@
 // otherwise: causal mask inside the round (Section 3.1), compensation token with its count as the initial
 // softmax state of a head's first part (Eq. 5), split over the tokens with partial records merged afterwards.
 //
-// A work item is (KV head, tile of 128 query rows, a run of 128-token blocks of the head's slot stream).
-// Persistent CTAs pull items from a queue (longest first).  Roles in a CTA of ten warps:
-//   * warp 0, one thread: TMA copies of K and V, one 16-token page at a time.  A page of the pool is
-//     [16 K rows][16 V rows] with the 16-byte chunks of a row XOR-swizzled by the token index; a tensor map
-//     over the pool with a box of (64 elements, 16 tokens) lands each half row at a 128-byte pitch, which is
-//     exactly the 128-byte-swizzled operand layout of the matrix unit: K as a K-major operand of S = Q K^T,
-//     V as an MN-major operand of O = P V.  Three stages of 128 tokens each for K and for V;
+// A work item is (KV head, tile of 128 query rows, a run of 128-token blocks of the head's slot stream); a CTA
+// takes it in steps of 64 tokens.  Persistent CTAs pull items from a queue (longest first), TWO CTAs to an SM:
+// each has half of the tensor memory (256 columns) and less than half of the shared memory, and because the
+// two run independently, one's softmax (transcendental unit, ALU) overlaps the other's waits and matrix
+// products - inside one CTA the phases of a step follow each other.  Roles in a CTA of six warps:
+//   * warp 0: TMA copies of K and V, one 16-token page at a time.  A page of the pool is [16 K rows][16 V rows]
+//     with the 16-byte chunks of a row XOR-swizzled by the token index; a tensor map over the pool with a box of
+//     (64 elements, 16 tokens) lands each half row at a 128-byte pitch, which is exactly the 128-byte-swizzled
+//     operand layout of the matrix unit: K as a K-major operand of S = Q K^T, V as an MN-major operand of
+//     O = P V.  Two stages of 64 tokens each for K and for V;
 //   * warp 1, one thread: issues the matrix instructions and commits them onto the barriers;
-//   * warps 2-9: softmax.  A warp owns 16 query rows (tensor-memory lanes) in the fragment layout of the 16-lane
-//     loads: four threads per row, each with every fourth pair of columns, so a row's maximum is two shuffles and
-//     two warps share a scheduler.  A thread reads its scores of S from tensor memory, masks, keeps a reference
-//     max and its share of the sum, and writes P - a bf16 head plus a bf16 remainder per weight - into one of two
-//     buffers in tensor memory, in the layout the matrix unit reads operand A in.  Scale, subtraction, sums and
-//     remainders work on two scores per instruction (f32x2).  O accumulates in tensor memory over the item's
-//     blocks; the reference max may lag the true one by a factor of 2^8, and only when a row outruns it is the
-//     accumulator rescaled in place.
-// Tensor memory (512 columns): S in [0, 128), O in [128, 256), P in [256, 384) and [384, 512).
+//   * warps 2-5: softmax, a thread per query row (tensor-memory lane).  It reads its 64 scores of S, masks, keeps
+//     a reference max and the sum, and writes P - a bf16 head plus a bf16 remainder per weight - into tensor
+//     memory in the layout the matrix unit reads operand A in.  Scale, subtraction, sums and remainders work on
+//     two scores per instruction (f32x2).  O accumulates in tensor memory over the item's steps; the reference
+//     max may lag the true one by a factor of 2^8, and only when a row outruns it is the accumulator rescaled.
+// Tensor memory of a CTA (256 columns): S in [0, 64), P in [64, 128) (heads, then remainders), O in [128, 256).
 // (Tried and dropped: P through shared memory - the matrix unit's own operand reads, the TMA writes and the
-// softmax stores then share the shared-memory port; a thread per query row - one warp per scheduler leaves the
-// pipes idle in turn; exponentials partly as a polynomial on the FMA pipe - it costs more issue slots than the
-// transcendental unit saves here; the load of the next block's scores issued ahead of the wait for this block's
-// stores - no faster.)
+// softmax stores then share the shared-memory port; one CTA per SM with 128-token steps, first with a thread per
+// row, then with eight softmax warps and four threads per row - its warps move through the phases of a step
+// together; exponentials partly as a polynomial on the FMA pipe.)
 // Every wait is bounded in time; a wait that runs out sets the CTA's abort flag and a bit of the device status
 // word, copies and instructions in flight are waited for, tensor memory is released.
 #include <math_constants.h>
@@ -42,37 +41,41 @@ namespace razor {
 namespace {
 
 constexpr int kRows = kRoundTileRows;      // query rows per tile = accumulator rows = tensor-memory lanes
-constexpr int kBlk = kRoundBlockTokens;    // tokens per block = columns of S
-constexpr int kKvStages = 3;
-constexpr int kRoundThreads = 10 * 32;
-constexpr int kSoftmaxThreads = 256;
-constexpr int kHalfBytes = kRows * 128;    // one 64-element half of a 128-row operand tile
+constexpr int kBlk = kRoundBlockTokens;    // tokens per block of a work item
+constexpr int kStep = 64;                  // tokens per step = columns of S
+constexpr int kStepsPerBlock = kBlk / kStep;
+constexpr int kKvStages = 2;
+constexpr int kRoundThreads = 6 * 32;
+constexpr int kSoftmaxThreads = 128;
+constexpr int kCtasPerSm = 2;
+constexpr int kQHalfBytes = kRows * 128;   // one 64-element half of the 128-row query tile
+constexpr int kKvHalfBytes = kStep * 128;  // one 64-element half of a 64-token K or V stage
 
 struct RoundCtl {
   uint64_t q_ready;               // softmax threads -> MMA: the query tile is in shared memory
-  uint64_t k_full[kKvStages];     // TMA -> MMA: the stage holds 128 tokens of K
+  uint64_t k_full[kKvStages];     // TMA -> MMA: the stage holds 64 tokens of K
   uint64_t k_empty[kKvStages];    // MMA (commit of S = Q K^T) -> TMA
   uint64_t v_full[kKvStages];     // the same for V; a V stage is free once O += P V has run
   uint64_t v_empty[kKvStages];
-  uint64_t s_full;                // MMA (commit) -> softmax: S holds a block's scores
+  uint64_t s_full;                // MMA (commit) -> softmax: S holds a step's scores
   uint64_t s_empty;               // softmax -> MMA: S read out into registers
-  uint64_t p_full[2];             // softmax -> MMA: P of the block is in its tensor-memory buffer
-  uint64_t p_empty[2];            // MMA (commit) -> softmax: the product that read the buffer has run
+  uint64_t p_full;                // softmax -> MMA: P of the step is in tensor memory
+  uint64_t p_empty;               // MMA (commit) -> softmax: the product that read P has run
   uint64_t o_read;                // softmax -> MMA: the item's output accumulator has been read out of tensor memory
   uint64_t item_ready;            // producer -> everyone: the next item index is in `item`
   uint64_t item_taken;            // MMA warp + softmax threads -> producer: `item` has been read
-  uint64_t blk_sync;              // the softmax threads among themselves, once per masked block (a bounded wait, unlike bar.sync)
+  uint64_t blk_sync;              // the softmax threads among themselves, once per masked step (a bounded wait, unlike bar.sync)
   uint64_t drain;
   uint32_t tmem_base;
   int abort_flag;
   int item;                       // index of the current work item, -1: no more
-  int32_t col_pos[2][kBlk];       // token position of each column of a masked block (two may be in progress)
+  int32_t col_pos[2][kStep];      // token position of each column of a masked step (two may be in progress)
 };
 
 template <int D>
 constexpr size_t round_smem_bytes() {
   // 1 KB alignment slack, Q tile, K and V stages, control block
-  return 1024 + (size_t)kRows * D * 2 + (size_t)kKvStages * 2 * kBlk * D * 2 + sizeof(RoundCtl);
+  return 1024 + (size_t)kRows * D * 2 + (size_t)kKvStages * 2 * kStep * D * 2 + sizeof(RoundCtl);
 }
 
 // One page half: 16 tokens x 64 elements of K or V of pool page `pid` into shared memory (2 KB).
@@ -99,42 +102,26 @@ __device__ __forceinline__ uint32_t pack2_bf16(float lo, float hi) {
   return *(const uint32_t*)&v;
 }
 
-// Fragment-shaped accesses: a warp touches 16 lanes (taddr's lane, a multiple of 16, onwards).  Thread t of the warp
-// owns lanes t / 4 and t / 4 + 8 and, in each group of columns, the columns picked by t % 4:
-//   .16x256b (groups of 8 columns): registers 4j .. 4j + 3 of group j are (lane t/4, columns 8j + 2(t%4) and + 1),
-//                                   (lane t/4 + 8, the same two columns);
-//   .16x128b (groups of 4 columns): registers 2j, 2j + 1 of group j are (lane t/4, column 4j + t%4), (lane t/4 + 8,
-//                                   the same column).
-// So the two fp32 values a thread reads from columns 2c, 2c + 1 of S become, as a bf16 pair, its column c of P.
-#define RAZOR_R8(v, o) "r"(v[o]), "r"(v[o + 1]), "r"(v[o + 2]), "r"(v[o + 3]), "r"(v[o + 4]), "r"(v[o + 5]), "r"(v[o + 6]), "r"(v[o + 7])
-#define RAZOR_W8(v, o) "=r"(v[o]), "=r"(v[o + 1]), "=r"(v[o + 2]), "=r"(v[o + 3]), "=r"(v[o + 4]), "=r"(v[o + 5]), "=r"(v[o + 6]), "=r"(v[o + 7])
-// 64 columns (8 groups of 8) of 16 lanes into 32 registers; valid after tmem_ld_wait_all().
-__device__ __forceinline__ void tmem_ld_frag64(uint32_t taddr, uint32_t* v) {
+// 32 or 16 consecutive columns of this thread's lane into tensor memory; complete after tmem_st_wait_all().
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* v) {
   asm volatile(
-      "tcgen05.ld.sync.aligned.16x256b.x8.b32 "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
-      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-      : RAZOR_W8(v, 0), RAZOR_W8(v, 8), RAZOR_W8(v, 16), RAZOR_W8(v, 24)
-      : "r"(taddr)
-      : "memory");
-}
-// The store of the same shape; complete after tmem_st_wait_all().
-__device__ __forceinline__ void tmem_st_frag64(uint32_t taddr, const uint32_t* v) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.16x256b.x8.b32 [%0], "
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
       "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
       "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
       :
-      : "r"(taddr), RAZOR_R8(v, 0), RAZOR_R8(v, 8), RAZOR_R8(v, 16), RAZOR_R8(v, 24)
+      : "r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]),
+        "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]), "r"(v[16]), "r"(v[17]),
+        "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]), "r"(v[24]), "r"(v[25]), "r"(v[26]),
+        "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
       : "memory");
 }
-// 32 columns (8 groups of 4) of 16 lanes out of 16 registers.
-__device__ __forceinline__ void tmem_st_frag32(uint32_t taddr, const uint32_t* v) {
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* v) {
   asm volatile(
-      "tcgen05.st.sync.aligned.16x128b.x8.b32 [%0], "
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
       "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
       :
-      : "r"(taddr), RAZOR_R8(v, 0), RAZOR_R8(v, 8)
+      : "r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]),
+        "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
       : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait_all() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
@@ -148,22 +135,22 @@ __device__ __forceinline__ int slot_pos(int s, int n_sink, int ring_head, int wi
 }
 
 template <int D>
-__global__ void __launch_bounds__(kRoundThreads, 1)
+__global__ void __launch_bounds__(kRoundThreads, kCtasPerSm)
     round_kernel(DeviceView dv, const __grid_constant__ CUtensorMap map_pool, int layer, RoundJobs jb,
                  const __nv_bfloat16* __restrict__ q, float* __restrict__ out) {
   constexpr int HALVES = D / 64;
-  constexpr int Q_BYTES = kRows * D * 2, KV_TILE = kBlk * D * 2;
-  constexpr uint32_t kIdescQK = instr_desc_bf16(kRows, kBlk, false);
+  constexpr int Q_BYTES = kRows * D * 2, KV_TILE = kStep * D * 2;
+  constexpr uint32_t kIdescQK = instr_desc_bf16(kRows, kStep, false);
   constexpr uint32_t kIdescPV = instr_desc_bf16(kRows, D, true);
-  constexpr uint32_t kTmemCols = 512;
-  // tensor memory: S in columns [0, 128), the output accumulator in [128, 128 + D), two buffers of P in [256, 384) and
-  // [384, 512): a row's 128 weights as 64 columns of bf16 pairs (the heads) and 64 more (the remainders)
-  constexpr uint32_t kOCol = kBlk, kPCol = 2 * kBlk, kPBuf = kBlk, kPLo = kBlk / 2;
+  // tensor memory: S in columns [0, 64), P in [64, 128) - a row's 64 weights as 32 columns of bf16 pairs (the
+  // heads) and 32 more (the remainders) -, the output accumulator in [128, 128 + D)
+  constexpr uint32_t kTmemCols = 256;
+  constexpr uint32_t kPCol = kStep, kPLo = kStep / 2, kOCol = 2 * kStep;
 
   extern __shared__ uint8_t round_smem_raw[];
   uint8_t* base = round_smem_raw + ((1024u - (smem_u32(round_smem_raw) & 1023u)) & 1023u);
   uint8_t* q_tile = base;
-  uint8_t* k_tile = q_tile + Q_BYTES;                    // [stage][half][128 tokens][128 B]
+  uint8_t* k_tile = q_tile + Q_BYTES;                    // [stage][half][64 tokens][128 B]
   uint8_t* v_tile = k_tile + kKvStages * KV_TILE;
   RoundCtl* ctl = (RoundCtl*)(v_tile + kKvStages * KV_TILE);
 
@@ -181,10 +168,8 @@ __global__ void __launch_bounds__(kRoundThreads, 1)
     }
     mbar_init(&ctl->s_full, 1);
     mbar_init(&ctl->s_empty, kSoftmaxThreads);
-    for (int s = 0; s < 2; ++s) {
-      mbar_init(&ctl->p_full[s], kSoftmaxThreads);
-      mbar_init(&ctl->p_empty[s], 1);
-    }
+    mbar_init(&ctl->p_full, kSoftmaxThreads);
+    mbar_init(&ctl->p_empty, 1);
     mbar_init(&ctl->o_read, kSoftmaxThreads);
     mbar_init(&ctl->item_ready, 1);
     mbar_init(&ctl->item_taken, kSoftmaxThreads + 1);
@@ -193,7 +178,7 @@ __global__ void __launch_bounds__(kRoundThreads, 1)
     ctl->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 1) {   // the MMA warp owns the tensor-memory allocation
+  if (warp == 1) {   // the MMA warp owns the tensor-memory allocation (half of the SM's: the other CTA has the rest)
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)),
                  "r"(kTmemCols)
                  : "memory");
@@ -205,10 +190,15 @@ __global__ void __launch_bounds__(kRoundThreads, 1)
   const uint32_t tmem = ctl->tmem_base;
   const int G = dv.group;               // query heads per KV head
   const int tok_per_tile = kRows / G;   // query tokens of a tile
+  // Steps of a work item: its blocks in halves, without the steps that lie wholly beyond the head's length.
+  auto first_step = [](const RoundItem& w) { return w.blk_begin * kStepsPerBlock; };
+  auto end_step = [](const RoundItem& w, int len) {
+    return max(w.blk_begin * kStepsPerBlock, min(w.blk_end * kStepsPerBlock, (len + kStep - 1) / kStep));
+  };
 
   if (warp == 0) {
     // ================================================================ producer: work items and TMA copies
-    unsigned gb = 0;       // blocks issued so far by this CTA
+    unsigned gb = 0;       // steps issued so far by this CTA
     unsigned issued_k = 0, issued_v = 0;
     for (unsigned gi = 0;; ++gi) {
       int it = 0;
@@ -228,34 +218,36 @@ __global__ void __launch_bounds__(kRoundThreads, 1)
       const int head_pages = (st.len + kPageTokens - 1) / kPageTokens;
       const int32_t* pt = dv.page_table + hs * dv.max_pages;
       bool ok = true;
-      // lane p < 8 handles page p of a block (past the head's end: a page of it again - finite data, masked);
-      // the ids of the next block are fetched while this one is being issued
-      auto page_of = [&](int blk) { return lane < 8 ? pt[min(blk * 8 + lane, max(head_pages - 1, 0))] : 0; };
-      int pid = w.blk_begin < w.blk_end ? page_of(w.blk_begin) : 0;
-      for (int blk = w.blk_begin; blk < w.blk_end && ok; ++blk, ++gb) {
+      // lane p < 4 handles page p of a step (past the head's end: a page of it again - finite data, masked);
+      // the ids of the next step are fetched while this one is being issued
+      constexpr int kStepPages = kStep / kPageTokens;
+      auto page_of = [&](int step) { return lane < kStepPages ? pt[min(step * kStepPages + lane, max(head_pages - 1, 0))] : 0; };
+      const int s_begin = first_step(w), s_end = end_step(w, st.len);
+      int pid = s_begin < s_end ? page_of(s_begin) : 0;
+      for (int step = s_begin; step < s_end && ok; ++step, ++gb) {
         const int s = gb % kKvStages;
         const unsigned use = gb / kKvStages;   // how often the stage has been filled before
-        const int pid_next = blk + 1 < w.blk_end ? page_of(blk + 1) : 0;
-        // K of the block: its stage is free as soon as the scores of three blocks ago have been computed
+        const int pid_next = step + 1 < s_end ? page_of(step + 1) : 0;
+        // K of the step: its stage is free as soon as the scores of two steps ago have been computed
         if (gb >= kKvStages) ok = __all_sync(0xffffffffu, mbar_wait(&ctl->k_empty[s], (use - 1) & 1, abort_flag));
         if (!ok) break;
         if (lane == 0) mbar_arrive_expect_tx(&ctl->k_full[s], (uint32_t)KV_TILE);
         __syncwarp();
-        if (lane < 8) {
+        if (lane < kStepPages) {
 #pragma unroll
           for (int h = 0; h < HALVES; ++h)
-            tma_load_page_half<D>(k_tile + s * KV_TILE + h * kHalfBytes + lane * 2048, &map_pool, h, 0, pid, &ctl->k_full[s]);
+            tma_load_page_half<D>(k_tile + s * KV_TILE + h * kKvHalfBytes + lane * 2048, &map_pool, h, 0, pid, &ctl->k_full[s]);
         }
         issued_k = gb + 1;
-        // V of the block: its stage is free once the product of two blocks ago has run
+        // V of the step: its stage is free once the product of two steps ago has run
         if (gb >= kKvStages) ok = __all_sync(0xffffffffu, mbar_wait(&ctl->v_empty[s], (use - 1) & 1, abort_flag));
         if (!ok) break;
         if (lane == 0) mbar_arrive_expect_tx(&ctl->v_full[s], (uint32_t)KV_TILE);
         __syncwarp();
-        if (lane < 8) {
+        if (lane < kStepPages) {
 #pragma unroll
           for (int h = 0; h < HALVES; ++h)
-            tma_load_page_half<D>(v_tile + s * KV_TILE + h * kHalfBytes + lane * 2048, &map_pool, h, 1, pid, &ctl->v_full[s]);
+            tma_load_page_half<D>(v_tile + s * KV_TILE + h * kKvHalfBytes + lane * 2048, &map_pool, h, 1, pid, &ctl->v_full[s]);
         }
         issued_v = gb + 1;
         pid = pid_next;
@@ -287,26 +279,26 @@ __global__ void __launch_bounds__(kRoundThreads, 1)
       unsigned gb = 0;
       bool ok = true;
       const uint32_t q0 = smem_u32(q_tile);
-      // O = sum over the item's blocks of P V, accumulated in tensor memory (the softmax threads rescale it there on
+      // O = sum over the item's steps of P V, accumulated in tensor memory (the softmax threads rescale it there on
       // the rare occasions a row's reference maximum moves).  P is read out of tensor memory (operand A), V out of
       // shared memory.
       auto issue_pv = [&](unsigned g, bool first_of_item, unsigned gi) -> bool {
-        const int s = g % kKvStages, pb = g & 1;
-        if (!mbar_wait(&ctl->p_full[pb], (g >> 1) & 1, abort_flag)) return false;
+        const int s = g % kKvStages;
+        if (!mbar_wait(&ctl->p_full, g & 1, abort_flag)) return false;
         if (!mbar_wait(&ctl->v_full[s], (g / kKvStages) & 1, abort_flag)) return false;
         // the first product of an item overwrites the accumulator: the item before must have been read out
         if (first_of_item && gi >= 1 && !mbar_wait(&ctl->o_read, (gi - 1) & 1, abort_flag)) return false;
         tc_fence_after();
         const uint32_t v0 = smem_u32(v_tile + s * KV_TILE);
-        const uint32_t p0 = tmem + kPCol + (uint32_t)pb * kPBuf;
+        const uint32_t p0 = tmem + kPCol;
 #pragma unroll
-        for (int kk = 0; kk < kBlk / 16; ++kk) {   // 16 tokens per instruction: 8 columns of bf16 pairs
-          const uint64_t db = operand_desc_mn(v0 + (uint32_t)(kk * 16 * 128), kHalfBytes, 1024);
+        for (int kk = 0; kk < kStep / 16; ++kk) {   // 16 tokens per instruction: 8 columns of bf16 pairs
+          const uint64_t db = operand_desc_mn(v0 + (uint32_t)(kk * 16 * 128), kKvHalfBytes, 1024);
           umma_bf16_tmem_a(tmem + kOCol, p0 + (uint32_t)(kk * 8), db, kIdescPV, (kk > 0 || !first_of_item) ? 1u : 0u);
           umma_bf16_tmem_a(tmem + kOCol, p0 + kPLo + (uint32_t)(kk * 8), db, kIdescPV, 1);
         }
         umma_commit(&ctl->v_empty[s]);
-        umma_commit(&ctl->p_empty[pb]);
+        umma_commit(&ctl->p_empty);
         return true;
       };
       for (unsigned gi = 0; ok; ++gi) {
@@ -316,25 +308,27 @@ __global__ void __launch_bounds__(kRoundThreads, 1)
         mbar_arrive(&ctl->item_taken);
         if (it < 0) break;
         const RoundItem w = items[it];
-        const int nb = w.blk_end - w.blk_begin;
+        const HeadState st = dv.state[(size_t)layer * dv.n_heads + w.head];
+        const int nb = end_step(w, st.len) - first_step(w);
         ok = mbar_wait(&ctl->q_ready, gi & 1, abort_flag);
         for (int i = 0; i < nb && ok; ++i) {
           const unsigned g = gb + i;
           const int s = g % kKvStages;
           ok = mbar_wait(&ctl->k_full[s], (g / kKvStages) & 1, abort_flag);
-          // S is overwritten: the softmax threads must have the scores of the block before in registers
+          // S is overwritten: the softmax threads must have the scores of the step before in registers
           if (ok && g >= 1) ok = mbar_wait(&ctl->s_empty, (g - 1) & 1, abort_flag);
           if (!ok) break;
           tc_fence_after();
           const uint32_t k0 = smem_u32(k_tile + s * KV_TILE);
 #pragma unroll
           for (int kk = 0; kk < D / 16; ++kk) {   // 16 elements = 32 bytes along the swizzled half row
-            const uint32_t off = (uint32_t)((kk >> 2) * kHalfBytes + (kk & 3) * 32);
-            umma_bf16_desc(tmem, operand_desc(q0 + off), operand_desc(k0 + off), kIdescQK, kk > 0);
+            const uint32_t q_off = (uint32_t)((kk >> 2) * kQHalfBytes + (kk & 3) * 32);
+            const uint32_t k_off = (uint32_t)((kk >> 2) * kKvHalfBytes + (kk & 3) * 32);
+            umma_bf16_desc(tmem, operand_desc(q0 + q_off), operand_desc(k0 + k_off), kIdescQK, kk > 0);
           }
           umma_commit(&ctl->k_empty[s]);
           umma_commit(&ctl->s_full);
-          if (i >= 1) ok = issue_pv(g - 1, i == 1, gi);   // behind the next block's scores, so that its softmax overlaps this product
+          if (i >= 1) ok = issue_pv(g - 1, i == 1, gi);   // behind the next step's scores, so that its softmax overlaps this product
         }
         if (ok && nb > 0) ok = issue_pv(gb + nb - 1, nb == 1, gi);
         gb += nb;
@@ -347,17 +341,12 @@ __global__ void __launch_bounds__(kRoundThreads, 1)
     }
     __syncwarp();
   } else {
-    // ================================================================ softmax and epilogue: four threads per query row
-    // A warp works on 16 tensor-memory lanes (query rows) in the fragment layout of the .16x256b loads: thread t has
-    // rows t / 4 and t / 4 + 8 of them and, of every 8 columns, the pair 2 (t % 4), 2 (t % 4) + 1.  Two warps share a
-    // lane quarter (and a scheduler), so one's transcendental and conversion work overlaps the other's arithmetic.
-    const int tid = (int)threadIdx.x - 64;                 // 0 .. 255 among the softmax threads
-    const int lane0 = (warp & 3) * 32 + ((warp - 2) >> 2) * 16;   // first of the warp's 16 lanes (a warp may access the quarter warp % 4)
-    const int cq = lane & 3;
-    const int row0 = lane0 + (lane >> 2);                  // the thread's rows: row0 and row0 + 8
-    const uint32_t lane_addr = tmem + ((uint32_t)lane0 << 16);
+    // ================================================================ softmax and epilogue: a thread per query row
+    const int sw = warp & 3;                     // tensor-memory lane quarter this warp may access
+    const int row = sw * 32 + lane;
+    const uint32_t lane_addr = tmem + ((uint32_t)(sw * 32) << 16);
     const float scale_log2 = dv.scale_log2;
-    unsigned gb = 0, n_sync = 0;   // blocks so far; exchanges of column positions so far
+    unsigned gb = 0, n_sync = 0;   // steps so far; exchanges of column positions so far
     bool ok = true;
     for (unsigned gi = 0; ok; ++gi) {
       ok = mbar_wait(&ctl->item_ready, gi & 1, abort_flag);
@@ -370,74 +359,43 @@ __global__ void __launch_bounds__(kRoundThreads, 1)
       const HeadState st = dv.state[hs];
       const int b = w.head / dv.n_kv_heads, g_kv = w.head % dv.n_kv_heads;
       const int total = st.len + st.n_drop;
-      // row -> query token t (within the round) and query head j of the group
-      auto row_token = [&](int row) { return w.q_tile * tok_per_tile + row / G; };
-      auto row_offset = [&](int row) {
-        const int t = row_token(row), j = row % G;
-        return (((size_t)b * jb.n_tok + min(t, jb.n_tok - 1)) * ((size_t)dv.n_kv_heads * G) + (size_t)g_kv * G + j) * D;
-      };
-      bool row_live[2];
-      int q_pos[2];
-      size_t row_off[2];
-#pragma unroll
-      for (int r = 0; r < 2; ++r) {
-        const int t = row_token(row0 + 8 * r);
-        row_live[r] = t < jb.n_tok;
-        q_pos[r] = total - jb.n_tok + t;
-        row_off[r] = row_offset(row0 + 8 * r);
-      }
+      // this row: query token t (within the round), query head j of the group
+      const int t = w.q_tile * tok_per_tile + row / G, j = row % G;
+      const bool row_live = t < jb.n_tok;
+      const int q_pos = total - jb.n_tok + t;
+      const size_t row_off = (((size_t)b * jb.n_tok + min(t, jb.n_tok - 1)) * ((size_t)dv.n_kv_heads * G) + (size_t)g_kv * G + j) * D;
 
-      // ---- the query tile into shared memory (operand layout: 128-byte half rows, chunks swizzled by the row):
-      // two threads per row, half a row each
+      // ---- the query row into shared memory (operand layout: 128-byte half rows, chunks swizzled by the row)
+      const bool seed = w.part_idx == 0 && dv.use_comp && st.n_drop > 0 && st.window >= 0;
+      float s_c = 0.f;
       {
-        const int qr = tid >> 1;
-        const bool live = row_token(qr) < jb.n_tok;
-        const uint4* src = (const uint4*)(q + row_offset(qr));
+        const uint4* src = (const uint4*)(q + row_off);
+        const float* k_hat = dv.comp_mean + hs * 2 * D;
 #pragma unroll
-        for (int cc = 0; cc < D / 16; ++cc) {
-          const int c = (tid & 1) * (D / 16) + cc;
-          const uint4 u = live ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);
-          *(uint4*)(q_tile + (c >> 3) * kHalfBytes + qr * 128 + (((c & 7) ^ (qr & 7)) << 4)) = u;
+        for (int c = 0; c < D / 8; ++c) {
+          uint4 u = row_live ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);
+          *(uint4*)(q_tile + (c >> 3) * kQHalfBytes + row * 128 + (((c & 7) ^ (row & 7)) << 4)) = u;
+          if (seed) {
+            float f[8];
+            Elem<__nv_bfloat16>::unpack(u, f);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) s_c = fmaf(f[e], k_hat[c * 8 + e], s_c);
+          }
         }
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       mbar_arrive(&ctl->q_ready);
 
-      // ---- the compensation token's score q . k_hat of the thread's two rows: a quarter of the row each, summed
-      // over the four threads
-      const bool seed = w.part_idx == 0 && dv.use_comp && st.n_drop > 0 && st.window >= 0;
-      float s_c[2] = {0.f, 0.f};
-      if (seed) {
-        const float* k_hat = dv.comp_mean + hs * 2 * D;
-#pragma unroll
-        for (int r = 0; r < 2; ++r) {
-          const uint4* src = (const uint4*)(q + row_off[r]);
-#pragma unroll
-          for (int cc = 0; cc < D / 32; ++cc) {
-            const int c = cq * (D / 32) + cc;
-            const uint4 u = row_live[r] ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);
-            float f[8];
-            Elem<__nv_bfloat16>::unpack(u, f);
-#pragma unroll
-            for (int e = 0; e < 8; ++e) s_c[r] = fmaf(f[e], k_hat[c * 8 + e], s_c[r]);
-          }
-          s_c[r] += __shfl_xor_sync(0xffffffffu, s_c[r], 1);
-          s_c[r] += __shfl_xor_sync(0xffffffffu, s_c[r], 2);
-        }
-      }
-
       // Online softmax against a reference maximum m_ref that is allowed to lag: weights are 2^(s - m_ref), at
       // most 2^kLag, and the accumulator in tensor memory is rescaled only when a row's maximum has outrun the
-      // reference by more than kLag (rare after the first blocks).  The compensation token (Eq. 4, Eq. 5: weight
-      // N_d exp(s_c), value v_hat) is carried as a scalar weight w_seed and added at the end.  A thread keeps the
-      // sum of its own columns' weights; the four partial sums of a row meet at the end.
+      // reference by more than kLag (rare after the first steps).  The compensation token (Eq. 4, Eq. 5: weight
+      // N_d exp(s_c), value v_hat) is carried as a scalar weight w_seed and added at the end.
       constexpr float kLag = 8.f;
-      float m_ref[2], l_part[2], w_seed[2];
-#pragma unroll
-      for (int r = 0; r < 2; ++r) {
-        m_ref[r] = seed ? s_c[r] * scale_log2 + log2f((float)st.n_drop) : -CUDART_INF_F;
-        l_part[r] = (seed && cq == 0) ? 1.f : 0.f;
-        w_seed[r] = seed ? 1.f : 0.f;
+      float m_ref = -CUDART_INF_F, l_run = 0.f, w_seed = 0.f;
+      if (seed) {
+        m_ref = s_c * scale_log2 + log2f((float)st.n_drop);
+        l_run = 1.f;
+        w_seed = 1.f;
       }
       const bool in_order = st.window < 0 || st.n_drop == 0;               // slot = position
       const int q_pos_min = total - jb.n_tok + w.q_tile * tok_per_tile;    // the tile's earliest query
@@ -448,26 +406,26 @@ __global__ void __launch_bounds__(kRoundThreads, 1)
         else if (lo < st.ring_head) { new_lo = dv.n_sink + lo; new_hi = dv.n_sink + st.ring_head; }
         else { new_lo = dv.n_sink + lo; new_hi = dv.n_sink + st.window; new_lo2 = dv.n_sink; new_hi2 = dv.n_sink + st.ring_head; }
       }
-      const int nb = w.blk_end - w.blk_begin;
+      const int s_begin = first_step(w);
+      const int nb = end_step(w, st.len) - s_begin;
       for (int i = 0; i < nb && ok; ++i) {
         const unsigned g = gb + i;
-        const int pb = g & 1, blk = w.blk_begin + i;
-        const int slot0 = blk * kBlk;
-        // Does the block need masking?  Slots beyond the head's length, or tokens of the round (the newest n_tok: the
+        const int slot0 = (s_begin + i) * kStep;
+        // Does the step need masking?  Slots beyond the head's length, or tokens of the round (the newest n_tok: the
         // last slots of a head whose slots are in position order, a cyclic run of the ring otherwise) that come
         // after some query of the tile.  Every thread finds the same answer from the head's state, so the common
-        // case costs no exchange; in a block that does need it the position of each column is worked out by one
-        // thread and traded through shared memory.
-        const int slot1 = slot0 + kBlk;
+        // case costs no exchange; in a step that does need it each of the first 64 threads works out the position
+        // of one column and the four warps trade them through shared memory.
+        const int slot1 = slot0 + kStep;
         bool masked = slot1 > st.len;
         if (in_order) masked |= slot1 - 1 > q_pos_min;
         else masked |= (slot0 < new_hi && new_lo < slot1) || (slot0 < new_hi2 && new_lo2 < slot1);
         const int32_t* col_pos = ctl->col_pos[n_sync & 1];
         if (masked) {
-          // (double-buffered: a thread may still be reading the positions of the masked block before)
-          if (tid < kBlk) {
-            const int s = slot0 + tid;   // column tid of the block
-            ctl->col_pos[n_sync & 1][tid] = s < st.len ? slot_pos(s, dv.n_sink, st.ring_head, st.window, st.n_drop, total) : 0x7fffffff;
+          // (double-buffered: a thread may still be reading the positions of the masked step before)
+          if (row < kStep) {
+            const int s = slot0 + row;   // column `row` of the step
+            ctl->col_pos[n_sync & 1][row] = s < st.len ? slot_pos(s, dv.n_sink, st.ring_head, st.window, st.n_drop, total) : 0x7fffffff;
           }
           mbar_arrive(&ctl->blk_sync);
           ok = mbar_wait(&ctl->blk_sync, n_sync & 1, abort_flag);
@@ -478,185 +436,142 @@ __global__ void __launch_bounds__(kRoundThreads, 1)
         if (!ok) break;
         tc_fence_after();
 
-        // ---- the thread's 2 x 64 scores, in registers: v[4j + 2r + e] is row r, column 8j + 2cq + e
-        uint32_t v[64];
-        tmem_ld_frag64(lane_addr, v);
-        tmem_ld_frag64(lane_addr + 64u, v + 32);
+        // ---- this row's 64 scores, in registers
+        uint32_t v[kStep];
+#pragma unroll
+        for (int c = 0; c < kStep / 32; ++c) tmem_ld32_issue(lane_addr + (uint32_t)(c * 32), v + c * 32);
         tmem_ld_wait_all();
 #pragma unroll
-        for (int e = 0; e < 64; ++e) asm volatile("" : "+r"(v[e]));
+        for (int e = 0; e < kStep; ++e) asm volatile("" : "+r"(v[e]));
         tc_fence_before();
         mbar_arrive(&ctl->s_empty);
         if (masked) {
 #pragma unroll
-          for (int j = 0; j < kBlk / 8; ++j)
-#pragma unroll
-            for (int e = 0; e < 2; ++e) {
-              const int cp = col_pos[8 * j + 2 * cq + e];
-              if (cp > q_pos[0]) v[4 * j + e] = 0xff800000u;   // -inf
-              if (cp > q_pos[1]) v[4 * j + 2 + e] = 0xff800000u;
-            }
+          for (int e = 0; e < kStep; ++e)
+            if (col_pos[e] > q_pos) v[e] = 0xff800000u;   // -inf
         }
-        // ---- the rows' maxima over the block: own columns, then the four threads of a row
-        float m_blk[2];
+        float mx0 = -CUDART_INF_F, mx1 = -CUDART_INF_F;
 #pragma unroll
-        for (int r = 0; r < 2; ++r) {
-          float mx0 = -CUDART_INF_F, mx1 = -CUDART_INF_F;
-#pragma unroll
-          for (int j = 0; j < kBlk / 8; j += 2) {
-            mx0 = max3(mx0, __uint_as_float(v[4 * j + 2 * r]), __uint_as_float(v[4 * j + 2 * r + 1]));
-            mx1 = max3(mx1, __uint_as_float(v[4 * j + 4 + 2 * r]), __uint_as_float(v[4 * j + 4 + 2 * r + 1]));
-          }
-          float mx = fmaxf(mx0, mx1);
-          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-          m_blk[r] = mx * scale_log2;   // (the scale is positive: the max of the scaled scores is the scaled max)
+        for (int e = 0; e < kStep; e += 4) {
+          mx0 = max3(mx0, __uint_as_float(v[e]), __uint_as_float(v[e + 1]));
+          mx1 = max3(mx1, __uint_as_float(v[e + 2]), __uint_as_float(v[e + 3]));
         }
+        // (the scale is positive: the max of the scaled scores is the scaled max)
+        const float m_blk = fmaxf(mx0, mx1) * scale_log2;
 
-        // ---- the product that read this buffer of P (two blocks ago) must have run before it is overwritten
-        if (g >= 2) ok = mbar_wait(&ctl->p_empty[pb], ((g >> 1) - 1) & 1, abort_flag);
+        // ---- the product of the step before must have run before P is overwritten (and before O is touched)
+        if (g >= 1) ok = mbar_wait(&ctl->p_empty, (g - 1) & 1, abort_flag);
         if (!ok) break;
-        // ---- move the reference maxima?  Tensor-memory loads and stores are warp-wide, so the warp decides as one.
-        bool want = false;
-#pragma unroll
-        for (int r = 0; r < 2; ++r) want |= m_blk[r] > m_ref[r] + kLag || (m_ref[r] == -CUDART_INF_F && m_blk[r] > -CUDART_INF_F);
+        // ---- move the reference maximum?  Tensor-memory loads and stores are warp-wide, so the warp decides as one.
+        const bool want = m_blk > m_ref + kLag || (m_ref == -CUDART_INF_F && m_blk > -CUDART_INF_F);
         if (__any_sync(0xffffffffu, want)) {
-          float f[2];
-#pragma unroll
-          for (int r = 0; r < 2; ++r) {
-            const float m_to = fmaxf(m_ref[r], m_blk[r]);
-            f[r] = (m_to == -CUDART_INF_F || m_ref[r] == -CUDART_INF_F) ? 0.f : fast_exp2(m_ref[r] - m_to);   // 1 for a row that stays
-            l_part[r] *= f[r];
-            w_seed[r] *= f[r];
-            m_ref[r] = m_to;
-          }
-          if (i >= 1) {   // the accumulator holds products of this item: rescale this warp's rows, once the last has run
-            ok = mbar_wait(&ctl->p_empty[pb ^ 1], ((g - 1) >> 1) & 1, abort_flag);
-            if (!ok) break;
+          const float m_to = fmaxf(m_ref, m_blk);
+          const float f = (m_to == -CUDART_INF_F || m_ref == -CUDART_INF_F) ? 0.f : fast_exp2(m_ref - m_to);   // 1 for a row that stays
+          if (i >= 1) {   // the accumulator holds products of this item: rescale this warp's rows
             tc_fence_after();
 #pragma unroll
-            for (int c = 0; c < D / 64; ++c) {
+            for (int c = 0; c < D / 32; ++c) {
               uint32_t o[32];
-              tmem_ld_frag64(lane_addr + kOCol + (uint32_t)(c * 64), o);
+              tmem_ld32_issue(lane_addr + kOCol + (uint32_t)(c * 32), o);
               tmem_ld_wait_all();
 #pragma unroll
               for (int e = 0; e < 32; ++e) {
                 asm volatile("" : "+r"(o[e]));
-                o[e] = __float_as_uint(__uint_as_float(o[e]) * f[(e >> 1) & 1]);
+                o[e] = __float_as_uint(__uint_as_float(o[e]) * f);
               }
-              tmem_st_frag64(lane_addr + kOCol + (uint32_t)(c * 64), o);
+              tmem_st32(lane_addr + kOCol + (uint32_t)(c * 32), o);
             }
             tmem_st_wait_all();
             tc_fence_before();
           }
+          l_run *= f;
+          w_seed *= f;
+          m_ref = m_to;
         }
-        float m_use[2];
-#pragma unroll
-        for (int r = 0; r < 2; ++r) m_use[r] = (m_ref[r] == -CUDART_INF_F) ? 0.f : m_ref[r];
+        const float m_use = (m_ref == -CUDART_INF_F) ? 0.f : m_ref;
 
-        // ---- weights, their sums, and P into its tensor-memory buffer: column c of the head half holds the bf16 pair of
-        // tokens 2c and 2c + 1 (the operand-A layout of the matrix unit), the remainder half the same
-        // A weight goes into the product as a bf16 head (its upper 16 bits) plus a bf16 remainder - two products - so
-        // that it keeps fp32-like accuracy: a single bf16 would put 2^-9 of a large weight times its V row into the result.
-        const uint64_t scale2 = f2_pack(scale_log2, scale_log2);
-        uint64_t neg_m2[2], psum2[2][2];
+        // ---- weights, their sum, and P into tensor memory: column c of the head half holds the bf16 pair of tokens
+        // 2c and 2c + 1 (the operand-A layout of the matrix unit), the remainder half the same.  A weight goes into
+        // the product as a bf16 head (its upper 16 bits) plus a bf16 remainder - two products - so that it keeps
+        // fp32-like accuracy: a single bf16 would put 2^-9 of a large weight times its V row into the result.
+        const uint64_t scale2 = f2_pack(scale_log2, scale_log2), neg_m2 = f2_pack(-m_use, -m_use);
+        uint64_t psum2[2] = {f2_pack(0.f, 0.f), f2_pack(0.f, 0.f)};
+        const uint32_t p_addr = lane_addr + kPCol;
 #pragma unroll
-        for (int r = 0; r < 2; ++r) {
-          neg_m2[r] = f2_pack(-m_use[r], -m_use[r]);
-          psum2[r][0] = psum2[r][1] = f2_pack(0.f, 0.f);
-        }
-        const uint32_t p_addr = lane_addr + kPCol + (uint32_t)pb * kPBuf;
-#pragma unroll
-        for (int hh = 0; hh < 2; ++hh) {   // 64 tokens = 32 columns of pairs at a time
+        for (int c = 0; c < kStep / 32; ++c) {   // 32 tokens = 16 columns of pairs
           uint32_t hi[16], lo[16];
 #pragma unroll
-          for (int jj = 0; jj < 8; ++jj) {
-            const int j = hh * 8 + jj;
-#pragma unroll
-            for (int r = 0; r < 2; ++r) {
-              float t0, t1, l0, l1;
-              f2_unpack(f2_fma(f2_pack(__uint_as_float(v[4 * j + 2 * r]), __uint_as_float(v[4 * j + 2 * r + 1])), scale2, neg_m2[r]), t0, t1);
-              const float w0 = fast_exp2(t0), w1 = fast_exp2(t1);
-              const uint64_t w2 = f2_pack(w0, w1);
-              psum2[r][jj & 1] = f2_add(psum2[r][jj & 1], w2);
-              const uint32_t b0 = __float_as_uint(w0), b1 = __float_as_uint(w1);
-              hi[2 * jj + r] = __byte_perm(b0, b1, 0x7632);
-              f2_unpack(f2_sub(w2, f2_pack(__uint_as_float(b0 & 0xffff0000u), __uint_as_float(b1 & 0xffff0000u))), l0, l1);
-              lo[2 * jj + r] = pack2_bf16(l0, l1);
-            }
+          for (int e2 = 0; e2 < 16; ++e2) {
+            const int e = c * 32 + e2 * 2;
+            float t0, t1, l0, l1;
+            f2_unpack(f2_fma(f2_pack(__uint_as_float(v[e]), __uint_as_float(v[e + 1])), scale2, neg_m2), t0, t1);
+            const float w0 = fast_exp2(t0), w1 = fast_exp2(t1);
+            const uint64_t w2 = f2_pack(w0, w1);
+            psum2[e2 & 1] = f2_add(psum2[e2 & 1], w2);
+            const uint32_t b0 = __float_as_uint(w0), b1 = __float_as_uint(w1);
+            hi[e2] = __byte_perm(b0, b1, 0x7632);
+            f2_unpack(f2_sub(w2, f2_pack(__uint_as_float(b0 & 0xffff0000u), __uint_as_float(b1 & 0xffff0000u))), l0, l1);
+            lo[e2] = pack2_bf16(l0, l1);
           }
-          tmem_st_frag32(p_addr + (uint32_t)(hh * 32), hi);
-          tmem_st_frag32(p_addr + kPLo + (uint32_t)(hh * 32), lo);
+          tmem_st16(p_addr + (uint32_t)(c * 16), hi);
+          tmem_st16(p_addr + kPLo + (uint32_t)(c * 16), lo);
         }
-#pragma unroll
-        for (int r = 0; r < 2; ++r) {
+        {
           float a0, a1;
-          f2_unpack(f2_add(psum2[r][0], psum2[r][1]), a0, a1);
-          l_part[r] += a0 + a1;
+          f2_unpack(f2_add(psum2[0], psum2[1]), a0, a1);
+          l_run += a0 + a1;
         }
         // V rows of slots beyond the head's length may hold anything (a zero weight times a NaN is a NaN): zero them
-        if (slot0 + kBlk > st.len) {
+        if (slot0 + kStep > st.len) {
           ok = mbar_wait(&ctl->v_full[g % kKvStages], (g / kKvStages) & 1, abort_flag);   // the rows must have landed before they are overwritten
           if (!ok) break;
           const int first_bad = max(st.len - slot0, 0);
           uint8_t* vt = v_tile + (g % kKvStages) * KV_TILE;
-          for (int idx = first_bad * 8 + tid; idx < kBlk * 8; idx += kSoftmaxThreads) {   // 16-byte chunks of the bad rows
+          for (int idx = first_bad * 8 + row; idx < kStep * 8; idx += kSoftmaxThreads) {   // 16-byte chunks of the bad rows
 #pragma unroll
-            for (int h = 0; h < HALVES; ++h) *(uint4*)(vt + h * kHalfBytes + idx * 16) = make_uint4(0u, 0u, 0u, 0u);
+            for (int h = 0; h < HALVES; ++h) *(uint4*)(vt + h * kKvHalfBytes + idx * 16) = make_uint4(0u, 0u, 0u, 0u);
           }
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         }
         tmem_st_wait_all();
         tc_fence_before();
-        mbar_arrive(&ctl->p_full[pb]);
+        mbar_arrive(&ctl->p_full);
       }
       if (!ok) break;
-      // ---- the rows' results: accumulator out of tensor memory once the last product is done, plus the
+      // ---- the row's result: accumulator out of tensor memory once the last product is done, plus the
       // compensation token's share; the output when the unit is in one part, else a partial record
       if (nb > 0) {
-        ok = mbar_wait(&ctl->p_empty[(gb + nb - 1) & 1], ((gb + nb - 1) >> 1) & 1, abort_flag);
+        ok = mbar_wait(&ctl->p_empty, (gb + nb - 1) & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
       }
       gb += nb;
       const bool direct = w.n_parts == 1;
-      float inv[2];
-      float* dst[2];
-#pragma unroll
-      for (int r = 0; r < 2; ++r) {
-        float l = l_part[r];
-        l += __shfl_xor_sync(0xffffffffu, l, 1);
-        l += __shfl_xor_sync(0xffffffffu, l, 2);
-        l_part[r] = l;
-        inv[r] = direct ? (l > 0.f ? 1.f / l : 0.f) : 1.f;
-        const size_t rr = (size_t)w.rec_base + (size_t)w.part_idx * kRows + (size_t)(row0 + 8 * r);
-        dst[r] = direct ? out + row_off[r] : dv.rec_o + rr * D;
-        if (!direct && cq == 0) dv.rec_ml[rr] = make_float2(m_ref[r], l);
-      }
+      const float inv = direct ? (l_run > 0.f ? 1.f / l_run : 0.f) : 1.f;
+      const size_t r = (size_t)w.rec_base + (size_t)w.part_idx * kRows + row;
+      float* dst = direct ? out + row_off : dv.rec_o + r * D;
       const float* v_hat = dv.comp_mean + hs * 2 * D + D;
 #pragma unroll
-      for (int c = 0; c < D / 64; ++c) {
+      for (int c = 0; c < D / 32; ++c) {
         uint32_t o[32];
         if (nb > 0) {
-          tmem_ld_frag64(lane_addr + kOCol + (uint32_t)(c * 64), o);
+          tmem_ld32_issue(lane_addr + kOCol + (uint32_t)(c * 32), o);
           tmem_ld_wait_all();
         }
 #pragma unroll
-        for (int jj = 0; jj < 8; ++jj) {
-          const int col = c * 64 + 8 * jj + 2 * cq;
+        for (int e = 0; e < 32; ++e) {
+          asm volatile("" : "+r"(o[e]));
+          float x = nb > 0 ? __uint_as_float(o[e]) : 0.f;
+          if (seed) x = fmaf(w_seed, v_hat[c * 32 + e], x);
+          o[e] = __float_as_uint(x * inv);
+        }
+        if (direct ? row_live : true) {
 #pragma unroll
-          for (int r = 0; r < 2; ++r) {
-            asm volatile("" : "+r"(o[4 * jj + 2 * r]), "+r"(o[4 * jj + 2 * r + 1]));
-            float x0 = nb > 0 ? __uint_as_float(o[4 * jj + 2 * r]) : 0.f;
-            float x1 = nb > 0 ? __uint_as_float(o[4 * jj + 2 * r + 1]) : 0.f;
-            if (seed) {
-              x0 = fmaf(w_seed[r], v_hat[col], x0);
-              x1 = fmaf(w_seed[r], v_hat[col + 1], x1);
-            }
-            if (direct ? row_live[r] : true) *(float2*)(dst[r] + col) = make_float2(x0 * inv[r], x1 * inv[r]);
-          }
+          for (int e = 0; e < 32; e += 4)
+            *(float4*)(dst + c * 32 + e) = make_float4(__uint_as_float(o[e]), __uint_as_float(o[e + 1]), __uint_as_float(o[e + 2]), __uint_as_float(o[e + 3]));
         }
       }
+      if (!direct) dv.rec_ml[r] = make_float2(m_ref, l_run);
       tc_fence_before();
       mbar_arrive(&ctl->o_read);
     }
@@ -739,9 +654,12 @@ cudaError_t round_launch(const DeviceView& dv, long long pool_pages, int layer, 
   if (dev < 0 || dev >= 64 || !opted_in[dev]) {
     e = cudaFuncSetAttribute(round_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)round_smem_bytes<D>());
     if (e != cudaSuccess) return e;
+    // two CTAs to an SM need the largest shared-memory split
+    e = cudaFuncSetAttribute(round_kernel<D>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) opted_in[dev] = true;
   }
-  const int grid = std::max(1, std::min(n_sms, jb.n_items));
+  const int grid = std::max(1, std::min(n_sms * kCtasPerSm, jb.n_items));
   round_kernel<D><<<grid, kRoundThreads, round_smem_bytes<D>(), s>>>(dv, map, layer, jb, (const __nv_bfloat16*)q, out);
   e = cudaGetLastError();
   if (e != cudaSuccess || jb.n_units == 0) return e;
