@@ -666,8 +666,19 @@ int razor_append_many(razor_cache_t* c, int32_t layer, const void* k_new, const 
   if (n_tokens >= kAppendChunkMin) {
     const long long nh = c->dv.n_heads;
     const long long room = ((long long)kCompressSliceBudget + nh) / (2 * nh);   // two sets of sums per slice
-    slices = (int)std::max(1LL, std::min({(long long)ceil_div((long long)c->n_sms * 8, nh), room,
-                                           (long long)(n_tokens / 32)}));
+    const long long cap = std::max(1LL, std::min(room, (long long)(n_tokens / 32)));
+    const long long s0 = std::max(1LL, std::min((long long)ceil_div((long long)c->n_sms * 8, nh), cap));
+    // two CTAs of the kernel are resident per SM: among s0 .. 1.5 s0 slices take the count whose CTAs fill their
+    // last wave best
+    const long long resident = 2LL * c->n_sms;
+    long long best = s0;
+    double best_fill = 0.0;
+    for (long long sl = s0; sl <= std::min(cap, s0 + s0 / 2); ++sl) {
+      const long long n = sl * nh, waves = (n + resident - 1) / resident;
+      const double fill = (double)n / (double)(waves * resident);
+      if (fill > best_fill + 1e-9) { best_fill = fill; best = sl; }
+    }
+    slices = (int)best;
   }
   RZ_CUDA(launch_append_many(c->dv, c->cfg.dtype, layer, k_new, v_new, n_tokens, slices, (cudaStream_t)stream));
   c->note_write(layer, razor_cache::kWriteBulk);

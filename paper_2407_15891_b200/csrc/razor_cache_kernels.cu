@@ -414,36 +414,50 @@ __global__ void __launch_bounds__(256) append_chunk_kernel(DeviceView dv, int la
   float accK[EPL], accV[EPL], ringK[EPL], ringV[EPL];
 #pragma unroll
   for (int i = 0; i < EPL; ++i) accK[i] = accV[i] = ringK[i] = ringV[i] = 0.f;
-  for (int a = a0 + grp; a < a1; a += NGRP) {
-    const size_t row = (((size_t)b * n_tok + a) * dv.n_kv_heads + g) * D;
-    const uint4 kf = ld_stream((const uint4*)(k_new + row) + lir);
-    const uint4 vf = ld_stream((const uint4*)(v_new + row) + lir);
-    const AppendFate fate = append_fate(st, n_sink, n_tok, a);
-    const int slot = fate.slot;
-    const bool stays = slot >= 0, had_old = fate.evicts_old;
-    float a_k[EPL], a_v[EPL];
-    if (stays) {
-      const size_t page = (size_t)pt[slot >> 4];
-      uint4* dst = (uint4*)(dv.pool + page * dv.page_bytes + (size_t)(slot & 15) * Geo::kRowBytes) + swz(slot, lir);
-      if (had_old && !skip_old) {
-        Elem<T>::unpack(dst[0], a_k);
-        Elem<T>::unpack(dst[kPageTokens * LPR], a_v);
+  constexpr int U = 4;   // rows of a thread group in flight
+  for (int a_first = a0 + grp; a_first < a1; a_first += NGRP * U) {
+    uint4 kfs[U], vfs[U];
 #pragma unroll
-        for (int i = 0; i < EPL; ++i) { accK[i] += a_k[i]; accV[i] += a_v[i]; }
+    for (int u = 0; u < U; ++u) {
+      const int a = a_first + u * NGRP;
+      if (a < a1) {
+        const size_t row = (((size_t)b * n_tok + a) * dv.n_kv_heads + g) * D;
+        kfs[u] = ld_stream((const uint4*)(k_new + row) + lir);
+        vfs[u] = ld_stream((const uint4*)(v_new + row) + lir);
       }
-      dst[0] = kf;
-      dst[kPageTokens * LPR] = vf;
-      if (st.window >= 0 && slot >= n_sink) {   // a row of the new window
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const int a = a_first + u * NGRP;
+      if (a >= a1) break;
+      const uint4 kf = kfs[u], vf = vfs[u];
+      const AppendFate fate = append_fate(st, n_sink, n_tok, a);
+      const int slot = fate.slot;
+      const bool stays = slot >= 0, had_old = fate.evicts_old;
+      float a_k[EPL], a_v[EPL];
+      if (stays) {
+        const size_t page = (size_t)pt[slot >> 4];
+        uint4* dst = (uint4*)(dv.pool + page * dv.page_bytes + (size_t)(slot & 15) * Geo::kRowBytes) + swz(slot, lir);
+        if (had_old && !skip_old) {
+          Elem<T>::unpack(dst[0], a_k);
+          Elem<T>::unpack(dst[kPageTokens * LPR], a_v);
+#pragma unroll
+          for (int i = 0; i < EPL; ++i) { accK[i] += a_k[i]; accV[i] += a_v[i]; }
+        }
+        dst[0] = kf;
+        dst[kPageTokens * LPR] = vf;
+        if (st.window >= 0 && slot >= n_sink) {   // a row of the new window
+          Elem<T>::unpack(kf, a_k);
+          Elem<T>::unpack(vf, a_v);
+#pragma unroll
+          for (int i = 0; i < EPL; ++i) { ringK[i] += a_k[i]; ringV[i] += a_v[i]; }
+        }
+      } else {
         Elem<T>::unpack(kf, a_k);
         Elem<T>::unpack(vf, a_v);
 #pragma unroll
-        for (int i = 0; i < EPL; ++i) { ringK[i] += a_k[i]; ringV[i] += a_v[i]; }
+        for (int i = 0; i < EPL; ++i) { accK[i] += a_k[i]; accV[i] += a_v[i]; }
       }
-    } else {
-      Elem<T>::unpack(kf, a_k);
-      Elem<T>::unpack(vf, a_v);
-#pragma unroll
-      for (int i = 0; i < EPL; ++i) { accK[i] += a_k[i]; accV[i] += a_v[i]; }
     }
   }
   // two sets of sums per slice: rows that join the dropped set, rows stored into the window
