@@ -107,7 +107,7 @@ def test_round_longer_than_one_launch_runs_block_by_block(group, T, D):
 
 
 @pytest.mark.parametrize("group,T,D", [(1, 64, 128), (1, 200, 128), (4, 40, 128), (2, 300, 64), (8, 16, 128), (1, 512, 64),
-                                        (4, 512, 128)])
+                                        (4, 512, 128), (1, 2048, 128), (4, 2048, 64)])
 def test_prompt_sized_round_on_the_query_tiled_kernel(group, T, D):
     """Rounds with at least 64 query rows per KV head run on the query-tiled tensor-core kernel: ragged batch (one
     sequence shorter than a block, one whose window evicts and wraps during the rounds), two rounds in a row,
