@@ -102,7 +102,7 @@ __device__ __forceinline__ uint32_t pack2_bf16(float lo, float hi) {
   return *(const uint32_t*)&v;
 }
 
-// 32 or 16 consecutive columns of this thread's lane into tensor memory; complete after tmem_st_wait_all().
+// 32 consecutive columns of this thread's lane into tensor memory; complete after tmem_st_wait_all().
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* v) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
@@ -113,15 +113,6 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* v) {
         "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]), "r"(v[16]), "r"(v[17]),
         "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]), "r"(v[24]), "r"(v[25]), "r"(v[26]),
         "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
-      : "memory");
-}
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* v) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
-      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
-      :
-      : "r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]),
-        "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
       : "memory");
 }
 __device__ __forceinline__ void tmem_st_wait_all() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
@@ -459,12 +450,18 @@ __global__ void __launch_bounds__(kRoundThreads, kCtasPerSm)
         // (the scale is positive: the max of the scaled scores is the scaled max)
         const float m_blk = fmaxf(mx0, mx1) * scale_log2;
 
-        // ---- the product of the step before must have run before P is overwritten (and before O is touched)
-        if (g >= 1) ok = mbar_wait(&ctl->p_empty, (g - 1) & 1, abort_flag);
-        if (!ok) break;
+        // The product of the step before must have run before P is overwritten and before O is touched.  The
+        // weights themselves need neither, so in the common case (no rescaling) they are computed into registers
+        // first and the wait comes just before the stores: the product's latency hides behind the arithmetic.
+        bool p_free = g == 0;
         // ---- move the reference maximum?  Tensor-memory loads and stores are warp-wide, so the warp decides as one.
         const bool want = m_blk > m_ref + kLag || (m_ref == -CUDART_INF_F && m_blk > -CUDART_INF_F);
         if (__any_sync(0xffffffffu, want)) {
+          if (!p_free) {
+            ok = mbar_wait(&ctl->p_empty, (g - 1) & 1, abort_flag);
+            if (!ok) break;
+            p_free = true;
+          }
           const float m_to = fmaxf(m_ref, m_blk);
           const float f = (m_to == -CUDART_INF_F || m_ref == -CUDART_INF_F) ? 0.f : fast_exp2(m_ref - m_to);   // 1 for a row that stays
           if (i >= 1) {   // the accumulator holds products of this item: rescale this warp's rows
@@ -497,25 +494,26 @@ __global__ void __launch_bounds__(kRoundThreads, kCtasPerSm)
         const uint64_t scale2 = f2_pack(scale_log2, scale_log2), neg_m2 = f2_pack(-m_use, -m_use);
         uint64_t psum2[2] = {f2_pack(0.f, 0.f), f2_pack(0.f, 0.f)};
         const uint32_t p_addr = lane_addr + kPCol;
+        uint32_t hi[kStep / 2], lo[kStep / 2];
 #pragma unroll
-        for (int c = 0; c < kStep / 32; ++c) {   // 32 tokens = 16 columns of pairs
-          uint32_t hi[16], lo[16];
-#pragma unroll
-          for (int e2 = 0; e2 < 16; ++e2) {
-            const int e = c * 32 + e2 * 2;
-            float t0, t1, l0, l1;
-            f2_unpack(f2_fma(f2_pack(__uint_as_float(v[e]), __uint_as_float(v[e + 1])), scale2, neg_m2), t0, t1);
-            const float w0 = fast_exp2(t0), w1 = fast_exp2(t1);
-            const uint64_t w2 = f2_pack(w0, w1);
-            psum2[e2 & 1] = f2_add(psum2[e2 & 1], w2);
-            const uint32_t b0 = __float_as_uint(w0), b1 = __float_as_uint(w1);
-            hi[e2] = __byte_perm(b0, b1, 0x7632);
-            f2_unpack(f2_sub(w2, f2_pack(__uint_as_float(b0 & 0xffff0000u), __uint_as_float(b1 & 0xffff0000u))), l0, l1);
-            lo[e2] = pack2_bf16(l0, l1);
-          }
-          tmem_st16(p_addr + (uint32_t)(c * 16), hi);
-          tmem_st16(p_addr + kPLo + (uint32_t)(c * 16), lo);
+        for (int e2 = 0; e2 < kStep / 2; ++e2) {
+          const int e = e2 * 2;
+          float t0, t1, l0, l1;
+          f2_unpack(f2_fma(f2_pack(__uint_as_float(v[e]), __uint_as_float(v[e + 1])), scale2, neg_m2), t0, t1);
+          const float w0 = fast_exp2(t0), w1 = fast_exp2(t1);
+          const uint64_t w2 = f2_pack(w0, w1);
+          psum2[e2 & 1] = f2_add(psum2[e2 & 1], w2);
+          const uint32_t b0 = __float_as_uint(w0), b1 = __float_as_uint(w1);
+          hi[e2] = __byte_perm(b0, b1, 0x7632);
+          f2_unpack(f2_sub(w2, f2_pack(__uint_as_float(b0 & 0xffff0000u), __uint_as_float(b1 & 0xffff0000u))), l0, l1);
+          lo[e2] = pack2_bf16(l0, l1);
         }
+        if (!p_free) {
+          ok = mbar_wait(&ctl->p_empty, (g - 1) & 1, abort_flag);
+          if (!ok) break;
+        }
+        tmem_st32(p_addr, hi);
+        tmem_st32(p_addr + kPLo, lo);
         {
           float a0, a1;
           f2_unpack(f2_add(psum2[0], psum2[1]), a0, a1);
