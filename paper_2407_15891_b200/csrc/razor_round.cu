@@ -353,6 +353,9 @@ __global__ void __launch_bounds__(kRoundThreads, kCtasPerSm)
       // this row: query token t (within the round), query head j of the group
       const int t = w.q_tile * tok_per_tile + row / G, j = row % G;
       const bool row_live = t < jb.n_tok;
+      // A warp none of whose rows is a query of the round (the last tile of a round is seldom full) keeps the pace of
+      // the barriers and computes nothing: its rows of P and O hold whatever they held, and nobody reads them.
+      const bool warp_live = __any_sync(0xffffffffu, row_live);
       const int q_pos = total - jb.n_tok + t;
       const size_t row_off = (((size_t)b * jb.n_tok + min(t, jb.n_tok - 1)) * ((size_t)dv.n_kv_heads * G) + (size_t)g_kv * G + j) * D;
 
@@ -399,6 +402,20 @@ __global__ void __launch_bounds__(kRoundThreads, kCtasPerSm)
       }
       const int s_begin = first_step(w);
       const int nb = end_step(w, st.len) - s_begin;
+      // V rows of slots beyond the head's length may hold anything (a zero weight times a NaN is a NaN): the softmax
+      // threads zero them in shared memory before the step's product is released.
+      auto zero_rows_beyond_the_end = [&](unsigned g, int slot0) -> bool {
+        if (slot0 + kStep <= st.len) return true;
+        if (!mbar_wait(&ctl->v_full[g % kKvStages], (g / kKvStages) & 1, abort_flag)) return false;   // the rows must have landed before they are overwritten
+        const int first_bad = max(st.len - slot0, 0);
+        uint8_t* vt = v_tile + (g % kKvStages) * KV_TILE;
+        for (int idx = first_bad * 8 + row; idx < kStep * 8; idx += kSoftmaxThreads) {   // 16-byte chunks of the bad rows
+#pragma unroll
+          for (int h = 0; h < HALVES; ++h) *(uint4*)(vt + h * kKvHalfBytes + idx * 16) = make_uint4(0u, 0u, 0u, 0u);
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        return true;
+      };
       for (int i = 0; i < nb && ok; ++i) {
         const unsigned g = gb + i;
         const int slot0 = (s_begin + i) * kStep;
@@ -426,6 +443,15 @@ __global__ void __launch_bounds__(kRoundThreads, kCtasPerSm)
         ok = mbar_wait(&ctl->s_full, g & 1, abort_flag);
         if (!ok) break;
         tc_fence_after();
+        if (!warp_live) {
+          tc_fence_before();
+          mbar_arrive(&ctl->s_empty);
+          if (g >= 1) ok = mbar_wait(&ctl->p_empty, (g - 1) & 1, abort_flag);   // (an arrival must not run into the phase before)
+          if (ok) ok = zero_rows_beyond_the_end(g, slot0);   // (every softmax thread has a share of that)
+          if (!ok) break;
+          mbar_arrive(&ctl->p_full);
+          continue;
+        }
 
         // ---- this row's 64 scores, in registers
         uint32_t v[kStep];
@@ -519,18 +545,8 @@ __global__ void __launch_bounds__(kRoundThreads, kCtasPerSm)
           f2_unpack(f2_add(psum2[0], psum2[1]), a0, a1);
           l_run += a0 + a1;
         }
-        // V rows of slots beyond the head's length may hold anything (a zero weight times a NaN is a NaN): zero them
-        if (slot0 + kStep > st.len) {
-          ok = mbar_wait(&ctl->v_full[g % kKvStages], (g / kKvStages) & 1, abort_flag);   // the rows must have landed before they are overwritten
-          if (!ok) break;
-          const int first_bad = max(st.len - slot0, 0);
-          uint8_t* vt = v_tile + (g % kKvStages) * KV_TILE;
-          for (int idx = first_bad * 8 + row; idx < kStep * 8; idx += kSoftmaxThreads) {   // 16-byte chunks of the bad rows
-#pragma unroll
-            for (int h = 0; h < HALVES; ++h) *(uint4*)(vt + h * kKvHalfBytes + idx * 16) = make_uint4(0u, 0u, 0u, 0u);
-          }
-          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        }
+        ok = zero_rows_beyond_the_end(g, slot0);
+        if (!ok) break;
         tmem_st_wait_all();
         tc_fence_before();
         mbar_arrive(&ctl->p_full);
@@ -550,7 +566,7 @@ __global__ void __launch_bounds__(kRoundThreads, kCtasPerSm)
       float* dst = direct ? out + row_off : dv.rec_o + r * D;
       const float* v_hat = dv.comp_mean + hs * 2 * D + D;
 #pragma unroll
-      for (int c = 0; c < D / 32; ++c) {
+      for (int c = 0; c < (warp_live ? D / 32 : 0); ++c) {
         uint32_t o[32];
         if (nb > 0) {
           tmem_ld32_issue(lane_addr + kOCol + (uint32_t)(c * 32), o);
@@ -569,7 +585,7 @@ __global__ void __launch_bounds__(kRoundThreads, kCtasPerSm)
             *(float4*)(dst + c * 32 + e) = make_float4(__uint_as_float(o[e]), __uint_as_float(o[e + 1]), __uint_as_float(o[e + 2]), __uint_as_float(o[e + 3]));
         }
       }
-      if (!direct) dv.rec_ml[r] = make_float2(m_ref, l_run);
+      if (!direct && warp_live) dv.rec_ml[r] = make_float2(m_ref, l_run);
       tc_fence_before();
       mbar_arrive(&ctl->o_read);
     }
