@@ -768,6 +768,11 @@ def main():
             line["round_of_512_tokens_32k"] = long_round_leg(rz, synth, dev)
         except Exception as ex:
             line["round_of_512_tokens_32k"] = {"unavailable": str(ex)[:200]}
+        try:   # a 32-token round (a short user turn): more rows than one launch of the streaming kernel takes, so the
+            # query-tiled kernel as well, most of whose 128 rows are then no query
+            line["round_of_32_tokens_32k"] = long_round_leg(rz, synth, dev, n_tok=32)
+        except Exception as ex:
+            line["round_of_32_tokens_32k"] = {"unavailable": str(ex)[:200]}
         try:   # a 4-token round (verify step) on the 32K MHA shape: same pages streamed, four queries per head
             line["round_of_4_tokens_32k"] = decode_only(rz, synth, "cfg2", 3, dev, peak, n_tok=4)
         except Exception as ex:

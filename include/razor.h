@@ -188,9 +188,11 @@ RAZOR_API int razor_decode_step(razor_cache_t* cache, int32_t layer, const void*
  *                                 n_tokens = 1 is razor_decode_attention.
  * Limits of the multi-token call: bf16; at least n_tokens tokens cached; every head that has dropped
  * tokens must have a window >= n_tokens (otherwise its mean would hold tokens that come after a query).
- * One launch takes a tile of 2, 4 or 8 rows per KV head (query heads of the group x query tokens, on
- * matrix instructions); a longer round runs as several launches, block by block, each streaming the
- * cache once and masking the round's tokens that come after its block.
+ * A round of at most 8 query rows per KV head (query heads of the group x query tokens) is one launch of
+ * the streaming kernel on a tile of 2, 4 or 8 rows (matrix instructions).  A longer round of a bf16 cache
+ * without ALiBi runs on the query-tiled tensor-core kernel (128 rows per tile; the threshold is
+ * RAZOR_OPT_ROUND_TILED_MIN_ROWS); otherwise it runs as several launches of the streaming kernel, block by
+ * block, each streaming the cache once and masking the round's tokens that come after its block.
  * Errors: NULL_PTR, INVALID_ARG, UNSUPPORTED_DIM, NOT_COMPRESSED, CAPACITY (append), MISALIGNED, CUDA.
  */
 RAZOR_API int razor_append_many(razor_cache_t* cache, int32_t layer, const void* k_new, const void* v_new,
@@ -272,11 +274,16 @@ enum {
                                            tile), 2 = never                                               */
   RAZOR_OPT_DECODE_STATIC_PERCENT = 6,  /* share of the pages handed out as per-CTA spans (0..100;
                                            default 80); 0 makes every job a tail item                     */
-  RAZOR_OPT_DECODE_EARLY_PREFETCH = 7   /* most pages (0..64; default 12) a CTA copies from the start of its span
+  RAZOR_OPT_DECODE_EARLY_PREFETCH = 7,  /* most pages (0..64; default 12) a CTA copies from the start of its span
                                            into shared memory before the kernel waits for the launch before it
                                            on the stream - only pages that no kernel still in flight can be
                                            writing (the host knows which page a preceding razor_append
                                            touched); 0: every copy waits                                   */
+  RAZOR_OPT_ROUND_TILED_MIN_ROWS = 8    /* razor_decode_attention_multi: rounds with at least this many query
+                                           rows per KV head (query heads of the group x new tokens; default 9,
+                                           i.e. more than one launch of the streaming kernel would take) run on
+                                           the query-tiled tensor-core kernel, shorter ones block by block on
+                                           the streaming kernel; bf16 caches without ALiBi only                */
 };
 RAZOR_API int razor_cache_set_option(razor_cache_t* cache, int32_t option, int32_t value);
 

@@ -249,7 +249,7 @@ def razor_schedule_plan(tokens, n_ctas: int = 148, static_percent: int = 80, tai
 
 
 OPT_DECODE_TAIL_ITEMS_PER_SM, OPT_DECODE_MIN_CHUNK_PAGES, OPT_DECODE_RING_KB, OPT_DECODE_CONSUMER_WARPS = 1, 2, 3, 4
-OPT_DECODE_TENSOR_CORES, OPT_DECODE_STATIC_PERCENT, OPT_DECODE_EARLY_PREFETCH = 5, 6, 7
+OPT_DECODE_TENSOR_CORES, OPT_DECODE_STATIC_PERCENT, OPT_DECODE_EARLY_PREFETCH, OPT_ROUND_TILED_MIN_ROWS = 5, 6, 7, 8
 
 
 def razor_cache_set_option(cache: int, option: int, value: int) -> None:

@@ -135,6 +135,7 @@ struct razor_cache {
   long long pool_pages = 0, next_page = 0;
   int n_sms = 148;
   DecodeTuning tune{3, 80, 32, 0, 0, 0, 12};
+  int round_tiled_min_rows = 9;   // rounds with at least this many query rows per KV head run on the query-tiled kernel
   std::vector<LayerHost> layers;
   WorkItem* pinned_items = nullptr;   // [L][max_items]
   int32_t* pinned_jobs = nullptr;     // [L][max_items + 1]
@@ -859,7 +860,7 @@ int razor_decode_attention_multi(razor_cache_t* c, int32_t layer, const void* q,
   const int group0 = c->cfg.n_q_heads / c->cfg.n_kv_heads;
   // A round with at least 64 query rows per KV head is a dense tile: the query-tiled kernel streams the cache once
   // per 128 rows (tensor cores).  ALiBi heads stay on the path below.
-  if ((long long)group0 * n_tokens >= kRoundTileRows / 2 && !c->dv.alibi) return round_impl(c, layer, q, out, n_tokens, stream);
+  if ((long long)group0 * n_tokens >= c->round_tiled_min_rows && !c->dv.alibi) return round_impl(c, layer, q, out, n_tokens, stream);
   // One launch takes a tile of 2, 4 or 8 rows per KV head (query heads of the group x query tokens).  A
   // longer round runs block by block, the largest block that fits; when the round is not a multiple of
   // the block, the last block is moved back to end with the round and recomputes a few tokens.
@@ -1034,6 +1035,10 @@ int razor_cache_set_option(razor_cache_t* c, int32_t option, int32_t value) {
     case RAZOR_OPT_DECODE_EARLY_PREFETCH:
       if (value < 0 || value > 64) return RAZOR_E_INVALID_ARG;
       c->tune.early_prefetch = value;
+      break;
+    case RAZOR_OPT_ROUND_TILED_MIN_ROWS:
+      if (value < 1) return RAZOR_E_INVALID_ARG;
+      c->round_tiled_min_rows = value;
       break;
     default:
       return RAZOR_E_INVALID_ARG;

@@ -78,13 +78,16 @@ def test_round_on_a_long_context_with_split_heads():
     cache.close()
 
 
+@pytest.mark.parametrize("tiled", [False, True])
 @pytest.mark.parametrize("group,T,D", [(1, 16, 128), (1, 9, 128), (1, 3, 64), (2, 5, 128), (4, 3, 128), (8, 2, 64), (1, 29, 128)])
-def test_round_longer_than_one_launch_runs_block_by_block(group, T, D):
-    """Rounds that do not fit one tile of 2, 4 or 8 rows: blocks of the largest size that fits, the last one moved
-    back to end with the round; every block masks the round's tokens that come after it."""
+def test_round_longer_than_one_launch(group, T, D, tiled):
+    """Rounds that do not fit one tile of 2, 4 or 8 rows of the streaming kernel.  Block by block on that kernel
+    (forced here by the threshold option; it is what ALiBi caches get): blocks of the largest size that fits, the
+    last one moved back to end with the round, every block masking the round's tokens that come after it.  And the
+    default: the query-tiled kernel, most of whose 128 rows are no query of such a short round."""
     Hkv = 2
     w = synth.Workload("long_round", 2, 1, Hkv * group, Hkv, D, "bf16", [700, 90], [120, 40], 4, 1, T, 777 + T + group)
-    cache = make_cache(w, max_new=T)
+    cache = make_cache(w, max_new=T, options=None if tiled else {rz.OPT_ROUND_TILED_MIN_ROWS: 1 << 30})
     K, V = synth.make_dense_kv(w, 0, DEV)
     retr = w.retrieval(0)
     cache.compress(0, K, V, w.ctx_len, retr, w.window)
