@@ -175,7 +175,7 @@ RAZOR_API int razor_decode_step(razor_cache_t* cache, int32_t layer, const void*
  *   razor_append_many             adds n_tokens tokens per sequence, k_new, v_new device
  *                                 [B, n_tokens, Hkv, D] contiguous: exactly what n_tokens razor_append
  *                                 calls would leave (window fixed, evicted tokens folded into Eq. 4).
- *                                 Any length up to the remaining max_new_tokens; runs of 64 tokens or more
+ *                                 Any length up to the remaining max_new_tokens; runs of 8 tokens or more
  *                                 are appended in parallel over the tokens.  This is also how a chunked
  *                                 prefill hands its K/V over without a dense cache of the whole context:
  *                                 razor_compress with ctx_len 0 (K, V may be NULL) fixes the layer's windows

@@ -343,7 +343,8 @@ int razor_cache_destroy(razor_cache_t* c) {
 
 namespace {
 
-constexpr int kAppendChunkMin = 64;   // razor_append_many: runs this long are appended in parallel over the tokens
+constexpr int kAppendChunkMin = 8;   // razor_append_many: runs this long are appended in parallel over the tokens
+                                     // (shorter ones token by token in one kernel: about 2 us per token)
 
 struct SeqIn {
   int b;
@@ -858,8 +859,8 @@ int razor_decode_attention_multi(razor_cache_t* c, int32_t layer, const void* q,
     if (h.n_drop > 0 && h.window < n_tokens) return RAZOR_E_INVALID_ARG;  // the mean would hold tokens after a query
   }
   const int group0 = c->cfg.n_q_heads / c->cfg.n_kv_heads;
-  // A round with at least 64 query rows per KV head is a dense tile: the query-tiled kernel streams the cache once
-  // per 128 rows (tensor cores).  ALiBi heads stay on the path below.
+  // A round of more query rows per KV head than one launch of the streaming kernel takes goes to the query-tiled
+  // kernel, which streams the cache once per 128 rows (tensor cores).  ALiBi heads stay on the path below.
   if ((long long)group0 * n_tokens >= c->round_tiled_min_rows && !c->dv.alibi) return round_impl(c, layer, q, out, n_tokens, stream);
   // One launch takes a tile of 2, 4 or 8 rows per KV head (query heads of the group x query tokens).  A
   // longer round runs block by block, the largest block that fits; when the round is not a multiple of

@@ -32,7 +32,7 @@ def test_cache_built_chunk_by_chunk_from_empty(dtype, D, group):
     """Chunks shorter and longer than the windows, runs below and above the parallel kernel's threshold, a window
     that fills in the middle of a chunk, a chunk that laps the ring several times."""
     Hkv = 3
-    chunks = [700, 1, 5, 64, 1500, 735, 100]
+    chunks = [700, 1, 5, 8, 7, 64, 1500, 735, 100]
     total = sum(chunks)
     w = synth.Workload("chunked", 2, 1, Hkv * group, Hkv, D, dtype, [0, 0], [600, 100], 4, 1, total, 9100 + D + group)
     cache = make_cache(w, max_new=total)
