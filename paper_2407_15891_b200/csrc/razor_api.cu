@@ -744,9 +744,15 @@ static int round_impl(razor_cache_t* c, int32_t layer, const void* q, float* out
       total_blocks += std::max(blocks, 0);
     }
   }
-  // parts: about four items per SM, never more than fit the item list or the record rows
+  // Parts.  Two CTAs run per SM, and an item costs some ten steps' worth of set-up and read-out, a unit in several
+  // parts a merge pass besides.  So a unit is cut only where balance asks for it: into parts of a CTA's average
+  // load when the longest unit is at most one and a half times that load (a round of many tiles: usually no cut at
+  // all), into parts of half of it otherwise; never more parts than fit the item list or the record rows.
   const long long rec_rows = (long long)c->lay.max_items * kMaxGroup;
-  long long chunk = std::max<long long>(1, ceil_div(total_blocks, (long long)c->n_sms * 4));
+  long long longest = 0;
+  for (const Unit& u : units) longest = std::max<long long>(longest, u.blocks);
+  const long long per_cta = std::max<long long>(1, ceil_div(total_blocks, (long long)c->n_sms * 2));
+  long long chunk = 2 * longest <= 3 * per_cta ? per_cta : std::max<long long>(1, ceil_div(per_cta, 2));
   std::vector<RoundItem> items;
   std::vector<RoundUnit> multi;
   for (;;) {
