@@ -73,10 +73,13 @@ def test_alibi_decode_steps_match_the_oracle(dtype, group, D):
     cache.close()
 
 
-def test_alibi_in_a_round_of_several_tokens():
-    Hkv, T, D = 3, 4, 128
+@pytest.mark.parametrize("T", [4, 20, 37])
+def test_alibi_in_a_round_of_several_tokens(T):
+    """T = 4: one launch (a tile of 8 rows); longer rounds run block by block on the streaming kernel, every block
+    masking the round's tokens that come after it (ALiBi caches do not use the query-tiled kernel)."""
+    Hkv, D = 3, 128
     w = synth.Workload("alibi_round", 2, 1, Hkv * 2, Hkv, D, "bf16", [700, 60], [300, 300], 0, 1, T, 99)
-    hw = [40, 300, 9]
+    hw = [40, 300, max(9, T)]
     slopes = _slopes(1, w.n_q_heads)
     cache = make_cache(w, max_new=T, use_comp=0)
     rz.razor_cache_set_alibi(cache.handle, slopes)
