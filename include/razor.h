@@ -189,10 +189,11 @@ RAZOR_API int razor_decode_step(razor_cache_t* cache, int32_t layer, const void*
  * Limits of the multi-token call: bf16; at least n_tokens tokens cached; every head that has dropped
  * tokens must have a window >= n_tokens (otherwise its mean would hold tokens that come after a query).
  * A round of at most 8 query rows per KV head (query heads of the group x query tokens) is one launch of
- * the streaming kernel on a tile of 2, 4 or 8 rows (matrix instructions).  A longer round of a bf16 cache
- * without ALiBi runs on the query-tiled tensor-core kernel (128 rows per tile; the threshold is
- * RAZOR_OPT_ROUND_TILED_MIN_ROWS); otherwise it runs as several launches of the streaming kernel, block by
- * block, each streaming the cache once and masking the round's tokens that come after its block.
+ * the streaming kernel on a tile of 2, 4 or 8 rows (matrix instructions).  A longer round runs on the
+ * query-tiled tensor-core kernel (128 rows per tile; the threshold is RAZOR_OPT_ROUND_TILED_MIN_ROWS; with
+ * ALiBi it adds Eq. 1's distance penalty to every score) - except in an ALiBi cache that keeps sink tokens,
+ * or below the threshold: there it runs as several launches of the streaming kernel, block by block, each
+ * streaming the cache once and masking the round's tokens that come after its block.
  * Errors: NULL_PTR, INVALID_ARG, UNSUPPORTED_DIM, NOT_COMPRESSED, CAPACITY (append), MISALIGNED, CUDA.
  */
 RAZOR_API int razor_append_many(razor_cache_t* cache, int32_t layer, const void* k_new, const void* v_new,
@@ -283,7 +284,7 @@ enum {
                                            rows per KV head (query heads of the group x new tokens; default 9,
                                            i.e. more than one launch of the streaming kernel would take) run on
                                            the query-tiled tensor-core kernel, shorter ones block by block on
-                                           the streaming kernel; bf16 caches without ALiBi only                */
+                                           the streaming kernel                                                */
 };
 RAZOR_API int razor_cache_set_option(razor_cache_t* cache, int32_t option, int32_t value);
 

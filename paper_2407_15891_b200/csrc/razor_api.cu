@@ -866,8 +866,10 @@ int razor_decode_attention_multi(razor_cache_t* c, int32_t layer, const void* q,
   }
   const int group0 = c->cfg.n_q_heads / c->cfg.n_kv_heads;
   // A round of more query rows per KV head than one launch of the streaming kernel takes goes to the query-tiled
-  // kernel, which streams the cache once per 128 rows (tensor cores).  ALiBi heads stay on the path below.
-  if ((long long)group0 * n_tokens >= c->round_tiled_min_rows && !c->dv.alibi) return round_impl(c, layer, q, out, n_tokens, stream);
+  // kernel, which streams the cache once per 128 rows (tensor cores).  (An ALiBi cache with sink tokens stays on the
+  // path below.)
+  if ((long long)group0 * n_tokens >= c->round_tiled_min_rows && (!c->dv.alibi || c->cfg.n_sink == 0))
+    return round_impl(c, layer, q, out, n_tokens, stream);
   // One launch takes a tile of 2, 4 or 8 rows per KV head (query heads of the group x query tokens).  A
   // longer round runs block by block, the largest block that fits; when the round is not a multiple of
   // the block, the last block is moved back to end with the round and recomputes a few tokens.

@@ -4,7 +4,8 @@
 // 5th-generation tensor cores: S = Q K^T with both operands in shared memory, O = P V with P read out of
 // tensor memory and V out of shared memory, accumulators in tensor memory.  Same arithmetic as the decode kernel
 // otherwise: causal mask inside the round (Section 3.1), compensation token with its count as the initial
-// softmax state of a head's first part (Eq. 5), split over the tokens with partial records merged afterwards.
+// softmax state of a head's first part (Eq. 5), split over the tokens with partial records merged afterwards;
+// for ALiBi caches (Section 3.1) a second instantiation adds Eq. 1's distance penalty to every score.
 //
 // A work item is (KV head, tile of 128 query rows, a run of 128-token blocks of the head's slot stream); a CTA
 // takes it in steps of 64 tokens.  Persistent CTAs pull items from a queue (longest first), TWO CTAs to an SM:
@@ -125,7 +126,7 @@ __device__ __forceinline__ int slot_pos(int s, int n_sink, int ring_head, int wi
   return total - window + j;
 }
 
-template <int D>
+template <int D, bool kAlibi>
 __global__ void __launch_bounds__(kRoundThreads, kCtasPerSm)
     round_kernel(DeviceView dv, const __grid_constant__ CUtensorMap map_pool, int layer, RoundJobs jb,
                  const __nv_bfloat16* __restrict__ q, float* __restrict__ out) {
@@ -392,6 +393,8 @@ __global__ void __launch_bounds__(kRoundThreads, kCtasPerSm)
         w_seed = 1.f;
       }
       const bool in_order = st.window < 0 || st.n_drop == 0;               // slot = position
+      float slope_l2 = 0.f;   // ALiBi slope of this row's query head (Section 3.1), log2 domain
+      if constexpr (kAlibi) slope_l2 = dv.alibi_slopes[((size_t)layer * dv.n_kv_heads + g_kv) * G + j];
       const int q_pos_min = total - jb.n_tok + w.q_tile * tok_per_tile;    // the tile's earliest query
       int new_lo = 0, new_hi = 0, new_lo2 = 0, new_hi2 = 0;                // slot ranges [lo, hi) holding the round's tokens
       if (!in_order) {
@@ -467,6 +470,29 @@ __global__ void __launch_bounds__(kRoundThreads, kCtasPerSm)
           for (int e = 0; e < kStep; ++e)
             if (col_pos[e] > q_pos) v[e] = 0xff800000u;   // -inf
         }
+        if constexpr (kAlibi) {
+          // Eq. 1: the logit of column e gets - l_h (m - n), with the slope already in the log2 domain.  The position
+          // n of column e runs up with e: slot0 + e in position order; in a ring total - window + (x0 + e), plus window
+          // for the columns before the wrap (x0 + e < 0).  (No sink tokens in an ALiBi cache on this path.)  The scores
+          // are put into the log2 domain here, so the scale below is one.
+          float pen_base, pen_wrap = 0.f;
+          int wrap_end = 0;
+          if (in_order) {
+            pen_base = slope_l2 * (float)(slot0 - q_pos);
+          } else {
+            const int x0 = slot0 - st.ring_head;
+            pen_base = slope_l2 * (float)(total - st.window + x0 - q_pos);
+            pen_wrap = slope_l2 * (float)st.window;
+            wrap_end = -x0;
+          }
+#pragma unroll
+          for (int e = 0; e < kStep; ++e) {
+            float pen = fmaf(slope_l2, (float)e, pen_base);
+            if (e < wrap_end) pen += pen_wrap;
+            v[e] = __float_as_uint(fmaf(__uint_as_float(v[e]), scale_log2, pen));
+          }
+        }
+        const float sc = kAlibi ? 1.f : scale_log2;
         float mx0 = -CUDART_INF_F, mx1 = -CUDART_INF_F;
 #pragma unroll
         for (int e = 0; e < kStep; e += 4) {
@@ -474,7 +500,7 @@ __global__ void __launch_bounds__(kRoundThreads, kCtasPerSm)
           mx1 = max3(mx1, __uint_as_float(v[e + 2]), __uint_as_float(v[e + 3]));
         }
         // (the scale is positive: the max of the scaled scores is the scaled max)
-        const float m_blk = fmaxf(mx0, mx1) * scale_log2;
+        const float m_blk = fmaxf(mx0, mx1) * sc;
 
         // The product of the step before must have run before P is overwritten and before O is touched.  The
         // weights themselves need neither, so in the common case (no rescaling) they are computed into registers
@@ -517,7 +543,7 @@ __global__ void __launch_bounds__(kRoundThreads, kCtasPerSm)
         // 2c and 2c + 1 (the operand-A layout of the matrix unit), the remainder half the same.  A weight goes into
         // the product as a bf16 head (its upper 16 bits) plus a bf16 remainder - two products - so that it keeps
         // fp32-like accuracy: a single bf16 would put 2^-9 of a large weight times its V row into the result.
-        const uint64_t scale2 = f2_pack(scale_log2, scale_log2), neg_m2 = f2_pack(-m_use, -m_use);
+        const uint64_t scale2 = f2_pack(sc, sc), neg_m2 = f2_pack(-m_use, -m_use);
         uint64_t psum2[2] = {f2_pack(0.f, 0.f), f2_pack(0.f, 0.f)};
         const uint32_t p_addr = lane_addr + kPCol;
         uint32_t hi[kStep / 2], lo[kStep / 2];
@@ -656,7 +682,7 @@ bool make_pool_map(CUtensorMap* map, const void* pool, long long n_pages) {
   }
 }
 
-template <int D>
+template <int D, bool kAlibi>
 cudaError_t round_launch(const DeviceView& dv, long long pool_pages, int layer, const RoundJobs& jb, const void* q,
                          float* out, int n_sms, cudaStream_t s) {
   CUtensorMap map;
@@ -666,15 +692,15 @@ cudaError_t round_launch(const DeviceView& dv, long long pool_pages, int layer, 
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= 64 || !opted_in[dev]) {
-    e = cudaFuncSetAttribute(round_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)round_smem_bytes<D>());
+    e = cudaFuncSetAttribute(round_kernel<D, kAlibi>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)round_smem_bytes<D>());
     if (e != cudaSuccess) return e;
     // two CTAs to an SM need the largest shared-memory split
-    e = cudaFuncSetAttribute(round_kernel<D>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
+    e = cudaFuncSetAttribute(round_kernel<D, kAlibi>, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared);
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) opted_in[dev] = true;
   }
   const int grid = std::max(1, std::min(n_sms * kCtasPerSm, jb.n_items));
-  round_kernel<D><<<grid, kRoundThreads, round_smem_bytes<D>(), s>>>(dv, map, layer, jb, (const __nv_bfloat16*)q, out);
+  round_kernel<D, kAlibi><<<grid, kRoundThreads, round_smem_bytes<D>(), s>>>(dv, map, layer, jb, (const __nv_bfloat16*)q, out);
   e = cudaGetLastError();
   if (e != cudaSuccess || jb.n_units == 0) return e;
   round_combine_kernel<D><<<dim3(jb.n_units, kRows / 4), 128, 0, s>>>(dv, jb, out);
@@ -685,8 +711,11 @@ cudaError_t round_launch(const DeviceView& dv, long long pool_pages, int layer, 
 
 cudaError_t launch_round(const DeviceView& dv, long long pool_pages, int layer, const RoundJobs& jb, const void* q,
                          float* out, int n_sms, cudaStream_t s) {
-  return dv.head_dim == 128 ? round_launch<128>(dv, pool_pages, layer, jb, q, out, n_sms, s)
-                            : round_launch<64>(dv, pool_pages, layer, jb, q, out, n_sms, s);
+  if (dv.alibi)
+    return dv.head_dim == 128 ? round_launch<128, true>(dv, pool_pages, layer, jb, q, out, n_sms, s)
+                              : round_launch<64, true>(dv, pool_pages, layer, jb, q, out, n_sms, s);
+  return dv.head_dim == 128 ? round_launch<128, false>(dv, pool_pages, layer, jb, q, out, n_sms, s)
+                            : round_launch<64, false>(dv, pool_pages, layer, jb, q, out, n_sms, s);
 }
 
 }  // namespace razor

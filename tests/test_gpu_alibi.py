@@ -73,15 +73,19 @@ def test_alibi_decode_steps_match_the_oracle(dtype, group, D):
     cache.close()
 
 
-@pytest.mark.parametrize("T", [4, 20, 37])
-def test_alibi_in_a_round_of_several_tokens(T):
-    """T = 4: one launch (a tile of 8 rows); longer rounds run block by block on the streaming kernel, every block
-    masking the round's tokens that come after it (ALiBi caches do not use the query-tiled kernel)."""
-    Hkv, D = 3, 128
-    w = synth.Workload("alibi_round", 2, 1, Hkv * 2, Hkv, D, "bf16", [700, 60], [300, 300], 0, 1, T, 99)
-    hw = [40, 300, max(9, T)]
+@pytest.mark.parametrize("T,tiled,group,D", [(4, True, 2, 128), (20, True, 2, 128), (20, False, 2, 128), (37, True, 2, 128),
+                                             (37, False, 2, 128), (150, True, 2, 128), (70, True, 1, 64), (9, True, 4, 128),
+                                             (33, True, 8, 64), (5, True, 4, 64)])
+def test_alibi_in_a_round_of_several_tokens(T, tiled, group, D):
+    """T = 4: one launch of the streaming kernel (a tile of 8 rows).  Longer rounds: the query-tiled kernel, which
+    adds Eq. 1's distance penalty to every score (heads in position order and ring heads that have wrapped), or -
+    forced here by the threshold option - block by block on the streaming kernel, every block masking the round's
+    tokens that come after it."""
+    Hkv = 3
+    w = synth.Workload("alibi_round", 2, 1, Hkv * group, Hkv, D, "bf16", [700, 60], [300, 300], 0, 1, T, 99 + group)
+    hw = [max(40, T), 300, max(9, T)]
     slopes = _slopes(1, w.n_q_heads)
-    cache = make_cache(w, max_new=T, use_comp=0)
+    cache = make_cache(w, max_new=T, use_comp=0, options=None if tiled else {rz.OPT_ROUND_TILED_MIN_ROWS: 1 << 30})
     rz.razor_cache_set_alibi(cache.handle, slopes)
     rz.razor_cache_set_head_windows(cache.handle, 0, hw)
     K, V = synth.make_dense_kv(w, 0, DEV)
@@ -99,8 +103,8 @@ def test_alibi_in_a_round_of_several_tokens(T):
             Kh = np.concatenate([to_f64(K[b, g, : w.ctx_len[b]]), to_f64(k[b, :, g])])
             Vh = np.concatenate([to_f64(V[b, g, : w.ctx_len[b]]), to_f64(v[b, :, g])])
             win = -1 if retr[g] else min(w.window[b], hw[g])
-            for j in range(2):
-                h = g * 2 + j
+            for j in range(group):
+                h = g * group + j
                 expect = orc.alibi_decode_head(to_f64(q[b, :, h]), Kh, Vh, win, float(slopes[0, h]), scale)
                 assert np.abs(out[b, :, h] - expect).max() <= TOL_OUT["bf16"]
     cache.close()
