@@ -95,6 +95,8 @@ inline long long head_capacity_tokens(const razor_config_t& c, int n_ctx, int wi
 }
 
 constexpr int kPlanSlots = 16;   // compression plans that may be on their way to the device at once
+constexpr int kRoundSlots = 8;   // work lists of the round kernel that may be on their way to the device at once
+constexpr size_t kRoundSlotBytes = (size_t)kRoundMaxItems * sizeof(RoundItem) + (size_t)kRoundMaxUnits * sizeof(RoundUnit);
 
 struct LayerHost {
   bool any = false;
@@ -147,8 +149,11 @@ struct razor_cache {
   cudaEvent_t plan_done[kPlanSlots] = {};
   int plan_next = 0;
   // Work list of the round kernel (razor_decode_attention_multi on long rounds): pinned staging, one upload in flight.
-  uint8_t* pinned_round = nullptr;   // RoundItem[kRoundMaxItems], then RoundUnit[kRoundMaxUnits]
-  cudaEvent_t round_done = nullptr;
+  // kRoundSlots staging areas used in turn (RoundItem[kRoundMaxItems], then RoundUnit[kRoundMaxUnits] each), so that
+  // the host waits for an upload only when it comes round to that upload's area again and can otherwise run ahead
+  uint8_t* pinned_round = nullptr;
+  cudaEvent_t round_done[kRoundSlots] = {};
+  int round_slot = 0;
   // Layer whose pages, state or sums the last kernel launched for this cache wrote (-1: it wrote none, a decode).
   // An append of another layer may read before it waits for that kernel.
   int last_writer_layer = -1;
@@ -279,8 +284,7 @@ int razor_cache_create(razor_cache_t** out, const razor_config_t* cfg, void* poo
   if (e == cudaSuccess)
     e = cudaHostAlloc((void**)&c->pinned_plan, (size_t)kPlanSlots * c->plan_bytes, cudaHostAllocDefault);
   if (e == cudaSuccess)
-    e = cudaHostAlloc((void**)&c->pinned_round, (size_t)kRoundMaxItems * sizeof(RoundItem) + (size_t)kRoundMaxUnits * sizeof(RoundUnit),
-                      cudaHostAllocDefault);
+    e = cudaHostAlloc((void**)&c->pinned_round, (size_t)kRoundSlots * kRoundSlotBytes, cudaHostAllocDefault);
   if (e != cudaSuccess) {
     note_cuda_error(e);
     if (c->pinned_items) cudaFreeHost(c->pinned_items);
@@ -332,7 +336,8 @@ int razor_cache_destroy(razor_cache_t* c) {
   if (c->pinned_multi) cudaFreeHost(c->pinned_multi);
   if (c->pinned_plan) cudaFreeHost(c->pinned_plan);
   if (c->pinned_round) cudaFreeHost(c->pinned_round);
-  if (c->round_done) cudaEventDestroy(c->round_done);
+  for (cudaEvent_t ev : c->round_done)
+    if (ev) cudaEventDestroy(ev);
   for (cudaEvent_t ev : c->plan_done)
     if (ev) cudaEventDestroy(ev);
   delete c;
@@ -782,16 +787,19 @@ static int round_impl(razor_cache_t* c, int32_t layer, const void* q, float* out
     return a.blk_end - a.blk_begin > b.blk_end - b.blk_begin;
   });
   cudaStream_t s = (cudaStream_t)stream;
-  if (c->round_done) RZ_CUDA(cudaEventSynchronize(c->round_done));   // the upload before has left the staging area
-  else RZ_CUDA(cudaEventCreateWithFlags(&c->round_done, cudaEventDisableTiming));
-  RoundItem* st_items = (RoundItem*)c->pinned_round;
-  RoundUnit* st_units = (RoundUnit*)(c->pinned_round + (size_t)kRoundMaxItems * sizeof(RoundItem));
+  const int slot = c->round_slot;
+  c->round_slot = (slot + 1) % kRoundSlots;
+  if (c->round_done[slot]) RZ_CUDA(cudaEventSynchronize(c->round_done[slot]));   // the upload that used this area last has left it
+  else RZ_CUDA(cudaEventCreateWithFlags(&c->round_done[slot], cudaEventDisableTiming));
+  uint8_t* area = c->pinned_round + (size_t)slot * kRoundSlotBytes;
+  RoundItem* st_items = (RoundItem*)area;
+  RoundUnit* st_units = (RoundUnit*)(area + (size_t)kRoundMaxItems * sizeof(RoundItem));
   std::memcpy(st_items, items.data(), items.size() * sizeof(RoundItem));
   if (!multi.empty()) std::memcpy(st_units, multi.data(), multi.size() * sizeof(RoundUnit));
   RZ_CUDA(cudaMemcpyAsync(c->dv.round_items, st_items, items.size() * sizeof(RoundItem), cudaMemcpyHostToDevice, s));
   if (!multi.empty())
     RZ_CUDA(cudaMemcpyAsync(c->dv.round_units, st_units, multi.size() * sizeof(RoundUnit), cudaMemcpyHostToDevice, s));
-  RZ_CUDA(cudaEventRecord(c->round_done, s));
+  RZ_CUDA(cudaEventRecord(c->round_done[slot], s));
   const RoundJobs jb{(int32_t)items.size(), (int32_t)multi.size(), n_tokens, 0};
   RZ_CUDA(launch_round(c->dv, c->pool_pages, layer, jb, q, out, c->n_sms, s));
   c->last_writer_layer = -1;
