@@ -85,7 +85,7 @@ def test_alibi_in_a_round_of_several_tokens(T, tiled, group, D):
     w = synth.Workload("alibi_round", 2, 1, Hkv * group, Hkv, D, "bf16", [700, 60], [300, 300], 0, 1, T, 99 + group)
     hw = [max(40, T), 300, max(9, T)]
     slopes = _slopes(1, w.n_q_heads)
-    cache = make_cache(w, max_new=T, use_comp=0, options=None if tiled else {rz.OPT_ROUND_TILED_MIN_ROWS: 1 << 30})
+    cache = make_cache(w, max_new=T, use_comp=0, options={rz.OPT_ROUND_TILED_MIN_ROWS: 9 if tiled else 1 << 30})
     rz.razor_cache_set_alibi(cache.handle, slopes)
     rz.razor_cache_set_head_windows(cache.handle, 0, hw)
     K, V = synth.make_dense_kv(w, 0, DEV)

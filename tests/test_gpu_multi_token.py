@@ -87,7 +87,7 @@ def test_round_longer_than_one_launch(group, T, D, tiled):
     default: the query-tiled kernel, most of whose 128 rows are no query of such a short round."""
     Hkv = 2
     w = synth.Workload("long_round", 2, 1, Hkv * group, Hkv, D, "bf16", [700, 90], [120, 40], 4, 1, T, 777 + T + group)
-    cache = make_cache(w, max_new=T, options=None if tiled else {rz.OPT_ROUND_TILED_MIN_ROWS: 1 << 30})
+    cache = make_cache(w, max_new=T, options={rz.OPT_ROUND_TILED_MIN_ROWS: 9 if tiled else 1 << 30})
     K, V = synth.make_dense_kv(w, 0, DEV)
     retr = w.retrieval(0)
     cache.compress(0, K, V, w.ctx_len, retr, w.window)
