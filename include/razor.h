@@ -281,11 +281,10 @@ enum {
                                            writing (the host knows which page a preceding razor_append
                                            touched); 0: every copy waits                                   */
   RAZOR_OPT_ROUND_TILED_MIN_ROWS = 8    /* razor_decode_attention_multi: rounds with at least this many query
-                                           rows per KV head (query heads of the group x new tokens) run on the
+                                           rows per KV head (query heads of the group x new tokens; default 9,
+                                           i.e. more than one launch of the streaming kernel takes) run on the
                                            query-tiled tensor-core kernel, shorter ones block by block on the
-                                           streaming kernel.  0 (default): automatic - 17 rows, i.e. what would
-                                           take a third launch of the streaming kernel, or 9 rows when the batch
-                                           has at least 64 KV heads                                            */
+                                           streaming kernel                                                    */
 };
 RAZOR_API int razor_cache_set_option(razor_cache_t* cache, int32_t option, int32_t value);
 

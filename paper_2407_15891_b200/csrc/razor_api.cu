@@ -137,7 +137,7 @@ struct razor_cache {
   long long pool_pages = 0, next_page = 0;
   int n_sms = 148;
   DecodeTuning tune{3, 80, 32, 0, 0, 0, 12};
-  int round_tiled_min_rows = 0;   // rounds with at least this many query rows per KV head run on the query-tiled kernel; 0: automatic
+  int round_tiled_min_rows = 9;   // rounds with at least this many query rows per KV head run on the query-tiled kernel
   std::vector<LayerHost> layers;
   WorkItem* pinned_items = nullptr;   // [L][max_items]
   int32_t* pinned_jobs = nullptr;     // [L][max_items + 1]
@@ -876,11 +876,9 @@ int razor_decode_attention_multi(razor_cache_t* c, int32_t layer, const void* q,
   // A round of more query rows per KV head than one launch of the streaming kernel takes goes to the query-tiled
   // kernel, which streams the cache once per 128 rows (tensor cores).  (An ALiBi cache with sink tokens stays on the
   // path below.)
-  // Automatic threshold: from 17 rows (a third launch of the streaming kernel) always; for 9-16 rows (a second launch)
-  // when the batch has many KV heads - there the streaming kernel's launches cost more than the tiled kernel's set-up
-  // (32K MHA, 256 heads: 0.31 against 0.44 ms; 128K GQA, 16 heads: 150 against 124 us).
-  const int min_rows = c->round_tiled_min_rows > 0 ? c->round_tiled_min_rows : (c->dv.n_heads >= 64 ? 9 : 17);
-  if ((long long)group0 * n_tokens >= min_rows && (!c->dv.alibi || c->cfg.n_sink == 0))
+  // (From 9 rows, a second launch of the streaming kernel: 32K MHA, 256 heads, 12 rows: 0.31 against 0.44 ms; 128K
+  // GQA, 16 heads, 16 rows: 113 against 128 us.)
+  if ((long long)group0 * n_tokens >= c->round_tiled_min_rows && (!c->dv.alibi || c->cfg.n_sink == 0))
     return round_impl(c, layer, q, out, n_tokens, stream);
   // One launch takes a tile of 2, 4 or 8 rows per KV head (query heads of the group x query tokens).  A
   // longer round runs block by block, the largest block that fits; when the round is not a multiple of
@@ -1058,7 +1056,7 @@ int razor_cache_set_option(razor_cache_t* c, int32_t option, int32_t value) {
       c->tune.early_prefetch = value;
       break;
     case RAZOR_OPT_ROUND_TILED_MIN_ROWS:
-      if (value < 0) return RAZOR_E_INVALID_ARG;
+      if (value < 1) return RAZOR_E_INVALID_ARG;
       c->round_tiled_min_rows = value;
       break;
     default:

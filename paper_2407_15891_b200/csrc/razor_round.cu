@@ -638,18 +638,29 @@ __global__ void __launch_bounds__(128) round_combine_kernel(DeviceView dv, Round
   float m = -CUDART_INF_F, l = 0.f;
   LaneVec<D> acc;
   acc.zero();
-  for (int p = 0; p < u.n_parts; ++p) {
-    const size_t r = (size_t)u.rec_base + (size_t)p * kRows + row;
-    const float2 ml = __ldcg(&dv.rec_ml[r]);
-    LaneVec<D> o;
-    o.load_l2(dv.rec_o + r * D, lane);
-    const float mn = fmaxf(m, ml.x);
-    const float mu = (mn == -CUDART_INF_F) ? 0.f : mn;
-    const float c_old = fast_exp2(m - mu), c_new = fast_exp2(ml.x - mu);
-    l = l * c_old + ml.y * c_new;
-    acc.scale(c_old);
-    acc.fma(c_new, o);
-    m = mn;
+  constexpr int U = 8;   // records in flight (a unit of a long head may be in a hundred parts)
+  for (int p0 = 0; p0 < u.n_parts; p0 += U) {
+    float2 mls[U];
+    LaneVec<D> os[U];
+#pragma unroll
+    for (int i = 0; i < U; ++i) {
+      const size_t r = (size_t)u.rec_base + (size_t)min(p0 + i, u.n_parts - 1) * kRows + row;   // beyond the end: re-read, unused
+      mls[i] = __ldcg(&dv.rec_ml[r]);
+      os[i].load_l2(dv.rec_o + r * D, lane);
+    }
+#pragma unroll
+    for (int i = 0; i < U; ++i) {
+      if (p0 + i < u.n_parts) {
+        const float2 ml = mls[i];
+        const float mn = fmaxf(m, ml.x);
+        const float mu = (mn == -CUDART_INF_F) ? 0.f : mn;
+        const float c_old = fast_exp2(m - mu), c_new = fast_exp2(ml.x - mu);
+        l = l * c_old + ml.y * c_new;
+        acc.scale(c_old);
+        acc.fma(c_new, os[i]);
+        m = mn;
+      }
+    }
   }
   acc.scale(l > 0.f ? 1.f / l : 0.f);
   const int b = u.head / dv.n_kv_heads, g_kv = u.head % dv.n_kv_heads;
